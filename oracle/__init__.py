@@ -1,0 +1,209 @@
+"""ctypes front end of the plain CPU oracle (``kvq_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  Nothing in the CUDA package imports it, and it
+imports nothing from the CUDA package.
+
+All arithmetic lives in the C file; this module only marshals numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "kvq_oracle.c")
+_LIB = os.path.join(_HERE, "libkvq_oracle.so")
+
+CFLAGS = ["-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-shared", "-fPIC"]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc if the shared object is missing or stale."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + ".tmp.%d" % os.getpid()
+    subprocess.check_call(["gcc", *CFLAGS, "-o", tmp, _SRC, "-lm"])
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.oracle_half_to_float.restype = C.c_float
+        _lib.oracle_half_to_float.argtypes = [C.c_uint16]
+        _lib.oracle_float_to_half.restype = C.c_uint16
+        _lib.oracle_float_to_half.argtypes = [C.c_float]
+        _lib.oracle_num_threads.restype = C.c_int
+    return _lib
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _c(a, dtype) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _u16(a) -> np.ndarray:
+    """fp16 arrays are passed as their bit patterns."""
+    a = np.asarray(a)
+    if a.dtype == np.float16:
+        a = a.view(np.uint16)
+    return np.ascontiguousarray(a, dtype=np.uint16)
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def half_to_float(h: np.ndarray) -> np.ndarray:
+    h = _u16(h)
+    out = np.empty(h.shape, dtype=np.float32)
+    lib().oracle_half_to_float_array(_p(h), C.c_int(h.size), _p(out))
+    return out
+
+
+def float_to_half(f: np.ndarray) -> np.ndarray:
+    f = _c(f, np.float32)
+    out = np.empty(f.shape, dtype=np.uint16)
+    lib().oracle_float_to_half_array(_p(f), C.c_int(f.size), _p(out))
+    return out
+
+
+def select_bits(feats, hidden, W1, b1, W2, b2, W3, b3
+                ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Controller decision for feats [..., 4] -> (bits u8 [...], logits [...,4], gap [...])."""
+    feats = _c(feats, np.float32)
+    shape = feats.shape[:-1]
+    n = int(np.prod(shape)) if shape else 1
+    W1, b1, W2, b2, W3, b3 = (_c(x, np.float32) for x in (W1, b1, W2, b2, W3, b3))
+    assert W1.shape == (hidden, 4) and W2.shape == (hidden, hidden) and W3.shape == (4, hidden)
+    bits = np.empty(n, dtype=np.uint8)
+    logits = np.empty((n, 4), dtype=np.float32)
+    gap = np.empty(n, dtype=np.float32)
+    rc = lib().oracle_select_bits(_p(feats), C.c_int(n), C.c_int(hidden),
+                                  _p(W1), _p(b1), _p(W2), _p(b2), _p(W3), _p(b3),
+                                  _p(bits), _p(logits), _p(gap))
+    if rc != 0:
+        raise ValueError("oracle_select_bits failed: %d" % rc)
+    return bits.reshape(shape), logits.reshape(shape + (4,)), gap.reshape(shape)
+
+
+def assign_slots(bits, counts: Optional[np.ndarray] = None
+                 ) -> Tuple[np.ndarray, np.ndarray]:
+    """(pool<<30 | slot) for one sequence's tokens in position order; returns (pool_slot, counts)."""
+    bits = _c(bits, np.uint8)
+    counts = np.zeros(4, dtype=np.uint32) if counts is None else _c(counts, np.uint32).copy()
+    ps = np.empty(bits.shape[0], dtype=np.uint32)
+    rc = lib().oracle_assign_slots(_p(bits), C.c_int(bits.shape[0]), _p(counts), _p(ps))
+    if rc != 0:
+        raise ValueError("oracle_assign_slots failed: %d" % rc)
+    return ps, counts
+
+
+def quantize_row(x, bits: int) -> Tuple[np.ndarray, np.ndarray]:
+    """One fp16 row -> (codes u8 [D*bits/8], meta u16 [2] = {scale, zero-point} bit patterns)."""
+    x = _u16(x)
+    D = x.shape[0]
+    codes = np.zeros(D * bits // 8, dtype=np.uint8)
+    meta = np.zeros(2, dtype=np.uint16)
+    rc = lib().oracle_quantize_row(_p(x), C.c_int(D), C.c_int(bits), _p(codes), _p(meta))
+    if rc != 0:
+        raise ValueError("oracle_quantize_row failed: %d" % rc)
+    return codes, meta
+
+
+def dequantize_row(codes, meta, D: int, bits: int) -> np.ndarray:
+    codes = _c(codes, np.uint8)
+    meta = _c(meta, np.uint16)
+    out = np.empty(D, dtype=np.float32)
+    rc = lib().oracle_dequantize_row(_p(codes), _p(meta), C.c_int(D), C.c_int(bits), _p(out))
+    if rc != 0:
+        raise ValueError("oracle_dequantize_row failed: %d" % rc)
+    return out
+
+
+def append(K, V, bits):
+    """K, V fp16 [B][n][Hkv][D], bits u8 [B][n] -> (kcodes, kmeta, vcodes, vmeta).
+
+    codes u8 [B][n][Hkv][2*D] (row stride 2*D, tail zero), meta u16 [B][n][Hkv][2].
+    """
+    K, V = _u16(K), _u16(V)
+    bits = _c(bits, np.uint8)
+    B, n, H, D = K.shape
+    assert V.shape == K.shape and bits.shape == (B, n)
+    kc = np.empty((B, n, H, 2 * D), dtype=np.uint8)
+    vc = np.empty((B, n, H, 2 * D), dtype=np.uint8)
+    km = np.empty((B, n, H, 2), dtype=np.uint16)
+    vm = np.empty((B, n, H, 2), dtype=np.uint16)
+    rc = lib().oracle_append(_p(K), _p(V), _p(bits), C.c_int(B), C.c_int(n), C.c_int(H),
+                             C.c_int(D), _p(kc), _p(km), _p(vc), _p(vm))
+    if rc != 0:
+        raise ValueError("oracle_append failed: %d" % rc)
+    return kc, km, vc, vm
+
+
+def decode_attn(Q, q_heads: int, kv_heads: int, bits, kc, km, vc, vm,
+                want64: bool = False):
+    """Q fp16 [B][Hq][D] over the cache written by ``append`` -> O fp16 bit patterns [B][Hq][D]."""
+    Q = _u16(Q)
+    B, Hq, D = Q.shape
+    bits = _c(bits, np.uint8)
+    n = bits.shape[1]
+    kc, vc = _c(kc, np.uint8), _c(vc, np.uint8)
+    km, vm = _c(km, np.uint16), _c(vm, np.uint16)
+    assert Hq == q_heads and kc.shape == (B, n, kv_heads, 2 * D)
+    out = np.empty((B, Hq, D), dtype=np.uint16)
+    out64 = np.empty((B, Hq, D), dtype=np.float64) if want64 else None
+    rc = lib().oracle_decode_attn(_p(Q), C.c_int(B), C.c_int(q_heads), C.c_int(kv_heads),
+                                  C.c_int(D), C.c_int(n), _p(bits), _p(kc), _p(km),
+                                  _p(vc), _p(vm), _p(out), _p(out64))
+    if rc != 0:
+        raise ValueError("oracle_decode_attn failed: %d" % rc)
+    return (out, out64) if want64 else out
+
+
+class OracleCache:
+    """Position-ordered mixed-precision cache of one layer: append rows, then attend."""
+
+    def __init__(self, batch: int, q_heads: int, kv_heads: int, head_dim: int = 64):
+        self.B, self.Hq, self.Hkv, self.D = batch, q_heads, kv_heads, head_dim
+        self.bits = np.zeros((batch, 0), dtype=np.uint8)
+        self.kc = np.zeros((batch, 0, kv_heads, 2 * head_dim), dtype=np.uint8)
+        self.vc = np.zeros_like(self.kc)
+        self.km = np.zeros((batch, 0, kv_heads, 2), dtype=np.uint16)
+        self.vm = np.zeros_like(self.km)
+        self.counts = np.zeros((batch, 4), dtype=np.uint32)
+        self.pool_slot = np.zeros((batch, 0), dtype=np.uint32)
+
+    def __len__(self) -> int:
+        return self.bits.shape[1]
+
+    def append(self, K, V, bits) -> None:
+        bits = _c(bits, np.uint8)
+        kc, km, vc, vm = append(K, V, bits)
+        ps = np.empty(bits.shape, dtype=np.uint32)
+        for b in range(self.B):
+            ps[b], self.counts[b] = assign_slots(bits[b], self.counts[b])
+        self.bits = np.concatenate([self.bits, bits], axis=1)
+        self.kc = np.concatenate([self.kc, kc], axis=1)
+        self.vc = np.concatenate([self.vc, vc], axis=1)
+        self.km = np.concatenate([self.km, km], axis=1)
+        self.vm = np.concatenate([self.vm, vm], axis=1)
+        self.pool_slot = np.concatenate([self.pool_slot, ps], axis=1)
+
+    def decode_attn(self, Q, want64: bool = False):
+        return decode_attn(Q, self.Hq, self.Hkv, self.bits, self.kc, self.km,
+                           self.vc, self.vm, want64=want64)
