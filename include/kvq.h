@@ -1,0 +1,206 @@
+/*
+ * kvq.h -- C ABI of the B200 (sm_100a) adaptive mixed-precision KV cache.
+ *
+ * The library implements the data-parallel hot path of "Don't Waste Bits!"
+ * adaptive KV-cache quantization:
+ *
+ *   features --(controller MLP, Eq. 19-23)--> bit-width per token in {2,4,8,16}
+ *   K,V rows --(Q_b of Eq. 24, append of Eq. 4)--> packed mixed-precision cache
+ *   query    --(decode attention, Eq. 5)--> output, reading that cache
+ *
+ * Quantizer (the paper names Q_b in Eq. 24 without defining it; this is the
+ * reading the library implements): per token and per KV head, asymmetric
+ * min-max over the 64 head channels; scale = (max-min)/(2^b-1) computed in
+ * fp32 and stored as fp16; zero-point = row minimum (fp16, -0 stored as +0);
+ * code_i = clamp(rint((x_i-min) * (1/scale_fp16)), 0, 2^b-1), ties to even;
+ * dequantized value = code*scale + zero-point.  16 "bits" keeps the fp16 row.
+ * One bit-width per token is used for its K row and its V row, in every KV
+ * head.  Class index <-> bit-width: 0,1,2,3 <-> 2,4,8,16 (Algorithm 1).
+ *
+ * Store: one pool per precision; inside a pool the rows of one (layer,
+ * sequence, KV head) are contiguous in slot order; slot = number of earlier
+ * tokens of that (layer, sequence) with the same precision.  A per-token
+ * index word (pool << 30 | slot) is kept per (layer, sequence, position).
+ *
+ * Conventions
+ *   - Every function returns 0 (KVQ_OK) or a negative KVQ_ERR_* code, except
+ *     kvq_strerror.  Nothing throws, aborts or traps the device.
+ *   - "dev" pointers are device memory owned by the caller (for instance a
+ *     torch tensor's data_ptr()) on the device that was current at
+ *     kvq_create; they must stay valid until the work queued on `stream` has
+ *     finished.  "host" pointers are ordinary host memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls that take a stream only enqueue work; they do not synchronize.
+ *     Calls without a stream argument synchronize the device.
+ *   - All sequences of the batch advance together: every append adds the same
+ *     number of tokens to each of the `batch` sequences of that layer.
+ *   - fp16 tensors are IEEE binary16, row-major, innermost dimension last.
+ *   - The handle is not thread-safe; use one handle from one thread at a time.
+ */
+#ifndef KVQ_H
+#define KVQ_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KVQ_OK                 0
+#define KVQ_ERR_ARG           -1   /* NULL pointer, value out of range, unsupported shape   */
+#define KVQ_ERR_CAPACITY      -2   /* append would exceed max_ctx                           */
+#define KVQ_ERR_NO_CONTROLLER -3   /* controller weights were never set                     */
+#define KVQ_ERR_CUDA          -4   /* a CUDA call failed; see kvq_last_cuda_error           */
+#define KVQ_ERR_EMPTY         -5   /* decode attention on a layer that holds no token       */
+#define KVQ_ERR_DEVICE_FLAG   -6   /* a kernel recorded a problem (e.g. a bit-width not in
+                                      {2,4,8,16}); see kvq_device_status                     */
+#define KVQ_ERR_NOMEM         -7   /* host or device allocation failed                      */
+
+typedef struct kvq_ctx kvq_ctx;    /* opaque; owned by the library */
+
+/* Row size of the canonical export format, bytes per (token, KV head, tensor). */
+#define KVQ_EXPORT_ROW_BYTES 128
+
+/*
+ * Create a cache for `layers` layers, `batch` sequences, `q_heads` query heads
+ * sharing `kv_heads` KV heads (q_heads % kv_heads == 0; query head h reads KV
+ * head h / (q_heads/kv_heads)), head_dim == 64, up to `max_ctx` tokens per
+ * sequence (Eq. 4: the cache that decode steps append to).  Allocates every
+ * pool at its worst-case size on the current device (504 bytes per token, KV
+ * head and layer) plus index, counters and split-attention scratch, and zeroes
+ * them.  *out receives the handle.  KVQ_ERR_ARG for unsupported shapes,
+ * KVQ_ERR_NOMEM / KVQ_ERR_CUDA if allocation fails (nothing is leaked).
+ */
+int kvq_create(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim,
+               int max_ctx, int batch);
+
+/* Free everything the handle owns.  NULL is a no-op.  Synchronizes the device. */
+int kvq_destroy(kvq_ctx* ctx);
+
+/*
+ * Install the controller of Eq. 19-21: a 4 -> hidden -> hidden -> 4 MLP with
+ * ReLU after the first two layers.  Host pointers, fp32, row-major [out][in]:
+ * W1 [hidden][4], b1 [hidden], W2 [hidden][hidden], b2 [hidden], W3 [4][hidden],
+ * b3 [4].  The values are copied to the device; 1 <= hidden <= 128 (the paper's
+ * width; the whole parameter block is kept in shared memory).
+ */
+int kvq_set_controller(kvq_ctx* ctx, int hidden,
+                       const float* W1, const float* b1,
+                       const float* W2, const float* b2,
+                       const float* W3, const float* b3);
+
+/*
+ * Controller decision (Eq. 19-23) for n tokens.  feats: dev fp32 [n][4].
+ * bits: dev uint8 [n], receives 2, 4, 8 or 16.  logits_opt: dev fp32 [n][4] or
+ * NULL.  Arithmetic: fp32, each product rounded, then each sum rounded, inputs
+ * in ascending order starting from the bias; argmax takes the lowest class on
+ * ties; a NaN logit selects 16.  n == 0 is a no-op.
+ */
+int kvq_select_bits(kvq_ctx* ctx, const float* feats, int n, uint8_t* bits,
+                    float* logits_opt, void* stream);
+
+/*
+ * Quantize-append (Eq. 24, then Eq. 4) of n_new tokens per sequence to `layer`.
+ * K, V: dev fp16 [batch][n_new][kv_heads][64].  bits: dev uint8 [batch][n_new]
+ * with values in {2,4,8,16}; any other value stores the token as fp16 and sets
+ * the device flag KVQ_FLAG_BAD_BITS.  KVQ_ERR_CAPACITY (nothing is queued) if
+ * the layer would exceed max_ctx.  n_new == 0 is a no-op.
+ */
+int kvq_append(kvq_ctx* ctx, int layer, const void* K, const void* V,
+               const uint8_t* bits, int n_new, void* stream);
+
+/*
+ * Same as kvq_select_bits followed by kvq_append, with the decision taken
+ * inside the append launch: feats is dev fp32 [batch][n_new][4].  bits_out_opt
+ * (dev uint8 [batch][n_new] or NULL) receives the decisions.
+ */
+int kvq_append_fused(kvq_ctx* ctx, int layer, const void* K, const void* V,
+                     const float* feats, int n_new, uint8_t* bits_out_opt, void* stream);
+
+/*
+ * Decode-step attention (Eq. 5) of one query row per (sequence, query head)
+ * over every token cached in `layer`, dequantizing on the fly:
+ * O = Softmax(q K^T / 8) V.  Q, O: dev fp16 [batch][q_heads][64].  fp32
+ * accumulation, online softmax, split over the sequence and merged.
+ * KVQ_ERR_EMPTY if the layer holds no token.
+ */
+int kvq_decode_attn(kvq_ctx* ctx, int layer, const void* Q, void* O, void* stream);
+
+/*
+ * One decode step from HOST buffers, copies included: controller decision for
+ * the step's `batch` tokens, quantize-append of their K/V rows to `layer`,
+ * attention of Q over the layer, result copied back.  feats host fp32
+ * [batch][4]; K, V host fp16 [batch][1][kv_heads][64]; Q host fp16
+ * [batch][q_heads][64]; O host fp16 [batch][q_heads][64] (written);
+ * bits_out_opt host uint8 [batch] or NULL.  Uses staging buffers owned by the
+ * handle; returns after the stream has been synchronized.
+ */
+int kvq_decode_step_host(kvq_ctx* ctx, int layer, const float* feats, const void* K,
+                         const void* V, const void* Q, void* O, uint8_t* bits_out_opt,
+                         void* stream);
+
+/* Forget all cached tokens of every layer (pools keep their bytes, counters go to 0). */
+int kvq_reset(kvq_ctx* ctx, void* stream);
+
+/* Tokens cached per sequence in `layer` (host-side mirror; no device access). */
+int kvq_seq_len(kvq_ctx* ctx, int layer, int* host_len_out);
+
+/*
+ * Number of sequence splits used by kvq_decode_attn: 0 = choose from the
+ * cached length and the device's SM count (default), otherwise 1..64.
+ */
+int kvq_set_splits(kvq_ctx* ctx, int splits);
+
+/*
+ * Canonical copy of tokens [pos0, pos0+n) of every sequence of `layer`, for
+ * comparison with other implementations.  All outputs are dev pointers:
+ *   bits      uint8  [batch][n]                 2,4,8,16
+ *   pool_slot uint32 [batch][n]                 pool << 30 | slot
+ *   k_codes, v_codes uint8 [batch][n][kv_heads][128]: packed codes, element i in
+ *             bits [(i*b)%8, +b) of byte floor(i*b/8); for b == 16 the fp16 row,
+ *             little-endian; bytes past 64*b/8 are zero
+ *   k_meta, v_meta  uint16 [batch][n][kv_heads][2]: fp16 bit patterns of
+ *             {scale, zero-point}; {0,0} for b == 16
+ * Any output pointer may be NULL to skip it.
+ */
+int kvq_export_range(kvq_ctx* ctx, int layer, int pos0, int n,
+                     uint8_t* bits, uint32_t* pool_slot,
+                     void* k_codes, void* v_codes, uint16_t* k_meta, uint16_t* v_meta,
+                     void* stream);
+
+/* The same for one token of one sequence, into HOST buffers ([kv_heads][128] and
+ * [kv_heads][2]); synchronizes. */
+int kvq_export_token(kvq_ctx* ctx, int layer, int b, int pos,
+                     uint8_t* bits, uint32_t* pool_slot,
+                     void* k_codes, void* v_codes, uint16_t* k_meta, uint16_t* v_meta);
+
+/*
+ * Pool fill of `layer`: host_counts (host uint32 [batch][4], may be NULL)
+ * receives tokens per precision class; resident_bytes (host, may be NULL) the
+ * bytes of packed rows in use, sum over tokens of kv_heads * {40,72,136,256};
+ * expected_bits (host, may be NULL) the mean bit-width sum_c count_c*b_c / tokens
+ * (the paper's E[b], Eq. 11).  Synchronizes.
+ */
+int kvq_stats(kvq_ctx* ctx, int layer, uint32_t* host_counts, uint64_t* resident_bytes,
+              double* expected_bits);
+
+/* Device flags recorded by kernels since the last call (host uint32, cleared on read). */
+#define KVQ_FLAG_BAD_BITS 1u      /* a bit-width outside {2,4,8,16} was appended (stored as fp16) */
+int kvq_device_status(kvq_ctx* ctx, uint32_t* host_flags_out);
+
+/* Bytes of device memory the handle holds (pools + index + scratch). */
+int kvq_device_bytes(kvq_ctx* ctx, uint64_t* host_bytes_out);
+
+/* Kernels this handle has launched since creation (for launch accounting). */
+int kvq_launch_count(kvq_ctx* ctx, uint64_t* host_count_out);
+
+/* cudaError_t value of the last failing CUDA call of this handle (0 if none). */
+int kvq_last_cuda_error(kvq_ctx* ctx);
+
+/* Static, human-readable text for a return code. */
+const char* kvq_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVQ_H */

@@ -1,0 +1,93 @@
+// Controller MLP of Eq. 19-23: 4 -> H -> H -> 4, ReLU after the first two
+// layers, argmax over the four logits, class index -> bit-width (Algorithm 1's
+// label map {2,4,8,16} <-> {0,1,2,3}).
+//
+// One thread per token.  The decision must be reproducible bit for bit, so the
+// arithmetic is pinned: fp32, every product rounded (__fmul_rn), then every sum
+// rounded (__fadd_rn), inputs in ascending order starting from the bias -- the
+// intrinsics also keep the compiler from contracting them into FMAs.  Softmax
+// (Eq. 22) is monotone, so the argmax of Eq. 23 is taken on the logits; ties go
+// to the lowest class and a NaN logit selects the fp16 class.
+//
+// Weights live in shared memory in the order W1[H][4] b1[H] W2[H][H] b2[H]
+// W3[4][H] b3[4]; every lane reads the same word at the same time (broadcast).
+#pragma once
+#include "kvq_common.cuh"
+
+namespace kvq {
+
+__host__ __device__ inline int controller_floats(int H) { return 4 * H + H + H * H + H + 4 * H + 4; }
+
+// Copy the parameter block to shared memory (all threads of the CTA take part).
+__device__ __forceinline__ void controller_stage(float* sW, const float* __restrict__ gW, int H) {
+    int n = controller_floats(H);
+    for (int i = threadIdx.x; i < n; i += blockDim.x) sW[i] = gW[i];
+}
+
+// HC > 0: hidden width known at compile time (fully unrolled, h1 in registers);
+// HC == 0: runtime width H <= kMaxHidden (h1 in local memory).
+template <int HC>
+__device__ __forceinline__ int controller_decide(const float* sW, int Hrt, float x0, float x1, float x2,
+                                                 float x3, float logits[4]) {
+    const int H = HC > 0 ? HC : Hrt;
+    const float* W1 = sW;
+    const float* b1 = W1 + 4 * H;
+    const float* W2 = b1 + H;
+    const float* b2 = W2 + H * H;
+    const float* W3 = b2 + H;
+    const float* b3 = W3 + 4 * H;
+    float h1[HC > 0 ? HC : kMaxHidden];
+#pragma unroll
+    for (int j = 0; j < H; ++j) {
+        float acc = b1[j];
+        acc = __fadd_rn(acc, __fmul_rn(W1[4 * j + 0], x0));
+        acc = __fadd_rn(acc, __fmul_rn(W1[4 * j + 1], x1));
+        acc = __fadd_rn(acc, __fmul_rn(W1[4 * j + 2], x2));
+        acc = __fadd_rn(acc, __fmul_rn(W1[4 * j + 3], x3));
+        h1[j] = acc > 0.0f ? acc : 0.0f;
+    }
+    float o0 = b3[0], o1 = b3[1], o2 = b3[2], o3 = b3[3];
+#pragma unroll 4
+    for (int j = 0; j < H; ++j) {
+        float acc = b2[j];
+#pragma unroll
+        for (int i = 0; i < H; ++i) acc = __fadd_rn(acc, __fmul_rn(W2[j * H + i], h1[i]));
+        float h2 = acc > 0.0f ? acc : 0.0f;
+        o0 = __fadd_rn(o0, __fmul_rn(W3[0 * H + j], h2));
+        o1 = __fadd_rn(o1, __fmul_rn(W3[1 * H + j], h2));
+        o2 = __fadd_rn(o2, __fmul_rn(W3[2 * H + j], h2));
+        o3 = __fadd_rn(o3, __fmul_rn(W3[3 * H + j], h2));
+    }
+    logits[0] = o0; logits[1] = o1; logits[2] = o2; logits[3] = o3;
+    if (o0 != o0 || o1 != o1 || o2 != o2 || o3 != o3) return 3;
+    int cls = 0;
+    float best = o0;
+    if (o1 > best) { best = o1; cls = 1; }
+    if (o2 > best) { best = o2; cls = 2; }
+    if (o3 > best) { best = o3; cls = 3; }
+    return cls;
+}
+
+__device__ __forceinline__ int controller_decide_any(const float* sW, int H, float x0, float x1, float x2,
+                                                     float x3, float logits[4]) {
+    if (H == 32) return controller_decide<32>(sW, H, x0, x1, x2, x3, logits);
+    return controller_decide<0>(sW, H, x0, x1, x2, x3, logits);
+}
+
+// kvq_select_bits: one thread per token.
+__global__ void __launch_bounds__(128)
+k_select_bits(const float* __restrict__ feats, int n, const float* __restrict__ gW, int H,
+              uint8_t* __restrict__ bits, float* __restrict__ logits_opt) {
+    extern __shared__ float sW[];
+    controller_stage(sW, gW, H);
+    __syncthreads();
+    int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n) return;
+    float4 f = reinterpret_cast<const float4*>(feats)[t];
+    float lg[4];
+    int cls = controller_decide_any(sW, H, f.x, f.y, f.z, f.w, lg);
+    bits[t] = (uint8_t)pool_bits(cls);
+    if (logits_opt) reinterpret_cast<float4*>(logits_opt)[t] = make_float4(lg[0], lg[1], lg[2], lg[3]);
+}
+
+}  // namespace kvq

@@ -1,0 +1,60 @@
+// Canonical copy of cached tokens, position by position: looks every token up
+// through the per-token index word (pool << 30 | slot) and de-interleaves its
+// rows from the tile records into plain 128-byte rows (packed codes first,
+// zero tail) plus {scale, zero-point} pairs.  Used to compare the store with
+// other implementations of the quantizer named in Eq. 24.
+#pragma once
+#include "kvq_common.cuh"
+
+namespace kvq {
+
+struct ExportParams {
+    StoreView store;
+    int layer, b0, nb, pos0, n;
+    uint8_t* bits;          // [nb][n]
+    uint32_t* pool_slot;    // [nb][n]
+    uint4* k_codes;         // [nb][n][kv_heads][8] (16-byte units)
+    uint4* v_codes;
+    uint16_t* k_meta;       // [nb][n][kv_heads][2]
+    uint16_t* v_meta;
+};
+
+// grid = (n, nb), block = 128.
+__global__ void __launch_bounds__(128)
+k_export(ExportParams p) {
+    const int i = blockIdx.x, bi = blockIdx.y, b = p.b0 + bi;
+    const StoreView& s = p.store;
+    const uint32_t word = s.index[((size_t)p.layer * s.batch + b) * s.max_ctx + p.pos0 + i];
+    const int cls = (int)(word >> 30);
+    const uint32_t slot = word & 0x3fffffffu;
+    const int W = pool_chunks(cls);
+    const size_t tok = (size_t)bi * p.n + i;
+    if (threadIdx.x == 0) {
+        if (p.bits) p.bits[tok] = (uint8_t)pool_bits(cls);
+        if (p.pool_slot) p.pool_slot[tok] = word;
+    }
+    const int items = s.kv_heads * 2 * 8;              // (head, tensor, 16-byte chunk)
+    for (int it = threadIdx.x; it < items; it += blockDim.x) {
+        const int j = it & 7, tensor = (it >> 3) & 1, h = it >> 4;
+        uint4* dst = tensor ? p.v_codes : p.k_codes;
+        if (!dst) continue;
+        const uint8_t* rec = s.pool[cls] + tile_offset(s, cls, p.layer, b, h, (int)(slot >> 5));
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (j < W) v = *reinterpret_cast<const uint4*>(rec + (size_t)tensor * W * 512 + j * 512 + (slot & 31) * 16);
+        dst[(tok * s.kv_heads + h) * 8 + j] = v;
+    }
+    for (int it = threadIdx.x; it < s.kv_heads * 2; it += blockDim.x) {
+        const int tensor = it & 1, h = it >> 1;
+        uint16_t* dst = tensor ? p.v_meta : p.k_meta;
+        if (!dst) continue;
+        uint32_t m = 0;
+        if (cls < 3) {
+            const uint8_t* rec = s.pool[cls] + tile_offset(s, cls, p.layer, b, h, (int)(slot >> 5));
+            m = *reinterpret_cast<const uint32_t*>(rec + 2 * W * 512 + tensor * 128 + (slot & 31) * 4);
+        }
+        dst[(tok * s.kv_heads + h) * 2 + 0] = (uint16_t)(m & 0xffffu);
+        dst[(tok * s.kv_heads + h) * 2 + 1] = (uint16_t)(m >> 16);
+    }
+}
+
+}  // namespace kvq

@@ -1,0 +1,493 @@
+// Host side of the C ABI declared in include/kvq.h: handle, argument checks,
+// launch planning.  All arithmetic of the method runs in the kernels included
+// below; nothing here computes on the CPU.
+#include "../../include/kvq.h"
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kvq_common.cuh"
+#include "k_controller.cuh"
+#include "k_append.cuh"
+#include "k_decode.cuh"
+#include "k_export.cuh"
+
+using namespace kvq;
+
+struct kvq_ctx {
+    int device = 0, sm_count = 0;
+    int layers = 0, q_heads = 0, kv_heads = 0, max_ctx = 0, batch = 0;
+    StoreView store{};
+    uint8_t* pool_block = nullptr;       // the four pools, one allocation
+    uint32_t* counts = nullptr;          // [2][layers][batch][4], double-buffered pool fills
+    std::vector<int> len;                // host mirror: tokens per sequence, per layer
+    std::vector<int> cur;                // which counts buffer is current, per layer
+    uint8_t* cls = nullptr;              // append scratch [batch][max_ctx]
+    uint4* hist = nullptr;               // append scratch [batch][max chunks]
+    float* ctrl = nullptr;               // controller parameter block
+    int hidden = 0;
+    float* part_o = nullptr;             // decode scratch [batch][q_heads][kMaxSplits][64]
+    float2* part_ml = nullptr;           //                [batch][q_heads][kMaxSplits]
+    int splits_override = 0;
+    uint32_t* flags = nullptr;
+    // device staging for the host-buffer entry points
+    float* st_feats = nullptr;
+    __half *st_K = nullptr, *st_V = nullptr, *st_Q = nullptr, *st_O = nullptr;
+    uint8_t* st_bits = nullptr;
+    uint8_t* st_export = nullptr;
+    uint64_t device_bytes = 0, launches = 0;
+    cudaError_t last_err = cudaSuccess;
+};
+
+namespace {
+
+struct DeviceGuard {                     // make the handle's device current for the duration of a call
+    int prev = -1;
+    explicit DeviceGuard(int dev) {
+        cudaGetDevice(&prev);
+        if (prev != dev) cudaSetDevice(dev);
+        else prev = -1;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+#define KVQ_CUDA(ctx, call)                         \
+    do {                                            \
+        cudaError_t e__ = (call);                   \
+        if (e__ != cudaSuccess) {                   \
+            (ctx)->last_err = e__;                  \
+            return KVQ_ERR_CUDA;                    \
+        }                                           \
+    } while (0)
+
+template <typename T>
+cudaError_t dev_alloc(kvq_ctx* c, T** p, size_t bytes) {
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), bytes ? bytes : 1);
+    if (e == cudaSuccess) c->device_bytes += bytes;
+    return e;
+}
+
+void free_all(kvq_ctx* c) {
+    cudaFree(c->pool_block);
+    cudaFree(c->store.index);
+    cudaFree(c->counts);
+    cudaFree(c->cls);
+    cudaFree(c->hist);
+    cudaFree(c->ctrl);
+    cudaFree(c->part_o);
+    cudaFree(c->part_ml);
+    cudaFree(c->flags);
+    cudaFree(c->st_feats);
+    cudaFree(c->st_K);
+    cudaFree(c->st_V);
+    cudaFree(c->st_Q);
+    cudaFree(c->st_O);
+    cudaFree(c->st_bits);
+    cudaFree(c->st_export);
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline uint32_t* counts_of(kvq_ctx* c, int which, int layer) {
+    return c->counts + ((size_t)which * c->layers + layer) * c->batch * 4;
+}
+
+int check_layer(kvq_ctx* c, int layer) { return (c && layer >= 0 && layer < c->layers) ? KVQ_OK : KVQ_ERR_ARG; }
+
+size_t controller_smem(int hidden) { return sizeof(float) * (size_t)controller_floats(hidden); }
+
+// Shared by kvq_append and kvq_append_fused.
+int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8_t* bits, const float* feats,
+                uint8_t* bits_out, int n_new, cudaStream_t st) {
+    if (check_layer(c, layer) != KVQ_OK || n_new < 0) return KVQ_ERR_ARG;
+    if (n_new == 0) return KVQ_OK;
+    if (!K || !V || !aligned16(K) || !aligned16(V)) return KVQ_ERR_ARG;
+    const bool fused = feats != nullptr;
+    if (fused) {
+        if (!aligned16(feats)) return KVQ_ERR_ARG;
+        if (c->hidden == 0) return KVQ_ERR_NO_CONTROLLER;
+    } else if (!bits) {
+        return KVQ_ERR_ARG;
+    }
+    if (c->len[layer] + n_new > c->max_ctx) return KVQ_ERR_CAPACITY;
+    DeviceGuard guard(c->device);
+
+    AppendParams p{};
+    p.store = c->store;
+    p.K = static_cast<const __half*>(K);
+    p.V = static_cast<const __half*>(V);
+    p.bits = bits;
+    p.feats = feats;
+    p.ctrl = c->ctrl;
+    p.hidden = c->hidden;
+    p.bits_out = bits_out;
+    p.cls = c->cls;
+    p.hist = c->hist;
+    p.counts_in = counts_of(c, c->cur[layer], layer);
+    p.counts_out = counts_of(c, c->cur[layer] ^ 1, layer);
+    p.layer = layer;
+    p.n_new = n_new;
+    p.pos0 = c->len[layer];
+    p.nchunks = (n_new + kChunkTokens - 1) / kChunkTokens;
+    // enough CTAs to fill the device: split the KV heads into groups when chunks x batch is small
+    int want_groups = (2 * c->sm_count + p.nchunks * c->batch - 1) / (p.nchunks * c->batch);
+    int groups = want_groups < 1 ? 1 : (want_groups > c->kv_heads ? c->kv_heads : want_groups);
+    p.heads_per_group = (c->kv_heads + groups - 1) / groups;
+    groups = (c->kv_heads + p.heads_per_group - 1) / p.heads_per_group;
+
+    const size_t smem = fused ? controller_smem(c->hidden) : 0;
+    dim3 grid_q(p.nchunks, groups, c->batch);
+    if (p.nchunks == 1) {
+        if (fused) k_quant_pack<2><<<grid_q, kChunkTokens, smem, st>>>(p);
+        else k_quant_pack<1><<<grid_q, kChunkTokens, 0, st>>>(p);
+        c->launches += 1;
+    } else {
+        dim3 grid_c(p.nchunks, c->batch);
+        if (fused) k_classify<true><<<grid_c, kChunkTokens, smem, st>>>(p);
+        else k_classify<false><<<grid_c, kChunkTokens, 0, st>>>(p);
+        k_quant_pack<0><<<grid_q, kChunkTokens, 0, st>>>(p);
+        c->launches += 2;
+    }
+    KVQ_CUDA(c, cudaGetLastError());
+    c->cur[layer] ^= 1;
+    c->len[layer] += n_new;
+    return KVQ_OK;
+}
+
+int choose_splits(kvq_ctx* c, int len) {
+    if (c->splits_override > 0) return c->splits_override;
+    const int tiles = (len + kTileTokens - 1) / kTileTokens + (kNumPools - 1);
+    const int units = c->batch * c->q_heads;
+    int s = (24 * c->sm_count + units - 1) / units;              // ~8 waves of 3 CTAs per SM
+    const int by_work = tiles / (2 * kDecodeWarps);              // at least two tiles per warp
+    if (s > by_work) s = by_work;
+    if (s > kMaxSplits) s = kMaxSplits;
+    if (s < 1) s = 1;
+    return s;
+}
+
+int export_impl(kvq_ctx* c, int layer, int b0, int nb, int pos0, int n, uint8_t* bits, uint32_t* pool_slot,
+                void* k_codes, void* v_codes, uint16_t* k_meta, uint16_t* v_meta, cudaStream_t st) {
+    ExportParams p{};
+    p.store = c->store;
+    p.layer = layer;
+    p.b0 = b0;
+    p.nb = nb;
+    p.pos0 = pos0;
+    p.n = n;
+    p.bits = bits;
+    p.pool_slot = pool_slot;
+    p.k_codes = static_cast<uint4*>(k_codes);
+    p.v_codes = static_cast<uint4*>(v_codes);
+    p.k_meta = k_meta;
+    p.v_meta = v_meta;
+    k_export<<<dim3(n, nb), 128, 0, st>>>(p);
+    c->launches += 1;
+    KVQ_CUDA(c, cudaGetLastError());
+    return KVQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int kvq_create(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch) {
+    if (!out) return KVQ_ERR_ARG;
+    *out = nullptr;
+    if (layers < 1 || q_heads < 1 || kv_heads < 1 || batch < 1 || max_ctx < 1) return KVQ_ERR_ARG;
+    if (head_dim != kHeadDim || q_heads % kv_heads != 0) return KVQ_ERR_ARG;
+    if (max_ctx > (1 << 30) - 1 || batch > 65535 || q_heads > 65535) return KVQ_ERR_ARG;
+    kvq_ctx* c = new (std::nothrow) kvq_ctx();
+    if (!c) return KVQ_ERR_NOMEM;
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
+    if (e != cudaSuccess) {
+        delete c;
+        return KVQ_ERR_CUDA;
+    }
+    c->layers = layers;
+    c->q_heads = q_heads;
+    c->kv_heads = kv_heads;
+    c->max_ctx = max_ctx;
+    c->batch = batch;
+    c->len.assign(layers, 0);
+    c->cur.assign(layers, 0);
+    StoreView& s = c->store;
+    s.layers = layers;
+    s.batch = batch;
+    s.kv_heads = kv_heads;
+    s.q_heads = q_heads;
+    s.max_ctx = max_ctx;
+    s.cap_tiles = (max_ctx + kTileTokens - 1) / kTileTokens;
+
+    const size_t seqs = (size_t)layers * batch * kv_heads;
+    size_t pool_bytes[kNumPools], total = 0;
+    for (int k = 0; k < kNumPools; ++k) {
+        pool_bytes[k] = seqs * s.cap_tiles * (size_t)pool_rec_bytes(k);
+        total += pool_bytes[k];
+    }
+    const size_t max_chunks = (size_t)(max_ctx + kChunkTokens - 1) / kChunkTokens;
+    const size_t units = (size_t)batch * q_heads;
+    bool ok = dev_alloc(c, &c->pool_block, total) == cudaSuccess;
+    ok = ok && dev_alloc(c, &s.index, sizeof(uint32_t) * (size_t)layers * batch * max_ctx) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->counts, sizeof(uint32_t) * 2 * (size_t)layers * batch * 4) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->cls, (size_t)batch * max_ctx) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->hist, sizeof(uint4) * batch * max_chunks) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->ctrl, controller_smem(kMaxHidden)) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->part_o, sizeof(float) * units * kMaxSplits * kHeadDim) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->part_ml, sizeof(float2) * units * kMaxSplits) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->flags, sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->st_feats, sizeof(float) * 4 * batch) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->st_K, sizeof(__half) * (size_t)batch * kv_heads * kHeadDim) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->st_V, sizeof(__half) * (size_t)batch * kv_heads * kHeadDim) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->st_Q, sizeof(__half) * units * kHeadDim) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->st_O, sizeof(__half) * units * kHeadDim) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->st_bits, (size_t)batch) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->st_export, (size_t)kv_heads * (2 * KVQ_EXPORT_ROW_BYTES + 8) + 16) == cudaSuccess;
+    if (ok) {
+        size_t off = 0;
+        for (int k = 0; k < kNumPools; ++k) {
+            s.pool[k] = c->pool_block + off;
+            off += pool_bytes[k];
+        }
+        s.flags = c->flags;
+        ok = cudaMemset(c->pool_block, 0, total) == cudaSuccess;
+        ok = ok && cudaMemset(s.index, 0, sizeof(uint32_t) * (size_t)layers * batch * max_ctx) == cudaSuccess;
+        ok = ok && cudaMemset(c->counts, 0, sizeof(uint32_t) * 2 * (size_t)layers * batch * 4) == cudaSuccess;
+        ok = ok && cudaMemset(c->flags, 0, sizeof(uint32_t)) == cudaSuccess;
+        // the controller block may exceed the default 48 KB of dynamic shared memory
+        const int smem_max = (int)controller_smem(kMaxHidden);
+        ok = ok && cudaFuncSetAttribute(k_select_bits, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(k_classify<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(k_quant_pack<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
+        ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+    }
+    if (!ok) {
+        cudaError_t err = cudaGetLastError();
+        free_all(c);
+        delete c;
+        return err == cudaErrorMemoryAllocation ? KVQ_ERR_NOMEM : KVQ_ERR_CUDA;
+    }
+    *out = c;
+    return KVQ_OK;
+}
+
+int kvq_destroy(kvq_ctx* c) {
+    if (!c) return KVQ_OK;
+    DeviceGuard guard(c->device);
+    cudaDeviceSynchronize();
+    free_all(c);
+    delete c;
+    return KVQ_OK;
+}
+
+int kvq_set_controller(kvq_ctx* c, int hidden, const float* W1, const float* b1, const float* W2, const float* b2,
+                       const float* W3, const float* b3) {
+    if (!c || hidden < 1 || hidden > kMaxHidden || !W1 || !b1 || !W2 || !b2 || !W3 || !b3) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    std::vector<float> blk;
+    blk.reserve(controller_floats(hidden));
+    blk.insert(blk.end(), W1, W1 + 4 * hidden);
+    blk.insert(blk.end(), b1, b1 + hidden);
+    blk.insert(blk.end(), W2, W2 + (size_t)hidden * hidden);
+    blk.insert(blk.end(), b2, b2 + hidden);
+    blk.insert(blk.end(), W3, W3 + 4 * hidden);
+    blk.insert(blk.end(), b3, b3 + 4);
+    KVQ_CUDA(c, cudaDeviceSynchronize());                          // earlier launches may still read the old block
+    KVQ_CUDA(c, cudaMemcpy(c->ctrl, blk.data(), sizeof(float) * blk.size(), cudaMemcpyHostToDevice));
+    c->hidden = hidden;
+    return KVQ_OK;
+}
+
+int kvq_select_bits(kvq_ctx* c, const float* feats, int n, uint8_t* bits, float* logits_opt, void* stream) {
+    if (!c || n < 0) return KVQ_ERR_ARG;
+    if (n == 0) return KVQ_OK;
+    if (!feats || !bits || !aligned16(feats) || (logits_opt && !aligned16(logits_opt))) return KVQ_ERR_ARG;
+    if (c->hidden == 0) return KVQ_ERR_NO_CONTROLLER;
+    DeviceGuard guard(c->device);
+    k_select_bits<<<(n + 127) / 128, 128, controller_smem(c->hidden), static_cast<cudaStream_t>(stream)>>>(
+        feats, n, c->ctrl, c->hidden, bits, logits_opt);
+    c->launches += 1;
+    KVQ_CUDA(c, cudaGetLastError());
+    return KVQ_OK;
+}
+
+int kvq_append(kvq_ctx* c, int layer, const void* K, const void* V, const uint8_t* bits, int n_new, void* stream) {
+    if (!c) return KVQ_ERR_ARG;
+    return append_impl(c, layer, K, V, bits, nullptr, nullptr, n_new, static_cast<cudaStream_t>(stream));
+}
+
+int kvq_append_fused(kvq_ctx* c, int layer, const void* K, const void* V, const float* feats, int n_new,
+                     uint8_t* bits_out_opt, void* stream) {
+    if (!c || (n_new > 0 && !feats)) return KVQ_ERR_ARG;
+    return append_impl(c, layer, K, V, nullptr, feats, bits_out_opt, n_new, static_cast<cudaStream_t>(stream));
+}
+
+int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream) {
+    if (check_layer(c, layer) != KVQ_OK || !Q || !O) return KVQ_ERR_ARG;
+    if (c->len[layer] == 0) return KVQ_ERR_EMPTY;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DecodeParams p{};
+    p.store = c->store;
+    p.counts = counts_of(c, c->cur[layer], layer);
+    p.Q = static_cast<const __half*>(Q);
+    p.O = static_cast<__half*>(O);
+    p.part_o = c->part_o;
+    p.part_ml = c->part_ml;
+    p.layer = layer;
+    p.splits = choose_splits(c, c->len[layer]);
+    p.group = c->q_heads / c->kv_heads;
+    k_decode_split<<<dim3(p.splits, c->q_heads, c->batch), kDecodeThreads, 0, st>>>(p);
+    k_decode_merge<<<c->batch * c->q_heads, kHeadDim, 0, st>>>(p);
+    c->launches += 2;
+    KVQ_CUDA(c, cudaGetLastError());
+    return KVQ_OK;
+}
+
+int kvq_decode_step_host(kvq_ctx* c, int layer, const float* feats, const void* K, const void* V, const void* Q,
+                         void* O, uint8_t* bits_out_opt, void* stream) {
+    if (check_layer(c, layer) != KVQ_OK || !feats || !K || !V || !Q || !O) return KVQ_ERR_ARG;
+    if (c->hidden == 0) return KVQ_ERR_NO_CONTROLLER;
+    if (c->len[layer] + 1 > c->max_ctx) return KVQ_ERR_CAPACITY;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t kv_bytes = sizeof(__half) * (size_t)c->batch * c->kv_heads * kHeadDim;
+    const size_t q_bytes = sizeof(__half) * (size_t)c->batch * c->q_heads * kHeadDim;
+    KVQ_CUDA(c, cudaMemcpyAsync(c->st_feats, feats, sizeof(float) * 4 * c->batch, cudaMemcpyHostToDevice, st));
+    KVQ_CUDA(c, cudaMemcpyAsync(c->st_K, K, kv_bytes, cudaMemcpyHostToDevice, st));
+    KVQ_CUDA(c, cudaMemcpyAsync(c->st_V, V, kv_bytes, cudaMemcpyHostToDevice, st));
+    KVQ_CUDA(c, cudaMemcpyAsync(c->st_Q, Q, q_bytes, cudaMemcpyHostToDevice, st));
+    int rc = kvq_append_fused(c, layer, c->st_K, c->st_V, c->st_feats, 1, c->st_bits, stream);
+    if (rc != KVQ_OK) return rc;
+    rc = kvq_decode_attn(c, layer, c->st_Q, c->st_O, stream);
+    if (rc != KVQ_OK) return rc;
+    KVQ_CUDA(c, cudaMemcpyAsync(O, c->st_O, q_bytes, cudaMemcpyDeviceToHost, st));
+    if (bits_out_opt) KVQ_CUDA(c, cudaMemcpyAsync(bits_out_opt, c->st_bits, c->batch, cudaMemcpyDeviceToHost, st));
+    KVQ_CUDA(c, cudaStreamSynchronize(st));
+    return KVQ_OK;
+}
+
+int kvq_reset(kvq_ctx* c, void* stream) {
+    if (!c) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    KVQ_CUDA(c, cudaMemsetAsync(c->counts, 0, sizeof(uint32_t) * 2 * (size_t)c->layers * c->batch * 4,
+                                static_cast<cudaStream_t>(stream)));
+    for (int l = 0; l < c->layers; ++l) {
+        c->len[l] = 0;
+        c->cur[l] = 0;
+    }
+    return KVQ_OK;
+}
+
+int kvq_seq_len(kvq_ctx* c, int layer, int* host_len_out) {
+    if (check_layer(c, layer) != KVQ_OK || !host_len_out) return KVQ_ERR_ARG;
+    *host_len_out = c->len[layer];
+    return KVQ_OK;
+}
+
+int kvq_set_splits(kvq_ctx* c, int splits) {
+    if (!c || splits < 0 || splits > kMaxSplits) return KVQ_ERR_ARG;
+    c->splits_override = splits;
+    return KVQ_OK;
+}
+
+int kvq_export_range(kvq_ctx* c, int layer, int pos0, int n, uint8_t* bits, uint32_t* pool_slot, void* k_codes,
+                     void* v_codes, uint16_t* k_meta, uint16_t* v_meta, void* stream) {
+    if (check_layer(c, layer) != KVQ_OK || pos0 < 0 || n < 0 || pos0 + n > c->len[layer]) return KVQ_ERR_ARG;
+    if (n == 0) return KVQ_OK;
+    if ((k_codes && !aligned16(k_codes)) || (v_codes && !aligned16(v_codes))) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    return export_impl(c, layer, 0, c->batch, pos0, n, bits, pool_slot, k_codes, v_codes, k_meta, v_meta,
+                       static_cast<cudaStream_t>(stream));
+}
+
+int kvq_export_token(kvq_ctx* c, int layer, int b, int pos, uint8_t* bits, uint32_t* pool_slot, void* k_codes,
+                     void* v_codes, uint16_t* k_meta, uint16_t* v_meta) {
+    if (check_layer(c, layer) != KVQ_OK || b < 0 || b >= c->batch || pos < 0 || pos >= c->len[layer])
+        return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    const size_t row = (size_t)c->kv_heads * KVQ_EXPORT_ROW_BYTES, meta = (size_t)c->kv_heads * 4;
+    uint8_t* d_k = c->st_export;
+    uint8_t* d_v = d_k + row;
+    uint8_t* d_km = d_v + row;
+    uint8_t* d_vm = d_km + meta;
+    uint8_t* d_ps = d_vm + meta;           // 4 bytes pool_slot, then 1 byte bits
+    KVQ_CUDA(c, cudaDeviceSynchronize());
+    int rc = export_impl(c, layer, b, 1, pos, 1, d_ps + 4, reinterpret_cast<uint32_t*>(d_ps), d_k, d_v,
+                         reinterpret_cast<uint16_t*>(d_km), reinterpret_cast<uint16_t*>(d_vm), nullptr);
+    if (rc != KVQ_OK) return rc;
+    if (k_codes) KVQ_CUDA(c, cudaMemcpy(k_codes, d_k, row, cudaMemcpyDeviceToHost));
+    if (v_codes) KVQ_CUDA(c, cudaMemcpy(v_codes, d_v, row, cudaMemcpyDeviceToHost));
+    if (k_meta) KVQ_CUDA(c, cudaMemcpy(k_meta, d_km, meta, cudaMemcpyDeviceToHost));
+    if (v_meta) KVQ_CUDA(c, cudaMemcpy(v_meta, d_vm, meta, cudaMemcpyDeviceToHost));
+    if (pool_slot) KVQ_CUDA(c, cudaMemcpy(pool_slot, d_ps, 4, cudaMemcpyDeviceToHost));
+    if (bits) KVQ_CUDA(c, cudaMemcpy(bits, d_ps + 4, 1, cudaMemcpyDeviceToHost));
+    KVQ_CUDA(c, cudaDeviceSynchronize());
+    return KVQ_OK;
+}
+
+int kvq_stats(kvq_ctx* c, int layer, uint32_t* host_counts, uint64_t* resident_bytes, double* expected_bits) {
+    if (check_layer(c, layer) != KVQ_OK) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    std::vector<uint32_t> cnt((size_t)c->batch * 4);
+    KVQ_CUDA(c, cudaDeviceSynchronize());
+    KVQ_CUDA(c, cudaMemcpy(cnt.data(), counts_of(c, c->cur[layer], layer), sizeof(uint32_t) * cnt.size(),
+                           cudaMemcpyDeviceToHost));
+    uint64_t bytes = 0, tokens = 0, bit_sum = 0;
+    for (int b = 0; b < c->batch; ++b)
+        for (int k = 0; k < kNumPools; ++k) {
+            const uint64_t n = cnt[(size_t)b * 4 + k];
+            bytes += n * (uint64_t)c->kv_heads * pool_row_bytes(k);
+            tokens += n;
+            bit_sum += n * (uint64_t)pool_bits(k);
+        }
+    if (host_counts) memcpy(host_counts, cnt.data(), sizeof(uint32_t) * cnt.size());
+    if (resident_bytes) *resident_bytes = bytes;
+    if (expected_bits) *expected_bits = tokens ? (double)bit_sum / (double)tokens : 0.0;
+    return KVQ_OK;
+}
+
+int kvq_device_status(kvq_ctx* c, uint32_t* host_flags_out) {
+    if (!c || !host_flags_out) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    KVQ_CUDA(c, cudaDeviceSynchronize());
+    KVQ_CUDA(c, cudaMemcpy(host_flags_out, c->flags, sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    KVQ_CUDA(c, cudaMemset(c->flags, 0, sizeof(uint32_t)));
+    return *host_flags_out ? KVQ_ERR_DEVICE_FLAG : KVQ_OK;
+}
+
+int kvq_device_bytes(kvq_ctx* c, uint64_t* host_bytes_out) {
+    if (!c || !host_bytes_out) return KVQ_ERR_ARG;
+    *host_bytes_out = c->device_bytes;
+    return KVQ_OK;
+}
+
+int kvq_launch_count(kvq_ctx* c, uint64_t* host_count_out) {
+    if (!c || !host_count_out) return KVQ_ERR_ARG;
+    *host_count_out = c->launches;
+    return KVQ_OK;
+}
+
+int kvq_last_cuda_error(kvq_ctx* c) { return c ? (int)c->last_err : 0; }
+
+const char* kvq_strerror(int code) {
+    switch (code) {
+    case KVQ_OK: return "ok";
+    case KVQ_ERR_ARG: return "invalid argument";
+    case KVQ_ERR_CAPACITY: return "append would exceed max_ctx";
+    case KVQ_ERR_NO_CONTROLLER: return "controller weights not set";
+    case KVQ_ERR_CUDA: return "CUDA call failed";
+    case KVQ_ERR_EMPTY: return "layer holds no token";
+    case KVQ_ERR_DEVICE_FLAG: return "a kernel recorded a problem";
+    case KVQ_ERR_NOMEM: return "out of memory";
+    default: return "unknown error";
+    }
+}
+
+}  // extern "C"
