@@ -184,6 +184,17 @@ int kvq_export_token(kvq_ctx* ctx, int layer, int b, int pos,
 int kvq_stats(kvq_ctx* ctx, int layer, uint32_t* host_counts, uint64_t* resident_bytes,
               double* expected_bits);
 
+/*
+ * Timing hooks for benchmarks.  While profiling is on, kvq_decode_attn records CUDA
+ * events on its stream before the split kernel, between the two kernels and after the
+ * merge kernel (up to 1024 calls are kept; later calls are not recorded).
+ * kvq_profile_read synchronizes, adds up the elapsed times of the recorded calls into
+ * split_ms_total / merge_ms_total (host doubles, may be NULL), stores their number in
+ * calls (host int, may be NULL) and forgets them.
+ */
+int kvq_set_profiling(kvq_ctx* ctx, int on);
+int kvq_profile_read(kvq_ctx* ctx, double* split_ms_total, double* merge_ms_total, int* calls);
+
 /* Device flags recorded by kernels since the last call (host uint32, cleared on read). */
 #define KVQ_FLAG_BAD_BITS 1u      /* a bit-width outside {2,4,8,16} was appended (stored as fp16) */
 int kvq_device_status(kvq_ctx* ctx, uint32_t* host_flags_out);

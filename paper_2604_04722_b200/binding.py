@@ -43,6 +43,8 @@ SIGNATURES = {
     "kvq_export_range": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvq_export_token": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvq_stats": (_i, [_vp, _i, _vp, _u64p, C.POINTER(C.c_double)]),
+    "kvq_set_profiling": (_i, [_vp, _i]),
+    "kvq_profile_read": (_i, [_vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_i)]),
     "kvq_device_status": (_i, [_vp, C.POINTER(C.c_uint32)]),
     "kvq_device_bytes": (_i, [_vp, _u64p]),
     "kvq_launch_count": (_i, [_vp, _u64p]),
@@ -183,6 +185,17 @@ def kvq_stats(ctx: int, layer: int, batch: int):
     eb = C.c_double()
     check(lib().kvq_stats(ctx, layer, _ptr(counts), C.byref(rb), C.byref(eb)), "kvq_stats")
     return counts, rb.value, eb.value
+
+
+def kvq_set_profiling(ctx: int, on: bool) -> None:
+    check(lib().kvq_set_profiling(ctx, int(bool(on))), "kvq_set_profiling")
+
+
+def kvq_profile_read(ctx: int):
+    """Returns (split_ms_total, merge_ms_total, calls) of the decode calls recorded since the last read."""
+    a, b, n = C.c_double(), C.c_double(), _i()
+    check(lib().kvq_profile_read(ctx, C.byref(a), C.byref(b), C.byref(n)), "kvq_profile_read")
+    return a.value, b.value, n.value
 
 
 def kvq_device_status(ctx: int) -> int:

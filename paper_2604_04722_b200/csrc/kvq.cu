@@ -38,6 +38,9 @@ struct kvq_ctx {
     __half *st_K = nullptr, *st_V = nullptr, *st_Q = nullptr, *st_O = nullptr;
     uint8_t* st_bits = nullptr;
     uint8_t* st_export = nullptr;
+    bool profiling = false;              // decode timing hooks
+    std::vector<cudaEvent_t> prof_ev;    // 3 events per recorded call
+    int prof_calls = 0;
     uint64_t device_bytes = 0, launches = 0;
     cudaError_t last_err = cudaSuccess;
 };
@@ -72,7 +75,11 @@ cudaError_t dev_alloc(kvq_ctx* c, T** p, size_t bytes) {
     return e;
 }
 
+constexpr int kProfMaxCalls = 1024;
+
 void free_all(kvq_ctx* c) {
+    for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+    c->prof_ev.clear();
     cudaFree(c->pool_block);
     cudaFree(c->store.index);
     cudaFree(c->counts);
@@ -343,8 +350,16 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
     p.layer = layer;
     p.splits = choose_splits(c, c->len[layer]);
     p.group = c->q_heads / c->kv_heads;
+    const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
+    cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 3] : nullptr;
+    if (rec) cudaEventRecord(ev[0], st);
     k_decode_split<<<dim3(p.splits, c->q_heads, c->batch), kDecodeThreads, 0, st>>>(p);
+    if (rec) cudaEventRecord(ev[1], st);
     k_decode_merge<<<c->batch * c->q_heads, kHeadDim, 0, st>>>(p);
+    if (rec) {
+        cudaEventRecord(ev[2], st);
+        c->prof_calls += 1;
+    }
     c->launches += 2;
     KVQ_CUDA(c, cudaGetLastError());
     return KVQ_OK;
@@ -450,6 +465,44 @@ int kvq_stats(kvq_ctx* c, int layer, uint32_t* host_counts, uint64_t* resident_b
     if (host_counts) memcpy(host_counts, cnt.data(), sizeof(uint32_t) * cnt.size());
     if (resident_bytes) *resident_bytes = bytes;
     if (expected_bits) *expected_bits = tokens ? (double)bit_sum / (double)tokens : 0.0;
+    return KVQ_OK;
+}
+
+int kvq_set_profiling(kvq_ctx* c, int on) {
+    if (!c) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    if (on && c->prof_ev.empty()) {
+        c->prof_ev.resize((size_t)kProfMaxCalls * 3);
+        for (size_t i = 0; i < c->prof_ev.size(); ++i) {
+            cudaError_t e = cudaEventCreate(&c->prof_ev[i]);
+            if (e != cudaSuccess) {
+                for (size_t j = 0; j < i; ++j) cudaEventDestroy(c->prof_ev[j]);
+                c->prof_ev.clear();
+                c->last_err = e;
+                return KVQ_ERR_CUDA;
+            }
+        }
+    }
+    c->profiling = on != 0;
+    return KVQ_OK;
+}
+
+int kvq_profile_read(kvq_ctx* c, double* split_ms_total, double* merge_ms_total, int* calls) {
+    if (!c) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    KVQ_CUDA(c, cudaDeviceSynchronize());
+    double s_ms = 0.0, m_ms = 0.0;
+    for (int i = 0; i < c->prof_calls; ++i) {
+        float a = 0.f, b = 0.f;
+        KVQ_CUDA(c, cudaEventElapsedTime(&a, c->prof_ev[(size_t)i * 3], c->prof_ev[(size_t)i * 3 + 1]));
+        KVQ_CUDA(c, cudaEventElapsedTime(&b, c->prof_ev[(size_t)i * 3 + 1], c->prof_ev[(size_t)i * 3 + 2]));
+        s_ms += a;
+        m_ms += b;
+    }
+    if (split_ms_total) *split_ms_total = s_ms;
+    if (merge_ms_total) *merge_ms_total = m_ms;
+    if (calls) *calls = c->prof_calls;
+    c->prof_calls = 0;
     return KVQ_OK;
 }
 

@@ -31,6 +31,7 @@ regenerated alone):
 from __future__ import annotations
 
 import math
+import os
 from dataclasses import dataclass, field
 from typing import Dict, Optional, Tuple
 
@@ -104,8 +105,10 @@ def _rows(seed: int, tag: int, layer: int, b: int, t0: int, n: int,
     rng = _rng(seed, tag, layer, b, t0)
     x = rng.standard_normal((n, kv_heads, head_dim), dtype=np.float32)
     ch = outlier_channels(seed, layer, kv_heads, head_dim, tag)
+    scale = np.ones((kv_heads, head_dim), dtype=np.float32)
     for h in range(kv_heads):
-        x[:, h, ch[h]] *= np.float32(8.0)
+        scale[h, ch[h]] = 8.0
+    x *= scale[None]
     return x.astype(np.float16)
 
 
@@ -122,10 +125,27 @@ def kv_rows(seed: int, layer: int, b: int, t0: int, n: int, kv_heads: int,
 
 def kv_batch(seed: int, layer: int, batch: int, t0: int, n: int, kv_heads: int,
              head_dim: int = 64) -> Tuple[np.ndarray, np.ndarray]:
-    """fp16 [batch][n][kv_heads][head_dim] for K and V."""
-    ks, vs = zip(*(kv_rows(seed, layer, b, t0, n, kv_heads, head_dim)
-                   for b in range(batch)))
-    return np.stack(ks), np.stack(vs)
+    """fp16 [batch][n][kv_heads][head_dim] for K and V.
+
+    Blocks are independent streams, so large batches are drawn by a thread pool
+    (numpy's generators release the GIL); the values do not depend on it.
+    """
+    K = np.empty((batch, n, kv_heads, head_dim), dtype=np.float16)
+    V = np.empty_like(K)
+
+    def fill(job):
+        b, tag, out = job
+        out[b] = _rows(seed, tag, layer, b, t0, n, kv_heads, head_dim)
+
+    jobs = [(b, tag, out) for b in range(batch) for tag, out in ((_TAG_K, K), (_TAG_V, V))]
+    if batch * n * kv_heads * head_dim < (1 << 22):
+        for j in jobs:
+            fill(j)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 1)) as ex:
+            list(ex.map(fill, jobs))
+    return K, V
 
 
 def queries(seed: int, layer: int, step: int, batch: int, q_heads: int,
