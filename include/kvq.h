@@ -197,6 +197,8 @@ int kvq_profile_read(kvq_ctx* ctx, double* split_ms_total, double* merge_ms_tota
 
 /* Device flags recorded by kernels since the last call (host uint32, cleared on read). */
 #define KVQ_FLAG_BAD_BITS 1u      /* a bit-width outside {2,4,8,16} was appended (stored as fp16) */
+#define KVQ_FLAG_WAIT_TIMEOUT 2u  /* a bounded wait on an async copy expired in kvq_decode_attn; that
+                                     call's output is invalid */
 int kvq_device_status(kvq_ctx* ctx, uint32_t* host_flags_out);
 
 /* Bytes of device memory the handle holds (pools + index + scratch). */

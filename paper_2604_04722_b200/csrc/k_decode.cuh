@@ -8,9 +8,18 @@
 // each CTA keeps an online softmax in fp32 and emits (m, l, o[64]); a second
 // kernel merges the parts.
 //
-// Work layout inside a CTA: one lane per token (a warp reads one 32-token tile
-// with coalesced 16-byte loads), so the q.k dot product needs no shuffles and
-// the output accumulators are per-lane partial sums reduced once at the end.
+// Data movement: the tiles of a part are cut into chunks of up to kStageBytes
+// contiguous bytes; chunks are dealt round-robin to the CTA's warps, and every
+// warp runs its own ring of kStages shared-memory buffers filled by 1-D bulk
+// async copies (cp.async.bulk, completion on an mbarrier), issued kStages
+// chunks ahead by lane 0.  No CTA-wide synchronisation happens in the main
+// loop.  Every mbarrier wait is bounded: on expiry the warp records
+// KVQ_FLAG_WAIT_TIMEOUT and leaves the loop.
+//
+// Work layout inside a warp: one lane per token (a 32-token tile is read with
+// conflict-free 16-byte shared loads), so the q.k dot product needs no
+// shuffles and the output accumulators are per-lane partial sums reduced once
+// at the end.
 //
 // Dequantization is hoisted out of the inner loops:
 //   q.khat = s_k * sum_i q_i c_i + z_k * sum_i q_i
@@ -25,13 +34,30 @@
 #pragma once
 #include "kvq_common.cuh"
 
+#ifndef KVQ_DECODE_STAGES
+#define KVQ_DECODE_STAGES 3
+#endif
+#ifndef KVQ_DECODE_WARPS
+#define KVQ_DECODE_WARPS 4
+#endif
+#ifndef KVQ_DECODE_MIN_CTAS
+#define KVQ_DECODE_MIN_CTAS 2
+#endif
+
 namespace kvq {
 
-constexpr int kDecodeThreads = 128;
-constexpr int kDecodeWarps = kDecodeThreads / 32;
+constexpr int kDecodeWarps = KVQ_DECODE_WARPS;
+constexpr int kDecodeThreads = kDecodeWarps * 32;
+constexpr int kStages = KVQ_DECODE_STAGES;
+constexpr int kStageBytes = 8704;                // two 8-bit tiles; 6 / 3 / 2 / 1 tiles of the four classes
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleSlack = 8.0f;            // the running maximum may lag by 2^8 before a rescale
 constexpr float kNegBig = -1.0e30f;
+constexpr uint32_t kWaitLimit = 1u << 20;        // mbarrier polls before a wait is abandoned
+constexpr uint32_t kFlagWaitTimeout = 2u;
+
+__host__ __device__ constexpr int tiles_per_stage(int c) { return kStageBytes / pool_rec_bytes(c); }
+constexpr size_t kDecodeSmemBytes = (size_t)kDecodeWarps * kStages * kStageBytes;
 
 struct DecodeParams {
     StoreView store;
@@ -42,6 +68,48 @@ struct DecodeParams {
     float2* part_ml;               // [batch][q_heads][splits]      (m in log2 units, l)
     int layer, splits, group;      // group = q_heads / kv_heads
 };
+
+// ---------------------------------------------------------------- PTX helpers
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t arrivals) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+// Bounded wait; false if the phase did not complete within kWaitLimit polls.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (uint32_t it = 0; it < kWaitLimit; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// 1-D bulk async copy global -> shared, completion counted in bytes on `bar`.
+// dst, src 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 __device__ __forceinline__ float pow2f(int e) { return __int_as_float((127 + e) << 23); }
 
@@ -81,40 +149,45 @@ struct Softmax {
 __device__ __forceinline__ float softmax_step(Softmax& st, float (&acc)[kHeadDim], float y) {
     const float tmax = warp_max(y);
     if (tmax > st.m + kRescaleSlack) {                 // warp-uniform
-        const float f = exp2f(st.m - tmax);
+        const float f = fast_exp2(st.m - tmax);
         st.m = tmax;
         st.l *= f;
         st.bsum *= f;
 #pragma unroll
         for (int j = 0; j < kHeadDim; ++j) acc[j] *= f;
     }
-    const float p = exp2f(y - st.m);
+    const float p = fast_exp2(y - st.m);
     st.l += p;
     return p;
 }
 
-// Walk the tiles [lo, hi) of one quantized pool that belong to this warp.
+// ---------------------------------------------------------------- tile consumers (data in shared memory)
+
 template <int CLS>
-__device__ __forceinline__ void walk_quantized(const uint8_t* __restrict__ base, int first, int hi, uint32_t cnt,
-                                               int lane, const float* q_s, float sumq, Softmax& st,
-                                               float (&acc)[kHeadDim]) {
-    constexpr int BITS = pool_bits(CLS), W = pool_chunks(CLS), REC = pool_rec_bytes(CLS);
-    constexpr int EPW = 32 / BITS;                     // elements per 32-bit word
-    constexpr int EPC = 4 * EPW;                       // elements per 16-byte chunk
-    float qk[kHeadDim];
+struct Quantized {
+    static constexpr int BITS = pool_bits(CLS), W = pool_chunks(CLS), REC = pool_rec_bytes(CLS);
+    static constexpr int EPW = 32 / BITS;              // elements per 32-bit word
+    static constexpr int EPC = 4 * EPW;                // elements per 16-byte chunk
+
+    // pre-scaled query and accumulator exponent domain of this class
+    __device__ static __forceinline__ void enter(const float* q_s, float (&qk)[kHeadDim], float (&acc)[kHeadDim]) {
 #pragma unroll
-    for (int i = 0; i < kHeadDim; ++i) {
-        qk[i] = q_s[i] * pow2f(100 - field_pos<BITS>(i % EPW));
-        acc[i] *= pow2f(field_pos<BITS>(i % EPW) - 49);           // into this pool's exponent domain
+        for (int i = 0; i < kHeadDim; ++i) {
+            qk[i] = q_s[i] * pow2f(100 - field_pos<BITS>(i % EPW));
+            acc[i] *= pow2f(field_pos<BITS>(i % EPW) - 49);
+        }
     }
-    for (int t = first; t < hi; t += kDecodeWarps) {
-        const uint8_t* rec = base + (size_t)t * REC;
-        const bool valid = (uint32_t)(t * kTileTokens + lane) < cnt;
-        // ---- K: sum_i q_i c_i
+    __device__ static __forceinline__ void leave(float (&acc)[kHeadDim]) {
+#pragma unroll
+        for (int i = 0; i < kHeadDim; ++i) acc[i] *= pow2f(49 - field_pos<BITS>(i % EPW));
+    }
+    // one 32-token tile whose record starts at `rec` (shared memory)
+    __device__ static __forceinline__ void tile(const uint8_t* rec, bool valid, int lane, const float (&qk)[kHeadDim],
+                                                float sumq, Softmax& st, float (&acc)[kHeadDim]) {
         float d[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < W; ++j) {
-            const uint4 w4 = __ldg(reinterpret_cast<const uint4*>(rec + j * 512) + lane);
+            const uint4 w4 = reinterpret_cast<const uint4*>(rec + j * 512)[lane];
             const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi) {
@@ -124,22 +197,21 @@ __device__ __forceinline__ void walk_quantized(const uint8_t* __restrict__ base,
                     d[wi] = fmaf(field_as_float<BITS>(w[wi], hi8, e), qk[j * EPC + wi * EPW + e], d[wi]);
             }
         }
-        const uint32_t kmeta = __ldg(reinterpret_cast<const uint32_t*>(rec + 2 * W * 512) + lane);
-        const uint32_t vmeta = __ldg(reinterpret_cast<const uint32_t*>(rec + 2 * W * 512 + 128) + lane);
+        const uint32_t kmeta = reinterpret_cast<const uint32_t*>(rec + 2 * W * 512)[lane];
+        const uint32_t vmeta = reinterpret_cast<const uint32_t*>(rec + 2 * W * 512 + 128)[lane];
         const float sk = __half2float(__ushort_as_half((unsigned short)(kmeta & 0xffffu)));
         const float zk = __half2float(__ushort_as_half((unsigned short)(kmeta >> 16)));
         const float dot = (d[0] + d[1]) + (d[2] + d[3]);
         float y = fmaf(sk * pow2f(49), dot, zk * sumq) * (0.125f * kLog2e);
         y = valid ? y : -INFINITY;
         const float p = softmax_step(st, acc, y);
-        // ---- V: acc_j += (p s_v) c_j, and sum p z_v on the side
         const float sv = __half2float(__ushort_as_half((unsigned short)(vmeta & 0xffffu)));
         const float zv = __half2float(__ushort_as_half((unsigned short)(vmeta >> 16)));
         const float wv = (p * sv) * pow2f(100);
         st.bsum = fmaf(p, zv, st.bsum);
 #pragma unroll
         for (int j = 0; j < W; ++j) {
-            const uint4 w4 = __ldg(reinterpret_cast<const uint4*>(rec + W * 512 + j * 512) + lane);
+            const uint4 w4 = reinterpret_cast<const uint4*>(rec + W * 512 + j * 512)[lane];
             const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi) {
@@ -152,27 +224,28 @@ __device__ __forceinline__ void walk_quantized(const uint8_t* __restrict__ base,
             }
         }
     }
-#pragma unroll
-    for (int i = 0; i < kHeadDim; ++i) acc[i] *= pow2f(49 - field_pos<BITS>(i % EPW));   // back to plain values
-}
+};
 
-// The fp16 pool: rows are stored unchanged.
-__device__ __forceinline__ void walk_fp16(const uint8_t* __restrict__ base, int first, int hi, uint32_t cnt, int lane,
-                                          const float* q_s, Softmax& st, float (&acc)[kHeadDim]) {
-    constexpr int W = pool_chunks(3), REC = pool_rec_bytes(3);
-    for (int t = first; t < hi; t += kDecodeWarps) {
-        const uint8_t* rec = base + (size_t)t * REC;
-        const bool valid = (uint32_t)(t * kTileTokens + lane) < cnt;
+// The fp16 pool: rows are stored unchanged; qk holds the plain query.
+struct Fp16Rows {
+    static constexpr int W = pool_chunks(3), REC = pool_rec_bytes(3);
+    __device__ static __forceinline__ void enter(const float* q_s, float (&qk)[kHeadDim], float (&)[kHeadDim]) {
+#pragma unroll
+        for (int i = 0; i < kHeadDim; ++i) qk[i] = q_s[i];
+    }
+    __device__ static __forceinline__ void leave(float (&)[kHeadDim]) {}
+    __device__ static __forceinline__ void tile(const uint8_t* rec, bool valid, int lane, const float (&qk)[kHeadDim],
+                                                float, Softmax& st, float (&acc)[kHeadDim]) {
         float d[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < W; ++j) {
-            const uint4 w4 = __ldg(reinterpret_cast<const uint4*>(rec + j * 512) + lane);
+            const uint4 w4 = reinterpret_cast<const uint4*>(rec + j * 512)[lane];
             const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi) {
                 const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[wi]));
-                d[wi] = fmaf(f.x, q_s[j * 8 + wi * 2], d[wi]);
-                d[wi] = fmaf(f.y, q_s[j * 8 + wi * 2 + 1], d[wi]);
+                d[wi] = fmaf(f.x, qk[j * 8 + wi * 2], d[wi]);
+                d[wi] = fmaf(f.y, qk[j * 8 + wi * 2 + 1], d[wi]);
             }
         }
         float y = ((d[0] + d[1]) + (d[2] + d[3])) * (0.125f * kLog2e);
@@ -180,7 +253,7 @@ __device__ __forceinline__ void walk_fp16(const uint8_t* __restrict__ base, int 
         const float p = softmax_step(st, acc, y);
 #pragma unroll
         for (int j = 0; j < W; ++j) {
-            uint4 w4 = __ldg(reinterpret_cast<const uint4*>(rec + W * 512 + j * 512) + lane);
+            uint4 w4 = reinterpret_cast<const uint4*>(rec + W * 512 + j * 512)[lane];
             if (!valid) w4 = make_uint4(0, 0, 0, 0);               // stale bytes may hold anything
             const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
@@ -191,11 +264,31 @@ __device__ __forceinline__ void walk_fp16(const uint8_t* __restrict__ base, int 
             }
         }
     }
+};
+
+// ---------------------------------------------------------------- the split kernel
+
+// The part of the sequence this CTA owns, as a list of chunks: chunk g in [pre[c], pre[c+1])
+// belongs to class c and covers tiles [lo[c] + (g-pre[c])*TPS, ...) of that class's pool.
+struct ChunkMap {
+    int lo[kNumPools], hi[kNumPools], pre[kNumPools + 1];
+    uint32_t cnt[kNumPools];
+};
+
+__device__ __forceinline__ void chunk_at(const ChunkMap& m, int g, int& c, int& tile0, int& ntiles) {
+    c = (g >= m.pre[1]) + (g >= m.pre[2]) + (g >= m.pre[3]);
+    const int tps = c == 0 ? tiles_per_stage(0) : c == 1 ? tiles_per_stage(1) : c == 2 ? tiles_per_stage(2)
+                                                                                      : tiles_per_stage(3);
+    tile0 = m.lo[c] + (g - m.pre[c]) * tps;
+    ntiles = min(tps, m.hi[c] - tile0);
 }
 
-// grid = (splits, q_heads, batch), block = 128.
-__global__ void __launch_bounds__(kDecodeThreads)
+// grid = (splits, q_heads, batch), block = kDecodeThreads, dynamic smem = kDecodeSmemBytes.
+__global__ void __launch_bounds__(kDecodeThreads, KVQ_DECODE_MIN_CTAS)
 k_decode_split(DecodeParams P) {
+    extern __shared__ __align__(128) uint8_t ring[];   // [warps][stages][kStageBytes]
+    __shared__ uint64_t bars[kDecodeWarps][kStages];
+    __shared__ ChunkMap map;
     __shared__ float q_s[kHeadDim];
     __shared__ float red_o[kDecodeWarps][kHeadDim];
     __shared__ float2 red_ml[kDecodeWarps];
@@ -205,32 +298,103 @@ k_decode_split(DecodeParams P) {
 
     if (threadIdx.x < kHeadDim)
         q_s[threadIdx.x] = __half2float(P.Q[((size_t)b * P.store.q_heads + qh) * kHeadDim + threadIdx.x]);
+    if (threadIdx.x == 0) {
+        const uint32_t* cnt = P.counts + (size_t)b * 4;
+        int pre = 0;
+        for (int c = 0; c < kNumPools; ++c) {
+            const uint32_t n = cnt[c];
+            const int ntiles = (int)((n + kTileTokens - 1) / kTileTokens);
+            map.cnt[c] = n;
+            map.lo[c] = (int)((long long)ntiles * split / P.splits);
+            map.hi[c] = (int)((long long)ntiles * (split + 1) / P.splits);
+            map.pre[c] = pre;
+            pre += (map.hi[c] - map.lo[c] + tiles_per_stage(c) - 1) / tiles_per_stage(c);
+        }
+        map.pre[kNumPools] = pre;
+        for (int w = 0; w < kDecodeWarps; ++w)
+            for (int s = 0; s < kStages; ++s) mbar_init(&bars[w][s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     __syncthreads();
     float sumq = 0.f;
 #pragma unroll
     for (int i = 0; i < kHeadDim; ++i) sumq += q_s[i];
+
+    const int total = map.pre[kNumPools];
+    const int n_mine = total > warp ? (total - warp + kDecodeWarps - 1) / kDecodeWarps : 0;   // chunks of this warp
+    uint8_t* my_ring = ring + (size_t)warp * kStages * kStageBytes;
+
+    // lane 0 starts the copy of this warp's i-th chunk into ring slot `slot`
+    auto issue = [&](int i, int slot) {
+        if (lane == 0) {
+            int c, tile0, ntiles;
+            chunk_at(map, warp + i * kDecodeWarps, c, tile0, ntiles);
+            const uint32_t bytes = (uint32_t)ntiles * (uint32_t)pool_rec_bytes(c);
+            const uint8_t* src = P.store.pool[c] + tile_offset(P.store, c, P.layer, b, kvh, tile0);
+            mbar_arrive_expect_tx(&bars[warp][slot], bytes);
+            bulk_load(my_ring + (size_t)slot * kStageBytes, src, bytes, &bars[warp][slot]);
+        }
+    };
+    int issued = 0;
+    for (; issued < kStages && issued < n_mine; ++issued) issue(issued, issued);
 
     Softmax st = {kNegBig, 0.f, 0.f};
     float acc[kHeadDim];
 #pragma unroll
     for (int i = 0; i < kHeadDim; ++i) acc[i] = 0.f;
 
-    const uint32_t* cnt = P.counts + (size_t)b * 4;
-    int rr = 0;                                        // tiles handed out so far (mod warps): round robin
-#pragma unroll
-    for (int c = 0; c < kNumPools; ++c) {
-        const uint32_t n = cnt[c];
-        const int ntiles = (int)((n + kTileTokens - 1) / kTileTokens);
-        const int lo = (int)((long long)ntiles * split / P.splits);
-        const int hi = (int)((long long)ntiles * (split + 1) / P.splits);
-        const int first = lo + ((warp - rr) & (kDecodeWarps - 1));
-        rr = (rr + (hi - lo)) & (kDecodeWarps - 1);
-        if (first >= hi) continue;                     // warp-uniform
-        const uint8_t* base = P.store.pool[c] + tile_offset(P.store, c, P.layer, b, kvh, 0);
-        if (c == 0) walk_quantized<0>(base, first, hi, n, lane, q_s, sumq, st, acc);
-        else if (c == 1) walk_quantized<1>(base, first, hi, n, lane, q_s, sumq, st, acc);
-        else if (c == 2) walk_quantized<2>(base, first, hi, n, lane, q_s, sumq, st, acc);
-        else walk_fp16(base, first, hi, n, lane, q_s, st, acc);
+    int ic = 0, slot = 0;                              // next chunk to consume, its ring slot
+    uint32_t parity = 0;                               // phase parity of `slot`
+    bool failed = false;
+
+    auto walk = [&](auto cls_tag, auto consumer) {
+        constexpr int CLS = decltype(cls_tag)::value;
+        using C = decltype(consumer);
+        const int i_end = (map.pre[CLS + 1] - warp + kDecodeWarps - 1) / kDecodeWarps;      // my chunks below pre[CLS+1]
+        if (ic >= i_end || failed) return;
+        float qk[kHeadDim];
+        C::enter(q_s, qk, acc);
+        for (; ic < i_end; ++ic) {
+            if (!mbar_wait(&bars[warp][slot], parity)) {
+                failed = true;
+                break;
+            }
+            const int g = warp + ic * kDecodeWarps;
+            const int tile0 = map.lo[CLS] + (g - map.pre[CLS]) * tiles_per_stage(CLS);
+            const int ntiles = min(tiles_per_stage(CLS), map.hi[CLS] - tile0);
+            const uint8_t* buf = my_ring + (size_t)slot * kStageBytes;
+            for (int t = 0; t < ntiles; ++t) {
+                const bool valid = (uint32_t)((tile0 + t) * kTileTokens + lane) < map.cnt[CLS];
+                C::tile(buf + (size_t)t * C::REC, valid, lane, qk, sumq, st, acc);
+            }
+            __syncwarp();                              // every lane is done with the slot before it is refilled
+            if (issued < n_mine) {
+                issue(issued, slot);
+                ++issued;
+            }
+            if (++slot == kStages) {
+                slot = 0;
+                parity ^= 1u;
+            }
+        }
+        C::leave(acc);
+    };
+    walk(std::integral_constant<int, 0>{}, Quantized<0>{});
+    walk(std::integral_constant<int, 1>{}, Quantized<1>{});
+    walk(std::integral_constant<int, 2>{}, Quantized<2>{});
+    walk(std::integral_constant<int, 3>{}, Fp16Rows{});
+
+    if (failed) {
+        // Copies that were started but not consumed may still land in this CTA's shared memory:
+        // give each a bounded wait before the CTA can retire, then report.
+        for (int i = ic + 1; i < issued; ++i) {
+            if (++slot == kStages) {
+                slot = 0;
+                parity ^= 1u;
+            }
+            mbar_wait(&bars[warp][slot], parity);
+        }
+        if (lane == 0) atomicOr(P.store.flags, kFlagWaitTimeout);
     }
 
     // ---- reduce the per-lane partial sums: after five halving steps lane L holds elements 2L, 2L+1
@@ -284,7 +448,7 @@ k_decode_split(DecodeParams P) {
         float L = 0.f, o = 0.f;
 #pragma unroll
         for (int w = 0; w < kDecodeWarps; ++w) {
-            const float f = exp2f(red_ml[w].x - M);
+            const float f = fast_exp2(red_ml[w].x - M);
             L = fmaf(red_ml[w].y, f, L);
             o = fmaf(red_o[w][threadIdx.x], f, o);
         }
@@ -304,7 +468,7 @@ k_decode_merge(DecodeParams P) {
     float L = 0.f, o = 0.f;
     for (int s = 0; s < P.splits; ++s) {
         const float2 ml = P.part_ml[unit0 + s];
-        const float f = exp2f(ml.x - M);
+        const float f = fast_exp2(ml.x - M);
         L = fmaf(ml.y, f, L);
         o = fmaf(P.part_o[(unit0 + s) * kHeadDim + threadIdx.x], f, o);
     }

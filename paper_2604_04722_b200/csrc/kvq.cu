@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <type_traits>
 #include <vector>
 
 #include "kvq_common.cuh"
@@ -272,6 +273,8 @@ int kvq_create(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_di
         ok = ok && cudaFuncSetAttribute(k_select_bits, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(k_classify<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(k_quant_pack<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(k_decode_split, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)kDecodeSmemBytes) == cudaSuccess;
         ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     }
     if (!ok) {
@@ -353,7 +356,7 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
     const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
     cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 3] : nullptr;
     if (rec) cudaEventRecord(ev[0], st);
-    k_decode_split<<<dim3(p.splits, c->q_heads, c->batch), kDecodeThreads, 0, st>>>(p);
+    k_decode_split<<<dim3(p.splits, c->q_heads, c->batch), kDecodeThreads, kDecodeSmemBytes, st>>>(p);
     if (rec) cudaEventRecord(ev[1], st);
     k_decode_merge<<<c->batch * c->q_heads, kHeadDim, 0, st>>>(p);
     if (rec) {
