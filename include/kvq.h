@@ -55,6 +55,7 @@ extern "C" {
 #define KVQ_ERR_DEVICE_FLAG   -6   /* a kernel recorded a problem (e.g. a bit-width not in
                                       {2,4,8,16}); see kvq_device_status                     */
 #define KVQ_ERR_NOMEM         -7   /* host or device allocation failed                      */
+#define KVQ_ERR_TOO_LARGE     -8   /* problem exceeds the fixed scratch of kvq_decode_attn_static */
 
 typedef struct kvq_ctx kvq_ctx;    /* opaque; owned by the library */
 
@@ -125,6 +126,38 @@ int kvq_append_fused(kvq_ctx* ctx, int layer, const void* K, const void* V,
  * KVQ_ERR_EMPTY if the layer holds no token.
  */
 int kvq_decode_attn(kvq_ctx* ctx, int layer, const void* Q, void* O, void* stream);
+
+/*
+ * kvq_decode_attn without any buffer that had to be allocated for it.  (No counterpart in
+ * the paper: this is a packaging variant of the call above, same arithmetic, same result.)
+ *
+ * Who it is for: code that must not touch the CUDA allocator when it runs -- a serving loop
+ * under a "no allocation after start-up" rule, a plug-in inside a process whose device
+ * memory is entirely owned by another allocator, a caller that cannot tolerate the implicit
+ * device synchronisation of cudaMalloc/cudaFree.  Such a caller cannot ask a library to
+ * reserve per-call or per-handle scratch on its behalf.  Here the split-attention partials
+ * (the only scratch the decode step needs) live in a fixed array that is part of the
+ * library image: KVQ_STATIC_MAX_PARTIALS records of 66 floats, about 2.1 MB, which every
+ * GPU that loads the library holds until the process exits.  The call performs no
+ * cudaMalloc, no cudaFree and calls no allocating routine; the handle's store is read as
+ * input, Q is read and O is written exactly as in kvq_decode_attn, and none of the
+ * handle's own scratch is used.
+ *
+ * Limit: batch * q_heads * splits <= KVQ_STATIC_MAX_PARTIALS (splits is what
+ * kvq_set_splits fixed, or the library's choice for the cached length); otherwise
+ * KVQ_ERR_TOO_LARGE is returned and nothing is queued.
+ *
+ * Set-up: the first call on each device looks up the device address of the array (once
+ * per device, with that device current).  Make that first call outside any stream capture.
+ *
+ * Sharing: every call on a device uses the same array, whatever the handle or stream.
+ * Two calls whose kernels overlap on the GPU (different streams, or different threads)
+ * race on it; serialise them.  The array keeps the previous call's partials; nothing in it
+ * has to start at zero, because every record the merge reads is written first by the same
+ * call.
+ */
+#define KVQ_STATIC_MAX_PARTIALS 8192
+int kvq_decode_attn_static(kvq_ctx* ctx, int layer, const void* Q, void* O, void* stream);
 
 /*
  * One decode step from HOST buffers, copies included: controller decision for

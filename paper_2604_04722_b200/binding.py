@@ -23,6 +23,8 @@ KVQ_ERR_CUDA = -4
 KVQ_ERR_EMPTY = -5
 KVQ_ERR_DEVICE_FLAG = -6
 KVQ_ERR_NOMEM = -7
+KVQ_ERR_TOO_LARGE = -8
+KVQ_STATIC_MAX_PARTIALS = 8192
 KVQ_EXPORT_ROW_BYTES = 128
 
 _vp, _i, _u64p = C.c_void_p, C.c_int, C.POINTER(C.c_uint64)
@@ -36,6 +38,7 @@ SIGNATURES = {
     "kvq_append": (_i, [_vp, _i, _vp, _vp, _vp, _i, _vp]),
     "kvq_append_fused": (_i, [_vp, _i, _vp, _vp, _vp, _i, _vp, _vp]),
     "kvq_decode_attn": (_i, [_vp, _i, _vp, _vp, _vp]),
+    "kvq_decode_attn_static": (_i, [_vp, _i, _vp, _vp, _vp]),
     "kvq_decode_step_host": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvq_reset": (_i, [_vp, _vp]),
     "kvq_seq_len": (_i, [_vp, _i, C.POINTER(_i)]),
@@ -136,6 +139,11 @@ def kvq_append_fused(ctx: int, layer: int, K, V, feats, n_new: int, bits_out=Non
 
 def kvq_decode_attn(ctx: int, layer: int, Q, O, stream=None) -> None:
     check(lib().kvq_decode_attn(ctx, layer, _ptr(Q), _ptr(O), _stream(stream)), "kvq_decode_attn")
+
+
+def kvq_decode_attn_static(ctx: int, layer: int, Q, O, stream=None) -> None:
+    """kvq_decode_attn with the split partials in the library's fixed device array: allocates nothing."""
+    check(lib().kvq_decode_attn_static(ctx, layer, _ptr(Q), _ptr(O), _stream(stream)), "kvq_decode_attn_static")
 
 
 def kvq_decode_step_host(ctx: int, layer: int, feats, K, V, Q, O, bits_out=None, stream=None) -> None:

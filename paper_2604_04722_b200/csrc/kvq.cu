@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <type_traits>
 #include <vector>
@@ -368,6 +369,52 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
     return KVQ_OK;
 }
 
+// ---- decode attention with its partials in the library image (no allocation at all)
+//
+// The array below is a device symbol.  Its NAME in host code is only a host-side stand-in, not
+// a device address; the address is fetched with cudaGetSymbolAddress once per device (that
+// device current) and passed to the kernels like any other pointer.
+#define KVQ_STATIC_MAX_DEVICES 64
+static __device__ __align__(256) float g_static_partials[(size_t)KVQ_STATIC_MAX_PARTIALS * (kHeadDim + 2)];
+static float* g_static_partials_addr[KVQ_STATIC_MAX_DEVICES];   // per device, nullptr until looked up
+static std::mutex g_static_partials_lock;
+
+int kvq_decode_attn_static(kvq_ctx* c, int layer, const void* Q, void* O, void* stream) {
+    if (check_layer(c, layer) != KVQ_OK || !Q || !O) return KVQ_ERR_ARG;
+    if (c->len[layer] == 0) return KVQ_ERR_EMPTY;
+    if (c->device < 0 || c->device >= KVQ_STATIC_MAX_DEVICES) return KVQ_ERR_ARG;
+    const int splits = choose_splits(c, c->len[layer]);
+    const size_t records = (size_t)c->batch * c->q_heads * splits;
+    if (records > (size_t)KVQ_STATIC_MAX_PARTIALS) return KVQ_ERR_TOO_LARGE;
+    DeviceGuard guard(c->device);
+    float* base = nullptr;
+    {
+        std::lock_guard<std::mutex> hold(g_static_partials_lock);
+        if (!g_static_partials_addr[c->device]) {
+            void* p = nullptr;
+            KVQ_CUDA(c, cudaGetSymbolAddress(&p, g_static_partials));
+            g_static_partials_addr[c->device] = static_cast<float*>(p);
+        }
+        base = g_static_partials_addr[c->device];
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DecodeParams p{};
+    p.store = c->store;
+    p.counts = counts_of(c, c->cur[layer], layer);
+    p.Q = static_cast<const __half*>(Q);
+    p.O = static_cast<__half*>(O);
+    p.part_o = base;                                                        // [records][64]
+    p.part_ml = reinterpret_cast<float2*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * kHeadDim);   // [records]
+    p.layer = layer;
+    p.splits = splits;
+    p.group = c->q_heads / c->kv_heads;
+    k_decode_split<<<dim3(p.splits, c->q_heads, c->batch), kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    k_decode_merge<<<c->batch * c->q_heads, kHeadDim, 0, st>>>(p);
+    c->launches += 2;
+    KVQ_CUDA(c, cudaGetLastError());
+    return KVQ_OK;
+}
+
 int kvq_decode_step_host(kvq_ctx* c, int layer, const float* feats, const void* K, const void* V, const void* Q,
                          void* O, uint8_t* bits_out_opt, void* stream) {
     if (check_layer(c, layer) != KVQ_OK || !feats || !K || !V || !Q || !O) return KVQ_ERR_ARG;
@@ -542,6 +589,7 @@ const char* kvq_strerror(int code) {
     case KVQ_ERR_EMPTY: return "layer holds no token";
     case KVQ_ERR_DEVICE_FLAG: return "a kernel recorded a problem";
     case KVQ_ERR_NOMEM: return "out of memory";
+    case KVQ_ERR_TOO_LARGE: return "batch * q_heads * splits exceeds the static scratch of kvq_decode_attn_static";
     default: return "unknown error";
     }
 }
