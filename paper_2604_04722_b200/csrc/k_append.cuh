@@ -131,26 +131,28 @@ __device__ __forceinline__ void quantize_store_row(const StoreView& s, uint4 raw
     const uint32_t lo_next = __shfl_down_sync(0xffffffffu, lo, 1);
     if (!valid) return;
 
-    const int W = pool_chunks(cls);
-    uint8_t* rec = s.pool[cls] + tile_offset(s, cls, layer, b, h, (int)(slot >> 5));
-    uint8_t* row = rec + (size_t)tensor * W * 512 + (slot & 31) * 16;
+    const int t = (int)(slot & (kTileTokens - 1));
+    uint8_t* rec = s.pool[cls] + tile_offset(s, cls, layer, b, h, (int)(slot / kTileTokens));
+    uint8_t* codes = rec + (size_t)tensor * pool_codes_bytes(cls);
+    const int half = sub >> 2, q = sub & 3;            // this lane's 8 elements: quarter q of half-row `half`
     switch (cls) {
-    case 0:                                            // 16 bits per lane -> 4-byte words from even lanes
-        if ((sub & 1) == 0) *reinterpret_cast<uint32_t*>(row + (sub >> 1) * 4) = (lo & 0xffffu) | (lo_next << 16);
+    case 0:                                            // 2 bytes per lane -> 4-byte words from even lanes
+        if ((sub & 1) == 0)
+            *reinterpret_cast<uint32_t*>(codes + unit_offset(0, half, 0, t) + (q >> 1) * 4) = (lo & 0xffffu) | (lo_next << 16);
         break;
-    case 1:                                            // 4 bytes per lane: row bytes [4*sub, +4)
-        *reinterpret_cast<uint32_t*>(row + (sub >> 2) * 512 + (sub & 3) * 4) = lo;
+    case 1:                                            // 4 bytes per lane
+        *reinterpret_cast<uint32_t*>(codes + unit_offset(1, half, 0, t) + q * 4) = lo;
         break;
-    case 2:                                            // 8 bytes per lane: row bytes [8*sub, +8)
-        *reinterpret_cast<uint2*>(row + (sub >> 1) * 512 + (sub & 1) * 8) = make_uint2(lo, hi);
+    case 2:                                            // 8 bytes per lane
+        *reinterpret_cast<uint2*>(codes + unit_offset(2, half, q >> 1, t) + (q & 1) * 8) = make_uint2(lo, hi);
         break;
-    default:                                           // fp16: the lane's 16 input bytes are chunk `sub`
-        *reinterpret_cast<uint4*>(row + sub * 512) = raw;
+    default:                                           // fp16: the lane's 16 input bytes are one unit
+        *reinterpret_cast<uint4*>(codes + unit_offset(3, half, q, t)) = raw;
         break;
     }
     if (cls < 3 && sub == 0) {
         uint32_t meta = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(__float2half_rn(mn)) << 16);
-        *reinterpret_cast<uint32_t*>(rec + 2 * W * 512 + tensor * 128 + (slot & 31) * 4) = meta;
+        *reinterpret_cast<uint32_t*>(rec + meta_offset(cls, tensor, t)) = meta;
     }
 }
 

@@ -16,10 +16,13 @@
 // loop.  Every mbarrier wait is bounded: on expiry the warp records
 // KVQ_FLAG_WAIT_TIMEOUT and leaves the loop.
 //
-// Work layout inside a warp: one lane per token (a 32-token tile is read with
-// conflict-free 16-byte shared loads), so the q.k dot product needs no
-// shuffles and the output accumulators are per-lane partial sums reduced once
-// at the end.
+// Work layout inside a warp: two lanes per token.  Lane l handles half l/16
+// (elements 32*(l/16) .. +32) of slot l%16 of a 16-token tile, so it keeps 32
+// pre-scaled query values and 32 output accumulators in registers (about half
+// the registers of a lane-per-token mapping: 16 warps stay resident per SM and
+// hide the latency of the dependent FMA chains).  The two half dot products
+// meet through one xor-16 shuffle; the output accumulators are per-lane
+// partial sums reduced once at the end.
 //
 // Dequantization is hoisted out of the inner loops:
 //   q.khat = s_k * sum_i q_i c_i + z_k * sum_i q_i
@@ -41,21 +44,28 @@
 #define KVQ_DECODE_WARPS 4
 #endif
 #ifndef KVQ_DECODE_MIN_CTAS
-#define KVQ_DECODE_MIN_CTAS 2
+#define KVQ_DECODE_MIN_CTAS 4
+#endif
+#ifndef KVQ_DECODE_STAGE_BYTES
+#define KVQ_DECODE_STAGE_BYTES 4352
 #endif
 
 namespace kvq {
 
 constexpr int kDecodeWarps = KVQ_DECODE_WARPS;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
+constexpr int kDecodeCtasPerSm = KVQ_DECODE_MIN_CTAS;
 constexpr int kStages = KVQ_DECODE_STAGES;
-constexpr int kStageBytes = 8704;                // two 8-bit tiles; 6 / 3 / 2 / 1 tiles of the four classes
+constexpr int kStageBytes = KVQ_DECODE_STAGE_BYTES;   // two 8-bit tiles; 6 / 3 / 2 / 1 tiles of the four classes
+constexpr int kHalfDim = kHeadDim / 2;           // elements per lane
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLogitScale = 0.125f * kLog2e;   // 1/sqrt(64), in log2 units
 constexpr float kRescaleSlack = 8.0f;            // the running maximum may lag by 2^8 before a rescale
 constexpr float kNegBig = -1.0e30f;
 constexpr uint32_t kWaitLimit = 1u << 20;        // mbarrier polls before a wait is abandoned
 constexpr uint32_t kFlagWaitTimeout = 2u;
 
+static_assert(kStageBytes % 16 == 0 && kStageBytes >= pool_rec_bytes(3), "a stage must hold one fp16 tile");
 __host__ __device__ constexpr int tiles_per_stage(int c) { return kStageBytes / pool_rec_bytes(c); }
 constexpr size_t kDecodeSmemBytes = (size_t)kDecodeWarps * kStages * kStageBytes;
 
@@ -145,82 +155,94 @@ struct Softmax {
     float m, l, bsum;              // running max (log2 units), sum of p, sum of p * zero-point
 };
 
-// Fold a tile's logits into the running state and return this lane's p.
-__device__ __forceinline__ float softmax_step(Softmax& st, float (&acc)[kHeadDim], float y) {
-    const float tmax = warp_max(y);
-    if (tmax > st.m + kRescaleSlack) {                 // warp-uniform
+// Fold a tile's logits into the running state and return this lane's p.  The running maximum
+// is only raised when some logit exceeds it by more than kRescaleSlack (one vote per tile).
+__device__ __forceinline__ float softmax_step(Softmax& st, float (&acc)[kHalfDim], float y) {
+    if (__any_sync(0xffffffffu, y > st.m + kRescaleSlack)) {       // warp-uniform
+        const float tmax = warp_max(y);
         const float f = fast_exp2(st.m - tmax);
         st.m = tmax;
         st.l *= f;
         st.bsum *= f;
 #pragma unroll
-        for (int j = 0; j < kHeadDim; ++j) acc[j] *= f;
+        for (int j = 0; j < kHalfDim; ++j) acc[j] *= f;
     }
     const float p = fast_exp2(y - st.m);
     st.l += p;
     return p;
 }
 
+__device__ __forceinline__ float2 meta_to_float2(uint32_t m) {     // {scale, zero-point}
+    return __half22float2(*reinterpret_cast<const __half2*>(&m));
+}
+
 // ---------------------------------------------------------------- tile consumers (data in shared memory)
+// Every consumer sees one 16-token tile record `rec`; the lane handles half `half` of slot `t`.
 
 template <int CLS>
 struct Quantized {
-    static constexpr int BITS = pool_bits(CLS), W = pool_chunks(CLS), REC = pool_rec_bytes(CLS);
+    static constexpr int BITS = pool_bits(CLS), REC = pool_rec_bytes(CLS);
     static constexpr int EPW = 32 / BITS;              // elements per 32-bit word
-    static constexpr int EPC = 4 * EPW;                // elements per 16-byte chunk
+    static constexpr int WORDS = pool_half_bytes(CLS) / 4;         // words per half-row: 2, 4, 8
+    static constexpr int UNITS = pool_units(CLS), UWORDS = pool_unit_bytes(CLS) / 4;
 
     // pre-scaled query and accumulator exponent domain of this class
-    __device__ static __forceinline__ void enter(const float* q_s, float (&qk)[kHeadDim], float (&acc)[kHeadDim]) {
+    __device__ static __forceinline__ void enter(const float* q_half, float (&qk)[kHalfDim], float (&acc)[kHalfDim]) {
 #pragma unroll
-        for (int i = 0; i < kHeadDim; ++i) {
-            qk[i] = q_s[i] * pow2f(100 - field_pos<BITS>(i % EPW));
+        for (int i = 0; i < kHalfDim; ++i) {
+            qk[i] = q_half[i] * pow2f(100 - field_pos<BITS>(i % EPW));
             acc[i] *= pow2f(field_pos<BITS>(i % EPW) - 49);
         }
     }
-    __device__ static __forceinline__ void leave(float (&acc)[kHeadDim]) {
+    __device__ static __forceinline__ void leave(float (&acc)[kHalfDim]) {
 #pragma unroll
-        for (int i = 0; i < kHeadDim; ++i) acc[i] *= pow2f(49 - field_pos<BITS>(i % EPW));
+        for (int i = 0; i < kHalfDim; ++i) acc[i] *= pow2f(49 - field_pos<BITS>(i % EPW));
     }
-    // one 32-token tile whose record starts at `rec` (shared memory)
-    __device__ static __forceinline__ void tile(const uint8_t* rec, bool valid, int lane, const float (&qk)[kHeadDim],
-                                                float sumq, Softmax& st, float (&acc)[kHeadDim]) {
-        float d[4] = {0.f, 0.f, 0.f, 0.f};
+    __device__ static __forceinline__ void load_half_row(const uint8_t* codes, int half, int t, uint32_t (&w)[WORDS]) {
 #pragma unroll
-        for (int j = 0; j < W; ++j) {
-            const uint4 w4 = reinterpret_cast<const uint4*>(rec + j * 512)[lane];
-            const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
-#pragma unroll
-            for (int wi = 0; wi < 4; ++wi) {
-                const uint32_t hi8 = w[wi] >> 8;
-#pragma unroll
-                for (int e = 0; e < EPW; ++e)
-                    d[wi] = fmaf(field_as_float<BITS>(w[wi], hi8, e), qk[j * EPC + wi * EPW + e], d[wi]);
+        for (int u = 0; u < UNITS; ++u) {
+            if (UWORDS == 2) {
+                const uint2 v = *reinterpret_cast<const uint2*>(codes + unit_offset(CLS, half, u, t));
+                w[0] = v.x; w[1] = v.y;
+            } else {
+                const uint4 v = *reinterpret_cast<const uint4*>(codes + unit_offset(CLS, half, u, t));
+                w[4 * u] = v.x; w[4 * u + 1] = v.y; w[4 * u + 2] = v.z; w[4 * u + 3] = v.w;
             }
         }
-        const uint32_t kmeta = reinterpret_cast<const uint32_t*>(rec + 2 * W * 512)[lane];
-        const uint32_t vmeta = reinterpret_cast<const uint32_t*>(rec + 2 * W * 512 + 128)[lane];
-        const float sk = __half2float(__ushort_as_half((unsigned short)(kmeta & 0xffffu)));
-        const float zk = __half2float(__ushort_as_half((unsigned short)(kmeta >> 16)));
-        const float dot = (d[0] + d[1]) + (d[2] + d[3]);
-        float y = fmaf(sk * pow2f(49), dot, zk * sumq) * (0.125f * kLog2e);
+    }
+    __device__ static __forceinline__ void tile(const uint8_t* rec, bool valid, int half, int t,
+                                                const float (&qk)[kHalfDim], float sumq_scaled, Softmax& st,
+                                                float (&acc)[kHalfDim]) {
+        uint32_t w[WORDS];
+        load_half_row(rec, half, t, w);
+        const float2 km = meta_to_float2(*reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 0, t)));
+        float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int wi = 0; wi < WORDS; ++wi) {
+            const uint32_t hi8 = w[wi] >> 8;
+#pragma unroll
+            for (int e = 0; e < EPW; ++e) {
+                const int i = wi * EPW + e;
+                d[i & 3] = fmaf(field_as_float<BITS>(w[wi], hi8, e), qk[i], d[i & 3]);
+            }
+        }
+        float dot = (d[0] + d[1]) + (d[2] + d[3]);
+        dot += __shfl_xor_sync(0xffffffffu, dot, 16);              // the other half of the row
+        float y = fmaf(km.x * (pow2f(49) * kLogitScale), dot, km.y * sumq_scaled);
         y = valid ? y : -INFINITY;
         const float p = softmax_step(st, acc, y);
-        const float sv = __half2float(__ushort_as_half((unsigned short)(vmeta & 0xffffu)));
-        const float zv = __half2float(__ushort_as_half((unsigned short)(vmeta >> 16)));
-        const float wv = (p * sv) * pow2f(100);
-        st.bsum = fmaf(p, zv, st.bsum);
+
+        load_half_row(rec + pool_codes_bytes(CLS), half, t, w);
+        const float2 vm = meta_to_float2(*reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 1, t)));
+        const float wv = (p * vm.x) * pow2f(100);
+        st.bsum = fmaf(p, vm.y, st.bsum);
 #pragma unroll
-        for (int j = 0; j < W; ++j) {
-            const uint4 w4 = reinterpret_cast<const uint4*>(rec + W * 512 + j * 512)[lane];
-            const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+        for (int wi = 0; wi < WORDS; ++wi) {
+            const uint32_t hi8 = w[wi] >> 8;
 #pragma unroll
-            for (int wi = 0; wi < 4; ++wi) {
-                const uint32_t hi8 = w[wi] >> 8;
-#pragma unroll
-                for (int e = 0; e < EPW; ++e) {
-                    const int i = j * EPC + wi * EPW + e;
-                    acc[i] = fmaf(field_as_float<BITS>(w[wi], hi8, e), wv, acc[i]);
-                }
+            for (int e = 0; e < EPW; ++e) {
+                const int i = wi * EPW + e;
+                acc[i] = fmaf(field_as_float<BITS>(w[wi], hi8, e), wv, acc[i]);
             }
         }
     }
@@ -228,39 +250,42 @@ struct Quantized {
 
 // The fp16 pool: rows are stored unchanged; qk holds the plain query.
 struct Fp16Rows {
-    static constexpr int W = pool_chunks(3), REC = pool_rec_bytes(3);
-    __device__ static __forceinline__ void enter(const float* q_s, float (&qk)[kHeadDim], float (&)[kHeadDim]) {
+    static constexpr int REC = pool_rec_bytes(3), UNITS = pool_units(3), WORDS = pool_half_bytes(3) / 4;
+    __device__ static __forceinline__ void enter(const float* q_half, float (&qk)[kHalfDim], float (&)[kHalfDim]) {
 #pragma unroll
-        for (int i = 0; i < kHeadDim; ++i) qk[i] = q_s[i];
+        for (int i = 0; i < kHalfDim; ++i) qk[i] = q_half[i];
     }
-    __device__ static __forceinline__ void leave(float (&)[kHeadDim]) {}
-    __device__ static __forceinline__ void tile(const uint8_t* rec, bool valid, int lane, const float (&qk)[kHeadDim],
-                                                float, Softmax& st, float (&acc)[kHeadDim]) {
+    __device__ static __forceinline__ void leave(float (&)[kHalfDim]) {}
+    __device__ static __forceinline__ void tile(const uint8_t* rec, bool valid, int half, int t,
+                                                const float (&qk)[kHalfDim], float, Softmax& st,
+                                                float (&acc)[kHalfDim]) {
         float d[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int j = 0; j < W; ++j) {
-            const uint4 w4 = reinterpret_cast<const uint4*>(rec + j * 512)[lane];
+        for (int u = 0; u < UNITS; ++u) {
+            const uint4 w4 = *reinterpret_cast<const uint4*>(rec + unit_offset(3, half, u, t));
             const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi) {
                 const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[wi]));
-                d[wi] = fmaf(f.x, qk[j * 8 + wi * 2], d[wi]);
-                d[wi] = fmaf(f.y, qk[j * 8 + wi * 2 + 1], d[wi]);
+                d[wi] = fmaf(f.x, qk[u * 8 + wi * 2], d[wi]);
+                d[wi] = fmaf(f.y, qk[u * 8 + wi * 2 + 1], d[wi]);
             }
         }
-        float y = ((d[0] + d[1]) + (d[2] + d[3])) * (0.125f * kLog2e);
+        float dot = (d[0] + d[1]) + (d[2] + d[3]);
+        dot += __shfl_xor_sync(0xffffffffu, dot, 16);
+        float y = dot * kLogitScale;
         y = valid ? y : -INFINITY;
         const float p = softmax_step(st, acc, y);
 #pragma unroll
-        for (int j = 0; j < W; ++j) {
-            uint4 w4 = reinterpret_cast<const uint4*>(rec + W * 512 + j * 512)[lane];
+        for (int u = 0; u < UNITS; ++u) {
+            uint4 w4 = *reinterpret_cast<const uint4*>(rec + pool_codes_bytes(3) + unit_offset(3, half, u, t));
             if (!valid) w4 = make_uint4(0, 0, 0, 0);               // stale bytes may hold anything
             const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi) {
                 const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[wi]));
-                acc[j * 8 + wi * 2] = fmaf(p, f.x, acc[j * 8 + wi * 2]);
-                acc[j * 8 + wi * 2 + 1] = fmaf(p, f.y, acc[j * 8 + wi * 2 + 1]);
+                acc[u * 8 + wi * 2] = fmaf(p, f.x, acc[u * 8 + wi * 2]);
+                acc[u * 8 + wi * 2 + 1] = fmaf(p, f.y, acc[u * 8 + wi * 2 + 1]);
             }
         }
     }
@@ -295,6 +320,7 @@ k_decode_split(DecodeParams P) {
     const int split = blockIdx.x, qh = blockIdx.y, b = blockIdx.z;
     const int kvh = qh / P.group;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int half = lane >> 4, t = lane & 15;
 
     if (threadIdx.x < kHeadDim)
         q_s[threadIdx.x] = __half2float(P.Q[((size_t)b * P.store.q_heads + qh) * kHeadDim + threadIdx.x]);
@@ -316,9 +342,9 @@ k_decode_split(DecodeParams P) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    float sumq = 0.f;
-#pragma unroll
-    for (int i = 0; i < kHeadDim; ++i) sumq += q_s[i];
+    float sumq = q_s[lane] + q_s[lane + 32];
+    sumq = warp_sum(sumq) * kLogitScale;               // sum_i q_i, in logit units
+    const float* q_half = q_s + half * kHalfDim;
 
     const int total = map.pre[kNumPools];
     const int n_mine = total > warp ? (total - warp + kDecodeWarps - 1) / kDecodeWarps : 0;   // chunks of this warp
@@ -339,9 +365,9 @@ k_decode_split(DecodeParams P) {
     for (; issued < kStages && issued < n_mine; ++issued) issue(issued, issued);
 
     Softmax st = {kNegBig, 0.f, 0.f};
-    float acc[kHeadDim];
+    float acc[kHalfDim];
 #pragma unroll
-    for (int i = 0; i < kHeadDim; ++i) acc[i] = 0.f;
+    for (int i = 0; i < kHalfDim; ++i) acc[i] = 0.f;
 
     int ic = 0, slot = 0;                              // next chunk to consume, its ring slot
     uint32_t parity = 0;                               // phase parity of `slot`
@@ -352,8 +378,8 @@ k_decode_split(DecodeParams P) {
         using C = decltype(consumer);
         const int i_end = (map.pre[CLS + 1] - warp + kDecodeWarps - 1) / kDecodeWarps;      // my chunks below pre[CLS+1]
         if (ic >= i_end || failed) return;
-        float qk[kHeadDim];
-        C::enter(q_s, qk, acc);
+        float qk[kHalfDim];
+        C::enter(q_half, qk, acc);
         for (; ic < i_end; ++ic) {
             if (!mbar_wait(&bars[warp][slot], parity)) {
                 failed = true;
@@ -363,9 +389,9 @@ k_decode_split(DecodeParams P) {
             const int tile0 = map.lo[CLS] + (g - map.pre[CLS]) * tiles_per_stage(CLS);
             const int ntiles = min(tiles_per_stage(CLS), map.hi[CLS] - tile0);
             const uint8_t* buf = my_ring + (size_t)slot * kStageBytes;
-            for (int t = 0; t < ntiles; ++t) {
-                const bool valid = (uint32_t)((tile0 + t) * kTileTokens + lane) < map.cnt[CLS];
-                C::tile(buf + (size_t)t * C::REC, valid, lane, qk, sumq, st, acc);
+            for (int i = 0; i < ntiles; ++i) {
+                const bool valid = (uint32_t)((tile0 + i) * kTileTokens + t) < map.cnt[CLS];
+                C::tile(buf + (size_t)i * C::REC, valid, half, t, qk, sumq, st, acc);
             }
             __syncwarp();                              // every lane is done with the slot before it is refilled
             if (issued < n_mine) {
@@ -397,19 +423,13 @@ k_decode_split(DecodeParams P) {
         if (lane == 0) atomicOr(P.store.flags, kFlagWaitTimeout);
     }
 
-    // ---- reduce the per-lane partial sums: after five halving steps lane L holds elements 2L, 2L+1
-    float r32[32];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        const bool up = lane & 16;
-        const float keep = up ? acc[j + 32] : acc[j], send = up ? acc[j] : acc[j + 32];
-        r32[j] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-    }
+    // ---- reduce the per-lane partial sums over the 16 slots of a half: after four halving steps
+    //      lane L holds elements 2L, 2L+1 of the row
     float r16[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
         const bool up = lane & 8;
-        const float keep = up ? r32[j + 16] : r32[j], send = up ? r32[j] : r32[j + 16];
+        const float keep = up ? acc[j + 16] : acc[j], send = up ? acc[j] : acc[j + 16];
         r16[j] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
     }
     float r8[8];
@@ -433,8 +453,9 @@ k_decode_split(DecodeParams P) {
         const float keep = up ? r4[j + 2] : r4[j], send = up ? r4[j] : r4[j + 2];
         r2[j] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
     }
-    const float l_w = warp_sum(st.l);
-    const float b_w = warp_sum(st.bsum);
+    // both lanes of a token added its p and p * zero-point: halve the warp sums
+    const float l_w = 0.5f * warp_sum(st.l);
+    const float b_w = 0.5f * warp_sum(st.bsum);
     red_o[warp][2 * lane] = r2[0] + b_w;
     red_o[warp][2 * lane + 1] = r2[1] + b_w;
     if (lane == 0) red_ml[warp] = make_float2(st.m, l_w);

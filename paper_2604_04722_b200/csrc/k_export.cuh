@@ -1,6 +1,6 @@
 // Canonical copy of cached tokens, position by position: looks every token up
-// through the per-token index word (pool << 30 | slot) and de-interleaves its
-// rows from the tile records into plain 128-byte rows (packed codes first,
+// through the per-token index word (pool << 30 | slot) and gathers the units of
+// its rows from the tile records into plain 128-byte rows (packed codes first,
 // zero tail) plus {scale, zero-point} pairs.  Used to compare the store with
 // other implementations of the quantizer named in Eq. 24.
 #pragma once
@@ -33,14 +33,24 @@ k_export(ExportParams p) {
         if (p.bits) p.bits[tok] = (uint8_t)pool_bits(cls);
         if (p.pool_slot) p.pool_slot[tok] = word;
     }
-    const int items = s.kv_heads * 2 * 8;              // (head, tensor, 16-byte chunk)
+    const int t = (int)(slot & (kTileTokens - 1)), tile = (int)(slot / kTileTokens);
+    const int items = s.kv_heads * 2 * 8;              // (head, tensor, 16-byte chunk of the canonical row)
     for (int it = threadIdx.x; it < items; it += blockDim.x) {
         const int j = it & 7, tensor = (it >> 3) & 1, h = it >> 4;
         uint4* dst = tensor ? p.v_codes : p.k_codes;
         if (!dst) continue;
-        const uint8_t* rec = s.pool[cls] + tile_offset(s, cls, p.layer, b, h, (int)(slot >> 5));
+        const uint8_t* codes = s.pool[cls] + tile_offset(s, cls, p.layer, b, h, tile) + (size_t)tensor * pool_codes_bytes(cls);
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (j < W) v = *reinterpret_cast<const uint4*>(rec + (size_t)tensor * W * 512 + j * 512 + (slot & 31) * 16);
+        if (j < W) {
+            if (cls == 0) {                            // the 16-byte row is two 8-byte half-rows
+                const uint2 lo = *reinterpret_cast<const uint2*>(codes + unit_offset(0, 0, 0, t));
+                const uint2 hi = *reinterpret_cast<const uint2*>(codes + unit_offset(0, 1, 0, t));
+                v = make_uint4(lo.x, lo.y, hi.x, hi.y);
+            } else {                                   // chunk j = unit j % units of half j / units
+                const int units = pool_units(cls);
+                v = *reinterpret_cast<const uint4*>(codes + unit_offset(cls, j / units, j % units, t));
+            }
+        }
         dst[(tok * s.kv_heads + h) * 8 + j] = v;
     }
     for (int it = threadIdx.x; it < s.kv_heads * 2; it += blockDim.x) {
@@ -49,8 +59,8 @@ k_export(ExportParams p) {
         if (!dst) continue;
         uint32_t m = 0;
         if (cls < 3) {
-            const uint8_t* rec = s.pool[cls] + tile_offset(s, cls, p.layer, b, h, (int)(slot >> 5));
-            m = *reinterpret_cast<const uint32_t*>(rec + 2 * W * 512 + tensor * 128 + (slot & 31) * 4);
+            const uint8_t* rec = s.pool[cls] + tile_offset(s, cls, p.layer, b, h, tile);
+            m = *reinterpret_cast<const uint32_t*>(rec + meta_offset(cls, tensor, t));
         }
         dst[(tok * s.kv_heads + h) * 2 + 0] = (uint16_t)(m & 0xffffu);
         dst[(tok * s.kv_heads + h) * 2 + 1] = (uint16_t)(m >> 16);

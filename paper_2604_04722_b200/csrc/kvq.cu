@@ -168,16 +168,32 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
     return KVQ_OK;
 }
 
+// Number of sequence splits.  Every (sequence, query head) unit is cut into the same number of
+// parts; the grid is units x splits CTAs and kDecodeCtasPerSm CTAs are resident per SM.  Few CTAs:
+// take as many splits as the work allows (a warp should still own a few chunks).  Many CTAs: aim
+// at a handful of full waves and pick the count whose last wave is fullest.
 int choose_splits(kvq_ctx* c, int len) {
     if (c->splits_override > 0) return c->splits_override;
     const int tiles = (len + kTileTokens - 1) / kTileTokens + (kNumPools - 1);
     const int units = c->batch * c->q_heads;
-    int s = (24 * c->sm_count + units - 1) / units;              // ~8 waves of 3 CTAs per SM
-    const int by_work = tiles / (2 * kDecodeWarps);              // at least two tiles per warp
-    if (s > by_work) s = by_work;
-    if (s > kMaxSplits) s = kMaxSplits;
-    if (s < 1) s = 1;
-    return s;
+    const int slots = kDecodeCtasPerSm * c->sm_count;
+    int smax = tiles / (8 * kDecodeWarps);                       // at least eight tiles per warp
+    const int by_waves = (8 * slots + units - 1) / units;        // at most about eight waves
+    if (smax > by_waves) smax = by_waves;
+    if (smax > kMaxSplits) smax = kMaxSplits;
+    if (smax < 1) smax = 1;
+    int best = 1;
+    double best_score = -1.0;
+    for (int s = 1; s <= smax; ++s) {
+        const double fill = (double)units * s / slots;
+        const double waves = fill <= 1.0 ? 1.0 : (double)(long long)(fill + 0.999999);
+        const double score = fill / waves;                       // share of the resident slots kept busy
+        if (score > best_score + 1e-9) {
+            best_score = score;
+            best = s;
+        }
+    }
+    return best;
 }
 
 int export_impl(kvq_ctx* c, int layer, int b0, int nb, int pos0, int n, uint8_t* bits, uint32_t* pool_slot,
