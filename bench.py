@@ -183,9 +183,9 @@ def run_reference(args, wl):
 
 
 def workload_config(wl):
-    return {"workload": "%s stress: 1 SmolLM-1.7B-shaped layer, 32 q / 32 kv heads, head_dim 64, batch 16, "
+    return {"workload": "%s stress: 1 SmolLM-1.7B-shaped layer, 32 q / 32 kv heads, head_dim 64, batch %d, "
                         "context %d, bits iid {2:.50,4:.30,8:.15,16:.05} seed 0; each step appends 1 "
-                        "controller-decided token per sequence and attends" % (wl.name, wl.context),
+                        "controller-decided token per sequence and attends" % (wl.name, wl.batch, wl.context),
             "layers": wl.layers, "batch": wl.batch, "q_heads": wl.q_heads, "kv_heads": wl.kv_heads,
             "head_dim": wl.head_dim, "context": wl.context,
             "l2": "inputs larger than L2 (about 1.25 GB of packed KV is streamed per step; L2 is 126 MB)"}
@@ -408,12 +408,16 @@ def main():
     ap.add_argument("--context", type=int, default=0,
                     help="shorter cached context than the workload's 32768, for profiler captures that must "
                          "stay small; the printed config names it and the line is not a benchmark result")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="fewer sequences than the workload's 16, likewise for profiler captures only")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     wl = synth.CONFIGS["cfg5"]
     if args.context > 0:
-        wl = dataclasses.replace(wl, context=args.context, name="cfg5-context-%d" % args.context)
+        wl = dataclasses.replace(wl, context=args.context, name="%s-context-%d" % (wl.name, args.context))
+    if args.batch > 0:
+        wl = dataclasses.replace(wl, batch=args.batch, name="%s-batch-%d" % (wl.name, args.batch))
     if args.impl == "reference":
         run_reference(args, wl)
     else:

@@ -122,7 +122,8 @@ int kvq_append_fused(kvq_ctx* ctx, int layer, const void* K, const void* V,
  * Decode-step attention (Eq. 5) of one query row per (sequence, query head)
  * over every token cached in `layer`, dequantizing on the fly:
  * O = Softmax(q K^T / 8) V.  Q, O: dev fp16 [batch][q_heads][64].  fp32
- * accumulation, online softmax, split over the sequence and merged.
+ * accumulation, online softmax; the work is split over warps (see kvq_set_splits) whose
+ * partial results a second kernel merges.
  * KVQ_ERR_EMPTY if the layer holds no token.
  */
 int kvq_decode_attn(kvq_ctx* ctx, int layer, const void* Q, void* O, void* stream);
@@ -143,8 +144,9 @@ int kvq_decode_attn(kvq_ctx* ctx, int layer, const void* Q, void* O, void* strea
  * input, Q is read and O is written exactly as in kvq_decode_attn, and none of the
  * handle's own scratch is used.
  *
- * Limit: batch * q_heads * splits <= KVQ_STATIC_MAX_PARTIALS (splits is what
- * kvq_set_splits fixed, or the library's choice for the cached length); otherwise
+ * Limit: batch * q_heads * (parts + 1) <= KVQ_STATIC_MAX_PARTIALS, where parts is the value
+ * given to kvq_set_splits or, in automatic mode, ceil(W / (batch * q_heads)) with W the
+ * number of warps the launch uses (at most 16 per SM of the device); otherwise
  * KVQ_ERR_TOO_LARGE is returned and nothing is queued.
  *
  * Set-up: the first call on each device looks up the device address of the array (once
@@ -179,8 +181,9 @@ int kvq_reset(kvq_ctx* ctx, void* stream);
 int kvq_seq_len(kvq_ctx* ctx, int layer, int* host_len_out);
 
 /*
- * Number of sequence splits used by kvq_decode_attn: 0 = choose from the
- * cached length and the device's SM count (default), otherwise 1..64.
+ * How kvq_decode_attn cuts the work: 0 = automatic (default): one launch of as many warps as
+ * stay resident on the device, each taking an equal share of all (sequence, query head)
+ * units; 1..64 = every unit is cut into exactly that many equal parts, one warp each.
  */
 int kvq_set_splits(kvq_ctx* ctx, int splits);
 

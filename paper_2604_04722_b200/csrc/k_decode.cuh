@@ -3,26 +3,33 @@
 //
 // Softmax attention does not depend on the order of the cached tokens, so the
 // kernel never touches the per-token index: it walks each precision pool of a
-// (sequence, KV head) front to back.  The sequence is cut into `splits` parts
-// (every part takes the same fraction of every pool, hence the same bytes);
-// each CTA keeps an online softmax in fp32 and emits (m, l, o[64]); a second
-// kernel merges the parts.
+// (sequence, KV head) front to back.
 //
-// Data movement: the tiles of a part are cut into chunks of up to kStageBytes
-// contiguous bytes; chunks are dealt round-robin to the CTA's warps, and every
-// warp runs its own ring of kStages shared-memory buffers filled by 1-D bulk
-// async copies (cp.async.bulk, completion on an mbarrier), issued kStages
-// chunks ahead by lane 0.  No CTA-wide synchronisation happens in the main
-// loop.  Every mbarrier wait is bounded: on expiry the warp records
-// KVQ_FLAG_WAIT_TIMEOUT and leaves the loop.
+// Work split.  The (sequence, query head) units are laid end to end on an axis
+// x, every unit gw ticks long; working warp j of gw owns ticks
+// [j*units, (j+1)*units), i.e. an equal share of the whole launch, cut into
+// SEGMENTS where it crosses unit borders.  A segment [a0, a1) of a unit takes
+// tiles [nt*a0/gw, nt*a1/gw) of EVERY pool of that unit (the same fraction of
+// every pool, hence the same byte and instruction mix for every warp).  Warps
+// are independent: each has its own ring, softmax state and accumulators, and
+// writes one partial (m, l, o[64]) per segment into the slot of its unit; a
+// second kernel merges the slots of a unit.  The launch is persistent when gw
+// is the number of warps resident on the device; nothing in the kernel waits
+// for another warp.
+//
+// Data movement: the tiles of a segment are cut into chunks of up to
+// kStageBytes contiguous bytes; every warp runs its own ring of kStages
+// shared-memory buffers filled by 1-D bulk async copies (cp.async.bulk,
+// completion on an mbarrier), issued kStages chunks ahead by lane 0.  Every
+// mbarrier wait is bounded: on expiry the warp records KVQ_FLAG_WAIT_TIMEOUT
+// and stops.
 //
 // Work layout inside a warp: two lanes per token.  Lane l handles half l/16
 // (elements 32*(l/16) .. +32) of slot l%16 of a 16-token tile, so it keeps 32
-// pre-scaled query values and 32 output accumulators in registers (about half
-// the registers of a lane-per-token mapping: 16 warps stay resident per SM and
-// hide the latency of the dependent FMA chains).  The two half dot products
-// meet through one xor-16 shuffle; the output accumulators are per-lane
-// partial sums reduced once at the end.
+// pre-scaled query values and 32 output accumulators in registers (16 warps
+// stay resident per SM and hide the latency of the dependent FMA chains).  The
+// two half dot products meet through one xor-16 shuffle; the output
+// accumulators are per-lane partial sums reduced once per segment.
 //
 // Dequantization is hoisted out of the inner loops:
 //   q.khat = s_k * sum_i q_i c_i + z_k * sum_i q_i
@@ -74,10 +81,23 @@ struct DecodeParams {
     const uint32_t* counts;        // [batch][4] pool fills of this layer
     const __half* Q;               // [batch][q_heads][64]
     __half* O;                     // [batch][q_heads][64]
-    float* part_o;                 // [batch][q_heads][splits][64]  unnormalised
-    float2* part_ml;               // [batch][q_heads][splits]      (m in log2 units, l)
-    int layer, splits, group;      // group = q_heads / kv_heads
+    float* part_o;                 // [units][pslots][64]  unnormalised
+    float2* part_ml;               // [units][pslots]      (m in log2 units, l)
+    int layer, group;              // group = q_heads / kv_heads
+    uint32_t units;                // batch * q_heads
+    uint32_t gw;                   // working warps = parts the x axis is cut into
+    uint32_t pslots;               // partial slots per unit = decode_pslots(units, gw)
 };
+
+// Warps that can overlap one unit: ceil(gw/units) + 1.
+__host__ __device__ inline uint32_t decode_pslots(uint32_t units, uint32_t gw) { return (gw + units - 1) / units + 1; }
+// First warp whose share overlaps unit u, and the number of warps that do.
+__host__ __device__ inline uint32_t decode_first_warp(uint32_t u, uint32_t units, uint32_t gw) {
+    return (uint32_t)((uint64_t)u * gw / units);
+}
+__host__ __device__ inline uint32_t decode_warps_of_unit(uint32_t u, uint32_t units, uint32_t gw) {
+    return (uint32_t)(((uint64_t)(u + 1) * gw - 1) / units) - decode_first_warp(u, units, gw) + 1;
+}
 
 // ---------------------------------------------------------------- PTX helpers
 
@@ -293,207 +313,214 @@ struct Fp16Rows {
 
 // ---------------------------------------------------------------- the split kernel
 
-// The part of the sequence this CTA owns, as a list of chunks: chunk g in [pre[c], pre[c+1])
-// belongs to class c and covers tiles [lo[c] + (g-pre[c])*TPS, ...) of that class's pool.
-struct ChunkMap {
-    int lo[kNumPools], hi[kNumPools], pre[kNumPools + 1];
-    uint32_t cnt[kNumPools];
+// Per-warp scratch in shared memory: the segment being worked on.
+struct WarpScratch {
+    uint64_t bars[kStages];
+    const uint8_t* base[kNumPools];    // first tile of this (layer, sequence, KV head) in each pool
+    int lo[kNumPools], hi[kNumPools];  // tile range of the segment in each pool
+    uint32_t cnt[kNumPools];           // tokens in each pool
+    float q[kHeadDim + 4];             // query row; half 1 starts at q[36] so the two halves sit in different banks
 };
+constexpr int kQHalfStride = kHalfDim + 4;
 
-__device__ __forceinline__ void chunk_at(const ChunkMap& m, int g, int& c, int& tile0, int& ntiles) {
-    c = (g >= m.pre[1]) + (g >= m.pre[2]) + (g >= m.pre[3]);
-    const int tps = c == 0 ? tiles_per_stage(0) : c == 1 ? tiles_per_stage(1) : c == 2 ? tiles_per_stage(2)
-                                                                                      : tiles_per_stage(3);
-    tile0 = m.lo[c] + (g - m.pre[c]) * tps;
-    ntiles = min(tps, m.hi[c] - tile0);
+__device__ __forceinline__ int tps_of(int c) {
+    return c == 0 ? tiles_per_stage(0) : c == 1 ? tiles_per_stage(1) : c == 2 ? tiles_per_stage(2) : tiles_per_stage(3);
 }
 
-// grid = (splits, q_heads, batch), block = kDecodeThreads, dynamic smem = kDecodeSmemBytes.
+// grid = ceil(gw / kDecodeWarps), block = kDecodeThreads, dynamic smem = kDecodeSmemBytes.
 __global__ void __launch_bounds__(kDecodeThreads, KVQ_DECODE_MIN_CTAS)
 k_decode_split(DecodeParams P) {
     extern __shared__ __align__(128) uint8_t ring[];   // [warps][stages][kStageBytes]
-    __shared__ uint64_t bars[kDecodeWarps][kStages];
-    __shared__ ChunkMap map;
-    __shared__ float q_s[kHeadDim];
-    __shared__ float red_o[kDecodeWarps][kHeadDim];
-    __shared__ float2 red_ml[kDecodeWarps];
-    const int split = blockIdx.x, qh = blockIdx.y, b = blockIdx.z;
-    const int kvh = qh / P.group;
+    __shared__ WarpScratch scratch[kDecodeWarps];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int half = lane >> 4, t = lane & 15;
-
-    if (threadIdx.x < kHeadDim)
-        q_s[threadIdx.x] = __half2float(P.Q[((size_t)b * P.store.q_heads + qh) * kHeadDim + threadIdx.x]);
-    if (threadIdx.x == 0) {
-        const uint32_t* cnt = P.counts + (size_t)b * 4;
-        int pre = 0;
-        for (int c = 0; c < kNumPools; ++c) {
-            const uint32_t n = cnt[c];
-            const int ntiles = (int)((n + kTileTokens - 1) / kTileTokens);
-            map.cnt[c] = n;
-            map.lo[c] = (int)((long long)ntiles * split / P.splits);
-            map.hi[c] = (int)((long long)ntiles * (split + 1) / P.splits);
-            map.pre[c] = pre;
-            pre += (map.hi[c] - map.lo[c] + tiles_per_stage(c) - 1) / tiles_per_stage(c);
-        }
-        map.pre[kNumPools] = pre;
-        for (int w = 0; w < kDecodeWarps; ++w)
-            for (int s = 0; s < kStages; ++s) mbar_init(&bars[w][s], 1);
+    const uint32_t j = blockIdx.x * kDecodeWarps + warp;
+    if (j >= P.gw) return;                             // warps never wait for one another
+    WarpScratch& ws = scratch[warp];
+    uint8_t* my_ring = ring + (size_t)warp * kStages * kStageBytes;
+    if (lane == 0) {
+        for (int s = 0; s < kStages; ++s) mbar_init(&ws.bars[s], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    __syncthreads();
-    float sumq = q_s[lane] + q_s[lane + 32];
-    sumq = warp_sum(sumq) * kLogitScale;               // sum_i q_i, in logit units
-    const float* q_half = q_s + half * kHalfDim;
+    __syncwarp();
 
-    const int total = map.pre[kNumPools];
-    const int n_mine = total > warp ? (total - warp + kDecodeWarps - 1) / kDecodeWarps : 0;   // chunks of this warp
-    uint8_t* my_ring = ring + (size_t)warp * kStages * kStageBytes;
-
-    // lane 0 starts the copy of this warp's i-th chunk into ring slot `slot`
-    auto issue = [&](int i, int slot) {
-        if (lane == 0) {
-            int c, tile0, ntiles;
-            chunk_at(map, warp + i * kDecodeWarps, c, tile0, ntiles);
-            const uint32_t bytes = (uint32_t)ntiles * (uint32_t)pool_rec_bytes(c);
-            const uint8_t* src = P.store.pool[c] + tile_offset(P.store, c, P.layer, b, kvh, tile0);
-            mbar_arrive_expect_tx(&bars[warp][slot], bytes);
-            bulk_load(my_ring + (size_t)slot * kStageBytes, src, bytes, &bars[warp][slot]);
-        }
-    };
-    int issued = 0;
-    for (; issued < kStages && issued < n_mine; ++issued) issue(issued, issued);
-
-    Softmax st = {kNegBig, 0.f, 0.f};
-    float acc[kHalfDim];
-#pragma unroll
-    for (int i = 0; i < kHalfDim; ++i) acc[i] = 0.f;
-
-    int ic = 0, slot = 0;                              // next chunk to consume, its ring slot
-    uint32_t parity = 0;                               // phase parity of `slot`
+    int pslot = 0, cslot = 0;                          // ring slot the next copy goes to / the next chunk is read from
+    uint32_t parity = 0;                               // phase parity of cslot
     bool failed = false;
+    uint64_t x = (uint64_t)j * P.units;
+    const uint64_t xend = x + P.units;
 
-    auto walk = [&](auto cls_tag, auto consumer) {
-        constexpr int CLS = decltype(cls_tag)::value;
-        using C = decltype(consumer);
-        const int i_end = (map.pre[CLS + 1] - warp + kDecodeWarps - 1) / kDecodeWarps;      // my chunks below pre[CLS+1]
-        if (ic >= i_end || failed) return;
-        float qk[kHalfDim];
-        C::enter(q_half, qk, acc);
-        for (; ic < i_end; ++ic) {
-            if (!mbar_wait(&bars[warp][slot], parity)) {
-                failed = true;
-                break;
-            }
-            const int g = warp + ic * kDecodeWarps;
-            const int tile0 = map.lo[CLS] + (g - map.pre[CLS]) * tiles_per_stage(CLS);
-            const int ntiles = min(tiles_per_stage(CLS), map.hi[CLS] - tile0);
-            const uint8_t* buf = my_ring + (size_t)slot * kStageBytes;
-            for (int i = 0; i < ntiles; ++i) {
-                const bool valid = (uint32_t)((tile0 + i) * kTileTokens + t) < map.cnt[CLS];
-                C::tile(buf + (size_t)i * C::REC, valid, half, t, qk, sumq, st, acc);
-            }
-            __syncwarp();                              // every lane is done with the slot before it is refilled
-            if (issued < n_mine) {
-                issue(issued, slot);
-                ++issued;
-            }
-            if (++slot == kStages) {
-                slot = 0;
-                parity ^= 1u;
-            }
+    while (x < xend && !failed) {
+        // ---- this segment: ticks [a0, a1) of unit u
+        const uint32_t u = (uint32_t)(x / P.gw);
+        const uint32_t a0 = (uint32_t)(x - (uint64_t)u * P.gw);
+        const uint64_t room = xend - x;
+        const uint32_t a1 = room < (uint64_t)(P.gw - a0) ? a0 + (uint32_t)room : P.gw;
+        x += a1 - a0;
+        const uint32_t b = u / (uint32_t)P.store.q_heads, qh = u - b * (uint32_t)P.store.q_heads;
+        const int kvh = (int)qh / P.group;
+        if (lane < kNumPools) {                        // lane c plans pool c
+            const int c = lane;
+            const uint32_t n = P.counts[(size_t)b * 4 + c];
+            const uint64_t nt = (n + kTileTokens - 1) / kTileTokens;
+            ws.cnt[c] = n;
+            ws.lo[c] = (int)(nt * a0 / P.gw);
+            ws.hi[c] = (int)(nt * a1 / P.gw);
+            const uint8_t* pool = c == 0 ? P.store.pool[0] : c == 1 ? P.store.pool[1] : c == 2 ? P.store.pool[2]
+                                                                                              : P.store.pool[3];
+            ws.base[c] = pool + tile_offset(P.store, c, P.layer, (int)b, kvh, 0);
         }
-        C::leave(acc);
-    };
-    walk(std::integral_constant<int, 0>{}, Quantized<0>{});
-    walk(std::integral_constant<int, 1>{}, Quantized<1>{});
-    walk(std::integral_constant<int, 2>{}, Quantized<2>{});
-    walk(std::integral_constant<int, 3>{}, Fp16Rows{});
+        {
+            const float2 q2 = __half22float2(reinterpret_cast<const __half2*>(P.Q + (size_t)u * kHeadDim)[lane]);
+            const int i = 2 * lane;                    // elements i, i+1 (same half)
+            float* dst = ws.q + (i >> 5) * kQHalfStride + (i & 31);
+            dst[0] = q2.x;
+            dst[1] = q2.y;
+        }
+        __syncwarp();
+        float sumq = ws.q[lane] + ws.q[kQHalfStride + lane];
+        sumq = warp_sum(sumq) * kLogitScale;           // sum_i q_i, in logit units
+        const float* q_half = ws.q + half * kQHalfStride;
 
-    if (failed) {
-        // Copies that were started but not consumed may still land in this CTA's shared memory:
-        // give each a bounded wait before the CTA can retire, then report.
-        for (int i = ic + 1; i < issued; ++i) {
-            if (++slot == kStages) {
-                slot = 0;
-                parity ^= 1u;
+        // ---- producer cursor (warp-uniform; lane 0 issues)
+        int p_c = 0, p_tile = ws.lo[0];
+        while (p_tile >= ws.hi[p_c]) {
+            if (++p_c >= kNumPools) break;
+            p_tile = ws.lo[p_c];
+        }
+        auto issue_next = [&]() {
+            if (p_c >= kNumPools) return;
+            const int n = min(tps_of(p_c), ws.hi[p_c] - p_tile);
+            if (lane == 0) {
+                const uint32_t rec = (uint32_t)pool_rec_bytes(p_c);
+                const uint32_t bytes = (uint32_t)n * rec;
+                mbar_arrive_expect_tx(&ws.bars[pslot], bytes);
+                bulk_load(my_ring + (size_t)pslot * kStageBytes, ws.base[p_c] + (size_t)p_tile * rec, bytes,
+                          &ws.bars[pslot]);
             }
-            mbar_wait(&bars[warp][slot], parity);
-        }
-        if (lane == 0) atomicOr(P.store.flags, kFlagWaitTimeout);
-    }
+            if (++pslot == kStages) pslot = 0;
+            p_tile += n;
+            while (p_tile >= ws.hi[p_c]) {
+                if (++p_c >= kNumPools) break;
+                p_tile = ws.lo[p_c];
+            }
+        };
+        int in_flight = 0;
+        for (; in_flight < kStages && p_c < kNumPools; ++in_flight) issue_next();
 
-    // ---- reduce the per-lane partial sums over the 16 slots of a half: after four halving steps
-    //      lane L holds elements 2L, 2L+1 of the row
-    float r16[16];
+        Softmax st = {kNegBig, 0.f, 0.f};
+        float acc[kHalfDim];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        const bool up = lane & 8;
-        const float keep = up ? acc[j + 16] : acc[j], send = up ? acc[j] : acc[j + 16];
-        r16[j] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-    }
-    float r8[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const bool up = lane & 4;
-        const float keep = up ? r16[j + 8] : r16[j], send = up ? r16[j] : r16[j + 8];
-        r8[j] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-    }
-    float r4[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const bool up = lane & 2;
-        const float keep = up ? r8[j + 4] : r8[j], send = up ? r8[j] : r8[j + 4];
-        r4[j] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-    }
-    float r2[2];
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-        const bool up = lane & 1;
-        const float keep = up ? r4[j + 2] : r4[j], send = up ? r4[j] : r4[j + 2];
-        r2[j] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
-    }
-    // both lanes of a token added its p and p * zero-point: halve the warp sums
-    const float l_w = 0.5f * warp_sum(st.l);
-    const float b_w = 0.5f * warp_sum(st.bsum);
-    red_o[warp][2 * lane] = r2[0] + b_w;
-    red_o[warp][2 * lane + 1] = r2[1] + b_w;
-    if (lane == 0) red_ml[warp] = make_float2(st.m, l_w);
-    __syncthreads();
+        for (int i = 0; i < kHalfDim; ++i) acc[i] = 0.f;
 
-    // ---- combine the warps and emit this split's partial
-    if (threadIdx.x < kHeadDim) {
-        float M = red_ml[0].x;
-#pragma unroll
-        for (int w = 1; w < kDecodeWarps; ++w) M = fmaxf(M, red_ml[w].x);
-        float L = 0.f, o = 0.f;
-#pragma unroll
-        for (int w = 0; w < kDecodeWarps; ++w) {
-            const float f = fast_exp2(red_ml[w].x - M);
-            L = fmaf(red_ml[w].y, f, L);
-            o = fmaf(red_o[w][threadIdx.x], f, o);
+        auto walk = [&](auto cls_tag, auto consumer) {
+            constexpr int CLS = decltype(cls_tag)::value;
+            using C = decltype(consumer);
+            int tile0 = ws.lo[CLS];
+            const int hi = ws.hi[CLS];
+            if (tile0 >= hi || failed) return;
+            const uint32_t cnt = ws.cnt[CLS];
+            float qk[kHalfDim];
+            C::enter(q_half, qk, acc);
+            while (tile0 < hi) {
+                if (!mbar_wait(&ws.bars[cslot], parity)) {
+                    failed = true;
+                    break;
+                }
+                const int ntiles = min(tiles_per_stage(CLS), hi - tile0);
+                const uint8_t* buf = my_ring + (size_t)cslot * kStageBytes;
+                for (int i = 0; i < ntiles; ++i) {
+                    const bool valid = (uint32_t)((tile0 + i) * kTileTokens + t) < cnt;
+                    C::tile(buf + (size_t)i * C::REC, valid, half, t, qk, sumq, st, acc);
+                }
+                tile0 += ntiles;
+                --in_flight;
+                __syncwarp();                          // every lane is done with the slot before it is refilled
+                if (p_c < kNumPools) {
+                    issue_next();
+                    ++in_flight;
+                }
+                if (++cslot == kStages) {
+                    cslot = 0;
+                    parity ^= 1u;
+                }
+            }
+            C::leave(acc);
+        };
+        walk(std::integral_constant<int, 0>{}, Quantized<0>{});
+        walk(std::integral_constant<int, 1>{}, Quantized<1>{});
+        walk(std::integral_constant<int, 2>{}, Quantized<2>{});
+        walk(std::integral_constant<int, 3>{}, Fp16Rows{});
+
+        if (failed) {
+            // Copies that were started but not consumed may still land in this warp's ring: give
+            // each a bounded wait before the warp can retire, then report.
+            for (int i = 1; i < in_flight; ++i) {
+                if (++cslot == kStages) {
+                    cslot = 0;
+                    parity ^= 1u;
+                }
+                mbar_wait(&ws.bars[cslot], parity);
+            }
+            if (lane == 0) atomicOr(P.store.flags, kFlagWaitTimeout);
         }
-        const size_t unit = ((size_t)b * P.store.q_heads + qh) * P.splits + split;
-        P.part_o[unit * kHeadDim + threadIdx.x] = o;
-        if (threadIdx.x == 0) P.part_ml[unit] = make_float2(M, L);
+
+        // ---- reduce the per-lane partial sums over the 16 slots of a half: after four halving
+        //      steps lane L holds elements 2L, 2L+1 of the row
+        float r16[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const bool up = lane & 8;
+            const float keep = up ? acc[k + 16] : acc[k], send = up ? acc[k] : acc[k + 16];
+            r16[k] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+        }
+        float r8[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const bool up = lane & 4;
+            const float keep = up ? r16[k + 8] : r16[k], send = up ? r16[k] : r16[k + 8];
+            r8[k] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+        }
+        float r4[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const bool up = lane & 2;
+            const float keep = up ? r8[k + 4] : r8[k], send = up ? r8[k] : r8[k + 4];
+            r4[k] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+        }
+        float r2[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const bool up = lane & 1;
+            const float keep = up ? r4[k + 2] : r4[k], send = up ? r4[k] : r4[k + 2];
+            r2[k] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
+        }
+        // both lanes of a token added its p and p * zero-point: halve the warp sums
+        const float l_w = 0.5f * warp_sum(st.l);
+        const float b_w = 0.5f * warp_sum(st.bsum);
+        const size_t recno = (size_t)u * P.pslots + (j - decode_first_warp(u, P.units, P.gw));
+        reinterpret_cast<float2*>(P.part_o + recno * kHeadDim)[lane] = make_float2(r2[0] + b_w, r2[1] + b_w);
+        if (lane == 0) P.part_ml[recno] = make_float2(st.m, l_w);
     }
 }
 
-// Merge the splits: M = max m_j, l = sum l_j 2^(m_j-M), O = sum o_j 2^(m_j-M) / l.
-// grid = batch*q_heads, block = 64.
+// Merge the partials of a unit: M = max m_j, l = sum l_j 2^(m_j-M), O = sum o_j 2^(m_j-M) / l.
+// grid = units, block = 64.
 __global__ void __launch_bounds__(kHeadDim)
 k_decode_merge(DecodeParams P) {
-    const size_t unit0 = (size_t)blockIdx.x * P.splits;
+    const uint32_t u = blockIdx.x;
+    const uint32_t n = decode_warps_of_unit(u, P.units, P.gw);
+    const size_t rec0 = (size_t)u * P.pslots;
     float M = kNegBig;
-    for (int s = 0; s < P.splits; ++s) M = fmaxf(M, P.part_ml[unit0 + s].x);
+    for (uint32_t s = 0; s < n; ++s) M = fmaxf(M, P.part_ml[rec0 + s].x);
     float L = 0.f, o = 0.f;
-    for (int s = 0; s < P.splits; ++s) {
-        const float2 ml = P.part_ml[unit0 + s];
+    for (uint32_t s = 0; s < n; ++s) {
+        const float2 ml = P.part_ml[rec0 + s];
         const float f = fast_exp2(ml.x - M);
         L = fmaf(ml.y, f, L);
-        o = fmaf(P.part_o[(unit0 + s) * kHeadDim + threadIdx.x], f, o);
+        o = fmaf(P.part_o[(rec0 + s) * kHeadDim + threadIdx.x], f, o);
     }
-    P.O[(size_t)blockIdx.x * kHeadDim + threadIdx.x] = __float2half_rn(o / L);
+    P.O[(size_t)u * kHeadDim + threadIdx.x] = __float2half_rn(o / L);
 }
 
 }  // namespace kvq

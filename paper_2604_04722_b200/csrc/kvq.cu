@@ -31,8 +31,8 @@ struct kvq_ctx {
     uint4* hist = nullptr;               // append scratch [batch][max chunks]
     float* ctrl = nullptr;               // controller parameter block
     int hidden = 0;
-    float* part_o = nullptr;             // decode scratch [batch][q_heads][kMaxSplits][64]
-    float2* part_ml = nullptr;           //                [batch][q_heads][kMaxSplits]
+    float* part_o = nullptr;             // decode scratch [units][partial slots][64]
+    float2* part_ml = nullptr;           //                [units][partial slots]
     int splits_override = 0;
     uint32_t* flags = nullptr;
     // device staging for the host-buffer entry points
@@ -168,32 +168,44 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
     return KVQ_OK;
 }
 
-// Number of sequence splits.  Every (sequence, query head) unit is cut into the same number of
-// parts; the grid is units x splits CTAs and kDecodeCtasPerSm CTAs are resident per SM.  Few CTAs:
-// take as many splits as the work allows (a warp should still own a few chunks).  Many CTAs: aim
-// at a handful of full waves and pick the count whose last wave is fullest.
-int choose_splits(kvq_ctx* c, int len) {
-    if (c->splits_override > 0) return c->splits_override;
-    const int tiles = (len + kTileTokens - 1) / kTileTokens + (kNumPools - 1);
-    const int units = c->batch * c->q_heads;
-    const int slots = kDecodeCtasPerSm * c->sm_count;
-    int smax = tiles / (8 * kDecodeWarps);                       // at least eight tiles per warp
-    const int by_waves = (8 * slots + units - 1) / units;        // at most about eight waves
-    if (smax > by_waves) smax = by_waves;
-    if (smax > kMaxSplits) smax = kMaxSplits;
-    if (smax < 1) smax = 1;
-    int best = 1;
-    double best_score = -1.0;
-    for (int s = 1; s <= smax; ++s) {
-        const double fill = (double)units * s / slots;
-        const double waves = fill <= 1.0 ? 1.0 : (double)(long long)(fill + 0.999999);
-        const double score = fill / waves;                       // share of the resident slots kept busy
-        if (score > best_score + 1e-9) {
-            best_score = score;
-            best = s;
-        }
-    }
-    return best;
+// Number of working warps of a decode launch (the x axis is cut into that many equal parts).
+// With an explicit split count every (sequence, query head) unit is cut into exactly that many
+// parts.  Otherwise: as many warps as stay resident on the device (a persistent launch), but not
+// more than the work supports -- a warp should own about eight tiles to pay for its set-up.
+uint32_t choose_warps(kvq_ctx* c, int len) {
+    const uint64_t units = (uint64_t)c->batch * c->q_heads;
+    if (c->splits_override > 0) return (uint32_t)(units * (uint64_t)c->splits_override);
+    const uint64_t tiles = units * (uint64_t)((len + kTileTokens - 1) / kTileTokens + (kNumPools - 1));
+    const uint64_t resident = (uint64_t)kDecodeWarps * kDecodeCtasPerSm * c->sm_count;
+    uint64_t gw = tiles / 8;
+    if (gw > resident) gw = resident;
+    if (gw < 1) gw = 1;
+    return (uint32_t)gw;
+}
+
+// Partial records a handle may need: explicit splits up to kMaxSplits, or a persistent launch.
+size_t max_partial_records(const kvq_ctx* c) {
+    const size_t units = (size_t)c->batch * c->q_heads;
+    const size_t resident = (size_t)kDecodeWarps * kDecodeCtasPerSm * c->sm_count;
+    const size_t by_splits = units * (kMaxSplits + 1);
+    const size_t by_residency = resident + 2 * units;
+    return by_splits > by_residency ? by_splits : by_residency;
+}
+
+// Fill the launch parameters of a decode call and queue split + merge on `st`.
+void fill_decode_params(kvq_ctx* c, int layer, const void* Q, void* O, float* part_o, float2* part_ml, uint32_t gw,
+                        DecodeParams& p) {
+    p.store = c->store;
+    p.counts = counts_of(c, c->cur[layer], layer);
+    p.Q = static_cast<const __half*>(Q);
+    p.O = static_cast<__half*>(O);
+    p.part_o = part_o;
+    p.part_ml = part_ml;
+    p.layer = layer;
+    p.group = c->q_heads / c->kv_heads;
+    p.units = (uint32_t)c->batch * (uint32_t)c->q_heads;
+    p.gw = gw;
+    p.pslots = decode_pslots(p.units, gw);
 }
 
 int export_impl(kvq_ctx* c, int layer, int b0, int nb, int pos0, int n, uint8_t* bits, uint32_t* pool_slot,
@@ -264,8 +276,8 @@ int kvq_create(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_di
     ok = ok && dev_alloc(c, &c->cls, (size_t)batch * max_ctx) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->hist, sizeof(uint4) * batch * max_chunks) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->ctrl, controller_smem(kMaxHidden)) == cudaSuccess;
-    ok = ok && dev_alloc(c, &c->part_o, sizeof(float) * units * kMaxSplits * kHeadDim) == cudaSuccess;
-    ok = ok && dev_alloc(c, &c->part_ml, sizeof(float2) * units * kMaxSplits) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->part_o, sizeof(float) * max_partial_records(c) * kHeadDim) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->part_ml, sizeof(float2) * max_partial_records(c)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->flags, sizeof(uint32_t)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_feats, sizeof(float) * 4 * batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_K, sizeof(__half) * (size_t)batch * kv_heads * kHeadDim) == cudaSuccess;
@@ -361,21 +373,14 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
     DeviceGuard guard(c->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DecodeParams p{};
-    p.store = c->store;
-    p.counts = counts_of(c, c->cur[layer], layer);
-    p.Q = static_cast<const __half*>(Q);
-    p.O = static_cast<__half*>(O);
-    p.part_o = c->part_o;
-    p.part_ml = c->part_ml;
-    p.layer = layer;
-    p.splits = choose_splits(c, c->len[layer]);
-    p.group = c->q_heads / c->kv_heads;
+    fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, choose_warps(c, c->len[layer]), p);
+    const unsigned grid = (p.gw + kDecodeWarps - 1) / kDecodeWarps;
     const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
     cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 3] : nullptr;
     if (rec) cudaEventRecord(ev[0], st);
-    k_decode_split<<<dim3(p.splits, c->q_heads, c->batch), kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    k_decode_split<<<grid, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
     if (rec) cudaEventRecord(ev[1], st);
-    k_decode_merge<<<c->batch * c->q_heads, kHeadDim, 0, st>>>(p);
+    k_decode_merge<<<p.units, kHeadDim, 0, st>>>(p);
     if (rec) {
         cudaEventRecord(ev[2], st);
         c->prof_calls += 1;
@@ -399,8 +404,8 @@ int kvq_decode_attn_static(kvq_ctx* c, int layer, const void* Q, void* O, void* 
     if (check_layer(c, layer) != KVQ_OK || !Q || !O) return KVQ_ERR_ARG;
     if (c->len[layer] == 0) return KVQ_ERR_EMPTY;
     if (c->device < 0 || c->device >= KVQ_STATIC_MAX_DEVICES) return KVQ_ERR_ARG;
-    const int splits = choose_splits(c, c->len[layer]);
-    const size_t records = (size_t)c->batch * c->q_heads * splits;
+    const uint32_t gw = choose_warps(c, c->len[layer]);
+    const size_t records = (size_t)c->batch * c->q_heads * decode_pslots((uint32_t)c->batch * c->q_heads, gw);
     if (records > (size_t)KVQ_STATIC_MAX_PARTIALS) return KVQ_ERR_TOO_LARGE;
     DeviceGuard guard(c->device);
     float* base = nullptr;
@@ -415,17 +420,10 @@ int kvq_decode_attn_static(kvq_ctx* c, int layer, const void* Q, void* O, void* 
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DecodeParams p{};
-    p.store = c->store;
-    p.counts = counts_of(c, c->cur[layer], layer);
-    p.Q = static_cast<const __half*>(Q);
-    p.O = static_cast<__half*>(O);
-    p.part_o = base;                                                        // [records][64]
-    p.part_ml = reinterpret_cast<float2*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * kHeadDim);   // [records]
-    p.layer = layer;
-    p.splits = splits;
-    p.group = c->q_heads / c->kv_heads;
-    k_decode_split<<<dim3(p.splits, c->q_heads, c->batch), kDecodeThreads, kDecodeSmemBytes, st>>>(p);
-    k_decode_merge<<<c->batch * c->q_heads, kHeadDim, 0, st>>>(p);
+    fill_decode_params(c, layer, Q, O, base, reinterpret_cast<float2*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * kHeadDim),
+                       gw, p);
+    k_decode_split<<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    k_decode_merge<<<p.units, kHeadDim, 0, st>>>(p);
     c->launches += 2;
     KVQ_CUDA(c, cudaGetLastError());
     return KVQ_OK;
@@ -605,7 +603,7 @@ const char* kvq_strerror(int code) {
     case KVQ_ERR_EMPTY: return "layer holds no token";
     case KVQ_ERR_DEVICE_FLAG: return "a kernel recorded a problem";
     case KVQ_ERR_NOMEM: return "out of memory";
-    case KVQ_ERR_TOO_LARGE: return "batch * q_heads * splits exceeds the static scratch of kvq_decode_attn_static";
+    case KVQ_ERR_TOO_LARGE: return "batch * q_heads * (parts + 1) exceeds the static scratch of kvq_decode_attn_static";
     default: return "unknown error";
     }
 }

@@ -76,17 +76,17 @@ def test_static_scratch_entry_rejects_what_does_not_fit(gu):
     try:
         Qd = gu.dev(synth.queries(7, 0, 0, g.B, g.Hq).view(np.uint16))
         O = torch.zeros_like(Qd)
-        kq.kvq_set_splits(g.ctx, 64)                      # 16 * 9 * 64 = 9216 records > 8192
-        assert 16 * 9 * 64 > kq.KVQ_STATIC_MAX_PARTIALS
+        kq.kvq_set_splits(g.ctx, 64)                      # 16 * 9 * (64 + 1) = 9360 records > 8192
+        assert 16 * 9 * 65 > kq.KVQ_STATIC_MAX_PARTIALS
         with pytest.raises(kq.KvqError) as err:
             kq.kvq_decode_attn_static(g.ctx, 0, Qd, O)
         assert err.value.code == kq.KVQ_ERR_TOO_LARGE
         assert "static scratch" in str(err.value)
-        kq.kvq_set_splits(g.ctx, 56)                      # 8064 records fit
+        kq.kvq_set_splits(g.ctx, 55)                      # 16 * 9 * 56 = 8064 records fit
         kq.kvq_decode_attn_static(g.ctx, 0, Qd, O)
         want = torch.zeros_like(Qd)
         kq.kvq_decode_attn(g.ctx, 0, Qd, want)
         torch.cuda.synchronize()
-        gu.assert_attention_close(O.cpu().numpy().view(np.uint16), want.cpu().numpy().view(np.uint16), "56 splits")
+        gu.assert_attention_close(O.cpu().numpy().view(np.uint16), want.cpu().numpy().view(np.uint16), "55 parts")
     finally:
         g.close()
