@@ -45,7 +45,7 @@
 #include "kvq_common.cuh"
 
 #ifndef KVQ_DECODE_STAGES
-#define KVQ_DECODE_STAGES 3
+#define KVQ_DECODE_STAGES 2
 #endif
 #ifndef KVQ_DECODE_WARPS
 #define KVQ_DECODE_WARPS 4
@@ -54,7 +54,7 @@
 #define KVQ_DECODE_MIN_CTAS 4
 #endif
 #ifndef KVQ_DECODE_STAGE_BYTES
-#define KVQ_DECODE_STAGE_BYTES 4352
+#define KVQ_DECODE_STAGE_BYTES 6528
 #endif
 
 namespace kvq {
@@ -63,7 +63,7 @@ constexpr int kDecodeWarps = KVQ_DECODE_WARPS;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kDecodeCtasPerSm = KVQ_DECODE_MIN_CTAS;
 constexpr int kStages = KVQ_DECODE_STAGES;
-constexpr int kStageBytes = KVQ_DECODE_STAGE_BYTES;   // two 8-bit tiles; 6 / 3 / 2 / 1 tiles of the four classes
+constexpr int kStageBytes = KVQ_DECODE_STAGE_BYTES;   // three 8-bit tiles; 10 / 5 / 3 / 1 tiles of the four classes
 constexpr int kHalfDim = kHeadDim / 2;           // elements per lane
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLogitScale = 0.125f * kLog2e;   // 1/sqrt(64), in log2 units
@@ -173,15 +173,17 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 struct Softmax {
     float m, l, bsum;              // running max (log2 units), sum of p, sum of p * zero-point
+    float thr;                     // m + kRescaleSlack: a logit above it forces a rescale
 };
 
 // Fold a tile's logits into the running state and return this lane's p.  The running maximum
 // is only raised when some logit exceeds it by more than kRescaleSlack (one vote per tile).
 __device__ __forceinline__ float softmax_step(Softmax& st, float (&acc)[kHalfDim], float y) {
-    if (__any_sync(0xffffffffu, y > st.m + kRescaleSlack)) {       // warp-uniform
+    if (__any_sync(0xffffffffu, y > st.thr)) {                     // warp-uniform
         const float tmax = warp_max(y);
         const float f = fast_exp2(st.m - tmax);
         st.m = tmax;
+        st.thr = tmax + kRescaleSlack;
         st.l *= f;
         st.bsum *= f;
 #pragma unroll
@@ -326,6 +328,11 @@ constexpr int kQHalfStride = kHalfDim + 4;
 __device__ __forceinline__ int tps_of(int c) {
     return c == 0 ? tiles_per_stage(0) : c == 1 ? tiles_per_stage(1) : c == 2 ? tiles_per_stage(2) : tiles_per_stage(3);
 }
+// floor(n * a / g) for a <= g < 65536 in 32-bit arithmetic: n = q*g + r gives q*a + floor(r*a/g).
+__device__ __forceinline__ uint32_t scale_by_fraction(uint32_t n, uint32_t a, uint32_t g) {
+    const uint32_t q = n / g, r = n - q * g;
+    return q * a + r * a / g;
+}
 
 // grid = ceil(gw / kDecodeWarps), block = kDecodeThreads, dynamic smem = kDecodeSmemBytes.
 __global__ void __launch_bounds__(kDecodeThreads, KVQ_DECODE_MIN_CTAS)
@@ -352,7 +359,7 @@ k_decode_split(DecodeParams P) {
 
     while (x < xend && !failed) {
         // ---- this segment: ticks [a0, a1) of unit u
-        const uint32_t u = (uint32_t)(x / P.gw);
+        const uint32_t u = (x >> 32) ? (uint32_t)(x / P.gw) : (uint32_t)x / P.gw;
         const uint32_t a0 = (uint32_t)(x - (uint64_t)u * P.gw);
         const uint64_t room = xend - x;
         const uint32_t a1 = room < (uint64_t)(P.gw - a0) ? a0 + (uint32_t)room : P.gw;
@@ -362,10 +369,15 @@ k_decode_split(DecodeParams P) {
         if (lane < kNumPools) {                        // lane c plans pool c
             const int c = lane;
             const uint32_t n = P.counts[(size_t)b * 4 + c];
-            const uint64_t nt = (n + kTileTokens - 1) / kTileTokens;
+            const uint32_t nt = (n + kTileTokens - 1) / kTileTokens;
             ws.cnt[c] = n;
-            ws.lo[c] = (int)(nt * a0 / P.gw);
-            ws.hi[c] = (int)(nt * a1 / P.gw);
+            if (P.gw < 65536u) {
+                ws.lo[c] = (int)scale_by_fraction(nt, a0, P.gw);
+                ws.hi[c] = (int)scale_by_fraction(nt, a1, P.gw);
+            } else {
+                ws.lo[c] = (int)((uint64_t)nt * a0 / P.gw);
+                ws.hi[c] = (int)((uint64_t)nt * a1 / P.gw);
+            }
             const uint8_t* pool = c == 0 ? P.store.pool[0] : c == 1 ? P.store.pool[1] : c == 2 ? P.store.pool[2]
                                                                                               : P.store.pool[3];
             ws.base[c] = pool + tile_offset(P.store, c, P.layer, (int)b, kvh, 0);
@@ -382,33 +394,36 @@ k_decode_split(DecodeParams P) {
         sumq = warp_sum(sumq) * kLogitScale;           // sum_i q_i, in logit units
         const float* q_half = ws.q + half * kQHalfStride;
 
-        // ---- producer cursor (warp-uniform; lane 0 issues)
-        int p_c = 0, p_tile = ws.lo[0];
-        while (p_tile >= ws.hi[p_c]) {
-            if (++p_c >= kNumPools) break;
-            p_tile = ws.lo[p_c];
-        }
-        auto issue_next = [&]() {
-            if (p_c >= kNumPools) return;
-            const int n = min(tps_of(p_c), ws.hi[p_c] - p_tile);
-            if (lane == 0) {
-                const uint32_t rec = (uint32_t)pool_rec_bytes(p_c);
-                const uint32_t bytes = (uint32_t)n * rec;
-                mbar_arrive_expect_tx(&ws.bars[pslot], bytes);
-                bulk_load(my_ring + (size_t)pslot * kStageBytes, ws.base[p_c] + (size_t)p_tile * rec, bytes,
-                          &ws.bars[pslot]);
-            }
-            if (++pslot == kStages) pslot = 0;
-            p_tile += n;
-            while (p_tile >= ws.hi[p_c]) {
-                if (++p_c >= kNumPools) break;
-                p_tile = ws.lo[p_c];
+        // ---- producer cursor (warp-uniform; lane 0 issues): next tile to fetch, tiles left in its pool
+        int p_c = -1, p_left = 0, p_tps = 0;
+        uint32_t p_rec = 0;
+        const uint8_t* p_ptr = nullptr;
+        auto next_pool = [&]() {                       // move to the next pool that has tiles in this segment
+            while (p_left == 0 && ++p_c < kNumPools) {
+                const int lo = ws.lo[p_c];
+                p_left = ws.hi[p_c] - lo;
+                p_tps = tps_of(p_c);
+                p_rec = (uint32_t)pool_rec_bytes(p_c);
+                p_ptr = ws.base[p_c] + (size_t)lo * p_rec;
             }
         };
+        next_pool();
+        auto issue_next = [&]() {
+            const int n = min(p_tps, p_left);
+            const uint32_t bytes = (uint32_t)n * p_rec;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(&ws.bars[pslot], bytes);
+                bulk_load(my_ring + (size_t)pslot * kStageBytes, p_ptr, bytes, &ws.bars[pslot]);
+            }
+            if (++pslot == kStages) pslot = 0;
+            p_ptr += bytes;
+            p_left -= n;
+            if (p_left == 0) next_pool();
+        };
         int in_flight = 0;
-        for (; in_flight < kStages && p_c < kNumPools; ++in_flight) issue_next();
+        for (; in_flight < kStages && p_left > 0; ++in_flight) issue_next();
 
-        Softmax st = {kNegBig, 0.f, 0.f};
+        Softmax st = {kNegBig, 0.f, 0.f, kNegBig};
         float acc[kHalfDim];
 #pragma unroll
         for (int i = 0; i < kHalfDim; ++i) acc[i] = 0.f;
@@ -436,7 +451,7 @@ k_decode_split(DecodeParams P) {
                 tile0 += ntiles;
                 --in_flight;
                 __syncwarp();                          // every lane is done with the slot before it is refilled
-                if (p_c < kNumPools) {
+                if (p_left > 0) {
                     issue_next();
                     ++in_flight;
                 }
