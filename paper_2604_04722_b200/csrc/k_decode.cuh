@@ -34,13 +34,20 @@
 // Dequantization is hoisted out of the inner loops:
 //   q.khat = s_k * sum_i q_i c_i + z_k * sum_i q_i
 //   sum_t p_t vhat_t = sum_t (p_t s_t) c_t + sum_t p_t z_t
-// and the integer codes enter the fp32 FMAs without any int->float conversion:
-// a bit field of a packed word that lies inside bits [0,24) of a 32-bit word,
-// read as an fp32 bit pattern, IS the number code * 2^(k-149) (subnormal /
-// first-binade encoding is linear), so one AND per element isolates it and the
-// power of two is folded into a pre-scaled copy of q (for K) or into the
-// accumulator's exponent (for V).  Products stay in the normal range, so the
-// arithmetic is exact fp32 FMA work: ~2 issue slots per cached element.
+//
+// K side: sum_i q_i c_i is an integer dot product.  q is put on a 16-bit fixed-point grid once
+// per segment (q_i * R rounded to nearest, R the power of two that brings max|q| just below
+// 2^15: an error below 2^-16 of max|q| per element, against fp16's own 2^-11 of each element),
+// the codes are masked IN PLACE into byte lanes (2-bit: four masks 0x03030303 << 2k per word,
+// 4-bit: two masks, 8-bit: none) and dp2a multiplies two 16-bit q values by two code bytes and
+// accumulates exactly in int32; the planes' weights 4^k / 16^k are undone by a Horner step on
+// the integer sums.  That is 0.75 / 0.75 / 0.5 issue slots per element instead of 2.
+//
+// V side: the integer codes enter fp32 FMAs without any int->float conversion: a bit field of a
+// packed word that lies inside bits [0,24) of a 32-bit word, read as an fp32 bit pattern, IS the
+// number code * 2^(k-149) (subnormal / first-binade encoding is linear), so one AND per element
+// isolates it and the power of two is folded into the accumulator's exponent.  Products stay in
+// the normal range, so the arithmetic is exact fp32 FMA work: 2 issue slots per element.
 #pragma once
 #include "kvq_common.cuh"
 
@@ -141,6 +148,18 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// d = c + a.h0 * b.b0 + a.h1 * b.b1 (lo) or a.h0 * b.b2 + a.h1 * b.b3 (hi); a signed 16-bit, b unsigned 8-bit.
+__device__ __forceinline__ int dp2a_lo(uint32_t a, uint32_t b, int c) {
+    int d;
+    asm("dp2a.lo.s32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ int dp2a_hi(uint32_t a, uint32_t b, int c) {
+    int d;
+    asm("dp2a.hi.s32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 __device__ __forceinline__ float pow2f(int e) { return __int_as_float((127 + e) << 23); }
 
 // Exponent offset of element e (0-based inside its 32-bit word) for BITS-wide codes:
@@ -201,20 +220,42 @@ __device__ __forceinline__ float2 meta_to_float2(uint32_t m) {     // {scale, ze
 // ---------------------------------------------------------------- tile consumers (data in shared memory)
 // Every consumer sees one 16-token tile record `rec`; the lane handles half `half` of slot `t`.
 
+// What a consumer needs to know about the query of the current segment.
+struct QueryInfo {
+    const float* q_half;           // this lane's 32 query values (shared memory)
+    float fix_scale;               // R: q * R is the 16-bit fixed-point query
+    float inv_fix;                 // kLogitScale / R
+    float sumq;                    // kLogitScale * sum_i q_i
+};
+constexpr int kQRegs = kHalfDim;   // registers a consumer may use for its copy of the query
+
 template <int CLS>
 struct Quantized {
     static constexpr int BITS = pool_bits(CLS), REC = pool_rec_bytes(CLS);
     static constexpr int EPW = 32 / BITS;              // elements per 32-bit word
     static constexpr int WORDS = pool_half_bytes(CLS) / 4;         // words per half-row: 2, 4, 8
     static constexpr int UNITS = pool_units(CLS), UWORDS = pool_unit_bytes(CLS) / 4;
+    static constexpr int PLANES = 8 / BITS;            // codes per byte: 4, 2, 1
+    static constexpr uint32_t PLANE0 = 0x01010101u * ((1u << BITS) - 1u);   // mask of plane 0
 
-    // pre-scaled query and accumulator exponent domain of this class
-    __device__ static __forceinline__ void enter(const float* q_half, float (&qk)[kHalfDim], float (&acc)[kHalfDim]) {
+    // Element (inside the half-row) that sits in byte j of plane k of word wi.
+    __device__ static constexpr int element(int wi, int k, int j) { return wi * EPW + j * PLANES + k; }
+
+    // qreg[0..15]: the fixed-point query as 16-bit pairs, pair (wi, k, hh) = bytes 2hh, 2hh+1 of plane k of
+    // word wi.  The accumulators move to this class's exponent domain (for the V side).
+    __device__ static __forceinline__ void enter(const QueryInfo& qi, uint32_t (&qreg)[kQRegs], float (&acc)[kHalfDim]) {
 #pragma unroll
-        for (int i = 0; i < kHalfDim; ++i) {
-            qk[i] = q_half[i] * pow2f(100 - field_pos<BITS>(i % EPW));
-            acc[i] *= pow2f(field_pos<BITS>(i % EPW) - 49);
-        }
+        for (int wi = 0; wi < WORDS; ++wi)
+#pragma unroll
+            for (int k = 0; k < PLANES; ++k)
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int lo = __float2int_rn(qi.q_half[element(wi, k, 2 * hh)] * qi.fix_scale);
+                    const int hi = __float2int_rn(qi.q_half[element(wi, k, 2 * hh + 1)] * qi.fix_scale);
+                    qreg[(wi * PLANES + k) * 2 + hh] = ((uint32_t)lo & 0xffffu) | ((uint32_t)hi << 16);
+                }
+#pragma unroll
+        for (int i = 0; i < kHalfDim; ++i) acc[i] *= pow2f(field_pos<BITS>(i % EPW) - 49);
     }
     __device__ static __forceinline__ void leave(float (&acc)[kHalfDim]) {
 #pragma unroll
@@ -233,24 +274,28 @@ struct Quantized {
         }
     }
     __device__ static __forceinline__ void tile(const uint8_t* rec, bool valid, int half, int t,
-                                                const float (&qk)[kHalfDim], float sumq_scaled, Softmax& st,
+                                                const uint32_t (&qreg)[kQRegs], const QueryInfo& qi, Softmax& st,
                                                 float (&acc)[kHalfDim]) {
         uint32_t w[WORDS];
         load_half_row(rec, half, t, w);
         const float2 km = meta_to_float2(*reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 0, t)));
-        float d[4] = {0.f, 0.f, 0.f, 0.f};
+        int d[PLANES];
 #pragma unroll
-        for (int wi = 0; wi < WORDS; ++wi) {
-            const uint32_t hi8 = w[wi] >> 8;
+        for (int k = 0; k < PLANES; ++k) d[k] = 0;
 #pragma unroll
-            for (int e = 0; e < EPW; ++e) {
-                const int i = wi * EPW + e;
-                d[i & 3] = fmaf(field_as_float<BITS>(w[wi], hi8, e), qk[i], d[i & 3]);
+        for (int wi = 0; wi < WORDS; ++wi)
+#pragma unroll
+            for (int k = 0; k < PLANES; ++k) {
+                const uint32_t plane = PLANES == 1 ? w[wi] : (w[wi] & (PLANE0 << (k * BITS)));   // bytes = code << k*BITS
+                d[k] = dp2a_lo(qreg[(wi * PLANES + k) * 2], plane, d[k]);
+                d[k] = dp2a_hi(qreg[(wi * PLANES + k) * 2 + 1], plane, d[k]);
             }
-        }
-        float dot = (d[0] + d[1]) + (d[2] + d[3]);
+        int dsum = d[0];                               // Horner: sum_k d[k] * 2^(BITS*(PLANES-1-k))
+#pragma unroll
+        for (int k = 1; k < PLANES; ++k) dsum = (dsum << BITS) + d[k];
+        float dot = (float)dsum;
         dot += __shfl_xor_sync(0xffffffffu, dot, 16);              // the other half of the row
-        float y = fmaf(km.x * (pow2f(49) * kLogitScale), dot, km.y * sumq_scaled);
+        float y = fmaf(km.x * (qi.inv_fix * (1.0f / (float)(1 << (BITS * (PLANES - 1))))), dot, km.y * qi.sumq);
         y = valid ? y : -INFINITY;
         const float p = softmax_step(st, acc, y);
 
@@ -273,13 +318,13 @@ struct Quantized {
 // The fp16 pool: rows are stored unchanged; qk holds the plain query.
 struct Fp16Rows {
     static constexpr int REC = pool_rec_bytes(3), UNITS = pool_units(3), WORDS = pool_half_bytes(3) / 4;
-    __device__ static __forceinline__ void enter(const float* q_half, float (&qk)[kHalfDim], float (&)[kHalfDim]) {
+    __device__ static __forceinline__ void enter(const QueryInfo& qi, uint32_t (&qreg)[kQRegs], float (&)[kHalfDim]) {
 #pragma unroll
-        for (int i = 0; i < kHalfDim; ++i) qk[i] = q_half[i];
+        for (int i = 0; i < kHalfDim; ++i) qreg[i] = __float_as_uint(qi.q_half[i] * kLogitScale);
     }
     __device__ static __forceinline__ void leave(float (&)[kHalfDim]) {}
     __device__ static __forceinline__ void tile(const uint8_t* rec, bool valid, int half, int t,
-                                                const float (&qk)[kHalfDim], float, Softmax& st,
+                                                const uint32_t (&qreg)[kQRegs], const QueryInfo&, Softmax& st,
                                                 float (&acc)[kHalfDim]) {
         float d[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -289,13 +334,12 @@ struct Fp16Rows {
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi) {
                 const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[wi]));
-                d[wi] = fmaf(f.x, qk[u * 8 + wi * 2], d[wi]);
-                d[wi] = fmaf(f.y, qk[u * 8 + wi * 2 + 1], d[wi]);
+                d[wi] = fmaf(f.x, __uint_as_float(qreg[u * 8 + wi * 2]), d[wi]);
+                d[wi] = fmaf(f.y, __uint_as_float(qreg[u * 8 + wi * 2 + 1]), d[wi]);
             }
         }
-        float dot = (d[0] + d[1]) + (d[2] + d[3]);
-        dot += __shfl_xor_sync(0xffffffffu, dot, 16);
-        float y = dot * kLogitScale;
+        float y = (d[0] + d[1]) + (d[2] + d[3]);
+        y += __shfl_xor_sync(0xffffffffu, y, 16);
         y = valid ? y : -INFINITY;
         const float p = softmax_step(st, acc, y);
 #pragma unroll
@@ -390,9 +434,17 @@ k_decode_split(DecodeParams P) {
             dst[1] = q2.y;
         }
         __syncwarp();
-        float sumq = ws.q[lane] + ws.q[kQHalfStride + lane];
-        sumq = warp_sum(sumq) * kLogitScale;           // sum_i q_i, in logit units
-        const float* q_half = ws.q + half * kQHalfStride;
+        QueryInfo qi;
+        {
+            const float qa = ws.q[lane], qb = ws.q[kQHalfStride + lane];
+            qi.sumq = warp_sum(qa + qb) * kLogitScale; // sum_i q_i, in logit units
+            // R = 2^(14 - floor(log2 max|q|)), max|q| taken as at least the smallest normal fp16
+            const float qmax = fmaxf(warp_max(fmaxf(fabsf(qa), fabsf(qb))), 6.103515625e-05f);
+            const uint32_t e = __float_as_uint(qmax) >> 23;        // biased exponent, 113..142
+            qi.fix_scale = __uint_as_float((268u - e) << 23);
+            qi.inv_fix = __uint_as_float((e - 14u) << 23) * kLogitScale;
+            qi.q_half = ws.q + half * kQHalfStride;
+        }
 
         // ---- producer cursor (warp-uniform; lane 0 issues): next tile to fetch, tiles left in its pool
         int p_c = -1, p_left = 0, p_tps = 0;
@@ -435,8 +487,8 @@ k_decode_split(DecodeParams P) {
             const int hi = ws.hi[CLS];
             if (tile0 >= hi || failed) return;
             const uint32_t cnt = ws.cnt[CLS];
-            float qk[kHalfDim];
-            C::enter(q_half, qk, acc);
+            uint32_t qreg[kQRegs];
+            C::enter(qi, qreg, acc);
             while (tile0 < hi) {
                 if (!mbar_wait(&ws.bars[cslot], parity)) {
                     failed = true;
@@ -446,7 +498,7 @@ k_decode_split(DecodeParams P) {
                 const uint8_t* buf = my_ring + (size_t)cslot * kStageBytes;
                 for (int i = 0; i < ntiles; ++i) {
                     const bool valid = (uint32_t)((tile0 + i) * kTileTokens + t) < cnt;
-                    C::tile(buf + (size_t)i * C::REC, valid, half, t, qk, sumq, st, acc);
+                    C::tile(buf + (size_t)i * C::REC, valid, half, t, qreg, qi, st, acc);
                 }
                 tile0 += ntiles;
                 --in_flight;
