@@ -35,13 +35,15 @@
 //   q.khat = s_k * sum_i q_i c_i + z_k * sum_i q_i
 //   sum_t p_t vhat_t = sum_t (p_t s_t) c_t + sum_t p_t z_t
 //
-// K side: sum_i q_i c_i is an integer dot product.  q is put on a 16-bit fixed-point grid once
-// per segment (q_i * R rounded to nearest, R the power of two that brings max|q| just below
-// 2^15: an error below 2^-16 of max|q| per element, against fp16's own 2^-11 of each element),
-// the codes are masked IN PLACE into byte lanes (2-bit: four masks 0x03030303 << 2k per word,
-// 4-bit: two masks, 8-bit: none) and dp2a multiplies two 16-bit q values by two code bytes and
-// accumulates exactly in int32; the planes' weights 4^k / 16^k are undone by a Horner step on
-// the integer sums.  That is 0.75 / 0.75 / 0.5 issue slots per element instead of 2.
+// K side: sum_i q_i c_i is an integer dot product.  q is put on a 24-bit fixed-point grid once
+// per segment: T_i = rint(q_i * 256 R), R the power of two that brings max|q| R just below 2^15
+// (an error below 2^-24 of max|q| per element, so elements up to 2^13 times smaller than the
+// largest keep fp16's own 11 bits), and T_i = 256 * hi_i + lo_i with a signed 16-bit hi and a
+// signed 8-bit lo.  The codes are masked IN PLACE into byte lanes (2-bit: four masks
+// 0x03030303 << 2k per word, 4-bit: two masks, 8-bit: none); dp2a multiplies two hi values by
+// two code bytes, dp4a four lo values by four code bytes, both accumulate exactly in int32, and
+// the planes' weights 4^k / 16^k are undone by a Horner step on the integer sums.  That is about
+// 1 / 1 / 0.75 issue slots per element instead of 2, on fewer of the half-rate integer ALU slots.
 //
 // V side: the integer codes enter fp32 FMAs without any int->float conversion: a bit field of a
 // packed word that lies inside bits [0,24) of a 32-bit word, read as an fp32 bit pattern, IS the
@@ -160,6 +162,13 @@ __device__ __forceinline__ int dp2a_hi(uint32_t a, uint32_t b, int c) {
     return d;
 }
 
+// d = c + sum_j a.b_j * b.b_j; a signed 8-bit, b unsigned 8-bit.
+__device__ __forceinline__ int dp4a_su(uint32_t a, uint32_t b, int c) {
+    int d;
+    asm("dp4a.s32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 __device__ __forceinline__ float pow2f(int e) { return __int_as_float((127 + e) << 23); }
 
 // Exponent offset of element e (0-based inside its 32-bit word) for BITS-wide codes:
@@ -223,8 +232,8 @@ __device__ __forceinline__ float2 meta_to_float2(uint32_t m) {     // {scale, ze
 // What a consumer needs to know about the query of the current segment.
 struct QueryInfo {
     const float* q_half;           // this lane's 32 query values (shared memory)
-    float fix_scale;               // R: q * R is the 16-bit fixed-point query
-    float inv_fix;                 // kLogitScale / R
+    float fix_scale;               // 256 R: rint(q * 256 R) is the 24-bit fixed-point query
+    float inv_fix;                 // kLogitScale / (256 R)
     float sumq;                    // kLogitScale * sum_i q_i
 };
 constexpr int kQRegs = kHalfDim;   // registers a consumer may use for its copy of the query
@@ -241,19 +250,26 @@ struct Quantized {
     // Element (inside the half-row) that sits in byte j of plane k of word wi.
     __device__ static constexpr int element(int wi, int k, int j) { return wi * EPW + j * PLANES + k; }
 
-    // qreg[0..15]: the fixed-point query as 16-bit pairs, pair (wi, k, hh) = bytes 2hh, 2hh+1 of plane k of
-    // word wi.  The accumulators move to this class's exponent domain (for the V side).
+    // The fixed-point query T = 256 * hi + lo.  qreg[0..15]: hi as 16-bit pairs, pair (wi, k, hh) = bytes
+    // 2hh, 2hh+1 of plane k of word wi; qreg[16..23]: lo as 8-bit quads, quad (wi, k) = bytes 0..3 of that
+    // plane.  The accumulators move to this class's exponent domain (for the V side).
     __device__ static __forceinline__ void enter(const QueryInfo& qi, uint32_t (&qreg)[kQRegs], float (&acc)[kHalfDim]) {
 #pragma unroll
         for (int wi = 0; wi < WORDS; ++wi)
 #pragma unroll
-            for (int k = 0; k < PLANES; ++k)
+            for (int k = 0; k < PLANES; ++k) {
+                uint32_t hi[4], lo[4];
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int lo = __float2int_rn(qi.q_half[element(wi, k, 2 * hh)] * qi.fix_scale);
-                    const int hi = __float2int_rn(qi.q_half[element(wi, k, 2 * hh + 1)] * qi.fix_scale);
-                    qreg[(wi * PLANES + k) * 2 + hh] = ((uint32_t)lo & 0xffffu) | ((uint32_t)hi << 16);
+                for (int j = 0; j < 4; ++j) {
+                    const int T = __float2int_rn(qi.q_half[element(wi, k, j)] * qi.fix_scale);
+                    const int h = (T + 128) >> 8;                  // T = 256 h + l, -128 <= l <= 127
+                    hi[j] = (uint32_t)h & 0xffffu;
+                    lo[j] = (uint32_t)(T - (h << 8)) & 0xffu;
                 }
+                qreg[(wi * PLANES + k) * 2] = hi[0] | (hi[1] << 16);
+                qreg[(wi * PLANES + k) * 2 + 1] = hi[2] | (hi[3] << 16);
+                qreg[16 + wi * PLANES + k] = lo[0] | (lo[1] << 8) | (lo[2] << 16) | (lo[3] << 24);
+            }
 #pragma unroll
         for (int i = 0; i < kHalfDim; ++i) acc[i] *= pow2f(field_pos<BITS>(i % EPW) - 49);
     }
@@ -279,21 +295,25 @@ struct Quantized {
         uint32_t w[WORDS];
         load_half_row(rec, half, t, w);
         const float2 km = meta_to_float2(*reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 0, t)));
-        int d[PLANES];
+        int dh[PLANES], dl[PLANES];
 #pragma unroll
-        for (int k = 0; k < PLANES; ++k) d[k] = 0;
+        for (int k = 0; k < PLANES; ++k) dh[k] = dl[k] = 0;
 #pragma unroll
         for (int wi = 0; wi < WORDS; ++wi)
 #pragma unroll
             for (int k = 0; k < PLANES; ++k) {
                 const uint32_t plane = PLANES == 1 ? w[wi] : (w[wi] & (PLANE0 << (k * BITS)));   // bytes = code << k*BITS
-                d[k] = dp2a_lo(qreg[(wi * PLANES + k) * 2], plane, d[k]);
-                d[k] = dp2a_hi(qreg[(wi * PLANES + k) * 2 + 1], plane, d[k]);
+                dh[k] = dp2a_lo(qreg[(wi * PLANES + k) * 2], plane, dh[k]);
+                dh[k] = dp2a_hi(qreg[(wi * PLANES + k) * 2 + 1], plane, dh[k]);
+                dl[k] = dp4a_su(qreg[16 + wi * PLANES + k], plane, dl[k]);
             }
-        int dsum = d[0];                               // Horner: sum_k d[k] * 2^(BITS*(PLANES-1-k))
+        int hsum = dh[0], lsum = dl[0];                // Horner: sum_k d[k] * 2^(BITS*(PLANES-1-k))
 #pragma unroll
-        for (int k = 1; k < PLANES; ++k) dsum = (dsum << BITS) + d[k];
-        float dot = (float)dsum;
+        for (int k = 1; k < PLANES; ++k) {
+            hsum = (hsum << BITS) + dh[k];
+            lsum = (lsum << BITS) + dl[k];
+        }
+        float dot = fmaf((float)hsum, 256.0f, (float)lsum);
         dot += __shfl_xor_sync(0xffffffffu, dot, 16);              // the other half of the row
         float y = fmaf(km.x * (qi.inv_fix * (1.0f / (float)(1 << (BITS * (PLANES - 1))))), dot, km.y * qi.sumq);
         y = valid ? y : -INFINITY;
@@ -438,11 +458,11 @@ k_decode_split(DecodeParams P) {
         {
             const float qa = ws.q[lane], qb = ws.q[kQHalfStride + lane];
             qi.sumq = warp_sum(qa + qb) * kLogitScale; // sum_i q_i, in logit units
-            // R = 2^(14 - floor(log2 max|q|)), max|q| taken as at least the smallest normal fp16
+            // 256 R = 2^(22 - floor(log2 max|q|)), max|q| taken as at least the smallest normal fp16
             const float qmax = fmaxf(warp_max(fmaxf(fabsf(qa), fabsf(qb))), 6.103515625e-05f);
             const uint32_t e = __float_as_uint(qmax) >> 23;        // biased exponent, 113..142
-            qi.fix_scale = __uint_as_float((268u - e) << 23);
-            qi.inv_fix = __uint_as_float((e - 14u) << 23) * kLogitScale;
+            qi.fix_scale = __uint_as_float((276u - e) << 23);
+            qi.inv_fix = __uint_as_float((e - 22u) << 23) * kLogitScale;
             qi.q_half = ws.q + half * kQHalfStride;
         }
 

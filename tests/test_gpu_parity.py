@@ -246,6 +246,26 @@ def test_decode_peaked_softmax_and_large_logits(gu, oracle):
     _attend_case(gu, oracle, rng, B, Hq, H, n, bits, splits=(0, 5), kscale=12.0)
 
 
+@pytest.mark.parametrize("qscale,spread", [(1.0, 8.0), (0.01, 8.0), (30.0, 1.0), (1.0, 64.0), (1.0, 1000.0)])
+def test_decode_query_dynamic_range(gu, oracle, qscale, spread):
+    """The K-side dot product runs on a fixed-point copy of the query row: rows with outlier
+    channels (some elements `spread` times larger than the rest), very small and very large rows must
+    stay inside the attention tolerance.  The quantized keys carry x8 outlier channels as well."""
+    rng = np.random.default_rng(int(qscale * 100 + spread))
+    B, Hq, H, n = 2, 6, 2, 1100
+    bits = BITS[rng.choice(4, size=(B, n), p=[.4, .35, .2, .05])]
+    K, V = _kv(rng, B, n, H)
+    K[:, :, :, [3, 17, 40, 55]] *= np.float16(8.0)
+    Q = rng.standard_normal((B, Hq, 64)).astype(np.float32) * qscale
+    Q[:, :, [5, 17, 33, 60]] *= spread
+    Q = Q.astype(np.float16)
+    oc = oracle.OracleCache(B, Hq, H)
+    oc.append(K, V, bits)
+    with gu.GpuCache(1, B, Hq, H, n) as g:
+        g.append(0, K, V, bits)
+        gu.assert_attention_close(g.decode(0, Q), oc.decode_attn(Q), "qscale=%g spread=%g" % (qscale, spread))
+
+
 def test_decode_after_incremental_steps(gu, oracle):
     """Prefill, then decode steps that append one token and attend (Eq. 4 then Eq. 5 each step)."""
     rng = np.random.default_rng(17)
