@@ -42,9 +42,11 @@ ROW_BYTES = {2: 40, 4: 72, 8: 136, 16: 256}          # K+V bytes per (token, KV 
 METRIC = "decode_step_kv_bandwidth"
 UNIT = "GB/s"
 
-# DRAM traffic of one k_decode_split launch on this workload, from the ncu capture summarised in
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM traffic of one k_decode_split launch on this workload (dram__bytes_read.sum +
+# dram__bytes_write.sum): captured with a quarter of the sequences (profiles/k_decode_split_cfg5_batch4.md,
+# 320.7 MB per launch) and scaled by the rows read (x 4); every row is read exactly once, so traffic
+# grows in proportion.  Set to None whenever the kernel changes after the capture.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 320.7e6
 
 
 def measured_peak_gbs():
