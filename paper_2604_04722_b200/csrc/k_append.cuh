@@ -10,10 +10,14 @@
 // double-buffered (read `counts_in`, write `counts_out`) so no CTA reads a
 // counter another CTA of the same launch writes.
 //
-// Row quantizer: eight lanes per row, 16 bytes (8 fp16) per lane; min/max by
-// three xor-shuffles; fp32 scale with IEEE divide, fp16 round, IEEE reciprocal,
-// codes by round-to-nearest-even -- all with explicit _rn intrinsics so the
-// result is the same bit pattern on every build.
+// Row quantizer: a warp quantizes one 16-slot tile of one (class, KV head) at a time, with the
+// lane mapping of the store (lane l: half-row l/16 of slot l%16), so the tokens of a chunk are
+// first grouped by class (a list per class in slot order) and every store of the warp is one
+// contiguous run of the tile record.  Min/max in packed fp16 (exact), one xor-16 shuffle, fp32
+// scale with IEEE divide, fp16 round, IEEE reciprocal, codes by round-to-nearest-even (adding
+// 1.5 * 2^23 rounds a float in [0, 2^22) to an integer exactly as rint does) -- all with explicit
+// _rn intrinsics so the result is the same bit pattern on every build.  Codes are packed in the
+// float domain (sums of code * 2^(b*i) below 2^16 are exact) or, for bytes, by byte permutes.
 #pragma once
 #include "kvq_common.cuh"
 #include "k_controller.cuh"
@@ -87,90 +91,101 @@ k_classify(AppendParams p) {
     }
 }
 
-// Quantize one row held by an 8-lane group (x = this lane's 8 elements) and store it.
-// cls: class of the token; slot: its slot in that class's pool; tensor 0 = K, 1 = V.
-__device__ __forceinline__ void quantize_store_row(const StoreView& s, uint4 raw, bool valid, int cls, int layer,
-                                                   int b, int h, uint32_t slot, int tensor, int sub) {
-    const __half2* hp = reinterpret_cast<const __half2*>(&raw);
-    float x[8];
+constexpr float kRoundMagic = 12582912.0f;             // 1.5 * 2^23
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// Quantize the half-row this lane holds (raw = its 32 fp16 values = 64 bytes of the input row) with
+// class CLS < 3 and store it: the lane's units of the tile's code block `codes`, and (half 0 only)
+// the {scale, zero-point} word at `meta`.  Both lanes of a slot (l, l ^ 16) must call together.
+template <int CLS>
+__device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], bool active, int half, int t,
+                                                        uint8_t* codes, uint8_t* meta) {
+    constexpr int BITS = pool_bits(CLS);
+    constexpr float LEVELS = (float)((1 << BITS) - 1);
+    const __half2* hp = reinterpret_cast<const __half2*>(raw);
+    __half2 mn2 = hp[0], mx2 = hp[0];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float2 f = __half22float2(hp[i]);
-        x[2 * i] = f.x;
-        x[2 * i + 1] = f.y;
+    for (int i = 1; i < 16; ++i) {
+        mn2 = __hmin2(mn2, hp[i]);
+        mx2 = __hmax2(mx2, hp[i]);
     }
-    float mn = x[0], mx = x[0];
-#pragma unroll
-    for (int i = 1; i < 8; ++i) {
-        mn = fminf(mn, x[i]);
-        mx = fmaxf(mx, x[i]);
-    }
-#pragma unroll
-    for (int d = 1; d < 8; d <<= 1) {
-        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, d));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
-    }
+    float mn = fminf(__low2float(mn2), __high2float(mn2));
+    float mx = fmaxf(__low2float(mx2), __high2float(mx2));
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 16));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
     if (mn == 0.0f) mn = 0.0f;                         // -0 is stored as +0
     if (mx == 0.0f) mx = 0.0f;
-    const int bits = cls < 3 ? pool_bits(cls) : 8;     // fp16 rows skip the codes; keep the shifts in range
-    const int levels = (1 << bits) - 1;
-    const float s32 = __fdiv_rn(__fsub_rn(mx, mn), (float)levels);
+    const float s32 = __fdiv_rn(__fsub_rn(mx, mn), LEVELS);
     const __half s16 = __float2half_rn(s32);
     const float sf = __half2float(s16);
     const float inv = sf == 0.0f ? 0.0f : __frcp_rn(sf);
-    uint32_t lo = 0, hi = 0;                           // this lane's packed codes (up to 64 bits)
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        int c = __float2int_rn(__fmul_rn(__fsub_rn(x[i], mn), inv));
-        c = min(max(c, 0), levels);
-        int pos = i * bits;                            // < 64 for bits <= 8
-        if (pos < 32) lo |= (uint32_t)c << pos;
-        else hi |= (uint32_t)c << (pos - 32);
-    }
-    // pair up 16-bit halves for the 2-bit class (executed by every lane, used by one branch)
-    const uint32_t lo_next = __shfl_down_sync(0xffffffffu, lo, 1);
-    if (!valid) return;
 
-    const int t = (int)(slot & (kTileTokens - 1));
-    uint8_t* rec = s.pool[cls] + tile_offset(s, cls, layer, b, h, (int)(slot / kTileTokens));
-    uint8_t* codes = rec + (size_t)tensor * pool_codes_bytes(cls);
-    const int half = sub >> 2, q = sub & 3;            // this lane's 8 elements: quarter q of half-row `half`
-    switch (cls) {
-    case 0:                                            // 2 bytes per lane -> 4-byte words from even lanes
-        if ((sub & 1) == 0)
-            *reinterpret_cast<uint32_t*>(codes + unit_offset(0, half, 0, t) + (q >> 1) * 4) = (lo & 0xffffu) | (lo_next << 16);
-        break;
-    case 1:                                            // 4 bytes per lane
-        *reinterpret_cast<uint32_t*>(codes + unit_offset(1, half, 0, t) + q * 4) = lo;
-        break;
-    case 2:                                            // 8 bytes per lane
-        *reinterpret_cast<uint2*>(codes + unit_offset(2, half, q >> 1, t) + (q & 1) * 8) = make_uint2(lo, hi);
-        break;
-    default:                                           // fp16: the lane's 16 input bytes are one unit
-        *reinterpret_cast<uint4*>(codes + unit_offset(3, half, q, t)) = raw;
-        break;
+    // r[i] = clamp(rint((x_i - mn) * inv), 0, LEVELS) as a float; the product is never negative
+    float r[32];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float2 f = __half22float2(hp[i]);
+        const float v0 = fminf(__fmul_rn(__fsub_rn(f.x, mn), inv), LEVELS);
+        const float v1 = fminf(__fmul_rn(__fsub_rn(f.y, mn), inv), LEVELS);
+        r[2 * i] = __fadd_rn(v0, kRoundMagic);
+        r[2 * i + 1] = __fadd_rn(v1, kRoundMagic);
     }
-    if (cls < 3 && sub == 0) {
-        uint32_t meta = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(__float2half_rn(mn)) << 16);
-        *reinterpret_cast<uint32_t*>(rec + meta_offset(cls, tensor, t)) = meta;
+    if (!active) return;
+    if (CLS == 2) {                                    // the code is the low byte of r's bit pattern
+        uint32_t w[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t lo = prmt(__float_as_uint(r[4 * k]), __float_as_uint(r[4 * k + 1]), 0x0040u);
+            const uint32_t hi = prmt(__float_as_uint(r[4 * k + 2]), __float_as_uint(r[4 * k + 3]), 0x0040u);
+            w[k] = prmt(lo, hi, 0x5410u);
+        }
+        *reinterpret_cast<uint4*>(codes + unit_offset(2, half, 0, t)) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(codes + unit_offset(2, half, 1, t)) = make_uint4(w[4], w[5], w[6], w[7]);
+    } else {                                           // 16-bit groups summed exactly in fp32
+        constexpr int PER = 16 / BITS;                 // elements per 16-bit group: 8 or 4
+        constexpr int GROUPS = 32 / PER;               // 4 or 8
+        uint32_t g16[GROUPS];
+#pragma unroll
+        for (int g = 0; g < GROUPS; ++g) {
+            float a = 0.f;
+#pragma unroll
+            for (int e = 0; e < PER; ++e) a = fmaf(__fsub_rn(r[g * PER + e], kRoundMagic), (float)(1 << (BITS * e)), a);
+            g16[g] = __float2uint_rn(a);
+        }
+        if (CLS == 0) {
+            *reinterpret_cast<uint2*>(codes + unit_offset(0, half, 0, t)) =
+                make_uint2(g16[0] | (g16[1] << 16), g16[2] | (g16[3] << 16));
+        } else {
+            *reinterpret_cast<uint4*>(codes + unit_offset(1, half, 0, t)) =
+                make_uint4(g16[0] | (g16[1] << 16), g16[2] | (g16[3] << 16), g16[4] | (g16[5] << 16),
+                           g16[6] | (g16[7] << 16));
+        }
     }
+    if (half == 0)
+        *reinterpret_cast<uint32_t*>(meta) =
+            (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(__float2half_rn(mn)) << 16);
 }
 
 // Launch 2.  MODE 0: classes come from k_classify (several chunks per sequence);
 // MODE 1: one chunk, classes from `bits`; MODE 2: one chunk, classes from the controller.
 // grid = (nchunks, head_groups, batch), block = 256.
 template <int MODE>
-__global__ void __launch_bounds__(kChunkTokens)
+__global__ void __launch_bounds__(kChunkTokens, 2)
 k_quant_pack(AppendParams p) {
     extern __shared__ float sW[];
     __shared__ uint32_t wtot[kChunkTokens / 32][4];
     __shared__ uint32_t base[4];
-    __shared__ uint32_t tok_slot[kChunkTokens];
+    __shared__ uint8_t list[4][kChunkTokens];         // tokens of the chunk by class, in slot order
     const int chunk = blockIdx.x, hg = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int t = chunk * kChunkTokens + threadIdx.x;
-    const bool live = t < p.n_new;
-    const size_t tok = (size_t)b * p.n_new + t;
+    const int tok_i = chunk * kChunkTokens + threadIdx.x;
+    const bool live = tok_i < p.n_new;
+    const size_t tok = (size_t)b * p.n_new + tok_i;
 
     // ---- class of this thread's token
     int c = -1;
@@ -220,42 +235,93 @@ k_quant_pack(AppendParams p) {
     }
     __syncthreads();
     if (live) {
-        uint32_t slot = base[c] + rank;
-        for (int w = 0; w < warp; ++w) slot += wtot[w][c];
-        uint32_t word = ((uint32_t)c << 30) | slot;
-        tok_slot[threadIdx.x] = word;
-        if (hg == 0) p.store.index[((size_t)p.layer * p.store.batch + b) * p.store.max_ctx + p.pos0 + t] = word;
+        for (int w = 0; w < warp; ++w) rank += wtot[w][c];
+        list[c][rank] = (uint8_t)threadIdx.x;
+        if (hg == 0)
+            p.store.index[((size_t)p.layer * p.store.batch + b) * p.store.max_ctx + p.pos0 + tok_i] =
+                ((uint32_t)c << 30) | (base[c] + rank);
     }
-    if (hg == 0 && chunk == p.nchunks - 1 && threadIdx.x < 4) {
-        uint32_t tot = base[threadIdx.x];
-        for (int w = 0; w < kChunkTokens / 32; ++w) tot += wtot[w][threadIdx.x];
-        p.counts_out[(size_t)b * 4 + threadIdx.x] = tot;
+    uint32_t ncls[4];                                  // tokens of each class in this chunk
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        ncls[k] = 0;
+        for (int w = 0; w < kChunkTokens / 32; ++w) ncls[k] += wtot[w][k];
     }
+    if (hg == 0 && chunk == p.nchunks - 1 && threadIdx.x < 4)
+        p.counts_out[(size_t)b * 4 + threadIdx.x] = base[threadIdx.x] + ncls[threadIdx.x];
     __syncthreads();
 
-    // ---- rows: 8 lanes per row, K and V of (token i, head h) together
-    const int ntok = min(kChunkTokens, p.n_new - chunk * kChunkTokens);
+    // ---- tiles: class k touches tiles [first[k], first[k] + nt[k]) of its pool
+    uint32_t first[4], pre[5];
+    pre[0] = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        first[k] = base[k] / kTileTokens;
+        const uint32_t nt = ncls[k] ? (base[k] + ncls[k] - 1) / kTileTokens - first[k] + 1 : 0;
+        pre[k + 1] = pre[k] + nt;
+    }
     const int h0 = hg * p.heads_per_group;
     const int nh = min(p.heads_per_group, p.store.kv_heads - h0);
-    const int items = ntok * nh;
-    const int group = threadIdx.x >> 3, sub = threadIdx.x & 7;
-    const size_t row_stride = kHeadDim;                                  // halves
-    for (int r0 = 0; r0 < items; r0 += kChunkTokens / 8) {
-        const int r = r0 + group;
-        const bool valid = r < items;
-        const int i = valid ? r / nh : 0;
-        const int h = h0 + (valid ? r % nh : 0);
-        const size_t src = (((size_t)b * p.n_new + (size_t)chunk * kChunkTokens + i) * p.store.kv_heads + h) * row_stride;
-        uint4 kraw = make_uint4(0, 0, 0, 0), vraw = kraw;
-        if (valid) {
-            kraw = __ldg(reinterpret_cast<const uint4*>(p.K + src) + sub);
-            vraw = __ldg(reinterpret_cast<const uint4*>(p.V + src) + sub);
+    const int half = lane >> 4, t = lane & 15;
+    // work items (tile tau, head hh), heads fastest, dealt round-robin to the warps
+    uint32_t tau = 0;
+    int hh = warp;
+    while (hh >= nh) {
+        hh -= nh;
+        ++tau;
+    }
+    while (tau < pre[4]) {
+        const int k = (tau >= pre[1]) + (tau >= pre[2]) + (tau >= pre[3]);
+        const uint32_t basek = k == 0 ? base[0] : k == 1 ? base[1] : k == 2 ? base[2] : base[3];
+        const uint32_t nk = k == 0 ? ncls[0] : k == 1 ? ncls[1] : k == 2 ? ncls[2] : ncls[3];
+        const uint32_t tile = (k == 0 ? first[0] : k == 1 ? first[1] : k == 2 ? first[2] : first[3]) +
+                              (tau - (k == 0 ? pre[0] : k == 1 ? pre[1] : k == 2 ? pre[2] : pre[3]));
+        const uint32_t r = tile * kTileTokens + t - basek;       // rank of this lane's slot in the chunk (wraps if before)
+        const bool active = r < nk;
+        const int h = h0 + hh;
+        uint4 kraw[4], vraw[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) kraw[i] = vraw[i] = make_uint4(0, 0, 0, 0);
+        if (active) {
+            const int i_tok = list[k][r];
+            const size_t src = (((size_t)b * p.n_new + (size_t)chunk * kChunkTokens + i_tok) * p.store.kv_heads + h) * kHeadDim +
+                               half * (kHeadDim / 2);
+            const uint4* ks = reinterpret_cast<const uint4*>(p.K + src);
+            const uint4* vs = reinterpret_cast<const uint4*>(p.V + src);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) kraw[i] = __ldg(ks + i);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) vraw[i] = __ldg(vs + i);
         }
-        const uint32_t word = tok_slot[i];
-        const int cls = (int)(word >> 30);
-        const uint32_t slot = word & 0x3fffffffu;
-        quantize_store_row(p.store, kraw, valid, cls, p.layer, b, h, slot, 0, sub);
-        quantize_store_row(p.store, vraw, valid, cls, p.layer, b, h, slot, 1, sub);
+        uint8_t* rec = p.store.pool[k] + tile_offset(p.store, k, p.layer, b, h, (int)tile);
+        switch (k) {
+        case 0:
+            quantize_store_half_row<0>(kraw, active, half, t, rec, rec + meta_offset(0, 0, t));
+            quantize_store_half_row<0>(vraw, active, half, t, rec + pool_codes_bytes(0), rec + meta_offset(0, 1, t));
+            break;
+        case 1:
+            quantize_store_half_row<1>(kraw, active, half, t, rec, rec + meta_offset(1, 0, t));
+            quantize_store_half_row<1>(vraw, active, half, t, rec + pool_codes_bytes(1), rec + meta_offset(1, 1, t));
+            break;
+        case 2:
+            quantize_store_half_row<2>(kraw, active, half, t, rec, rec + meta_offset(2, 0, t));
+            quantize_store_half_row<2>(vraw, active, half, t, rec + pool_codes_bytes(2), rec + meta_offset(2, 1, t));
+            break;
+        default:                                       // fp16: the lane's 64 input bytes are its four units
+            if (active) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    *reinterpret_cast<uint4*>(rec + unit_offset(3, half, u, t)) = kraw[u];
+                    *reinterpret_cast<uint4*>(rec + pool_codes_bytes(3) + unit_offset(3, half, u, t)) = vraw[u];
+                }
+            }
+            break;
+        }
+        hh += kChunkTokens / 32;
+        while (hh >= nh) {
+            hh -= nh;
+            ++tau;
+        }
     }
 }
 
