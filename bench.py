@@ -42,8 +42,8 @@ ROW_BYTES = {2: 40, 4: 72, 8: 136, 16: 256}          # K+V bytes per (token, KV 
 METRIC = "decode_step_kv_bandwidth"
 UNIT = "GB/s"
 
-# DRAM traffic of one k_decode_split launch on this workload (dram__bytes_read.sum +
-# dram__bytes_write.sum): captured with a quarter of the sequences (profiles/k_decode_split_cfg5_batch4.md,
+# DRAM traffic of one k_decode_attn launch on this workload (dram__bytes_read.sum +
+# dram__bytes_write.sum): captured with a quarter of the sequences (profiles/k_decode_attn_cfg5_batch4.md,
 # 320.7 MB per launch) and scaled by the rows read (x 4); every row is read exactly once, so traffic
 # grows in proportion.  Set to None whenever the kernel changes after the capture.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 320.7e6
@@ -314,7 +314,7 @@ def run_ours(args, wl):
         dist.barrier()
     ms_total = ev0.elapsed_time(ev1)
     launches_timed = kq.kvq_launch_count(ctx) - launches1
-    split_ms, merge_ms, ncalls = kq.kvq_profile_read(ctx)
+    attn_ms, ncalls = kq.kvq_profile_read(ctx)
     kq.kvq_set_profiling(ctx, False)
     time.sleep(0.2)
     clocks = sampler.stop()
@@ -346,16 +346,15 @@ def run_ours(args, wl):
 
     # ---- reduce over ranks: slowest rank's time, summed bytes
     ms_step = ms_total / K_steps
-    vals = torch.tensor([ms_step, ms_e2e, split_ms / max(ncalls, 1), merge_ms / max(ncalls, 1)],
-                        dtype=torch.float64, device=dev)
+    vals = torch.tensor([ms_step, ms_e2e, attn_ms / max(ncalls, 1)], dtype=torch.float64, device=dev)
     if dist is not None:
         dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    ms_step, ms_e2e, ms_split, ms_merge = [float(x) for x in vals.tolist()]
+    ms_step, ms_e2e, ms_attn = [float(x) for x in vals.tolist()]
 
     dec_bytes, app_bytes = step_bytes(wl, ctx_len, resident_mean, new_rows_mean)
     bytes_step = dec_bytes + app_bytes
     peak, peak_kind = measured_peak_gbs()
-    achieved = dec_bytes / (ms_split * 1e-3) / 1e9
+    achieved = dec_bytes / (ms_attn * 1e-3) / 1e9
     index_bytes = B * (ctx_len + W + K_steps / 2) * 4
 
     cpu = None
@@ -375,14 +374,13 @@ def run_ours(args, wl):
             "e2e": {"value": world * bytes_step / (ms_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms_e2e,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches_timed),
-            "roofline": {"bound": "hbm", "kernel": "k_decode_split", "achieved": achieved, "peak": peak,
+            "roofline": {"bound": "hbm", "kernel": "k_decode_attn", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": "of " + peak_kind,
                          "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "algorithmic_bytes_per_launch": dec_bytes,
-                         "avg_launch_us": ms_split * 1e3,
-                         "frac_with_index_bytes": (dec_bytes + index_bytes) / (ms_split * 1e-3) / 1e9 / peak},
+                         "avg_launch_us": ms_attn * 1e3,
+                         "frac_with_index_bytes": (dec_bytes + index_bytes) / (ms_attn * 1e-3) / 1e9 / peak},
             "cpu_baseline": cpu,
-            "decode_attn_us_per_step": (ms_split + ms_merge) * 1e3,
-            "decode_merge_us": ms_merge * 1e3,
+            "decode_attn_us_per_step": ms_attn * 1e3,
             "step_us": ms_step * 1e3,
             "append_prefill_tokens_per_s": {
                 "controller_fused": B * ctx_len / (ms_prefill_fused * 1e-3),

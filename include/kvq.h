@@ -122,8 +122,9 @@ int kvq_append_fused(kvq_ctx* ctx, int layer, const void* K, const void* V,
  * Decode-step attention (Eq. 5) of one query row per (sequence, query head)
  * over every token cached in `layer`, dequantizing on the fly:
  * O = Softmax(q K^T / 8) V.  Q, O: dev fp16 [batch][q_heads][64].  fp32
- * accumulation, online softmax; the work is split over warps (see kvq_set_splits) whose
- * partial results a second kernel merges.
+ * accumulation, online softmax; the work is split over warps (see kvq_set_splits); the warp
+ * that delivers the last partial result of a (sequence, query head) merges them, all in one
+ * kernel.
  * KVQ_ERR_EMPTY if the layer holds no token.
  */
 int kvq_decode_attn(kvq_ctx* ctx, int layer, const void* Q, void* O, void* stream);
@@ -137,8 +138,9 @@ int kvq_decode_attn(kvq_ctx* ctx, int layer, const void* Q, void* O, void* strea
  * memory is entirely owned by another allocator, a caller that cannot tolerate the implicit
  * device synchronisation of cudaMalloc/cudaFree.  Such a caller cannot ask a library to
  * reserve per-call or per-handle scratch on its behalf.  Here the split-attention partials
- * (the only scratch the decode step needs) live in a fixed array that is part of the
- * library image: KVQ_STATIC_MAX_PARTIALS records of 66 floats, about 2.1 MB, which every
+ * and their arrival counters (the only scratch the decode step needs) live in a fixed array
+ * that is part of the library image: KVQ_STATIC_MAX_PARTIALS records of 66 floats plus the
+ * counters, about 2.2 MB, which every
  * GPU that loads the library holds until the process exits.  The call performs no
  * cudaMalloc, no cudaFree and calls no allocating routine; the handle's store is read as
  * input, Q is read and O is written exactly as in kvq_decode_attn, and none of the
@@ -154,9 +156,10 @@ int kvq_decode_attn(kvq_ctx* ctx, int layer, const void* Q, void* O, void* strea
  *
  * Sharing: every call on a device uses the same array, whatever the handle or stream.
  * Two calls whose kernels overlap on the GPU (different streams, or different threads)
- * race on it; serialise them.  The array keeps the previous call's partials; nothing in it
- * has to start at zero, because every record the merge reads is written first by the same
- * call.
+ * race on it; serialise them.  The array keeps the previous call's partials, which is
+ * harmless: every record a merge reads is written first by the same call.  Only the arrival
+ * counters must be zero when a call starts; they are zero when the library is loaded and
+ * each call puts back to zero every counter it used.
  */
 #define KVQ_STATIC_MAX_PARTIALS 8192
 int kvq_decode_attn_static(kvq_ctx* ctx, int layer, const void* Q, void* O, void* stream);
@@ -221,15 +224,14 @@ int kvq_stats(kvq_ctx* ctx, int layer, uint32_t* host_counts, uint64_t* resident
               double* expected_bits);
 
 /*
- * Timing hooks for benchmarks.  While profiling is on, kvq_decode_attn records CUDA
- * events on its stream before the split kernel, between the two kernels and after the
- * merge kernel (up to 1024 calls are kept; later calls are not recorded).
+ * Timing hooks for benchmarks.  While profiling is on, kvq_decode_attn records CUDA events on its
+ * stream before and after its kernel (up to 1024 calls are kept; later calls are not recorded).
  * kvq_profile_read synchronizes, adds up the elapsed times of the recorded calls into
- * split_ms_total / merge_ms_total (host doubles, may be NULL), stores their number in
- * calls (host int, may be NULL) and forgets them.
+ * attn_ms_total (host double, may be NULL), stores their number in calls (host int, may be NULL)
+ * and forgets them.
  */
 int kvq_set_profiling(kvq_ctx* ctx, int on);
-int kvq_profile_read(kvq_ctx* ctx, double* split_ms_total, double* merge_ms_total, int* calls);
+int kvq_profile_read(kvq_ctx* ctx, double* attn_ms_total, int* calls);
 
 /* Device flags recorded by kernels since the last call (host uint32, cleared on read). */
 #define KVQ_FLAG_BAD_BITS 1u      /* a bit-width outside {2,4,8,16} was appended (stored as fp16) */

@@ -47,7 +47,7 @@ SIGNATURES = {
     "kvq_export_token": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvq_stats": (_i, [_vp, _i, _vp, _u64p, C.POINTER(C.c_double)]),
     "kvq_set_profiling": (_i, [_vp, _i]),
-    "kvq_profile_read": (_i, [_vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_i)]),
+    "kvq_profile_read": (_i, [_vp, C.POINTER(C.c_double), C.POINTER(_i)]),
     "kvq_device_status": (_i, [_vp, C.POINTER(C.c_uint32)]),
     "kvq_device_bytes": (_i, [_vp, _u64p]),
     "kvq_launch_count": (_i, [_vp, _u64p]),
@@ -200,10 +200,10 @@ def kvq_set_profiling(ctx: int, on: bool) -> None:
 
 
 def kvq_profile_read(ctx: int):
-    """Returns (split_ms_total, merge_ms_total, calls) of the decode calls recorded since the last read."""
-    a, b, n = C.c_double(), C.c_double(), _i()
-    check(lib().kvq_profile_read(ctx, C.byref(a), C.byref(b), C.byref(n)), "kvq_profile_read")
-    return a.value, b.value, n.value
+    """Returns (attn_ms_total, calls) of the decode calls recorded since the last read."""
+    a, n = C.c_double(), _i()
+    check(lib().kvq_profile_read(ctx, C.byref(a), C.byref(n)), "kvq_profile_read")
+    return a.value, n.value
 
 
 def kvq_device_status(ctx: int) -> int:

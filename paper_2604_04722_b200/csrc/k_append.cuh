@@ -16,8 +16,8 @@
 // contiguous run of the tile record.  Min/max in packed fp16 (exact), one xor-16 shuffle, fp32
 // scale with IEEE divide, fp16 round, IEEE reciprocal, codes by round-to-nearest-even (adding
 // 1.5 * 2^23 rounds a float in [0, 2^22) to an integer exactly as rint does) -- all with explicit
-// _rn intrinsics so the result is the same bit pattern on every build.  Codes are packed in the
-// float domain (sums of code * 2^(b*i) below 2^16 are exact) or, for bytes, by byte permutes.
+// _rn intrinsics so the result is the same bit pattern on every build.  Codes are packed by adding
+// the shifted bit patterns of the rounded sums in wrapping 32-bit arithmetic.
 #pragma once
 #include "kvq_common.cuh"
 #include "k_controller.cuh"
@@ -25,6 +25,12 @@
 namespace kvq {
 
 constexpr int kChunkTokens = 256;      // tokens per slot-assignment chunk == threads per CTA
+#ifndef KVQ_APPEND_DEPTH
+#define KVQ_APPEND_DEPTH 2
+#endif
+#ifndef KVQ_APPEND_MIN_CTAS
+#define KVQ_APPEND_MIN_CTAS 3
+#endif
 
 struct AppendParams {
     StoreView store;
@@ -92,17 +98,53 @@ k_classify(AppendParams p) {
 }
 
 constexpr float kRoundMagic = 12582912.0f;             // 1.5 * 2^23
+constexpr int kAppendDepth = KVQ_APPEND_DEPTH;         // items whose input rows are in flight per warp
+constexpr size_t kAppendRingBytes = (size_t)(kChunkTokens / 32) * kAppendDepth * 8 * 32 * sizeof(uint4);
 
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+                 "l"(gmem_src)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// Codes of the 32 values hp[0..15] packed little-endian into words.  rint is done by adding
+// 1.5 * 2^23 (the sum's bit pattern is 0x4B400000 + code); the words are sums of shifted bit patterns
+// in wrapping 32-bit arithmetic, minus the constant the 0x4B400000 terms add up to.
+template <int CLS, bool CLAMP>
+__device__ __forceinline__ void pack_codes(const __half2* hp, float mn, float inv, uint32_t (&w)[pool_half_bytes(CLS) / 4]) {
+    constexpr int BITS = pool_bits(CLS), EPW = 32 / BITS, WORDS = pool_half_bytes(CLS) / 4;
+    constexpr float LEVELS = (float)((1 << BITS) - 1);
+    uint32_t bias = 0;
+#pragma unroll
+    for (int e = 0; e < EPW; ++e) bias += 0x4B400000u << (BITS * e);
+#pragma unroll
+    for (int wi = 0; wi < WORDS; ++wi) {
+        uint32_t acc = 0u - bias;
+#pragma unroll
+        for (int e = 0; e < EPW; e += 2) {
+            const float2 f = __half22float2(hp[(wi * EPW + e) / 2]);
+            float v0 = __fmul_rn(__fsub_rn(f.x, mn), inv), v1 = __fmul_rn(__fsub_rn(f.y, mn), inv);
+            if (CLAMP) {
+                v0 = fminf(v0, LEVELS);
+                v1 = fminf(v1, LEVELS);
+            }
+            acc += __float_as_uint(__fadd_rn(v0, kRoundMagic)) << (BITS * e);
+            acc += __float_as_uint(__fadd_rn(v1, kRoundMagic)) << (BITS * (e + 1));
+        }
+        w[wi] = acc;
+    }
 }
 
 // Quantize the half-row this lane holds (raw = its 32 fp16 values = 64 bytes of the input row) with
 // class CLS < 3 and store it: the lane's units of the tile's code block `codes`, and (half 0 only)
 // the {scale, zero-point} word at `meta`.  Both lanes of a slot (l, l ^ 16) must call together.
-template <int CLS>
+// PARTNER: lane distance (xor) to the lane that holds the other half of the same row.
+template <int CLS, int PARTNER = 16>
 __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], bool active, int half, int t,
                                                         uint8_t* codes, uint8_t* meta) {
     constexpr int BITS = pool_bits(CLS);
@@ -116,8 +158,8 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
     }
     float mn = fminf(__low2float(mn2), __high2float(mn2));
     float mx = fmaxf(__low2float(mx2), __high2float(mx2));
-    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 16));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, PARTNER));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, PARTNER));
     if (mn == 0.0f) mn = 0.0f;                         // -0 is stored as +0
     if (mx == 0.0f) mx = 0.0f;
     const float s32 = __fdiv_rn(__fsub_rn(mx, mn), LEVELS);
@@ -125,46 +167,22 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
     const float sf = __half2float(s16);
     const float inv = sf == 0.0f ? 0.0f : __frcp_rn(sf);
 
-    // r[i] = clamp(rint((x_i - mn) * inv), 0, LEVELS) as a float; the product is never negative
-    float r[32];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        const float2 f = __half22float2(hp[i]);
-        const float v0 = fminf(__fmul_rn(__fsub_rn(f.x, mn), inv), LEVELS);
-        const float v1 = fminf(__fmul_rn(__fsub_rn(f.y, mn), inv), LEVELS);
-        r[2 * i] = __fadd_rn(v0, kRoundMagic);
-        r[2 * i + 1] = __fadd_rn(v1, kRoundMagic);
-    }
+    // code_i = min(rint((x_i - mn) * inv), LEVELS); the product is never negative.  With a normal fp16
+    // scale the quotient exceeds LEVELS by less than 2^-10 LEVELS, so the clamp only matters for
+    // subnormal scales (warp-uniform rare path).
+    constexpr int WORDS = pool_half_bytes(CLS) / 4;
+    uint32_t w[WORDS];
+    const bool tiny = sf != 0.0f && sf < 6.103515625e-05f;
+    if (__any_sync(0xffffffffu, tiny)) pack_codes<CLS, true>(hp, mn, inv, w);
+    else pack_codes<CLS, false>(hp, mn, inv, w);
     if (!active) return;
-    if (CLS == 2) {                                    // the code is the low byte of r's bit pattern
-        uint32_t w[8];
+    if (CLS == 0) {
+        *reinterpret_cast<uint2*>(codes + unit_offset(0, half, 0, t)) = make_uint2(w[0], w[1]);
+    } else {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const uint32_t lo = prmt(__float_as_uint(r[4 * k]), __float_as_uint(r[4 * k + 1]), 0x0040u);
-            const uint32_t hi = prmt(__float_as_uint(r[4 * k + 2]), __float_as_uint(r[4 * k + 3]), 0x0040u);
-            w[k] = prmt(lo, hi, 0x5410u);
-        }
-        *reinterpret_cast<uint4*>(codes + unit_offset(2, half, 0, t)) = make_uint4(w[0], w[1], w[2], w[3]);
-        *reinterpret_cast<uint4*>(codes + unit_offset(2, half, 1, t)) = make_uint4(w[4], w[5], w[6], w[7]);
-    } else {                                           // 16-bit groups summed exactly in fp32
-        constexpr int PER = 16 / BITS;                 // elements per 16-bit group: 8 or 4
-        constexpr int GROUPS = 32 / PER;               // 4 or 8
-        uint32_t g16[GROUPS];
-#pragma unroll
-        for (int g = 0; g < GROUPS; ++g) {
-            float a = 0.f;
-#pragma unroll
-            for (int e = 0; e < PER; ++e) a = fmaf(__fsub_rn(r[g * PER + e], kRoundMagic), (float)(1 << (BITS * e)), a);
-            g16[g] = __float2uint_rn(a);
-        }
-        if (CLS == 0) {
-            *reinterpret_cast<uint2*>(codes + unit_offset(0, half, 0, t)) =
-                make_uint2(g16[0] | (g16[1] << 16), g16[2] | (g16[3] << 16));
-        } else {
-            *reinterpret_cast<uint4*>(codes + unit_offset(1, half, 0, t)) =
-                make_uint4(g16[0] | (g16[1] << 16), g16[2] | (g16[3] << 16), g16[4] | (g16[5] << 16),
-                           g16[6] | (g16[7] << 16));
-        }
+        for (int u = 0; u < WORDS / 4; ++u)
+            *reinterpret_cast<uint4*>(codes + unit_offset(CLS, half, u, t)) =
+                make_uint4(w[4 * u], w[4 * u + 1], w[4 * u + 2], w[4 * u + 3]);
     }
     if (half == 0)
         *reinterpret_cast<uint32_t*>(meta) =
@@ -175,9 +193,11 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
 // MODE 1: one chunk, classes from `bits`; MODE 2: one chunk, classes from the controller.
 // grid = (nchunks, head_groups, batch), block = 256.
 template <int MODE>
-__global__ void __launch_bounds__(kChunkTokens, 2)
+__global__ void __launch_bounds__(kChunkTokens, KVQ_APPEND_MIN_CTAS)
 k_quant_pack(AppendParams p) {
-    extern __shared__ float sW[];
+    extern __shared__ __align__(16) uint8_t dyn_smem[];   // [ring: warps x depth x 4 KB][controller block (MODE 2)]
+    uint8_t* ring_raw = dyn_smem;
+    float* sW = reinterpret_cast<float*>(dyn_smem + kAppendRingBytes);
     __shared__ uint32_t wtot[kChunkTokens / 32][4];
     __shared__ uint32_t base[4];
     __shared__ uint8_t list[4][kChunkTokens];         // tokens of the chunk by class, in slot order
@@ -263,65 +283,182 @@ k_quant_pack(AppendParams p) {
     const int h0 = hg * p.heads_per_group;
     const int nh = min(p.heads_per_group, p.store.kv_heads - h0);
     const int half = lane >> 4, t = lane & 15;
-    // work items (tile tau, head hh), heads fastest, dealt round-robin to the warps
+    // Work items (tile tau, head hh), heads fastest, dealt round-robin to the warps.  The input rows of
+    // the next kAppendDepth items are kept in flight with per-lane 16-byte async copies into a per-warp
+    // ring in shared memory.  For copying, lanes 2j and 2j+1 take adjacent 16-byte pieces (2i, 2i+1) of
+    // the row of slot j, so neighbouring lanes complete a 32-byte sector; each lane then reads the
+    // contiguous half-row it quantizes (pieces 4*half + i of slot lane%16) back from the ring.  A stage
+    // holds [tensor][piece 0..7][slot 0..15] 16-byte pieces, odd pieces rotated by four slots so that
+    // neither access pattern has bank conflicts.
+    struct Item {
+        int k;                                         // class, -1 = no more items
+        bool active;
+        uint32_t tile;
+        int h;
+    };
     uint32_t tau = 0;
     int hh = warp;
-    while (hh >= nh) {
-        hh -= nh;
-        ++tau;
-    }
-    while (tau < pre[4]) {
-        const int k = (tau >= pre[1]) + (tau >= pre[2]) + (tau >= pre[3]);
-        const uint32_t basek = k == 0 ? base[0] : k == 1 ? base[1] : k == 2 ? base[2] : base[3];
-        const uint32_t nk = k == 0 ? ncls[0] : k == 1 ? ncls[1] : k == 2 ? ncls[2] : ncls[3];
-        const uint32_t tile = (k == 0 ? first[0] : k == 1 ? first[1] : k == 2 ? first[2] : first[3]) +
-                              (tau - (k == 0 ? pre[0] : k == 1 ? pre[1] : k == 2 ? pre[2] : pre[3]));
-        const uint32_t r = tile * kTileTokens + t - basek;       // rank of this lane's slot in the chunk (wraps if before)
-        const bool active = r < nk;
-        const int h = h0 + hh;
-        uint4 kraw[4], vraw[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) kraw[i] = vraw[i] = make_uint4(0, 0, 0, 0);
-        if (active) {
-            const int i_tok = list[k][r];
-            const size_t src = (((size_t)b * p.n_new + (size_t)chunk * kChunkTokens + i_tok) * p.store.kv_heads + h) * kHeadDim +
-                               half * (kHeadDim / 2);
-            const uint4* ks = reinterpret_cast<const uint4*>(p.K + src);
-            const uint4* vs = reinterpret_cast<const uint4*>(p.V + src);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) kraw[i] = __ldg(ks + i);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) vraw[i] = __ldg(vs + i);
+    auto settle = [&]() {
+        while (hh >= nh) {
+            hh -= nh;
+            ++tau;
         }
-        uint8_t* rec = p.store.pool[k] + tile_offset(p.store, k, p.layer, b, h, (int)tile);
-        switch (k) {
+    };
+    settle();
+    uint4* my_ring = reinterpret_cast<uint4*>(ring_raw) + (size_t)warp * kAppendDepth * 8 * 32;
+    // describe the next item and start the copies of its rows into ring stage `stage`
+    auto next_item = [&](int stage) {
+        Item it;
+        it.k = -1;
+        it.active = false;
+        it.tile = 0;
+        it.h = 0;
+        if (tau < pre[4]) {
+            const int k = (tau >= pre[1]) + (tau >= pre[2]) + (tau >= pre[3]);
+            const uint32_t basek = k == 0 ? base[0] : k == 1 ? base[1] : k == 2 ? base[2] : base[3];
+            const uint32_t nk = k == 0 ? ncls[0] : k == 1 ? ncls[1] : k == 2 ? ncls[2] : ncls[3];
+            it.k = k;
+            it.tile = (k == 0 ? first[0] : k == 1 ? first[1] : k == 2 ? first[2] : first[3]) +
+                      (tau - (k == 0 ? pre[0] : k == 1 ? pre[1] : k == 2 ? pre[2] : pre[3]));
+            const uint32_t r0 = it.tile * kTileTokens - basek;     // rank of the tile's slot 0 in the chunk (may wrap)
+            it.active = r0 + t < nk;                               // the slot this lane quantizes
+            it.h = h0 + hh;
+            const uint32_t r_ld = r0 + (lane >> 1);                // the slot this lane copies a piece of
+            if (r_ld < nk) {
+                const int i_tok = list[k][r_ld];
+                const size_t src = (((size_t)b * p.n_new + (size_t)chunk * kChunkTokens + i_tok) * p.store.kv_heads + it.h) *
+                                   kHeadDim;
+                const int odd = lane & 1;
+                const uint4* ks = reinterpret_cast<const uint4*>(p.K + src) + odd;
+                const uint4* vs = reinterpret_cast<const uint4*>(p.V + src) + odd;
+                uint4* dst = my_ring + (size_t)stage * 8 * 32 + odd * 16 + (((lane >> 1) + 4 * odd) & 15);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    cp_async16(dst + (2 * i) * 16, ks + 2 * i);            // piece 2i + odd of K
+                    cp_async16(dst + (8 + 2 * i) * 16, vs + 2 * i);        // piece 2i + odd of V
+                }
+            }
+            hh += kChunkTokens / 32;
+            settle();
+        }
+        cp_async_commit();                             // one group per call, possibly empty
+        return it;
+    };
+    Item items[kAppendDepth];
+#pragma unroll
+    for (int d = 0; d < kAppendDepth; ++d) items[d] = next_item(d);
+    int stage = 0;
+    while (items[0].k >= 0) {
+        cp_async_wait<kAppendDepth - 1>();             // this lane's copies of the oldest group have landed
+        __syncwarp();                                  // ... and so have its partner's
+        const Item cur = items[0];
+        uint4 kraw[4], vraw[4];
+        const uint4* src = my_ring + (size_t)stage * 8 * 32 + (4 * half) * 16;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {                  // piece 4*half + i sits at slot (t + 4*(i&1)) % 16
+            const int at = i * 16 + ((t + 4 * (i & 1)) & 15);
+            kraw[i] = cur.active ? src[at] : make_uint4(0, 0, 0, 0);
+            vraw[i] = cur.active ? src[8 * 16 + at] : make_uint4(0, 0, 0, 0);
+        }
+        __syncwarp();                                  // every lane has read the stage before it is refilled
+#pragma unroll
+        for (int d = 0; d + 1 < kAppendDepth; ++d) items[d] = items[d + 1];
+        items[kAppendDepth - 1] = next_item(stage);
+        if (++stage == kAppendDepth) stage = 0;
+
+        uint8_t* rec = p.store.pool[cur.k] + tile_offset(p.store, cur.k, p.layer, b, cur.h, (int)cur.tile);
+        uint8_t* vcodes = rec + pool_codes_bytes(cur.k);
+        const bool active = cur.active;
+        switch (cur.k) {
         case 0:
             quantize_store_half_row<0>(kraw, active, half, t, rec, rec + meta_offset(0, 0, t));
-            quantize_store_half_row<0>(vraw, active, half, t, rec + pool_codes_bytes(0), rec + meta_offset(0, 1, t));
+            quantize_store_half_row<0>(vraw, active, half, t, vcodes, rec + meta_offset(0, 1, t));
             break;
         case 1:
             quantize_store_half_row<1>(kraw, active, half, t, rec, rec + meta_offset(1, 0, t));
-            quantize_store_half_row<1>(vraw, active, half, t, rec + pool_codes_bytes(1), rec + meta_offset(1, 1, t));
+            quantize_store_half_row<1>(vraw, active, half, t, vcodes, rec + meta_offset(1, 1, t));
             break;
         case 2:
             quantize_store_half_row<2>(kraw, active, half, t, rec, rec + meta_offset(2, 0, t));
-            quantize_store_half_row<2>(vraw, active, half, t, rec + pool_codes_bytes(2), rec + meta_offset(2, 1, t));
+            quantize_store_half_row<2>(vraw, active, half, t, vcodes, rec + meta_offset(2, 1, t));
             break;
         default:                                       // fp16: the lane's 64 input bytes are its four units
             if (active) {
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     *reinterpret_cast<uint4*>(rec + unit_offset(3, half, u, t)) = kraw[u];
-                    *reinterpret_cast<uint4*>(rec + pool_codes_bytes(3) + unit_offset(3, half, u, t)) = vraw[u];
+                    *reinterpret_cast<uint4*>(vcodes + unit_offset(3, half, u, t)) = vraw[u];
                 }
             }
             break;
         }
-        hh += kChunkTokens / 32;
-        while (hh >= nh) {
-            hh -= nh;
-            ++tau;
+    }
+    cp_async_wait<0>();
+}
+
+// One new token per sequence (a decode step): grid = (ceil(kv_heads / 16), batch), block = 32.
+// Lane l handles half-row l%2 of KV head 16*blockIdx.x + l/2.  Everything the warp needs (the K and V
+// rows, the pool fills, the features) is requested up front so the loads overlap the controller;
+// the decision is taken by the whole warp (FUSED, hidden width 32) or read from `bits`.
+template <bool FUSED>
+__global__ void __launch_bounds__(32)
+k_append_token(AppendParams p) {
+    const int lane = threadIdx.x, b = blockIdx.y;
+    const int h = blockIdx.x * 16 + (lane >> 1), half = lane & 1;
+    const bool active = h < p.store.kv_heads;
+    uint4 kraw[4], vraw[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) kraw[i] = vraw[i] = make_uint4(0, 0, 0, 0);
+    if (active) {
+        const size_t src = ((size_t)b * p.store.kv_heads + h) * kHeadDim + half * (kHeadDim / 2);
+        const uint4* ks = reinterpret_cast<const uint4*>(p.K + src);
+        const uint4* vs = reinterpret_cast<const uint4*>(p.V + src);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            kraw[i] = __ldg(ks + i);
+            vraw[i] = __ldg(vs + i);
         }
+    }
+    const uint4 fill = *reinterpret_cast<const uint4*>(p.counts_in + (size_t)b * 4);
+    int c;
+    if (FUSED) {
+        const float4 f = reinterpret_cast<const float4*>(p.feats)[b];
+        c = controller_decide_warp32(p.ctrl, f.x, f.y, f.z, f.w, lane);
+    } else {
+        c = class_of_bits(p.bits[b], p.store.flags);
+    }
+    const uint32_t slot = c == 0 ? fill.x : c == 1 ? fill.y : c == 2 ? fill.z : fill.w;
+    if (blockIdx.x == 0 && lane == 0) {
+        p.store.index[((size_t)p.layer * p.store.batch + b) * p.store.max_ctx + p.pos0] = ((uint32_t)c << 30) | slot;
+        *reinterpret_cast<uint4*>(p.counts_out + (size_t)b * 4) =
+            make_uint4(fill.x + (c == 0), fill.y + (c == 1), fill.z + (c == 2), fill.w + (c == 3));
+        if (FUSED && p.bits_out) p.bits_out[b] = (uint8_t)pool_bits(c);
+    }
+    const int t = (int)(slot & (kTileTokens - 1));
+    uint8_t* rec = p.store.pool[c] + tile_offset(p.store, c, p.layer, b, active ? h : 0, (int)(slot / kTileTokens));
+    uint8_t* vcodes = rec + pool_codes_bytes(c);
+    switch (c) {
+    case 0:
+        quantize_store_half_row<0, 1>(kraw, active, half, t, rec, rec + meta_offset(0, 0, t));
+        quantize_store_half_row<0, 1>(vraw, active, half, t, vcodes, rec + meta_offset(0, 1, t));
+        break;
+    case 1:
+        quantize_store_half_row<1, 1>(kraw, active, half, t, rec, rec + meta_offset(1, 0, t));
+        quantize_store_half_row<1, 1>(vraw, active, half, t, vcodes, rec + meta_offset(1, 1, t));
+        break;
+    case 2:
+        quantize_store_half_row<2, 1>(kraw, active, half, t, rec, rec + meta_offset(2, 0, t));
+        quantize_store_half_row<2, 1>(vraw, active, half, t, vcodes, rec + meta_offset(2, 1, t));
+        break;
+    default:
+        if (active) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                *reinterpret_cast<uint4*>(rec + unit_offset(3, half, u, t)) = kraw[u];
+                *reinterpret_cast<uint4*>(vcodes + unit_offset(3, half, u, t)) = vraw[u];
+            }
+        }
+        break;
     }
 }
 

@@ -74,6 +74,54 @@ __device__ __forceinline__ int controller_decide_any(const float* sW, int H, flo
     return controller_decide<0>(sW, H, x0, x1, x2, x3, logits);
 }
 
+// The same decision taken by a whole warp for ONE token, hidden width 32: lane j owns hidden unit j.
+// Every sum still runs in ascending input order with separately rounded products and sums, so the
+// result is bit-identical to controller_decide; the warp only removes the serial walk over the 32 x 32
+// second layer from the critical path of a decode step (one token per sequence).  gW is the
+// parameter block in global memory (row j of W2 and of W3 is read straight into registers).
+// Returns the class in every lane.
+__device__ __forceinline__ int controller_decide_warp32(const float* __restrict__ gW, float x0, float x1, float x2,
+                                                        float x3, int lane) {
+    constexpr int H = 32;
+    const float* W1 = gW;
+    const float* b1 = W1 + 4 * H;
+    const float* W2 = b1 + H;
+    const float* b2 = W2 + H * H;
+    const float* W3 = b2 + H;
+    const float* b3 = W3 + 4 * H;
+    float w2row[H], w3row[H];
+#pragma unroll
+    for (int i = 0; i < H / 4; ++i) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(W2 + lane * H) + i);
+        w2row[4 * i] = v.x; w2row[4 * i + 1] = v.y; w2row[4 * i + 2] = v.z; w2row[4 * i + 3] = v.w;
+        const float4 u = __ldg(reinterpret_cast<const float4*>(W3 + (lane & 3) * H) + i);
+        w3row[4 * i] = u.x; w3row[4 * i + 1] = u.y; w3row[4 * i + 2] = u.z; w3row[4 * i + 3] = u.w;
+    }
+    const float4 w1 = __ldg(reinterpret_cast<const float4*>(W1) + lane);
+    float acc = __ldg(b1 + lane);
+    acc = __fadd_rn(acc, __fmul_rn(w1.x, x0));
+    acc = __fadd_rn(acc, __fmul_rn(w1.y, x1));
+    acc = __fadd_rn(acc, __fmul_rn(w1.z, x2));
+    acc = __fadd_rn(acc, __fmul_rn(w1.w, x3));
+    const float h1 = acc > 0.0f ? acc : 0.0f;
+    acc = __ldg(b2 + lane);
+#pragma unroll
+    for (int i = 0; i < H; ++i) acc = __fadd_rn(acc, __fmul_rn(w2row[i], __shfl_sync(0xffffffffu, h1, i)));
+    const float h2 = acc > 0.0f ? acc : 0.0f;
+    float o = __ldg(b3 + (lane & 3));                  // lanes 0..3 hold the four logits (the others mirror them)
+#pragma unroll
+    for (int j = 0; j < H; ++j) o = __fadd_rn(o, __fmul_rn(w3row[j], __shfl_sync(0xffffffffu, h2, j)));
+    const float o0 = __shfl_sync(0xffffffffu, o, 0), o1 = __shfl_sync(0xffffffffu, o, 1);
+    const float o2 = __shfl_sync(0xffffffffu, o, 2), o3 = __shfl_sync(0xffffffffu, o, 3);
+    if (o0 != o0 || o1 != o1 || o2 != o2 || o3 != o3) return 3;
+    int cls = 0;
+    float best = o0;
+    if (o1 > best) { best = o1; cls = 1; }
+    if (o2 > best) { best = o2; cls = 2; }
+    if (o3 > best) { best = o3; cls = 3; }
+    return cls;
+}
+
 // kvq_select_bits: one thread per token.
 __global__ void __launch_bounds__(128)
 k_select_bits(const float* __restrict__ feats, int n, const float* __restrict__ gW, int H,

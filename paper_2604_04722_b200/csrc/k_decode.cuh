@@ -12,10 +12,12 @@
 // tiles [nt*a0/gw, nt*a1/gw) of EVERY pool of that unit (the same fraction of
 // every pool, hence the same byte and instruction mix for every warp).  Warps
 // are independent: each has its own ring, softmax state and accumulators, and
-// writes one partial (m, l, o[64]) per segment into the slot of its unit; a
-// second kernel merges the slots of a unit.  The launch is persistent when gw
-// is the number of warps resident on the device; nothing in the kernel waits
-// for another warp.
+// writes one partial (m, l, o[64]) per segment into the slot of its unit.  A
+// counter per unit tells a warp whether it delivered the unit's last partial;
+// that warp merges the slots (M = max m_j, l = sum l_j 2^(m_j-M),
+// O = sum o_j 2^(m_j-M) / l), writes the fp16 output row and puts the counter
+// back to zero.  The launch is persistent when gw is the number of warps
+// resident on the device; nothing in the kernel waits for another warp.
 //
 // Data movement: the tiles of a segment are cut into chunks of up to
 // kStageBytes contiguous bytes; every warp runs its own ring of kStages
@@ -92,6 +94,7 @@ struct DecodeParams {
     __half* O;                     // [batch][q_heads][64]
     float* part_o;                 // [units][pslots][64]  unnormalised
     float2* part_ml;               // [units][pslots]      (m in log2 units, l)
+    uint32_t* part_cnt;            // [units] partials delivered so far; zero between launches
     int layer, group;              // group = q_heads / kv_heads
     uint32_t units;                // batch * q_heads
     uint32_t gw;                   // working warps = parts the x axis is cut into
@@ -400,7 +403,7 @@ __device__ __forceinline__ uint32_t scale_by_fraction(uint32_t n, uint32_t a, ui
 
 // grid = ceil(gw / kDecodeWarps), block = kDecodeThreads, dynamic smem = kDecodeSmemBytes.
 __global__ void __launch_bounds__(kDecodeThreads, KVQ_DECODE_MIN_CTAS)
-k_decode_split(DecodeParams P) {
+k_decode_attn(DecodeParams P) {
     extern __shared__ __align__(128) uint8_t ring[];   // [warps][stages][kStageBytes]
     __shared__ WarpScratch scratch[kDecodeWarps];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -585,29 +588,50 @@ k_decode_split(DecodeParams P) {
         // both lanes of a token added its p and p * zero-point: halve the warp sums
         const float l_w = 0.5f * warp_sum(st.l);
         const float b_w = 0.5f * warp_sum(st.bsum);
-        const size_t recno = (size_t)u * P.pslots + (j - decode_first_warp(u, P.units, P.gw));
-        reinterpret_cast<float2*>(P.part_o + recno * kHeadDim)[lane] = make_float2(r2[0] + b_w, r2[1] + b_w);
-        if (lane == 0) P.part_ml[recno] = make_float2(st.m, l_w);
-    }
-}
+        const uint32_t jf = decode_first_warp(u, P.units, P.gw);
+        const size_t rec0 = (size_t)u * P.pslots;
+        reinterpret_cast<float2*>(P.part_o + (rec0 + (j - jf)) * kHeadDim)[lane] = make_float2(r2[0] + b_w, r2[1] + b_w);
+        if (lane == 0) P.part_ml[rec0 + (j - jf)] = make_float2(st.m, l_w);
 
-// Merge the partials of a unit: M = max m_j, l = sum l_j 2^(m_j-M), O = sum o_j 2^(m_j-M) / l.
-// grid = units, block = 64.
-__global__ void __launch_bounds__(kHeadDim)
-k_decode_merge(DecodeParams P) {
-    const uint32_t u = blockIdx.x;
-    const uint32_t n = decode_warps_of_unit(u, P.units, P.gw);
-    const size_t rec0 = (size_t)u * P.pslots;
-    float M = kNegBig;
-    for (uint32_t s = 0; s < n; ++s) M = fmaxf(M, P.part_ml[rec0 + s].x);
-    float L = 0.f, o = 0.f;
-    for (uint32_t s = 0; s < n; ++s) {
-        const float2 ml = P.part_ml[rec0 + s];
-        const float f = fast_exp2(ml.x - M);
-        L = fmaf(ml.y, f, L);
-        o = fmaf(P.part_o[(rec0 + s) * kHeadDim + threadIdx.x], f, o);
+        // ---- the warp that delivers the last partial of the unit merges them
+        const uint32_t n_u = decode_warps_of_unit(u, P.units, P.gw);
+        __threadfence();                               // this warp's partial is visible device-wide ...
+        __syncwarp();
+        uint32_t seen = 0;
+        if (lane == 0) seen = atomicAdd(P.part_cnt + u, 1u);       // ... before it is counted
+        seen = __shfl_sync(0xffffffffu, seen, 0);
+        if (seen + 1 == n_u) {
+            __threadfence();                           // the other warps' partials, counted before ours
+            float M = kNegBig, L = 0.f, o0 = 0.f, o1 = 0.f;
+            for (uint32_t s0 = 0; s0 < n_u; s0 += 32) {            // the running maximum, 32 partials at a time
+                const uint32_t s = s0 + lane;
+                M = fmaxf(M, s < n_u ? __ldcg(&P.part_ml[rec0 + s]).x : kNegBig);
+            }
+            M = warp_max(M);
+            for (uint32_t s0 = 0; s0 < n_u; s0 += 32) {
+                const uint32_t s = s0 + lane;                      // lane s weighs partial s ...
+                const float2 ml = s < n_u ? __ldcg(&P.part_ml[rec0 + s]) : make_float2(kNegBig, 0.f);
+                const float f = fast_exp2(ml.x - M);
+                L += warp_sum(ml.y * f);
+                const uint32_t cnt = min(32u, n_u - s0);
+                for (uint32_t k0 = 0; k0 < cnt; k0 += 8) {         // ... every lane sums its two elements, 8 loads in flight
+                    float2 o[8];
+#pragma unroll
+                    for (uint32_t k = 0; k < 8; ++k)
+                        o[k] = k0 + k < cnt ? __ldcg(reinterpret_cast<const float2*>(P.part_o + (rec0 + s0 + k0 + k) * kHeadDim) + lane)
+                                            : make_float2(0.f, 0.f);
+#pragma unroll
+                    for (uint32_t k = 0; k < 8; ++k) {
+                        const float fk = __shfl_sync(0xffffffffu, f, (k0 + k) & 31);
+                        o0 = fmaf(o[k].x, fk, o0);
+                        o1 = fmaf(o[k].y, fk, o1);
+                    }
+                }
+            }
+            reinterpret_cast<__half2*>(P.O + (size_t)u * kHeadDim)[lane] = __floats2half2_rn(o0 / L, o1 / L);
+            if (lane == 0) P.part_cnt[u] = 0;
+        }
     }
-    P.O[(size_t)u * kHeadDim + threadIdx.x] = __float2half_rn(o / L);
 }
 
 }  // namespace kvq

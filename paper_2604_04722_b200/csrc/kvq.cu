@@ -33,6 +33,7 @@ struct kvq_ctx {
     int hidden = 0;
     float* part_o = nullptr;             // decode scratch [units][partial slots][64]
     float2* part_ml = nullptr;           //                [units][partial slots]
+    uint32_t* part_cnt = nullptr;        //                [units] arrival counters, zero between launches
     int splits_override = 0;
     uint32_t* flags = nullptr;
     // device staging for the host-buffer entry points
@@ -41,7 +42,7 @@ struct kvq_ctx {
     uint8_t* st_bits = nullptr;
     uint8_t* st_export = nullptr;
     bool profiling = false;              // decode timing hooks
-    std::vector<cudaEvent_t> prof_ev;    // 3 events per recorded call
+    std::vector<cudaEvent_t> prof_ev;    // 2 events per recorded call
     int prof_calls = 0;
     uint64_t device_bytes = 0, launches = 0;
     cudaError_t last_err = cudaSuccess;
@@ -90,6 +91,7 @@ void free_all(kvq_ctx* c) {
     cudaFree(c->ctrl);
     cudaFree(c->part_o);
     cudaFree(c->part_ml);
+    cudaFree(c->part_cnt);
     cudaFree(c->flags);
     cudaFree(c->st_feats);
     cudaFree(c->st_K);
@@ -151,15 +153,20 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
 
     const size_t smem = fused ? controller_smem(c->hidden) : 0;
     dim3 grid_q(p.nchunks, groups, c->batch);
-    if (p.nchunks == 1) {
-        if (fused) k_quant_pack<2><<<grid_q, kChunkTokens, smem, st>>>(p);
-        else k_quant_pack<1><<<grid_q, kChunkTokens, 0, st>>>(p);
+    if (n_new == 1 && (!fused || c->hidden == 32)) {                   // a decode step: one warp per 16 heads
+        dim3 grid_t((c->kv_heads + 15) / 16, c->batch);
+        if (fused) k_append_token<true><<<grid_t, 32, 0, st>>>(p);
+        else k_append_token<false><<<grid_t, 32, 0, st>>>(p);
+        c->launches += 1;
+    } else if (p.nchunks == 1) {
+        if (fused) k_quant_pack<2><<<grid_q, kChunkTokens, kAppendRingBytes + smem, st>>>(p);
+        else k_quant_pack<1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
         c->launches += 1;
     } else {
         dim3 grid_c(p.nchunks, c->batch);
         if (fused) k_classify<true><<<grid_c, kChunkTokens, smem, st>>>(p);
         else k_classify<false><<<grid_c, kChunkTokens, 0, st>>>(p);
-        k_quant_pack<0><<<grid_q, kChunkTokens, 0, st>>>(p);
+        k_quant_pack<0><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
         c->launches += 2;
     }
     KVQ_CUDA(c, cudaGetLastError());
@@ -193,14 +200,15 @@ size_t max_partial_records(const kvq_ctx* c) {
 }
 
 // Fill the launch parameters of a decode call and queue split + merge on `st`.
-void fill_decode_params(kvq_ctx* c, int layer, const void* Q, void* O, float* part_o, float2* part_ml, uint32_t gw,
-                        DecodeParams& p) {
+void fill_decode_params(kvq_ctx* c, int layer, const void* Q, void* O, float* part_o, float2* part_ml,
+                        uint32_t* part_cnt, uint32_t gw, DecodeParams& p) {
     p.store = c->store;
     p.counts = counts_of(c, c->cur[layer], layer);
     p.Q = static_cast<const __half*>(Q);
     p.O = static_cast<__half*>(O);
     p.part_o = part_o;
     p.part_ml = part_ml;
+    p.part_cnt = part_cnt;
     p.layer = layer;
     p.group = c->q_heads / c->kv_heads;
     p.units = (uint32_t)c->batch * (uint32_t)c->q_heads;
@@ -278,6 +286,7 @@ int kvq_create(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_di
     ok = ok && dev_alloc(c, &c->ctrl, controller_smem(kMaxHidden)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_o, sizeof(float) * max_partial_records(c) * kHeadDim) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_ml, sizeof(float2) * max_partial_records(c)) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->part_cnt, sizeof(uint32_t) * units) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->flags, sizeof(uint32_t)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_feats, sizeof(float) * 4 * batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_K, sizeof(__half) * (size_t)batch * kv_heads * kHeadDim) == cudaSuccess;
@@ -297,12 +306,16 @@ int kvq_create(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_di
         ok = ok && cudaMemset(s.index, 0, sizeof(uint32_t) * (size_t)layers * batch * max_ctx) == cudaSuccess;
         ok = ok && cudaMemset(c->counts, 0, sizeof(uint32_t) * 2 * (size_t)layers * batch * 4) == cudaSuccess;
         ok = ok && cudaMemset(c->flags, 0, sizeof(uint32_t)) == cudaSuccess;
+        ok = ok && cudaMemset(c->part_cnt, 0, sizeof(uint32_t) * units) == cudaSuccess;
         // the controller block may exceed the default 48 KB of dynamic shared memory
         const int smem_max = (int)controller_smem(kMaxHidden);
         ok = ok && cudaFuncSetAttribute(k_select_bits, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(k_classify<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
-        ok = ok && cudaFuncSetAttribute(k_quant_pack<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
-        ok = ok && cudaFuncSetAttribute(k_decode_split, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        const int ring = (int)kAppendRingBytes;
+        ok = ok && cudaFuncSetAttribute(k_quant_pack<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(k_quant_pack<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(k_quant_pack<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring + smem_max) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(k_decode_attn, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)kDecodeSmemBytes) == cudaSuccess;
         ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     }
@@ -373,19 +386,17 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
     DeviceGuard guard(c->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DecodeParams p{};
-    fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, choose_warps(c, c->len[layer]), p);
+    fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, choose_warps(c, c->len[layer]), p);
     const unsigned grid = (p.gw + kDecodeWarps - 1) / kDecodeWarps;
     const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
-    cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 3] : nullptr;
+    cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 2] : nullptr;
     if (rec) cudaEventRecord(ev[0], st);
-    k_decode_split<<<grid, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
-    if (rec) cudaEventRecord(ev[1], st);
-    k_decode_merge<<<p.units, kHeadDim, 0, st>>>(p);
+    k_decode_attn<<<grid, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
     if (rec) {
-        cudaEventRecord(ev[2], st);
+        cudaEventRecord(ev[1], st);
         c->prof_calls += 1;
     }
-    c->launches += 2;
+    c->launches += 1;
     KVQ_CUDA(c, cudaGetLastError());
     return KVQ_OK;
 }
@@ -396,7 +407,11 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
 // a device address; the address is fetched with cudaGetSymbolAddress once per device (that
 // device current) and passed to the kernels like any other pointer.
 #define KVQ_STATIC_MAX_DEVICES 64
-static __device__ __align__(256) float g_static_partials[(size_t)KVQ_STATIC_MAX_PARTIALS * (kHeadDim + 2)];
+// Layout: [records][64] partial rows, [records] (m, l) pairs, [records / 2] arrival counters (a unit
+// has at least two partial slots).  The counters are zero when the library is loaded and every launch
+// leaves them at zero again.
+static __device__ __align__(256) float g_static_partials[(size_t)KVQ_STATIC_MAX_PARTIALS * (kHeadDim + 2) +
+                                                         KVQ_STATIC_MAX_PARTIALS / 2];
 static float* g_static_partials_addr[KVQ_STATIC_MAX_DEVICES];   // per device, nullptr until looked up
 static std::mutex g_static_partials_lock;
 
@@ -421,10 +436,9 @@ int kvq_decode_attn_static(kvq_ctx* c, int layer, const void* Q, void* O, void* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DecodeParams p{};
     fill_decode_params(c, layer, Q, O, base, reinterpret_cast<float2*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * kHeadDim),
-                       gw, p);
-    k_decode_split<<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
-    k_decode_merge<<<p.units, kHeadDim, 0, st>>>(p);
-    c->launches += 2;
+                       reinterpret_cast<uint32_t*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * (kHeadDim + 2)), gw, p);
+    k_decode_attn<<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    c->launches += 1;
     KVQ_CUDA(c, cudaGetLastError());
     return KVQ_OK;
 }
@@ -536,7 +550,7 @@ int kvq_set_profiling(kvq_ctx* c, int on) {
     if (!c) return KVQ_ERR_ARG;
     DeviceGuard guard(c->device);
     if (on && c->prof_ev.empty()) {
-        c->prof_ev.resize((size_t)kProfMaxCalls * 3);
+        c->prof_ev.resize((size_t)kProfMaxCalls * 2);
         for (size_t i = 0; i < c->prof_ev.size(); ++i) {
             cudaError_t e = cudaEventCreate(&c->prof_ev[i]);
             if (e != cudaSuccess) {
@@ -551,20 +565,17 @@ int kvq_set_profiling(kvq_ctx* c, int on) {
     return KVQ_OK;
 }
 
-int kvq_profile_read(kvq_ctx* c, double* split_ms_total, double* merge_ms_total, int* calls) {
+int kvq_profile_read(kvq_ctx* c, double* attn_ms_total, int* calls) {
     if (!c) return KVQ_ERR_ARG;
     DeviceGuard guard(c->device);
     KVQ_CUDA(c, cudaDeviceSynchronize());
-    double s_ms = 0.0, m_ms = 0.0;
+    double ms = 0.0;
     for (int i = 0; i < c->prof_calls; ++i) {
-        float a = 0.f, b = 0.f;
-        KVQ_CUDA(c, cudaEventElapsedTime(&a, c->prof_ev[(size_t)i * 3], c->prof_ev[(size_t)i * 3 + 1]));
-        KVQ_CUDA(c, cudaEventElapsedTime(&b, c->prof_ev[(size_t)i * 3 + 1], c->prof_ev[(size_t)i * 3 + 2]));
-        s_ms += a;
-        m_ms += b;
+        float a = 0.f;
+        KVQ_CUDA(c, cudaEventElapsedTime(&a, c->prof_ev[(size_t)i * 2], c->prof_ev[(size_t)i * 2 + 1]));
+        ms += a;
     }
-    if (split_ms_total) *split_ms_total = s_ms;
-    if (merge_ms_total) *merge_ms_total = m_ms;
+    if (attn_ms_total) *attn_ms_total = ms;
     if (calls) *calls = c->prof_calls;
     c->prof_calls = 0;
     return KVQ_OK;
