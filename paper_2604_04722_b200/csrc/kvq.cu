@@ -180,9 +180,9 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
 // parts.  Otherwise the count is taken from a small cost model.  A warp should own about eight
 // tiles to pay for its set-up, which bounds the count for small problems.  For large ones the
 // candidates are a persistent launch (as many warps as stay resident; warps whose share crosses a
-// unit border work on two units and finish last, measured at about 0.93 of the ideal) and whole
+// unit border work on two units and finish last, measured at about 0.9 of the ideal) and whole
 // numbers of parts per unit (every warp does the same single piece of work; what counts is how
-// full the last wave of CTAs is, minus a little set-up per wave).
+// full the last wave of CTAs is and how much of a warp's time goes into set-up).
 uint32_t choose_warps(kvq_ctx* c, int len) {
     const uint64_t units = (uint64_t)c->batch * c->q_heads;
     if (c->splits_override > 0) return (uint32_t)(units * (uint64_t)c->splits_override);
@@ -191,13 +191,18 @@ uint32_t choose_warps(kvq_ctx* c, int len) {
     uint64_t cap = tiles / 8;
     if (cap < 1) cap = 1;
     if (cap <= resident) return (uint32_t)(cap >= units ? cap / units * units : cap);
+    // set-up, ring fill and the final reduction cost a warp about as much as fifteen tiles per part
+    // (constants fitted to measured sweeps over the split count on four workload shapes)
+    const double tiles_d = (double)tiles;
     uint64_t best = resident;
-    double best_score = 0.93;
+    const double tpw_p = tiles_d / (double)resident;
+    double best_score = 0.90 * tpw_p / (tpw_p + 25.0);           // some warps work on two parts
     for (uint64_t s = 1; s <= (uint64_t)kMaxSplits && units * s <= cap; ++s) {
         const double fill = (double)(units * s) / (double)resident;
         const double waves = (double)(uint64_t)(fill + 0.999999);
         if (waves > 8.0) break;
-        const double score = fill / waves - 0.01 * waves;
+        const double tpw = tiles_d / (double)(units * s);
+        const double score = fill / waves * tpw / (tpw + 15.0);
         if (score > best_score + 1e-9) {
             best_score = score;
             best = units * s;
