@@ -292,12 +292,27 @@ struct Quantized {
             }
         }
     }
-    __device__ static __forceinline__ void tile(const uint8_t* rec, bool valid, int half, int t,
+    // The K half-row and K meta word of a tile, fetched from shared memory one tile ahead of their use.
+    struct KIn {
+        uint32_t w[WORDS];
+        uint32_t meta;
+    };
+    __device__ static __forceinline__ KIn load_k(const uint8_t* rec, int half, int t) {
+        KIn k;
+        load_half_row(rec, half, t, k.w);
+        k.meta = *reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 0, t));
+        return k;
+    }
+    __device__ static __forceinline__ void tile(const uint8_t* rec, const KIn& kin, bool valid, int half, int t,
                                                 const uint32_t (&qreg)[kQRegs], const QueryInfo& qi, Softmax& st,
                                                 float (&acc)[kHalfDim]) {
         uint32_t w[WORDS];
-        load_half_row(rec, half, t, w);
-        const float2 km = meta_to_float2(*reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 0, t)));
+#pragma unroll
+        for (int i = 0; i < WORDS; ++i) w[i] = kin.w[i];
+        const float2 km = meta_to_float2(kin.meta);
+        uint32_t wv_codes[WORDS];                      // the V side's inputs are requested before the K arithmetic
+        load_half_row(rec + pool_codes_bytes(CLS), half, t, wv_codes);
+        const uint32_t vmeta = *reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 1, t));
         int dh[PLANES], dl[PLANES];
 #pragma unroll
         for (int k = 0; k < PLANES; ++k) dh[k] = dl[k] = 0;
@@ -322,8 +337,9 @@ struct Quantized {
         y = valid ? y : -INFINITY;
         const float p = softmax_step(st, acc, y);
 
-        load_half_row(rec + pool_codes_bytes(CLS), half, t, w);
-        const float2 vm = meta_to_float2(*reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 1, t)));
+#pragma unroll
+        for (int i = 0; i < WORDS; ++i) w[i] = wv_codes[i];
+        const float2 vm = meta_to_float2(vmeta);
         const float wv = (p * vm.x) * pow2f(100);
         st.bsum = fmaf(p, vm.y, st.bsum);
 #pragma unroll
@@ -346,7 +362,9 @@ struct Fp16Rows {
         for (int i = 0; i < kHalfDim; ++i) qreg[i] = __float_as_uint(qi.q_half[i] * kLogitScale);
     }
     __device__ static __forceinline__ void leave(float (&)[kHalfDim]) {}
-    __device__ static __forceinline__ void tile(const uint8_t* rec, bool valid, int half, int t,
+    struct KIn {};                                     // fp16 rows are read where they are used
+    __device__ static __forceinline__ KIn load_k(const uint8_t*, int, int) { return KIn{}; }
+    __device__ static __forceinline__ void tile(const uint8_t* rec, const KIn&, bool valid, int half, int t,
                                                 const uint32_t (&qreg)[kQRegs], const QueryInfo&, Softmax& st,
                                                 float (&acc)[kHalfDim]) {
         float d[4] = {0.f, 0.f, 0.f, 0.f};
@@ -519,9 +537,13 @@ k_decode_attn(DecodeParams P) {
                 }
                 const int ntiles = min(tiles_per_stage(CLS), hi - tile0);
                 const uint8_t* buf = my_ring + (size_t)cslot * kStageBytes;
+                typename C::KIn kin = C::load_k(buf, half, t);
                 for (int i = 0; i < ntiles; ++i) {
                     const bool valid = (uint32_t)((tile0 + i) * kTileTokens + t) < cnt;
-                    C::tile(buf + (size_t)i * C::REC, valid, half, t, qreg, qi, st, acc);
+                    // the next tile's K side (the last tile fetches itself again)
+                    const typename C::KIn knext = C::load_k(buf + (size_t)min(i + 1, ntiles - 1) * C::REC, half, t);
+                    C::tile(buf + (size_t)i * C::REC, kin, valid, half, t, qreg, qi, st, acc);
+                    kin = knext;
                 }
                 tile0 += ntiles;
                 --in_flight;
