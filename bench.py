@@ -159,7 +159,7 @@ def oracle_leg(wl, seqs, steps, warmup):
         "value": float(np.sum(nbytes)) / total_t / 1e9,
         "ms_per_step": 1e3 * total_t / len(times),
         "cores": oracle.num_threads(),
-        "sample": "%d of %d sequences of cfg5 (whole sequences, all 32 heads, context %d); %d steps; "
+        "sample": "%d of %d sequences of the workload (whole sequences, every head, one layer, context %d); %d steps; "
                   "prefill quantize-append of the sample took %.1f s (%.0f tokens/s)" % (
                       nb, wl.batch, wl.context, len(times), prefill_s, nb * wl.context / prefill_s),
         "append_prefill_tokens_per_s": nb * wl.context / prefill_s,
@@ -184,13 +184,34 @@ def run_reference(args, wl):
     print(json.dumps(line))
 
 
-def workload_config(wl):
-    return {"workload": "%s stress: 1 SmolLM-1.7B-shaped layer, 32 q / 32 kv heads, head_dim 64, batch %d, "
-                        "context %d, bits iid {2:.50,4:.30,8:.15,16:.05} seed 0; each step appends 1 "
-                        "controller-decided token per sequence and attends" % (wl.name, wl.batch, wl.context),
-            "layers": wl.layers, "batch": wl.batch, "q_heads": wl.q_heads, "kv_heads": wl.kv_heads,
-            "head_dim": wl.head_dim, "context": wl.context,
-            "l2": "inputs larger than L2 (about 1.25 GB of packed KV is streamed per step; L2 is 126 MB)"}
+WORKLOAD_TEXT = {
+    "cfg1": "SmolLM-135M-shaped single layer, 9 q / 3 kv heads, batch 1, context 512, bits iid {2:.40,4:.35,8:.20,16:.05}",
+    "cfg2": "SmolLM-135M-shaped full cache, 30 layers, 9 q / 3 kv heads, batch 1, context 2048, controller bits",
+    "cfg3": "SmolLM-360M-shaped, 32 layers, 15 q / 5 kv heads, batch 8, context 4096, controller bits",
+    "cfg4": "SmolLM-1.7B-shaped, 24 layers, 32 q / 32 kv heads, batch 16, context 8192, bits in geometric runs "
+            "{2:.25,4:.40,8:.25,16:.10} (or uniform with --uniform-bits)",
+    "cfg5": "stress: 1 SmolLM-1.7B-shaped layer, 32 q / 32 kv heads, batch 16, context 32768, bits iid "
+            "{2:.50,4:.30,8:.15,16:.05} seed 0",
+}
+
+
+def workload_config(wl, cold=None, kv_bytes_all_layers=None):
+    base = wl.name.split("-")[0]
+    cfg = {"workload": "%s: %s; head_dim 64; each step appends 1 controller-decided token per sequence to every "
+                       "layer and attends (this run: batch %d, context %d)" % (
+                           wl.name, WORKLOAD_TEXT.get(base, base), wl.batch, wl.context),
+           "layers": wl.layers, "batch": wl.batch, "q_heads": wl.q_heads, "kv_heads": wl.kv_heads,
+           "head_dim": wl.head_dim, "context": wl.context}
+    if cold is None:
+        cfg["l2"] = "inputs larger than L2 (126 MB) for cfg4/cfg5; smaller workloads flush L2 between timed steps"
+    elif cold:
+        cfg["l2"] = ("L2 flushed between timed steps (a 256 MB buffer is overwritten outside the timed region): the "
+                     "packed KV of all layers is %.1f MB, it would stay resident in the 126 MB L2" % (
+                         kv_bytes_all_layers / 1e6))
+    else:
+        cfg["l2"] = "inputs larger than L2 (%.2f GB of packed KV is streamed per step; L2 is 126 MB)" % (
+            kv_bytes_all_layers / 1e9)
+    return cfg
 
 
 def run_ours(args, wl):
@@ -217,24 +238,33 @@ def run_ours(args, wl):
 
     W, K_steps = args.warmup, args.steps
     e2e_steps, e2e_warm = K_steps, max(3, W)
-    total_steps = W + K_steps + e2e_warm + e2e_steps
-    B, Hq, Hkv, D, ctx_len = wl.batch, wl.q_heads, wl.kv_heads, wl.head_dim, wl.context
+    total_steps = W + 2 * K_steps + e2e_warm + e2e_steps      # the flushed-L2 mode times its steps twice
+    L, B, Hq, Hkv, D, ctx_len = wl.layers, wl.batch, wl.q_heads, wl.kv_heads, wl.head_dim, wl.context
     seed = wl.seed + 1000 * rank                      # replicas draw their own data
     cw = synth.controller_weights(wl.mlp_seed, wl.hidden)
 
+    # Every layer is filled with the same seeded K/V block (layer 0's): drawing 24 layers of cfg4 on the
+    # host would take minutes and changes nothing the kernels see.
     t_gen = time.perf_counter()
     K, V = synth.kv_batch(seed, 0, B, 0, ctx_len, Hkv)
-    bits = np.stack([synth.bits_iid(seed, b, 0, ctx_len, wl.mix) for b in range(B)])
     feats_prefill = synth.features_batch(seed, B, 0, ctx_len)
+    if args.uniform_bits:
+        bits = np.full((B, ctx_len), args.uniform_bits, np.uint8)
+    elif wl.bits_mode == "controller":
+        bits = None                                   # decided on the device from the features
+    else:
+        wl_seeded = dataclasses.replace(wl, seed=seed)
+        bits = np.stack([synth.workload_bits(wl_seeded, b, 0, ctx_len) for b in range(B)])
     t_gen = time.perf_counter() - t_gen
 
     def to_dev(a, dt):
         return torch.from_numpy(np.ascontiguousarray(a).view(dt)).to(dev)
 
-    ctx = kq.kvq_create(1, Hq, Hkv, D, ctx_len + total_steps, B)
+    ctx = kq.kvq_create(L, Hq, Hkv, D, ctx_len + total_steps, B)
     kq.kvq_set_controller(ctx, cw.hidden, *cw.as_tuple())
     Kd, Vd = to_dev(K, np.int16), to_dev(V, np.int16)
-    bits_d, feats_d = to_dev(bits, np.uint8), to_dev(feats_prefill, np.float32)
+    feats_d = to_dev(feats_prefill, np.float32)
+    bits_d = to_dev(bits, np.uint8) if bits is not None else None
     stream = torch.cuda.current_stream().cuda_stream
 
     def timed(fn, reps):
@@ -247,7 +277,7 @@ def run_ours(args, wl):
         torch.cuda.synchronize()
         return ev0.elapsed_time(ev1) / reps
 
-    # ---- prefill quantize-append, phase (i): bits decided by the controller inside the launch
+    # ---- prefill quantize-append of one layer, timed both ways (kvq_reset empties every layer)
     launches0 = kq.kvq_launch_count(ctx)
     ctl_bits = torch.zeros((B, ctx_len), dtype=torch.uint8, device=dev)
 
@@ -259,8 +289,10 @@ def run_ours(args, wl):
     ms_prefill_fused = timed(prefill_fused, 3)
     ctl_hist = {int(b): int((ctl_bits == b).sum().item()) for b in (2, 4, 8, 16)}
     ctl_written = sum(ROW_BYTES[b] * n for b, n in ctl_hist.items()) * Hkv
+    if bits_d is None:                                # controller workloads keep the controller's decisions
+        bits_d = ctl_bits
+        bits = ctl_bits.cpu().numpy()
 
-    # ---- phase (ii): the stated i.i.d. mix, which the decode steps then read
     def prefill_given():
         kq.kvq_reset(ctx)
         kq.kvq_append(ctx, 0, Kd, Vd, bits_d, ctx_len)
@@ -268,10 +300,13 @@ def run_ours(args, wl):
     ms_prefill_given = timed(prefill_given, 3)
     given_hist = {int(b): int((bits == b).sum()) for b in (2, 4, 8, 16)}
     given_written = sum(ROW_BYTES[b] * n for b, n in given_hist.items()) * Hkv
+    for layer in range(1, L):                         # the other layers get the same tokens (untimed)
+        kq.kvq_append(ctx, layer, Kd, Vd, bits_d, ctx_len)
+    torch.cuda.synchronize()
     del Kd, Vd, feats_d
     torch.cuda.empty_cache()
 
-    # ---- per-step inputs, resident on the device
+    # ---- per-step inputs, resident on the device (shared by the layers)
     f_steps = np.stack([synth.features_batch(seed, B, ctx_len + s, 1) for s in range(total_steps)])   # [S][B][1][4]
     kv_steps = [synth.kv_batch(seed, 0, B, ctx_len + s, 1, Hkv) for s in range(total_steps)]
     k_steps = np.stack([kv[0] for kv in kv_steps])
@@ -286,9 +321,14 @@ def run_ours(args, wl):
 
     def one_step():
         s = step_no[0]
-        kq.kvq_append_fused(ctx, 0, k_d[s], v_d[s], f_d[s], 1, step_bits_d[s], stream)
-        kq.kvq_decode_attn(ctx, 0, q_d[s], O_d, stream)
+        for layer in range(L):
+            kq.kvq_append_fused(ctx, layer, k_d[s], v_d[s], f_d[s], 1, step_bits_d[s], stream)
+            kq.kvq_decode_attn(ctx, layer, q_d[s], O_d, stream)
         step_no[0] = s + 1
+
+    _, resident_layer0, _ = kq.kvq_stats(ctx, 0, B)
+    cold = L * resident_layer0 < 2 * 126e6            # the whole cache would sit in L2: flush it between steps
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if cold else None
 
     for _ in range(W):
         one_step()
@@ -303,24 +343,43 @@ def run_ours(args, wl):
     if dist is not None:
         dist.barrier()
     launches1 = kq.kvq_launch_count(ctx)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    ev0.record()
-    for _ in range(K_steps):
-        one_step()
-    ev1.record()
-    torch.cuda.synchronize()
+    attn_ms, ncalls = 0.0, 0
+    if cold:
+        # one pair of events per step; the flush runs between the pairs, outside the timed regions
+        ms_total = 0.0
+        for _ in range(K_steps):
+            flush_buf.fill_(step_no[0] & 0xff)
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            ev0.record()
+            one_step()
+            ev1.record()
+            torch.cuda.synchronize()
+            ms_total += ev0.elapsed_time(ev1)
+            a_ms, n = kq.kvq_profile_read(ctx)
+            attn_ms, ncalls = attn_ms + a_ms, ncalls + n
+        ms_warm = timed(one_step, K_steps)            # the same steps again with whatever stays in L2
+        kq.kvq_profile_read(ctx)
+    else:
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        ev0.record()
+        for _ in range(K_steps):
+            one_step()
+        ev1.record()
+        torch.cuda.synchronize()
+        ms_total = ev0.elapsed_time(ev1)
+        attn_ms, ncalls = kq.kvq_profile_read(ctx)
+        ms_warm = None
     if dist is not None:
         dist.barrier()
-    ms_total = ev0.elapsed_time(ev1)
-    launches_timed = kq.kvq_launch_count(ctx) - launches1
-    attn_ms, ncalls = kq.kvq_profile_read(ctx)
+    launches_timed = (kq.kvq_launch_count(ctx) - launches1) // (2 if cold else 1)
     kq.kvq_set_profiling(ctx, False)
     time.sleep(0.2)
     clocks = sampler.stop()
     _, resident1, ebits = kq.kvq_stats(ctx, 0, B)
-    resident_mean = 0.5 * (resident0 + resident1)
-    new_rows_mean = (resident1 - resident0) / K_steps
+    resident_mean = 0.5 * (resident0 + resident1)     # per layer
+    new_rows_mean = (resident1 - resident0) / max(1, step_no[0] - W)
 
     # ---- end to end through the host-buffer entry point (pinned buffers, copies timed)
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
@@ -330,8 +389,9 @@ def run_ours(args, wl):
 
     def one_step_host():
         s = step_no[0]
-        kq.kvq_decode_step_host(ctx, 0, f_h[s].data_ptr(), k_h[s].data_ptr(), v_h[s].data_ptr(), q_h[s].data_ptr(),
-                                O_h.data_ptr(), None, stream)
+        for layer in range(L):
+            kq.kvq_decode_step_host(ctx, layer, f_h[s].data_ptr(), k_h[s].data_ptr(), v_h[s].data_ptr(),
+                                    q_h[s].data_ptr(), O_h.data_ptr(), None, stream)
         step_no[0] = s + 1
 
     for _ in range(e2e_warm):
@@ -341,8 +401,8 @@ def run_ours(args, wl):
     ms_e2e = timed(one_step_host, e2e_steps)
     if dist is not None:
         dist.barrier()
-    h2d = B * 16 + 2 * B * Hkv * D * 2 + B * Hq * D * 2
-    d2h = B * Hq * D * 2
+    h2d = L * (B * 16 + 2 * B * Hkv * D * 2 + B * Hq * D * 2)
+    d2h = L * B * Hq * D * 2
 
     # ---- reduce over ranks: slowest rank's time, summed bytes
     ms_step = ms_total / K_steps
@@ -351,45 +411,51 @@ def run_ours(args, wl):
         dist.all_reduce(vals, op=dist.ReduceOp.MAX)
     ms_step, ms_e2e, ms_attn = [float(x) for x in vals.tolist()]
 
-    dec_bytes, app_bytes = step_bytes(wl, ctx_len, resident_mean, new_rows_mean)
-    bytes_step = dec_bytes + app_bytes
+    dec_bytes, app_bytes = step_bytes(wl, ctx_len, resident_mean, new_rows_mean)    # per layer
+    bytes_step = L * (dec_bytes + app_bytes)
     peak, peak_kind = measured_peak_gbs()
     achieved = dec_bytes / (ms_attn * 1e-3) / 1e9
     index_bytes = B * (ctx_len + W + K_steps / 2) * 4
+    is_headline = wl.name == "cfg5" and not args.uniform_bits
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and is_headline:
         leg = oracle_leg(wl, [0, 1], 20, 1)
         cpu = {"value": leg["value"], "unit": UNIT, "cores": leg["cores"], "kind": "oracle", "sample": leg["sample"],
                "ms_per_step_of_sample": leg["ms_per_step"],
                "append_prefill_tokens_per_s": leg["append_prefill_tokens_per_s"]}
 
     if rank == 0:
+        cfg = workload_config(wl, cold, L * resident_mean)
+        if args.uniform_bits:
+            cfg["uniform_bits"] = args.uniform_bits
         line = {
             "metric": METRIC, "value": world * bytes_step / (ms_step * 1e-3) / 1e9, "unit": UNIT,
             "n_gpus": world, "steps": K_steps, "warmup": W, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(wl),
+            "config": cfg,
             "clocks": clocks,
             "e2e": {"value": world * bytes_step / (ms_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms_e2e,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches_timed),
             "roofline": {"bound": "hbm", "kernel": "k_decode_attn", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": "of " + peak_kind,
-                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "algorithmic_bytes_per_launch": dec_bytes,
+                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if is_headline and B == 16 and ctx_len == 32768 else None,
+                         "algorithmic_bytes_per_launch": dec_bytes,
                          "avg_launch_us": ms_attn * 1e3,
                          "frac_with_index_bytes": (dec_bytes + index_bytes) / (ms_attn * 1e-3) / 1e9 / peak},
             "cpu_baseline": cpu,
-            "decode_attn_us_per_step": ms_attn * 1e3,
+            "decode_attn_us_per_layer": ms_attn * 1e3,
             "step_us": ms_step * 1e3,
+            "step_us_warm_l2": None if ms_warm is None else ms_warm * 1e3,
             "append_prefill_tokens_per_s": {
                 "controller_fused": B * ctx_len / (ms_prefill_fused * 1e-3),
                 "bits_given": B * ctx_len / (ms_prefill_given * 1e-3),
                 "ms_fused": ms_prefill_fused, "ms_bits_given": ms_prefill_given,
                 "GBps_fused": (B * ctx_len * Hkv * 256 + ctl_written) / (ms_prefill_fused * 1e-3) / 1e9,
                 "GBps_bits_given": (B * ctx_len * Hkv * 256 + given_written) / (ms_prefill_given * 1e-3) / 1e9,
-                "controller_class_histogram": ctl_hist},
-            "kv_bytes_per_step": dec_bytes, "expected_bits": ebits,
+                "controller_class_histogram": ctl_hist, "note": "one layer"},
+            "kv_bytes_per_layer": dec_bytes, "expected_bits": ebits,
             "device_bytes": kq.kvq_device_bytes(ctx), "input_generation_s": t_gen,
         }
         print(json.dumps(line))
@@ -408,12 +474,16 @@ def main():
     ap.add_argument("--context", type=int, default=0,
                     help="shorter cached context than the workload's 32768, for profiler captures that must "
                          "stay small; the printed config names it and the line is not a benchmark result")
+    ap.add_argument("--workload", choices=sorted(synth.CONFIGS), default="cfg5",
+                    help="cfg5 (default) is the workload the metric is quoted on; the others are reported in DESIGN.md")
+    ap.add_argument("--uniform-bits", type=int, choices=[2, 4, 8, 16], default=0,
+                    help="store every prefill token at this precision (the static baselines of cfg4)")
     ap.add_argument("--batch", type=int, default=0,
                     help="fewer sequences than the workload's 16, likewise for profiler captures only")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    wl = synth.CONFIGS["cfg5"]
+    wl = synth.CONFIGS[args.workload]
     if args.context > 0:
         wl = dataclasses.replace(wl, context=args.context, name="%s-context-%d" % (wl.name, args.context))
     if args.batch > 0:
