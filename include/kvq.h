@@ -66,14 +66,35 @@ typedef struct kvq_ctx kvq_ctx;    /* opaque; owned by the library */
  * Create a cache for `layers` layers, `batch` sequences, `q_heads` query heads
  * sharing `kv_heads` KV heads (q_heads % kv_heads == 0; query head h reads KV
  * head h / (q_heads/kv_heads)), head_dim == 64, up to `max_ctx` tokens per
- * sequence (Eq. 4: the cache that decode steps append to).  Allocates every
- * pool at its worst-case size on the current device (504 bytes per token, KV
- * head and layer) plus index, counters and split-attention scratch, and zeroes
+ * sequence (Eq. 4: the cache that decode steps append to).  Allocates the
+ * arena of packed rows at its worst-case size on the current device (about 504
+ * bytes per token, KV head and layer: every token could take any precision)
+ * plus block tables, index, counters and split-attention scratch, and zeroes
  * them.  *out receives the handle.  KVQ_ERR_ARG for unsupported shapes,
  * KVQ_ERR_NOMEM / KVQ_ERR_CUDA if allocation fails (nothing is leaked).
  */
 int kvq_create(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim,
                int max_ctx, int batch);
+
+/*
+ * The same with a chosen budget for the packed rows.  The rows live in an arena of 64 KB
+ * blocks; a block serves one (layer, sequence, KV head, precision) stream and is taken from
+ * the arena when an append first reaches it, so the memory in use is the sum of the stored row
+ * bytes (40 / 72 / 136 / 256 per token and KV head, against 256 for an fp16 cache) plus at most
+ * one partly filled block per stream -- the footprint reduction the paper's abstract claims,
+ * measurable with kvq_arena_usage.  arena_bytes is rounded down to whole blocks; 0 means the
+ * worst case (what kvq_create takes).  An append that finds the arena exhausted stores nothing
+ * for the tokens that did not fit, sets the device flag KVQ_FLAG_ARENA_FULL (see
+ * kvq_device_status) and leaves the cache unusable until kvq_reset.
+ */
+int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim,
+                     int max_ctx, int batch, uint64_t arena_bytes);
+
+/*
+ * Arena fill: blocks handed out so far, blocks available, bytes per block (host uint64, any
+ * may be NULL).  Synchronizes.
+ */
+int kvq_arena_usage(kvq_ctx* ctx, uint64_t* blocks_in_use, uint64_t* blocks_total, uint64_t* block_bytes);
 
 /* Free everything the handle owns.  NULL is a no-op.  Synchronizes the device. */
 int kvq_destroy(kvq_ctx* ctx);
@@ -177,7 +198,7 @@ int kvq_decode_step_host(kvq_ctx* ctx, int layer, const float* feats, const void
                          const void* V, const void* Q, void* O, uint8_t* bits_out_opt,
                          void* stream);
 
-/* Forget all cached tokens of every layer (pools keep their bytes, counters go to 0). */
+/* Forget all cached tokens of every layer (counters go to 0, every arena block is free again). */
 int kvq_reset(kvq_ctx* ctx, void* stream);
 
 /* Tokens cached per sequence in `layer` (host-side mirror; no device access). */
@@ -235,6 +256,7 @@ int kvq_profile_read(kvq_ctx* ctx, double* attn_ms_total, int* calls);
 
 /* Device flags recorded by kernels since the last call (host uint32, cleared on read). */
 #define KVQ_FLAG_BAD_BITS 1u      /* a bit-width outside {2,4,8,16} was appended (stored as fp16) */
+#define KVQ_FLAG_ARENA_FULL 4u    /* an append ran out of arena blocks; the tokens that did not fit are lost */
 #define KVQ_FLAG_WAIT_TIMEOUT 2u  /* a bounded wait on an async copy expired in kvq_decode_attn; that
                                      call's output is invalid */
 int kvq_device_status(kvq_ctx* ctx, uint32_t* host_flags_out);

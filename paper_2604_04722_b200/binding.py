@@ -32,6 +32,8 @@ _vp, _i, _u64p = C.c_void_p, C.c_int, C.POINTER(C.c_uint64)
 # name -> (restype, argtypes); mirrors include/kvq.h one to one
 SIGNATURES = {
     "kvq_create": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i]),
+    "kvq_create_arena": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, C.c_uint64]),
+    "kvq_arena_usage": (_i, [_vp, _u64p, _u64p, _u64p]),
     "kvq_destroy": (_i, [_vp]),
     "kvq_set_controller": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvq_select_bits": (_i, [_vp, _vp, _i, _vp, _vp, _vp]),
@@ -111,6 +113,21 @@ def kvq_create(layers: int, q_heads: int, kv_heads: int, head_dim: int, max_ctx:
     h = _vp()
     check(lib().kvq_create(C.byref(h), layers, q_heads, kv_heads, head_dim, max_ctx, batch), "kvq_create")
     return h.value
+
+
+def kvq_create_arena(layers: int, q_heads: int, kv_heads: int, head_dim: int, max_ctx: int, batch: int,
+                     arena_bytes: int) -> int:
+    h = _vp()
+    check(lib().kvq_create_arena(C.byref(h), layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes),
+          "kvq_create_arena")
+    return h.value
+
+
+def kvq_arena_usage(ctx: int):
+    """Returns (blocks_in_use, blocks_total, block_bytes)."""
+    a, b, c = C.c_uint64(), C.c_uint64(), C.c_uint64()
+    check(lib().kvq_arena_usage(ctx, C.byref(a), C.byref(b), C.byref(c)), "kvq_arena_usage")
+    return a.value, b.value, c.value
 
 
 def kvq_destroy(ctx: int) -> None:

@@ -144,8 +144,11 @@ __device__ __forceinline__ void pack_codes(const __half2* hp, float mn, float in
 // class CLS < 3 and store it: the lane's units of the tile's code block `codes`, and (half 0 only)
 // the {scale, zero-point} word at `meta`.  Both lanes of a slot (l, l ^ 16) must call together.
 // PARTNER: lane distance (xor) to the lane that holds the other half of the same row.
+// `tail`: the lane's slot lies beyond the stream's fill (it will be written by a later append); its
+// {scale, zero-point} word is cleared so that a reader, which gives such a slot weight zero, never
+// multiplies that zero with whatever a recycled block held before.
 template <int CLS, int PARTNER = 16>
-__device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], bool active, int half, int t,
+__device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], bool active, bool tail, int half, int t,
                                                         uint8_t* codes, uint8_t* meta) {
     constexpr int BITS = pool_bits(CLS);
     constexpr float LEVELS = (float)((1 << BITS) - 1);
@@ -175,7 +178,10 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
     const bool tiny = sf != 0.0f && sf < 6.103515625e-05f;
     if (__any_sync(0xffffffffu, tiny)) pack_codes<CLS, true>(hp, mn, inv, w);
     else pack_codes<CLS, false>(hp, mn, inv, w);
-    if (!active) return;
+    if (!active) {
+        if (tail && half == 0) *reinterpret_cast<uint32_t*>(meta) = 0u;
+        return;
+    }
     if (CLS == 0) {
         *reinterpret_cast<uint2*>(codes + unit_offset(0, half, 0, t)) = make_uint2(w[0], w[1]);
     } else {
@@ -187,6 +193,39 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
     if (half == 0)
         *reinterpret_cast<uint32_t*>(meta) =
             (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(__float2half_rn(mn)) << 16);
+}
+
+// Reserve the blocks that class c of the streams (layer, b, heads h0 .. h0+nh) grows into when its fill
+// goes from n_old to n_new tokens.  Called by one warp; the new table entries are visible to the
+// CTA after its next barrier and to later launches.
+__device__ __forceinline__ void reserve_blocks(const StoreView& s, int c, int layer, int b, int h0, int nh,
+                                               uint32_t n_old, uint32_t n_new, int lane) {
+    const uint32_t have = blocks_for(c, n_old), want = blocks_for(c, n_new);
+    if (want == have) return;
+    const uint32_t per = want - have;
+    uint32_t first = 0;
+    if (lane == 0) first = arena_take(s, per * (uint32_t)nh);
+    first = __shfl_sync(0xffffffffu, first, 0);
+    for (uint32_t i = lane; i < per * (uint32_t)nh; i += 32) {
+        const uint32_t hh = i / per, j = i - hh * per;
+        stream_table(s, c, layer, b, h0 + (int)hh)[have + j] = first ? first + i : 0u;
+    }
+}
+
+// Launch between k_classify and k_quant_pack<0> (several chunks per sequence): reserve the blocks every
+// stream of the layer grows into.  grid = batch, block = 128 (warp c handles class c).
+__global__ void __launch_bounds__(128)
+k_reserve_blocks(AppendParams p) {
+    const int b = blockIdx.x, c = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint32_t add = 0;
+    for (int cc = lane; cc < p.nchunks; cc += 32) {
+        const uint4 v = p.hist[(size_t)b * p.nchunks + cc];
+        add += c == 0 ? v.x : c == 1 ? v.y : c == 2 ? v.z : v.w;
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) add += __shfl_xor_sync(0xffffffffu, add, d);
+    const uint32_t n_old = p.counts_in[(size_t)b * 4 + c];
+    reserve_blocks(p.store, c, p.layer, b, 0, p.store.kv_heads, n_old, n_old + add, lane);
 }
 
 // Launch 2.  MODE 0: classes come from k_classify (several chunks per sequence);
@@ -269,6 +308,13 @@ k_quant_pack(AppendParams p) {
     }
     if (hg == 0 && chunk == p.nchunks - 1 && threadIdx.x < 4)
         p.counts_out[(size_t)b * 4 + threadIdx.x] = base[threadIdx.x] + ncls[threadIdx.x];
+    const int h0 = hg * p.heads_per_group;
+    const int nh = min(p.heads_per_group, p.store.kv_heads - h0);
+    if (MODE != 0) {
+        // One chunk per sequence: this CTA is the only one that writes the streams of its heads, so it
+        // reserves the blocks they grow into itself (with several chunks k_reserve_blocks did it before).
+        if (warp < kNumPools) reserve_blocks(p.store, warp, p.layer, b, h0, nh, base[warp], base[warp] + ncls[warp], lane);
+    }
     __syncthreads();
 
     // ---- tiles: class k touches tiles [first[k], first[k] + nt[k]) of its pool
@@ -277,11 +323,12 @@ k_quant_pack(AppendParams p) {
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
         first[k] = base[k] / kTileTokens;
-        const uint32_t nt = ncls[k] ? (base[k] + ncls[k] - 1) / kTileTokens - first[k] + 1 : 0;
+        uint32_t nt = ncls[k] ? (base[k] + ncls[k] - 1) / kTileTokens - first[k] + 1 : 0;
+        // The append's last chunk also visits the partly filled last tile of a class that got no token in
+        // this chunk, only to clear the {scale, zero-point} words of its unused slots (see `tail`).
+        if (ncls[k] == 0 && chunk == p.nchunks - 1 && base[k] % kTileTokens != 0) nt = 1;
         pre[k + 1] = pre[k] + nt;
     }
-    const int h0 = hg * p.heads_per_group;
-    const int nh = min(p.heads_per_group, p.store.kv_heads - h0);
     const int half = lane >> 4, t = lane & 15;
     // Work items (tile tau, head hh), heads fastest, dealt round-robin to the warps.  The input rows of
     // the next kAppendDepth items are kept in flight with per-lane 16-byte async copies into a per-warp
@@ -292,9 +339,8 @@ k_quant_pack(AppendParams p) {
     // neither access pattern has bank conflicts.
     struct Item {
         int k;                                         // class, -1 = no more items
-        bool active;
-        uint32_t tile;
-        int h;
+        bool active, tail;                             // the lane's slot gets a token / lies beyond the fill
+        uint8_t* rec;                                  // the tile record (found through the stream's block table)
     };
     uint32_t tau = 0;
     int hh = warp;
@@ -310,23 +356,25 @@ k_quant_pack(AppendParams p) {
     auto next_item = [&](int stage) {
         Item it;
         it.k = -1;
-        it.active = false;
-        it.tile = 0;
-        it.h = 0;
+        it.active = it.tail = false;
+        it.rec = nullptr;
         if (tau < pre[4]) {
             const int k = (tau >= pre[1]) + (tau >= pre[2]) + (tau >= pre[3]);
             const uint32_t basek = k == 0 ? base[0] : k == 1 ? base[1] : k == 2 ? base[2] : base[3];
             const uint32_t nk = k == 0 ? ncls[0] : k == 1 ? ncls[1] : k == 2 ? ncls[2] : ncls[3];
             it.k = k;
-            it.tile = (k == 0 ? first[0] : k == 1 ? first[1] : k == 2 ? first[2] : first[3]) +
-                      (tau - (k == 0 ? pre[0] : k == 1 ? pre[1] : k == 2 ? pre[2] : pre[3]));
-            const uint32_t r0 = it.tile * kTileTokens - basek;     // rank of the tile's slot 0 in the chunk (may wrap)
+            const uint32_t tile = (k == 0 ? first[0] : k == 1 ? first[1] : k == 2 ? first[2] : first[3]) +
+                                  (tau - (k == 0 ? pre[0] : k == 1 ? pre[1] : k == 2 ? pre[2] : pre[3]));
+            const uint32_t r0 = tile * kTileTokens - basek;        // rank of the tile's slot 0 in the chunk (may wrap)
             it.active = r0 + t < nk;                               // the slot this lane quantizes
-            it.h = h0 + hh;
+            // beyond the fill only in the append's last chunk (otherwise the next chunk's tokens go there)
+            it.tail = !it.active && (int32_t)(r0 + t) >= 0 && chunk == p.nchunks - 1;
+            const int h = h0 + hh;
+            it.rec = tile_ptr(p.store, k, stream_table(p.store, k, p.layer, b, h), tile);
             const uint32_t r_ld = r0 + (lane >> 1);                // the slot this lane copies a piece of
             if (r_ld < nk) {
                 const int i_tok = list[k][r_ld];
-                const size_t src = (((size_t)b * p.n_new + (size_t)chunk * kChunkTokens + i_tok) * p.store.kv_heads + it.h) *
+                const size_t src = (((size_t)b * p.n_new + (size_t)chunk * kChunkTokens + i_tok) * p.store.kv_heads + h) *
                                    kHeadDim;
                 const int odd = lane & 1;
                 const uint4* ks = reinterpret_cast<const uint4*>(p.K + src) + odd;
@@ -366,21 +414,21 @@ k_quant_pack(AppendParams p) {
         items[kAppendDepth - 1] = next_item(stage);
         if (++stage == kAppendDepth) stage = 0;
 
-        uint8_t* rec = p.store.pool[cur.k] + tile_offset(p.store, cur.k, p.layer, b, cur.h, (int)cur.tile);
+        uint8_t* rec = cur.rec;
         uint8_t* vcodes = rec + pool_codes_bytes(cur.k);
         const bool active = cur.active;
         switch (cur.k) {
         case 0:
-            quantize_store_half_row<0>(kraw, active, half, t, rec, rec + meta_offset(0, 0, t));
-            quantize_store_half_row<0>(vraw, active, half, t, vcodes, rec + meta_offset(0, 1, t));
+            quantize_store_half_row<0>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(0, 0, t));
+            quantize_store_half_row<0>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(0, 1, t));
             break;
         case 1:
-            quantize_store_half_row<1>(kraw, active, half, t, rec, rec + meta_offset(1, 0, t));
-            quantize_store_half_row<1>(vraw, active, half, t, vcodes, rec + meta_offset(1, 1, t));
+            quantize_store_half_row<1>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(1, 0, t));
+            quantize_store_half_row<1>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(1, 1, t));
             break;
         case 2:
-            quantize_store_half_row<2>(kraw, active, half, t, rec, rec + meta_offset(2, 0, t));
-            quantize_store_half_row<2>(vraw, active, half, t, vcodes, rec + meta_offset(2, 1, t));
+            quantize_store_half_row<2>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(2, 0, t));
+            quantize_store_half_row<2>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(2, 1, t));
             break;
         default:                                       // fp16: the lane's 64 input bytes are its four units
             if (active) {
@@ -394,6 +442,41 @@ k_quant_pack(AppendParams p) {
         }
     }
     cp_async_wait<0>();
+}
+
+// The stores of k_append_token: both tensors of the lane's half-row into the tile record `rec`.
+__device__ __forceinline__ void token_store(int c, const uint4 (&kraw)[4], const uint4 (&vraw)[4], bool active, int half,
+                                            int t, uint8_t* rec) {
+    uint8_t* vcodes = rec + pool_codes_bytes(c);
+    if (t == 0 && c < 3 && active) {                   // the token opens a tile: clear the tile's {scale, zero-point} words
+        uint4* m = reinterpret_cast<uint4*>(rec + meta_offset(c, half, 0));        // half 0: K words, half 1: V words
+#pragma unroll
+        for (int i = 0; i < 4; ++i) m[i] = make_uint4(0, 0, 0, 0);
+    }
+    __syncwarp();                                      // slot 0's own word is written after the clearing
+    switch (c) {
+    case 0:
+        quantize_store_half_row<0, 1>(kraw, active, false, half, t, rec, rec + meta_offset(0, 0, t));
+        quantize_store_half_row<0, 1>(vraw, active, false, half, t, vcodes, rec + meta_offset(0, 1, t));
+        break;
+    case 1:
+        quantize_store_half_row<1, 1>(kraw, active, false, half, t, rec, rec + meta_offset(1, 0, t));
+        quantize_store_half_row<1, 1>(vraw, active, false, half, t, vcodes, rec + meta_offset(1, 1, t));
+        break;
+    case 2:
+        quantize_store_half_row<2, 1>(kraw, active, false, half, t, rec, rec + meta_offset(2, 0, t));
+        quantize_store_half_row<2, 1>(vraw, active, false, half, t, vcodes, rec + meta_offset(2, 1, t));
+        break;
+    default:
+        if (active) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                *reinterpret_cast<uint4*>(rec + unit_offset(3, half, u, t)) = kraw[u];
+                *reinterpret_cast<uint4*>(vcodes + unit_offset(3, half, u, t)) = vraw[u];
+            }
+        }
+        break;
+    }
 }
 
 // One new token per sequence (a decode step): grid = (ceil(kv_heads / 16), batch), block = 32.
@@ -435,31 +518,21 @@ k_append_token(AppendParams p) {
         if (FUSED && p.bits_out) p.bits_out[b] = (uint8_t)pool_bits(c);
     }
     const int t = (int)(slot & (kTileTokens - 1));
-    uint8_t* rec = p.store.pool[c] + tile_offset(p.store, c, p.layer, b, active ? h : 0, (int)(slot / kTileTokens));
-    uint8_t* vcodes = rec + pool_codes_bytes(c);
-    switch (c) {
-    case 0:
-        quantize_store_half_row<0, 1>(kraw, active, half, t, rec, rec + meta_offset(0, 0, t));
-        quantize_store_half_row<0, 1>(vraw, active, half, t, vcodes, rec + meta_offset(0, 1, t));
-        break;
-    case 1:
-        quantize_store_half_row<1, 1>(kraw, active, half, t, rec, rec + meta_offset(1, 0, t));
-        quantize_store_half_row<1, 1>(vraw, active, half, t, vcodes, rec + meta_offset(1, 1, t));
-        break;
-    case 2:
-        quantize_store_half_row<2, 1>(kraw, active, half, t, rec, rec + meta_offset(2, 0, t));
-        quantize_store_half_row<2, 1>(vraw, active, half, t, vcodes, rec + meta_offset(2, 1, t));
-        break;
-    default:
-        if (active) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                *reinterpret_cast<uint4*>(rec + unit_offset(3, half, u, t)) = kraw[u];
-                *reinterpret_cast<uint4*>(vcodes + unit_offset(3, half, u, t)) = vraw[u];
-            }
+    const uint32_t tile = slot / kTileTokens;
+    uint32_t* tab = stream_table(p.store, c, p.layer, b, active ? h : 0);
+    if (slot % (kTileTokens * block_tiles(c)) == 0) {              // the token opens a new block of its stream
+        uint32_t id = 0;
+        if (active && half == 0) {
+            id = arena_take(p.store, 1);
+            tab[tile / block_tiles(c)] = id;
         }
-        break;
+        id = __shfl_sync(0xffffffffu, id, lane & ~1);
+        // the partner lane must not read the table before the entry is written: hand it the address instead
+        uint8_t* rec_new = p.store.arena + (size_t)id * kBlockBytes;
+        token_store(c, kraw, vraw, active, half, t, rec_new);
+        return;
     }
+    token_store(c, kraw, vraw, active, half, t, tile_ptr(p.store, c, tab, tile));
 }
 
 }  // namespace kvq

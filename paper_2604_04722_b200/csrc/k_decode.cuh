@@ -84,6 +84,9 @@ constexpr uint32_t kWaitLimit = 1u << 20;        // mbarrier polls before a wait
 constexpr uint32_t kFlagWaitTimeout = 2u;
 
 static_assert(kStageBytes % 16 == 0 && kStageBytes >= pool_rec_bytes(3), "a stage must hold one fp16 tile");
+static_assert(block_tiles(0) % (kStageBytes / pool_rec_bytes(0)) == 0 && block_tiles(1) % (kStageBytes / pool_rec_bytes(1)) == 0 &&
+                  block_tiles(2) % (kStageBytes / pool_rec_bytes(2)) == 0 && block_tiles(3) % (kStageBytes / pool_rec_bytes(3)) == 0,
+              "an arena block must hold a whole number of ring stages");
 __host__ __device__ constexpr int tiles_per_stage(int c) { return kStageBytes / pool_rec_bytes(c); }
 constexpr size_t kDecodeSmemBytes = (size_t)kDecodeWarps * kStages * kStageBytes;
 
@@ -403,7 +406,7 @@ struct Fp16Rows {
 // Per-warp scratch in shared memory: the segment being worked on.
 struct WarpScratch {
     uint64_t bars[kStages];
-    const uint8_t* base[kNumPools];    // first tile of this (layer, sequence, KV head) in each pool
+    const uint32_t* tab[kNumPools];    // block table of this (layer, sequence, KV head) in each pool
     int lo[kNumPools], hi[kNumPools];  // tile range of the segment in each pool
     uint32_t cnt[kNumPools];           // tokens in each pool
     float q[kHeadDim + 4];             // query row; half 1 starts at q[36] so the two halves sit in different banks
@@ -463,9 +466,7 @@ k_decode_attn(DecodeParams P) {
                 ws.lo[c] = (int)((uint64_t)nt * a0 / P.gw);
                 ws.hi[c] = (int)((uint64_t)nt * a1 / P.gw);
             }
-            const uint8_t* pool = c == 0 ? P.store.pool[0] : c == 1 ? P.store.pool[1] : c == 2 ? P.store.pool[2]
-                                                                                              : P.store.pool[3];
-            ws.base[c] = pool + tile_offset(P.store, c, P.layer, (int)b, kvh, 0);
+            ws.tab[c] = stream_table(P.store, c, P.layer, (int)b, kvh);
         }
         {
             const float2 q2 = __half22float2(reinterpret_cast<const __half2*>(P.Q + (size_t)u * kHeadDim)[lane]);
@@ -488,21 +489,33 @@ k_decode_attn(DecodeParams P) {
         }
 
         // ---- producer cursor (warp-uniform; lane 0 issues): next tile to fetch, tiles left in its pool
-        int p_c = -1, p_left = 0, p_tps = 0;
-        uint32_t p_rec = 0;
+        // Chunks end at absolute multiples of the pool's tiles-per-stage, and a block holds a whole number
+        // of stages, so a chunk never crosses a 64 KB block of the arena; the id of the block after the
+        // current one is fetched from the stream's table a whole block ahead of its first use.
+        int p_c = -1, p_left = 0, p_tps = 0, p_in_block = 0, p_phase = 0;
+        uint32_t p_rec = 0, p_next_id = 0;
         const uint8_t* p_ptr = nullptr;
+        const uint32_t* p_tab = nullptr;               // entry of the block after the current one
         auto next_pool = [&]() {                       // move to the next pool that has tiles in this segment
             while (p_left == 0 && ++p_c < kNumPools) {
                 const int lo = ws.lo[p_c];
                 p_left = ws.hi[p_c] - lo;
+                if (p_left == 0) continue;
                 p_tps = tps_of(p_c);
                 p_rec = (uint32_t)pool_rec_bytes(p_c);
-                p_ptr = ws.base[p_c] + (size_t)lo * p_rec;
+                const int bt = (int)block_tiles(p_c);
+                const int blk = lo / bt;
+                p_in_block = bt - (lo - blk * bt);
+                p_phase = p_tps - lo % p_tps;          // tiles up to the next stage boundary
+                p_tab = ws.tab[p_c] + blk + 1;
+                p_ptr = P.store.arena + (size_t)p_tab[-1] * kBlockBytes + (size_t)(lo - blk * bt) * p_rec;
+                p_next_id = p_tab[0];
             }
         };
         next_pool();
         auto issue_next = [&]() {
-            const int n = min(p_tps, p_left);
+            const int n = min(p_phase, p_left);
+            p_phase = p_tps;
             const uint32_t bytes = (uint32_t)n * p_rec;
             if (lane == 0) {
                 mbar_arrive_expect_tx(&ws.bars[pslot], bytes);
@@ -511,7 +524,15 @@ k_decode_attn(DecodeParams P) {
             if (++pslot == kStages) pslot = 0;
             p_ptr += bytes;
             p_left -= n;
-            if (p_left == 0) next_pool();
+            p_in_block -= n;
+            if (p_left == 0) {
+                next_pool();
+            } else if (p_in_block == 0) {              // on to the stream's next block
+                p_ptr = P.store.arena + (size_t)p_next_id * kBlockBytes;
+                p_in_block = (int)block_tiles(p_c);
+                ++p_tab;
+                p_next_id = p_tab[0];
+            }
         };
         int in_flight = 0;
         for (; in_flight < kStages && p_left > 0; ++in_flight) issue_next();
@@ -528,6 +549,7 @@ k_decode_attn(DecodeParams P) {
             const int hi = ws.hi[CLS];
             if (tile0 >= hi || failed) return;
             const uint32_t cnt = ws.cnt[CLS];
+            int phase = tiles_per_stage(CLS) - tile0 % tiles_per_stage(CLS);        // tiles up to the next stage boundary
             uint32_t qreg[kQRegs];
             C::enter(qi, qreg, acc);
             while (tile0 < hi) {
@@ -535,7 +557,8 @@ k_decode_attn(DecodeParams P) {
                     failed = true;
                     break;
                 }
-                const int ntiles = min(tiles_per_stage(CLS), hi - tile0);
+                const int ntiles = min(phase, hi - tile0);
+                phase = tiles_per_stage(CLS);
                 const uint8_t* buf = my_ring + (size_t)cslot * kStageBytes;
                 typename C::KIn kin = C::load_k(buf, half, t);
                 for (int i = 0; i < ntiles; ++i) {

@@ -39,7 +39,8 @@ k_export(ExportParams p) {
         const int j = it & 7, tensor = (it >> 3) & 1, h = it >> 4;
         uint4* dst = tensor ? p.v_codes : p.k_codes;
         if (!dst) continue;
-        const uint8_t* codes = s.pool[cls] + tile_offset(s, cls, p.layer, b, h, tile) + (size_t)tensor * pool_codes_bytes(cls);
+        const uint8_t* codes = tile_ptr(s, cls, stream_table(s, cls, p.layer, b, h), (uint32_t)tile) +
+                               (size_t)tensor * pool_codes_bytes(cls);
         uint4 v = make_uint4(0, 0, 0, 0);
         if (j < W) {
             if (cls == 0) {                            // the 16-byte row is two 8-byte half-rows
@@ -59,7 +60,7 @@ k_export(ExportParams p) {
         if (!dst) continue;
         uint32_t m = 0;
         if (cls < 3) {
-            const uint8_t* rec = s.pool[cls] + tile_offset(s, cls, p.layer, b, h, tile);
+            const uint8_t* rec = tile_ptr(s, cls, stream_table(s, cls, p.layer, b, h), (uint32_t)tile);
             m = *reinterpret_cast<const uint32_t*>(rec + meta_offset(cls, tensor, t));
         }
         dst[(tok * s.kv_heads + h) * 2 + 0] = (uint16_t)(m & 0xffffu);

@@ -23,7 +23,9 @@ struct kvq_ctx {
     int device = 0, sm_count = 0;
     int layers = 0, q_heads = 0, kv_heads = 0, max_ctx = 0, batch = 0;
     StoreView store{};
-    uint8_t* pool_block = nullptr;       // the four pools, one allocation
+    uint8_t* arena = nullptr;            // the tile records: blocks of kBlockBytes
+    uint32_t* table = nullptr;           // block tables of all streams
+    uint32_t* arena_used = nullptr;      // device counter of blocks handed out
     uint32_t* counts = nullptr;          // [2][layers][batch][4], double-buffered pool fills
     std::vector<int> len;                // host mirror: tokens per sequence, per layer
     std::vector<int> cur;                // which counts buffer is current, per layer
@@ -83,7 +85,9 @@ constexpr int kProfMaxCalls = 1024;
 void free_all(kvq_ctx* c) {
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     c->prof_ev.clear();
-    cudaFree(c->pool_block);
+    cudaFree(c->arena);
+    cudaFree(c->table);
+    cudaFree(c->arena_used);
     cudaFree(c->store.index);
     cudaFree(c->counts);
     cudaFree(c->cls);
@@ -166,8 +170,9 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
         dim3 grid_c(p.nchunks, c->batch);
         if (fused) k_classify<true><<<grid_c, kChunkTokens, smem, st>>>(p);
         else k_classify<false><<<grid_c, kChunkTokens, 0, st>>>(p);
+        k_reserve_blocks<<<c->batch, 128, 0, st>>>(p);
         k_quant_pack<0><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
-        c->launches += 2;
+        c->launches += 3;
     }
     KVQ_CUDA(c, cudaGetLastError());
     c->cur[layer] ^= 1;
@@ -263,6 +268,11 @@ int export_impl(kvq_ctx* c, int layer, int b0, int nb, int pos0, int n, uint8_t*
 extern "C" {
 
 int kvq_create(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch) {
+    return kvq_create_arena(out, layers, q_heads, kv_heads, head_dim, max_ctx, batch, 0);
+}
+
+int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
+                     uint64_t arena_bytes) {
     if (!out) return KVQ_ERR_ARG;
     *out = nullptr;
     if (layers < 1 || q_heads < 1 || kv_heads < 1 || batch < 1 || max_ctx < 1) return KVQ_ERR_ARG;
@@ -291,15 +301,30 @@ int kvq_create(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_di
     s.max_ctx = max_ctx;
     s.cap_tiles = (max_ctx + kTileTokens - 1) / kTileTokens;
 
-    const size_t seqs = (size_t)layers * batch * kv_heads;
-    size_t pool_bytes[kNumPools], total = 0;
+    // block tables: one row per stream, class k at table_off[k]; one spare entry at the very end because
+    // the decode kernel reads the entry after the block it is working on
+    const size_t streams = (size_t)layers * batch * kv_heads;
+    uint32_t row = 0;
     for (int k = 0; k < kNumPools; ++k) {
-        pool_bytes[k] = seqs * s.cap_tiles * (size_t)pool_rec_bytes(k);
-        total += pool_bytes[k];
+        s.table_off[k] = row;
+        row += blocks_for(k, (uint32_t)max_ctx);
     }
+    s.table_stride = row;
+    const uint64_t worst_blocks = (uint64_t)streams * row + 1;           // every token in every class, plus block 0
+    uint64_t blocks = arena_bytes ? arena_bytes / kBlockBytes : worst_blocks;
+    if (blocks > worst_blocks) blocks = worst_blocks;
+    if (blocks < 2 || blocks > 0xffffffffull) {
+        delete c;
+        return KVQ_ERR_ARG;
+    }
+    s.arena_blocks = (uint32_t)blocks;
+    const size_t total = (size_t)blocks * kBlockBytes;
+    const size_t table_bytes = sizeof(uint32_t) * (streams * row + 1);
     const size_t max_chunks = (size_t)(max_ctx + kChunkTokens - 1) / kChunkTokens;
     const size_t units = (size_t)batch * q_heads;
-    bool ok = dev_alloc(c, &c->pool_block, total) == cudaSuccess;
+    bool ok = dev_alloc(c, &c->arena, total) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->table, table_bytes) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->arena_used, sizeof(uint32_t)) == cudaSuccess;
     ok = ok && dev_alloc(c, &s.index, sizeof(uint32_t) * (size_t)layers * batch * max_ctx) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->counts, sizeof(uint32_t) * 2 * (size_t)layers * batch * 4) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->cls, (size_t)batch * max_ctx) == cudaSuccess;
@@ -317,13 +342,13 @@ int kvq_create(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_di
     ok = ok && dev_alloc(c, &c->st_bits, (size_t)batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_export, (size_t)kv_heads * (2 * KVQ_EXPORT_ROW_BYTES + 8) + 16) == cudaSuccess;
     if (ok) {
-        size_t off = 0;
-        for (int k = 0; k < kNumPools; ++k) {
-            s.pool[k] = c->pool_block + off;
-            off += pool_bytes[k];
-        }
+        s.arena = c->arena;
+        s.table = c->table;
+        s.arena_used = c->arena_used;
         s.flags = c->flags;
-        ok = cudaMemset(c->pool_block, 0, total) == cudaSuccess;
+        ok = cudaMemset(c->arena, 0, total) == cudaSuccess;
+        ok = ok && cudaMemset(c->table, 0, table_bytes) == cudaSuccess;
+        ok = ok && cudaMemset(c->arena_used, 0, sizeof(uint32_t)) == cudaSuccess;
         ok = ok && cudaMemset(s.index, 0, sizeof(uint32_t) * (size_t)layers * batch * max_ctx) == cudaSuccess;
         ok = ok && cudaMemset(c->counts, 0, sizeof(uint32_t) * 2 * (size_t)layers * batch * 4) == cudaSuccess;
         ok = ok && cudaMemset(c->flags, 0, sizeof(uint32_t)) == cudaSuccess;
@@ -492,6 +517,7 @@ int kvq_reset(kvq_ctx* c, void* stream) {
     DeviceGuard guard(c->device);
     KVQ_CUDA(c, cudaMemsetAsync(c->counts, 0, sizeof(uint32_t) * 2 * (size_t)c->layers * c->batch * 4,
                                 static_cast<cudaStream_t>(stream)));
+    KVQ_CUDA(c, cudaMemsetAsync(c->arena_used, 0, sizeof(uint32_t), static_cast<cudaStream_t>(stream)));
     for (int l = 0; l < c->layers; ++l) {
         c->len[l] = 0;
         c->cur[l] = 0;
@@ -564,6 +590,19 @@ int kvq_stats(kvq_ctx* c, int layer, uint32_t* host_counts, uint64_t* resident_b
     if (host_counts) memcpy(host_counts, cnt.data(), sizeof(uint32_t) * cnt.size());
     if (resident_bytes) *resident_bytes = bytes;
     if (expected_bits) *expected_bits = tokens ? (double)bit_sum / (double)tokens : 0.0;
+    return KVQ_OK;
+}
+
+int kvq_arena_usage(kvq_ctx* c, uint64_t* blocks_in_use, uint64_t* blocks_total, uint64_t* block_bytes) {
+    if (!c) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    uint32_t used = 0;
+    KVQ_CUDA(c, cudaDeviceSynchronize());
+    KVQ_CUDA(c, cudaMemcpy(&used, c->arena_used, sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    const uint64_t total = c->store.arena_blocks - 1;                     // block 0 is never handed out
+    if (blocks_in_use) *blocks_in_use = used < total ? used : total;
+    if (blocks_total) *blocks_total = total;
+    if (block_bytes) *block_bytes = kBlockBytes;
     return KVQ_OK;
 }
 

@@ -22,8 +22,13 @@
 // [(i*b)%8, +b) of byte floor(i*b/8)); half h is bytes [h*8<<c, (h+1)*8<<c) of
 // the canonical row.
 //
-// The tiles of one (layer, sequence, KV head, class) are contiguous, in slot
-// order, cap_tiles = ceil(max_ctx/16) of them.
+// Placement.  All tile records live in one ARENA of 64 KB blocks.  A block belongs to one
+// STREAM = (layer, sequence, KV head, class) and holds 100 / 55 / 30 / 16 consecutive tiles of it
+// (1600 / 880 / 480 / 256 tokens; the tail of a block that no whole tile fits is unused).  A block
+// table per stream lists its blocks in slot order; blocks are handed out by a device-side counter
+// when an append first reaches them, so the memory in use follows what was actually stored: the
+// sum of the row bytes plus at most one partly filled block per stream.  Block 0 is never handed
+// out: writes that find the arena exhausted land there and set KVQ_FLAG_ARENA_FULL.
 #pragma once
 #include <cuda_runtime.h>
 #include <cuda_fp16.h>
@@ -58,17 +63,46 @@ __host__ __device__ constexpr int meta_offset(int c, int tensor, int t) {
     return 2 * pool_codes_bytes(c) + tensor * pool_meta_bytes(c) + 4 * t;
 }
 
+constexpr uint32_t kBlockBytes = 65536;
+// Tiles per block: a whole number of ring stages of the decode kernel (10 / 5 / 3 / 1 tiles).
+__host__ __device__ constexpr uint32_t block_tiles(int c) { return c == 0 ? 100u : c == 1 ? 55u : c == 2 ? 30u : 16u; }
+constexpr uint32_t kFlagArenaFull = 4u;
+
 // Everything a kernel needs to find a row.
 struct StoreView {
-    uint8_t* pool[kNumPools];     // base of each class's region
+    uint8_t* arena;               // blocks of kBlockBytes
+    uint32_t* table;              // [streams][table_stride] block ids, class c at table_off[c]
+    uint32_t* arena_used;         // blocks handed out so far (block ids are 1 + the old value)
+    uint32_t arena_blocks;        // capacity in blocks, block 0 included
+    uint32_t table_stride, table_off[kNumPools];
     uint32_t* index;              // [layers][batch][max_ctx]   pool<<30 | slot
     uint32_t* flags;              // device flag word
     int layers, batch, kv_heads, q_heads, max_ctx, cap_tiles;
 };
 
-__host__ __device__ inline size_t tile_offset(const StoreView& s, int c, int layer, int b, int h, int tile) {
-    size_t seq = ((size_t)layer * s.batch + b) * s.kv_heads + h;
-    return (seq * (size_t)s.cap_tiles + (size_t)tile) * (size_t)pool_rec_bytes(c);
+// The block-table row of class c of stream (layer, b, h).
+__host__ __device__ inline uint32_t* stream_table(const StoreView& s, int c, int layer, int b, int h) {
+    const size_t stream = ((size_t)layer * s.batch + b) * s.kv_heads + h;
+    return s.table + stream * s.table_stride + s.table_off[c];
+}
+// Address of tile `tile` of a stream whose table row is `tab`.
+__device__ __forceinline__ uint8_t* tile_ptr(const StoreView& s, int c, const uint32_t* tab, uint32_t tile) {
+    const uint32_t bt = block_tiles(c);
+    const uint32_t blk = tile / bt;
+    return s.arena + (size_t)tab[blk] * kBlockBytes + (size_t)(tile - blk * bt) * (uint32_t)pool_rec_bytes(c);
+}
+// Hand out `n` consecutive blocks; returns the id of the first (0 = the arena is exhausted: flagged).
+__device__ __forceinline__ uint32_t arena_take(const StoreView& s, uint32_t n) {
+    const uint32_t first = 1u + atomicAdd(s.arena_used, n);
+    if (first + n > s.arena_blocks) {
+        atomicOr(s.flags, kFlagArenaFull);
+        return 0u;
+    }
+    return first;
+}
+// Blocks a stream of class c needs for n tokens.
+__host__ __device__ constexpr uint32_t blocks_for(int c, uint32_t n) {
+    return ((n + kTileTokens - 1) / kTileTokens + block_tiles(c) - 1) / block_tiles(c);
 }
 
 __device__ __forceinline__ int bits_to_class(int bits) {
