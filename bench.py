@@ -44,9 +44,9 @@ UNIT = "GB/s"
 
 # DRAM traffic of one k_decode_attn launch on this workload (dram__bytes_read.sum +
 # dram__bytes_write.sum): captured with a quarter of the sequences (profiles/k_decode_attn_cfg5_batch4.md,
-# 319.6 MB per launch) and scaled by the rows read (x 4); every row is read exactly once, so traffic
+# 319.2 MB per launch) and scaled by the rows read (x 4); every row is read exactly once, so traffic
 # grows in proportion.  Set to None whenever the kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 319.6e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 319.2e6
 
 
 def measured_peak_gbs():
@@ -378,6 +378,7 @@ def run_ours(args, wl):
     time.sleep(0.2)
     clocks = sampler.stop()
     _, resident1, ebits = kq.kvq_stats(ctx, 0, B)
+    arena_used, arena_total, arena_block = kq.kvq_arena_usage(ctx)
     resident_mean = 0.5 * (resident0 + resident1)     # per layer
     new_rows_mean = (resident1 - resident0) / max(1, step_no[0] - W)
 
@@ -455,6 +456,11 @@ def run_ours(args, wl):
                 "GBps_fused": (B * ctx_len * Hkv * 256 + ctl_written) / (ms_prefill_fused * 1e-3) / 1e9,
                 "GBps_bits_given": (B * ctx_len * Hkv * 256 + given_written) / (ms_prefill_given * 1e-3) / 1e9,
                 "controller_class_histogram": ctl_hist, "note": "one layer"},
+            "memory": {"packed_row_bytes": int(L * resident1), "arena_bytes_in_use": int(arena_used * arena_block),
+                       "arena_bytes_reserved": int(arena_total * arena_block),
+                       "fp16_cache_bytes": int(L * B * Hkv * (ctx_len + step_no[0]) * 256),
+                       "note": "arena blocks are taken on demand; kvq_create reserves the worst case, "
+                               "kvq_create_arena any budget"},
             "kv_bytes_per_layer": dec_bytes, "expected_bits": ebits,
             "device_bytes": kq.kvq_device_bytes(ctx), "input_generation_s": t_gen,
         }

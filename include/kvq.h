@@ -17,10 +17,11 @@
  * One bit-width per token is used for its K row and its V row, in every KV
  * head.  Class index <-> bit-width: 0,1,2,3 <-> 2,4,8,16 (Algorithm 1).
  *
- * Store: one pool per precision; inside a pool the rows of one (layer,
- * sequence, KV head) are contiguous in slot order; slot = number of earlier
- * tokens of that (layer, sequence) with the same precision.  A per-token
- * index word (pool << 30 | slot) is kept per (layer, sequence, position).
+ * Store: one pool per precision; the rows of one (layer, sequence, KV head,
+ * precision) stream are kept in slot order in 64 KB blocks of a common arena
+ * that are taken when an append first reaches them; slot = number of earlier
+ * tokens of that (layer, sequence) with the same precision.  A per-token index
+ * word (pool << 30 | slot) is kept per (layer, sequence, position).
  *
  * Conventions
  *   - Every function returns 0 (KVQ_OK) or a negative KVQ_ERR_* code, except
