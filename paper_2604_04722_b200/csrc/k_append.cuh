@@ -503,6 +503,14 @@ k_append_token(AppendParams p) {
         }
     }
     const uint4 fill = *reinterpret_cast<const uint4*>(p.counts_in + (size_t)b * 4);
+    // The block-table entry is needed once the class is known; the four candidates (one per class) are
+    // requested now, so that they travel while the controller runs.  An entry of a block that is not
+    // reserved yet may hold anything and is not used.
+    const int hs = active ? h : 0;
+    const uint32_t id0 = stream_table(p.store, 0, p.layer, b, hs)[fill.x / (kTileTokens * block_tiles(0))];
+    const uint32_t id1 = stream_table(p.store, 1, p.layer, b, hs)[fill.y / (kTileTokens * block_tiles(1))];
+    const uint32_t id2 = stream_table(p.store, 2, p.layer, b, hs)[fill.z / (kTileTokens * block_tiles(2))];
+    const uint32_t id3 = stream_table(p.store, 3, p.layer, b, hs)[fill.w / (kTileTokens * block_tiles(3))];
     int c;
     if (FUSED) {
         const float4 f = reinterpret_cast<const float4*>(p.feats)[b];
@@ -532,7 +540,9 @@ k_append_token(AppendParams p) {
         token_store(c, kraw, vraw, active, half, t, rec_new);
         return;
     }
-    token_store(c, kraw, vraw, active, half, t, tile_ptr(p.store, c, tab, tile));
+    const uint32_t id = c == 0 ? id0 : c == 1 ? id1 : c == 2 ? id2 : id3;
+    token_store(c, kraw, vraw, active, half, t,
+                p.store.arena + (size_t)id * kBlockBytes + (size_t)(tile % block_tiles(c)) * (uint32_t)pool_rec_bytes(c));
 }
 
 }  // namespace kvq
