@@ -123,6 +123,18 @@ class ClockSampler:
         return out
 
 
+def aggregate_over_ranks(times_ms, step_bytes_this_rank, dist, device):
+    """The whole job's figures from one rank's: every time becomes the slowest rank's (max), the bytes
+    of a step become the sum over the ranks' replicas.  `dist` is torch.distributed or None."""
+    import torch
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    nbytes = torch.tensor([float(step_bytes_this_rank)], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(nbytes, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t.tolist()], float(nbytes.item())
+
+
 def oracle_leg(wl, seqs, steps, warmup):
     """The CPU oracle, as it stands, on a bounded sample of the workload: `seqs` whole sequences.
     Each step = decision for the new tokens + quantize-append + attention over everything cached."""
@@ -407,13 +419,9 @@ def run_ours(args, wl):
 
     # ---- reduce over ranks: slowest rank's time, summed bytes
     ms_step = ms_total / K_steps
-    vals = torch.tensor([ms_step, ms_e2e, attn_ms / max(ncalls, 1)], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    ms_step, ms_e2e, ms_attn = [float(x) for x in vals.tolist()]
-
-    dec_bytes, app_bytes = step_bytes(wl, ctx_len, resident_mean, new_rows_mean)    # per layer
-    bytes_step = L * (dec_bytes + app_bytes)
+    dec_bytes, app_bytes = step_bytes(wl, ctx_len, resident_mean, new_rows_mean)    # per layer, this rank's replica
+    (ms_step, ms_e2e, ms_attn), bytes_job = aggregate_over_ranks(
+        [ms_step, ms_e2e, attn_ms / max(ncalls, 1)], L * (dec_bytes + app_bytes), dist, dev)
     peak, peak_kind = measured_peak_gbs()
     achieved = dec_bytes / (ms_attn * 1e-3) / 1e9
     index_bytes = B * (ctx_len + W + K_steps / 2) * 4
@@ -431,12 +439,12 @@ def run_ours(args, wl):
         if args.uniform_bits:
             cfg["uniform_bits"] = args.uniform_bits
         line = {
-            "metric": METRIC, "value": world * bytes_step / (ms_step * 1e-3) / 1e9, "unit": UNIT,
+            "metric": METRIC, "value": bytes_job / (ms_step * 1e-3) / 1e9, "unit": UNIT,
             "n_gpus": world, "steps": K_steps, "warmup": W, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": cfg,
             "clocks": clocks,
-            "e2e": {"value": world * bytes_step / (ms_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms_e2e,
+            "e2e": {"value": bytes_job / (ms_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms_e2e,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches_timed),
             "roofline": {"bound": "hbm", "kernel": "k_decode_attn", "achieved": achieved, "peak": peak,
