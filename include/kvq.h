@@ -152,6 +152,17 @@ int kvq_append_fused(kvq_ctx* ctx, int layer, const void* K, const void* V,
 int kvq_decode_attn(kvq_ctx* ctx, int layer, const void* Q, void* O, void* stream);
 
 /*
+ * Causal attention of several query rows over the cache (Eq. 5 applied at each of the last
+ * n_queries cached positions): query row i belongs to the token at position len - n_queries + i
+ * and attends over positions <= its own, the rows after it stay invisible.  This is what a
+ * speculative or chunked decode step needs after appending n_queries tokens at once.
+ * Q, O: dev fp16 [batch][n_queries][q_heads][64].  1 <= n_queries <= cached length
+ * (KVQ_ERR_ARG otherwise); n_queries == 1 is kvq_decode_attn.  Rows are served eight per
+ * launch; every row reads the cache on its own (no sharing between rows).
+ */
+int kvq_attend_last(kvq_ctx* ctx, int layer, const void* Q, void* O, int n_queries, void* stream);
+
+/*
  * kvq_decode_attn without any buffer that had to be allocated for it.  (No counterpart in
  * the paper: this is a packaging variant of the call above, same arithmetic, same result.)
  *

@@ -207,3 +207,17 @@ class OracleCache:
     def decode_attn(self, Q, want64: bool = False):
         return decode_attn(Q, self.Hq, self.Hkv, self.bits, self.kc, self.km,
                            self.vc, self.vm, want64=want64)
+
+    def attend_last(self, Q):
+        """Causal attention of the last T cached positions (Eq. 5 at each of them): Q fp16 [B][T][Hq][D];
+        row i sees the first len - T + i + 1 tokens.  Written as T plain calls on truncated caches."""
+        Q = _u16(Q)
+        B, T, Hq, D = Q.shape
+        n = len(self)
+        assert 1 <= T <= n
+        out = np.empty((B, T, Hq, D), dtype=np.uint16)
+        for i in range(T):
+            m = n - T + i + 1
+            out[:, i] = decode_attn(np.ascontiguousarray(Q[:, i]), self.Hq, self.Hkv, self.bits[:, :m],
+                                    self.kc[:, :m], self.km[:, :m], self.vc[:, :m], self.vm[:, :m])
+        return out

@@ -40,6 +40,7 @@ SIGNATURES = {
     "kvq_append": (_i, [_vp, _i, _vp, _vp, _vp, _i, _vp]),
     "kvq_append_fused": (_i, [_vp, _i, _vp, _vp, _vp, _i, _vp, _vp]),
     "kvq_decode_attn": (_i, [_vp, _i, _vp, _vp, _vp]),
+    "kvq_attend_last": (_i, [_vp, _i, _vp, _vp, _i, _vp]),
     "kvq_decode_attn_static": (_i, [_vp, _i, _vp, _vp, _vp]),
     "kvq_decode_step_host": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvq_reset": (_i, [_vp, _vp]),
@@ -156,6 +157,10 @@ def kvq_append_fused(ctx: int, layer: int, K, V, feats, n_new: int, bits_out=Non
 
 def kvq_decode_attn(ctx: int, layer: int, Q, O, stream=None) -> None:
     check(lib().kvq_decode_attn(ctx, layer, _ptr(Q), _ptr(O), _stream(stream)), "kvq_decode_attn")
+
+
+def kvq_attend_last(ctx: int, layer: int, Q, O, n_queries: int, stream=None) -> None:
+    check(lib().kvq_attend_last(ctx, layer, _ptr(Q), _ptr(O), n_queries, _stream(stream)), "kvq_attend_last")
 
 
 def kvq_decode_attn_static(ctx: int, layer: int, Q, O, stream=None) -> None:

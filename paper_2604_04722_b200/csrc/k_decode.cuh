@@ -93,13 +93,17 @@ constexpr size_t kDecodeSmemBytes = (size_t)kDecodeWarps * kStages * kStageBytes
 struct DecodeParams {
     StoreView store;
     const uint32_t* counts;        // [batch][4] pool fills of this layer
-    const __half* Q;               // [batch][q_heads][64]
-    __half* O;                     // [batch][q_heads][64]
+    const __half* Q;               // [batch][t_total][q_heads][64]
+    __half* O;                     // [batch][t_total][q_heads][64]
     float* part_o;                 // [units][pslots][64]  unnormalised
     float2* part_ml;               // [units][pslots]      (m in log2 units, l)
     uint32_t* part_cnt;            // [units] partials delivered so far; zero between launches
     int layer, group;              // group = q_heads / kv_heads
-    uint32_t units;                // batch * q_heads
+    // Query rows per sequence.  A decode step has one (tq = t_total = 1, t0 = 0).  With several (the last
+    // t_total cached tokens each ask, causally), a launch serves rows t0 .. t0+tq of every sequence and
+    // `counts` has one row of visible pool fills per (sequence, query row of the launch).
+    uint32_t tq, t_total, t0;
+    uint32_t units;                // batch * tq * q_heads
     uint32_t gw;                   // working warps = parts the x axis is cut into
     uint32_t pslots;               // partial slots per unit = decode_pslots(units, gw)
 };
@@ -452,11 +456,13 @@ k_decode_attn(DecodeParams P) {
         const uint64_t room = xend - x;
         const uint32_t a1 = room < (uint64_t)(P.gw - a0) ? a0 + (uint32_t)room : P.gw;
         x += a1 - a0;
-        const uint32_t b = u / (uint32_t)P.store.q_heads, qh = u - b * (uint32_t)P.store.q_heads;
+        const uint32_t row = u / (uint32_t)P.store.q_heads, qh = u - row * (uint32_t)P.store.q_heads;
+        const uint32_t b = row / P.tq;                 // row = b * tq + (query row - t0)
+        const size_t qo = (((size_t)b * P.t_total + P.t0 + (row - b * P.tq)) * P.store.q_heads + qh) * kHeadDim;
         const int kvh = (int)qh / P.group;
         if (lane < kNumPools) {                        // lane c plans pool c
             const int c = lane;
-            const uint32_t n = P.counts[(size_t)b * 4 + c];
+            const uint32_t n = P.counts[(size_t)row * 4 + c];
             const uint32_t nt = (n + kTileTokens - 1) / kTileTokens;
             ws.cnt[c] = n;
             if (P.gw < 65536u) {
@@ -469,7 +475,7 @@ k_decode_attn(DecodeParams P) {
             ws.tab[c] = stream_table(P.store, c, P.layer, (int)b, kvh);
         }
         {
-            const float2 q2 = __half22float2(reinterpret_cast<const __half2*>(P.Q + (size_t)u * kHeadDim)[lane]);
+            const float2 q2 = __half22float2(reinterpret_cast<const __half2*>(P.Q + qo)[lane]);
             const int i = 2 * lane;                    // elements i, i+1 (same half)
             float* dst = ws.q + (i >> 5) * kQHalfStride + (i & 31);
             dst[0] = q2.x;
@@ -684,10 +690,30 @@ k_decode_attn(DecodeParams P) {
                     }
                 }
             }
-            reinterpret_cast<__half2*>(P.O + (size_t)u * kHeadDim)[lane] = __floats2half2_rn(o0 / L, o1 / L);
+            reinterpret_cast<__half2*>(P.O + qo)[lane] = __floats2half2_rn(o0 / L, o1 / L);
             if (lane == 0) P.part_cnt[u] = 0;
         }
     }
+}
+
+// Pool fills each of the last t_total cached tokens may see when it asks as a query (causal
+// attention over the mixed cache).  Slots of a pool are handed out in position order, so query row i
+// (position len - t_total + i) sees every slot of pool c except those of the later rows of that class:
+// vis[b][i - t0][c] = fill[b][c] - #{ j > i : class(position of row j) == c }, for rows t0 .. t0+tq.
+// grid = batch, block = tq threads.
+__global__ void k_visible_counts(StoreView s, const uint32_t* __restrict__ fill, int layer, int len, uint32_t t_total,
+                                 uint32_t t0, uint32_t tq, uint32_t* __restrict__ vis) {
+    const uint32_t b = blockIdx.x, il = threadIdx.x;
+    if (il >= tq) return;
+    const uint32_t i = t0 + il;
+    uint32_t l0 = 0, l1 = 0, l2 = 0, l3 = 0;
+    const uint32_t* idx = s.index + ((size_t)layer * s.batch + b) * s.max_ctx + (len - (int)t_total);
+    for (uint32_t j = i + 1; j < t_total; ++j) {
+        const uint32_t c = idx[j] >> 30;
+        l0 += c == 0; l1 += c == 1; l2 += c == 2; l3 += c == 3;
+    }
+    const uint4 f = *reinterpret_cast<const uint4*>(fill + (size_t)b * 4);
+    *reinterpret_cast<uint4*>(vis + ((size_t)b * tq + il) * 4) = make_uint4(f.x - l0, f.y - l1, f.z - l2, f.w - l3);
 }
 
 }  // namespace kvq

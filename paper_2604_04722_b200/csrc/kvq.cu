@@ -36,6 +36,7 @@ struct kvq_ctx {
     float* part_o = nullptr;             // decode scratch [units][partial slots][64]
     float2* part_ml = nullptr;           //                [units][partial slots]
     uint32_t* part_cnt = nullptr;        //                [units] arrival counters, zero between launches
+    uint32_t* vis = nullptr;             // kvq_attend_last: visible pool fills [batch][query rows of a launch][4]
     int splits_override = 0;
     uint32_t* flags = nullptr;
     // device staging for the host-buffer entry points
@@ -96,6 +97,7 @@ void free_all(kvq_ctx* c) {
     cudaFree(c->part_o);
     cudaFree(c->part_ml);
     cudaFree(c->part_cnt);
+    cudaFree(c->vis);
     cudaFree(c->flags);
     cudaFree(c->st_feats);
     cudaFree(c->st_K);
@@ -188,9 +190,13 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
 // unit border work on two units and finish last, measured at about 0.9 of the ideal) and whole
 // numbers of parts per unit (every warp does the same single piece of work; what counts is how
 // full the last wave of CTAs is and how much of a warp's time goes into set-up).
-uint32_t choose_warps(kvq_ctx* c, int len) {
-    const uint64_t units = (uint64_t)c->batch * c->q_heads;
-    if (c->splits_override > 0) return (uint32_t)(units * (uint64_t)c->splits_override);
+constexpr int kMaxQueryRows = 8;       // query rows per sequence that one launch of kvq_attend_last serves
+
+size_t max_partial_records(const kvq_ctx* c);
+
+uint32_t choose_warps(kvq_ctx* c, int len, uint64_t units) {
+    if (c->splits_override > 0 && units * (uint64_t)(c->splits_override + 1) <= max_partial_records(c))
+        return (uint32_t)(units * (uint64_t)c->splits_override);
     const uint64_t tiles = units * (uint64_t)((len + kTileTokens - 1) / kTileTokens + (kNumPools - 1));
     const uint64_t resident = (uint64_t)kDecodeWarps * kDecodeCtasPerSm * c->sm_count;
     uint64_t cap = tiles / 8;
@@ -202,7 +208,8 @@ uint32_t choose_warps(kvq_ctx* c, int len) {
     uint64_t best = resident;
     const double tpw_p = tiles_d / (double)resident;
     double best_score = 0.90 * tpw_p / (tpw_p + 25.0);           // some warps work on two parts
-    for (uint64_t s = 1; s <= (uint64_t)kMaxSplits && units * s <= cap; ++s) {
+    const uint64_t room = max_partial_records(c);                 // partial records the handle has scratch for
+    for (uint64_t s = 1; s <= (uint64_t)kMaxSplits && units * s <= cap && units * (s + 1) <= room; ++s) {
         const double fill = (double)(units * s) / (double)resident;
         const double waves = (double)(uint64_t)(fill + 0.999999);
         if (waves > 8.0) break;
@@ -221,7 +228,7 @@ size_t max_partial_records(const kvq_ctx* c) {
     const size_t units = (size_t)c->batch * c->q_heads;
     const size_t resident = (size_t)kDecodeWarps * kDecodeCtasPerSm * c->sm_count;
     const size_t by_splits = units * (kMaxSplits + 1);
-    const size_t by_residency = resident + 2 * units;
+    const size_t by_residency = resident + 2 * units * kMaxQueryRows;
     return by_splits > by_residency ? by_splits : by_residency;
 }
 
@@ -237,6 +244,8 @@ void fill_decode_params(kvq_ctx* c, int layer, const void* Q, void* O, float* pa
     p.part_cnt = part_cnt;
     p.layer = layer;
     p.group = c->q_heads / c->kv_heads;
+    p.tq = p.t_total = 1;
+    p.t0 = 0;
     p.units = (uint32_t)c->batch * (uint32_t)c->q_heads;
     p.gw = gw;
     p.pslots = decode_pslots(p.units, gw);
@@ -332,7 +341,8 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
     ok = ok && dev_alloc(c, &c->ctrl, controller_smem(kMaxHidden)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_o, sizeof(float) * max_partial_records(c) * kHeadDim) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_ml, sizeof(float2) * max_partial_records(c)) == cudaSuccess;
-    ok = ok && dev_alloc(c, &c->part_cnt, sizeof(uint32_t) * units) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->part_cnt, sizeof(uint32_t) * units * kMaxQueryRows) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->vis, sizeof(uint32_t) * 4 * (size_t)batch * kMaxQueryRows) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->flags, sizeof(uint32_t)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_feats, sizeof(float) * 4 * batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_K, sizeof(__half) * (size_t)batch * kv_heads * kHeadDim) == cudaSuccess;
@@ -352,7 +362,7 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
         ok = ok && cudaMemset(s.index, 0, sizeof(uint32_t) * (size_t)layers * batch * max_ctx) == cudaSuccess;
         ok = ok && cudaMemset(c->counts, 0, sizeof(uint32_t) * 2 * (size_t)layers * batch * 4) == cudaSuccess;
         ok = ok && cudaMemset(c->flags, 0, sizeof(uint32_t)) == cudaSuccess;
-        ok = ok && cudaMemset(c->part_cnt, 0, sizeof(uint32_t) * units) == cudaSuccess;
+        ok = ok && cudaMemset(c->part_cnt, 0, sizeof(uint32_t) * units * kMaxQueryRows) == cudaSuccess;
         // the controller block may exceed the default 48 KB of dynamic shared memory
         const int smem_max = (int)controller_smem(kMaxHidden);
         ok = ok && cudaFuncSetAttribute(k_select_bits, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
@@ -432,7 +442,7 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
     DeviceGuard guard(c->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DecodeParams p{};
-    fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, choose_warps(c, c->len[layer]), p);
+    fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, choose_warps(c, c->len[layer], (uint64_t)c->batch * c->q_heads), p);
     const unsigned grid = (p.gw + kDecodeWarps - 1) / kDecodeWarps;
     const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
     cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 2] : nullptr;
@@ -443,6 +453,32 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
         c->prof_calls += 1;
     }
     c->launches += 1;
+    KVQ_CUDA(c, cudaGetLastError());
+    return KVQ_OK;
+}
+
+int kvq_attend_last(kvq_ctx* c, int layer, const void* Q, void* O, int n_queries, void* stream) {
+    if (check_layer(c, layer) != KVQ_OK || !Q || !O || n_queries < 1) return KVQ_ERR_ARG;
+    if (c->len[layer] == 0) return KVQ_ERR_EMPTY;
+    if (n_queries > c->len[layer]) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int t0 = 0; t0 < n_queries; t0 += kMaxQueryRows) {
+        const int tq = n_queries - t0 < kMaxQueryRows ? n_queries - t0 : kMaxQueryRows;
+        k_visible_counts<<<c->batch, tq, 0, st>>>(c->store, counts_of(c, c->cur[layer], layer), layer, c->len[layer],
+                                                  (uint32_t)n_queries, (uint32_t)t0, (uint32_t)tq, c->vis);
+        const uint64_t units = (uint64_t)c->batch * tq * c->q_heads;
+        DecodeParams p{};
+        fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, choose_warps(c, c->len[layer], units), p);
+        p.counts = c->vis;
+        p.tq = (uint32_t)tq;
+        p.t_total = (uint32_t)n_queries;
+        p.t0 = (uint32_t)t0;
+        p.units = (uint32_t)units;
+        p.pslots = decode_pslots(p.units, p.gw);
+        k_decode_attn<<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+        c->launches += 2;
+    }
     KVQ_CUDA(c, cudaGetLastError());
     return KVQ_OK;
 }
@@ -465,7 +501,7 @@ int kvq_decode_attn_static(kvq_ctx* c, int layer, const void* Q, void* O, void* 
     if (check_layer(c, layer) != KVQ_OK || !Q || !O) return KVQ_ERR_ARG;
     if (c->len[layer] == 0) return KVQ_ERR_EMPTY;
     if (c->device < 0 || c->device >= KVQ_STATIC_MAX_DEVICES) return KVQ_ERR_ARG;
-    const uint32_t gw = choose_warps(c, c->len[layer]);
+    const uint32_t gw = choose_warps(c, c->len[layer], (uint64_t)c->batch * c->q_heads);
     const size_t records = (size_t)c->batch * c->q_heads * decode_pslots((uint32_t)c->batch * c->q_heads, gw);
     if (records > (size_t)KVQ_STATIC_MAX_PARTIALS) return KVQ_ERR_TOO_LARGE;
     DeviceGuard guard(c->device);

@@ -311,3 +311,35 @@ def test_decode_step_host_matches_device_path(gu, oracle):
             oc.append(K, V, want_bits)
             gu.assert_attention_close(O, oc.decode_attn(Q), "host step %d" % step)
         gu.assert_store_equals_oracle(g, 0, oc)
+
+
+# ------------------------------------------------------------------ several causal query rows
+
+@pytest.mark.parametrize("T,n", [(1, 200), (4, 333), (8, 1500), (11, 90), (20, 700)])
+def test_attend_last_is_causal_attention_at_each_of_the_last_positions(gu, oracle, T, n):
+    """kvq_attend_last: query row i sits at position n - T + i and sees positions <= its own (Eq. 5 applied
+    at each of the last T positions).  The oracle computes every row on a cache truncated after its
+    position; rows 8 and up go through a second launch."""
+    import torch
+    from paper_2604_04722_b200 import binding as kq
+    rng = np.random.default_rng(1000 * T + n)
+    B, Hq, H = 2, 6, 2
+    bits = BITS[rng.choice(4, size=(B, n), p=[.4, .3, .2, .1])]
+    K, V = _kv(rng, B, n, H)
+    Q = rng.standard_normal((B, T, Hq, 64)).astype(np.float16)
+    oc = oracle.OracleCache(B, Hq, H)
+    oc.append(K, V, bits)
+    want = oc.attend_last(Q)
+    with gu.GpuCache(1, B, Hq, H, n) as g:
+        g.append(0, K[:, :n - T], V[:, :n - T], bits[:, :n - T])       # the cache, then the T new tokens at once
+        g.append(0, K[:, n - T:], V[:, n - T:], bits[:, n - T:])
+        Qd = gu.dev(Q.view(np.uint16))
+        for splits in (0, 3):
+            kq.kvq_set_splits(g.ctx, splits)
+            O = torch.zeros_like(Qd)
+            kq.kvq_attend_last(g.ctx, 0, Qd, O, T)
+            torch.cuda.synchronize()
+            gu.assert_attention_close(O.cpu().numpy().view(np.uint16), want, "T=%d n=%d splits=%d" % (T, n, splits))
+        # the last row is the ordinary decode step
+        gu.assert_attention_close(g.decode(0, np.ascontiguousarray(Q[:, T - 1])), want[:, T - 1], "last row")
+        assert kq.lib().kvq_attend_last(g.ctx, 0, Qd.data_ptr(), O.data_ptr(), n + 1, None) == kq.KVQ_ERR_ARG

@@ -175,3 +175,34 @@ def test_workload_table_matches_the_backbones():
     r = synth.bits_runs(0, 0, 0, 100000, c["cfg4"].mix, 16)
     changes = np.count_nonzero(np.diff(r.astype(int))) + 1
     assert 12 < 100000 / changes < 30          # mean run near 16 (equal neighbours merge)
+
+
+def test_attend_last_matches_library_causal_attention_and_ignores_the_future(oracle):
+    """Causal attention of the last T positions: an all-fp16 cache must equal a library routine with a
+    causal mask (fp64), and a row's result must not move when later tokens change."""
+    import torch
+    rng = np.random.default_rng(21)
+    B, Hq, H, n, T = 2, 4, 2, 60, 5
+    K = rng.standard_normal((B, n, H, 64)).astype(np.float16)
+    V = rng.standard_normal((B, n, H, 64)).astype(np.float16)
+    Q = rng.standard_normal((B, T, Hq, 64)).astype(np.float16)
+    oc = oracle.OracleCache(B, Hq, H)
+    oc.append(K, V, np.full((B, n), 16, np.uint8))
+    got = oc.attend_last(Q).view(np.float16).astype(np.float64)                    # [B][T][Hq][D]
+    q = torch.from_numpy(Q.astype(np.float64)).permute(0, 2, 1, 3)                 # [B][Hq][T][D]
+    k = torch.from_numpy(K.astype(np.float64)).permute(0, 2, 1, 3).repeat_interleave(Hq // H, 1)
+    v = torch.from_numpy(V.astype(np.float64)).permute(0, 2, 1, 3).repeat_interleave(Hq // H, 1)
+    mask = torch.ones(T, n, dtype=torch.bool).tril(diagonal=n - T)                 # row i sees keys <= n - T + i
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, attn_mask=mask).permute(0, 2, 1, 3).numpy()
+    assert np.max(np.abs(got - ref)) < 2e-3
+    # change the last token only: rows 0 .. T-2 stay bit-identical, the last row moves
+    K2, V2 = K.copy(), V.copy()
+    K2[:, -1] *= np.float16(-3.0)
+    V2[:, -1] += np.float16(5.0)
+    oc2 = oracle.OracleCache(B, Hq, H)
+    oc2.append(K2, V2, np.full((B, n), 16, np.uint8))
+    got2 = oc2.attend_last(Q)
+    assert np.array_equal(got2[:, :T - 1], oc.attend_last(Q)[:, :T - 1])
+    assert not np.array_equal(got2[:, T - 1], oc.attend_last(Q)[:, T - 1])
+    # one row is the plain decode step
+    assert np.array_equal(oc.attend_last(Q[:, -1:])[:, 0], oc.decode_attn(np.ascontiguousarray(Q[:, -1])))
