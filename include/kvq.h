@@ -141,6 +141,24 @@ int kvq_append_fused(kvq_ctx* ctx, int layer, const void* K, const void* V,
                      const float* feats, int n_new, uint8_t* bits_out_opt, void* stream);
 
 /*
+ * Ragged batches: the same append with a different number of new tokens per sequence.  K, V
+ * (and bits, or feats) keep n_max rows per sequence; sequence b appends its first
+ * host_lens[b] rows (host int [batch], 0 <= host_lens[b] <= n_max), the rest is ignored.
+ * Exactly one of bits (dev uint8 [batch][n_max]) and feats (dev fp32 [batch][n_max][4], the
+ * controller decides; bits_out_opt as in kvq_append_fused) is given, the other is NULL.
+ * Afterwards the sequences of the layer differ in length: kvq_seq_lens reports them,
+ * kvq_seq_len the longest, kvq_decode_attn attends for every sequence over what it holds
+ * (a sequence that holds nothing gets a zero row), kvq_export_range and kvq_attend_last are
+ * limited by the shortest.  Synchronizes the stream once (the lengths travel to the device).
+ */
+int kvq_append_ragged(kvq_ctx* ctx, int layer, const void* K, const void* V, const uint8_t* bits,
+                      const float* feats, int n_max, const int* host_lens, uint8_t* bits_out_opt,
+                      void* stream);
+
+/* Tokens cached per sequence in `layer` (host int [batch]; host-side mirror, no device access). */
+int kvq_seq_lens(kvq_ctx* ctx, int layer, int* host_lens_out);
+
+/*
  * Decode-step attention (Eq. 5) of one query row per (sequence, query head)
  * over every token cached in `layer`, dequantizing on the fly:
  * O = Softmax(q K^T / 8) V.  Q, O: dev fp16 [batch][q_heads][64].  fp32
@@ -213,7 +231,7 @@ int kvq_decode_step_host(kvq_ctx* ctx, int layer, const float* feats, const void
 /* Forget all cached tokens of every layer (counters go to 0, every arena block is free again). */
 int kvq_reset(kvq_ctx* ctx, void* stream);
 
-/* Tokens cached per sequence in `layer` (host-side mirror; no device access). */
+/* Tokens cached by the longest sequence of `layer` (host-side mirror; no device access). */
 int kvq_seq_len(kvq_ctx* ctx, int layer, int* host_len_out);
 
 /*

@@ -39,6 +39,8 @@ SIGNATURES = {
     "kvq_select_bits": (_i, [_vp, _vp, _i, _vp, _vp, _vp]),
     "kvq_append": (_i, [_vp, _i, _vp, _vp, _vp, _i, _vp]),
     "kvq_append_fused": (_i, [_vp, _i, _vp, _vp, _vp, _i, _vp, _vp]),
+    "kvq_append_ragged": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _i, _vp, _vp, _vp]),
+    "kvq_seq_lens": (_i, [_vp, _i, _vp]),
     "kvq_decode_attn": (_i, [_vp, _i, _vp, _vp, _vp]),
     "kvq_attend_last": (_i, [_vp, _i, _vp, _vp, _i, _vp]),
     "kvq_decode_attn_static": (_i, [_vp, _i, _vp, _vp, _vp]),
@@ -153,6 +155,20 @@ def kvq_append(ctx: int, layer: int, K, V, bits, n_new: int, stream=None) -> Non
 def kvq_append_fused(ctx: int, layer: int, K, V, feats, n_new: int, bits_out=None, stream=None) -> None:
     check(lib().kvq_append_fused(ctx, layer, _ptr(K), _ptr(V), _ptr(feats), n_new, _ptr(bits_out), _stream(stream)),
           "kvq_append_fused")
+
+
+def kvq_append_ragged(ctx: int, layer: int, K, V, bits, feats, n_max: int, lens, bits_out=None, stream=None) -> None:
+    import numpy as np
+    lens = np.ascontiguousarray(lens, dtype=np.int32)
+    check(lib().kvq_append_ragged(ctx, layer, _ptr(K), _ptr(V), _ptr(bits), _ptr(feats), n_max, lens.ctypes.data,
+                                  _ptr(bits_out), _stream(stream)), "kvq_append_ragged")
+
+
+def kvq_seq_lens(ctx: int, layer: int, batch: int):
+    import numpy as np
+    out = np.zeros(batch, np.int32)
+    check(lib().kvq_seq_lens(ctx, layer, out.ctypes.data), "kvq_seq_lens")
+    return out
 
 
 def kvq_decode_attn(ctx: int, layer: int, Q, O, stream=None) -> None:

@@ -46,7 +46,14 @@ struct AppendParams {
     const uint32_t* counts_in;         // [batch][4] of this layer
     uint32_t* counts_out;              // [batch][4] of this layer
     int layer, n_new, pos0, nchunks, heads_per_group;
+    // Ragged batches: tokens each sequence adds in this call (nullptr: n_new for all; the input tensors keep
+    // n_new rows per sequence) and position of each sequence's first new token (nullptr: pos0 for all).
+    const int* lens;
+    const int* pos;
 };
+
+__device__ __forceinline__ int new_tokens_of(const AppendParams& p, int b) { return p.lens ? p.lens[b] : p.n_new; }
+__device__ __forceinline__ int first_pos_of(const AppendParams& p, int b) { return p.pos ? p.pos[b] : p.pos0; }
 
 // Class of one token from its bit-width; anything outside {2,4,8,16} is kept as fp16 and flagged.
 __device__ __forceinline__ int class_of_bits(int bits, uint32_t* flags) {
@@ -66,7 +73,7 @@ k_classify(AppendParams p) {
     __shared__ uint32_t wtot[kChunkTokens / 32][4];
     const int chunk = blockIdx.x, b = blockIdx.y;
     const int t = chunk * kChunkTokens + threadIdx.x;
-    const bool live = t < p.n_new;
+    const bool live = t < new_tokens_of(p, b);
     int c = -1;
     if (FUSED) {
         controller_stage(sW, p.ctrl, p.hidden);
@@ -243,7 +250,7 @@ k_quant_pack(AppendParams p) {
     const int chunk = blockIdx.x, hg = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tok_i = chunk * kChunkTokens + threadIdx.x;
-    const bool live = tok_i < p.n_new;
+    const bool live = tok_i < new_tokens_of(p, b);
     const size_t tok = (size_t)b * p.n_new + tok_i;
 
     // ---- class of this thread's token
@@ -297,7 +304,7 @@ k_quant_pack(AppendParams p) {
         for (int w = 0; w < warp; ++w) rank += wtot[w][c];
         list[c][rank] = (uint8_t)threadIdx.x;
         if (hg == 0)
-            p.store.index[((size_t)p.layer * p.store.batch + b) * p.store.max_ctx + p.pos0 + tok_i] =
+            p.store.index[((size_t)p.layer * p.store.batch + b) * p.store.max_ctx + first_pos_of(p, b) + tok_i] =
                 ((uint32_t)c << 30) | (base[c] + rank);
     }
     uint32_t ncls[4];                                  // tokens of each class in this chunk
@@ -520,7 +527,7 @@ k_append_token(AppendParams p) {
     }
     const uint32_t slot = c == 0 ? fill.x : c == 1 ? fill.y : c == 2 ? fill.z : fill.w;
     if (blockIdx.x == 0 && lane == 0) {
-        p.store.index[((size_t)p.layer * p.store.batch + b) * p.store.max_ctx + p.pos0] = ((uint32_t)c << 30) | slot;
+        p.store.index[((size_t)p.layer * p.store.batch + b) * p.store.max_ctx + first_pos_of(p, b)] = ((uint32_t)c << 30) | slot;
         *reinterpret_cast<uint4*>(p.counts_out + (size_t)b * 4) =
             make_uint4(fill.x + (c == 0), fill.y + (c == 1), fill.z + (c == 2), fill.w + (c == 3));
         if (FUSED && p.bits_out) p.bits_out[b] = (uint8_t)pool_bits(c);

@@ -690,7 +690,8 @@ k_decode_attn(DecodeParams P) {
                     }
                 }
             }
-            reinterpret_cast<__half2*>(P.O + qo)[lane] = __floats2half2_rn(o0 / L, o1 / L);
+            const float inv = L > 0.f ? 1.0f / L : 0.f;            // a sequence that holds no token yet gets zeros
+            reinterpret_cast<__half2*>(P.O + qo)[lane] = __floats2half2_rn(o0 * inv, o1 * inv);
             if (lane == 0) P.part_cnt[u] = 0;
         }
     }
@@ -701,10 +702,13 @@ k_decode_attn(DecodeParams P) {
 // (position len - t_total + i) sees every slot of pool c except those of the later rows of that class:
 // vis[b][i - t0][c] = fill[b][c] - #{ j > i : class(position of row j) == c }, for rows t0 .. t0+tq.
 // grid = batch, block = tq threads.
-__global__ void k_visible_counts(StoreView s, const uint32_t* __restrict__ fill, int layer, int len, uint32_t t_total,
-                                 uint32_t t0, uint32_t tq, uint32_t* __restrict__ vis) {
+// lens: cached tokens per sequence (nullptr: `len` for all).
+__global__ void k_visible_counts(StoreView s, const uint32_t* __restrict__ fill, int layer, int len,
+                                 const int* __restrict__ lens, uint32_t t_total, uint32_t t0, uint32_t tq,
+                                 uint32_t* __restrict__ vis) {
     const uint32_t b = blockIdx.x, il = threadIdx.x;
     if (il >= tq) return;
+    if (lens) len = lens[b];
     const uint32_t i = t0 + il;
     uint32_t l0 = 0, l1 = 0, l2 = 0, l3 = 0;
     const uint32_t* idx = s.index + ((size_t)layer * s.batch + b) * s.max_ctx + (len - (int)t_total);

@@ -5,6 +5,7 @@
 
 #include <cstdio>
 #include <cstdlib>
+#include <algorithm>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -27,7 +28,10 @@ struct kvq_ctx {
     uint32_t* table = nullptr;           // block tables of all streams
     uint32_t* arena_used = nullptr;      // device counter of blocks handed out
     uint32_t* counts = nullptr;          // [2][layers][batch][4], double-buffered pool fills
-    std::vector<int> len;                // host mirror: tokens per sequence, per layer
+    std::vector<int> len;                // host mirror: tokens of the longest sequence, per layer
+    std::vector<int> lens;               // host mirror: tokens per (layer, sequence)
+    std::vector<char> ragged;            // per layer: sequences differ in length
+    int* d_lens = nullptr;               // device scratch [3][batch]: this call's new tokens, first positions, lengths
     std::vector<int> cur;                // which counts buffer is current, per layer
     uint8_t* cls = nullptr;              // append scratch [batch][max_ctx]
     uint4* hist = nullptr;               // append scratch [batch][max chunks]
@@ -98,6 +102,7 @@ void free_all(kvq_ctx* c) {
     cudaFree(c->part_ml);
     cudaFree(c->part_cnt);
     cudaFree(c->vis);
+    cudaFree(c->d_lens);
     cudaFree(c->flags);
     cudaFree(c->st_feats);
     cudaFree(c->st_K);
@@ -118,11 +123,20 @@ int check_layer(kvq_ctx* c, int layer) { return (c && layer >= 0 && layer < c->l
 
 size_t controller_smem(int hidden) { return sizeof(float) * (size_t)controller_floats(hidden); }
 
-// Shared by kvq_append and kvq_append_fused.
+// Shared by kvq_append, kvq_append_fused and kvq_append_ragged.  host_lens: tokens each sequence adds (host
+// int [batch], each 0..n_new) or nullptr for n_new everywhere.
 int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8_t* bits, const float* feats,
-                uint8_t* bits_out, int n_new, cudaStream_t st) {
+                uint8_t* bits_out, int n_new, const int* host_lens, cudaStream_t st) {
     if (check_layer(c, layer) != KVQ_OK || n_new < 0) return KVQ_ERR_ARG;
     if (n_new == 0) return KVQ_OK;
+    int* cur_lens = &c->lens[(size_t)layer * c->batch];
+    bool call_ragged = false;
+    if (host_lens) {
+        for (int b = 0; b < c->batch; ++b) {
+            if (host_lens[b] < 0 || host_lens[b] > n_new) return KVQ_ERR_ARG;
+            call_ragged = call_ragged || host_lens[b] != n_new;
+        }
+    }
     if (!K || !V || !aligned16(K) || !aligned16(V)) return KVQ_ERR_ARG;
     const bool fused = feats != nullptr;
     if (fused) {
@@ -131,7 +145,8 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
     } else if (!bits) {
         return KVQ_ERR_ARG;
     }
-    if (c->len[layer] + n_new > c->max_ctx) return KVQ_ERR_CAPACITY;
+    for (int b = 0; b < c->batch; ++b)
+        if (cur_lens[b] + (host_lens ? host_lens[b] : n_new) > c->max_ctx) return KVQ_ERR_CAPACITY;
     DeviceGuard guard(c->device);
 
     AppendParams p{};
@@ -150,6 +165,17 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
     p.layer = layer;
     p.n_new = n_new;
     p.pos0 = c->len[layer];
+    if (call_ragged || c->ragged[layer]) {             // per-sequence counts and positions travel with the call
+        std::vector<int> blk(2 * (size_t)c->batch);
+        for (int b = 0; b < c->batch; ++b) {
+            blk[b] = host_lens ? host_lens[b] : n_new;
+            blk[c->batch + b] = cur_lens[b];
+        }
+        KVQ_CUDA(c, cudaMemcpyAsync(c->d_lens, blk.data(), sizeof(int) * blk.size(), cudaMemcpyHostToDevice, st));
+        KVQ_CUDA(c, cudaStreamSynchronize(st));        // blk is pageable and about to go out of scope
+        p.lens = c->d_lens;
+        p.pos = c->d_lens + c->batch;
+    }
     p.nchunks = (n_new + kChunkTokens - 1) / kChunkTokens;
     // enough CTAs to fill the device: split the KV heads into groups when chunks x batch is small
     int want_groups = (2 * c->sm_count + p.nchunks * c->batch - 1) / (p.nchunks * c->batch);
@@ -159,7 +185,7 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
 
     const size_t smem = fused ? controller_smem(c->hidden) : 0;
     dim3 grid_q(p.nchunks, groups, c->batch);
-    if (n_new == 1 && (!fused || c->hidden == 32)) {                   // a decode step: one warp per 16 heads
+    if (n_new == 1 && !call_ragged && (!fused || c->hidden == 32)) {   // a decode step: one warp per 16 heads
         dim3 grid_t((c->kv_heads + 15) / 16, c->batch);
         if (fused) k_append_token<true><<<grid_t, 32, 0, st>>>(p);
         else k_append_token<false><<<grid_t, 32, 0, st>>>(p);
@@ -178,8 +204,21 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
     }
     KVQ_CUDA(c, cudaGetLastError());
     c->cur[layer] ^= 1;
-    c->len[layer] += n_new;
+    int longest = 0;
+    for (int b = 0; b < c->batch; ++b) {
+        cur_lens[b] += host_lens ? host_lens[b] : n_new;
+        longest = cur_lens[b] > longest ? cur_lens[b] : longest;
+    }
+    c->len[layer] = longest;
+    c->ragged[layer] = c->ragged[layer] || call_ragged;
     return KVQ_OK;
+}
+
+// Shortest sequence of a layer.
+int min_len(const kvq_ctx* c, int layer) {
+    int m = c->lens[(size_t)layer * c->batch];
+    for (int b = 1; b < c->batch; ++b) m = c->lens[(size_t)layer * c->batch + b] < m ? c->lens[(size_t)layer * c->batch + b] : m;
+    return m;
 }
 
 // Number of working warps of a decode launch (the x axis is cut into that many equal parts).
@@ -301,6 +340,8 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
     c->max_ctx = max_ctx;
     c->batch = batch;
     c->len.assign(layers, 0);
+    c->lens.assign((size_t)layers * batch, 0);
+    c->ragged.assign(layers, 0);
     c->cur.assign(layers, 0);
     StoreView& s = c->store;
     s.layers = layers;
@@ -343,6 +384,7 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
     ok = ok && dev_alloc(c, &c->part_ml, sizeof(float2) * max_partial_records(c)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_cnt, sizeof(uint32_t) * units * kMaxQueryRows) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->vis, sizeof(uint32_t) * 4 * (size_t)batch * kMaxQueryRows) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->d_lens, sizeof(int) * 3 * (size_t)batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->flags, sizeof(uint32_t)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_feats, sizeof(float) * 4 * batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_K, sizeof(__half) * (size_t)batch * kv_heads * kHeadDim) == cudaSuccess;
@@ -427,13 +469,26 @@ int kvq_select_bits(kvq_ctx* c, const float* feats, int n, uint8_t* bits, float*
 
 int kvq_append(kvq_ctx* c, int layer, const void* K, const void* V, const uint8_t* bits, int n_new, void* stream) {
     if (!c) return KVQ_ERR_ARG;
-    return append_impl(c, layer, K, V, bits, nullptr, nullptr, n_new, static_cast<cudaStream_t>(stream));
+    return append_impl(c, layer, K, V, bits, nullptr, nullptr, n_new, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 int kvq_append_fused(kvq_ctx* c, int layer, const void* K, const void* V, const float* feats, int n_new,
                      uint8_t* bits_out_opt, void* stream) {
     if (!c || (n_new > 0 && !feats)) return KVQ_ERR_ARG;
-    return append_impl(c, layer, K, V, nullptr, feats, bits_out_opt, n_new, static_cast<cudaStream_t>(stream));
+    return append_impl(c, layer, K, V, nullptr, feats, bits_out_opt, n_new, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+int kvq_append_ragged(kvq_ctx* c, int layer, const void* K, const void* V, const uint8_t* bits, const float* feats,
+                      int n_max, const int* host_lens, uint8_t* bits_out_opt, void* stream) {
+    if (!c || !host_lens || (!bits && !feats) || (bits && feats)) return KVQ_ERR_ARG;
+    return append_impl(c, layer, K, V, bits, feats, feats ? bits_out_opt : nullptr, n_max, host_lens,
+                       static_cast<cudaStream_t>(stream));
+}
+
+int kvq_seq_lens(kvq_ctx* c, int layer, int* host_lens_out) {
+    if (check_layer(c, layer) != KVQ_OK || !host_lens_out) return KVQ_ERR_ARG;
+    for (int b = 0; b < c->batch; ++b) host_lens_out[b] = c->lens[(size_t)layer * c->batch + b];
+    return KVQ_OK;
 }
 
 int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream) {
@@ -460,13 +515,20 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
 int kvq_attend_last(kvq_ctx* c, int layer, const void* Q, void* O, int n_queries, void* stream) {
     if (check_layer(c, layer) != KVQ_OK || !Q || !O || n_queries < 1) return KVQ_ERR_ARG;
     if (c->len[layer] == 0) return KVQ_ERR_EMPTY;
-    if (n_queries > c->len[layer]) return KVQ_ERR_ARG;
+    if (n_queries > min_len(c, layer)) return KVQ_ERR_ARG;
     DeviceGuard guard(c->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int* d_len = nullptr;
+    if (c->ragged[layer]) {
+        KVQ_CUDA(c, cudaMemcpyAsync(c->d_lens + 2 * c->batch, &c->lens[(size_t)layer * c->batch], sizeof(int) * c->batch,
+                                    cudaMemcpyHostToDevice, st));
+        KVQ_CUDA(c, cudaStreamSynchronize(st));
+        d_len = c->d_lens + 2 * c->batch;
+    }
     for (int t0 = 0; t0 < n_queries; t0 += kMaxQueryRows) {
         const int tq = n_queries - t0 < kMaxQueryRows ? n_queries - t0 : kMaxQueryRows;
         k_visible_counts<<<c->batch, tq, 0, st>>>(c->store, counts_of(c, c->cur[layer], layer), layer, c->len[layer],
-                                                  (uint32_t)n_queries, (uint32_t)t0, (uint32_t)tq, c->vis);
+                                                  d_len, (uint32_t)n_queries, (uint32_t)t0, (uint32_t)tq, c->vis);
         const uint64_t units = (uint64_t)c->batch * tq * c->q_heads;
         DecodeParams p{};
         fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, choose_warps(c, c->len[layer], units), p);
@@ -554,9 +616,11 @@ int kvq_reset(kvq_ctx* c, void* stream) {
     KVQ_CUDA(c, cudaMemsetAsync(c->counts, 0, sizeof(uint32_t) * 2 * (size_t)c->layers * c->batch * 4,
                                 static_cast<cudaStream_t>(stream)));
     KVQ_CUDA(c, cudaMemsetAsync(c->arena_used, 0, sizeof(uint32_t), static_cast<cudaStream_t>(stream)));
+    std::fill(c->lens.begin(), c->lens.end(), 0);
     for (int l = 0; l < c->layers; ++l) {
         c->len[l] = 0;
         c->cur[l] = 0;
+        c->ragged[l] = 0;
     }
     return KVQ_OK;
 }
@@ -575,7 +639,7 @@ int kvq_set_splits(kvq_ctx* c, int splits) {
 
 int kvq_export_range(kvq_ctx* c, int layer, int pos0, int n, uint8_t* bits, uint32_t* pool_slot, void* k_codes,
                      void* v_codes, uint16_t* k_meta, uint16_t* v_meta, void* stream) {
-    if (check_layer(c, layer) != KVQ_OK || pos0 < 0 || n < 0 || pos0 + n > c->len[layer]) return KVQ_ERR_ARG;
+    if (check_layer(c, layer) != KVQ_OK || pos0 < 0 || n < 0 || pos0 + n > min_len(c, layer)) return KVQ_ERR_ARG;
     if (n == 0) return KVQ_OK;
     if ((k_codes && !aligned16(k_codes)) || (v_codes && !aligned16(v_codes))) return KVQ_ERR_ARG;
     DeviceGuard guard(c->device);
@@ -585,7 +649,8 @@ int kvq_export_range(kvq_ctx* c, int layer, int pos0, int n, uint8_t* bits, uint
 
 int kvq_export_token(kvq_ctx* c, int layer, int b, int pos, uint8_t* bits, uint32_t* pool_slot, void* k_codes,
                      void* v_codes, uint16_t* k_meta, uint16_t* v_meta) {
-    if (check_layer(c, layer) != KVQ_OK || b < 0 || b >= c->batch || pos < 0 || pos >= c->len[layer])
+    if (check_layer(c, layer) != KVQ_OK || b < 0 || b >= c->batch || pos < 0 ||
+        pos >= c->lens[(size_t)layer * c->batch + (b < 0 || b >= c->batch ? 0 : b)])
         return KVQ_ERR_ARG;
     DeviceGuard guard(c->device);
     const size_t row = (size_t)c->kv_heads * KVQ_EXPORT_ROW_BYTES, meta = (size_t)c->kv_heads * 4;
