@@ -489,7 +489,7 @@ def main():
                     help="shorter cached context than the workload's 32768, for profiler captures that must "
                          "stay small; the printed config names it and the line is not a benchmark result")
     ap.add_argument("--workload", choices=sorted(synth.CONFIGS), default="cfg5",
-                    help="cfg5 (default) is the workload the metric is quoted on; the others are reported in DESIGN.md")
+                    help="cfg5 (default) is the workload the metric is quoted on; cfg1..cfg4 are the other SmolLM-shaped workloads")
     ap.add_argument("--uniform-bits", type=int, choices=[2, 4, 8, 16], default=0,
                     help="store every prefill token at this precision (the static baselines of cfg4)")
     ap.add_argument("--batch", type=int, default=0,
