@@ -175,6 +175,56 @@ def decode_attn(Q, q_heads: int, kv_heads: int, bits, kc, km, vc, vm,
     return (out, out64) if want64 else out
 
 
+def decode_probs(Q, q_heads: int, kv_heads: int, bits, kc, km, vc, vm) -> np.ndarray:
+    """The attention weights of ``decode_attn``: fp64 [B][Hq][n]."""
+    Q = _u16(Q)
+    B, Hq, D = Q.shape
+    bits = _c(bits, np.uint8)
+    n = bits.shape[1]
+    kc, vc = _c(kc, np.uint8), _c(vc, np.uint8)
+    km, vm = _c(km, np.uint16), _c(vm, np.uint16)
+    probs = np.empty((B, Hq, n), dtype=np.float64)
+    rc = lib().oracle_decode_probs(_p(Q), C.c_int(B), C.c_int(q_heads), C.c_int(kv_heads), C.c_int(D), C.c_int(n),
+                                   _p(bits), _p(kc), _p(km), _p(vc), _p(vm), _p(probs))
+    if rc != 0:
+        raise ValueError("oracle_decode_probs failed: %d" % rc)
+    return probs
+
+
+# ---- token-level saliency features (Section 3.2), plain fp64 numpy from the definitions
+
+def token_entropy(logits) -> np.ndarray:
+    """Eq. 14: H_t = -sum_v p_t(v) log p_t(v), p_t = Softmax(z_t); logits [n][V] -> [n] (natural log)."""
+    z = np.asarray(logits, dtype=np.float64)
+    z = z - z.max(axis=1, keepdims=True)
+    p = np.exp(z)
+    p /= p.sum(axis=1, keepdims=True)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        t = np.where(p > 0, p * np.log(p), 0.0)
+    return -t.sum(axis=1)
+
+
+def token_confidence(logits) -> np.ndarray:
+    """The confidence term C_t of Eq. 17, which the paper names without defining: taken as the largest
+    next-token probability, max_v Softmax(z_t)_v."""
+    z = np.asarray(logits, dtype=np.float64)
+    z = z - z.max(axis=1, keepdims=True)
+    p = np.exp(z)
+    return (p / p.sum(axis=1, keepdims=True)).max(axis=1)
+
+
+def token_rarity(token_ids, counts, total: int, observed: int) -> np.ndarray:
+    """Eq. 15: R_t = -log((c(x_t) + 1) / (N + |V_obs| + 1)); counts [V] running counts, total = N."""
+    c = np.asarray(counts, dtype=np.float64)[np.asarray(token_ids, dtype=np.int64)]
+    return -np.log((c + 1.0) / (float(total) + float(observed) + 1.0))
+
+
+def attention_variance(probs) -> np.ndarray:
+    """Eq. 16: V_t = (1/h) sum_i Var(A_i), with Var taken over the cached positions the query row of head i
+    attends to (population variance); probs [B][h][n] -> [B]."""
+    return np.var(np.asarray(probs, dtype=np.float64), axis=2).mean(axis=1)
+
+
 class OracleCache:
     """Position-ordered mixed-precision cache of one layer: append rows, then attend."""
 
@@ -207,6 +257,9 @@ class OracleCache:
     def decode_attn(self, Q, want64: bool = False):
         return decode_attn(Q, self.Hq, self.Hkv, self.bits, self.kc, self.km,
                            self.vc, self.vm, want64=want64)
+
+    def decode_probs(self, Q) -> np.ndarray:
+        return decode_probs(Q, self.Hq, self.Hkv, self.bits, self.kc, self.km, self.vc, self.vm)
 
     def attend_last(self, Q):
         """Causal attention of the last T cached positions (Eq. 5 at each of them): Q fp16 [B][T][Hq][D];

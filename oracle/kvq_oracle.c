@@ -358,7 +358,7 @@ static void attend_one_head(const uint16_t *q, int D, int n, const uint8_t *bits
                             const uint8_t *kc, const uint16_t *km,
                             const uint8_t *vc, const uint16_t *vm,
                             size_t row_stride, size_t meta_stride,
-                            double *out)
+                            double *out, double *probs)
 {
     double *z = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
     float *row = (float *)malloc(sizeof(float) * (size_t)D);
@@ -382,6 +382,8 @@ static void attend_one_head(const uint16_t *q, int D, int n, const uint8_t *bits
         out[i] = 0.0;
     for (int t = 0; t < n; ++t) {
         double p = z[t] / denom;
+        if (probs)
+            probs[t] = p;
         oracle_dequantize_row(vc + t * row_stride, vm + t * meta_stride, D, bits[t], row);
         for (int i = 0; i < D; ++i)
             out[i] += p * (double)row[i];
@@ -416,12 +418,42 @@ int oracle_decode_attn(const uint16_t *q, int batch, int q_heads, int kv_heads, 
         attend_one_head(q + (size_t)u * D, D, n, bits + (size_t)b * n,
                         kcodes + base * 2 * D, kmeta + base * 2,
                         vcodes + base * 2 * D, vmeta + base * 2,
-                        row_stride, meta_stride, acc);
+                        row_stride, meta_stride, acc, NULL);
         for (int i = 0; i < D; ++i) {
             out[(size_t)u * D + i] = double_to_half(acc[i]);
             if (out64)
                 out64[(size_t)u * D + i] = acc[i];
         }
+        free(acc);
+    }
+    return ORACLE_OK;
+}
+
+/* The attention weights of Eq. 5 themselves: probs [batch][q_heads][n] (fp64), same arguments as
+ * oracle_decode_attn.  Used for the attention-variance feature of Eq. 16. */
+int oracle_decode_probs(const uint16_t *q, int batch, int q_heads, int kv_heads, int D, int n,
+                        const uint8_t *bits,
+                        const uint8_t *kcodes, const uint16_t *kmeta,
+                        const uint8_t *vcodes, const uint16_t *vmeta,
+                        double *probs)
+{
+    if (!q || !bits || !kcodes || !kmeta || !vcodes || !vmeta || !probs)
+        return ORACLE_ERR_ARG;
+    if (batch < 1 || q_heads < 1 || kv_heads < 1 || q_heads % kv_heads || n < 1 || D < 1)
+        return ORACLE_ERR_ARG;
+    int g = q_heads / kv_heads;
+    size_t row_stride = (size_t)kv_heads * 2 * D;
+    size_t meta_stride = (size_t)kv_heads * 2;
+    int units = batch * q_heads;
+#pragma omp parallel for schedule(dynamic)
+    for (int u = 0; u < units; ++u) {
+        int b = u / q_heads, h = u % q_heads, kvh = h / g;
+        double *acc = (double *)malloc(sizeof(double) * (size_t)D);
+        size_t base = (size_t)b * n * kv_heads + kvh;
+        attend_one_head(q + (size_t)u * D, D, n, bits + (size_t)b * n,
+                        kcodes + base * 2 * D, kmeta + base * 2,
+                        vcodes + base * 2 * D, vmeta + base * 2,
+                        row_stride, meta_stride, acc, probs + (size_t)u * n);
         free(acc);
     }
     return ORACLE_OK;
