@@ -331,11 +331,20 @@ def run_ours(args, wl):
 
     step_no = [0]
 
+    # The timed loop passes plain addresses to the C calls: slicing tensors and re-deriving their pointers
+    # costs more host time per call than a small workload's kernels take.
+    clib = kq.lib()
+    ptr = lambda t: [t[i].data_ptr() for i in range(t.shape[0])]
+    k_p, v_p, f_p, q_p, sb_p = ptr(k_d), ptr(v_d), ptr(f_d), ptr(q_d), ptr(step_bits_d)
+    O_p = O_d.data_ptr()
+
     def one_step():
         s = step_no[0]
         for layer in range(L):
-            kq.kvq_append_fused(ctx, layer, k_d[s], v_d[s], f_d[s], 1, step_bits_d[s], stream)
-            kq.kvq_decode_attn(ctx, layer, q_d[s], O_d, stream)
+            rc = clib.kvq_append_fused(ctx, layer, k_p[s], v_p[s], f_p[s], 1, sb_p[s], stream)
+            rc = rc or clib.kvq_decode_attn(ctx, layer, q_p[s], O_p, stream)
+            if rc:
+                raise kq.KvqError(rc, "decode step")
         step_no[0] = s + 1
 
     _, resident_layer0, _ = kq.kvq_stats(ctx, 0, B)
@@ -400,11 +409,14 @@ def run_ours(args, wl):
         pin(q_steps.view(np.int16))
     O_h = torch.zeros((B, Hq, D), dtype=torch.int16).pin_memory()
 
+    fh_p, kh_p, vh_p, qh_p, Oh_p = ptr(f_h), ptr(k_h), ptr(v_h), ptr(q_h), O_h.data_ptr()
+
     def one_step_host():
         s = step_no[0]
         for layer in range(L):
-            kq.kvq_decode_step_host(ctx, layer, f_h[s].data_ptr(), k_h[s].data_ptr(), v_h[s].data_ptr(),
-                                    q_h[s].data_ptr(), O_h.data_ptr(), None, stream)
+            rc = clib.kvq_decode_step_host(ctx, layer, fh_p[s], kh_p[s], vh_p[s], qh_p[s], Oh_p, None, stream)
+            if rc:
+                raise kq.KvqError(rc, "decode step from host buffers")
         step_no[0] = s + 1
 
     for _ in range(e2e_warm):

@@ -170,6 +170,34 @@ int kvq_seq_lens(kvq_ctx* ctx, int layer, int* host_lens_out);
 int kvq_decode_attn(kvq_ctx* ctx, int layer, const void* Q, void* O, void* stream);
 
 /*
+ * kvq_decode_attn that also returns the attention-variance feature of Eq. 16 for the step's
+ * tokens: var_out (dev fp32 [batch]) receives V = (1/h) sum over the query heads of the variance
+ * of that head's attention weights over the cached tokens of the sequence.  (The paper takes
+ * the last transformer layer; which layer to ask is the caller's choice.)  One extra
+ * multiply-add per cached token and a small second kernel.
+ */
+int kvq_decode_attn_var(kvq_ctx* ctx, int layer, const void* Q, void* O, float* var_out, void* stream);
+
+/*
+ * The controller's input vector of Eq. 17 for n tokens, s_t = [H_t, R_t, V_t, C_t], computed on
+ * the device.  No handle is needed.
+ *   logits      dev [n][vocab], fp16 (logits_are_fp32 == 0) or fp32: the pre-softmax scores z_t
+ *   H_t         entropy of Softmax(z_t), natural logarithm (Eq. 14)
+ *   C_t         confidence; the paper names it without a definition: max_v Softmax(z_t)_v
+ *   token_ids   dev int32 [n], counts dev uint32 [vocab], total_count = N, observed_tokens =
+ *               |V_obs|: R_t = -log((counts[token] + 1) / (N + |V_obs| + 1)) (Eq. 15)
+ *   attn_var_opt dev fp32 [n] or NULL (then V_t = 0): the attention variance of Eq. 16, e.g. from
+ *               kvq_decode_attn_var
+ *   feats       dev fp32 [n][4] in the order H, R, V, C of Eq. 17 (16-byte aligned)
+ * The logits are read once; rows are read with 16-byte loads when vocab % 8 == 0 and the base
+ * is 32-byte aligned.  The library treats the controller's inputs as four opaque numbers, so a
+ * controller must have been trained on this order to be fed from here.
+ */
+int kvq_token_features(const void* logits, int logits_are_fp32, int n, int vocab,
+                       const int32_t* token_ids, const uint32_t* counts, uint64_t total_count,
+                       uint32_t observed_tokens, const float* attn_var_opt, float* feats, void* stream);
+
+/*
  * Causal attention of several query rows over the cache (Eq. 5 applied at each of the last
  * n_queries cached positions): query row i belongs to the token at position len - n_queries + i
  * and attends over positions <= its own, the rows after it stay invisible.  This is what a

@@ -42,6 +42,8 @@ SIGNATURES = {
     "kvq_append_ragged": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _i, _vp, _vp, _vp]),
     "kvq_seq_lens": (_i, [_vp, _i, _vp]),
     "kvq_decode_attn": (_i, [_vp, _i, _vp, _vp, _vp]),
+    "kvq_decode_attn_var": (_i, [_vp, _i, _vp, _vp, _vp, _vp]),
+    "kvq_token_features": (_i, [_vp, _i, _i, _i, _vp, _vp, C.c_uint64, C.c_uint32, _vp, _vp, _vp]),
     "kvq_attend_last": (_i, [_vp, _i, _vp, _vp, _i, _vp]),
     "kvq_decode_attn_static": (_i, [_vp, _i, _vp, _vp, _vp]),
     "kvq_decode_step_host": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -173,6 +175,17 @@ def kvq_seq_lens(ctx: int, layer: int, batch: int):
 
 def kvq_decode_attn(ctx: int, layer: int, Q, O, stream=None) -> None:
     check(lib().kvq_decode_attn(ctx, layer, _ptr(Q), _ptr(O), _stream(stream)), "kvq_decode_attn")
+
+
+def kvq_decode_attn_var(ctx: int, layer: int, Q, O, var_out, stream=None) -> None:
+    check(lib().kvq_decode_attn_var(ctx, layer, _ptr(Q), _ptr(O), _ptr(var_out), _stream(stream)), "kvq_decode_attn_var")
+
+
+def kvq_token_features(logits, logits_are_fp32: bool, n: int, vocab: int, token_ids, counts, total_count: int,
+                       observed_tokens: int, attn_var, feats, stream=None) -> None:
+    check(lib().kvq_token_features(_ptr(logits), int(bool(logits_are_fp32)), n, vocab, _ptr(token_ids), _ptr(counts),
+                                   total_count, observed_tokens, _ptr(attn_var), _ptr(feats), _stream(stream)),
+          "kvq_token_features")
 
 
 def kvq_attend_last(ctx: int, layer: int, Q, O, n_queries: int, stream=None) -> None:

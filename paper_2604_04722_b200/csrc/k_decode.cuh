@@ -98,6 +98,8 @@ struct DecodeParams {
     float* part_o;                 // [units][pslots][64]  unnormalised
     float2* part_ml;               // [units][pslots]      (m in log2 units, l)
     uint32_t* part_cnt;            // [units] partials delivered so far; zero between launches
+    float* part_s2;                // [units][pslots] sum of p^2 (statistics variant only)
+    float* unit_var;               // [units] variance of the unit's attention weights (statistics variant only)
     int layer, group;              // group = q_heads / kv_heads
     // Query rows per sequence.  A decode step has one (tq = t_total = 1, t0 = 0).  With several (the last
     // t_total cached tokens each ask, causally), a launch serves rows t0 .. t0+tq of every sequence and
@@ -209,14 +211,18 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-struct Softmax {
+// STATS: also keep the sum of squared weights (for the attention-variance feature of Eq. 16).
+template <bool STATS>
+struct SoftmaxT {
     float m, l, bsum;              // running max (log2 units), sum of p, sum of p * zero-point
     float thr;                     // m + kRescaleSlack: a logit above it forces a rescale
+    float s2;                      // sum of p^2 (STATS only)
 };
 
 // Fold a tile's logits into the running state and return this lane's p.  The running maximum
 // is only raised when some logit exceeds it by more than kRescaleSlack (one vote per tile).
-__device__ __forceinline__ float softmax_step(Softmax& st, float (&acc)[kHalfDim], float y) {
+template <bool STATS>
+__device__ __forceinline__ float softmax_step(SoftmaxT<STATS>& st, float (&acc)[kHalfDim], float y) {
     if (__any_sync(0xffffffffu, y > st.thr)) {                     // warp-uniform
         const float tmax = warp_max(y);
         const float f = fast_exp2(st.m - tmax);
@@ -224,11 +230,13 @@ __device__ __forceinline__ float softmax_step(Softmax& st, float (&acc)[kHalfDim
         st.thr = tmax + kRescaleSlack;
         st.l *= f;
         st.bsum *= f;
+        if (STATS) st.s2 *= f * f;
 #pragma unroll
         for (int j = 0; j < kHalfDim; ++j) acc[j] *= f;
     }
     const float p = fast_exp2(y - st.m);
     st.l += p;
+    if (STATS) st.s2 = fmaf(p, p, st.s2);
     return p;
 }
 
@@ -310,8 +318,9 @@ struct Quantized {
         k.meta = *reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 0, t));
         return k;
     }
+    template <class SM>
     __device__ static __forceinline__ void tile(const uint8_t* rec, const KIn& kin, bool valid, int half, int t,
-                                                const uint32_t (&qreg)[kQRegs], const QueryInfo& qi, Softmax& st,
+                                                const uint32_t (&qreg)[kQRegs], const QueryInfo& qi, SM& st,
                                                 float (&acc)[kHalfDim]) {
         uint32_t w[WORDS];
 #pragma unroll
@@ -371,8 +380,9 @@ struct Fp16Rows {
     __device__ static __forceinline__ void leave(float (&)[kHalfDim]) {}
     struct KIn {};                                     // fp16 rows are read where they are used
     __device__ static __forceinline__ KIn load_k(const uint8_t*, int, int) { return KIn{}; }
+    template <class SM>
     __device__ static __forceinline__ void tile(const uint8_t* rec, const KIn&, bool valid, int half, int t,
-                                                const uint32_t (&qreg)[kQRegs], const QueryInfo&, Softmax& st,
+                                                const uint32_t (&qreg)[kQRegs], const QueryInfo&, SM& st,
                                                 float (&acc)[kHalfDim]) {
         float d[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -427,6 +437,8 @@ __device__ __forceinline__ uint32_t scale_by_fraction(uint32_t n, uint32_t a, ui
 }
 
 // grid = ceil(gw / kDecodeWarps), block = kDecodeThreads, dynamic smem = kDecodeSmemBytes.
+// STATS: also emit, per unit, the variance of its attention weights over the cached tokens.
+template <bool STATS>
 __global__ void __launch_bounds__(kDecodeThreads, KVQ_DECODE_MIN_CTAS)
 k_decode_attn(DecodeParams P) {
     extern __shared__ __align__(128) uint8_t ring[];   // [warps][stages][kStageBytes]
@@ -543,7 +555,7 @@ k_decode_attn(DecodeParams P) {
         int in_flight = 0;
         for (; in_flight < kStages && p_left > 0; ++in_flight) issue_next();
 
-        Softmax st = {kNegBig, 0.f, 0.f, kNegBig};
+        SoftmaxT<STATS> st = {kNegBig, 0.f, 0.f, kNegBig, 0.f};
         float acc[kHalfDim];
 #pragma unroll
         for (int i = 0; i < kHalfDim; ++i) acc[i] = 0.f;
@@ -643,6 +655,10 @@ k_decode_attn(DecodeParams P) {
         const size_t rec0 = (size_t)u * P.pslots;
         reinterpret_cast<float2*>(P.part_o + (rec0 + (j - jf)) * kHeadDim)[lane] = make_float2(r2[0] + b_w, r2[1] + b_w);
         if (lane == 0) P.part_ml[rec0 + (j - jf)] = make_float2(st.m, l_w);
+        if (STATS) {
+            const float s2_w = 0.5f * warp_sum(st.s2);
+            if (lane == 0) P.part_s2[rec0 + (j - jf)] = s2_w;
+        }
 
         // ---- the warp that delivers the last partial of the unit merges them
         const uint32_t n_u = decode_warps_of_unit(u, P.units, P.gw);
@@ -692,6 +708,23 @@ k_decode_attn(DecodeParams P) {
             }
             const float inv = L > 0.f ? 1.0f / L : 0.f;            // a sequence that holds no token yet gets zeros
             reinterpret_cast<__half2*>(P.O + qo)[lane] = __floats2half2_rn(o0 * inv, o1 * inv);
+            if (STATS) {
+                // weights a_t = p_t / L sum to one over the n cached tokens: Var = sum a_t^2 / n - 1 / n^2
+                float S2 = 0.f;
+                for (uint32_t s0 = 0; s0 < n_u; s0 += 32) {
+                    const uint32_t s = s0 + lane;
+                    if (s < n_u) {
+                        const float f = fast_exp2(__ldcg(&P.part_ml[rec0 + s]).x - M);
+                        S2 = fmaf(__ldcg(&P.part_s2[rec0 + s]), f * f, S2);
+                    }
+                }
+                S2 = warp_sum(S2);
+                if (lane == 0) {
+                    const uint4 cnt = *reinterpret_cast<const uint4*>(P.counts + (size_t)row * 4);
+                    const float n = (float)(cnt.x + cnt.y + cnt.z + cnt.w);
+                    P.unit_var[u] = n > 0.f ? (S2 * inv * inv) / n - 1.0f / (n * n) : 0.f;
+                }
+            }
             if (lane == 0) P.part_cnt[u] = 0;
         }
     }
@@ -718,6 +751,15 @@ __global__ void k_visible_counts(StoreView s, const uint32_t* __restrict__ fill,
     }
     const uint4 f = *reinterpret_cast<const uint4*>(fill + (size_t)b * 4);
     *reinterpret_cast<uint4*>(vis + ((size_t)b * tq + il) * 4) = make_uint4(f.x - l0, f.y - l1, f.z - l2, f.w - l3);
+}
+
+// Eq. 16: V = (1/h) sum over the query heads of the variance of the head's attention weights.
+// unit_var [batch][q_heads] -> var_out [batch].  grid = batch, block = 32.
+__global__ void k_head_mean(const float* __restrict__ unit_var, int q_heads, float* __restrict__ var_out) {
+    float s = 0.f;
+    for (int h = threadIdx.x; h < q_heads; h += 32) s += unit_var[(size_t)blockIdx.x * q_heads + h];
+    s = warp_sum(s);
+    if (threadIdx.x == 0) var_out[blockIdx.x] = s / (float)q_heads;
 }
 
 }  // namespace kvq

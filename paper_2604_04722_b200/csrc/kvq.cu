@@ -17,6 +17,7 @@
 #include "k_append.cuh"
 #include "k_decode.cuh"
 #include "k_export.cuh"
+#include "k_features.cuh"
 
 using namespace kvq;
 
@@ -40,6 +41,8 @@ struct kvq_ctx {
     float* part_o = nullptr;             // decode scratch [units][partial slots][64]
     float2* part_ml = nullptr;           //                [units][partial slots]
     uint32_t* part_cnt = nullptr;        //                [units] arrival counters, zero between launches
+    float* part_s2 = nullptr;            //                [units][partial slots] sum of squared weights (kvq_decode_attn_var)
+    float* unit_var = nullptr;           //                [units] variance of a unit's attention weights
     uint32_t* vis = nullptr;             // kvq_attend_last: visible pool fills [batch][query rows of a launch][4]
     int splits_override = 0;
     uint32_t* flags = nullptr;
@@ -102,6 +105,8 @@ void free_all(kvq_ctx* c) {
     cudaFree(c->part_ml);
     cudaFree(c->part_cnt);
     cudaFree(c->vis);
+    cudaFree(c->part_s2);
+    cudaFree(c->unit_var);
     cudaFree(c->d_lens);
     cudaFree(c->flags);
     cudaFree(c->st_feats);
@@ -281,6 +286,8 @@ void fill_decode_params(kvq_ctx* c, int layer, const void* Q, void* O, float* pa
     p.part_o = part_o;
     p.part_ml = part_ml;
     p.part_cnt = part_cnt;
+    p.part_s2 = c->part_s2;
+    p.unit_var = c->unit_var;
     p.layer = layer;
     p.group = c->q_heads / c->kv_heads;
     p.tq = p.t_total = 1;
@@ -383,6 +390,8 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
     ok = ok && dev_alloc(c, &c->part_o, sizeof(float) * max_partial_records(c) * kHeadDim) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_ml, sizeof(float2) * max_partial_records(c)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_cnt, sizeof(uint32_t) * units * kMaxQueryRows) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->part_s2, sizeof(float) * max_partial_records(c)) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->unit_var, sizeof(float) * units) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->vis, sizeof(uint32_t) * 4 * (size_t)batch * kMaxQueryRows) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->d_lens, sizeof(int) * 3 * (size_t)batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->flags, sizeof(uint32_t)) == cudaSuccess;
@@ -413,7 +422,9 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
         ok = ok && cudaFuncSetAttribute(k_quant_pack<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(k_quant_pack<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(k_quant_pack<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring + smem_max) == cudaSuccess;
-        ok = ok && cudaFuncSetAttribute(k_decode_attn, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        ok = ok && cudaFuncSetAttribute(k_decode_attn<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)kDecodeSmemBytes) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(k_decode_attn<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)kDecodeSmemBytes) == cudaSuccess;
         ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     }
@@ -502,7 +513,7 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
     const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
     cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 2] : nullptr;
     if (rec) cudaEventRecord(ev[0], st);
-    k_decode_attn<<<grid, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    k_decode_attn<false><<<grid, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
     if (rec) {
         cudaEventRecord(ev[1], st);
         c->prof_calls += 1;
@@ -510,6 +521,40 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
     c->launches += 1;
     KVQ_CUDA(c, cudaGetLastError());
     return KVQ_OK;
+}
+
+int kvq_decode_attn_var(kvq_ctx* c, int layer, const void* Q, void* O, float* var_out, void* stream) {
+    if (check_layer(c, layer) != KVQ_OK || !Q || !O || !var_out) return KVQ_ERR_ARG;
+    if (c->len[layer] == 0) return KVQ_ERR_EMPTY;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DecodeParams p{};
+    fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt,
+                       choose_warps(c, c->len[layer], (uint64_t)c->batch * c->q_heads), p);
+    k_decode_attn<true><<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    k_head_mean<<<c->batch, 32, 0, st>>>(c->unit_var, c->q_heads, var_out);
+    c->launches += 2;
+    KVQ_CUDA(c, cudaGetLastError());
+    return KVQ_OK;
+}
+
+int kvq_token_features(const void* logits, int logits_are_fp32, int n, int vocab, const int32_t* token_ids,
+                       const uint32_t* counts, uint64_t total_count, uint32_t observed_tokens,
+                       const float* attn_var_opt, float* feats, void* stream) {
+    if (n < 0 || vocab < 1) return KVQ_ERR_ARG;
+    if (n == 0) return KVQ_OK;
+    if (!logits || !token_ids || !counts || !feats || !aligned16(feats)) return KVQ_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const float denom = (float)((double)total_count + (double)observed_tokens + 1.0);
+    const bool vec = vocab % 8 == 0 && (reinterpret_cast<uintptr_t>(logits) & 31u) == 0;
+    const int threads = n <= 1024 ? kFeatureThreadsFew : kFeatureThreads;
+    if (logits_are_fp32)
+        k_token_features<float><<<n, threads, 0, st>>>(static_cast<const float*>(logits), vocab, vec, token_ids,
+                                                               counts, denom, attn_var_opt, feats);
+    else
+        k_token_features<__half><<<n, threads, 0, st>>>(static_cast<const __half*>(logits), vocab, vec, token_ids,
+                                                                counts, denom, attn_var_opt, feats);
+    return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA;
 }
 
 int kvq_attend_last(kvq_ctx* c, int layer, const void* Q, void* O, int n_queries, void* stream) {
@@ -538,7 +583,7 @@ int kvq_attend_last(kvq_ctx* c, int layer, const void* Q, void* O, int n_queries
         p.t0 = (uint32_t)t0;
         p.units = (uint32_t)units;
         p.pslots = decode_pslots(p.units, p.gw);
-        k_decode_attn<<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+        k_decode_attn<false><<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
         c->launches += 2;
     }
     KVQ_CUDA(c, cudaGetLastError());
@@ -581,7 +626,7 @@ int kvq_decode_attn_static(kvq_ctx* c, int layer, const void* Q, void* O, void* 
     DecodeParams p{};
     fill_decode_params(c, layer, Q, O, base, reinterpret_cast<float2*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * kHeadDim),
                        reinterpret_cast<uint32_t*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * (kHeadDim + 2)), gw, p);
-    k_decode_attn<<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    k_decode_attn<false><<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
     c->launches += 1;
     KVQ_CUDA(c, cudaGetLastError());
     return KVQ_OK;
