@@ -670,7 +670,7 @@ k_decode_attn(DecodeParams P) {
         if (seen + 1 == n_u) {
             __threadfence();                           // the other warps' partials, counted before ours
             float M = kNegBig, L = 0.f, o0 = 0.f, o1 = 0.f;
-            if (n_u <= 8) {                            // the usual case: every load is issued before any is used
+            if (n_u <= 32) {                           // the usual case: lane s weighs partial s; loads go out eight at a time
                 const float2 ml = lane < n_u ? __ldcg(&P.part_ml[rec0 + lane]) : make_float2(kNegBig, 0.f);
                 float2 o[8];
 #pragma unroll
@@ -678,13 +678,25 @@ k_decode_attn(DecodeParams P) {
                     o[k] = k < n_u ? __ldcg(reinterpret_cast<const float2*>(P.part_o + (rec0 + k) * kHeadDim) + lane)
                                    : make_float2(0.f, 0.f);
                 M = warp_max(ml.x);
-                const float f = fast_exp2(ml.x - M);   // lane s weighs partial s
+                const float f = fast_exp2(ml.x - M);
                 L = warp_sum(ml.y * f);
 #pragma unroll
                 for (uint32_t k = 0; k < 8; ++k) {
                     const float fk = __shfl_sync(0xffffffffu, f, k);
                     o0 = fmaf(o[k].x, fk, o0);
                     o1 = fmaf(o[k].y, fk, o1);
+                }
+                for (uint32_t k0 = 8; k0 < n_u; k0 += 8) {
+#pragma unroll
+                    for (uint32_t k = 0; k < 8; ++k)
+                        o[k] = k0 + k < n_u ? __ldcg(reinterpret_cast<const float2*>(P.part_o + (rec0 + k0 + k) * kHeadDim) + lane)
+                                            : make_float2(0.f, 0.f);
+#pragma unroll
+                    for (uint32_t k = 0; k < 8; ++k) {
+                        const float fk = __shfl_sync(0xffffffffu, f, (k0 + k) & 31);
+                        o0 = fmaf(o[k].x, fk, o0);
+                        o1 = fmaf(o[k].y, fk, o1);
+                    }
                 }
             } else {
                 for (uint32_t s0 = 0; s0 < n_u; s0 += 32) {        // the maximum, 32 partials at a time
@@ -698,11 +710,18 @@ k_decode_attn(DecodeParams P) {
                     const float f = fast_exp2(ml.x - M);
                     L += warp_sum(ml.y * f);
                     const uint32_t cnt = min(32u, n_u - s0);
-                    for (uint32_t k = 0; k < cnt; ++k) {
-                        const float2 o = __ldcg(reinterpret_cast<const float2*>(P.part_o + (rec0 + s0 + k) * kHeadDim) + lane);
-                        const float fk = __shfl_sync(0xffffffffu, f, k);
-                        o0 = fmaf(o.x, fk, o0);
-                        o1 = fmaf(o.y, fk, o1);
+                    for (uint32_t k0 = 0; k0 < cnt; k0 += 8) {
+                        float2 o[8];
+#pragma unroll
+                        for (uint32_t k = 0; k < 8; ++k)
+                            o[k] = k0 + k < cnt ? __ldcg(reinterpret_cast<const float2*>(P.part_o + (rec0 + s0 + k0 + k) * kHeadDim) + lane)
+                                                : make_float2(0.f, 0.f);
+#pragma unroll
+                        for (uint32_t k = 0; k < 8; ++k) {
+                            const float fk = __shfl_sync(0xffffffffu, f, (k0 + k) & 31);
+                            o0 = fmaf(o[k].x, fk, o0);
+                            o1 = fmaf(o[k].y, fk, o1);
+                        }
                     }
                 }
             }
