@@ -274,3 +274,75 @@ class OracleCache:
             out[:, i] = decode_attn(np.ascontiguousarray(Q[:, i]), self.Hq, self.Hkv, self.bits[:, :m],
                                     self.kc[:, :m], self.km[:, :m], self.vc[:, :m], self.vm[:, :m])
         return out
+
+
+class GroupedOracleCache:
+    """The same cache with finer scale granularity: every row is cut into ``groups`` groups of
+    head_dim / groups consecutive channels and the row quantizer (the reading of Q_b in Eq. 24) is applied to
+    each group on its own, so a row carries ``groups`` {scale, zero-point} pairs.  Canonical form: the codes of
+    the groups back to back (element order unchanged), meta u16 [..][2 * groups].  Attention is Eq. 5 by its
+    definition (fp64) over the dequantized rows."""
+
+    def __init__(self, batch: int, q_heads: int, kv_heads: int, groups: int = 2, head_dim: int = 64):
+        assert head_dim % groups == 0
+        self.B, self.Hq, self.Hkv, self.D, self.G = batch, q_heads, kv_heads, head_dim, groups
+        self.bits = np.zeros((batch, 0), dtype=np.uint8)
+        self.kc = np.zeros((batch, 0, kv_heads, 2 * head_dim), dtype=np.uint8)
+        self.vc = np.zeros_like(self.kc)
+        self.km = np.zeros((batch, 0, kv_heads, 2 * groups), dtype=np.uint16)
+        self.vm = np.zeros_like(self.km)
+        self.khat = np.zeros((batch, 0, kv_heads, head_dim), dtype=np.float32)
+        self.vhat = np.zeros_like(self.khat)
+        self.counts = np.zeros((batch, 4), dtype=np.uint32)
+        self.pool_slot = np.zeros((batch, 0), dtype=np.uint32)
+
+    def __len__(self) -> int:
+        return self.bits.shape[1]
+
+    def _one(self, X, bits):
+        B, n, H, D = X.shape
+        G, Dg = self.G, D // self.G
+        Xg = np.ascontiguousarray(_u16(X).reshape(B, n, H * G, Dg))
+        cg, mg, _, _ = append(Xg, Xg, bits)                       # group rows: codes [B][n][H*G][2*Dg], meta [..][2]
+        codes = np.zeros((B, n, H, 2 * D), dtype=np.uint8)
+        hat = np.zeros((B, n, H, D), dtype=np.float32)
+        for b in range(B):
+            for t in range(n):
+                bt = int(bits[b, t])
+                gb = Dg * bt // 8
+                for h in range(H):
+                    for g in range(G):
+                        codes[b, t, h, g * gb:(g + 1) * gb] = cg[b, t, h * G + g, :gb]
+                        hat[b, t, h, g * Dg:(g + 1) * Dg] = dequantize_row(cg[b, t, h * G + g, :gb], mg[b, t, h * G + g], Dg, bt)
+        return codes, mg.reshape(B, n, H, 2 * G), hat
+
+    def append(self, K, V, bits) -> None:
+        bits = _c(bits, np.uint8)
+        kc, km, kh = self._one(K, bits)
+        vc, vm, vh = self._one(V, bits)
+        ps = np.empty(bits.shape, dtype=np.uint32)
+        for b in range(self.B):
+            ps[b], self.counts[b] = assign_slots(bits[b], self.counts[b])
+        self.bits = np.concatenate([self.bits, bits], axis=1)
+        self.kc = np.concatenate([self.kc, kc], axis=1)
+        self.vc = np.concatenate([self.vc, vc], axis=1)
+        self.km = np.concatenate([self.km, km], axis=1)
+        self.vm = np.concatenate([self.vm, vm], axis=1)
+        self.khat = np.concatenate([self.khat, kh], axis=1)
+        self.vhat = np.concatenate([self.vhat, vh], axis=1)
+        self.pool_slot = np.concatenate([self.pool_slot, ps], axis=1)
+
+    def decode_attn(self, Q) -> np.ndarray:
+        """fp16 bit patterns [B][Hq][D]: Softmax(q K^T / sqrt(D)) V over the dequantized rows, in fp64."""
+        q = half_to_float(_u16(Q)).astype(np.float64)
+        g = self.Hq // self.Hkv
+        out = np.empty((self.B, self.Hq, self.D), dtype=np.float64)
+        for b in range(self.B):
+            for h in range(self.Hq):
+                k = self.khat[b, :, h // g].astype(np.float64)
+                v = self.vhat[b, :, h // g].astype(np.float64)
+                z = k @ q[b, h] / np.sqrt(float(self.D))
+                p = np.exp(z - z.max())
+                p /= p.sum()
+                out[b, h] = p @ v
+        return np.asarray(out, dtype=np.float16).view(np.uint16)          # fp64 -> fp16, round to nearest even

@@ -49,23 +49,29 @@ __host__ __device__ constexpr int pool_half_bytes(int c) { return 8 << c; }     
 __host__ __device__ constexpr int pool_unit_bytes(int c) { return c == 0 ? 8 : 16; }
 __host__ __device__ constexpr int pool_units(int c) { return pool_half_bytes(c) / pool_unit_bytes(c); }   // 1,1,2,4
 __host__ __device__ constexpr int pool_codes_bytes(int c) { return 2 * pool_half_bytes(c) * kTileTokens; }  // per tile, per tensor
-__host__ __device__ constexpr int pool_meta_bytes(int c) { return pool_has_meta(c) ? 4 * kTileTokens : 0; }  // per tile, per tensor
-__host__ __device__ constexpr int pool_rec_bytes(int c) { return 2 * pool_codes_bytes(c) + 2 * pool_meta_bytes(c); }
-__host__ __device__ constexpr int pool_row_bytes(int c) {                        // K+V bytes per (token, KV head)
-    return pool_rec_bytes(c) / kTileTokens;                                      // 40, 72, 136, 256
+// Scale groups g: 1 = one {scale, zero-point} pair per row (the default), 2 = one pair per half-row (32
+// channels), stored as two planes of 16 words per tensor: [K half 0][K half 1][V half 0][V half 1].
+__host__ __device__ constexpr int pool_meta_bytes(int c, int g = 1) { return pool_has_meta(c) ? 4 * kTileTokens * g : 0; }  // per tile, per tensor
+__host__ __device__ constexpr int pool_rec_bytes(int c, int g = 1) { return 2 * pool_codes_bytes(c) + 2 * pool_meta_bytes(c, g); }
+__host__ __device__ constexpr int pool_row_bytes(int c, int g = 1) {             // K+V bytes per (token, KV head)
+    return pool_rec_bytes(c, g) / kTileTokens;                                   // 40, 72, 136, 256 (g = 2: 48, 80, 144, 256)
 }
 // Byte offset, inside one tensor's code block of a tile, of unit u of half h of slot t.
 __host__ __device__ constexpr int unit_offset(int c, int h, int u, int t) {
     return ((h * pool_units(c) + u) * kTileTokens + t) * pool_unit_bytes(c);
 }
 // Byte offset, inside the record, of the {scale, zero-point} pair of slot t (tensor 0 = K, 1 = V).
-__host__ __device__ constexpr int meta_offset(int c, int tensor, int t) {
-    return 2 * pool_codes_bytes(c) + tensor * pool_meta_bytes(c) + 4 * t;
+// With two scale groups `half` picks the plane of the half-row.
+__host__ __device__ constexpr int meta_offset(int c, int tensor, int t, int half = 0, int g = 1) {
+    return 2 * pool_codes_bytes(c) + tensor * pool_meta_bytes(c, g) + (g == 2 ? half * 4 * kTileTokens : 0) + 4 * t;
 }
 
 constexpr uint32_t kBlockBytes = 65536;
 // Tiles per block: a whole number of ring stages of the decode kernel (10 / 5 / 3 / 1 tiles).
-__host__ __device__ constexpr uint32_t block_tiles(int c) { return c == 0 ? 100u : c == 1 ? 55u : c == 2 ? 30u : 16u; }
+// (with two scale groups the records are 768 / 1280 / 2304 / 4096 bytes: 80 / 50 / 28 / 16 tiles)
+__host__ __device__ constexpr uint32_t block_tiles(int c, int g = 1) {
+    return g == 2 ? (c == 0 ? 80u : c == 1 ? 50u : c == 2 ? 28u : 16u) : (c == 0 ? 100u : c == 1 ? 55u : c == 2 ? 30u : 16u);
+}
 constexpr uint32_t kFlagArenaFull = 4u;
 
 // Everything a kernel needs to find a row.
@@ -75,6 +81,7 @@ struct StoreView {
     uint32_t* arena_used;         // blocks handed out so far (block ids are 1 + the old value)
     uint32_t arena_blocks;        // capacity in blocks, block 0 included
     uint32_t table_stride, table_off[kNumPools];
+    int groups;                   // scale groups per row: 1 or 2
     uint32_t* index;              // [layers][batch][max_ctx]   pool<<30 | slot
     uint32_t* flags;              // device flag word
     int layers, batch, kv_heads, q_heads, max_ctx, cap_tiles;
@@ -86,10 +93,10 @@ __host__ __device__ inline uint32_t* stream_table(const StoreView& s, int c, int
     return s.table + stream * s.table_stride + s.table_off[c];
 }
 // Address of tile `tile` of a stream whose table row is `tab`.
-__device__ __forceinline__ uint8_t* tile_ptr(const StoreView& s, int c, const uint32_t* tab, uint32_t tile) {
-    const uint32_t bt = block_tiles(c);
+__device__ __forceinline__ uint8_t* tile_ptr(const StoreView& s, int c, const uint32_t* tab, uint32_t tile, int g = 1) {
+    const uint32_t bt = block_tiles(c, g);
     const uint32_t blk = tile / bt;
-    return s.arena + (size_t)tab[blk] * kBlockBytes + (size_t)(tile - blk * bt) * (uint32_t)pool_rec_bytes(c);
+    return s.arena + (size_t)tab[blk] * kBlockBytes + (size_t)(tile - blk * bt) * (uint32_t)pool_rec_bytes(c, g);
 }
 // Hand out `n` consecutive blocks; returns the id of the first (0 = the arena is exhausted: flagged).
 __device__ __forceinline__ uint32_t arena_take(const StoreView& s, uint32_t n) {
@@ -101,8 +108,8 @@ __device__ __forceinline__ uint32_t arena_take(const StoreView& s, uint32_t n) {
     return first;
 }
 // Blocks a stream of class c needs for n tokens.
-__host__ __device__ constexpr uint32_t blocks_for(int c, uint32_t n) {
-    return ((n + kTileTokens - 1) / kTileTokens + block_tiles(c) - 1) / block_tiles(c);
+__host__ __device__ constexpr uint32_t blocks_for(int c, uint32_t n, int g = 1) {
+    return ((n + kTileTokens - 1) / kTileTokens + block_tiles(c, g) - 1) / block_tiles(c, g);
 }
 
 __device__ __forceinline__ int bits_to_class(int bits) {

@@ -199,3 +199,45 @@ def test_slot_assignment_is_a_bijection_per_pool(oracle):
         assert counts[p] == s.size
     with pytest.raises(ValueError):
         oracle.assign_slots(np.array([2, 3], np.uint8))
+
+
+def test_grouped_scales_reduce_to_the_row_quantizer_and_tighten_the_error(oracle):
+    """Two scale groups per row: each 32-channel group is quantized exactly as a 32-element row would be (codes
+    back to back, one {scale, zero-point} pair per group); with one group the cache equals the plain one and its
+    attention equals the C routine's; the per-element error bound s/2 now holds per group, and the mean error does
+    not grow."""
+    rng = np.random.default_rng(44)
+    B, Hq, H, n = 2, 4, 2, 40
+    K = (rng.standard_normal((B, n, H, 64)) * 2).astype(np.float16)
+    K[..., 5] *= np.float16(8.0)                                   # an outlier channel in the first group only
+    V = rng.standard_normal((B, n, H, 64)).astype(np.float16)
+    bits = np.array([2, 4, 8, 16], np.uint8)[rng.choice(4, size=(B, n))]
+    Q = rng.standard_normal((B, Hq, 64)).astype(np.float16)
+    plain = oracle.OracleCache(B, Hq, H)
+    plain.append(K, V, bits)
+    g1 = oracle.GroupedOracleCache(B, Hq, H, groups=1)
+    g1.append(K, V, bits)
+    assert np.array_equal(g1.kc, plain.kc) and np.array_equal(g1.km, plain.km) and np.array_equal(g1.vc, plain.vc)
+    a, b_ = g1.decode_attn(Q).view(np.float16).astype(np.float64), plain.decode_attn(Q).view(np.float16).astype(np.float64)
+    assert np.max(np.abs(a - b_)) <= 1e-3                          # same numbers up to the last fp16 rounding
+    g2 = oracle.GroupedOracleCache(B, Hq, H, groups=2)
+    g2.append(K, V, bits)
+    assert np.array_equal(g2.pool_slot, plain.pool_slot)
+    for b in range(B):
+        for t in range(n):
+            bt = int(bits[b, t])
+            for h in range(H):
+                for g in range(2):
+                    codes, meta = oracle.quantize_row(K[b, t, h, 32 * g:32 * g + 32], bt)
+                    gb = 32 * bt // 8
+                    assert np.array_equal(g2.kc[b, t, h, g * gb:(g + 1) * gb], codes)
+                    if bt < 16:
+                        assert np.array_equal(g2.km[b, t, h, 2 * g:2 * g + 2], meta)
+                        sf = float(oracle.half_to_float(meta[:1])[0])
+                        err = np.abs(g2.khat[b, t, h, 32 * g:32 * g + 32].astype(np.float64) -
+                                     K[b, t, h, 32 * g:32 * g + 32].astype(np.float64))
+                        assert np.all(err <= 0.5 * sf * (1 + 2 ** -9) + 1e-6)
+    q = bits < 16
+    e1 = np.abs(g1.khat.astype(np.float64) - K.astype(np.float64))[q].mean()
+    e2 = np.abs(g2.khat.astype(np.float64) - K.astype(np.float64))[q].mean()
+    assert e2 < e1                                                 # the outlier no longer stretches the second group's grid
