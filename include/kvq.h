@@ -92,6 +92,20 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
                      int max_ctx, int batch, uint64_t arena_bytes);
 
 /*
+ * The same with a chosen granularity of the min-max quantizer (Eq. 9-13 leave it open; the
+ * related work of Section 2 uses finer-grained scales).  scale_groups = 1: one {scale,
+ * zero-point} pair per (token, KV head) row of 64 channels, what kvq_create and
+ * kvq_create_arena build.  scale_groups = 2: one pair per group of 32 consecutive channels
+ * (channels 0..31 and 32..63), each group quantized by the row quantizer on its own values; the
+ * codes keep their place, a stored row grows by 8 bytes (48 / 80 / 144 / 256 bytes per token and
+ * KV head) and a 64 KB block holds 80 / 50 / 28 / 16 tiles.  Every other entry point behaves the
+ * same; the export calls return 2 * scale_groups meta words per (token, KV head, tensor).  Any
+ * other scale_groups is KVQ_ERR_ARG.
+ */
+int kvq_create_grouped(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim,
+                       int max_ctx, int batch, uint64_t arena_bytes, int scale_groups);
+
+/*
  * Arena fill: blocks handed out so far, blocks available, bytes per block (host uint64, any
  * may be NULL).  Synchronizes.
  */
@@ -278,7 +292,8 @@ int kvq_set_splits(kvq_ctx* ctx, int splits);
  *             bits [(i*b)%8, +b) of byte floor(i*b/8); for b == 16 the fp16 row,
  *             little-endian; bytes past 64*b/8 are zero
  *   k_meta, v_meta  uint16 [batch][n][kv_heads][2]: fp16 bit patterns of
- *             {scale, zero-point}; {0,0} for b == 16
+ *             {scale, zero-point}; {0,0} for b == 16.  A cache made with scale_groups = 2
+ *             returns [batch][n][kv_heads][2][2]: the pair of channels 0..31, then of 32..63
  * Any output pointer may be NULL to skip it.
  */
 int kvq_export_range(kvq_ctx* ctx, int layer, int pos0, int n,
@@ -287,7 +302,7 @@ int kvq_export_range(kvq_ctx* ctx, int layer, int pos0, int n,
                      void* stream);
 
 /* The same for one token of one sequence, into HOST buffers ([kv_heads][128] and
- * [kv_heads][2]); synchronizes. */
+ * [kv_heads][2 * scale_groups]); synchronizes. */
 int kvq_export_token(kvq_ctx* ctx, int layer, int b, int pos,
                      uint8_t* bits, uint32_t* pool_slot,
                      void* k_codes, void* v_codes, uint16_t* k_meta, uint16_t* v_meta);

@@ -33,6 +33,7 @@ _vp, _i, _u64p = C.c_void_p, C.c_int, C.POINTER(C.c_uint64)
 SIGNATURES = {
     "kvq_create": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i]),
     "kvq_create_arena": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, C.c_uint64]),
+    "kvq_create_grouped": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, C.c_uint64, _i]),
     "kvq_arena_usage": (_i, [_vp, _u64p, _u64p, _u64p]),
     "kvq_destroy": (_i, [_vp]),
     "kvq_set_controller": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -125,6 +126,14 @@ def kvq_create_arena(layers: int, q_heads: int, kv_heads: int, head_dim: int, ma
     h = _vp()
     check(lib().kvq_create_arena(C.byref(h), layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes),
           "kvq_create_arena")
+    return h.value
+
+
+def kvq_create_grouped(layers: int, q_heads: int, kv_heads: int, head_dim: int, max_ctx: int, batch: int,
+                       arena_bytes: int, scale_groups: int) -> int:
+    h = _vp()
+    check(lib().kvq_create_grouped(C.byref(h), layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes,
+                                   scale_groups), "kvq_create_grouped")
     return h.value
 
 
@@ -222,14 +231,14 @@ def kvq_export_range(ctx: int, layer: int, pos0: int, n: int, bits=None, pool_sl
                                  _ptr(k_meta), _ptr(v_meta), _stream(stream)), "kvq_export_range")
 
 
-def kvq_export_token(ctx: int, layer: int, b: int, pos: int, kv_heads: int):
-    """Returns (bits, pool_slot, k_codes [H][128] u8, v_codes, k_meta [H][2] u16, v_meta) as numpy."""
+def kvq_export_token(ctx: int, layer: int, b: int, pos: int, kv_heads: int, scale_groups: int = 1):
+    """Returns (bits, pool_slot, k_codes [H][128] u8, v_codes, k_meta [H][2 * scale_groups] u16, v_meta) as numpy."""
     import numpy as np
     bits = np.zeros(1, np.uint8)
     ps = np.zeros(1, np.uint32)
     kc = np.zeros((kv_heads, KVQ_EXPORT_ROW_BYTES), np.uint8)
     vc = np.zeros_like(kc)
-    km = np.zeros((kv_heads, 2), np.uint16)
+    km = np.zeros((kv_heads, 2 * scale_groups), np.uint16)
     vm = np.zeros_like(km)
     check(lib().kvq_export_token(ctx, layer, b, pos, _ptr(bits), _ptr(ps), _ptr(kc), _ptr(vc), _ptr(km), _ptr(vm)),
           "kvq_export_token")

@@ -154,7 +154,9 @@ __device__ __forceinline__ void pack_codes(const __half2* hp, float mn, float in
 // `tail`: the lane's slot lies beyond the stream's fill (it will be written by a later append); its
 // {scale, zero-point} word is cleared so that a reader, which gives such a slot weight zero, never
 // multiplies that zero with whatever a recycled block held before.
-template <int CLS, int PARTNER = 16>
+// G: scale groups per row.  With G == 2 the half-row is a group of its own: no exchange with the partner lane,
+// and every lane stores (or clears) the {scale, zero-point} word of its own group at `meta`.
+template <int CLS, int PARTNER = 16, int G = 1>
 __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], bool active, bool tail, int half, int t,
                                                         uint8_t* codes, uint8_t* meta) {
     constexpr int BITS = pool_bits(CLS);
@@ -168,8 +170,10 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
     }
     float mn = fminf(__low2float(mn2), __high2float(mn2));
     float mx = fmaxf(__low2float(mx2), __high2float(mx2));
-    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, PARTNER));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, PARTNER));
+    if (G == 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, PARTNER));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, PARTNER));
+    }
     if (mn == 0.0f) mn = 0.0f;                         // -0 is stored as +0
     if (mx == 0.0f) mx = 0.0f;
     const float s32 = __fdiv_rn(__fsub_rn(mx, mn), LEVELS);
@@ -186,7 +190,7 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
     if (__any_sync(0xffffffffu, tiny)) pack_codes<CLS, true>(hp, mn, inv, w);
     else pack_codes<CLS, false>(hp, mn, inv, w);
     if (!active) {
-        if (tail && half == 0) *reinterpret_cast<uint32_t*>(meta) = 0u;
+        if (tail && (G == 2 || half == 0)) *reinterpret_cast<uint32_t*>(meta) = 0u;
         return;
     }
     if (CLS == 0) {
@@ -197,7 +201,7 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
             *reinterpret_cast<uint4*>(codes + unit_offset(CLS, half, u, t)) =
                 make_uint4(w[4 * u], w[4 * u + 1], w[4 * u + 2], w[4 * u + 3]);
     }
-    if (half == 0)
+    if (G == 2 || half == 0)
         *reinterpret_cast<uint32_t*>(meta) =
             (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(__float2half_rn(mn)) << 16);
 }
@@ -207,7 +211,7 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
 // CTA after its next barrier and to later launches.
 __device__ __forceinline__ void reserve_blocks(const StoreView& s, int c, int layer, int b, int h0, int nh,
                                                uint32_t n_old, uint32_t n_new, int lane) {
-    const uint32_t have = blocks_for(c, n_old), want = blocks_for(c, n_new);
+    const uint32_t have = blocks_for(c, n_old, s.groups), want = blocks_for(c, n_new, s.groups);
     if (want == have) return;
     const uint32_t per = want - have;
     uint32_t first = 0;
@@ -238,7 +242,7 @@ k_reserve_blocks(AppendParams p) {
 // Launch 2.  MODE 0: classes come from k_classify (several chunks per sequence);
 // MODE 1: one chunk, classes from `bits`; MODE 2: one chunk, classes from the controller.
 // grid = (nchunks, head_groups, batch), block = 256.
-template <int MODE>
+template <int MODE, int G>
 __global__ void __launch_bounds__(kChunkTokens, KVQ_APPEND_MIN_CTAS)
 k_quant_pack(AppendParams p) {
     extern __shared__ __align__(16) uint8_t dyn_smem[];   // [ring: warps x depth x 4 KB][controller block (MODE 2)]
@@ -377,7 +381,7 @@ k_quant_pack(AppendParams p) {
             // beyond the fill only in the append's last chunk (otherwise the next chunk's tokens go there)
             it.tail = !it.active && (int32_t)(r0 + t) >= 0 && chunk == p.nchunks - 1;
             const int h = h0 + hh;
-            it.rec = tile_ptr(p.store, k, stream_table(p.store, k, p.layer, b, h), tile);
+            it.rec = tile_ptr(p.store, k, stream_table(p.store, k, p.layer, b, h), tile, G);
             const uint32_t r_ld = r0 + (lane >> 1);                // the slot this lane copies a piece of
             if (r_ld < nk) {
                 const int i_tok = list[k][r_ld];
@@ -426,16 +430,16 @@ k_quant_pack(AppendParams p) {
         const bool active = cur.active;
         switch (cur.k) {
         case 0:
-            quantize_store_half_row<0>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(0, 0, t));
-            quantize_store_half_row<0>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(0, 1, t));
+            quantize_store_half_row<0, 16, G>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(0, 0, t, half, G));
+            quantize_store_half_row<0, 16, G>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(0, 1, t, half, G));
             break;
         case 1:
-            quantize_store_half_row<1>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(1, 0, t));
-            quantize_store_half_row<1>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(1, 1, t));
+            quantize_store_half_row<1, 16, G>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(1, 0, t, half, G));
+            quantize_store_half_row<1, 16, G>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(1, 1, t, half, G));
             break;
         case 2:
-            quantize_store_half_row<2>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(2, 0, t));
-            quantize_store_half_row<2>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(2, 1, t));
+            quantize_store_half_row<2, 16, G>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(2, 0, t, half, G));
+            quantize_store_half_row<2, 16, G>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(2, 1, t, half, G));
             break;
         default:                                       // fp16: the lane's 64 input bytes are its four units
             if (active) {
@@ -452,27 +456,37 @@ k_quant_pack(AppendParams p) {
 }
 
 // The stores of k_append_token: both tensors of the lane's half-row into the tile record `rec`.
+template <int G>
 __device__ __forceinline__ void token_store(int c, const uint4 (&kraw)[4], const uint4 (&vraw)[4], bool active, int half,
                                             int t, uint8_t* rec) {
     uint8_t* vcodes = rec + pool_codes_bytes(c);
     if (t == 0 && c < 3 && active) {                   // the token opens a tile: clear the tile's {scale, zero-point} words
-        uint4* m = reinterpret_cast<uint4*>(rec + meta_offset(c, half, 0));        // half 0: K words, half 1: V words
+        if (G == 1) {
+            uint4* m = reinterpret_cast<uint4*>(rec + meta_offset(c, half, 0));    // half 0: K words, half 1: V words
 #pragma unroll
-        for (int i = 0; i < 4; ++i) m[i] = make_uint4(0, 0, 0, 0);
+            for (int i = 0; i < 4; ++i) m[i] = make_uint4(0, 0, 0, 0);
+        } else {                                       // the planes of this lane's group, for K and for V
+#pragma unroll
+            for (int tensor = 0; tensor < 2; ++tensor) {
+                uint4* m = reinterpret_cast<uint4*>(rec + meta_offset(c, tensor, 0, half, 2));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) m[i] = make_uint4(0, 0, 0, 0);
+            }
+        }
     }
     __syncwarp();                                      // slot 0's own word is written after the clearing
     switch (c) {
     case 0:
-        quantize_store_half_row<0, 1>(kraw, active, false, half, t, rec, rec + meta_offset(0, 0, t));
-        quantize_store_half_row<0, 1>(vraw, active, false, half, t, vcodes, rec + meta_offset(0, 1, t));
+        quantize_store_half_row<0, 1, G>(kraw, active, false, half, t, rec, rec + meta_offset(0, 0, t, half, G));
+        quantize_store_half_row<0, 1, G>(vraw, active, false, half, t, vcodes, rec + meta_offset(0, 1, t, half, G));
         break;
     case 1:
-        quantize_store_half_row<1, 1>(kraw, active, false, half, t, rec, rec + meta_offset(1, 0, t));
-        quantize_store_half_row<1, 1>(vraw, active, false, half, t, vcodes, rec + meta_offset(1, 1, t));
+        quantize_store_half_row<1, 1, G>(kraw, active, false, half, t, rec, rec + meta_offset(1, 0, t, half, G));
+        quantize_store_half_row<1, 1, G>(vraw, active, false, half, t, vcodes, rec + meta_offset(1, 1, t, half, G));
         break;
     case 2:
-        quantize_store_half_row<2, 1>(kraw, active, false, half, t, rec, rec + meta_offset(2, 0, t));
-        quantize_store_half_row<2, 1>(vraw, active, false, half, t, vcodes, rec + meta_offset(2, 1, t));
+        quantize_store_half_row<2, 1, G>(kraw, active, false, half, t, rec, rec + meta_offset(2, 0, t, half, G));
+        quantize_store_half_row<2, 1, G>(vraw, active, false, half, t, vcodes, rec + meta_offset(2, 1, t, half, G));
         break;
     default:
         if (active) {
@@ -490,7 +504,7 @@ __device__ __forceinline__ void token_store(int c, const uint4 (&kraw)[4], const
 // Lane l handles half-row l%2 of KV head 16*blockIdx.x + l/2.  Everything the warp needs (the K and V
 // rows, the pool fills, the features) is requested up front so the loads overlap the controller;
 // the decision is taken by the whole warp (FUSED, hidden width 32) or read from `bits`.
-template <bool FUSED>
+template <bool FUSED, int G>
 __global__ void __launch_bounds__(32)
 k_append_token(AppendParams p) {
     const int lane = threadIdx.x, b = blockIdx.y;
@@ -514,10 +528,10 @@ k_append_token(AppendParams p) {
     // requested now, so that they travel while the controller runs.  An entry of a block that is not
     // reserved yet may hold anything and is not used.
     const int hs = active ? h : 0;
-    const uint32_t id0 = stream_table(p.store, 0, p.layer, b, hs)[fill.x / (kTileTokens * block_tiles(0))];
-    const uint32_t id1 = stream_table(p.store, 1, p.layer, b, hs)[fill.y / (kTileTokens * block_tiles(1))];
-    const uint32_t id2 = stream_table(p.store, 2, p.layer, b, hs)[fill.z / (kTileTokens * block_tiles(2))];
-    const uint32_t id3 = stream_table(p.store, 3, p.layer, b, hs)[fill.w / (kTileTokens * block_tiles(3))];
+    const uint32_t id0 = stream_table(p.store, 0, p.layer, b, hs)[fill.x / (kTileTokens * block_tiles(0, G))];
+    const uint32_t id1 = stream_table(p.store, 1, p.layer, b, hs)[fill.y / (kTileTokens * block_tiles(1, G))];
+    const uint32_t id2 = stream_table(p.store, 2, p.layer, b, hs)[fill.z / (kTileTokens * block_tiles(2, G))];
+    const uint32_t id3 = stream_table(p.store, 3, p.layer, b, hs)[fill.w / (kTileTokens * block_tiles(3, G))];
     int c;
     if (FUSED) {
         const float4 f = reinterpret_cast<const float4*>(p.feats)[b];
@@ -535,21 +549,21 @@ k_append_token(AppendParams p) {
     const int t = (int)(slot & (kTileTokens - 1));
     const uint32_t tile = slot / kTileTokens;
     uint32_t* tab = stream_table(p.store, c, p.layer, b, active ? h : 0);
-    if (slot % (kTileTokens * block_tiles(c)) == 0) {              // the token opens a new block of its stream
+    if (slot % (kTileTokens * block_tiles(c, G)) == 0) {              // the token opens a new block of its stream
         uint32_t id = 0;
         if (active && half == 0) {
             id = arena_take(p.store, 1);
-            tab[tile / block_tiles(c)] = id;
+            tab[tile / block_tiles(c, G)] = id;
         }
         id = __shfl_sync(0xffffffffu, id, lane & ~1);
         // the partner lane must not read the table before the entry is written: hand it the address instead
         uint8_t* rec_new = p.store.arena + (size_t)id * kBlockBytes;
-        token_store(c, kraw, vraw, active, half, t, rec_new);
+        token_store<G>(c, kraw, vraw, active, half, t, rec_new);
         return;
     }
     const uint32_t id = c == 0 ? id0 : c == 1 ? id1 : c == 2 ? id2 : id3;
-    token_store(c, kraw, vraw, active, half, t,
-                p.store.arena + (size_t)id * kBlockBytes + (size_t)(tile % block_tiles(c)) * (uint32_t)pool_rec_bytes(c));
+    token_store<G>(c, kraw, vraw, active, half, t,
+                   p.store.arena + (size_t)id * kBlockBytes + (size_t)(tile % block_tiles(c, G)) * (uint32_t)pool_rec_bytes(c, G));
 }
 
 }  // namespace kvq

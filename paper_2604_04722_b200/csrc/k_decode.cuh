@@ -87,7 +87,10 @@ static_assert(kStageBytes % 16 == 0 && kStageBytes >= pool_rec_bytes(3), "a stag
 static_assert(block_tiles(0) % (kStageBytes / pool_rec_bytes(0)) == 0 && block_tiles(1) % (kStageBytes / pool_rec_bytes(1)) == 0 &&
                   block_tiles(2) % (kStageBytes / pool_rec_bytes(2)) == 0 && block_tiles(3) % (kStageBytes / pool_rec_bytes(3)) == 0,
               "an arena block must hold a whole number of ring stages");
-__host__ __device__ constexpr int tiles_per_stage(int c) { return kStageBytes / pool_rec_bytes(c); }
+__host__ __device__ constexpr int tiles_per_stage(int c, int g = 1) { return kStageBytes / pool_rec_bytes(c, g); }
+static_assert(block_tiles(0, 2) % tiles_per_stage(0, 2) == 0 && block_tiles(1, 2) % tiles_per_stage(1, 2) == 0 &&
+                  block_tiles(2, 2) % tiles_per_stage(2, 2) == 0 && block_tiles(3, 2) % tiles_per_stage(3, 2) == 0,
+              "the same with two scale groups per row");
 constexpr size_t kDecodeSmemBytes = (size_t)kDecodeWarps * kStages * kStageBytes;
 
 struct DecodeParams {
@@ -211,6 +214,12 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
+__device__ __forceinline__ float half_sum(float v) {    // over the 16 lanes of a half-warp
+#pragma unroll
+    for (int d = 8; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+    return v;
+}
+
 // STATS: also keep the sum of squared weights (for the attention-variance feature of Eq. 16).
 template <bool STATS>
 struct SoftmaxT {
@@ -252,13 +261,14 @@ struct QueryInfo {
     const float* q_half;           // this lane's 32 query values (shared memory)
     float fix_scale;               // 256 R: rint(q * 256 R) is the 24-bit fixed-point query
     float inv_fix;                 // kLogitScale / (256 R)
-    float sumq;                    // kLogitScale * sum_i q_i
+    float sumq;                    // kLogitScale * sum_i q_i over the row (over this lane's half with two scale groups)
 };
 constexpr int kQRegs = kHalfDim;   // registers a consumer may use for its copy of the query
 
-template <int CLS>
+// G: scale groups per row (1: one {scale, zero-point} per row; 2: one per half-row).
+template <int CLS, int G = 1>
 struct Quantized {
-    static constexpr int BITS = pool_bits(CLS), REC = pool_rec_bytes(CLS);
+    static constexpr int BITS = pool_bits(CLS), REC = pool_rec_bytes(CLS, G);
     static constexpr int EPW = 32 / BITS;              // elements per 32-bit word
     static constexpr int WORDS = pool_half_bytes(CLS) / 4;         // words per half-row: 2, 4, 8
     static constexpr int UNITS = pool_units(CLS), UWORDS = pool_unit_bytes(CLS) / 4;
@@ -315,7 +325,7 @@ struct Quantized {
     __device__ static __forceinline__ KIn load_k(const uint8_t* rec, int half, int t) {
         KIn k;
         load_half_row(rec, half, t, k.w);
-        k.meta = *reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 0, t));
+        k.meta = *reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 0, t, half, G));
         return k;
     }
     template <class SM>
@@ -328,7 +338,7 @@ struct Quantized {
         const float2 km = meta_to_float2(kin.meta);
         uint32_t wv_codes[WORDS];                      // the V side's inputs are requested before the K arithmetic
         load_half_row(rec + pool_codes_bytes(CLS), half, t, wv_codes);
-        const uint32_t vmeta = *reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 1, t));
+        const uint32_t vmeta = *reinterpret_cast<const uint32_t*>(rec + meta_offset(CLS, 1, t, half, G));
         int dh[PLANES], dl[PLANES];
 #pragma unroll
         for (int k = 0; k < PLANES; ++k) dh[k] = dl[k] = 0;
@@ -348,8 +358,9 @@ struct Quantized {
             lsum = (lsum << BITS) + dl[k];
         }
         float dot = fmaf((float)hsum, 256.0f, (float)lsum);
-        dot += __shfl_xor_sync(0xffffffffu, dot, 16);              // the other half of the row
+        if (G == 1) dot += __shfl_xor_sync(0xffffffffu, dot, 16);  // the other half of the row
         float y = fmaf(km.x * (qi.inv_fix * (1.0f / (float)(1 << (BITS * (PLANES - 1))))), dot, km.y * qi.sumq);
+        if (G == 2) y += __shfl_xor_sync(0xffffffffu, y, 16);      // each half carries its own scale and zero-point
         y = valid ? y : -INFINITY;
         const float p = softmax_step(st, acc, y);
 
@@ -427,8 +438,12 @@ struct WarpScratch {
 };
 constexpr int kQHalfStride = kHalfDim + 4;
 
+template <int G>
 __device__ __forceinline__ int tps_of(int c) {
-    return c == 0 ? tiles_per_stage(0) : c == 1 ? tiles_per_stage(1) : c == 2 ? tiles_per_stage(2) : tiles_per_stage(3);
+    return c == 0   ? tiles_per_stage(0, G)
+           : c == 1 ? tiles_per_stage(1, G)
+           : c == 2 ? tiles_per_stage(2, G)
+                    : tiles_per_stage(3, G);
 }
 // floor(n * a / g) for a <= g < 65536 in 32-bit arithmetic: n = q*g + r gives q*a + floor(r*a/g).
 __device__ __forceinline__ uint32_t scale_by_fraction(uint32_t n, uint32_t a, uint32_t g) {
@@ -438,7 +453,7 @@ __device__ __forceinline__ uint32_t scale_by_fraction(uint32_t n, uint32_t a, ui
 
 // grid = ceil(gw / kDecodeWarps), block = kDecodeThreads, dynamic smem = kDecodeSmemBytes.
 // STATS: also emit, per unit, the variance of its attention weights over the cached tokens.
-template <bool STATS>
+template <bool STATS, int G>
 __global__ void __launch_bounds__(kDecodeThreads, KVQ_DECODE_MIN_CTAS)
 k_decode_attn(DecodeParams P) {
     extern __shared__ __align__(128) uint8_t ring[];   // [warps][stages][kStageBytes]
@@ -497,7 +512,12 @@ k_decode_attn(DecodeParams P) {
         QueryInfo qi;
         {
             const float qa = ws.q[lane], qb = ws.q[kQHalfStride + lane];
-            qi.sumq = warp_sum(qa + qb) * kLogitScale; // sum_i q_i, in logit units
+            if (G == 1) {
+                qi.sumq = warp_sum(qa + qb) * kLogitScale;         // sum_i q_i, in logit units
+            } else {                                   // the sum over this lane's half: 32 elements over its 16 lanes
+                const float* qh_ = ws.q + half * kQHalfStride;
+                qi.sumq = half_sum(qh_[t] + qh_[16 + t]) * kLogitScale;
+            }
             // 256 R = 2^(22 - floor(log2 max|q|)), max|q| taken as at least the smallest normal fp16
             const float qmax = fmaxf(warp_max(fmaxf(fabsf(qa), fabsf(qb))), 6.103515625e-05f);
             const uint32_t e = __float_as_uint(qmax) >> 23;        // biased exponent, 113..142
@@ -519,9 +539,9 @@ k_decode_attn(DecodeParams P) {
                 const int lo = ws.lo[p_c];
                 p_left = ws.hi[p_c] - lo;
                 if (p_left == 0) continue;
-                p_tps = tps_of(p_c);
-                p_rec = (uint32_t)pool_rec_bytes(p_c);
-                const int bt = (int)block_tiles(p_c);
+                p_tps = tps_of<G>(p_c);
+                p_rec = (uint32_t)pool_rec_bytes(p_c, G);
+                const int bt = (int)block_tiles(p_c, G);
                 const int blk = lo / bt;
                 p_in_block = bt - (lo - blk * bt);
                 p_phase = p_tps - lo % p_tps;          // tiles up to the next stage boundary
@@ -547,7 +567,7 @@ k_decode_attn(DecodeParams P) {
                 next_pool();
             } else if (p_in_block == 0) {              // on to the stream's next block
                 p_ptr = P.store.arena + (size_t)p_next_id * kBlockBytes;
-                p_in_block = (int)block_tiles(p_c);
+                p_in_block = (int)block_tiles(p_c, G);
                 ++p_tab;
                 p_next_id = p_tab[0];
             }
@@ -567,7 +587,7 @@ k_decode_attn(DecodeParams P) {
             const int hi = ws.hi[CLS];
             if (tile0 >= hi || failed) return;
             const uint32_t cnt = ws.cnt[CLS];
-            int phase = tiles_per_stage(CLS) - tile0 % tiles_per_stage(CLS);        // tiles up to the next stage boundary
+            int phase = tiles_per_stage(CLS, G) - tile0 % tiles_per_stage(CLS, G);  // tiles up to the next stage boundary
             uint32_t qreg[kQRegs];
             C::enter(qi, qreg, acc);
             while (tile0 < hi) {
@@ -576,7 +596,7 @@ k_decode_attn(DecodeParams P) {
                     break;
                 }
                 const int ntiles = min(phase, hi - tile0);
-                phase = tiles_per_stage(CLS);
+                phase = tiles_per_stage(CLS, G);
                 const uint8_t* buf = my_ring + (size_t)cslot * kStageBytes;
                 typename C::KIn kin = C::load_k(buf, half, t);
                 for (int i = 0; i < ntiles; ++i) {
@@ -600,9 +620,9 @@ k_decode_attn(DecodeParams P) {
             }
             C::leave(acc);
         };
-        walk(std::integral_constant<int, 0>{}, Quantized<0>{});
-        walk(std::integral_constant<int, 1>{}, Quantized<1>{});
-        walk(std::integral_constant<int, 2>{}, Quantized<2>{});
+        walk(std::integral_constant<int, 0>{}, Quantized<0, G>{});
+        walk(std::integral_constant<int, 1>{}, Quantized<1, G>{});
+        walk(std::integral_constant<int, 2>{}, Quantized<2, G>{});
         walk(std::integral_constant<int, 3>{}, Fp16Rows{});
 
         if (failed) {
@@ -650,7 +670,8 @@ k_decode_attn(DecodeParams P) {
         }
         // both lanes of a token added its p and p * zero-point: halve the warp sums
         const float l_w = 0.5f * warp_sum(st.l);
-        const float b_w = 0.5f * warp_sum(st.bsum);
+        // (with two scale groups each half has its own zero-points: the sum stays inside the half)
+        const float b_w = G == 1 ? 0.5f * warp_sum(st.bsum) : half_sum(st.bsum);
         const uint32_t jf = decode_first_warp(u, P.units, P.gw);
         const size_t rec0 = (size_t)u * P.pslots;
         reinterpret_cast<float2*>(P.part_o + (rec0 + (j - jf)) * kHeadDim)[lane] = make_float2(r2[0] + b_w, r2[1] + b_w);

@@ -15,7 +15,7 @@ struct ExportParams {
     uint32_t* pool_slot;    // [nb][n]
     uint4* k_codes;         // [nb][n][kv_heads][8] (16-byte units)
     uint4* v_codes;
-    uint16_t* k_meta;       // [nb][n][kv_heads][2]
+    uint16_t* k_meta;       // [nb][n][kv_heads][2 * scale groups]
     uint16_t* v_meta;
 };
 
@@ -39,7 +39,7 @@ k_export(ExportParams p) {
         const int j = it & 7, tensor = (it >> 3) & 1, h = it >> 4;
         uint4* dst = tensor ? p.v_codes : p.k_codes;
         if (!dst) continue;
-        const uint8_t* codes = tile_ptr(s, cls, stream_table(s, cls, p.layer, b, h), (uint32_t)tile) +
+        const uint8_t* codes = tile_ptr(s, cls, stream_table(s, cls, p.layer, b, h), (uint32_t)tile, s.groups) +
                                (size_t)tensor * pool_codes_bytes(cls);
         uint4 v = make_uint4(0, 0, 0, 0);
         if (j < W) {
@@ -54,17 +54,18 @@ k_export(ExportParams p) {
         }
         dst[(tok * s.kv_heads + h) * 8 + j] = v;
     }
-    for (int it = threadIdx.x; it < s.kv_heads * 2; it += blockDim.x) {
-        const int tensor = it & 1, h = it >> 1;
+    const int G = s.groups;
+    for (int it = threadIdx.x; it < s.kv_heads * 2 * G; it += blockDim.x) {
+        const int g = it % G, tensor = (it / G) & 1, h = it / (2 * G);
         uint16_t* dst = tensor ? p.v_meta : p.k_meta;
         if (!dst) continue;
         uint32_t m = 0;
         if (cls < 3) {
-            const uint8_t* rec = tile_ptr(s, cls, stream_table(s, cls, p.layer, b, h), (uint32_t)tile);
-            m = *reinterpret_cast<const uint32_t*>(rec + meta_offset(cls, tensor, t));
+            const uint8_t* rec = tile_ptr(s, cls, stream_table(s, cls, p.layer, b, h), (uint32_t)tile, G);
+            m = *reinterpret_cast<const uint32_t*>(rec + meta_offset(cls, tensor, t, g, G));
         }
-        dst[(tok * s.kv_heads + h) * 2 + 0] = (uint16_t)(m & 0xffffu);
-        dst[(tok * s.kv_heads + h) * 2 + 1] = (uint16_t)(m >> 16);
+        dst[((tok * s.kv_heads + h) * G + g) * 2 + 0] = (uint16_t)(m & 0xffffu);
+        dst[((tok * s.kv_heads + h) * G + g) * 2 + 1] = (uint16_t)(m >> 16);
     }
 }
 

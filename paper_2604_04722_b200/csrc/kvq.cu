@@ -24,6 +24,7 @@ using namespace kvq;
 struct kvq_ctx {
     int device = 0, sm_count = 0;
     int layers = 0, q_heads = 0, kv_heads = 0, max_ctx = 0, batch = 0;
+    int groups = 1;                      // {scale, zero-point} pairs per quantized row: 1 or 2
     StoreView store{};
     uint8_t* arena = nullptr;            // the tile records: blocks of kBlockBytes
     uint32_t* table = nullptr;           // block tables of all streams
@@ -192,19 +193,30 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
     dim3 grid_q(p.nchunks, groups, c->batch);
     if (n_new == 1 && !call_ragged && (!fused || c->hidden == 32)) {   // a decode step: one warp per 16 heads
         dim3 grid_t((c->kv_heads + 15) / 16, c->batch);
-        if (fused) k_append_token<true><<<grid_t, 32, 0, st>>>(p);
-        else k_append_token<false><<<grid_t, 32, 0, st>>>(p);
+        if (c->groups == 1) {
+            if (fused) k_append_token<true, 1><<<grid_t, 32, 0, st>>>(p);
+            else k_append_token<false, 1><<<grid_t, 32, 0, st>>>(p);
+        } else {
+            if (fused) k_append_token<true, 2><<<grid_t, 32, 0, st>>>(p);
+            else k_append_token<false, 2><<<grid_t, 32, 0, st>>>(p);
+        }
         c->launches += 1;
     } else if (p.nchunks == 1) {
-        if (fused) k_quant_pack<2><<<grid_q, kChunkTokens, kAppendRingBytes + smem, st>>>(p);
-        else k_quant_pack<1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+        if (c->groups == 1) {
+            if (fused) k_quant_pack<2, 1><<<grid_q, kChunkTokens, kAppendRingBytes + smem, st>>>(p);
+            else k_quant_pack<1, 1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+        } else {
+            if (fused) k_quant_pack<2, 2><<<grid_q, kChunkTokens, kAppendRingBytes + smem, st>>>(p);
+            else k_quant_pack<1, 2><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+        }
         c->launches += 1;
     } else {
         dim3 grid_c(p.nchunks, c->batch);
         if (fused) k_classify<true><<<grid_c, kChunkTokens, smem, st>>>(p);
         else k_classify<false><<<grid_c, kChunkTokens, 0, st>>>(p);
         k_reserve_blocks<<<c->batch, 128, 0, st>>>(p);
-        k_quant_pack<0><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+        if (c->groups == 1) k_quant_pack<0, 1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+        else k_quant_pack<0, 2><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
         c->launches += 3;
     }
     KVQ_CUDA(c, cudaGetLastError());
@@ -297,6 +309,12 @@ void fill_decode_params(kvq_ctx* c, int layer, const void* Q, void* O, float* pa
     p.pslots = decode_pslots(p.units, gw);
 }
 
+template <bool STATS>
+void launch_decode(const kvq_ctx* c, uint32_t grid, const DecodeParams& p, cudaStream_t st) {
+    if (c->groups == 1) k_decode_attn<STATS, 1><<<grid, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    else k_decode_attn<STATS, 2><<<grid, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+}
+
 int export_impl(kvq_ctx* c, int layer, int b0, int nb, int pos0, int n, uint8_t* bits, uint32_t* pool_slot,
                 void* k_codes, void* v_codes, uint16_t* k_meta, uint16_t* v_meta, cudaStream_t st) {
     ExportParams p{};
@@ -328,8 +346,14 @@ int kvq_create(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_di
 
 int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
                      uint64_t arena_bytes) {
+    return kvq_create_grouped(out, layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes, 1);
+}
+
+int kvq_create_grouped(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
+                       uint64_t arena_bytes, int scale_groups) {
     if (!out) return KVQ_ERR_ARG;
     *out = nullptr;
+    if (scale_groups != 1 && scale_groups != 2) return KVQ_ERR_ARG;
     if (layers < 1 || q_heads < 1 || kv_heads < 1 || batch < 1 || max_ctx < 1) return KVQ_ERR_ARG;
     if (head_dim != kHeadDim || q_heads % kv_heads != 0) return KVQ_ERR_ARG;
     if (max_ctx > (1 << 30) - 1 || batch > 65535 || q_heads > 65535) return KVQ_ERR_ARG;
@@ -346,6 +370,7 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
     c->kv_heads = kv_heads;
     c->max_ctx = max_ctx;
     c->batch = batch;
+    c->groups = scale_groups;
     c->len.assign(layers, 0);
     c->lens.assign((size_t)layers * batch, 0);
     c->ragged.assign(layers, 0);
@@ -356,6 +381,7 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
     s.kv_heads = kv_heads;
     s.q_heads = q_heads;
     s.max_ctx = max_ctx;
+    s.groups = scale_groups;
     s.cap_tiles = (max_ctx + kTileTokens - 1) / kTileTokens;
 
     // block tables: one row per stream, class k at table_off[k]; one spare entry at the very end because
@@ -364,7 +390,7 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
     uint32_t row = 0;
     for (int k = 0; k < kNumPools; ++k) {
         s.table_off[k] = row;
-        row += blocks_for(k, (uint32_t)max_ctx);
+        row += blocks_for(k, (uint32_t)max_ctx, scale_groups);
     }
     s.table_stride = row;
     const uint64_t worst_blocks = (uint64_t)streams * row + 1;           // every token in every class, plus block 0
@@ -401,7 +427,7 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
     ok = ok && dev_alloc(c, &c->st_Q, sizeof(__half) * units * kHeadDim) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_O, sizeof(__half) * units * kHeadDim) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_bits, (size_t)batch) == cudaSuccess;
-    ok = ok && dev_alloc(c, &c->st_export, (size_t)kv_heads * (2 * KVQ_EXPORT_ROW_BYTES + 8) + 16) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->st_export, (size_t)kv_heads * (2 * KVQ_EXPORT_ROW_BYTES + 8 * scale_groups) + 16) == cudaSuccess;
     if (ok) {
         s.arena = c->arena;
         s.table = c->table;
@@ -419,13 +445,14 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
         ok = ok && cudaFuncSetAttribute(k_select_bits, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(k_classify<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) == cudaSuccess;
         const int ring = (int)kAppendRingBytes;
-        ok = ok && cudaFuncSetAttribute(k_quant_pack<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring) == cudaSuccess;
-        ok = ok && cudaFuncSetAttribute(k_quant_pack<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring) == cudaSuccess;
-        ok = ok && cudaFuncSetAttribute(k_quant_pack<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, ring + smem_max) == cudaSuccess;
-        ok = ok && cudaFuncSetAttribute(k_decode_attn<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)kDecodeSmemBytes) == cudaSuccess;
-        ok = ok && cudaFuncSetAttribute(k_decode_attn<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)kDecodeSmemBytes) == cudaSuccess;
+        auto dyn_smem = [](auto kernel, int bytes) {
+            return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+        };
+        ok = ok && dyn_smem(k_quant_pack<0, 1>, ring) && dyn_smem(k_quant_pack<0, 2>, ring);
+        ok = ok && dyn_smem(k_quant_pack<1, 1>, ring) && dyn_smem(k_quant_pack<1, 2>, ring);
+        ok = ok && dyn_smem(k_quant_pack<2, 1>, ring + smem_max) && dyn_smem(k_quant_pack<2, 2>, ring + smem_max);
+        ok = ok && dyn_smem(k_decode_attn<false, 1>, (int)kDecodeSmemBytes) && dyn_smem(k_decode_attn<false, 2>, (int)kDecodeSmemBytes);
+        ok = ok && dyn_smem(k_decode_attn<true, 1>, (int)kDecodeSmemBytes) && dyn_smem(k_decode_attn<true, 2>, (int)kDecodeSmemBytes);
         ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     }
     if (!ok) {
@@ -513,7 +540,7 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
     const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
     cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 2] : nullptr;
     if (rec) cudaEventRecord(ev[0], st);
-    k_decode_attn<false><<<grid, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    launch_decode<false>(c, grid, p, st);
     if (rec) {
         cudaEventRecord(ev[1], st);
         c->prof_calls += 1;
@@ -531,7 +558,7 @@ int kvq_decode_attn_var(kvq_ctx* c, int layer, const void* Q, void* O, float* va
     DecodeParams p{};
     fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt,
                        choose_warps(c, c->len[layer], (uint64_t)c->batch * c->q_heads), p);
-    k_decode_attn<true><<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    launch_decode<true>(c, (p.gw + kDecodeWarps - 1) / kDecodeWarps, p, st);
     k_head_mean<<<c->batch, 32, 0, st>>>(c->unit_var, c->q_heads, var_out);
     c->launches += 2;
     KVQ_CUDA(c, cudaGetLastError());
@@ -583,7 +610,7 @@ int kvq_attend_last(kvq_ctx* c, int layer, const void* Q, void* O, int n_queries
         p.t0 = (uint32_t)t0;
         p.units = (uint32_t)units;
         p.pslots = decode_pslots(p.units, p.gw);
-        k_decode_attn<false><<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+        launch_decode<false>(c, (p.gw + kDecodeWarps - 1) / kDecodeWarps, p, st);
         c->launches += 2;
     }
     KVQ_CUDA(c, cudaGetLastError());
@@ -626,7 +653,7 @@ int kvq_decode_attn_static(kvq_ctx* c, int layer, const void* Q, void* O, void* 
     DecodeParams p{};
     fill_decode_params(c, layer, Q, O, base, reinterpret_cast<float2*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * kHeadDim),
                        reinterpret_cast<uint32_t*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * (kHeadDim + 2)), gw, p);
-    k_decode_attn<false><<<(p.gw + kDecodeWarps - 1) / kDecodeWarps, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    launch_decode<false>(c, (p.gw + kDecodeWarps - 1) / kDecodeWarps, p, st);
     c->launches += 1;
     KVQ_CUDA(c, cudaGetLastError());
     return KVQ_OK;
@@ -698,7 +725,7 @@ int kvq_export_token(kvq_ctx* c, int layer, int b, int pos, uint8_t* bits, uint3
         pos >= c->lens[(size_t)layer * c->batch + (b < 0 || b >= c->batch ? 0 : b)])
         return KVQ_ERR_ARG;
     DeviceGuard guard(c->device);
-    const size_t row = (size_t)c->kv_heads * KVQ_EXPORT_ROW_BYTES, meta = (size_t)c->kv_heads * 4;
+    const size_t row = (size_t)c->kv_heads * KVQ_EXPORT_ROW_BYTES, meta = (size_t)c->kv_heads * 4 * c->groups;
     uint8_t* d_k = c->st_export;
     uint8_t* d_v = d_k + row;
     uint8_t* d_km = d_v + row;
@@ -729,7 +756,7 @@ int kvq_stats(kvq_ctx* c, int layer, uint32_t* host_counts, uint64_t* resident_b
     for (int b = 0; b < c->batch; ++b)
         for (int k = 0; k < kNumPools; ++k) {
             const uint64_t n = cnt[(size_t)b * 4 + k];
-            bytes += n * (uint64_t)c->kv_heads * pool_row_bytes(k);
+            bytes += n * (uint64_t)c->kv_heads * pool_row_bytes(k, c->groups);
             tokens += n;
             bit_sum += n * (uint64_t)pool_bits(k);
         }

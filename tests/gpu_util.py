@@ -24,9 +24,14 @@ def dev(a: np.ndarray) -> torch.Tensor:
 class GpuCache:
     """A kvq handle plus the shapes needed to size export buffers."""
 
-    def __init__(self, layers, batch, q_heads, kv_heads, max_ctx, head_dim=64):
+    def __init__(self, layers, batch, q_heads, kv_heads, max_ctx, head_dim=64, scale_groups=1, arena_bytes=0):
         self.L, self.B, self.Hq, self.Hkv, self.max_ctx = layers, batch, q_heads, kv_heads, max_ctx
-        self.ctx = kq.kvq_create(layers, q_heads, kv_heads, head_dim, max_ctx, batch)
+        self.G = scale_groups
+        if scale_groups == 1 and arena_bytes == 0:
+            self.ctx = kq.kvq_create(layers, q_heads, kv_heads, head_dim, max_ctx, batch)
+        else:
+            self.ctx = kq.kvq_create_grouped(layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes,
+                                             scale_groups)
 
     def close(self):
         if self.ctx:
@@ -76,7 +81,7 @@ class GpuCache:
         ps = torch.zeros((B, n), dtype=torch.int32, device=DEV)
         kc = torch.zeros((B, n, H, 128), dtype=torch.uint8, device=DEV)
         vc = torch.zeros_like(kc)
-        km = torch.zeros((B, n, H, 2), dtype=torch.int16, device=DEV)
+        km = torch.zeros((B, n, H, 2 * self.G), dtype=torch.int16, device=DEV)
         vm = torch.zeros_like(km)
         kq.kvq_export_range(self.ctx, layer, pos0, n, bits, ps, kc, vc, km, vm)
         torch.cuda.synchronize()
