@@ -61,6 +61,9 @@
 #ifndef KVQ_DECODE_WARPS
 #define KVQ_DECODE_WARPS 4
 #endif
+#ifndef KVQ_DECODE_FMA2
+#define KVQ_DECODE_FMA2 1          // V-side accumulation with packed two-lane fp32 FMAs
+#endif
 #ifndef KVQ_DECODE_MIN_CTAS
 #define KVQ_DECODE_MIN_CTAS 4
 #endif
@@ -201,6 +204,19 @@ __device__ __forceinline__ float field_as_float(uint32_t w, uint32_t w_shr8, int
     if (k + BITS <= 24) return __uint_as_float(w & (mask << k));
     if (BITS == 8) return __uint_as_float(w >> 24);
     return __uint_as_float(w_shr8 & (mask << (k - 8)));
+}
+
+// c0 += a0 * b, c1 += a1 * b as one packed instruction (two fp32 lanes in a 64-bit register pair).
+__device__ __forceinline__ void fma2(float& c0, float& c1, float a0, float a1, float b) {
+#if KVQ_DECODE_FMA2
+    asm("{ .reg .b64 a, b, c;\n mov.b64 a, {%2, %3};\n mov.b64 b, {%4, %4};\n mov.b64 c, {%0, %1};\n"
+        " fma.rn.f32x2 c, a, b, c;\n mov.b64 {%0, %1}, c; }"
+        : "+f"(c0), "+f"(c1)
+        : "f"(a0), "f"(a1), "f"(b));
+#else
+    c0 = fmaf(a0, b, c0);
+    c1 = fmaf(a1, b, c1);
+#endif
 }
 
 __device__ __forceinline__ float warp_max(float v) {
@@ -373,9 +389,9 @@ struct Quantized {
         for (int wi = 0; wi < WORDS; ++wi) {
             const uint32_t hi8 = w[wi] >> 8;
 #pragma unroll
-            for (int e = 0; e < EPW; ++e) {
+            for (int e = 0; e < EPW; e += 2) {
                 const int i = wi * EPW + e;
-                acc[i] = fmaf(field_as_float<BITS>(w[wi], hi8, e), wv, acc[i]);
+                fma2(acc[i], acc[i + 1], field_as_float<BITS>(w[wi], hi8, e), field_as_float<BITS>(w[wi], hi8, e + 1), wv);
             }
         }
     }
@@ -419,8 +435,7 @@ struct Fp16Rows {
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi) {
                 const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[wi]));
-                acc[u * 8 + wi * 2] = fmaf(p, f.x, acc[u * 8 + wi * 2]);
-                acc[u * 8 + wi * 2 + 1] = fmaf(p, f.y, acc[u * 8 + wi * 2 + 1]);
+                fma2(acc[u * 8 + wi * 2], acc[u * 8 + wi * 2 + 1], f.x, f.y, p);
             }
         }
     }
