@@ -44,9 +44,9 @@ UNIT = "GB/s"
 
 # DRAM traffic of one k_decode_attn launch on this workload (dram__bytes_read.sum +
 # dram__bytes_write.sum): captured with a quarter of the sequences (profiles/k_decode_attn_cfg5_batch4.md,
-# 320.7 MB per launch) and scaled by the rows read (x 4); every row is read exactly once, so traffic
+# 320.0 MB per launch) and scaled by the rows read (x 4); every row is read exactly once, so traffic
 # grows in proportion.  Set to None whenever the kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 320.7e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 320.0e6
 
 
 def measured_peak_gbs():

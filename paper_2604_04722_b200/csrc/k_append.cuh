@@ -119,6 +119,23 @@ __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+#ifndef KVQ_APPEND_F32X2
+#define KVQ_APPEND_F32X2 1         // the quantizer's subtract, multiply and rounding add as packed two-lane fp32 operations
+#endif
+// v0 = fl(fl(fl(x0 - mn) * inv) + magic), v1 likewise: three correctly rounded operations per lane, as packed
+// two-lane instructions (same results as the scalar ones).
+__device__ __forceinline__ void quantize_pair(float x0, float x1, float mn, float inv, float magic, float& v0, float& v1) {
+#if KVQ_APPEND_F32X2
+    asm("{ .reg .b64 x, m, s, g;\n mov.b64 x, {%2, %3};\n mov.b64 m, {%4, %4};\n mov.b64 s, {%5, %5};\n mov.b64 g, {%6, %6};\n"
+        " sub.rn.f32x2 x, x, m;\n mul.rn.f32x2 x, x, s;\n add.rn.f32x2 x, x, g;\n mov.b64 {%0, %1}, x; }"
+        : "=f"(v0), "=f"(v1)
+        : "f"(x0), "f"(x1), "f"(mn), "f"(inv), "f"(magic));
+#else
+    v0 = __fadd_rn(__fmul_rn(__fsub_rn(x0, mn), inv), magic);
+    v1 = __fadd_rn(__fmul_rn(__fsub_rn(x1, mn), inv), magic);
+#endif
+}
+
 // Codes of the 32 values hp[0..15] packed little-endian into words.  rint is done by adding
 // 1.5 * 2^23 (the sum's bit pattern is 0x4B400000 + code); the words are sums of shifted bit patterns
 // in wrapping 32-bit arithmetic, minus the constant the 0x4B400000 terms add up to.
@@ -135,13 +152,17 @@ __device__ __forceinline__ void pack_codes(const __half2* hp, float mn, float in
 #pragma unroll
         for (int e = 0; e < EPW; e += 2) {
             const float2 f = __half22float2(hp[(wi * EPW + e) / 2]);
-            float v0 = __fmul_rn(__fsub_rn(f.x, mn), inv), v1 = __fmul_rn(__fsub_rn(f.y, mn), inv);
+            float r0, r1;
             if (CLAMP) {
-                v0 = fminf(v0, LEVELS);
-                v1 = fminf(v1, LEVELS);
+                const float v0 = fminf(__fmul_rn(__fsub_rn(f.x, mn), inv), LEVELS);
+                const float v1 = fminf(__fmul_rn(__fsub_rn(f.y, mn), inv), LEVELS);
+                r0 = __fadd_rn(v0, kRoundMagic);
+                r1 = __fadd_rn(v1, kRoundMagic);
+            } else {
+                quantize_pair(f.x, f.y, mn, inv, kRoundMagic, r0, r1);
             }
-            acc += __float_as_uint(__fadd_rn(v0, kRoundMagic)) << (BITS * e);
-            acc += __float_as_uint(__fadd_rn(v1, kRoundMagic)) << (BITS * (e + 1));
+            acc += __float_as_uint(r0) << (BITS * e);
+            acc += __float_as_uint(r1) << (BITS * (e + 1));
         }
         w[wi] = acc;
     }
