@@ -120,16 +120,22 @@ __device__ __forceinline__ void cp_async_wait() {
 }
 
 #ifndef KVQ_APPEND_F32X2
-#define KVQ_APPEND_F32X2 1         // the quantizer's subtract, multiply and rounding add as packed two-lane fp32 operations
+#define KVQ_APPEND_F32X2 1         // the quantizer's subtract and multiply as packed two-lane fp32 operations
 #endif
-// v0 = fl(fl(fl(x0 - mn) * inv) + magic), v1 likewise: three correctly rounded operations per lane, as packed
-// two-lane instructions (same results as the scalar ones).
+// v0 = fl(fl(fl(x0 - mn) * inv) + magic), v1 likewise: three correctly rounded operations per lane.  The
+// subtraction and the product are packed two-lane instructions (same results as the scalar ones); the
+// rounding add stays scalar, because a packed product followed by a packed sum is contracted into one
+// fused operation by the assembler even with explicit rounding modifiers, and a fused product-sum
+// rounds differently where the product is within half an ulp of a tie.
 __device__ __forceinline__ void quantize_pair(float x0, float x1, float mn, float inv, float magic, float& v0, float& v1) {
 #if KVQ_APPEND_F32X2
-    asm("{ .reg .b64 x, m, s, g;\n mov.b64 x, {%2, %3};\n mov.b64 m, {%4, %4};\n mov.b64 s, {%5, %5};\n mov.b64 g, {%6, %6};\n"
-        " sub.rn.f32x2 x, x, m;\n mul.rn.f32x2 x, x, s;\n add.rn.f32x2 x, x, g;\n mov.b64 {%0, %1}, x; }"
-        : "=f"(v0), "=f"(v1)
-        : "f"(x0), "f"(x1), "f"(mn), "f"(inv), "f"(magic));
+    float p0, p1;
+    asm("{ .reg .b64 x, m, s;\n mov.b64 x, {%2, %3};\n mov.b64 m, {%4, %4};\n mov.b64 s, {%5, %5};\n"
+        " sub.rn.f32x2 x, x, m;\n mul.rn.f32x2 x, x, s;\n mov.b64 {%0, %1}, x; }"
+        : "=f"(p0), "=f"(p1)
+        : "f"(x0), "f"(x1), "f"(mn), "f"(inv));
+    v0 = __fadd_rn(p0, magic);
+    v1 = __fadd_rn(p1, magic);
 #else
     v0 = __fadd_rn(__fmul_rn(__fsub_rn(x0, mn), inv), magic);
     v1 = __fadd_rn(__fmul_rn(__fsub_rn(x1, mn), inv), magic);
