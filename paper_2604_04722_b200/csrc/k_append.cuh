@@ -534,6 +534,8 @@ __device__ __forceinline__ void token_store(int c, const uint4 (&kraw)[4], const
 template <bool FUSED, int G>
 __global__ void __launch_bounds__(32)
 k_append_token(AppendParams p) {
+    pdl_launch_dependents();
+    pdl_wait();                                        // the attention of the previous step still reads the store
     const int lane = threadIdx.x, b = blockIdx.y;
     const int h = blockIdx.x * 16 + (lane >> 1), half = lane & 1;
     const bool active = h < p.store.kv_heads;

@@ -484,6 +484,8 @@ k_decode_attn(DecodeParams P) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
+    pdl_launch_dependents();                           // the next step's append may be scheduled behind this launch
+    pdl_wait();                                        // the append before this launch has stored its token
 
     int pslot = 0, cslot = 0;                          // ring slot the next copy goes to / the next chunk is read from
     uint32_t parity = 0;                               // phase parity of cslot

@@ -91,6 +91,30 @@ cudaError_t dev_alloc(kvq_ctx* c, T** p, size_t bytes) {
 
 constexpr int kProfMaxCalls = 1024;
 
+#ifndef KVQ_OVERLAP_LAUNCHES
+#define KVQ_OVERLAP_LAUNCHES 1
+#endif
+// Launch with programmatic stream serialization (see pdl_wait): the kernel may be scheduled before the
+// kernel ahead of it in the stream has finished, if that kernel allows it; it waits inside for its end.
+template <class Params>
+void launch_overlapped(void (*kernel)(Params), dim3 grid, unsigned block, size_t smem, cudaStream_t st, const Params& p) {
+#if KVQ_OVERLAP_LAUNCHES
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, p);
+#else
+    kernel<<<grid, block, smem, st>>>(p);
+#endif
+}
+
 void free_all(kvq_ctx* c) {
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     c->prof_ev.clear();
@@ -194,11 +218,11 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
     if (n_new == 1 && !call_ragged && (!fused || c->hidden == 32)) {   // a decode step: one warp per 16 heads
         dim3 grid_t((c->kv_heads + 15) / 16, c->batch);
         if (c->groups == 1) {
-            if (fused) k_append_token<true, 1><<<grid_t, 32, 0, st>>>(p);
-            else k_append_token<false, 1><<<grid_t, 32, 0, st>>>(p);
+            if (fused) launch_overlapped(k_append_token<true, 1>, grid_t, 32, 0, st, p);
+            else launch_overlapped(k_append_token<false, 1>, grid_t, 32, 0, st, p);
         } else {
-            if (fused) k_append_token<true, 2><<<grid_t, 32, 0, st>>>(p);
-            else k_append_token<false, 2><<<grid_t, 32, 0, st>>>(p);
+            if (fused) launch_overlapped(k_append_token<true, 2>, grid_t, 32, 0, st, p);
+            else launch_overlapped(k_append_token<false, 2>, grid_t, 32, 0, st, p);
         }
         c->launches += 1;
     } else if (p.nchunks == 1) {
@@ -311,8 +335,8 @@ void fill_decode_params(kvq_ctx* c, int layer, const void* Q, void* O, float* pa
 
 template <bool STATS>
 void launch_decode(const kvq_ctx* c, uint32_t grid, const DecodeParams& p, cudaStream_t st) {
-    if (c->groups == 1) k_decode_attn<STATS, 1><<<grid, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
-    else k_decode_attn<STATS, 2><<<grid, kDecodeThreads, kDecodeSmemBytes, st>>>(p);
+    if (c->groups == 1) launch_overlapped(k_decode_attn<STATS, 1>, dim3(grid), kDecodeThreads, kDecodeSmemBytes, st, p);
+    else launch_overlapped(k_decode_attn<STATS, 2>, dim3(grid), kDecodeThreads, kDecodeSmemBytes, st, p);
 }
 
 int export_impl(kvq_ctx* c, int layer, int b0, int nb, int pos0, int n, uint8_t* bits, uint32_t* pool_slot,

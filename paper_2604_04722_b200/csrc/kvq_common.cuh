@@ -66,6 +66,14 @@ __host__ __device__ constexpr int meta_offset(int c, int tensor, int t, int half
     return 2 * pool_codes_bytes(c) + tensor * pool_meta_bytes(c, g) + (g == 2 ? half * 4 * kTileTokens : 0) + 4 * t;
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may be scheduled
+// while the kernel before it in the stream is still running, once every CTA of that kernel has called
+// pdl_launch_dependents (or exited); it must call pdl_wait before it touches memory the earlier kernel reads
+// or writes.  pdl_wait returns when the earlier kernel has completed and its writes are visible; without the
+// attribute both are no-ops.  Only the decode-step kernels use this, to hide each other's launch latency.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 constexpr uint32_t kBlockBytes = 65536;
 // Tiles per block: a whole number of ring stages of the decode kernel (10 / 5 / 3 / 1 tiles).
 // (with two scale groups the records are 768 / 1280 / 2304 / 4096 bytes: 80 / 50 / 28 / 16 tiles)

@@ -163,3 +163,51 @@ def test_ragged_batch_with_grouped_scales(gu, oracle):
         out = g.decode(0, Q)
         for b in range(B):
             gu.assert_attention_close(out[b:b + 1], ocs[b].decode_attn(Q[b:b + 1]), "sequence %d" % b)
+
+
+def test_the_other_attention_entry_points_on_a_grouped_cache(gu, oracle):
+    """Causal rows for the last positions, the statistics variant, the fixed-scratch variant and the host-buffer
+    step all run the same kernel template; with grouped scales each must agree with the grouped oracle."""
+    import torch
+    from paper_2604_04722_b200 import binding as kq
+    rng = np.random.default_rng(21)
+    B, Hq, H, n, T = 2, 4, 2, 300, 3
+    K, V = _kv(rng, B, n, H)
+    bits = BITS[rng.choice(4, size=(B, n), p=[.4, .3, .2, .1])]
+    Q = rng.standard_normal((B, T, Hq, 64)).astype(np.float16)
+    with gu.GpuCache(1, B, Hq, H, n + 1, scale_groups=2) as g:
+        g.append(0, K, V, bits)
+        Qd = gu.dev(Q.view(np.uint16))
+        O = torch.zeros_like(Qd)
+        kq.kvq_attend_last(g.ctx, 0, Qd, O, T)
+        torch.cuda.synchronize()
+        got = O.cpu().numpy().view(np.uint16)
+        for i in range(T):                              # row i sees positions <= n - T + i
+            upto = n - T + i + 1
+            oc = oracle.GroupedOracleCache(B, Hq, H, 2)
+            oc.append(K[:, :upto], V[:, :upto], bits[:, :upto])
+            gu.assert_attention_close(got[:, i], oc.decode_attn(np.ascontiguousarray(Q[:, i])), "row %d" % i)
+        want = oc.decode_attn(np.ascontiguousarray(Q[:, T - 1]))            # the whole cache, last query row
+        Ql = gu.dev(np.ascontiguousarray(Q[:, T - 1]).view(np.uint16))
+        O1, O2 = torch.zeros_like(Ql), torch.zeros_like(Ql)
+        var = torch.zeros(B, dtype=torch.float32, device=gu.DEV)
+        kq.kvq_decode_attn_var(g.ctx, 0, Ql, O1, var)
+        kq.kvq_decode_attn_static(g.ctx, 0, Ql, O2)
+        torch.cuda.synchronize()
+        gu.assert_attention_close(O1.cpu().numpy().view(np.uint16), want, "statistics variant")
+        gu.assert_attention_close(O2.cpu().numpy().view(np.uint16), want, "fixed-scratch variant")
+        assert np.all(np.isfinite(var.cpu().numpy())) and np.all(var.cpu().numpy() >= 0)
+        # one step from host buffers: append a controller-decided token, then attend
+        cw = synth.controller_weights(322, 32)
+        g.set_controller(cw)
+        Kn, Vn = _kv(rng, B, 1, H)
+        feats = synth.features_batch(3, B, 0, 1).astype(np.float32)
+        nb, _, _ = oracle.select_bits(feats, 32, *cw.as_tuple())
+        Qh = np.ascontiguousarray(Q[:, 0])
+        Oh = np.zeros_like(Qh)
+        bo = np.zeros((B, 1), np.uint8)
+        kq.kvq_decode_step_host(g.ctx, 0, feats, Kn.view(np.uint16), Vn.view(np.uint16), Qh.view(np.uint16),
+                                Oh.view(np.uint16), bo)
+        assert np.array_equal(bo, nb)
+        oc.append(Kn, Vn, nb)
+        gu.assert_attention_close(Oh.view(np.uint16), oc.decode_attn(Qh), "host-buffer step")
