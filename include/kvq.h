@@ -263,8 +263,12 @@ int kvq_decode_attn_static(kvq_ctx* ctx, int layer, const void* Q, void* O, void
  * attention of Q over the layer, result copied back.  feats host fp32
  * [batch][4]; K, V host fp16 [batch][1][kv_heads][64]; Q host fp16
  * [batch][q_heads][64]; O host fp16 [batch][q_heads][64] (written);
- * bits_out_opt host uint8 [batch] or NULL.  Uses staging buffers owned by the
- * handle; returns after the stream has been synchronized.
+ * bits_out_opt host uint8 [batch] or NULL.  Returns after the stream has been
+ * synchronized.  When feats, K, V, Q and O are all page-locked (cudaHostAlloc,
+ * cudaHostRegister, a pinned torch tensor) and 16-byte aligned, the kernels read
+ * and write them across the bus directly; otherwise the call copies through
+ * staging buffers owned by the handle.  Either way every byte of the step's
+ * inputs and of its result crosses the bus inside the call.
  */
 int kvq_decode_step_host(kvq_ctx* ctx, int layer, const float* feats, const void* K,
                          const void* V, const void* Q, void* O, uint8_t* bits_out_opt,

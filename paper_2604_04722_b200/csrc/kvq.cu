@@ -145,6 +145,18 @@ void free_all(kvq_ctx* c) {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The device's address for a page-locked host buffer, or nullptr if `p` is not one (pageable memory, or an
+// address the kernels' 16-byte accesses could not use).
+const void* device_view(const void* p) {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    if (a.type != cudaMemoryTypeHost || !a.devicePointer || !aligned16(a.devicePointer)) return nullptr;
+    return a.devicePointer;
+}
+
 inline uint32_t* counts_of(kvq_ctx* c, int which, int layer) {
     return c->counts + ((size_t)which * c->layers + layer) * c->batch * 4;
 }
@@ -692,15 +704,29 @@ int kvq_decode_step_host(kvq_ctx* c, int layer, const float* feats, const void* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t kv_bytes = sizeof(__half) * (size_t)c->batch * c->kv_heads * kHeadDim;
     const size_t q_bytes = sizeof(__half) * (size_t)c->batch * c->q_heads * kHeadDim;
-    KVQ_CUDA(c, cudaMemcpyAsync(c->st_feats, feats, sizeof(float) * 4 * c->batch, cudaMemcpyHostToDevice, st));
-    KVQ_CUDA(c, cudaMemcpyAsync(c->st_K, K, kv_bytes, cudaMemcpyHostToDevice, st));
-    KVQ_CUDA(c, cudaMemcpyAsync(c->st_V, V, kv_bytes, cudaMemcpyHostToDevice, st));
-    KVQ_CUDA(c, cudaMemcpyAsync(c->st_Q, Q, q_bytes, cudaMemcpyHostToDevice, st));
-    int rc = kvq_append_fused(c, layer, c->st_K, c->st_V, c->st_feats, 1, c->st_bits, stream);
+    // Page-locked host buffers are reachable from the device under unified addressing: the kernels then read
+    // the step's inputs and write its result across the bus themselves, which saves five copy launches.  Any
+    // buffer that is pageable (or misaligned for the kernels' 16-byte loads) sends the call through the
+    // staging buffers instead.
+    const void *d_feats = device_view(feats), *d_K = device_view(K), *d_V = device_view(V), *d_Q = device_view(Q);
+    void* d_O = const_cast<void*>(device_view(O));
+    const bool direct = d_feats && d_K && d_V && d_Q && d_O;
+    if (!direct) {
+        KVQ_CUDA(c, cudaMemcpyAsync(c->st_feats, feats, sizeof(float) * 4 * c->batch, cudaMemcpyHostToDevice, st));
+        KVQ_CUDA(c, cudaMemcpyAsync(c->st_K, K, kv_bytes, cudaMemcpyHostToDevice, st));
+        KVQ_CUDA(c, cudaMemcpyAsync(c->st_V, V, kv_bytes, cudaMemcpyHostToDevice, st));
+        KVQ_CUDA(c, cudaMemcpyAsync(c->st_Q, Q, q_bytes, cudaMemcpyHostToDevice, st));
+        d_feats = c->st_feats;
+        d_K = c->st_K;
+        d_V = c->st_V;
+        d_Q = c->st_Q;
+        d_O = c->st_O;
+    }
+    int rc = kvq_append_fused(c, layer, d_K, d_V, static_cast<const float*>(d_feats), 1, c->st_bits, stream);
     if (rc != KVQ_OK) return rc;
-    rc = kvq_decode_attn(c, layer, c->st_Q, c->st_O, stream);
+    rc = kvq_decode_attn(c, layer, d_Q, d_O, stream);
     if (rc != KVQ_OK) return rc;
-    KVQ_CUDA(c, cudaMemcpyAsync(O, c->st_O, q_bytes, cudaMemcpyDeviceToHost, st));
+    if (!direct) KVQ_CUDA(c, cudaMemcpyAsync(O, c->st_O, q_bytes, cudaMemcpyDeviceToHost, st));
     if (bits_out_opt) KVQ_CUDA(c, cudaMemcpyAsync(bits_out_opt, c->st_bits, c->batch, cudaMemcpyDeviceToHost, st));
     KVQ_CUDA(c, cudaStreamSynchronize(st));
     return KVQ_OK;

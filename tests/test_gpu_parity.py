@@ -285,13 +285,30 @@ def test_decode_after_incremental_steps(gu, oracle):
             gu.assert_attention_close(g.decode(0, Q), oc.decode_attn(Q), "step %d" % step)
 
 
-def test_decode_step_host_matches_device_path(gu, oracle):
-    """The host-buffer entry point (copies + fused append + attention) against the oracle."""
+@pytest.mark.parametrize("buffers", ["pageable", "page-locked", "page-locked but one", "page-locked, misaligned"])
+def test_decode_step_host_matches_device_path(gu, oracle, buffers):
+    """The host-buffer entry point (fused append + attention, the step's inputs and result crossing the bus)
+    against the oracle: with pageable buffers it copies through staging; with page-locked ones the kernels
+    reach them directly; one pageable buffer or a misaligned one sends the call back through staging."""
+    import torch
     from paper_2604_04722_b200 import binding as kq
     cw = synth.controller_weights(322, 32)
     rng = np.random.default_rng(19)
     B, Hq, H = 2, 6, 2
     oc = oracle.OracleCache(B, Hq, H)
+
+    def host(a, keep_pageable=False):
+        """numpy array a as the kind of host buffer under test (returns the object to pass and a numpy view)."""
+        a = np.ascontiguousarray(a)
+        raw = a.view(np.uint8).reshape(-1)
+        if buffers == "pageable" or keep_pageable:
+            return a, a
+        pad = 8 if buffers == "page-locked, misaligned" else 0
+        t = torch.zeros(raw.size + pad, dtype=torch.uint8).pin_memory()
+        t[pad:] = torch.from_numpy(raw.copy())
+        view = t[pad:].numpy().view(a.dtype).reshape(a.shape)
+        return t.data_ptr() + pad, view
+
     with gu.GpuCache(1, B, Hq, H, 80) as g:
         g.set_controller(cw)
         K, V = _kv(rng, B, 64, H)
@@ -303,13 +320,17 @@ def test_decode_step_host_matches_device_path(gu, oracle):
             K, V = _kv(rng, B, 1, H)
             feats = synth.features_batch(1, B, 64 + step, 1)
             Q = rng.standard_normal((B, Hq, 64)).astype(np.float16)
-            O = np.zeros((B, Hq, 64), np.uint16)
+            f_h, _ = host(feats[:, 0].astype(np.float32))
+            k_h, _ = host(K)
+            v_h, _ = host(V, keep_pageable=(buffers == "page-locked but one"))
+            q_h, _ = host(Q)
+            o_h, O = host(np.zeros((B, Hq, 64), np.uint16))
             got_bits = np.zeros(B, np.uint8)
-            kq.kvq_decode_step_host(g.ctx, 0, np.ascontiguousarray(feats[:, 0]), K, V, Q, O, got_bits)
+            kq.kvq_decode_step_host(g.ctx, 0, f_h, k_h, v_h, q_h, o_h, got_bits)
             want_bits, _, _ = oracle.select_bits(feats, 32, *cw.as_tuple())
             assert np.array_equal(got_bits, want_bits[:, 0])
             oc.append(K, V, want_bits)
-            gu.assert_attention_close(O, oc.decode_attn(Q), "host step %d" % step)
+            gu.assert_attention_close(O, oc.decode_attn(Q), "host step %d (%s)" % (step, buffers))
         gu.assert_store_equals_oracle(g, 0, oc)
 
 
