@@ -288,6 +288,14 @@ int kvq_seq_len(kvq_ctx* ctx, int layer, int* host_len_out);
 int kvq_set_splits(kvq_ctx* ctx, int splits);
 
 /*
+ * How a prefill append (more than 256 new tokens per sequence) cuts the new tokens into chunks
+ * for slot assignment and packing: 0 = automatic (default: 512-token chunks when that still
+ * leaves many CTAs, else 256), 256 or 512 = always that size.  The stored result does not depend
+ * on it; the setting exists for tuning and for tests.  Other values: KVQ_ERR_ARG.
+ */
+int kvq_set_append_chunk(kvq_ctx* ctx, int chunk_tokens);
+
+/*
  * Canonical copy of tokens [pos0, pos0+n) of every sequence of `layer`, for
  * comparison with other implementations.  All outputs are dev pointers:
  *   bits      uint8  [batch][n]                 2,4,8,16

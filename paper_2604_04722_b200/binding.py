@@ -51,6 +51,7 @@ SIGNATURES = {
     "kvq_reset": (_i, [_vp, _vp]),
     "kvq_seq_len": (_i, [_vp, _i, C.POINTER(_i)]),
     "kvq_set_splits": (_i, [_vp, _i]),
+    "kvq_set_append_chunk": (_i, [_vp, _i]),
     "kvq_export_range": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvq_export_token": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvq_stats": (_i, [_vp, _i, _vp, _u64p, C.POINTER(C.c_double)]),
@@ -219,6 +220,10 @@ def kvq_seq_len(ctx: int, layer: int) -> int:
     n = _i()
     check(lib().kvq_seq_len(ctx, layer, C.byref(n)), "kvq_seq_len")
     return n.value
+
+
+def kvq_set_append_chunk(ctx: int, chunk_tokens: int) -> None:
+    check(lib().kvq_set_append_chunk(ctx, chunk_tokens), "kvq_set_append_chunk")
 
 
 def kvq_set_splits(ctx: int, splits: int) -> None:

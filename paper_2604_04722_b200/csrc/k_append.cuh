@@ -24,7 +24,8 @@
 
 namespace kvq {
 
-constexpr int kChunkTokens = 256;      // tokens per slot-assignment chunk == threads per CTA
+constexpr int kChunkTokens = 256;      // threads per CTA of the chunked kernels; a chunk holds 256 * tpt tokens
+constexpr int kMaxTokensPerThread = 4; // (a thread takes tokens x, x + 256, ... of its chunk, so position order = pass order)
 #ifndef KVQ_APPEND_DEPTH
 #define KVQ_APPEND_DEPTH 2
 #endif
@@ -46,6 +47,7 @@ struct AppendParams {
     const uint32_t* counts_in;         // [batch][4] of this layer
     uint32_t* counts_out;              // [batch][4] of this layer
     int layer, n_new, pos0, nchunks, heads_per_group;
+    int tpt;                           // tokens per thread: a slot-assignment chunk is kChunkTokens * tpt tokens
     // Ragged batches: tokens each sequence adds in this call (nullptr: n_new for all; the input tensors keep
     // n_new rows per sequence) and position of each sequence's first new token (nullptr: pos0 for all).
     const int* lens;
@@ -72,27 +74,33 @@ k_classify(AppendParams p) {
     extern __shared__ float sW[];
     __shared__ uint32_t wtot[kChunkTokens / 32][4];
     const int chunk = blockIdx.x, b = blockIdx.y;
-    const int t = chunk * kChunkTokens + threadIdx.x;
-    const bool live = t < new_tokens_of(p, b);
-    int c = -1;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (FUSED) {
         controller_stage(sW, p.ctrl, p.hidden);
         __syncthreads();
-        if (live) {
-            float4 f = reinterpret_cast<const float4*>(p.feats)[(size_t)b * p.n_new + t];
-            float lg[4];
-            c = controller_decide_any(sW, p.hidden, f.x, f.y, f.z, f.w, lg);
-            if (p.bits_out) p.bits_out[(size_t)b * p.n_new + t] = (uint8_t)pool_bits(c);
-        }
-    } else if (live) {
-        c = class_of_bits(p.bits[(size_t)b * p.n_new + t], p.store.flags);
     }
-    if (live) p.cls[(size_t)b * p.n_new + t] = (uint8_t)c;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint32_t mine[4] = {0, 0, 0, 0};                   // lane 0: this warp's tokens per class over all passes
+    for (int r = 0; r < p.tpt; ++r) {
+        const int t = (chunk * p.tpt + r) * kChunkTokens + threadIdx.x;
+        const bool live = t < new_tokens_of(p, b);
+        int c = -1;
+        if (FUSED) {
+            if (live) {
+                float4 f = reinterpret_cast<const float4*>(p.feats)[(size_t)b * p.n_new + t];
+                float lg[4];
+                c = controller_decide_any(sW, p.hidden, f.x, f.y, f.z, f.w, lg);
+                if (p.bits_out) p.bits_out[(size_t)b * p.n_new + t] = (uint8_t)pool_bits(c);
+            }
+        } else if (live) {
+            c = class_of_bits(p.bits[(size_t)b * p.n_new + t], p.store.flags);
+        }
+        if (live) p.cls[(size_t)b * p.n_new + t] = (uint8_t)c;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        uint32_t m = __ballot_sync(0xffffffffu, c == k);
-        if (lane == 0) wtot[warp][k] = __popc(m);
+        for (int k = 0; k < 4; ++k) mine[k] += __popc(__ballot_sync(0xffffffffu, c == k));
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) wtot[warp][k] = mine[k];
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -268,37 +276,49 @@ k_reserve_blocks(AppendParams p) {
 
 // Launch 2.  MODE 0: classes come from k_classify (several chunks per sequence);
 // MODE 1: one chunk, classes from `bits`; MODE 2: one chunk, classes from the controller.
+// R: tokens per thread (= p.tpt): a chunk is 256 R tokens.  A 16-slot tile that a chunk only partly fills
+// costs as much as a full one, and every class has one at each end of a chunk, so long prefills take R = 4
+// (about 94 % of the slots a warp works on hold a token, against 81 % with R = 1).
 // grid = (nchunks, head_groups, batch), block = 256.
-template <int MODE, int G>
+template <int MODE, int G, int R = 1>
 __global__ void __launch_bounds__(kChunkTokens, KVQ_APPEND_MIN_CTAS)
 k_quant_pack(AppendParams p) {
+    static_assert(MODE == 0 || R == 1, "single-chunk appends hold at most 256 tokens per sequence");
+    constexpr int CT = kChunkTokens * R;               // tokens per chunk
     extern __shared__ __align__(16) uint8_t dyn_smem[];   // [ring: warps x depth x 4 KB][controller block (MODE 2)]
     uint8_t* ring_raw = dyn_smem;
     float* sW = reinterpret_cast<float*>(dyn_smem + kAppendRingBytes);
-    __shared__ uint32_t wtot[kChunkTokens / 32][4];
+    __shared__ uint32_t wtot[R][kChunkTokens / 32][4];
     __shared__ uint32_t base[4];
-    __shared__ uint8_t list[4][kChunkTokens];         // tokens of the chunk by class, in slot order
+    __shared__ uint16_t list[4][CT];                   // tokens of the chunk by class, in slot order
     const int chunk = blockIdx.x, hg = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tok_i = chunk * kChunkTokens + threadIdx.x;
-    const bool live = tok_i < new_tokens_of(p, b);
-    const size_t tok = (size_t)b * p.n_new + tok_i;
+    const int n_b = new_tokens_of(p, b);
 
-    // ---- class of this thread's token
-    int c = -1;
+    // ---- classes of this thread's tokens (pass r: token r * 256 + thread of the chunk)
+    int c[R];
     if (MODE == 2) {
         controller_stage(sW, p.ctrl, p.hidden);
         __syncthreads();
-        if (live) {
-            float4 f = reinterpret_cast<const float4*>(p.feats)[tok];
-            float lg[4];
-            c = controller_decide_any(sW, p.hidden, f.x, f.y, f.z, f.w, lg);
-            if (p.bits_out && hg == 0) p.bits_out[tok] = (uint8_t)pool_bits(c);
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int tok_i = chunk * CT + r * kChunkTokens + threadIdx.x;
+        const bool live = tok_i < n_b;
+        const size_t tok = (size_t)b * p.n_new + tok_i;
+        c[r] = -1;
+        if (MODE == 2) {
+            if (live) {
+                float4 f = reinterpret_cast<const float4*>(p.feats)[tok];
+                float lg[4];
+                c[r] = controller_decide_any(sW, p.hidden, f.x, f.y, f.z, f.w, lg);
+                if (p.bits_out && hg == 0) p.bits_out[tok] = (uint8_t)pool_bits(c[r]);
+            }
+        } else if (MODE == 1) {
+            if (live) c[r] = class_of_bits(p.bits[tok], p.store.flags);
+        } else {
+            if (live) c[r] = p.cls[tok];
         }
-    } else if (MODE == 1) {
-        if (live) c = class_of_bits(p.bits[tok], p.store.flags);
-    } else {
-        if (live) c = p.cls[tok];
     }
 
     // ---- fill of each pool before this chunk
@@ -322,27 +342,38 @@ k_quant_pack(AppendParams p) {
             base[0] = ci[0] + h.x; base[1] = ci[1] + h.y; base[2] = ci[2] + h.z; base[3] = ci[3] + h.w;
         }
     }
-    // ---- rank inside the chunk
-    uint32_t rank = 0;
+    // ---- rank inside the chunk: tokens of earlier passes, of earlier warps of the pass, of earlier lanes
+    uint32_t rank[R];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        uint32_t m = __ballot_sync(0xffffffffu, c == k);
-        if (c == k) rank = __popc(m & ((1u << lane) - 1u));
-        if (lane == 0) wtot[warp][k] = __popc(m);
+    for (int r = 0; r < R; ++r) {
+        rank[r] = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            uint32_t m = __ballot_sync(0xffffffffu, c[r] == k);
+            if (c[r] == k) rank[r] = __popc(m & ((1u << lane) - 1u));
+            if (lane == 0) wtot[r][warp][k] = __popc(m);
+        }
     }
     __syncthreads();
-    if (live) {
-        for (int w = 0; w < warp; ++w) rank += wtot[w][c];
-        list[c][rank] = (uint8_t)threadIdx.x;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        if (c[r] < 0) continue;
+        uint32_t before = rank[r];
+        for (int rr = 0; rr < r; ++rr)
+            for (int w = 0; w < kChunkTokens / 32; ++w) before += wtot[rr][w][c[r]];
+        for (int w = 0; w < warp; ++w) before += wtot[r][w][c[r]];
+        const int in_chunk = r * kChunkTokens + threadIdx.x;
+        list[c[r]][before] = (uint16_t)in_chunk;
         if (hg == 0)
-            p.store.index[((size_t)p.layer * p.store.batch + b) * p.store.max_ctx + first_pos_of(p, b) + tok_i] =
-                ((uint32_t)c << 30) | (base[c] + rank);
+            p.store.index[((size_t)p.layer * p.store.batch + b) * p.store.max_ctx + first_pos_of(p, b) + chunk * CT + in_chunk] =
+                ((uint32_t)c[r] << 30) | (base[c[r]] + before);
     }
     uint32_t ncls[4];                                  // tokens of each class in this chunk
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
         ncls[k] = 0;
-        for (int w = 0; w < kChunkTokens / 32; ++w) ncls[k] += wtot[w][k];
+        for (int r = 0; r < R; ++r)
+            for (int w = 0; w < kChunkTokens / 32; ++w) ncls[k] += wtot[r][w][k];
     }
     if (hg == 0 && chunk == p.nchunks - 1 && threadIdx.x < 4)
         p.counts_out[(size_t)b * 4 + threadIdx.x] = base[threadIdx.x] + ncls[threadIdx.x];
@@ -412,7 +443,7 @@ k_quant_pack(AppendParams p) {
             const uint32_t r_ld = r0 + (lane >> 1);                // the slot this lane copies a piece of
             if (r_ld < nk) {
                 const int i_tok = list[k][r_ld];
-                const size_t src = (((size_t)b * p.n_new + (size_t)chunk * kChunkTokens + i_tok) * p.store.kv_heads + h) *
+                const size_t src = (((size_t)b * p.n_new + (size_t)chunk * CT + i_tok) * p.store.kv_heads + h) *
                                    kHeadDim;
                 const int odd = lane & 1;
                 const uint4* ks = reinterpret_cast<const uint4*>(p.K + src) + odd;

@@ -46,6 +46,7 @@ struct kvq_ctx {
     float* unit_var = nullptr;           //                [units] variance of a unit's attention weights
     uint32_t* vis = nullptr;             // kvq_attend_last: visible pool fills [batch][query rows of a launch][4]
     int splits_override = 0;
+    int chunk_override = 0;              // kvq_set_append_chunk: 0 = automatic, else tokens per thread of a prefill chunk
     uint32_t* flags = nullptr;
     // device staging for the host-buffer entry points
     float* st_feats = nullptr;
@@ -91,6 +92,16 @@ cudaError_t dev_alloc(kvq_ctx* c, T** p, size_t bytes) {
 
 constexpr int kProfMaxCalls = 1024;
 
+#ifndef KVQ_APPEND_WAVES_SMALL
+#define KVQ_APPEND_WAVES_SMALL 2
+#endif
+#ifndef KVQ_APPEND_WAVES
+#define KVQ_APPEND_WAVES 24
+#endif
+#ifndef KVQ_APPEND_TOKENS_PER_THREAD
+#define KVQ_APPEND_TOKENS_PER_THREAD 2
+#endif
+static_assert(KVQ_APPEND_TOKENS_PER_THREAD >= 1 && KVQ_APPEND_TOKENS_PER_THREAD <= kMaxTokensPerThread, "chunk size");
 #ifndef KVQ_OVERLAP_LAUNCHES
 #define KVQ_OVERLAP_LAUNCHES 1
 #endif
@@ -218,9 +229,21 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
         p.lens = c->d_lens;
         p.pos = c->d_lens + c->batch;
     }
-    p.nchunks = (n_new + kChunkTokens - 1) / kChunkTokens;
+    // Long prefills use chunks of 1024 tokens (fewer partly filled tiles at chunk ends), as long as that still
+    // leaves several waves of CTAs once the KV heads are split into groups; everything else 256.
+    p.tpt = 1;
+    if (c->chunk_override) {
+        p.tpt = c->chunk_override;
+    } else if (KVQ_APPEND_TOKENS_PER_THREAD > 1) {
+        const long long big_chunks = (n_new + kChunkTokens * KVQ_APPEND_TOKENS_PER_THREAD - 1) / (kChunkTokens * KVQ_APPEND_TOKENS_PER_THREAD);
+        if (big_chunks * c->batch * c->kv_heads >= 12LL * c->sm_count * 2) p.tpt = KVQ_APPEND_TOKENS_PER_THREAD;
+    }
+    if (n_new <= kChunkTokens) p.tpt = 1;              // one CTA per (head group, sequence) does everything
+    const int chunk_tokens = kChunkTokens * p.tpt;
+    p.nchunks = (n_new + chunk_tokens - 1) / chunk_tokens;
     // enough CTAs to fill the device: split the KV heads into groups when chunks x batch is small
-    int want_groups = (2 * c->sm_count + p.nchunks * c->batch - 1) / (p.nchunks * c->batch);
+    const int waves = p.tpt > 1 ? KVQ_APPEND_WAVES : KVQ_APPEND_WAVES_SMALL;
+    int want_groups = (waves * c->sm_count + p.nchunks * c->batch - 1) / (p.nchunks * c->batch);
     int groups = want_groups < 1 ? 1 : (want_groups > c->kv_heads ? c->kv_heads : want_groups);
     p.heads_per_group = (c->kv_heads + groups - 1) / groups;
     groups = (c->kv_heads + p.heads_per_group - 1) / p.heads_per_group;
@@ -237,7 +260,7 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
             else launch_overlapped(k_append_token<false, 2>, grid_t, 32, 0, st, p);
         }
         c->launches += 1;
-    } else if (p.nchunks == 1) {
+    } else if (n_new <= kChunkTokens) {
         if (c->groups == 1) {
             if (fused) k_quant_pack<2, 1><<<grid_q, kChunkTokens, kAppendRingBytes + smem, st>>>(p);
             else k_quant_pack<1, 1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
@@ -251,8 +274,13 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
         if (fused) k_classify<true><<<grid_c, kChunkTokens, smem, st>>>(p);
         else k_classify<false><<<grid_c, kChunkTokens, 0, st>>>(p);
         k_reserve_blocks<<<c->batch, 128, 0, st>>>(p);
-        if (c->groups == 1) k_quant_pack<0, 1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
-        else k_quant_pack<0, 2><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+        if (p.tpt == 1) {
+            if (c->groups == 1) k_quant_pack<0, 1, 1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+            else k_quant_pack<0, 2, 1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+        } else {
+            if (c->groups == 1) k_quant_pack<0, 1, KVQ_APPEND_TOKENS_PER_THREAD><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+            else k_quant_pack<0, 2, KVQ_APPEND_TOKENS_PER_THREAD><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+        }
         c->launches += 3;
     }
     KVQ_CUDA(c, cudaGetLastError());
@@ -485,6 +513,8 @@ int kvq_create_grouped(kvq_ctx** out, int layers, int q_heads, int kv_heads, int
             return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
         };
         ok = ok && dyn_smem(k_quant_pack<0, 1>, ring) && dyn_smem(k_quant_pack<0, 2>, ring);
+        ok = ok && dyn_smem(k_quant_pack<0, 1, KVQ_APPEND_TOKENS_PER_THREAD>, ring) &&
+             dyn_smem(k_quant_pack<0, 2, KVQ_APPEND_TOKENS_PER_THREAD>, ring);
         ok = ok && dyn_smem(k_quant_pack<1, 1>, ring) && dyn_smem(k_quant_pack<1, 2>, ring);
         ok = ok && dyn_smem(k_quant_pack<2, 1>, ring + smem_max) && dyn_smem(k_quant_pack<2, 2>, ring + smem_max);
         ok = ok && dyn_smem(k_decode_attn<false, 1>, (int)kDecodeSmemBytes) && dyn_smem(k_decode_attn<false, 2>, (int)kDecodeSmemBytes);
@@ -750,6 +780,14 @@ int kvq_reset(kvq_ctx* c, void* stream) {
 int kvq_seq_len(kvq_ctx* c, int layer, int* host_len_out) {
     if (check_layer(c, layer) != KVQ_OK || !host_len_out) return KVQ_ERR_ARG;
     *host_len_out = c->len[layer];
+    return KVQ_OK;
+}
+
+int kvq_set_append_chunk(kvq_ctx* c, int chunk_tokens) {
+    if (!c) return KVQ_ERR_ARG;
+    if (chunk_tokens != 0 && chunk_tokens != kChunkTokens && chunk_tokens != kChunkTokens * KVQ_APPEND_TOKENS_PER_THREAD)
+        return KVQ_ERR_ARG;
+    c->chunk_override = chunk_tokens / kChunkTokens;
     return KVQ_OK;
 }
 
