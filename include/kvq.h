@@ -106,6 +106,21 @@ int kvq_create_grouped(kvq_ctx** out, int layers, int q_heads, int kv_heads, int
                        int max_ctx, int batch, uint64_t arena_bytes, int scale_groups);
 
 /*
+ * The same cache inside device memory that the caller owns (for instance one torch tensor), so that
+ * the library itself allocates no device memory for it.  kvq_workspace_bytes gives the size the other
+ * arguments need (host uint64; it reads the current device's properties, allocates nothing).
+ * kvq_create_in takes `workspace`, a dev pointer aligned to 256 bytes with at least that many bytes,
+ * carves every buffer of the handle out of it and zeroes what kvq_create zeroes.  The memory must stay
+ * valid until kvq_destroy, which leaves it alone.  KVQ_ERR_NOMEM if workspace_bytes is too small,
+ * KVQ_ERR_ARG for a NULL or misaligned workspace; otherwise as kvq_create_grouped.
+ */
+int kvq_workspace_bytes(int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
+                        uint64_t arena_bytes, int scale_groups, uint64_t* bytes_out);
+int kvq_create_in(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim,
+                  int max_ctx, int batch, uint64_t arena_bytes, int scale_groups,
+                  void* workspace, uint64_t workspace_bytes);
+
+/*
  * Arena fill: blocks handed out so far, blocks available, bytes per block (host uint64, any
  * may be NULL).  Synchronizes.
  */

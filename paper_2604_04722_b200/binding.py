@@ -34,6 +34,8 @@ SIGNATURES = {
     "kvq_create": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i]),
     "kvq_create_arena": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, C.c_uint64]),
     "kvq_create_grouped": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, C.c_uint64, _i]),
+    "kvq_workspace_bytes": (_i, [_i, _i, _i, _i, _i, _i, C.c_uint64, _i, C.POINTER(C.c_uint64)]),
+    "kvq_create_in": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, C.c_uint64, _i, _vp, C.c_uint64]),
     "kvq_arena_usage": (_i, [_vp, _u64p, _u64p, _u64p]),
     "kvq_destroy": (_i, [_vp]),
     "kvq_set_controller": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -135,6 +137,22 @@ def kvq_create_grouped(layers: int, q_heads: int, kv_heads: int, head_dim: int, 
     h = _vp()
     check(lib().kvq_create_grouped(C.byref(h), layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes,
                                    scale_groups), "kvq_create_grouped")
+    return h.value
+
+
+def kvq_workspace_bytes(layers: int, q_heads: int, kv_heads: int, head_dim: int, max_ctx: int, batch: int,
+                        arena_bytes: int = 0, scale_groups: int = 1) -> int:
+    n = C.c_uint64()
+    check(lib().kvq_workspace_bytes(layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes, scale_groups,
+                                    C.byref(n)), "kvq_workspace_bytes")
+    return n.value
+
+
+def kvq_create_in(layers: int, q_heads: int, kv_heads: int, head_dim: int, max_ctx: int, batch: int, arena_bytes: int,
+                  scale_groups: int, workspace, workspace_bytes: int) -> int:
+    h = _vp()
+    check(lib().kvq_create_in(C.byref(h), layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes, scale_groups,
+                              _ptr(workspace), workspace_bytes), "kvq_create_in")
     return h.value
 
 

@@ -57,6 +57,12 @@ struct kvq_ctx {
     std::vector<cudaEvent_t> prof_ev;    // 2 events per recorded call
     int prof_calls = 0;
     uint64_t device_bytes = 0, launches = 0;
+    // Where the device buffers come from: 0 = one cudaMalloc each; 1 = none, only their sizes are added up
+    // (kvq_workspace_bytes); 2 = carved out of the caller's workspace (kvq_create_in).
+    int mem_mode = 0;
+    uint8_t* slab = nullptr;
+    size_t slab_size = 0, slab_used = 0;
+    bool slab_short = false;             // the caller's workspace was too small
     cudaError_t last_err = cudaSuccess;
 };
 
@@ -85,6 +91,17 @@ struct DeviceGuard {                     // make the handle's device current for
 
 template <typename T>
 cudaError_t dev_alloc(kvq_ctx* c, T** p, size_t bytes) {
+    if (c->mem_mode != 0) {                          // 256-byte aligned pieces of one workspace
+        const size_t need = ((bytes ? bytes : 1) + 255) & ~(size_t)255;
+        if (c->mem_mode == 2 && c->slab_used + need > c->slab_size) {
+            c->slab_short = true;
+            return cudaErrorMemoryAllocation;
+        }
+        *p = c->mem_mode == 2 ? reinterpret_cast<T*>(c->slab + c->slab_used) : nullptr;
+        c->slab_used += need;
+        c->device_bytes += bytes;
+        return cudaSuccess;
+    }
     cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), bytes ? bytes : 1);
     if (e == cudaSuccess) c->device_bytes += bytes;
     return e;
@@ -129,6 +146,7 @@ void launch_overlapped(void (*kernel)(Params), dim3 grid, unsigned block, size_t
 void free_all(kvq_ctx* c) {
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     c->prof_ev.clear();
+    if (c->mem_mode != 0) return;                      // the buffers belong to the caller's workspace (or do not exist)
     cudaFree(c->arena);
     cudaFree(c->table);
     cudaFree(c->arena_used);
@@ -400,6 +418,10 @@ int export_impl(kvq_ctx* c, int layer, int b0, int nb, int pos0, int n, uint8_t*
     return KVQ_OK;
 }
 
+int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
+                uint64_t arena_bytes, int scale_groups, int mem_mode, void* workspace, uint64_t workspace_bytes,
+                uint64_t* bytes_out);
+
 }  // namespace
 
 extern "C" {
@@ -415,6 +437,31 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
 
 int kvq_create_grouped(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
                        uint64_t arena_bytes, int scale_groups) {
+    return create_impl(out, layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes, scale_groups, 0, nullptr, 0, nullptr);
+}
+
+int kvq_workspace_bytes(int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch, uint64_t arena_bytes,
+                        int scale_groups, uint64_t* bytes_out) {
+    if (!bytes_out) return KVQ_ERR_ARG;
+    kvq_ctx* none = nullptr;
+    return create_impl(&none, layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes, scale_groups, 1, nullptr, 0,
+                       bytes_out);
+}
+
+int kvq_create_in(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
+                  uint64_t arena_bytes, int scale_groups, void* workspace, uint64_t workspace_bytes) {
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return KVQ_ERR_ARG;
+    return create_impl(out, layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes, scale_groups, 2, workspace,
+                       workspace_bytes, nullptr);
+}
+
+}  // extern "C"
+
+namespace {
+
+int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
+                uint64_t arena_bytes, int scale_groups, int mem_mode, void* workspace, uint64_t workspace_bytes,
+                uint64_t* bytes_out) {
     if (!out) return KVQ_ERR_ARG;
     *out = nullptr;
     if (scale_groups != 1 && scale_groups != 2) return KVQ_ERR_ARG;
@@ -435,6 +482,9 @@ int kvq_create_grouped(kvq_ctx** out, int layers, int q_heads, int kv_heads, int
     c->max_ctx = max_ctx;
     c->batch = batch;
     c->groups = scale_groups;
+    c->mem_mode = mem_mode;
+    c->slab = static_cast<uint8_t*>(workspace);
+    c->slab_size = (size_t)workspace_bytes;
     c->len.assign(layers, 0);
     c->lens.assign((size_t)layers * batch, 0);
     c->ragged.assign(layers, 0);
@@ -492,6 +542,11 @@ int kvq_create_grouped(kvq_ctx** out, int layers, int q_heads, int kv_heads, int
     ok = ok && dev_alloc(c, &c->st_O, sizeof(__half) * units * kHeadDim) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_bits, (size_t)batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_export, (size_t)kv_heads * (2 * KVQ_EXPORT_ROW_BYTES + 8 * scale_groups) + 16) == cudaSuccess;
+    if (ok && mem_mode == 1) {                         // only the size was asked for
+        *bytes_out = c->slab_used;
+        delete c;
+        return KVQ_OK;
+    }
     if (ok) {
         s.arena = c->arena;
         s.table = c->table;
@@ -523,13 +578,18 @@ int kvq_create_grouped(kvq_ctx** out, int layers, int q_heads, int kv_heads, int
     }
     if (!ok) {
         cudaError_t err = cudaGetLastError();
+        const bool too_small = c->slab_short;
         free_all(c);
         delete c;
-        return err == cudaErrorMemoryAllocation ? KVQ_ERR_NOMEM : KVQ_ERR_CUDA;
+        return err == cudaErrorMemoryAllocation || too_small ? KVQ_ERR_NOMEM : KVQ_ERR_CUDA;
     }
     *out = c;
     return KVQ_OK;
 }
+
+}  // namespace
+
+extern "C" {
 
 int kvq_destroy(kvq_ctx* c) {
     if (!c) return KVQ_OK;
