@@ -19,6 +19,13 @@
 #include "k_export.cuh"
 #include "k_features.cuh"
 
+#ifndef KVQ_NVTX
+#define KVQ_NVTX 1                       // NVTX ranges around the entry points that launch the hot kernels
+#endif
+#if KVQ_NVTX
+#include <nvtx3/nvToolsExt.h>
+#endif
+
 using namespace kvq;
 
 struct kvq_ctx {
@@ -67,6 +74,15 @@ struct kvq_ctx {
 };
 
 namespace {
+
+struct TraceRange {                      // a named range for timeline tools; costs nothing when none is attached
+#if KVQ_NVTX
+    explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+    ~TraceRange() { nvtxRangePop(); }
+#else
+    explicit TraceRange(const char*) {}
+#endif
+};
 
 struct DeviceGuard {                     // make the handle's device current for the duration of a call
     int prev = -1;
@@ -198,6 +214,7 @@ size_t controller_smem(int hidden) { return sizeof(float) * (size_t)controller_f
 // int [batch], each 0..n_new) or nullptr for n_new everywhere.
 int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8_t* bits, const float* feats,
                 uint8_t* bits_out, int n_new, const int* host_lens, cudaStream_t st) {
+    TraceRange trace(feats ? "kvq_append (controller inside)" : "kvq_append");
     if (check_layer(c, layer) != KVQ_OK || n_new < 0) return KVQ_ERR_ARG;
     if (n_new == 0) return KVQ_OK;
     int* cur_lens = &c->lens[(size_t)layer * c->batch];
@@ -656,6 +673,7 @@ int kvq_seq_lens(kvq_ctx* c, int layer, int* host_lens_out) {
 }
 
 int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream) {
+    TraceRange trace("kvq_decode_attn");
     if (check_layer(c, layer) != KVQ_OK || !Q || !O) return KVQ_ERR_ARG;
     if (c->len[layer] == 0) return KVQ_ERR_EMPTY;
     DeviceGuard guard(c->device);
@@ -787,6 +805,7 @@ int kvq_decode_attn_static(kvq_ctx* c, int layer, const void* Q, void* O, void* 
 
 int kvq_decode_step_host(kvq_ctx* c, int layer, const float* feats, const void* K, const void* V, const void* Q,
                          void* O, uint8_t* bits_out_opt, void* stream) {
+    TraceRange trace("kvq_decode_step_host");
     if (check_layer(c, layer) != KVQ_OK || !feats || !K || !V || !Q || !O) return KVQ_ERR_ARG;
     if (c->hidden == 0) return KVQ_ERR_NO_CONTROLLER;
     if (c->len[layer] + 1 > c->max_ctx) return KVQ_ERR_CAPACITY;

@@ -364,3 +364,32 @@ def test_attend_last_is_causal_attention_at_each_of_the_last_positions(gu, oracl
         # the last row is the ordinary decode step
         gu.assert_attention_close(g.decode(0, np.ascontiguousarray(Q[:, T - 1])), want[:, T - 1], "last row")
         assert kq.lib().kvq_attend_last(g.ctx, 0, Qd.data_ptr(), O.data_ptr(), n + 1, None) == kq.KVQ_ERR_ARG
+
+
+# ------------------------------------------------------------------ determinism
+
+def test_two_runs_give_the_same_bits(gu):
+    """The same appends and the same query twice, on two handles: packed rows, scales and the attention output
+    are bitwise equal (slots come from a scan, not from atomics; partial results are merged in record order
+    whichever warp arrives last)."""
+    from paper_2604_04722_b200 import binding as kq
+    rng = np.random.default_rng(123)
+    B, Hq, H, n = 2, 8, 4, 3000
+    K, V = _kv(rng, B, n, H)
+    bits = BITS[rng.choice(4, size=(B, n), p=[.4, .3, .2, .1])]
+    Q = rng.standard_normal((B, Hq, 64)).astype(np.float16)
+    runs = []
+    for _ in range(2):
+        with gu.GpuCache(1, B, Hq, H, n) as g:
+            g.append(0, K[:, :2000], V[:, :2000], bits[:, :2000])
+            g.append(0, K[:, 2000:], V[:, 2000:], bits[:, 2000:])
+            outs = []
+            for splits in (0, 7):
+                kq.kvq_set_splits(g.ctx, splits)
+                outs += [g.decode(0, Q), g.decode(0, Q)]
+            runs.append((g.export(0, 0, n), outs))
+    for a, b in zip(runs[0][0], runs[1][0]):
+        assert np.array_equal(a, b)
+    for a, b in zip(runs[0][1], runs[1][1]):
+        assert np.array_equal(a, b)
+    assert np.array_equal(runs[0][1][0], runs[0][1][1]) and np.array_equal(runs[0][1][2], runs[0][1][3])
