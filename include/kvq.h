@@ -335,6 +335,20 @@ int kvq_export_token(kvq_ctx* ctx, int layer, int b, int pos,
                      void* k_codes, void* v_codes, uint16_t* k_meta, uint16_t* v_meta);
 
 /*
+ * Snapshot of the cache (every layer): the packed rows in use, block tables, per-token index, pool
+ * fills and sequence lengths, as one host blob that kvq_load_state puts back, into this handle or into
+ * another one created with the same shape arguments and scale_groups (its arena may have a different
+ * budget as long as the snapshot's blocks fit).  The controller weights are not part of it.
+ * kvq_state_bytes: size of a snapshot taken now (host uint64).  kvq_save_state: host_buf (host memory,
+ * host_bytes >= that size) receives it.  kvq_load_state: replaces the handle's contents; KVQ_ERR_ARG
+ * if the blob is truncated, was not written by kvq_save_state or belongs to another shape.  All three
+ * synchronize the device.
+ */
+int kvq_state_bytes(kvq_ctx* ctx, uint64_t* bytes_out);
+int kvq_save_state(kvq_ctx* ctx, void* host_buf, uint64_t host_bytes);
+int kvq_load_state(kvq_ctx* ctx, const void* host_buf, uint64_t host_bytes);
+
+/*
  * Pool fill of `layer`: host_counts (host uint32 [batch][4], may be NULL)
  * receives tokens per precision class; resident_bytes (host, may be NULL) the
  * bytes of packed rows in use, sum over tokens of kv_heads * {40,72,136,256};

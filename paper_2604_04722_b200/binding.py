@@ -53,6 +53,9 @@ SIGNATURES = {
     "kvq_reset": (_i, [_vp, _vp]),
     "kvq_seq_len": (_i, [_vp, _i, C.POINTER(_i)]),
     "kvq_set_splits": (_i, [_vp, _i]),
+    "kvq_state_bytes": (_i, [_vp, C.POINTER(C.c_uint64)]),
+    "kvq_save_state": (_i, [_vp, _vp, C.c_uint64]),
+    "kvq_load_state": (_i, [_vp, _vp, C.c_uint64]),
     "kvq_set_append_chunk": (_i, [_vp, _i]),
     "kvq_export_range": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvq_export_token": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -238,6 +241,20 @@ def kvq_seq_len(ctx: int, layer: int) -> int:
     n = _i()
     check(lib().kvq_seq_len(ctx, layer, C.byref(n)), "kvq_seq_len")
     return n.value
+
+
+def kvq_save_state(ctx: int):
+    """Returns the snapshot as a numpy uint8 array."""
+    import numpy as np
+    n = C.c_uint64()
+    check(lib().kvq_state_bytes(ctx, C.byref(n)), "kvq_state_bytes")
+    blob = np.empty(n.value, np.uint8)
+    check(lib().kvq_save_state(ctx, blob.ctypes.data, n.value), "kvq_save_state")
+    return blob
+
+
+def kvq_load_state(ctx: int, blob) -> None:
+    check(lib().kvq_load_state(ctx, blob.ctypes.data, blob.size), "kvq_load_state")
 
 
 def kvq_set_append_chunk(ctx: int, chunk_tokens: int) -> None:

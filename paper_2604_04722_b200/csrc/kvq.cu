@@ -70,6 +70,7 @@ struct kvq_ctx {
     uint8_t* slab = nullptr;
     size_t slab_size = 0, slab_used = 0;
     bool slab_short = false;             // the caller's workspace was too small
+    size_t table_bytes = 0;              // size of `table`
     cudaError_t last_err = cudaSuccess;
 };
 
@@ -534,6 +535,7 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
     s.arena_blocks = (uint32_t)blocks;
     const size_t total = (size_t)blocks * kBlockBytes;
     const size_t table_bytes = sizeof(uint32_t) * (streams * row + 1);
+    c->table_bytes = table_bytes;
     const size_t max_chunks = (size_t)(max_ctx + kChunkTokens - 1) / kChunkTokens;
     const size_t units = (size_t)batch * q_heads;
     bool ok = dev_alloc(c, &c->arena, total) == cudaSuccess;
@@ -943,6 +945,123 @@ int kvq_arena_usage(kvq_ctx* c, uint64_t* blocks_in_use, uint64_t* blocks_total,
     if (blocks_in_use) *blocks_in_use = used < total ? used : total;
     if (blocks_total) *blocks_total = total;
     if (block_bytes) *block_bytes = kBlockBytes;
+    return KVQ_OK;
+}
+
+// ---- snapshots: [StateHeader][len][lens][ragged][cur][arena blocks 0 .. used][table][index][counts]
+namespace {
+struct StateHeader {
+    uint32_t magic, version;
+    int32_t layers, q_heads, kv_heads, max_ctx, batch, groups;
+    uint32_t arena_blocks, blocks_used;
+    uint64_t table_bytes, index_bytes, counts_bytes, total_bytes;
+};
+constexpr uint32_t kStateMagic = 0x5156564bu, kStateVersion = 1;   // "KVVQ"
+
+int state_header(kvq_ctx* c, StateHeader& h) {
+    uint32_t used = 0;
+    KVQ_CUDA(c, cudaDeviceSynchronize());
+    KVQ_CUDA(c, cudaMemcpy(&used, c->arena_used, sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    if (used > c->store.arena_blocks - 1) used = c->store.arena_blocks - 1;       // an exhausted arena counts past its end
+    h = StateHeader{};
+    h.magic = kStateMagic;
+    h.version = kStateVersion;
+    h.layers = c->layers;
+    h.q_heads = c->q_heads;
+    h.kv_heads = c->kv_heads;
+    h.max_ctx = c->max_ctx;
+    h.batch = c->batch;
+    h.groups = c->groups;
+    h.arena_blocks = c->store.arena_blocks;
+    h.blocks_used = used;
+    h.table_bytes = c->table_bytes;
+    h.index_bytes = sizeof(uint32_t) * (uint64_t)c->layers * c->batch * c->max_ctx;
+    h.counts_bytes = sizeof(uint32_t) * 2 * (uint64_t)c->layers * c->batch * 4;
+    const uint64_t host_ints = (uint64_t)c->layers * 3 + (uint64_t)c->layers * c->batch;
+    h.total_bytes = sizeof(StateHeader) + sizeof(int32_t) * host_ints + (uint64_t)(used + 1) * kBlockBytes + h.table_bytes +
+                    h.index_bytes + h.counts_bytes;
+    return KVQ_OK;
+}
+}  // namespace
+
+int kvq_state_bytes(kvq_ctx* c, uint64_t* bytes_out) {
+    if (!c || !bytes_out) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    StateHeader h;
+    const int rc = state_header(c, h);
+    if (rc == KVQ_OK) *bytes_out = h.total_bytes;
+    return rc;
+}
+
+int kvq_save_state(kvq_ctx* c, void* host_buf, uint64_t host_bytes) {
+    if (!c || !host_buf) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    StateHeader h;
+    int rc = state_header(c, h);
+    if (rc != KVQ_OK) return rc;
+    if (host_bytes < h.total_bytes) return KVQ_ERR_ARG;
+    uint8_t* out = static_cast<uint8_t*>(host_buf);
+    std::memcpy(out, &h, sizeof(h));
+    out += sizeof(h);
+    auto put_ints = [&](auto&& get, size_t n) {
+        for (size_t i = 0; i < n; ++i) {
+            const int32_t v = (int32_t)get(i);
+            std::memcpy(out, &v, sizeof(v));
+            out += sizeof(v);
+        }
+    };
+    put_ints([&](size_t i) { return c->len[i]; }, c->len.size());
+    put_ints([&](size_t i) { return c->lens[i]; }, c->lens.size());
+    put_ints([&](size_t i) { return (int)c->ragged[i]; }, c->ragged.size());
+    put_ints([&](size_t i) { return c->cur[i]; }, c->cur.size());
+    const size_t arena_bytes = (size_t)(h.blocks_used + 1) * kBlockBytes;
+    KVQ_CUDA(c, cudaMemcpy(out, c->arena, arena_bytes, cudaMemcpyDeviceToHost));
+    out += arena_bytes;
+    KVQ_CUDA(c, cudaMemcpy(out, c->table, h.table_bytes, cudaMemcpyDeviceToHost));
+    out += h.table_bytes;
+    KVQ_CUDA(c, cudaMemcpy(out, c->store.index, h.index_bytes, cudaMemcpyDeviceToHost));
+    out += h.index_bytes;
+    KVQ_CUDA(c, cudaMemcpy(out, c->counts, h.counts_bytes, cudaMemcpyDeviceToHost));
+    return KVQ_OK;
+}
+
+int kvq_load_state(kvq_ctx* c, const void* host_buf, uint64_t host_bytes) {
+    if (!c || !host_buf || host_bytes < sizeof(StateHeader)) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    StateHeader h;
+    std::memcpy(&h, host_buf, sizeof(h));
+    if (h.magic != kStateMagic || h.version != kStateVersion || host_bytes < h.total_bytes) return KVQ_ERR_ARG;
+    if (h.layers != c->layers || h.q_heads != c->q_heads || h.kv_heads != c->kv_heads || h.max_ctx != c->max_ctx ||
+        h.batch != c->batch || h.groups != c->groups)
+        return KVQ_ERR_ARG;
+    // the arena may differ in size as long as the snapshot's blocks fit (block ids are positions in the arena)
+    if (h.blocks_used + 1 > c->store.arena_blocks || h.table_bytes != c->table_bytes) return KVQ_ERR_ARG;
+    const uint64_t host_ints = (uint64_t)c->layers * 3 + (uint64_t)c->layers * c->batch;
+    if (h.total_bytes != sizeof(StateHeader) + sizeof(int32_t) * host_ints + (uint64_t)(h.blocks_used + 1) * kBlockBytes +
+                             h.table_bytes + h.index_bytes + h.counts_bytes)
+        return KVQ_ERR_ARG;
+    const uint8_t* in = static_cast<const uint8_t*>(host_buf) + sizeof(h);
+    auto get_int = [&]() {
+        int32_t v;
+        std::memcpy(&v, in, sizeof(v));
+        in += sizeof(v);
+        return v;
+    };
+    KVQ_CUDA(c, cudaDeviceSynchronize());
+    for (auto& v : c->len) v = get_int();
+    for (auto& v : c->lens) v = get_int();
+    for (auto& v : c->ragged) v = (char)get_int();
+    for (auto& v : c->cur) v = get_int() & 1;
+    const size_t arena_bytes = (size_t)(h.blocks_used + 1) * kBlockBytes;
+    KVQ_CUDA(c, cudaMemcpy(c->arena, in, arena_bytes, cudaMemcpyHostToDevice));
+    in += arena_bytes;
+    KVQ_CUDA(c, cudaMemcpy(c->table, in, h.table_bytes, cudaMemcpyHostToDevice));
+    in += h.table_bytes;
+    KVQ_CUDA(c, cudaMemcpy(c->store.index, in, h.index_bytes, cudaMemcpyHostToDevice));
+    in += h.index_bytes;
+    KVQ_CUDA(c, cudaMemcpy(c->counts, in, h.counts_bytes, cudaMemcpyHostToDevice));
+    KVQ_CUDA(c, cudaMemcpy(c->arena_used, &h.blocks_used, sizeof(uint32_t), cudaMemcpyHostToDevice));
+    KVQ_CUDA(c, cudaMemset(c->flags, 0, sizeof(uint32_t)));
     return KVQ_OK;
 }
 

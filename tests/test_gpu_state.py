@@ -1,0 +1,93 @@
+"""Snapshots: kvq_save_state / kvq_load_state.  A cache restored from a snapshot, into the same handle or a fresh
+one, continues exactly like the one the snapshot was taken from."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+BITS = np.array([2, 4, 8, 16], np.uint8)
+
+
+@pytest.fixture(scope="module")
+def gu():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_04722_b200 import build
+    build.build()
+    import gpu_util
+    return gpu_util
+
+
+def _kv(rng, B, n, H):
+    K = (rng.standard_normal((B, n, H, 64)) * 2).astype(np.float16)
+    V = rng.standard_normal((B, n, H, 64)).astype(np.float16)
+    return K, V
+
+
+@pytest.mark.parametrize("groups", [1, 2])
+def test_restore_and_continue(gu, oracle, groups):
+    from paper_2604_04722_b200 import binding as kq
+    rng = np.random.default_rng(40 + groups)
+    L, B, Hq, H = 2, 3, 4, 2
+    lens = [500, 123, 0]
+    oc = [oracle.OracleCache(1, Hq, H) if groups == 1 else oracle.GroupedOracleCache(1, Hq, H, 2) for _ in range(B)]
+
+    def add(g, K, V, bits, ls=None):
+        if ls is None:
+            g.append(1, K, V, bits)
+        else:
+            kq.kvq_append_ragged(g.ctx, 1, gu.dev(K.view(np.uint16)), gu.dev(V.view(np.uint16)), gu.dev(bits), None, K.shape[1], ls)
+
+    K0, V0 = _kv(rng, B, 500, H)
+    b0 = BITS[rng.choice(4, size=(B, 500), p=[.4, .3, .2, .1])]
+    later = []
+    for n in (1, 40, 1):
+        K, V = _kv(rng, B, n, H)
+        later.append((K, V, BITS[rng.choice(4, size=(B, n))]))
+    Q = rng.standard_normal((B, Hq, 64)).astype(np.float16)
+
+    with gu.GpuCache(L, B, Hq, H, 600, scale_groups=groups) as g:
+        add(g, K0, V0, b0, lens)
+        blob = kq.kvq_save_state(g.ctx)
+        assert blob.size < 3 * 2 ** 20                  # rows in use, not the worst-case arena
+        for K, V, bits in later:
+            add(g, K, V, bits)
+        want_out = g.decode(1, Q)
+        want_store = g.export(1, 0, 42)                 # every sequence holds at least 42 tokens now
+        # back to the snapshot in the same handle
+        kq.kvq_load_state(g.ctx, blob)
+        assert kq.kvq_seq_lens(g.ctx, 1, B).tolist() == lens and kq.kvq_seq_len(g.ctx, 0) == 0
+        for K, V, bits in later:
+            add(g, K, V, bits)
+        assert np.array_equal(g.decode(1, Q), want_out)
+    # and in a fresh handle with a smaller arena
+    with gu.GpuCache(L, B, Hq, H, 600, scale_groups=groups, arena_bytes=64 * 65536) as g2:
+        kq.kvq_load_state(g2.ctx, blob)
+        for K, V, bits in later:
+            add(g2, K, V, bits)
+        assert np.array_equal(g2.decode(1, Q), want_out)
+        for a, b in zip(g2.export(1, 0, 42), want_store):
+            assert np.array_equal(a, b)
+        # against the oracle as well
+        for b in range(B):
+            if lens[b]:
+                oc[b].append(K0[b:b + 1, :lens[b]], V0[b:b + 1, :lens[b]], b0[b:b + 1, :lens[b]])
+            for K, V, bits in later:
+                oc[b].append(K[b:b + 1], V[b:b + 1], bits[b:b + 1])
+            gu.assert_attention_close(want_out[b:b + 1], oc[b].decode_attn(Q[b:b + 1]), "sequence %d" % b)
+
+
+def test_snapshots_of_other_shapes_are_refused(gu):
+    from paper_2604_04722_b200 import binding as kq
+    with gu.GpuCache(1, 1, 2, 2, 32) as a, gu.GpuCache(1, 1, 2, 1, 32) as b, gu.GpuCache(1, 1, 2, 2, 32, scale_groups=2) as c:
+        blob = kq.kvq_save_state(a.ctx)
+        L = kq.lib()
+        assert L.kvq_load_state(b.ctx, blob.ctypes.data, blob.size) == kq.KVQ_ERR_ARG
+        assert L.kvq_load_state(c.ctx, blob.ctypes.data, blob.size) == kq.KVQ_ERR_ARG
+        assert L.kvq_load_state(a.ctx, blob.ctypes.data, blob.size - 1) == kq.KVQ_ERR_ARG
+        bad = blob.copy()
+        bad[0] ^= 0xff
+        assert L.kvq_load_state(a.ctx, bad.ctypes.data, bad.size) == kq.KVQ_ERR_ARG
+        assert L.kvq_save_state(a.ctx, blob.ctypes.data, blob.size - 1) == kq.KVQ_ERR_ARG
+        kq.kvq_load_state(a.ctx, blob)
