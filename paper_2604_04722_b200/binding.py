@@ -243,13 +243,17 @@ def kvq_seq_len(ctx: int, layer: int) -> int:
     return n.value
 
 
+def kvq_state_bytes(ctx: int) -> int:
+    n = C.c_uint64()
+    check(lib().kvq_state_bytes(ctx, C.byref(n)), "kvq_state_bytes")
+    return n.value
+
+
 def kvq_save_state(ctx: int):
     """Returns the snapshot as a numpy uint8 array."""
     import numpy as np
-    n = C.c_uint64()
-    check(lib().kvq_state_bytes(ctx, C.byref(n)), "kvq_state_bytes")
-    blob = np.empty(n.value, np.uint8)
-    check(lib().kvq_save_state(ctx, blob.ctypes.data, n.value), "kvq_save_state")
+    blob = np.empty(kvq_state_bytes(ctx), np.uint8)
+    check(lib().kvq_save_state(ctx, blob.ctypes.data, blob.size), "kvq_save_state")
     return blob
 
 
