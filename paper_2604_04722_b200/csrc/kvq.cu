@@ -1047,6 +1047,53 @@ int kvq_load_state(kvq_ctx* c, const void* host_buf, uint64_t host_bytes) {
         in += sizeof(v);
         return v;
     };
+    // Nothing the kernels use as an address may point outside the handle's buffers: check lengths, fills,
+    // block ids and index words on the host before anything is replaced.
+    {
+        const uint8_t* q = in;
+        auto peek = [&]() {
+            int32_t v;
+            std::memcpy(&v, q, sizeof(v));
+            q += sizeof(v);
+            return v;
+        };
+        std::vector<int32_t> len(c->layers), lens((size_t)c->layers * c->batch), cur(c->layers);
+        for (auto& v : len) v = peek();
+        for (auto& v : lens) v = peek();
+        for (int l = 0; l < c->layers; ++l) peek();    // ragged flags
+        for (auto& v : cur) v = peek() & 1;
+        for (int l = 0; l < c->layers; ++l) {
+            int longest = 0;
+            for (int b = 0; b < c->batch; ++b) {
+                const int n = lens[(size_t)l * c->batch + b];
+                if (n < 0 || n > c->max_ctx) return KVQ_ERR_ARG;
+                longest = n > longest ? n : longest;
+            }
+            if (len[l] != longest) return KVQ_ERR_ARG;
+        }
+        const uint8_t* arena_blob = q;
+        const uint32_t* table = reinterpret_cast<const uint32_t*>(arena_blob + (size_t)(h.blocks_used + 1) * kBlockBytes);
+        for (size_t i = 0; i < h.table_bytes / sizeof(uint32_t); ++i) {
+            uint32_t id;
+            std::memcpy(&id, table + i, sizeof(id));
+            if (id > h.blocks_used) return KVQ_ERR_ARG;
+        }
+        const uint8_t* index = reinterpret_cast<const uint8_t*>(table) + h.table_bytes;
+        for (size_t i = 0; i < h.index_bytes / sizeof(uint32_t); ++i) {
+            uint32_t w;
+            std::memcpy(&w, index + i * sizeof(uint32_t), sizeof(w));
+            if ((w & 0x3fffffffu) >= (uint32_t)c->max_ctx) return KVQ_ERR_ARG;
+        }
+        const uint8_t* counts = index + h.index_bytes;
+        for (int which = 0; which < 2; ++which)
+            for (int l = 0; l < c->layers; ++l)
+                for (int b = 0; b < c->batch; ++b) {
+                    uint32_t f[4];
+                    std::memcpy(f, counts + sizeof(uint32_t) * 4 * (((size_t)which * c->layers + l) * c->batch + b), sizeof(f));
+                    const uint64_t sum = (uint64_t)f[0] + f[1] + f[2] + f[3];
+                    if (which == cur[l] ? sum != (uint64_t)lens[(size_t)l * c->batch + b] : sum > (uint64_t)c->max_ctx) return KVQ_ERR_ARG;
+                }
+    }
     KVQ_CUDA(c, cudaDeviceSynchronize());
     for (auto& v : c->len) v = get_int();
     for (auto& v : c->lens) v = get_int();

@@ -91,3 +91,36 @@ def test_snapshots_of_other_shapes_are_refused(gu):
         assert L.kvq_load_state(a.ctx, bad.ctypes.data, bad.size) == kq.KVQ_ERR_ARG
         assert L.kvq_save_state(a.ctx, blob.ctypes.data, blob.size - 1) == kq.KVQ_ERR_ARG
         kq.kvq_load_state(a.ctx, blob)
+
+
+def test_a_snapshot_that_points_outside_the_cache_is_refused(gu):
+    """Block ids, index words, fills and lengths of a blob are checked on the host before anything is loaded."""
+    import struct
+    from paper_2604_04722_b200 import binding as kq
+    rng = np.random.default_rng(2)
+    B, Hq, H, n = 1, 2, 2, 40
+    with gu.GpuCache(1, B, Hq, H, 64) as g:
+        K, V = _kv(rng, B, n, H)
+        g.append(0, K, V, BITS[rng.choice(4, size=(B, n))])
+        blob = kq.kvq_save_state(g.ctx)
+        head = struct.calcsize("<II6iII4Q")
+        used = struct.unpack_from("<I", blob, 4 * 9)[0]
+        table_bytes, index_bytes, counts_bytes, total = struct.unpack_from("<4Q", blob, head - 32)
+        assert total == blob.size
+        ints = 1 * 3 + 1 * B
+        table_at = head + 4 * ints + (used + 1) * 65536
+        index_at = table_at + table_bytes
+        counts_at = index_at + index_bytes
+        L = kq.lib()
+
+        def refused(at, value):
+            bad = blob.copy()
+            bad[at:at + 4] = np.frombuffer(struct.pack("<I", value), np.uint8)
+            return L.kvq_load_state(g.ctx, bad.ctypes.data, bad.size) == kq.KVQ_ERR_ARG
+
+        assert refused(table_at, used + 1)              # a block that was never handed out
+        assert refused(index_at, (1 << 30) | 64)        # a slot beyond max_ctx
+        assert refused(counts_at, 1000)                 # a pool fill that does not add up
+        assert refused(head + 4, 65)                    # a sequence longer than max_ctx
+        assert refused(head, 39)                        # longest length out of step with the lengths
+        kq.kvq_load_state(g.ctx, blob)                  # the untouched blob still loads
