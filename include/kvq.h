@@ -214,7 +214,8 @@ int kvq_decode_attn_var(kvq_ctx* ctx, int layer, const void* Q, void* O, float* 
  *   H_t         entropy of Softmax(z_t), natural logarithm (Eq. 14)
  *   C_t         confidence; the paper names it without a definition: max_v Softmax(z_t)_v
  *   token_ids   dev int32 [n], counts dev uint32 [vocab], total_count = N, observed_tokens =
- *               |V_obs|: R_t = -log((counts[token] + 1) / (N + |V_obs| + 1)) (Eq. 15)
+ *               |V_obs|: R_t = -log((counts[token] + 1) / (N + |V_obs| + 1)) (Eq. 15); a token id outside
+ *               [0, vocab) is taken as never seen (count 0)
  *   attn_var_opt dev fp32 [n] or NULL (then V_t = 0): the attention variance of Eq. 16, e.g. from
  *               kvq_decode_attn_var
  *   feats       dev fp32 [n][4] in the order H, R, V, C of Eq. 17 (16-byte aligned)

@@ -124,7 +124,8 @@ k_token_features(const T* __restrict__ logits, int vocab, bool vec, const int32_
         if (threadIdx.x != 0) return;
         const float H = logf(tot.s) - tot.w / tot.s;
         const float C = 1.0f / tot.s;
-        const float cnt = (float)counts[token_ids[tok]] + 1.0f;
+        const int32_t id = token_ids[tok];             // an id outside the table counts as never seen
+        const float cnt = ((uint32_t)id < (uint32_t)vocab ? (float)counts[id] : 0.0f) + 1.0f;
         const float R = -logf(cnt / rarity_denominator);
         reinterpret_cast<float4*>(feats)[tok] = make_float4(H, R, attn_var ? attn_var[tok] : 0.f, C);
     }

@@ -469,6 +469,12 @@ int kvq_workspace_bytes(int layers, int q_heads, int kv_heads, int head_dim, int
 int kvq_create_in(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
                   uint64_t arena_bytes, int scale_groups, void* workspace, uint64_t workspace_bytes) {
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return KVQ_ERR_ARG;
+    cudaPointerAttributes attr;                        // it has to be memory of a device, not of the host
+    if (cudaPointerGetAttributes(&attr, workspace) != cudaSuccess) {
+        cudaGetLastError();
+        return KVQ_ERR_ARG;
+    }
+    if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged) return KVQ_ERR_ARG;
     return create_impl(out, layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes, scale_groups, 2, workspace,
                        workspace_bytes, nullptr);
 }

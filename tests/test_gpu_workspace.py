@@ -35,7 +35,12 @@ def test_cache_in_a_caller_owned_workspace(gu, oracle, groups, arena_blocks):
     assert ws.data_ptr() % 256 == 0
     with pytest.raises(kq.KvqError):                   # one byte short
         kq.kvq_create_in(*shape, arena_blocks * 65536, groups, ws, need - 1)
-    assert kq.lib().kvq_create_in(None, *shape, 0, groups, ws.data_ptr() + 16, need) == kq.KVQ_ERR_ARG
+    import ctypes
+    handle = ctypes.c_void_p()
+    assert kq.lib().kvq_create_in(ctypes.byref(handle), *shape, 0, groups, ws.data_ptr() + 16, need) == kq.KVQ_ERR_ARG
+    host = torch.zeros(need + 256, dtype=torch.uint8)  # host memory is not a workspace
+    host_ptr = (host.data_ptr() + 255) & ~255
+    assert kq.lib().kvq_create_in(ctypes.byref(handle), *shape, 0, groups, host_ptr, need) == kq.KVQ_ERR_ARG
     ctx = kq.kvq_create_in(*shape, arena_blocks * 65536, groups, ws, need)
     oc = oracle.OracleCache(B, Hq, H) if groups == 1 else oracle.GroupedOracleCache(B, Hq, H, 2)
     g = gu.GpuCache.__new__(gu.GpuCache)               # the helper class around an existing handle
