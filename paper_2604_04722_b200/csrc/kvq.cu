@@ -1055,6 +1055,7 @@ int kvq_load_state(kvq_ctx* c, const void* host_buf, uint64_t host_bytes) {
     };
     // Nothing the kernels use as an address may point outside the handle's buffers: check lengths, fills,
     // block ids and index words on the host before anything is replaced.
+    std::vector<uint32_t> clean_table;
     {
         const uint8_t* q = in;
         auto peek = [&]() {
@@ -1078,13 +1079,8 @@ int kvq_load_state(kvq_ctx* c, const void* host_buf, uint64_t host_bytes) {
             if (len[l] != longest) return KVQ_ERR_ARG;
         }
         const uint8_t* arena_blob = q;
-        const uint32_t* table = reinterpret_cast<const uint32_t*>(arena_blob + (size_t)(h.blocks_used + 1) * kBlockBytes);
-        for (size_t i = 0; i < h.table_bytes / sizeof(uint32_t); ++i) {
-            uint32_t id;
-            std::memcpy(&id, table + i, sizeof(id));
-            if (id > h.blocks_used) return KVQ_ERR_ARG;
-        }
-        const uint8_t* index = reinterpret_cast<const uint8_t*>(table) + h.table_bytes;
+        const uint8_t* table = arena_blob + (size_t)(h.blocks_used + 1) * kBlockBytes;
+        const uint8_t* index = table + h.table_bytes;
         for (size_t i = 0; i < h.index_bytes / sizeof(uint32_t); ++i) {
             uint32_t w;
             std::memcpy(&w, index + i * sizeof(uint32_t), sizeof(w));
@@ -1099,6 +1095,25 @@ int kvq_load_state(kvq_ctx* c, const void* host_buf, uint64_t host_bytes) {
                     const uint64_t sum = (uint64_t)f[0] + f[1] + f[2] + f[3];
                     if (which == cur[l] ? sum != (uint64_t)lens[(size_t)l * c->batch + b] : sum > (uint64_t)c->max_ctx) return KVQ_ERR_ARG;
                 }
+        // Block tables: the entries that the current fills reach must name blocks of the snapshot; the rest
+        // (left over from before a reset) are not used and are cleared.
+        clean_table.assign(h.table_bytes / sizeof(uint32_t), 0u);
+        for (int l = 0; l < c->layers; ++l)
+            for (int b = 0; b < c->batch; ++b) {
+                uint32_t f[4];
+                std::memcpy(f, counts + sizeof(uint32_t) * 4 * (((size_t)cur[l] * c->layers + l) * c->batch + b), sizeof(f));
+                for (int hh = 0; hh < c->kv_heads; ++hh)
+                    for (int k = 0; k < kNumPools; ++k) {
+                        const size_t row = (((size_t)l * c->batch + b) * c->kv_heads + hh) * c->store.table_stride + c->store.table_off[k];
+                        const uint32_t reached = blocks_for(k, f[k], c->groups);
+                        for (uint32_t e = 0; e < reached; ++e) {
+                            uint32_t id;
+                            std::memcpy(&id, table + sizeof(uint32_t) * (row + e), sizeof(id));
+                            if (id > h.blocks_used) return KVQ_ERR_ARG;
+                            clean_table[row + e] = id;
+                        }
+                    }
+            }
     }
     KVQ_CUDA(c, cudaDeviceSynchronize());
     for (auto& v : c->len) v = get_int();
@@ -1108,7 +1123,7 @@ int kvq_load_state(kvq_ctx* c, const void* host_buf, uint64_t host_bytes) {
     const size_t arena_bytes = (size_t)(h.blocks_used + 1) * kBlockBytes;
     KVQ_CUDA(c, cudaMemcpy(c->arena, in, arena_bytes, cudaMemcpyHostToDevice));
     in += arena_bytes;
-    KVQ_CUDA(c, cudaMemcpy(c->table, in, h.table_bytes, cudaMemcpyHostToDevice));
+    KVQ_CUDA(c, cudaMemcpy(c->table, clean_table.data(), h.table_bytes, cudaMemcpyHostToDevice));
     in += h.table_bytes;
     KVQ_CUDA(c, cudaMemcpy(c->store.index, in, h.index_bytes, cudaMemcpyHostToDevice));
     in += h.index_bytes;

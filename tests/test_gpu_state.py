@@ -124,3 +124,26 @@ def test_a_snapshot_that_points_outside_the_cache_is_refused(gu):
         assert refused(head + 4, 65)                    # a sequence longer than max_ctx
         assert refused(head, 39)                        # longest length out of step with the lengths
         kq.kvq_load_state(g.ctx, blob)                  # the untouched blob still loads
+
+
+def test_snapshot_after_a_reset(gu):
+    """After kvq_reset the block tables still hold ids from before; they are beyond the fills, are not part of the
+    state, and must not make a snapshot unloadable (also not in a handle with a smaller arena)."""
+    from paper_2604_04722_b200 import binding as kq
+    rng = np.random.default_rng(6)
+    B, Hq, H = 2, 2, 2
+    with gu.GpuCache(1, B, Hq, H, 1200) as g:
+        K, V = _kv(rng, B, 1200, H)
+        g.append(0, K, V, BITS[rng.choice(4, size=(B, 1200))])      # several blocks per stream
+        kq.kvq_reset(g.ctx)
+        K, V = _kv(rng, B, 30, H)
+        bits = BITS[rng.choice(4, size=(B, 30))]
+        g.append(0, K, V, bits)
+        Q = rng.standard_normal((B, Hq, 64)).astype(np.float16)
+        want = g.decode(0, Q)
+        blob = kq.kvq_save_state(g.ctx)
+        kq.kvq_load_state(g.ctx, blob)
+        assert np.array_equal(g.decode(0, Q), want)
+    with gu.GpuCache(1, B, Hq, H, 1200, arena_bytes=40 * 65536) as g2:
+        kq.kvq_load_state(g2.ctx, blob)
+        assert np.array_equal(g2.decode(0, Q), want)
