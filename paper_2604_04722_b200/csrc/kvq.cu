@@ -356,6 +356,7 @@ uint32_t choose_warps(kvq_ctx* c, int len, uint64_t units) {
     const uint64_t tiles = units * (uint64_t)((len + kTileTokens - 1) / kTileTokens + (kNumPools - 1));
     const uint64_t resident = (uint64_t)kDecodeWarps * kDecodeCtasPerSm * c->sm_count;
     uint64_t cap = tiles / 8;
+    if (tiles / 4 <= resident) cap = tiles / 4;        // a small cache is a latency chain: shorter parts, while all warps fit at once
     if (cap < 1) cap = 1;
     if (cap <= resident) return (uint32_t)(cap >= units ? cap / units * units : cap);
     // set-up, ring fill and the final reduction cost a warp about as much as fifteen tiles per part
