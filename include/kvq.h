@@ -92,8 +92,8 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
                      int max_ctx, int batch, uint64_t arena_bytes);
 
 /*
- * The same with a chosen granularity of the min-max quantizer (Eq. 9-13 leave it open; the
- * related work of Section 2 uses finer-grained scales).  scale_groups = 1: one {scale,
+ * The same with a chosen granularity of the min-max quantizer (Eq. 24 only names Q_b and leaves its
+ * granularity open; the related work of Section 2 uses finer-grained scales).  scale_groups = 1: one {scale,
  * zero-point} pair per (token, KV head) row of 64 channels, what kvq_create and
  * kvq_create_arena build.  scale_groups = 2: one pair per group of 32 consecutive channels
  * (channels 0..31 and 32..63), each group quantized by the row quantizer on its own values; the
@@ -162,9 +162,13 @@ int kvq_append(kvq_ctx* ctx, int layer, const void* K, const void* V,
                const uint8_t* bits, int n_new, void* stream);
 
 /*
- * Same as kvq_select_bits followed by kvq_append, with the decision taken
- * inside the append launch: feats is dev fp32 [batch][n_new][4].  bits_out_opt
- * (dev uint8 [batch][n_new] or NULL) receives the decisions.
+ * Same as kvq_select_bits followed by kvq_append, with the controller (Eq. 19-23)
+ * evaluated inside the kernels that quantize and pack (Eq. 24): feats is dev fp32
+ * [batch][n_new][4].  bits_out_opt (dev uint8 [batch][n_new] or NULL) receives
+ * the decisions.  Launches: one kernel for up to 256 new tokens per sequence (a
+ * decode step included); a longer prefill runs three: the controller with a
+ * class histogram per chunk of tokens, the reservation of arena blocks, and the
+ * quantize-and-pack kernel, which reads the classes back from a scratch array.
  */
 int kvq_append_fused(kvq_ctx* ctx, int layer, const void* K, const void* V,
                      const float* feats, int n_new, uint8_t* bits_out_opt, void* stream);
@@ -255,10 +259,11 @@ int kvq_attend_last(kvq_ctx* ctx, int layer, const void* Q, void* O, int n_queri
  * input, Q is read and O is written exactly as in kvq_decode_attn, and none of the
  * handle's own scratch is used.
  *
- * Limit: batch * q_heads * (parts + 1) <= KVQ_STATIC_MAX_PARTIALS, where parts is the value
- * given to kvq_set_splits or, in automatic mode, ceil(W / (batch * q_heads)) with W the
- * number of warps the launch uses (at most 16 per SM of the device); otherwise
- * KVQ_ERR_TOO_LARGE is returned and nothing is queued.
+ * Limit: batch * q_heads * (parts + 1) <= KVQ_STATIC_MAX_PARTIALS, where parts is the number of
+ * pieces a (sequence, query head) unit is cut into.  A value given to kvq_set_splits is taken as
+ * it is, and KVQ_ERR_TOO_LARGE is returned (nothing is queued) if it does not fit.  In automatic
+ * mode the planner picks the best split that fits the array, which may be coarser than what
+ * kvq_decode_attn would pick; KVQ_ERR_TOO_LARGE only if 2 * batch * q_heads records do not fit.
  *
  * Set-up: the first call on each device looks up the device address of the array (once
  * per device, with that device current).  Make that first call outside any stream capture.
@@ -373,8 +378,21 @@ int kvq_profile_read(kvq_ctx* ctx, double* attn_ms_total, int* calls);
 #define KVQ_FLAG_BAD_BITS 1u      /* a bit-width outside {2,4,8,16} was appended (stored as fp16) */
 #define KVQ_FLAG_ARENA_FULL 4u    /* an append ran out of arena blocks; the tokens that did not fit are lost */
 #define KVQ_FLAG_WAIT_TIMEOUT 2u  /* a bounded wait on an async copy expired in kvq_decode_attn; that
-                                     call's output is invalid */
+                                     call's output is invalid.  The warp that gave up still hands in an
+                                     (empty) partial for the rest of its share, so every arrival counter
+                                     the call used is back at zero when it ends and later calls on the
+                                     handle are unaffected; kvq_device_status also runs kvq_recover when
+                                     it reports this flag. */
 int kvq_device_status(kvq_ctx* ctx, uint32_t* host_flags_out);
+
+/*
+ * Put the split-attention bookkeeping of the handle back into its start-up state: the arrival counters of
+ * the handle's scratch, those of the fixed array of kvq_decode_attn_static on the handle's device (if that
+ * call was ever used there) and the device flag word are set to zero.  Cached tokens are untouched.  For use
+ * after a decode call was cut short from outside (the process aborted a stream, a debugger killed a
+ * kernel); a call that ended by itself, even with KVQ_FLAG_WAIT_TIMEOUT, needs none.  Synchronizes.
+ */
+int kvq_recover(kvq_ctx* ctx);
 
 /* Bytes of device memory the handle holds (pools + index + scratch). */
 int kvq_device_bytes(kvq_ctx* ctx, uint64_t* host_bytes_out);

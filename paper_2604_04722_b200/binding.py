@@ -63,6 +63,7 @@ SIGNATURES = {
     "kvq_set_profiling": (_i, [_vp, _i]),
     "kvq_profile_read": (_i, [_vp, C.POINTER(C.c_double), C.POINTER(_i)]),
     "kvq_device_status": (_i, [_vp, C.POINTER(C.c_uint32)]),
+    "kvq_recover": (_i, [_vp]),
     "kvq_device_bytes": (_i, [_vp, _u64p]),
     "kvq_launch_count": (_i, [_vp, _u64p]),
     "kvq_last_cuda_error": (_i, [_vp]),
@@ -317,6 +318,10 @@ def kvq_device_status(ctx: int) -> int:
     if rc not in (KVQ_OK, KVQ_ERR_DEVICE_FLAG):
         raise KvqError(rc, "kvq_device_status")
     return f.value
+
+
+def kvq_recover(ctx: int) -> None:
+    check(lib().kvq_recover(ctx), "kvq_recover")
 
 
 def kvq_device_bytes(ctx: int) -> int:

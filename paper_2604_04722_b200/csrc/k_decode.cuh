@@ -493,7 +493,10 @@ k_decode_attn(DecodeParams P) {
     uint64_t x = (uint64_t)j * P.units;
     const uint64_t xend = x + P.units;
 
-    while (x < xend && !failed) {
+    while (x < xend) {
+        // After an expired wait the warp starts no further copy and walks no further tile, but it still
+        // delivers a (then empty) partial for every remaining segment of its share: the arrival counters of
+        // those units reach their totals and go back to zero, so the handle stays usable after the flag.
         // ---- this segment: ticks [a0, a1) of unit u
         const uint32_t u = (x >> 32) ? (uint32_t)(x / P.gw) : (uint32_t)x / P.gw;
         const uint32_t a0 = (uint32_t)(x - (uint64_t)u * P.gw);
@@ -567,7 +570,7 @@ k_decode_attn(DecodeParams P) {
                 p_next_id = p_tab[0];
             }
         };
-        next_pool();
+        if (!failed) next_pool();
         auto issue_next = [&]() {
             const int n = min(p_phase, p_left);
             p_phase = p_tps;
@@ -642,7 +645,7 @@ k_decode_attn(DecodeParams P) {
         walk(std::integral_constant<int, 2>{}, Quantized<2, G>{});
         walk(std::integral_constant<int, 3>{}, Fp16Rows{});
 
-        if (failed) {
+        if (failed && in_flight > 0) {
             // Copies that were started but not consumed may still land in this warp's ring: give
             // each a bounded wait before the warp can retire, then report.
             for (int i = 1; i < in_flight; ++i) {
@@ -652,6 +655,7 @@ k_decode_attn(DecodeParams P) {
                 }
                 mbar_wait(&ws.bars[cslot], parity);
             }
+            in_flight = 0;
             if (lane == 0) atomicOr(P.store.flags, kFlagWaitTimeout);
         }
 

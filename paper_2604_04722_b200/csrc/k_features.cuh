@@ -28,10 +28,14 @@ struct OnlineEntropy {
         }
         m = m2;
     }
+    // A term whose weight underflows to zero (a masked logit, z = -inf, in particular) adds nothing:
+    // p log p -> 0 as p -> 0 (Eq. 14), whereas d * e would be -inf * 0.
     __device__ __forceinline__ void add(float z) {             // z <= m
         const float d = z - m, e = __expf(d);
-        s += e;
-        w = fmaf(d, e, w);
+        if (e > 0.f) {
+            s += e;
+            w = fmaf(d, e, w);
+        }
     }
     __device__ __forceinline__ void merge(const OnlineEntropy& o) {
         if (o.m > m) {

@@ -350,22 +350,34 @@ constexpr int kMaxQueryRows = 8;       // query rows per sequence that one launc
 
 size_t max_partial_records(const kvq_ctx* c);
 
-uint32_t choose_warps(kvq_ctx* c, int len, uint64_t units) {
-    if (c->splits_override > 0 && units * (uint64_t)(c->splits_override + 1) <= max_partial_records(c))
+// room: partial records the caller has scratch for (0: the handle's own).  Returns 0 if not even one part
+// per unit fits.
+uint32_t choose_warps(kvq_ctx* c, int len, uint64_t units, uint64_t room = 0) {
+    if (room == 0) room = max_partial_records(c);
+    auto fits = [&](uint64_t gw) { return units * (uint64_t)decode_pslots((uint32_t)units, (uint32_t)gw) <= room; };
+    if (!fits(units)) return 0;
+    if (c->splits_override > 0 && units * (uint64_t)(c->splits_override + 1) <= room)
         return (uint32_t)(units * (uint64_t)c->splits_override);
     const uint64_t tiles = units * (uint64_t)((len + kTileTokens - 1) / kTileTokens + (kNumPools - 1));
     const uint64_t resident = (uint64_t)kDecodeWarps * kDecodeCtasPerSm * c->sm_count;
     uint64_t cap = tiles / 8;
     if (tiles / 4 <= resident) cap = tiles / 4;        // a small cache is a latency chain: shorter parts, while all warps fit at once
     if (cap < 1) cap = 1;
-    if (cap <= resident) return (uint32_t)(cap >= units ? cap / units * units : cap);
+    if (cap <= resident) {
+        uint64_t gw = cap >= units ? cap / units * units : cap;
+        if (!fits(gw)) gw = (room / units - 1) * units;            // the most whole parts per unit that fit
+        return (uint32_t)gw;
+    }
     // set-up, ring fill and the final reduction cost a warp about as much as fifteen tiles per part
     // (constants fitted to measured sweeps over the split count on four workload shapes)
     const double tiles_d = (double)tiles;
-    uint64_t best = resident;
-    const double tpw_p = tiles_d / (double)resident;
-    double best_score = 0.90 * tpw_p / (tpw_p + 25.0);           // some warps work on two parts
-    const uint64_t room = max_partial_records(c);                 // partial records the handle has scratch for
+    uint64_t best = units;
+    double best_score = 0.0;
+    if (fits(resident)) {
+        const double tpw_p = tiles_d / (double)resident;
+        best = resident;
+        best_score = 0.90 * tpw_p / (tpw_p + 25.0);               // some warps work on two parts
+    }
     for (uint64_t s = 1; s <= (uint64_t)kMaxSplits && units * s <= cap && units * (s + 1) <= room; ++s) {
         const double fill = (double)(units * s) / (double)resident;
         const double waves = (double)(uint64_t)(fill + 0.999999);
@@ -788,9 +800,11 @@ int kvq_decode_attn_static(kvq_ctx* c, int layer, const void* Q, void* O, void* 
     if (check_layer(c, layer) != KVQ_OK || !Q || !O) return KVQ_ERR_ARG;
     if (c->len[layer] == 0) return KVQ_ERR_EMPTY;
     if (c->device < 0 || c->device >= KVQ_STATIC_MAX_DEVICES) return KVQ_ERR_ARG;
-    const uint32_t gw = choose_warps(c, c->len[layer], (uint64_t)c->batch * c->q_heads);
-    const size_t records = (size_t)c->batch * c->q_heads * decode_pslots((uint32_t)c->batch * c->q_heads, gw);
-    if (records > (size_t)KVQ_STATIC_MAX_PARTIALS) return KVQ_ERR_TOO_LARGE;
+    const uint64_t units = (uint64_t)c->batch * c->q_heads;
+    // an explicit split count is taken as given; the automatic plan is the best one that fits the array
+    if (c->splits_override > 0 && units * (uint64_t)(c->splits_override + 1) > (uint64_t)KVQ_STATIC_MAX_PARTIALS) return KVQ_ERR_TOO_LARGE;
+    const uint32_t gw = choose_warps(c, c->len[layer], units, KVQ_STATIC_MAX_PARTIALS);
+    if (gw == 0) return KVQ_ERR_TOO_LARGE;
     DeviceGuard guard(c->device);
     float* base = nullptr;
     {
@@ -1041,10 +1055,14 @@ int kvq_load_state(kvq_ctx* c, const void* host_buf, uint64_t host_bytes) {
     if (h.layers != c->layers || h.q_heads != c->q_heads || h.kv_heads != c->kv_heads || h.max_ctx != c->max_ctx ||
         h.batch != c->batch || h.groups != c->groups)
         return KVQ_ERR_ARG;
-    // the arena may differ in size as long as the snapshot's blocks fit (block ids are positions in the arena)
-    if (h.blocks_used + 1 > c->store.arena_blocks || h.table_bytes != c->table_bytes) return KVQ_ERR_ARG;
+    // the arena may differ in size as long as the snapshot's blocks fit (block ids are positions in the arena);
+    // every other size in the header has to be this handle's own, whatever the blob claims
+    if ((uint64_t)h.blocks_used + 1 > (uint64_t)c->store.arena_blocks || h.table_bytes != c->table_bytes) return KVQ_ERR_ARG;
+    if (h.index_bytes != sizeof(uint32_t) * (uint64_t)c->layers * c->batch * c->max_ctx ||
+        h.counts_bytes != sizeof(uint32_t) * 2 * (uint64_t)c->layers * c->batch * 4)
+        return KVQ_ERR_ARG;
     const uint64_t host_ints = (uint64_t)c->layers * 3 + (uint64_t)c->layers * c->batch;
-    if (h.total_bytes != sizeof(StateHeader) + sizeof(int32_t) * host_ints + (uint64_t)(h.blocks_used + 1) * kBlockBytes +
+    if (h.total_bytes != sizeof(StateHeader) + sizeof(int32_t) * host_ints + ((uint64_t)h.blocks_used + 1) * kBlockBytes +
                              h.table_bytes + h.index_bytes + h.counts_bytes)
         return KVQ_ERR_ARG;
     const uint8_t* in = static_cast<const uint8_t*>(host_buf) + sizeof(h);
@@ -1175,7 +1193,28 @@ int kvq_device_status(kvq_ctx* c, uint32_t* host_flags_out) {
     KVQ_CUDA(c, cudaDeviceSynchronize());
     KVQ_CUDA(c, cudaMemcpy(host_flags_out, c->flags, sizeof(uint32_t), cudaMemcpyDeviceToHost));
     KVQ_CUDA(c, cudaMemset(c->flags, 0, sizeof(uint32_t)));
+    if (*host_flags_out & KVQ_FLAG_WAIT_TIMEOUT) {     // belt and braces: the kernel already left them at zero
+        const int rc = kvq_recover(c);
+        if (rc != KVQ_OK) return rc;
+    }
     return *host_flags_out ? KVQ_ERR_DEVICE_FLAG : KVQ_OK;
+}
+
+int kvq_recover(kvq_ctx* c) {
+    if (!c) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    KVQ_CUDA(c, cudaDeviceSynchronize());
+    KVQ_CUDA(c, cudaMemset(c->part_cnt, 0, sizeof(uint32_t) * (size_t)c->batch * c->q_heads * kMaxQueryRows));
+    KVQ_CUDA(c, cudaMemset(c->flags, 0, sizeof(uint32_t)));
+    float* base = nullptr;
+    if (c->device >= 0 && c->device < KVQ_STATIC_MAX_DEVICES) {
+        std::lock_guard<std::mutex> hold(g_static_partials_lock);
+        base = g_static_partials_addr[c->device];      // only if kvq_decode_attn_static ever ran on this device
+    }
+    if (base)
+        KVQ_CUDA(c, cudaMemset(base + (size_t)KVQ_STATIC_MAX_PARTIALS * (kHeadDim + 2), 0,
+                               sizeof(uint32_t) * (KVQ_STATIC_MAX_PARTIALS / 2)));
+    return KVQ_OK;
 }
 
 int kvq_device_bytes(kvq_ctx* c, uint64_t* host_bytes_out) {

@@ -17,3 +17,13 @@ def oracle():
     import oracle as _oracle
     _oracle.build()
     return _oracle
+
+
+def pytest_terminal_summary(terminalreporter):
+    """Near-tie controller decisions (top-two logit gap < 1e-5) are listed separately from the assertions."""
+    gu = sys.modules.get("gpu_util")
+    if gu is None or not gu.NEAR_TIE_REPORTS:
+        return
+    terminalreporter.section("controller decisions: near ties")
+    for line in gu.near_tie_summary_lines():
+        terminalreporter.write_line(line)

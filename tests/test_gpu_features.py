@@ -58,6 +58,32 @@ def test_token_features_match_the_definitions(gu, oracle, vocab, dtype, scale):
     assert np.all(no_var[:, 2] == 0.0) and np.allclose(no_var[:, [0, 1, 3]], got[:2][:, [0, 1, 3]])
 
 
+@pytest.mark.parametrize("vocab,dtype", [(49152, np.float16), (1001, np.float32), (4096, np.float32)])
+def test_token_features_with_masked_logits(gu, oracle, vocab, dtype):
+    """Vocabulary entries masked with -inf (p = 0, so p log p = 0 in Eq. 14) leave entropy and confidence
+    finite and equal to those of the unmasked entries: at the start of a row, in whole 8-element groups,
+    scattered, and all but one entry."""
+    rng = np.random.default_rng(vocab)
+    n = 9
+    logits = (rng.standard_normal((n, vocab)) * 3).astype(dtype)
+    logits[0, :16] = -np.inf                                  # the row starts with masked groups
+    logits[1, ::3] = -np.inf                                  # scattered
+    logits[2, vocab // 2:] = -np.inf                          # a masked tail
+    logits[3, :] = -np.inf
+    logits[3, 5] = dtype(0.75)                                # a single survivor: H = 0, C = 1
+    logits[4, :vocab - 3] = -np.inf                           # survivors only in the last group
+    token_ids = rng.integers(0, vocab, size=n)
+    counts = rng.integers(0, 50, size=vocab)
+    got = _features(gu, logits, token_ids, counts, int(counts.sum()), int((counts > 0).sum()), None)
+    with np.errstate(invalid="ignore"):
+        H = oracle.token_entropy(logits)
+        C = oracle.token_confidence(logits)
+    assert np.all(np.isfinite(got))
+    assert np.all(np.abs(got[:, 0] - H) <= 2e-4 + 2e-4 * np.abs(H)), (got[:, 0], H)
+    assert np.all(np.abs(got[:, 3] - C) <= 1e-3 * C + 1e-9)
+    assert got[3, 0] == 0.0 and got[3, 3] == 1.0
+
+
 @pytest.mark.parametrize("n,splits", [(1, 0), (17, 0), (700, 0), (700, 7), (3000, 0)])
 def test_attention_variance_of_the_decode_step(gu, oracle, n, splits):
     """kvq_decode_attn_var: V = mean over heads of the variance of the attention weights over the cached

@@ -123,6 +123,24 @@ def test_a_snapshot_that_points_outside_the_cache_is_refused(gu):
         assert refused(counts_at, 1000)                 # a pool fill that does not add up
         assert refused(head + 4, 65)                    # a sequence longer than max_ctx
         assert refused(head, 39)                        # longest length out of step with the lengths
+
+        # header fields that only have to be consistent with each other to pass a naive check: sizes that are
+        # not this handle's, and a block count that wraps around in 32-bit arithmetic
+        def header_refused(**fields):
+            bad = blob.copy()
+            names = ["magic", "version", "layers", "q_heads", "kv_heads", "max_ctx", "batch", "groups", "arena_blocks",
+                     "blocks_used", "table_bytes", "index_bytes", "counts_bytes", "total_bytes"]
+            vals = dict(zip(names, struct.unpack_from("<II6iII4Q", bad, 0)))
+            vals.update(fields)
+            struct.pack_into("<II6iII4Q", bad, 0, *[vals[k] for k in names])
+            return L.kvq_load_state(g.ctx, bad.ctypes.data, bad.size) == kq.KVQ_ERR_ARG
+
+        assert header_refused(index_bytes=index_bytes + 4096, counts_bytes=counts_bytes)                 # total no longer adds up
+        assert header_refused(index_bytes=index_bytes + 4096, total_bytes=total + 4096)                  # consistent, but too large
+        assert header_refused(index_bytes=index_bytes - 64, counts_bytes=counts_bytes + 64)              # consistent, shifted
+        assert header_refused(counts_bytes=counts_bytes - 16, total_bytes=total - 16)                    # a short fill table
+        assert header_refused(blocks_used=0xffffffff)                                                    # + 1 wraps to 0
+        assert header_refused(blocks_used=0xffffffff, total_bytes=total - (used + 1) * 65536)            # ... consistently
         kq.kvq_load_state(g.ctx, blob)                  # the untouched blob still loads
 
 

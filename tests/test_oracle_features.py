@@ -25,6 +25,20 @@ def test_entropy_closed_forms_and_library_routine(oracle):
     assert np.all(h >= 0) and np.all(h <= math.log(777) + 1e-12)
 
 
+def test_masked_logits_add_nothing_to_the_entropy(oracle):
+    """p log p is 0 at p = 0 (Eq. 14): a vocabulary entry masked with -inf drops out, so the entropy is that of
+    the remaining entries; the same for the confidence."""
+    rng = np.random.default_rng(3)
+    z = rng.standard_normal((4, 200)) * 2
+    masked = np.concatenate([np.full((4, 30), -np.inf), z, np.full((4, 7), -np.inf)], axis=1)
+    with np.errstate(invalid="ignore"):
+        assert np.allclose(oracle.token_entropy(masked), oracle.token_entropy(z), atol=1e-12)
+        assert np.allclose(oracle.token_confidence(masked), oracle.token_confidence(z), atol=1e-15)
+    one = np.full((1, 64), -np.inf)
+    one[0, 11] = 2.5
+    assert oracle.token_entropy(one)[0] == 0.0 and oracle.token_confidence(one)[0] == 1.0
+
+
 def test_confidence_is_the_largest_probability(oracle):
     V = 50
     assert abs(oracle.token_confidence(np.zeros((1, V)))[0] - 1.0 / V) < 1e-15
