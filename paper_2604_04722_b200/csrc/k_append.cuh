@@ -191,7 +191,12 @@ __device__ __forceinline__ void pack_codes(const __half2* hp, float mn, float in
 // multiplies that zero with whatever a recycled block held before.
 // G: scale groups per row.  With G == 2 the half-row is a group of its own: no exchange with the partner lane,
 // and every lane stores (or clears) the {scale, zero-point} word of its own group at `meta`.
-template <int CLS, int PARTNER = 16, int G = 1>
+// TENSOR: 0 = K, 1 = V.  With one scale group per row the codes go into the fragment layout of the decode
+// kernel (kvq_common.cuh): a K row's canonical words are scattered as 32-bit words; a V row's canonical bytes
+// sit slot-minor, four neighbouring slots per word, so in a tile-owning warp (PARTNER == 16) the four lanes of
+// slots 4q .. 4q+3 transpose their bytes among themselves first and store whole words where all four slots
+// belong to this append (single bytes otherwise: the other slots of the word hold tokens of an earlier call).
+template <int CLS, int PARTNER = 16, int G = 1, int TENSOR = 0>
 __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], bool active, bool tail, int half, int t,
                                                         uint8_t* codes, uint8_t* meta) {
     constexpr int BITS = pool_bits(CLS);
@@ -224,11 +229,42 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
     const bool tiny = sf != 0.0f && sf < 6.103515625e-05f;
     if (__any_sync(0xffffffffu, tiny)) pack_codes<CLS, true>(hp, mn, inv, w);
     else pack_codes<CLS, false>(hp, mn, inv, w);
+    if (G == 1 && TENSOR == 1 && PARTNER == 16) {
+        // 4 x 4 byte transposes among the lanes of slots 4q .. 4q+3 (same half): afterwards lane t holds, for every
+        // canonical word wi, byte t % 4 of that word from each of the four slots.  Every lane takes part.
+        const uint32_t group = (__ballot_sync(0xffffffffu, active) >> ((half * 16 + t) & ~3)) & 0xfu;
+        const uint32_t sel_a = (t & 2) ? 0x3276u : 0x5410u, sel_b = (t & 1) ? 0x3715u : 0x6240u;
+#pragma unroll
+        for (int wi = 0; wi < WORDS; ++wi) {
+            const uint32_t y = __byte_perm(w[wi], __shfl_xor_sync(0xffffffffu, w[wi], 2), sel_a);
+            const uint32_t o = __byte_perm(y, __shfl_xor_sync(0xffffffffu, y, 1), sel_b);
+            uint8_t* dst = codes + vfrag_byte_offset(CLS, t & ~3, 4 * (half * WORDS + wi) + (t & 3));
+            if (group == 0xfu) {
+                *reinterpret_cast<uint32_t*>(dst) = o;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (group & (1u << j)) dst[j] = (uint8_t)(o >> (8 * j));
+            }
+        }
+    }
     if (!active) {
         if (tail && (G == 2 || half == 0)) *reinterpret_cast<uint32_t*>(meta) = 0u;
         return;
     }
-    if (CLS == 0) {
+    if (G == 1 && TENSOR == 0) {
+#pragma unroll
+        for (int wi = 0; wi < WORDS; ++wi)
+            *reinterpret_cast<uint32_t*>(codes + kfrag_word_offset(CLS, t, half * WORDS + wi)) = w[wi];
+    } else if (G == 1 && PARTNER != 16) {              // a single token: its V bytes one by one
+#pragma unroll
+        for (int wi = 0; wi < WORDS; ++wi)
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+                codes[vfrag_byte_offset(CLS, t, 4 * (half * WORDS + wi) + b)] = (uint8_t)(w[wi] >> (8 * b));
+    } else if (G == 1) {
+        // stored above
+    } else if (CLS == 0) {
         *reinterpret_cast<uint2*>(codes + unit_offset(0, half, 0, t)) = make_uint2(w[0], w[1]);
     } else {
 #pragma unroll
@@ -489,15 +525,15 @@ k_quant_pack(AppendParams p) {
         switch (cur.k) {
         case 0:
             quantize_store_half_row<0, 16, G>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(0, 0, t, half, G));
-            quantize_store_half_row<0, 16, G>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(0, 1, t, half, G));
+            quantize_store_half_row<0, 16, G, 1>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(0, 1, t, half, G));
             break;
         case 1:
             quantize_store_half_row<1, 16, G>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(1, 0, t, half, G));
-            quantize_store_half_row<1, 16, G>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(1, 1, t, half, G));
+            quantize_store_half_row<1, 16, G, 1>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(1, 1, t, half, G));
             break;
         case 2:
             quantize_store_half_row<2, 16, G>(kraw, active, cur.tail, half, t, rec, rec + meta_offset(2, 0, t, half, G));
-            quantize_store_half_row<2, 16, G>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(2, 1, t, half, G));
+            quantize_store_half_row<2, 16, G, 1>(vraw, active, cur.tail, half, t, vcodes, rec + meta_offset(2, 1, t, half, G));
             break;
         default:                                       // fp16: the lane's 64 input bytes are its four units
             if (active) {
@@ -536,15 +572,15 @@ __device__ __forceinline__ void token_store(int c, const uint4 (&kraw)[4], const
     switch (c) {
     case 0:
         quantize_store_half_row<0, 1, G>(kraw, active, false, half, t, rec, rec + meta_offset(0, 0, t, half, G));
-        quantize_store_half_row<0, 1, G>(vraw, active, false, half, t, vcodes, rec + meta_offset(0, 1, t, half, G));
+        quantize_store_half_row<0, 1, G, 1>(vraw, active, false, half, t, vcodes, rec + meta_offset(0, 1, t, half, G));
         break;
     case 1:
         quantize_store_half_row<1, 1, G>(kraw, active, false, half, t, rec, rec + meta_offset(1, 0, t, half, G));
-        quantize_store_half_row<1, 1, G>(vraw, active, false, half, t, vcodes, rec + meta_offset(1, 1, t, half, G));
+        quantize_store_half_row<1, 1, G, 1>(vraw, active, false, half, t, vcodes, rec + meta_offset(1, 1, t, half, G));
         break;
     case 2:
         quantize_store_half_row<2, 1, G>(kraw, active, false, half, t, rec, rec + meta_offset(2, 0, t, half, G));
-        quantize_store_half_row<2, 1, G>(vraw, active, false, half, t, vcodes, rec + meta_offset(2, 1, t, half, G));
+        quantize_store_half_row<2, 1, G, 1>(vraw, active, false, half, t, vcodes, rec + meta_offset(2, 1, t, half, G));
         break;
     default:
         if (active) {

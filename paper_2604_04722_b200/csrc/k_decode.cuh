@@ -241,13 +241,17 @@ template <bool STATS>
 struct SoftmaxT {
     float m, l, bsum;              // running max (log2 units), sum of p, sum of p * zero-point
     float thr;                     // m + kRescaleSlack: a logit above it forces a rescale
+    static constexpr bool kStats = STATS;
     float s2;                      // sum of p^2 (STATS only)
+    float of[4];                   // fragment path: this lane's four output channels, sum of (p s) c so far
 };
 
 // Fold a tile's logits into the running state and return this lane's p.  The running maximum
 // is only raised when some logit exceeds it by more than kRescaleSlack (one vote per tile).
+// COUNT: whether this lane adds its p to the running sum (with two lanes per token only one of them may,
+// unless the sum is halved afterwards).
 template <bool STATS>
-__device__ __forceinline__ float softmax_step(SoftmaxT<STATS>& st, float (&acc)[kHalfDim], float y) {
+__device__ __forceinline__ float softmax_step(SoftmaxT<STATS>& st, float (&acc)[kHalfDim], float y, bool COUNT = true) {
     if (__any_sync(0xffffffffu, y > st.thr)) {                     // warp-uniform
         const float tmax = warp_max(y);
         const float f = fast_exp2(st.m - tmax);
@@ -257,11 +261,13 @@ __device__ __forceinline__ float softmax_step(SoftmaxT<STATS>& st, float (&acc)[
         st.bsum *= f;
         if (STATS) st.s2 *= f * f;
 #pragma unroll
+        for (int j = 0; j < 4; ++j) st.of[j] *= f;
+#pragma unroll
         for (int j = 0; j < kHalfDim; ++j) acc[j] *= f;
     }
     const float p = fast_exp2(y - st.m);
-    st.l += p;
-    if (STATS) st.s2 = fmaf(p, p, st.s2);
+    st.l += COUNT ? p : 0.f;
+    if (STATS) st.s2 = COUNT ? fmaf(p, p, st.s2) : st.s2;
     return p;
 }
 
@@ -398,6 +404,8 @@ struct Quantized {
 };
 
 // The fp16 pool: rows are stored unchanged; qk holds the plain query.
+// BOTH: both lanes of a token add its p to the running sum (which is then halved at the end of the segment).
+template <bool BOTH>
 struct Fp16Rows {
     static constexpr int REC = pool_rec_bytes(3), UNITS = pool_units(3), WORDS = pool_half_bytes(3) / 4;
     __device__ static __forceinline__ void enter(const QueryInfo& qi, uint32_t (&qreg)[kQRegs], float (&)[kHalfDim]) {
@@ -426,7 +434,7 @@ struct Fp16Rows {
         float y = (d[0] + d[1]) + (d[2] + d[3]);
         y += __shfl_xor_sync(0xffffffffu, y, 16);
         y = valid ? y : -INFINITY;
-        const float p = softmax_step(st, acc, y);
+        const float p = softmax_step(st, acc, y, BOTH || half == 0);
 #pragma unroll
         for (int u = 0; u < UNITS; ++u) {
             uint4 w4 = *reinterpret_cast<const uint4*>(rec + pool_codes_bytes(3) + unit_offset(3, half, u, t));
@@ -441,15 +449,233 @@ struct Fp16Rows {
     }
 };
 
+
+// ---------------------------------------------------------------- fragment path (one scale group per row)
+//
+// The quantized pools of a cache with one {scale, zero-point} pair per row are read with 8-bit integer matrix
+// instructions (mma.sync m16n8k32 / m16n8k16, int32 accumulation: exact), two 16-slot tiles (A, B) per loop
+// iteration.  Lane L = 4 g + q.
+//
+// K side: D[slot][column] = sum over the row's code bytes of code * digit, with the codes of a tile's 16 slots
+// as the row operand and the query as the column operand.  The byte planes of the packed words are masked IN
+// PLACE (code << 2p for plane p of a 2-bit byte, code << 4p of a 4-bit byte); the weight 4^p or 16^p that a
+// plane carries is undone on the query's side: q is put on a fixed-point grid once per segment,
+// T_i = rint(q_i * F * 4^(3-p)) for a channel that sits in plane p (16^(1-p) for 4-bit codes), so that every
+// product comes out as 64 F q c (16 F q c, F q c).  |q_i F| < 2^22, hence |T_i| < 2^28 = four balanced base-256
+// digits, T = d0 + 256 d1 + 65536 d2 + 2^24 d3, -128 <= d < 128.  Tile A's products use columns 0..3 = digits
+// 0..3 (columns 4..7 zero), tile B's columns 4..7, and both accumulate into the same registers: lane (g, q) then
+// holds, for q = 0: digits 0, 1 of A's slots g and g + 8, q = 1: digits 2, 3 of the same, q = 2, 3: the same of
+// tile B.  One exchange between lanes q and q ^ 1 gives every lane the dot product of ONE slot, which it OWNS:
+// slot g + 8 (q & 1) of tile A (q < 2) or B (q >= 2).  The owner evaluates the slot's logit, its softmax weight
+// p and its value weight w = p * scale_v.
+//
+// V side: D[channel group][column] += sum over a tile's 16 slots of code * digit of w, with the V codes stored
+// slot-minor (see kvq_common.cuh) as the row operand and the weights as the column operand: the owners put w
+// on a 24-bit unsigned grid X = rint(w * 2^(24-E)) shared by all tiles of an epoch, the 32 X of the two tiles
+// travel through shared memory, column n < 3 = digit n.  Four products per tile (one per byte plane of the
+// 2-bit and 4-bit codes, one per channel group of the 8-bit codes) accumulate in four int32 accumulators per
+// lane ACROSS tiles; they are turned into fp32 and added to the lane's four output channels only when the grid
+// changes: the running maximum moves, a weight would exceed the grid, or about a thousand tiles have been added
+// (int32 headroom).  Rounding w to the grid loses less than 2^-23 of the largest weight of the epoch per token,
+// the same order as fp32 accumulation.  The V products of a pair run one iteration after its K side: they do
+// not depend on the next pair's K side, and the weights have time to cross shared memory.
+__device__ __forceinline__ void mma_k32_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_k16_u8u8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+    asm("mma.sync.aligned.m16n8k16.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+        : "r"(a0), "r"(a1), "r"(b0));
+}
+__device__ __forceinline__ uint32_t byte_perm(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+constexpr float kGridLimit = 16777215.0f;          // weights on the grid stay below 2^24
+constexpr int kFlushTiles = 1000;                  // int32 headroom: 16 slots * 255 * 255 per tile and accumulator
+
+// The int32 accumulators of the V products and the grid they are on.
+struct ValueAcc {
+    int d[4][4];
+    float fix;                     // 2^(24-E): w * fix is the weight on the grid; +inf = no grid chosen yet
+    float ifix;                    // 2^(E-24)
+};
+
+template <int CLS>
+struct FragRows {
+    static constexpr int BITS = pool_bits(CLS), REC = pool_rec_bytes(CLS, 1);
+    static constexpr int NW = 2 << CLS;            // 32-bit words per lane of one tensor's codes: 2, 4, 8
+    static constexpr int PLANES = 8 / BITS;        // codes per byte: 4, 2, 1
+    static constexpr uint32_t MASK = CLS == 0 ? 0x03030303u : CLS == 1 ? 0x0f0f0f0fu : 0xffffffffu;
+    static constexpr float kDotScale = 1.0f / (float)(1 << (BITS * (PLANES - 1)));    // 1/64, 1/16, 1
+
+    // Channel in byte j of operand register r (0: bytes 4q.., 1: bytes 16+4q..) of K product u, and its byte plane.
+    __device__ static constexpr int k_plane(int u, int r) { return CLS == 0 ? 2 * u + r : CLS == 1 ? u : 0; }
+    __device__ static constexpr int k_element(int u, int r, int q, int j) {
+        return CLS == 0 ? 16 * q + 4 * j + (2 * u + r) : CLS == 1 ? 8 * (q + 4 * r) + 2 * j + u : 4 * (q + 8 * u + 4 * r) + j;
+    }
+    // Column operand of the K products: digit g & 3 of the fixed-point query (the same words serve tile A from
+    // the lanes with g < 4 and tile B from the lanes with g >= 4; see the walk).
+    __device__ static __forceinline__ void make_kb(const float* qrow, float fix_scale, int g, int q, uint32_t (&bk)[4]) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const float plane_scale = (float)(1 << (BITS * (PLANES - 1 - k_plane(u, r))));
+                uint32_t w = 0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int e = k_element(u, r, q, j);
+                    const int T = __float2int_rn(qrow[(e >> 5) * (kHalfDim + 4) + (e & 31)] * (fix_scale * plane_scale));
+                    const int h0 = (T + 128) >> 8, d0 = T - (h0 << 8);
+                    const int h1 = (h0 + 128) >> 8, d1 = h0 - (h1 << 8);
+                    const int h2 = (h1 + 128) >> 8, d2 = h1 - (h2 << 8);
+                    const int dg = (g & 3) == 0 ? d0 : (g & 3) == 1 ? d1 : (g & 3) == 2 ? d2 : h2;
+                    w |= ((uint32_t)dg & 0xffu) << (8 * j);
+                }
+                bk[2 * u + r] = w;
+            }
+    }
+    __device__ static __forceinline__ void load_words(const uint8_t* codes, int lane, uint32_t (&w)[NW]) {
+        if (CLS == 0) {
+            const uint2 v = *reinterpret_cast<const uint2*>(codes + lane * 8);
+            w[0] = v.x; w[1] = v.y;
+        } else {
+#pragma unroll
+            for (int u = 0; u < NW / 4; ++u) {
+                const uint4 v = *reinterpret_cast<const uint4*>(codes + (u * 32 + lane) * 16);
+                w[4 * u] = v.x; w[4 * u + 1] = v.y; w[4 * u + 2] = v.z; w[4 * u + 3] = v.w;
+            }
+        }
+    }
+    // The two K products of one tile, added to d.
+    __device__ static __forceinline__ void k_products(int (&d)[4], const uint32_t (&kw)[NW], const uint32_t (&bk)[4]) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (CLS == 0)
+                mma_k32_u8s8(d, kw[0] & (MASK << (4 * u)), kw[1] & (MASK << (4 * u)), kw[0] & (MASK << (4 * u + 2)),
+                             kw[1] & (MASK << (4 * u + 2)), bk[2 * u], bk[2 * u + 1]);
+            else if (CLS == 1)
+                mma_k32_u8s8(d, kw[0] & (MASK << (4 * u)), kw[1] & (MASK << (4 * u)), kw[2] & (MASK << (4 * u)),
+                             kw[3] & (MASK << (4 * u)), bk[2 * u], bk[2 * u + 1]);
+            else
+                mma_k32_u8s8(d, kw[4 * u], kw[4 * u + 1], kw[4 * u + 2], kw[4 * u + 3], bk[2 * u], bk[2 * u + 1]);
+        }
+    }
+    // Weight of V product m in the lane's output channels (the planes stay where they are in the byte).
+    __device__ static constexpr float plane_weight(int m) {
+        return CLS == 0 ? 1.0f / (float)(1 << (2 * m)) : CLS == 1 ? ((m & 1) ? 1.0f / 16.0f : 1.0f) : 1.0f;
+    }
+    // Move the int32 accumulators into fp32 and clear them.  Lane (g, 0) holds digits 0, 1 of channel groups g
+    // and g + 8, lane (g, 1) digit 2 (the other columns are zero): after one exchange per product lane (g, 0)
+    // has the four channels 4 g .. 4 g + 3 and lane (g, 1) the channels 4 (g + 8) .. + 3, in st.of.
+    template <class SM>
+    __device__ static __forceinline__ void flush(ValueAcc& va, SM& st, int q) {
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            const float c0 = (float)va.d[m][0], c1 = (float)va.d[m][1], c2 = (float)va.d[m][2], c3 = (float)va.d[m][3];
+            const float send = q == 0 ? fmaf(c3, 256.0f, c2) : c0 * 65536.0f;
+            const float mine = q == 0 ? fmaf(c1, 256.0f, c0) : c2 * 65536.0f;
+            const float tot = mine + __shfl_xor_sync(0xffffffffu, send, 1);
+            st.of[m] = fmaf(tot, va.ifix * plane_weight(m), st.of[m]);
+            va.d[m][0] = va.d[m][1] = va.d[m][2] = va.d[m][3] = 0;
+        }
+    }
+    // k_part: logits, softmax weights and value weights of a pair of tiles (recA, recB).  `valid`: the slot this
+    // lane owns holds a token.  The value weights go to xbuf (32 words of shared memory: tile A's 16 slots, then
+    // tile B's; two buffers alternate), the pair's V code words are returned for the v_part one iteration later.
+    template <class SM>
+    __device__ static __forceinline__ void k_part(const uint8_t* recA, const uint8_t* recB, bool valid, int lane, int g, int q,
+                                                  const uint32_t (&bkA)[4], const uint32_t (&bkB)[4], const QueryInfo& qi,
+                                                  SM& st, ValueAcc& va, uint32_t* xbuf, uint32_t (&vwA)[NW],
+                                                  uint32_t (&vwB)[NW]) {
+        uint32_t kwA[NW], kwB[NW];
+        load_words(recA, lane, kwA);
+        load_words(recB, lane, kwB);
+        const int slot = g + 8 * (q & 1);
+        const uint8_t* rec_own = q < 2 ? recA : recB;
+        const float2 km = meta_to_float2(*reinterpret_cast<const uint32_t*>(rec_own + meta_offset(CLS, 0, slot)));
+        const float2 vm = meta_to_float2(*reinterpret_cast<const uint32_t*>(rec_own + meta_offset(CLS, 1, slot)));
+        load_words(recA + pool_codes_bytes(CLS), lane, vwA);
+        load_words(recB + pool_codes_bytes(CLS), lane, vwB);
+
+        int d[4] = {0, 0, 0, 0};
+        k_products(d, kwA, bkA);
+        k_products(d, kwB, bkB);
+        // columns 2q, 2q+1 of slots g (d[0], d[1]) and g + 8 (d[2], d[3]): even q digits 0 and 1, odd q digits 2 and 3
+        const float w0 = (q & 1) ? 65536.0f : 1.0f, w1 = (q & 1) ? 16777216.0f : 256.0f;
+        const float lo = fmaf((float)d[1], w1, (float)d[0] * w0), hi = fmaf((float)d[3], w1, (float)d[2] * w0);
+        const float dot = ((q & 1) ? hi : lo) + __shfl_xor_sync(0xffffffffu, (q & 1) ? lo : hi, 1);
+        float y = fmaf(km.x * (qi.inv_fix * kDotScale), dot, km.y * qi.sumq);
+        y = valid ? y : -INFINITY;
+
+        float e = fast_exp2(y - st.m);                 // the weight under the current maximum
+        float x = (e * vm.x) * va.fix;                 // ... and its place on the current grid
+        if (__builtin_expect(__any_sync(0xffffffffu, y > st.thr || !(x < kGridLimit)), 0)) {   // warp-uniform, rare
+            flush(va, st, q);
+            if (__any_sync(0xffffffffu, y > st.thr)) {
+                const float tmax = warp_max(y);
+                const float f = fast_exp2(st.m - tmax);
+                st.m = tmax;
+                st.thr = tmax + kRescaleSlack;
+                st.l *= f;
+                st.bsum *= f;
+                if (SM::kStats) st.s2 *= f * f;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) st.of[j] *= f;
+                e = fast_exp2(y - st.m);
+            }
+            // a new grid: two bits of headroom above the largest weight of this pair of tiles
+            const float wmax = warp_max(e * vm.x);
+            uint32_t ew = __float_as_uint(wmax) >> 23;
+            ew = ew < 30u ? 30u : ew;
+            va.fix = wmax > 0.f ? __uint_as_float((275u - ew) << 23) : INFINITY;
+            va.ifix = __uint_as_float((ew - 21u) << 23);
+            x = (e * vm.x) * va.fix;
+            x = x < kGridLimit ? x : 0.f;              // no grid yet (every weight of the pair is zero)
+        }
+        st.l += e;
+        st.bsum = fmaf(e, vm.y, st.bsum);
+        if (SM::kStats) st.s2 = fmaf(e, e, st.s2);
+        xbuf[(q >> 1) * kTileTokens + slot] = __float2uint_rn(x);
+    }
+    // The four V products of one tile with the weights xs of its slots 4q .. 4q+3.
+    __device__ static __forceinline__ void v_products(ValueAcc& va, const uint32_t (&vw)[NW], const uint4 xs, uint32_t sel) {
+        const uint32_t bv = byte_perm(byte_perm(xs.x, xs.y, sel), byte_perm(xs.z, xs.w, sel), 0x5410u);
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            if (CLS == 0)
+                mma_k16_u8u8(va.d[m], vw[0] & (MASK << (2 * m)), vw[1] & (MASK << (2 * m)), bv);
+            else if (CLS == 1)
+                mma_k16_u8u8(va.d[m], vw[2 * (m >> 1)] & (MASK << (4 * (m & 1))), vw[2 * (m >> 1) + 1] & (MASK << (4 * (m & 1))), bv);
+            else
+                mma_k16_u8u8(va.d[m], vw[4 * (m >> 1) + 2 * (m & 1)], vw[4 * (m >> 1) + 2 * (m & 1) + 1], bv);
+        }
+    }
+    // v_part: the V products of a pair whose weights were written to xbuf before the warp last synchronised.
+    __device__ static __forceinline__ void v_part(const uint32_t (&vwA)[NW], const uint32_t (&vwB)[NW], const uint32_t* xbuf,
+                                                  int q, uint32_t sel, ValueAcc& va) {
+        v_products(va, vwA, *reinterpret_cast<const uint4*>(xbuf + 4 * q), sel);
+        v_products(va, vwB, *reinterpret_cast<const uint4*>(xbuf + kTileTokens + 4 * q), sel);
+    }
+};
+
 // ---------------------------------------------------------------- the split kernel
 
 // Per-warp scratch in shared memory: the segment being worked on.
-struct WarpScratch {
+struct alignas(16) WarpScratch {
     uint64_t bars[kStages];
     const uint32_t* tab[kNumPools];    // block table of this (layer, sequence, KV head) in each pool
     int lo[kNumPools], hi[kNumPools];  // tile range of the segment in each pool
     uint32_t cnt[kNumPools];           // tokens in each pool
     float q[kHeadDim + 4];             // query row; half 1 starts at q[36] so the two halves sit in different banks
+    uint32_t x[2][2 * kTileTokens];    // fragment path: the value weights of a pair of tiles on the integer grid (two pairs alternate)
+    float o[kHeadDim];                 // fragment path: the segment's output row, gathered from the lanes that own channels
 };
 constexpr int kQHalfStride = kHalfDim + 4;
 
@@ -541,8 +767,9 @@ k_decode_attn(DecodeParams P) {
             // 256 R = 2^(22 - floor(log2 max|q|)), max|q| taken as at least the smallest normal fp16
             const float qmax = fmaxf(warp_max(fmaxf(fabsf(qa), fabsf(qb))), 6.103515625e-05f);
             const uint32_t e = __float_as_uint(qmax) >> 23;        // biased exponent, 113..142
-            qi.fix_scale = __uint_as_float((276u - e) << 23);
-            qi.inv_fix = __uint_as_float((e - 22u) << 23) * kLogitScale;
+            // (the fragment path keeps one bit less, so that the top digit of three balanced base-256 digits fits)
+            qi.fix_scale = __uint_as_float(((G == 1 ? 275u : 276u) - e) << 23);
+            qi.inv_fix = __uint_as_float((e - (G == 1 ? 21u : 22u)) << 23) * kLogitScale;
             qi.q_half = ws.q + half * kQHalfStride;
         }
 
@@ -595,7 +822,7 @@ k_decode_attn(DecodeParams P) {
         int in_flight = 0;
         for (; in_flight < kStages && p_left > 0; ++in_flight) issue_next();
 
-        SoftmaxT<STATS> st = {kNegBig, 0.f, 0.f, kNegBig, 0.f};
+        SoftmaxT<STATS> st = {kNegBig, 0.f, 0.f, kNegBig, 0.f, {0.f, 0.f, 0.f, 0.f}};
         float acc[kHalfDim];
 #pragma unroll
         for (int i = 0; i < kHalfDim; ++i) acc[i] = 0.f;
@@ -640,10 +867,97 @@ k_decode_attn(DecodeParams P) {
             }
             C::leave(acc);
         };
-        walk(std::integral_constant<int, 0>{}, Quantized<0, G>{});
-        walk(std::integral_constant<int, 1>{}, Quantized<1, G>{});
-        walk(std::integral_constant<int, 2>{}, Quantized<2, G>{});
-        walk(std::integral_constant<int, 3>{}, Fp16Rows{});
+        // The same walk for the fragment path, two tiles (A, B) per iteration: lane L = 4 g + q owns slot
+        // g + 8 (q & 1) of tile A (q < 2) or of tile B (q >= 2).  A stage with an odd number of tiles ends with
+        // a pair whose B is absent: it points at A's record again and every one of its slots counts as empty.
+        auto walk_frag = [&](auto cls_tag) {
+            constexpr int CLS = decltype(cls_tag)::value;
+            using C = FragRows<CLS>;
+            int tile0 = ws.lo[CLS];
+            const int hi = ws.hi[CLS];
+            if (tile0 >= hi || failed) return;
+            const uint32_t cnt = ws.cnt[CLS];
+            const int g = lane >> 2, q = lane & 3;
+            const uint32_t my_slot = (uint32_t)((q >> 1) * kTileTokens + g + 8 * (q & 1));     // 0..15 in A, 16..31 in B
+            const uint32_t dg = g < 3 ? (uint32_t)g : 3u;                            // byte 3 of a weight on the grid is zero
+            const uint32_t sel = dg | ((4u + dg) << 4) | (dg << 8) | ((4u + dg) << 12);
+            int phase = tiles_per_stage(CLS, 1) - tile0 % tiles_per_stage(CLS, 1);
+            uint32_t bkA[4], bkB[4];
+            C::make_kb(ws.q, qi.fix_scale, g, q, bkA);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                bkB[i] = g >= 4 ? bkA[i] : 0u;
+                bkA[i] = g < 4 ? bkA[i] : 0u;
+            }
+            ValueAcc va;
+#pragma unroll
+            for (int m = 0; m < 4; ++m) va.d[m][0] = va.d[m][1] = va.d[m][2] = va.d[m][3] = 0;
+            va.fix = INFINITY;
+            va.ifix = 0.f;
+            int since_flush = 0;
+            // The V products of a pair run one iteration late: before the first pair there is a pair of zero
+            // weights, after the last one the pending products are drained.
+            uint32_t vpA[C::NW], vpB[C::NW];
+#pragma unroll
+            for (int i = 0; i < C::NW; ++i) vpA[i] = vpB[i] = 0u;
+            uint32_t pp = 0;                           // buffer the current pair writes its weights to
+            ws.x[1][lane] = 0u;
+            __syncwarp();
+            while (tile0 < hi) {
+                if (!mbar_wait(&ws.bars[cslot], parity)) {
+                    failed = true;
+                    break;
+                }
+                const int ntiles = min(phase, hi - tile0);
+                phase = tiles_per_stage(CLS, 1);
+                const uint8_t* buf = my_ring + (size_t)cslot * kStageBytes;
+                for (int i = 0; i < ntiles; i += 2) {
+                    const bool has_b = i + 1 < ntiles;
+                    const uint8_t* recA = buf + (size_t)i * C::REC;
+                    const uint8_t* recB = has_b ? recA + C::REC : recA;
+                    const bool valid = (uint32_t)((tile0 + i) * kTileTokens) + my_slot < cnt && (q < 2 || has_b);
+                    uint32_t vwA[C::NW], vwB[C::NW];
+                    C::v_part(vpA, vpB, ws.x[pp ^ 1u], q, sel, va);
+                    C::k_part(recA, recB, valid, lane, g, q, bkA, bkB, qi, st, va, ws.x[pp], vwA, vwB);
+                    __syncwarp();                      // the pair's weights are in shared memory
+                    pp ^= 1u;
+#pragma unroll
+                    for (int k = 0; k < C::NW; ++k) {
+                        vpA[k] = vwA[k];
+                        vpB[k] = vwB[k];
+                    }
+                }
+                tile0 += ntiles;
+                since_flush += ntiles;
+                if (since_flush >= kFlushTiles) {
+                    C::flush(va, st, q);
+                    since_flush = 0;
+                }
+                --in_flight;
+                __syncwarp();                          // every lane is done with the slot before it is refilled
+                if (p_left > 0) {
+                    issue_next();
+                    ++in_flight;
+                }
+                if (++cslot == kStages) {
+                    cslot = 0;
+                    parity ^= 1u;
+                }
+            }
+            C::v_part(vpA, vpB, ws.x[pp ^ 1u], q, sel, va);     // the last pair's products
+            C::flush(va, st, q);
+        };
+        if constexpr (G == 1) {
+            walk_frag(std::integral_constant<int, 0>{});
+            walk_frag(std::integral_constant<int, 1>{});
+            walk_frag(std::integral_constant<int, 2>{});
+            walk(std::integral_constant<int, 3>{}, Fp16Rows<false>{});
+        } else {
+            walk(std::integral_constant<int, 0>{}, Quantized<0, G>{});
+            walk(std::integral_constant<int, 1>{}, Quantized<1, G>{});
+            walk(std::integral_constant<int, 2>{}, Quantized<2, G>{});
+            walk(std::integral_constant<int, 3>{}, Fp16Rows<true>{});
+        }
 
         if (failed && in_flight > 0) {
             // Copies that were started but not consumed may still land in this warp's ring: give
@@ -689,16 +1003,31 @@ k_decode_attn(DecodeParams P) {
             const float keep = up ? r4[k + 2] : r4[k], send = up ? r4[k] : r4[k + 2];
             r2[k] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
         }
-        // both lanes of a token added its p and p * zero-point: halve the warp sums
-        const float l_w = 0.5f * warp_sum(st.l);
-        // (with two scale groups each half has its own zero-points: the sum stays inside the half)
-        const float b_w = G == 1 ? 0.5f * warp_sum(st.bsum) : half_sum(st.bsum);
+        // Two scale groups: both lanes of a token added its p and p * zero-point, so the warp sums are halved
+        // (each half has its own zero-points: that sum stays inside the half).  One scale group: every token was
+        // counted by exactly one lane; the quantized pools' part of the row sits with the lanes that own channels
+        // and is gathered through shared memory.
+        const float l_w = (G == 1 ? 1.0f : 0.5f) * warp_sum(st.l);
+        const float b_w = G == 1 ? warp_sum(st.bsum) : half_sum(st.bsum);
+        if (G == 1) {
+            if ((lane & 3) < 2)
+                *reinterpret_cast<float4*>(ws.o + 4 * ((lane >> 2) + 8 * (lane & 3))) =
+                    make_float4(st.of[0] + b_w, st.of[1] + b_w, st.of[2] + b_w, st.of[3] + b_w);
+            __syncwarp();
+            const float2 o2 = *reinterpret_cast<const float2*>(ws.o + 2 * lane);
+            r2[0] += o2.x;
+            r2[1] += o2.y;
+            __syncwarp();                              // ws.o is written again in the warp's next segment
+        } else {
+            r2[0] += b_w;
+            r2[1] += b_w;
+        }
         const uint32_t jf = decode_first_warp(u, P.units, P.gw);
         const size_t rec0 = (size_t)u * P.pslots;
-        reinterpret_cast<float2*>(P.part_o + (rec0 + (j - jf)) * kHeadDim)[lane] = make_float2(r2[0] + b_w, r2[1] + b_w);
+        reinterpret_cast<float2*>(P.part_o + (rec0 + (j - jf)) * kHeadDim)[lane] = make_float2(r2[0], r2[1]);
         if (lane == 0) P.part_ml[rec0 + (j - jf)] = make_float2(st.m, l_w);
         if (STATS) {
-            const float s2_w = 0.5f * warp_sum(st.s2);
+            const float s2_w = (G == 1 ? 1.0f : 0.5f) * warp_sum(st.s2);
             if (lane == 0) P.part_s2[rec0 + (j - jf)] = s2_w;
         }
 

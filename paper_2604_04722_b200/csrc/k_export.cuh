@@ -1,5 +1,6 @@
 // Canonical copy of cached tokens, position by position: looks every token up
-// through the per-token index word (pool << 30 | slot) and gathers the units of
+// through the per-token index word (pool << 30 | slot) and gathers the units (or,
+// in the fragment layout, the words and bytes) of
 // its rows from the tile records into plain 128-byte rows (packed codes first,
 // zero tail) plus {scale, zero-point} pairs.  Used to compare the store with
 // other implementations of the quantizer named in Eq. 24.
@@ -42,7 +43,21 @@ k_export(ExportParams p) {
         const uint8_t* codes = tile_ptr(s, cls, stream_table(s, cls, p.layer, b, h), (uint32_t)tile, s.groups) +
                                (size_t)tensor * pool_codes_bytes(cls);
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (j < W) {
+        if (j < W && cls < 3 && s.groups == 1) {       // fragment layout: K rows word by word, V rows byte by byte
+            uint32_t w[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (tensor == 0) {
+                    w[k] = *reinterpret_cast<const uint32_t*>(codes + kfrag_word_offset(cls, t, 4 * j + k));
+                } else {
+                    w[k] = 0;
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)
+                        w[k] |= (uint32_t)codes[vfrag_byte_offset(cls, t, 16 * j + 4 * k + b)] << (8 * b);
+                }
+            }
+            v = make_uint4(w[0], w[1], w[2], w[3]);
+        } else if (j < W) {
             if (cls == 0) {                            // the 16-byte row is two 8-byte half-rows
                 const uint2 lo = *reinterpret_cast<const uint2*>(codes + unit_offset(0, 0, 0, t));
                 const uint2 hi = *reinterpret_cast<const uint2*>(codes + unit_offset(0, 1, 0, t));

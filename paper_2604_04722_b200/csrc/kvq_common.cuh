@@ -66,6 +66,40 @@ __host__ __device__ constexpr int meta_offset(int c, int tensor, int t, int half
     return 2 * pool_codes_bytes(c) + tensor * pool_meta_bytes(c, g) + (g == 2 ? half * 4 * kTileTokens : 0) + 4 * t;
 }
 
+// ---- Fragment layout of the quantized classes (caches with one scale group per row).
+//
+// The decode kernel feeds the codes of a 16-slot tile straight into 8-bit integer matrix instructions
+// (16 rows x 8 columns per warp; a lane L = 4 g + q holds, of an operand with rows = slots, the four bytes
+// 4q .. 4q+3 of row g and of row g + 8).  Both code blocks of a tile record are therefore stored in the
+// order in which the lanes of the reading warp load them, so that one 8- or 16-byte load per lane yields
+// operand registers without any shuffling:
+//
+//   K codes  rows = slots, bytes = the row's canonical bytes.  Lane (g, q) holds, for slot g (i = 0) and slot
+//            g + 8 (i = 1), the canonical 32-bit words q, q + 4, q + 8, ... of the row (word wq = q + 4 wsel).
+//   V codes  rows = channel groups, bytes = SLOTS (the product sums over the tokens of the tile).  Row rho of
+//            an operand holds canonical byte(s) of index rho << c .. of the token rows, i.e. channels 4 rho ..
+//            4 rho + 3 in every class; lane (g, q) holds, for rho = g (i = 0) and rho = g + 8 (i = 1), the words
+//            whose byte j is that canonical byte of slot 4 q + j.
+//
+// Offsets below are relative to the start of the tensor's code block; the {scale, zero-point} words keep
+// their place behind the code blocks.  Caches with two scale groups per row keep the unit layout above.
+__host__ __device__ constexpr int frag_lane(int g, int q) { return 4 * g + q; }
+// canonical 32-bit word wq of the K row of slot t
+__host__ __device__ constexpr int kfrag_word_offset(int c, int t, int wq) {
+    const int lane = frag_lane(t & 7, wq & 3), i = t >> 3, wsel = wq >> 2;
+    return c == 0   ? lane * 8 + i * 4
+           : c == 1 ? lane * 16 + (wsel * 2 + i) * 4
+                    : ((wsel >> 1) * 32 + lane) * 16 + ((wsel & 1) * 2 + i) * 4;
+}
+// canonical byte cb of the V row of slot t
+__host__ __device__ constexpr int vfrag_byte_offset(int c, int t, int cb) {
+    const int rho = cb >> c, m = cb & ((1 << c) - 1);
+    const int lane = frag_lane(rho & 7, t >> 2), i = rho >> 3, j = t & 3;
+    return c == 0   ? lane * 8 + i * 4 + j
+           : c == 1 ? lane * 16 + (m * 2 + i) * 4 + j
+                    : ((m >> 1) * 32 + lane) * 16 + ((m & 1) * 2 + i) * 4 + j;
+}
+
 // Programmatic dependent launch: a kernel launched with the stream-serialization attribute may be scheduled
 // while the kernel before it in the stream is still running, once every CTA of that kernel has called
 // pdl_launch_dependents (or exited); it must call pdl_wait before it touches memory the earlier kernel reads
