@@ -19,8 +19,8 @@
 // back to zero.  The launch is persistent when gw is the number of warps
 // resident on the device; nothing in the kernel waits for another warp.
 //
-// Data movement: the tiles of a segment are cut into chunks of up to
-// kStageBytes contiguous bytes; every warp runs its own ring of kStages
+// Data movement: the tiles of a segment are cut into chunks of up to one stage of
+// contiguous bytes; every warp runs its own ring of a few stages (see DecodeGeom) of
 // shared-memory buffers filled by 1-D bulk async copies (cp.async.bulk,
 // completion on an mbarrier), issued kStages chunks ahead by lane 0.  Every
 // mbarrier wait is bounded: on expiry the warp records KVQ_FLAG_WAIT_TIMEOUT
@@ -55,29 +55,30 @@
 #pragma once
 #include "kvq_common.cuh"
 
-#ifndef KVQ_DECODE_STAGES
-#define KVQ_DECODE_STAGES 2
-#endif
-#ifndef KVQ_DECODE_WARPS
-#define KVQ_DECODE_WARPS 4
-#endif
 #ifndef KVQ_DECODE_FMA2
-#define KVQ_DECODE_FMA2 1          // V-side accumulation with packed two-lane fp32 FMAs
-#endif
-#ifndef KVQ_DECODE_MIN_CTAS
-#define KVQ_DECODE_MIN_CTAS 4
-#endif
-#ifndef KVQ_DECODE_STAGE_BYTES
-#define KVQ_DECODE_STAGE_BYTES 6528
+#define KVQ_DECODE_FMA2 1          // fp16 pool: V-side accumulation with packed two-lane fp32 FMAs
 #endif
 
 namespace kvq {
 
-constexpr int kDecodeWarps = KVQ_DECODE_WARPS;
-constexpr int kDecodeThreads = kDecodeWarps * 32;
-constexpr int kDecodeCtasPerSm = KVQ_DECODE_MIN_CTAS;
-constexpr int kStages = KVQ_DECODE_STAGES;
-constexpr int kStageBytes = KVQ_DECODE_STAGE_BYTES;   // three 8-bit tiles; 10 / 5 / 3 / 1 tiles of the four classes
+// Launch geometry.  The kernel is instantiated twice:
+//   Large: 4 warps per CTA, 4 CTAs per SM, per-warp rings of two 6.5 KB stages -- the bandwidth configuration
+//          (16 resident warps per SM, 209 KB of rings);
+//   Small: 8 warps per CTA, 1 CTA per SM, per-warp rings of four 4.25 KB stages -- for launches of few warps,
+//          where a warp's whole share is in flight at once and the parts of a (sequence, query head) unit sit in
+//          one CTA, which merges them through shared memory (no partial records, no global counter).
+template <int WARPS, int STAGES, int STAGE_BYTES, int MIN_CTAS>
+struct DecodeGeom {
+    static constexpr int kWarps = WARPS, kThreads = WARPS * 32, kStages = STAGES, kStageBytes = STAGE_BYTES, kCtasPerSm = MIN_CTAS;
+    static constexpr size_t kSmemBytes = (size_t)WARPS * STAGES * STAGE_BYTES;
+    static constexpr bool kCtaMerge = MIN_CTAS == 1;   // only the one-CTA-per-SM geometry merges inside the CTA
+    // tiles of class c that fit one stage
+    __host__ __device__ static constexpr int tps(int c, int g = 1) { return STAGE_BYTES / pool_rec_bytes(c, g); }
+    static_assert(STAGE_BYTES % 16 == 0 && STAGE_BYTES >= pool_rec_bytes(3), "a stage must hold one fp16 tile");
+};
+using GeomLarge = DecodeGeom<4, 2, 6528, 4>;          // 10 / 5 / 3 / 1 tiles of the four classes per stage
+using GeomSmall = DecodeGeom<8, 4, 4352, 1>;          //  6 / 3 / 2 / 1
+
 constexpr int kHalfDim = kHeadDim / 2;           // elements per lane
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLogitScale = 0.125f * kLog2e;   // 1/sqrt(64), in log2 units
@@ -85,16 +86,6 @@ constexpr float kRescaleSlack = 8.0f;            // the running maximum may lag 
 constexpr float kNegBig = -1.0e30f;
 constexpr uint32_t kWaitLimit = 1u << 20;        // mbarrier polls before a wait is abandoned
 constexpr uint32_t kFlagWaitTimeout = 2u;
-
-static_assert(kStageBytes % 16 == 0 && kStageBytes >= pool_rec_bytes(3), "a stage must hold one fp16 tile");
-static_assert(block_tiles(0) % (kStageBytes / pool_rec_bytes(0)) == 0 && block_tiles(1) % (kStageBytes / pool_rec_bytes(1)) == 0 &&
-                  block_tiles(2) % (kStageBytes / pool_rec_bytes(2)) == 0 && block_tiles(3) % (kStageBytes / pool_rec_bytes(3)) == 0,
-              "an arena block must hold a whole number of ring stages");
-__host__ __device__ constexpr int tiles_per_stage(int c, int g = 1) { return kStageBytes / pool_rec_bytes(c, g); }
-static_assert(block_tiles(0, 2) % tiles_per_stage(0, 2) == 0 && block_tiles(1, 2) % tiles_per_stage(1, 2) == 0 &&
-                  block_tiles(2, 2) % tiles_per_stage(2, 2) == 0 && block_tiles(3, 2) % tiles_per_stage(3, 2) == 0,
-              "the same with two scale groups per row");
-constexpr size_t kDecodeSmemBytes = (size_t)kDecodeWarps * kStages * kStageBytes;
 
 struct DecodeParams {
     StoreView store;
@@ -114,6 +105,7 @@ struct DecodeParams {
     uint32_t units;                // batch * tq * q_heads
     uint32_t gw;                   // working warps = parts the x axis is cut into
     uint32_t pslots;               // partial slots per unit = decode_pslots(units, gw)
+    uint32_t cta_parts;            // > 0: gw = units * cta_parts and the parts of a unit share a CTA, which merges them itself
 };
 
 // Warps that can overlap one unit: ceil(gw/units) + 1.
@@ -668,42 +660,145 @@ struct FragRows {
 // ---------------------------------------------------------------- the split kernel
 
 // Per-warp scratch in shared memory: the segment being worked on.
+template <int STAGES>
 struct alignas(16) WarpScratch {
-    uint64_t bars[kStages];
+    uint64_t bars[STAGES];
     const uint32_t* tab[kNumPools];    // block table of this (layer, sequence, KV head) in each pool
     int lo[kNumPools], hi[kNumPools];  // tile range of the segment in each pool
     uint32_t cnt[kNumPools];           // tokens in each pool
+    uint32_t id[kNumPools];            // arena block that holds tile lo of each pool
     float q[kHeadDim + 4];             // query row; half 1 starts at q[36] so the two halves sit in different banks
     uint32_t x[2][2 * kTileTokens];    // fragment path: the value weights of a pair of tiles on the integer grid (two pairs alternate)
-    float o[kHeadDim];                 // fragment path: the segment's output row, gathered from the lanes that own channels
+    float o[kHeadDim];                 // the segment's output row (fragment path: gathered from the lanes that own channels;
+                                       // CTA merge: this warp's partial)
+    float2 ml;                         // CTA merge: this warp's (m, l)
+    float s2;                          //            and its sum of squared weights
+    uint32_t arrived;                  // CTA merge: partials delivered to the unit whose first warp this is
 };
 constexpr int kQHalfStride = kHalfDim + 4;
 
-template <int G>
-__device__ __forceinline__ int tps_of(int c) {
-    return c == 0   ? tiles_per_stage(0, G)
-           : c == 1 ? tiles_per_stage(1, G)
-           : c == 2 ? tiles_per_stage(2, G)
-                    : tiles_per_stage(3, G);
-}
 // floor(n * a / g) for a <= g < 65536 in 32-bit arithmetic: n = q*g + r gives q*a + floor(r*a/g).
 __device__ __forceinline__ uint32_t scale_by_fraction(uint32_t n, uint32_t a, uint32_t g) {
     const uint32_t q = n / g, r = n - q * g;
     return q * a + r * a / g;
 }
+// Chunks of a stream end where a stage is full (counted from the start of the arena block, tps tiles per stage),
+// where the block ends, or where the segment's tiles of the pool end -- so a chunk is one contiguous run of bytes,
+// and the copying and the reading side cut the same chunks.  A cursor carries the tiles left up to the next stage
+// boundary and up to the end of the block.
+struct ChunkCursor {
+    int to_stage, to_block;
+    __device__ __forceinline__ void start(int in_block_index, int tps, int bt) {
+        to_stage = tps - in_block_index % tps;
+        to_block = bt - in_block_index;
+    }
+    __device__ __forceinline__ int next(int left) const { return min(min(to_stage, to_block), left); }
+    // true if the chunk of n tiles ended the block
+    __device__ __forceinline__ bool advance(int n, int tps, int bt) {
+        to_block -= n;
+        to_stage = to_stage == n ? tps : to_stage - n;
+        if (to_block != 0) return false;
+        to_block = bt;
+        to_stage = tps;
+        return true;
+    }
+};
 
-// grid = ceil(gw / kDecodeWarps), block = kDecodeThreads, dynamic smem = kDecodeSmemBytes.
+// Merge n_u partials (M = max m_j, l = sum l_j 2^(m_j - M), O = sum o_j 2^(m_j - M) / l) and write the fp16 row.
+// ml(s), o(s) [this lane's float2 of partial s], s2(s) read partial s, from global records or from shared memory.
+template <bool STATS, class LoadMl, class LoadO, class LoadS2>
+__device__ __forceinline__ void merge_partials(const DecodeParams& P, uint32_t u, uint32_t row, size_t qo, uint32_t n_u, int lane,
+                                               LoadMl ml_of, LoadO o_of, LoadS2 s2_of) {
+    float M = kNegBig, L = 0.f, o0 = 0.f, o1 = 0.f;
+    if (n_u <= 32) {                                   // the usual case: lane s weighs partial s; loads go out eight at a time
+        const float2 ml = lane < n_u ? ml_of(lane) : make_float2(kNegBig, 0.f);
+        float2 o[8];
+#pragma unroll
+        for (uint32_t k = 0; k < 8; ++k) o[k] = k < n_u ? o_of(k) : make_float2(0.f, 0.f);
+        M = warp_max(ml.x);
+        const float f = fast_exp2(ml.x - M);
+        L = warp_sum(ml.y * f);
+#pragma unroll
+        for (uint32_t k = 0; k < 8; ++k) {
+            const float fk = __shfl_sync(0xffffffffu, f, k);
+            o0 = fmaf(o[k].x, fk, o0);
+            o1 = fmaf(o[k].y, fk, o1);
+        }
+        for (uint32_t k0 = 8; k0 < n_u; k0 += 8) {
+#pragma unroll
+            for (uint32_t k = 0; k < 8; ++k) o[k] = k0 + k < n_u ? o_of(k0 + k) : make_float2(0.f, 0.f);
+#pragma unroll
+            for (uint32_t k = 0; k < 8; ++k) {
+                const float fk = __shfl_sync(0xffffffffu, f, (k0 + k) & 31);
+                o0 = fmaf(o[k].x, fk, o0);
+                o1 = fmaf(o[k].y, fk, o1);
+            }
+        }
+    } else {
+        for (uint32_t s0 = 0; s0 < n_u; s0 += 32) {    // the maximum, 32 partials at a time
+            const uint32_t s = s0 + lane;
+            M = fmaxf(M, s < n_u ? ml_of(s).x : kNegBig);
+        }
+        M = warp_max(M);
+        for (uint32_t s0 = 0; s0 < n_u; s0 += 32) {
+            const uint32_t s = s0 + lane;
+            const float2 ml = s < n_u ? ml_of(s) : make_float2(kNegBig, 0.f);
+            const float f = fast_exp2(ml.x - M);
+            L += warp_sum(ml.y * f);
+            const uint32_t cnt = min(32u, n_u - s0);
+            for (uint32_t k0 = 0; k0 < cnt; k0 += 8) {
+                float2 o[8];
+#pragma unroll
+                for (uint32_t k = 0; k < 8; ++k) o[k] = k0 + k < cnt ? o_of(s0 + k0 + k) : make_float2(0.f, 0.f);
+#pragma unroll
+                for (uint32_t k = 0; k < 8; ++k) {
+                    const float fk = __shfl_sync(0xffffffffu, f, (k0 + k) & 31);
+                    o0 = fmaf(o[k].x, fk, o0);
+                    o1 = fmaf(o[k].y, fk, o1);
+                }
+            }
+        }
+    }
+    const float inv = L > 0.f ? 1.0f / L : 0.f;        // a sequence that holds no token yet gets zeros
+    reinterpret_cast<__half2*>(P.O + qo)[lane] = __floats2half2_rn(o0 * inv, o1 * inv);
+    if (STATS) {
+        // weights a_t = p_t / L sum to one over the n cached tokens: Var = sum a_t^2 / n - 1 / n^2
+        float S2 = 0.f;
+        for (uint32_t s0 = 0; s0 < n_u; s0 += 32) {
+            const uint32_t s = s0 + lane;
+            if (s < n_u) {
+                const float f = fast_exp2(ml_of(s).x - M);
+                S2 = fmaf(s2_of(s), f * f, S2);
+            }
+        }
+        S2 = warp_sum(S2);
+        if (lane == 0) {
+            const uint4 cnt = *reinterpret_cast<const uint4*>(P.counts + (size_t)row * 4);
+            const float n = (float)(cnt.x + cnt.y + cnt.z + cnt.w);
+            P.unit_var[u] = n > 0.f ? (S2 * inv * inv) / n - 1.0f / (n * n) : 0.f;
+        }
+    }
+}
+
+// grid = ceil(gw / Geo::kWarps), block = Geo::kThreads, dynamic smem = Geo::kSmemBytes.
 // STATS: also emit, per unit, the variance of its attention weights over the cached tokens.
-template <bool STATS, int G>
-__global__ void __launch_bounds__(kDecodeThreads, KVQ_DECODE_MIN_CTAS)
+// P.cta_parts > 0: every unit is cut into that many parts (a divisor of Geo::kWarps), so all parts of a unit run in
+// one CTA, which merges them through shared memory.
+template <bool STATS, int G, class Geo>
+__global__ void __launch_bounds__(Geo::kThreads, Geo::kCtasPerSm)
 k_decode_attn(DecodeParams P) {
+    constexpr int kStages = Geo::kStages, kStageBytes = Geo::kStageBytes;
     extern __shared__ __align__(128) uint8_t ring[];   // [warps][stages][kStageBytes]
-    __shared__ WarpScratch scratch[kDecodeWarps];
+    __shared__ WarpScratch<kStages> scratch[Geo::kWarps];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int half = lane >> 4, t = lane & 15;
-    const uint32_t j = blockIdx.x * kDecodeWarps + warp;
+    const uint32_t j = blockIdx.x * Geo::kWarps + warp;
+    if (Geo::kCtaMerge && P.cta_parts) {               // the arrival counters of this CTA's units start at zero:
+        if (lane == 0) scratch[warp].arrived = 0u;     // the only barrier of the kernel, before any warp can wait
+        __syncthreads();
+    }
     if (j >= P.gw) return;                             // warps never wait for one another
-    WarpScratch& ws = scratch[warp];
+    WarpScratch<kStages>& ws = scratch[warp];
     uint8_t* my_ring = ring + (size_t)warp * kStages * kStageBytes;
     if (lane == 0) {
         for (int s = 0; s < kStages; ++s) mbar_init(&ws.bars[s], 1);
@@ -714,7 +809,7 @@ k_decode_attn(DecodeParams P) {
     pdl_wait();                                        // the append before this launch has stored its token
 
     int pslot = 0, cslot = 0;                          // ring slot the next copy goes to / the next chunk is read from
-    uint32_t parity = 0;                               // phase parity of cslot
+    uint32_t par_bits = 0;                             // phase parity of every ring slot (bit s: slot s)
     bool failed = false;
     uint64_t x = (uint64_t)j * P.units;
     const uint64_t xend = x + P.units;
@@ -735,17 +830,26 @@ k_decode_attn(DecodeParams P) {
         const int kvh = (int)qh / P.group;
         if (lane < kNumPools) {                        // lane c plans pool c
             const int c = lane;
+            const uint32_t* tab = stream_table(P.store, c, P.layer, (int)b, kvh);
+            // The id of the stream's first block is requested together with the pool fill: a short cache starts in
+            // it, and then the block table costs no memory round trip of its own.
+            const uint32_t id_first = tab[0];
             const uint32_t n = P.counts[(size_t)row * 4 + c];
             const uint32_t nt = (n + kTileTokens - 1) / kTileTokens;
             ws.cnt[c] = n;
+            int lo, hi;
             if (P.gw < 65536u) {
-                ws.lo[c] = (int)scale_by_fraction(nt, a0, P.gw);
-                ws.hi[c] = (int)scale_by_fraction(nt, a1, P.gw);
+                lo = (int)scale_by_fraction(nt, a0, P.gw);
+                hi = (int)scale_by_fraction(nt, a1, P.gw);
             } else {
-                ws.lo[c] = (int)((uint64_t)nt * a0 / P.gw);
-                ws.hi[c] = (int)((uint64_t)nt * a1 / P.gw);
+                lo = (int)((uint64_t)nt * a0 / P.gw);
+                hi = (int)((uint64_t)nt * a1 / P.gw);
             }
-            ws.tab[c] = stream_table(P.store, c, P.layer, (int)b, kvh);
+            ws.lo[c] = lo;
+            ws.hi[c] = hi;
+            ws.tab[c] = tab;
+            const uint32_t blk = (uint32_t)lo / block_tiles(c, G);
+            ws.id[c] = (blk == 0 || lo >= hi) ? id_first : tab[blk];
         }
         {
             const float2 q2 = __half22float2(reinterpret_cast<const __half2*>(P.Q + qo)[lane]);
@@ -767,17 +871,17 @@ k_decode_attn(DecodeParams P) {
             // 256 R = 2^(22 - floor(log2 max|q|)), max|q| taken as at least the smallest normal fp16
             const float qmax = fmaxf(warp_max(fmaxf(fabsf(qa), fabsf(qb))), 6.103515625e-05f);
             const uint32_t e = __float_as_uint(qmax) >> 23;        // biased exponent, 113..142
-            // (the fragment path keeps one bit less, so that the top digit of three balanced base-256 digits fits)
+            // (the fragment path keeps one bit less: |q F| < 2^22, see FragRows)
             qi.fix_scale = __uint_as_float(((G == 1 ? 275u : 276u) - e) << 23);
             qi.inv_fix = __uint_as_float((e - (G == 1 ? 21u : 22u)) << 23) * kLogitScale;
             qi.q_half = ws.q + half * kQHalfStride;
         }
 
-        // ---- producer cursor (warp-uniform; lane 0 issues): next tile to fetch, tiles left in its pool
-        // Chunks end at absolute multiples of the pool's tiles-per-stage, and a block holds a whole number
-        // of stages, so a chunk never crosses a 64 KB block of the arena; the id of the block after the
-        // current one is fetched from the stream's table a whole block ahead of its first use.
-        int p_c = -1, p_left = 0, p_tps = 0, p_in_block = 0, p_phase = 0;
+        // ---- producer cursor (warp-uniform; lane 0 issues): next tile to fetch, tiles left in its pool.
+        // A chunk never crosses a 64 KB block of the arena (see chunk_tiles); the id of the block after the current
+        // one is fetched from the stream's table a whole block ahead of its first use.
+        int p_c = -1, p_left = 0, p_tps = 0, p_bt = 0;
+        ChunkCursor p_cur = {0, 0};
         uint32_t p_rec = 0, p_next_id = 0;
         const uint8_t* p_ptr = nullptr;
         const uint32_t* p_tab = nullptr;               // entry of the block after the current one
@@ -786,21 +890,21 @@ k_decode_attn(DecodeParams P) {
                 const int lo = ws.lo[p_c];
                 p_left = ws.hi[p_c] - lo;
                 if (p_left == 0) continue;
-                p_tps = tps_of<G>(p_c);
+                p_tps = p_c == 0 ? Geo::tps(0, G) : p_c == 1 ? Geo::tps(1, G) : p_c == 2 ? Geo::tps(2, G) : Geo::tps(3, G);
                 p_rec = (uint32_t)pool_rec_bytes(p_c, G);
-                const int bt = (int)block_tiles(p_c, G);
-                const int blk = lo / bt;
-                p_in_block = bt - (lo - blk * bt);
-                p_phase = p_tps - lo % p_tps;          // tiles up to the next stage boundary
+                p_bt = (int)block_tiles(p_c, G);
+                const int blk = lo / p_bt, ib = lo - blk * p_bt;
+                p_cur.start(ib, p_tps, p_bt);
                 p_tab = ws.tab[p_c] + blk + 1;
-                p_ptr = P.store.arena + (size_t)p_tab[-1] * kBlockBytes + (size_t)(lo - blk * bt) * p_rec;
-                p_next_id = p_tab[0];
+                p_ptr = P.store.arena + (size_t)ws.id[p_c] * kBlockBytes + (size_t)ib * p_rec;
+                // (only a segment that goes on into the stream's next block asks for its id: a request that nobody
+                // waits for would still hold up the next request for the same register)
+                if (p_left > p_cur.to_block) p_next_id = p_tab[0];
             }
         };
         if (!failed) next_pool();
         auto issue_next = [&]() {
-            const int n = min(p_phase, p_left);
-            p_phase = p_tps;
+            const int n = p_cur.next(p_left);
             const uint32_t bytes = (uint32_t)n * p_rec;
             if (lane == 0) {
                 mbar_arrive_expect_tx(&ws.bars[pslot], bytes);
@@ -809,14 +913,13 @@ k_decode_attn(DecodeParams P) {
             if (++pslot == kStages) pslot = 0;
             p_ptr += bytes;
             p_left -= n;
-            p_in_block -= n;
+            const bool block_end = p_cur.advance(n, p_tps, p_bt);
             if (p_left == 0) {
                 next_pool();
-            } else if (p_in_block == 0) {              // on to the stream's next block
+            } else if (block_end) {                    // on to the stream's next block
                 p_ptr = P.store.arena + (size_t)p_next_id * kBlockBytes;
-                p_in_block = (int)block_tiles(p_c, G);
                 ++p_tab;
-                p_next_id = p_tab[0];
+                if (p_left > p_bt) p_next_id = p_tab[0];
             }
         };
         int in_flight = 0;
@@ -827,23 +930,38 @@ k_decode_attn(DecodeParams P) {
 #pragma unroll
         for (int i = 0; i < kHalfDim; ++i) acc[i] = 0.f;
 
+        // The reading side of the ring: wait for the chunk in slot cslot / hand the slot back and start the next copy.
+        auto chunk_wait = [&]() {
+            if (!mbar_wait(&ws.bars[cslot], (par_bits >> cslot) & 1u)) failed = true;
+            return !failed;
+        };
+        auto chunk_done = [&]() {
+            --in_flight;
+            __syncwarp();                              // every lane is done with the slot before it is refilled
+            if (p_left > 0) {
+                issue_next();
+                ++in_flight;
+            }
+            par_bits ^= 1u << cslot;
+            if (++cslot == kStages) cslot = 0;
+        };
+
         auto walk = [&](auto cls_tag, auto consumer) {
             constexpr int CLS = decltype(cls_tag)::value;
             using C = decltype(consumer);
+            constexpr int TPS = Geo::tps(CLS, G), BT = (int)block_tiles(CLS, G);
             int tile0 = ws.lo[CLS];
             const int hi = ws.hi[CLS];
             if (tile0 >= hi || failed) return;
             const uint32_t cnt = ws.cnt[CLS];
-            int phase = tiles_per_stage(CLS, G) - tile0 % tiles_per_stage(CLS, G);  // tiles up to the next stage boundary
+            ChunkCursor cur;
+            cur.start(tile0 % BT, TPS, BT);
             uint32_t qreg[kQRegs];
             C::enter(qi, qreg, acc);
             while (tile0 < hi) {
-                if (!mbar_wait(&ws.bars[cslot], parity)) {
-                    failed = true;
-                    break;
-                }
-                const int ntiles = min(phase, hi - tile0);
-                phase = tiles_per_stage(CLS, G);
+                if (!chunk_wait()) break;
+                const int ntiles = cur.next(hi - tile0);
+                cur.advance(ntiles, TPS, BT);
                 const uint8_t* buf = my_ring + (size_t)cslot * kStageBytes;
                 typename C::KIn kin = C::load_k(buf, half, t);
                 for (int i = 0; i < ntiles; ++i) {
@@ -854,25 +972,17 @@ k_decode_attn(DecodeParams P) {
                     kin = knext;
                 }
                 tile0 += ntiles;
-                --in_flight;
-                __syncwarp();                          // every lane is done with the slot before it is refilled
-                if (p_left > 0) {
-                    issue_next();
-                    ++in_flight;
-                }
-                if (++cslot == kStages) {
-                    cslot = 0;
-                    parity ^= 1u;
-                }
+                chunk_done();
             }
             C::leave(acc);
         };
         // The same walk for the fragment path, two tiles (A, B) per iteration: lane L = 4 g + q owns slot
-        // g + 8 (q & 1) of tile A (q < 2) or of tile B (q >= 2).  A stage with an odd number of tiles ends with
+        // g + 8 (q & 1) of tile A (q < 2) or of tile B (q >= 2).  A chunk with an odd number of tiles ends with
         // a pair whose B is absent: it points at A's record again and every one of its slots counts as empty.
         auto walk_frag = [&](auto cls_tag) {
             constexpr int CLS = decltype(cls_tag)::value;
             using C = FragRows<CLS>;
+            constexpr int TPS = Geo::tps(CLS, 1), BT = (int)block_tiles(CLS, 1);
             int tile0 = ws.lo[CLS];
             const int hi = ws.hi[CLS];
             if (tile0 >= hi || failed) return;
@@ -881,7 +991,8 @@ k_decode_attn(DecodeParams P) {
             const uint32_t my_slot = (uint32_t)((q >> 1) * kTileTokens + g + 8 * (q & 1));     // 0..15 in A, 16..31 in B
             const uint32_t dg = g < 3 ? (uint32_t)g : 3u;                            // byte 3 of a weight on the grid is zero
             const uint32_t sel = dg | ((4u + dg) << 4) | (dg << 8) | ((4u + dg) << 12);
-            int phase = tiles_per_stage(CLS, 1) - tile0 % tiles_per_stage(CLS, 1);
+            ChunkCursor cur;
+            cur.start(tile0 % BT, TPS, BT);
             uint32_t bkA[4], bkB[4];
             C::make_kb(ws.q, qi.fix_scale, g, q, bkA);
 #pragma unroll
@@ -904,12 +1015,9 @@ k_decode_attn(DecodeParams P) {
             ws.x[1][lane] = 0u;
             __syncwarp();
             while (tile0 < hi) {
-                if (!mbar_wait(&ws.bars[cslot], parity)) {
-                    failed = true;
-                    break;
-                }
-                const int ntiles = min(phase, hi - tile0);
-                phase = tiles_per_stage(CLS, 1);
+                if (!chunk_wait()) break;
+                const int ntiles = cur.next(hi - tile0);
+                cur.advance(ntiles, TPS, BT);
                 const uint8_t* buf = my_ring + (size_t)cslot * kStageBytes;
                 for (int i = 0; i < ntiles; i += 2) {
                     const bool has_b = i + 1 < ntiles;
@@ -933,16 +1041,7 @@ k_decode_attn(DecodeParams P) {
                     C::flush(va, st, q);
                     since_flush = 0;
                 }
-                --in_flight;
-                __syncwarp();                          // every lane is done with the slot before it is refilled
-                if (p_left > 0) {
-                    issue_next();
-                    ++in_flight;
-                }
-                if (++cslot == kStages) {
-                    cslot = 0;
-                    parity ^= 1u;
-                }
+                chunk_done();
             }
             C::v_part(vpA, vpB, ws.x[pp ^ 1u], q, sel, va);     // the last pair's products
             C::flush(va, st, q);
@@ -963,11 +1062,9 @@ k_decode_attn(DecodeParams P) {
             // Copies that were started but not consumed may still land in this warp's ring: give
             // each a bounded wait before the warp can retire, then report.
             for (int i = 1; i < in_flight; ++i) {
-                if (++cslot == kStages) {
-                    cslot = 0;
-                    parity ^= 1u;
-                }
-                mbar_wait(&ws.bars[cslot], parity);
+                par_bits ^= 1u << cslot;
+                if (++cslot == kStages) cslot = 0;
+                mbar_wait(&ws.bars[cslot], (par_bits >> cslot) & 1u);
             }
             in_flight = 0;
             if (lane == 0) atomicOr(P.store.flags, kFlagWaitTimeout);
@@ -1017,17 +1114,50 @@ k_decode_attn(DecodeParams P) {
             const float2 o2 = *reinterpret_cast<const float2*>(ws.o + 2 * lane);
             r2[0] += o2.x;
             r2[1] += o2.y;
-            __syncwarp();                              // ws.o is written again in the warp's next segment
+            __syncwarp();                              // ws.o is written again below or in the warp's next segment
         } else {
             r2[0] += b_w;
             r2[1] += b_w;
+        }
+        const float s2_w = STATS ? (G == 1 ? 1.0f : 0.5f) * warp_sum(st.s2) : 0.f;
+
+        if (Geo::kCtaMerge && P.cta_parts) {
+            // ---- all parts of the unit run in this CTA: partials and the arrival counter stay in shared memory
+            const uint32_t parts = P.cta_parts;
+            const int wf = warp - (int)(j % parts);    // the unit's first warp in this CTA holds its counter
+            reinterpret_cast<float2*>(ws.o)[lane] = make_float2(r2[0], r2[1]);
+            if (lane == 0) {
+                ws.ml = make_float2(st.m, l_w);
+                ws.s2 = s2_w;
+            }
+            __syncwarp();
+            uint32_t seen = 0;
+            if (lane == 0) {
+                __threadfence_block();                 // this warp's partial is visible to the CTA before it is counted
+                seen = atomicAdd(&scratch[wf].arrived, 1u);
+            }
+            seen = __shfl_sync(0xffffffffu, seen, 0);
+            if (seen + 1 == parts) {
+                __threadfence_block();
+                merge_partials<STATS>(
+                    P, u, row, qo, parts, lane,
+                    [&](uint32_t s) {
+                        const volatile float* pm = reinterpret_cast<const volatile float*>(&scratch[wf + s].ml);
+                        return make_float2(pm[0], pm[1]);
+                    },
+                    [&](uint32_t s) {
+                        const volatile float* po = scratch[wf + s].o + 2 * lane;
+                        return make_float2(po[0], po[1]);
+                    },
+                    [&](uint32_t s) { return *const_cast<const volatile float*>(&scratch[wf + s].s2); });
+            }
+            continue;                                  // (one segment per warp in this mode)
         }
         const uint32_t jf = decode_first_warp(u, P.units, P.gw);
         const size_t rec0 = (size_t)u * P.pslots;
         reinterpret_cast<float2*>(P.part_o + (rec0 + (j - jf)) * kHeadDim)[lane] = make_float2(r2[0], r2[1]);
         if (lane == 0) P.part_ml[rec0 + (j - jf)] = make_float2(st.m, l_w);
         if (STATS) {
-            const float s2_w = (G == 1 ? 1.0f : 0.5f) * warp_sum(st.s2);
             if (lane == 0) P.part_s2[rec0 + (j - jf)] = s2_w;
         }
 
@@ -1040,81 +1170,10 @@ k_decode_attn(DecodeParams P) {
         seen = __shfl_sync(0xffffffffu, seen, 0);
         if (seen + 1 == n_u) {
             __threadfence();                           // the other warps' partials, counted before ours
-            float M = kNegBig, L = 0.f, o0 = 0.f, o1 = 0.f;
-            if (n_u <= 32) {                           // the usual case: lane s weighs partial s; loads go out eight at a time
-                const float2 ml = lane < n_u ? __ldcg(&P.part_ml[rec0 + lane]) : make_float2(kNegBig, 0.f);
-                float2 o[8];
-#pragma unroll
-                for (uint32_t k = 0; k < 8; ++k)
-                    o[k] = k < n_u ? __ldcg(reinterpret_cast<const float2*>(P.part_o + (rec0 + k) * kHeadDim) + lane)
-                                   : make_float2(0.f, 0.f);
-                M = warp_max(ml.x);
-                const float f = fast_exp2(ml.x - M);
-                L = warp_sum(ml.y * f);
-#pragma unroll
-                for (uint32_t k = 0; k < 8; ++k) {
-                    const float fk = __shfl_sync(0xffffffffu, f, k);
-                    o0 = fmaf(o[k].x, fk, o0);
-                    o1 = fmaf(o[k].y, fk, o1);
-                }
-                for (uint32_t k0 = 8; k0 < n_u; k0 += 8) {
-#pragma unroll
-                    for (uint32_t k = 0; k < 8; ++k)
-                        o[k] = k0 + k < n_u ? __ldcg(reinterpret_cast<const float2*>(P.part_o + (rec0 + k0 + k) * kHeadDim) + lane)
-                                            : make_float2(0.f, 0.f);
-#pragma unroll
-                    for (uint32_t k = 0; k < 8; ++k) {
-                        const float fk = __shfl_sync(0xffffffffu, f, (k0 + k) & 31);
-                        o0 = fmaf(o[k].x, fk, o0);
-                        o1 = fmaf(o[k].y, fk, o1);
-                    }
-                }
-            } else {
-                for (uint32_t s0 = 0; s0 < n_u; s0 += 32) {        // the maximum, 32 partials at a time
-                    const uint32_t s = s0 + lane;
-                    M = fmaxf(M, s < n_u ? __ldcg(&P.part_ml[rec0 + s]).x : kNegBig);
-                }
-                M = warp_max(M);
-                for (uint32_t s0 = 0; s0 < n_u; s0 += 32) {
-                    const uint32_t s = s0 + lane;
-                    const float2 ml = s < n_u ? __ldcg(&P.part_ml[rec0 + s]) : make_float2(kNegBig, 0.f);
-                    const float f = fast_exp2(ml.x - M);
-                    L += warp_sum(ml.y * f);
-                    const uint32_t cnt = min(32u, n_u - s0);
-                    for (uint32_t k0 = 0; k0 < cnt; k0 += 8) {
-                        float2 o[8];
-#pragma unroll
-                        for (uint32_t k = 0; k < 8; ++k)
-                            o[k] = k0 + k < cnt ? __ldcg(reinterpret_cast<const float2*>(P.part_o + (rec0 + s0 + k0 + k) * kHeadDim) + lane)
-                                                : make_float2(0.f, 0.f);
-#pragma unroll
-                        for (uint32_t k = 0; k < 8; ++k) {
-                            const float fk = __shfl_sync(0xffffffffu, f, (k0 + k) & 31);
-                            o0 = fmaf(o[k].x, fk, o0);
-                            o1 = fmaf(o[k].y, fk, o1);
-                        }
-                    }
-                }
-            }
-            const float inv = L > 0.f ? 1.0f / L : 0.f;            // a sequence that holds no token yet gets zeros
-            reinterpret_cast<__half2*>(P.O + qo)[lane] = __floats2half2_rn(o0 * inv, o1 * inv);
-            if (STATS) {
-                // weights a_t = p_t / L sum to one over the n cached tokens: Var = sum a_t^2 / n - 1 / n^2
-                float S2 = 0.f;
-                for (uint32_t s0 = 0; s0 < n_u; s0 += 32) {
-                    const uint32_t s = s0 + lane;
-                    if (s < n_u) {
-                        const float f = fast_exp2(__ldcg(&P.part_ml[rec0 + s]).x - M);
-                        S2 = fmaf(__ldcg(&P.part_s2[rec0 + s]), f * f, S2);
-                    }
-                }
-                S2 = warp_sum(S2);
-                if (lane == 0) {
-                    const uint4 cnt = *reinterpret_cast<const uint4*>(P.counts + (size_t)row * 4);
-                    const float n = (float)(cnt.x + cnt.y + cnt.z + cnt.w);
-                    P.unit_var[u] = n > 0.f ? (S2 * inv * inv) / n - 1.0f / (n * n) : 0.f;
-                }
-            }
+            merge_partials<STATS>(
+                P, u, row, qo, n_u, lane, [&](uint32_t s) { return __ldcg(&P.part_ml[rec0 + s]); },
+                [&](uint32_t s) { return __ldcg(reinterpret_cast<const float2*>(P.part_o + (rec0 + s) * kHeadDim) + lane); },
+                [&](uint32_t s) { return __ldcg(&P.part_s2[rec0 + s]); });
             if (lane == 0) P.part_cnt[u] = 0;
         }
     }

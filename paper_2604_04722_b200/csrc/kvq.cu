@@ -350,23 +350,76 @@ constexpr int kMaxQueryRows = 8;       // query rows per sequence that one launc
 
 size_t max_partial_records(const kvq_ctx* c);
 
-// room: partial records the caller has scratch for (0: the handle's own).  Returns 0 if not even one part
-// per unit fits.
-uint32_t choose_warps(kvq_ctx* c, int len, uint64_t units, uint64_t room = 0) {
+// A launch plan: working warps, geometry, and (small geometry) parts per unit merged inside the CTA.
+struct DecodePlan {
+    uint32_t gw = 0;
+    bool small = false;
+    uint32_t cta_parts = 0;
+};
+// room: partial records the caller has scratch for (0: the handle's own).  gw == 0 if not even one part per unit
+// fits.  Launches of few warps take the small geometry (8 warps per CTA, one CTA per SM, deep rings): with 1, 2, 4
+// or 8 parts per unit the parts of a unit share a CTA and need no partial records at all.
+DecodePlan choose_plan(kvq_ctx* c, int len, uint64_t units, uint64_t room = 0) {
+    DecodePlan plan;
     if (room == 0) room = max_partial_records(c);
     auto fits = [&](uint64_t gw) { return units * (uint64_t)decode_pslots((uint32_t)units, (uint32_t)gw) <= room; };
-    if (!fits(units)) return 0;
-    if (c->splits_override > 0 && units * (uint64_t)(c->splits_override + 1) <= room)
-        return (uint32_t)(units * (uint64_t)c->splits_override);
-    const uint64_t tiles = units * (uint64_t)((len + kTileTokens - 1) / kTileTokens + (kNumPools - 1));
-    const uint64_t resident = (uint64_t)kDecodeWarps * kDecodeCtasPerSm * c->sm_count;
+    const uint64_t small_resident = (uint64_t)GeomSmall::kWarps * GeomSmall::kCtasPerSm * c->sm_count;
+    auto cta_mergeable = [&](uint64_t parts) { return parts == 1 || parts == 2 || parts == 4 || parts == 8; };
+    if (c->splits_override > 0) {
+        const uint64_t parts = (uint64_t)c->splits_override, gw = units * parts;
+        if (gw <= small_resident && cta_mergeable(parts)) {
+            plan.gw = (uint32_t)gw;
+            plan.small = true;
+            plan.cta_parts = (uint32_t)parts;
+            return plan;
+        }
+        if (units * (parts + 1) <= room) {
+            plan.gw = (uint32_t)gw;
+            plan.small = gw <= small_resident;
+            return plan;
+        }
+    }
+    const uint64_t tiles_per_unit = (uint64_t)((len + kTileTokens - 1) / kTileTokens + (kNumPools - 1));
+    const uint64_t tiles = units * tiles_per_unit;
+    const uint64_t resident = (uint64_t)GeomLarge::kWarps * GeomLarge::kCtasPerSm * c->sm_count;
+    if (!fits(units) && units > small_resident) return plan;
+    if (tiles / 4 <= resident) {
+        // A short cache is a chain of latencies, not a stream: a warp walks a tile in about kTileUs, parts merged
+        // inside their CTA cost about kCtaMergeUs, parts merged through global partial records about kGlobalMergeUs
+        // (measured on warps' own timestamps).  Take the cheaper of: 8 / 4 / 2 / 1 parts per unit in the small
+        // geometry, or as many parts as leave a warp four tiles, merged globally.
+        const double kTileUs = 0.3, kCtaMergeUs = 0.5, kGlobalMergeUs = 3.0;
+        double best_cost = 1e30;
+        for (uint64_t parts = 8; parts >= 1; parts /= 2) {
+            if (units * parts > small_resident) continue;
+            const double cost = kTileUs * (double)((tiles_per_unit + parts - 1) / parts) + kCtaMergeUs;
+            if (cost < best_cost) {
+                best_cost = cost;
+                plan.gw = (uint32_t)(units * parts);
+                plan.small = true;
+                plan.cta_parts = (uint32_t)parts;
+            }
+        }
+        uint64_t cap = tiles / 4 < 1 ? 1 : tiles / 4;
+        uint64_t gw = cap >= units ? cap / units * units : cap;
+        if (gw > 0 && !fits(gw)) gw = fits(units) ? (room / units - 1) * units : 0;
+        if (gw > 0) {
+            const double cost = kTileUs * (double)((tiles + gw - 1) / gw) + kGlobalMergeUs;
+            if (cost < best_cost) {
+                plan.gw = (uint32_t)gw;
+                plan.small = gw <= small_resident;
+                plan.cta_parts = 0;
+            }
+        }
+        return plan;
+    }
+    if (!fits(units)) return plan;
     uint64_t cap = tiles / 8;
-    if (tiles / 4 <= resident) cap = tiles / 4;        // a small cache is a latency chain: shorter parts, while all warps fit at once
-    if (cap < 1) cap = 1;
     if (cap <= resident) {
         uint64_t gw = cap >= units ? cap / units * units : cap;
         if (!fits(gw)) gw = (room / units - 1) * units;            // the most whole parts per unit that fit
-        return (uint32_t)gw;
+        plan.gw = (uint32_t)gw;
+        return plan;
     }
     // set-up, ring fill and the final reduction cost a warp about as much as fifteen tiles per part
     // (constants fitted to measured sweeps over the split count on four workload shapes)
@@ -389,13 +442,14 @@ uint32_t choose_warps(kvq_ctx* c, int len, uint64_t units, uint64_t room = 0) {
             best = units * s;
         }
     }
-    return (uint32_t)best;
+    plan.gw = (uint32_t)best;
+    return plan;
 }
 
 // Partial records a handle may need: explicit splits up to kMaxSplits, or a persistent launch.
 size_t max_partial_records(const kvq_ctx* c) {
     const size_t units = (size_t)c->batch * c->q_heads;
-    const size_t resident = (size_t)kDecodeWarps * kDecodeCtasPerSm * c->sm_count;
+    const size_t resident = (size_t)GeomLarge::kWarps * GeomLarge::kCtasPerSm * c->sm_count;
     const size_t by_splits = units * (kMaxSplits + 1);
     const size_t by_residency = resident + 2 * units * kMaxQueryRows;
     return by_splits > by_residency ? by_splits : by_residency;
@@ -403,7 +457,7 @@ size_t max_partial_records(const kvq_ctx* c) {
 
 // Fill the launch parameters of a decode call and queue split + merge on `st`.
 void fill_decode_params(kvq_ctx* c, int layer, const void* Q, void* O, float* part_o, float2* part_ml,
-                        uint32_t* part_cnt, uint32_t gw, DecodeParams& p) {
+                        uint32_t* part_cnt, const DecodePlan& plan, DecodeParams& p) {
     p.store = c->store;
     p.counts = counts_of(c, c->cur[layer], layer);
     p.Q = static_cast<const __half*>(Q);
@@ -418,14 +472,21 @@ void fill_decode_params(kvq_ctx* c, int layer, const void* Q, void* O, float* pa
     p.tq = p.t_total = 1;
     p.t0 = 0;
     p.units = (uint32_t)c->batch * (uint32_t)c->q_heads;
-    p.gw = gw;
-    p.pslots = decode_pslots(p.units, gw);
+    p.gw = plan.gw;
+    p.pslots = decode_pslots(p.units, plan.gw);
+    p.cta_parts = plan.cta_parts;
 }
 
+template <bool STATS, class Geo>
+void launch_decode_geo(const kvq_ctx* c, const DecodeParams& p, cudaStream_t st) {
+    const dim3 grid((p.gw + Geo::kWarps - 1) / Geo::kWarps);
+    if (c->groups == 1) launch_overlapped(k_decode_attn<STATS, 1, Geo>, grid, Geo::kThreads, Geo::kSmemBytes, st, p);
+    else launch_overlapped(k_decode_attn<STATS, 2, Geo>, grid, Geo::kThreads, Geo::kSmemBytes, st, p);
+}
 template <bool STATS>
-void launch_decode(const kvq_ctx* c, uint32_t grid, const DecodeParams& p, cudaStream_t st) {
-    if (c->groups == 1) launch_overlapped(k_decode_attn<STATS, 1>, dim3(grid), kDecodeThreads, kDecodeSmemBytes, st, p);
-    else launch_overlapped(k_decode_attn<STATS, 2>, dim3(grid), kDecodeThreads, kDecodeSmemBytes, st, p);
+void launch_decode(const kvq_ctx* c, const DecodePlan& plan, const DecodeParams& p, cudaStream_t st) {
+    if (plan.small) launch_decode_geo<STATS, GeomSmall>(c, p, st);
+    else launch_decode_geo<STATS, GeomLarge>(c, p, st);
 }
 
 int export_impl(kvq_ctx* c, int layer, int b0, int nb, int pos0, int n, uint8_t* bits, uint32_t* pool_slot,
@@ -610,8 +671,14 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
              dyn_smem(k_quant_pack<0, 2, KVQ_APPEND_TOKENS_PER_THREAD>, ring);
         ok = ok && dyn_smem(k_quant_pack<1, 1>, ring) && dyn_smem(k_quant_pack<1, 2>, ring);
         ok = ok && dyn_smem(k_quant_pack<2, 1>, ring + smem_max) && dyn_smem(k_quant_pack<2, 2>, ring + smem_max);
-        ok = ok && dyn_smem(k_decode_attn<false, 1>, (int)kDecodeSmemBytes) && dyn_smem(k_decode_attn<false, 2>, (int)kDecodeSmemBytes);
-        ok = ok && dyn_smem(k_decode_attn<true, 1>, (int)kDecodeSmemBytes) && dyn_smem(k_decode_attn<true, 2>, (int)kDecodeSmemBytes);
+        ok = ok && dyn_smem(k_decode_attn<false, 1, GeomLarge>, (int)GeomLarge::kSmemBytes) &&
+             dyn_smem(k_decode_attn<false, 2, GeomLarge>, (int)GeomLarge::kSmemBytes);
+        ok = ok && dyn_smem(k_decode_attn<true, 1, GeomLarge>, (int)GeomLarge::kSmemBytes) &&
+             dyn_smem(k_decode_attn<true, 2, GeomLarge>, (int)GeomLarge::kSmemBytes);
+        ok = ok && dyn_smem(k_decode_attn<false, 1, GeomSmall>, (int)GeomSmall::kSmemBytes) &&
+             dyn_smem(k_decode_attn<false, 2, GeomSmall>, (int)GeomSmall::kSmemBytes);
+        ok = ok && dyn_smem(k_decode_attn<true, 1, GeomSmall>, (int)GeomSmall::kSmemBytes) &&
+             dyn_smem(k_decode_attn<true, 2, GeomSmall>, (int)GeomSmall::kSmemBytes);
         ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     }
     if (!ok) {
@@ -700,12 +767,12 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
     DeviceGuard guard(c->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DecodeParams p{};
-    fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, choose_warps(c, c->len[layer], (uint64_t)c->batch * c->q_heads), p);
-    const unsigned grid = (p.gw + kDecodeWarps - 1) / kDecodeWarps;
+    const DecodePlan plan = choose_plan(c, c->len[layer], (uint64_t)c->batch * c->q_heads);
+    fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, plan, p);
     const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
     cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 2] : nullptr;
     if (rec) cudaEventRecord(ev[0], st);
-    launch_decode<false>(c, grid, p, st);
+    launch_decode<false>(c, plan, p, st);
     if (rec) {
         cudaEventRecord(ev[1], st);
         c->prof_calls += 1;
@@ -721,9 +788,9 @@ int kvq_decode_attn_var(kvq_ctx* c, int layer, const void* Q, void* O, float* va
     DeviceGuard guard(c->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DecodeParams p{};
-    fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt,
-                       choose_warps(c, c->len[layer], (uint64_t)c->batch * c->q_heads), p);
-    launch_decode<true>(c, (p.gw + kDecodeWarps - 1) / kDecodeWarps, p, st);
+    const DecodePlan plan = choose_plan(c, c->len[layer], (uint64_t)c->batch * c->q_heads);
+    fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, plan, p);
+    launch_decode<true>(c, plan, p, st);
     k_head_mean<<<c->batch, 32, 0, st>>>(c->unit_var, c->q_heads, var_out);
     c->launches += 2;
     KVQ_CUDA(c, cudaGetLastError());
@@ -768,14 +835,15 @@ int kvq_attend_last(kvq_ctx* c, int layer, const void* Q, void* O, int n_queries
                                                   d_len, (uint32_t)n_queries, (uint32_t)t0, (uint32_t)tq, c->vis);
         const uint64_t units = (uint64_t)c->batch * tq * c->q_heads;
         DecodeParams p{};
-        fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, choose_warps(c, c->len[layer], units), p);
+        const DecodePlan plan = choose_plan(c, c->len[layer], units);
+        fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, plan, p);
         p.counts = c->vis;
         p.tq = (uint32_t)tq;
         p.t_total = (uint32_t)n_queries;
         p.t0 = (uint32_t)t0;
         p.units = (uint32_t)units;
         p.pslots = decode_pslots(p.units, p.gw);
-        launch_decode<false>(c, (p.gw + kDecodeWarps - 1) / kDecodeWarps, p, st);
+        launch_decode<false>(c, plan, p, st);
         c->launches += 2;
     }
     KVQ_CUDA(c, cudaGetLastError());
@@ -803,8 +871,8 @@ int kvq_decode_attn_static(kvq_ctx* c, int layer, const void* Q, void* O, void* 
     const uint64_t units = (uint64_t)c->batch * c->q_heads;
     // an explicit split count is taken as given; the automatic plan is the best one that fits the array
     if (c->splits_override > 0 && units * (uint64_t)(c->splits_override + 1) > (uint64_t)KVQ_STATIC_MAX_PARTIALS) return KVQ_ERR_TOO_LARGE;
-    const uint32_t gw = choose_warps(c, c->len[layer], units, KVQ_STATIC_MAX_PARTIALS);
-    if (gw == 0) return KVQ_ERR_TOO_LARGE;
+    const DecodePlan plan = choose_plan(c, c->len[layer], units, KVQ_STATIC_MAX_PARTIALS);
+    if (plan.gw == 0) return KVQ_ERR_TOO_LARGE;
     DeviceGuard guard(c->device);
     float* base = nullptr;
     {
@@ -819,8 +887,8 @@ int kvq_decode_attn_static(kvq_ctx* c, int layer, const void* Q, void* O, void* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DecodeParams p{};
     fill_decode_params(c, layer, Q, O, base, reinterpret_cast<float2*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * kHeadDim),
-                       reinterpret_cast<uint32_t*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * (kHeadDim + 2)), gw, p);
-    launch_decode<false>(c, (p.gw + kDecodeWarps - 1) / kDecodeWarps, p, st);
+                       reinterpret_cast<uint32_t*>(base + (size_t)KVQ_STATIC_MAX_PARTIALS * (kHeadDim + 2)), plan, p);
+    launch_decode<false>(c, plan, p, st);
     c->launches += 1;
     KVQ_CUDA(c, cudaGetLastError());
     return KVQ_OK;
