@@ -1,0 +1,526 @@
+// Quantize-append (Q_b of Eq. 24, append of Eq. 4) for caches with one {scale, zero-point} pair per row, whose
+// code blocks are stored in the operand order of the decode kernel (the fragment layout of kvq_common.cuh).
+//
+// Ownership.  A warp quantizes one whole 16-slot tile of one (class, KV head) at a time and writes the record
+// with contiguous 8/16-byte stores straight from registers.  For that every tile must belong to exactly one
+// CTA although the tokens of a class do not stop at chunk borders: the CTA of a chunk owns the tiles of class k
+// whose FIRST slot one of the chunk's own tokens takes, and fetches the up to 15 tokens that complete its last
+// tile from the chunks that follow (a forward scan over the class bytes that the classify launch left behind).
+// Tokens at the start of a chunk that fall into a tile begun by an earlier chunk are left to that chunk.  Only
+// the tile that an EARLIER APPEND CALL left partly filled is special: the first chunk owns it and blends its
+// new slots into the words already stored (it is the only writer of the stream during the call).
+//
+// Lane mapping (lane L = 4 g + q, the reading warp's):
+//   K: lane (g, q) quantizes, of the rows of slots g and g + 8, the elements of the canonical words q, q + 4, ...
+//      that it will store (2-bit: one word of 16 elements, 4-bit: two words of 8, 8-bit: four words of 4);
+//      the row's minimum and maximum meet through two xor-shuffles inside the quad.
+//   V: lane (g, q) quantizes elements 4g .. 4g+3 and 32+4g .. 32+4g+3 of the rows of slots 4q .. 4q+3 (the
+//      bytes of its words); a row's minimum and maximum meet through three xor-shuffles over g.
+// The arithmetic per element is the row quantizer's (k_append.cuh): fl(fl(fl(x - mn) * inv) + 1.5 * 2^23), the
+// codes packed by adding shifted bit patterns.
+#pragma once
+#include "k_append.cuh"
+
+namespace kvq {
+
+// Input stage of a work item in shared memory: [tensor][slot 0..15][piece 0..7] 16-byte pieces, the piece index
+// xor-ed with a function of the slot so that every read pattern below (and the fp16 copy) is free of bank
+// conflicts: f(s) = 5 s0 ^ 2 s1 ^ 3 s2 ^ 4 s3 over the bits of s.
+__host__ __device__ constexpr int stage_swizzle(int s) {
+    return ((s & 1) ? 5 : 0) ^ ((s & 2) ? 2 : 0) ^ ((s & 4) ? 3 : 0) ^ ((s & 8) ? 4 : 0);
+}
+__device__ __forceinline__ int stage_piece_offset(int s, int p) { return ((s << 3) + (p ^ stage_swizzle(s))) << 4; }
+constexpr int kStageTensorBytes = kTileTokens * kHeadDim * 2;            // 2 KB: 16 rows of one tensor
+constexpr int kFragStageBytes = 2 * kStageTensorBytes;                   // K rows, then V rows
+constexpr size_t kFragRingBytes = (size_t)(kChunkTokens / 32) * kAppendDepth * kFragStageBytes;
+
+// 16-byte async copy that writes zeros when `live` is false (the source is not read then).
+__device__ __forceinline__ void cp_async16_or_zero(void* smem_dst, const void* gmem_src, bool live) {
+    const int n = live ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+                 "l"(gmem_src), "r"(n)
+                 : "memory");
+}
+
+// {scale fp16, reciprocal, minimum} of a row from its minimum and maximum (the row quantizer's set-up).
+struct RowScale {
+    uint32_t meta;                 // {scale, zero-point} fp16 bit patterns
+    float inv, mn;
+    bool tiny;                     // subnormal scale: the quotient may exceed the top code and is clamped
+};
+template <int CLS>
+__device__ __forceinline__ RowScale row_scale(float mn, float mx) {
+    constexpr float LEVELS = (float)((1 << pool_bits(CLS)) - 1);
+    if (mn == 0.0f) mn = 0.0f;                         // -0 is stored as +0
+    if (mx == 0.0f) mx = 0.0f;
+    const float s32 = __fdiv_rn(__fsub_rn(mx, mn), LEVELS);
+    const __half s16 = __float2half_rn(s32);
+    const float sf = __half2float(s16);
+    RowScale r;
+    r.inv = sf == 0.0f ? 0.0f : __frcp_rn(sf);
+    r.mn = mn;
+    r.meta = (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(__float2half_rn(mn)) << 16);
+    r.tiny = sf != 0.0f && sf < 6.103515625e-05f;
+    return r;
+}
+
+// (min, -max) of the 2 n fp16 values in h[0..n), as one half2: both halves then reduce with the same min.
+template <int N>
+__device__ __forceinline__ __half2 min_negmax(const __half2 (&h)[N]) {
+    __half2 mn2 = h[0], mx2 = h[0];
+#pragma unroll
+    for (int i = 1; i < N; ++i) {
+        mn2 = __hmin2(mn2, h[i]);
+        mx2 = __hmax2(mx2, h[i]);
+    }
+    const __half mn = __hmin(__low2half(mn2), __high2half(mn2)), mx = __hmax(__low2half(mx2), __high2half(mx2));
+    return __halves2half2(mn, __hneg(mx));
+}
+__device__ __forceinline__ __half2 shfl_min2(__half2 v, int lane_xor) {
+    uint32_t u = *reinterpret_cast<uint32_t*>(&v);
+    u = __shfl_xor_sync(0xffffffffu, u, lane_xor);
+    return __hmin2(v, *reinterpret_cast<__half2*>(&u));
+}
+
+// Code bit patterns of two values: 0x4B400000 + code each (see pack_codes in k_append.cuh).
+template <int CLS, bool CLAMP>
+__device__ __forceinline__ void code_pair(__half2 h, float mn, float inv, uint32_t& b0, uint32_t& b1) {
+    constexpr float LEVELS = (float)((1 << pool_bits(CLS)) - 1);
+    const float2 f = __half22float2(h);
+    float r0, r1;
+    if (CLAMP) {
+        r0 = __fadd_rn(fminf(__fmul_rn(__fsub_rn(f.x, mn), inv), LEVELS), kRoundMagic);
+        r1 = __fadd_rn(fminf(__fmul_rn(__fsub_rn(f.y, mn), inv), LEVELS), kRoundMagic);
+    } else {
+        quantize_pair(f.x, f.y, mn, inv, kRoundMagic, r0, r1);
+    }
+    b0 = __float_as_uint(r0);
+    b1 = __float_as_uint(r1);
+}
+
+// ---- K side of one tile.  stage: the 16 K rows (2 KB, swizzled).  Returns the lane's words of the K code block in
+// store order (see kfrag_word_offset) and, in lanes q < 2, the {scale, zero-point} word of slot g + 8 q.
+template <int CLS>
+struct FragK {
+    static constexpr int BITS = pool_bits(CLS), EPW = 32 / BITS, WT = 16 / EPW, NW = 2 * WT;     // words per token / per lane
+    // position of token i's word wsel in the lane's store vector
+    __device__ static constexpr int pos(int i, int wsel) { return CLS == 0 ? i : CLS == 1 ? wsel * 2 + i : 4 * (wsel >> 1) + (wsel & 1) * 2 + i; }
+
+    __device__ static __forceinline__ void load_token(const uint8_t* stage, int s, int q, __half2 (&h)[8]) {
+        if (CLS == 0) {                                // elements 16q .. 16q+15: pieces 2q, 2q+1
+            *reinterpret_cast<uint4*>(&h[0]) = *reinterpret_cast<const uint4*>(stage + stage_piece_offset(s, 2 * q));
+            *reinterpret_cast<uint4*>(&h[4]) = *reinterpret_cast<const uint4*>(stage + stage_piece_offset(s, 2 * q + 1));
+        } else if (CLS == 1) {                         // elements 8q .. 8q+7 and 32+8q ..: pieces q, 4+q
+            *reinterpret_cast<uint4*>(&h[0]) = *reinterpret_cast<const uint4*>(stage + stage_piece_offset(s, q));
+            *reinterpret_cast<uint4*>(&h[4]) = *reinterpret_cast<const uint4*>(stage + stage_piece_offset(s, 4 + q));
+        } else {                                       // elements 4q + 16 w .. +3: half q % 2 of piece 2w + q / 2
+#pragma unroll
+            for (int w = 0; w < 4; ++w)
+                *reinterpret_cast<uint2*>(&h[2 * w]) =
+                    *reinterpret_cast<const uint2*>(stage + stage_piece_offset(s, 2 * w + (q >> 1)) + 8 * (q & 1));
+        }
+    }
+    template <bool CLAMP>
+    __device__ static __forceinline__ void codes(const __half2 (&h)[8], float mn, float inv, int i, uint32_t (&kw)[NW]) {
+        uint32_t bias = 0;
+#pragma unroll
+        for (int e = 0; e < EPW; ++e) bias += 0x4B400000u << (BITS * e);
+#pragma unroll
+        for (int w = 0; w < WT; ++w) {
+            uint32_t acc = 0u - bias;
+#pragma unroll
+            for (int e = 0; e < EPW; e += 2) {
+                uint32_t b0, b1;
+                code_pair<CLS, CLAMP>(h[(w * EPW + e) / 2], mn, inv, b0, b1);
+                acc += b0 << (BITS * e);
+                acc += b1 << (BITS * (e + 1));
+            }
+            kw[pos(i, w)] = acc;
+        }
+    }
+    __device__ static __forceinline__ void tile(const uint8_t* stage, int g, int q, uint32_t (&kw)[NW], uint32_t& meta) {
+        __half2 h0[8], h1[8];
+        load_token(stage, g, q, h0);
+        load_token(stage, g + 8, q, h1);
+        __half2 m0 = min_negmax(h0), m1 = min_negmax(h1);
+        m0 = shfl_min2(shfl_min2(m0, 1), 2);
+        m1 = shfl_min2(shfl_min2(m1, 1), 2);
+        // even lanes set up slot g, odd lanes slot g + 8; the neighbour's result comes back through one exchange
+        const __half2 mine = (q & 1) ? m1 : m0;
+        const RowScale rs = row_scale<CLS>(__low2float(mine), -__high2float(mine));
+        meta = rs.meta;
+        const float inv_o = __shfl_xor_sync(0xffffffffu, rs.inv, 1), mn_o = __shfl_xor_sync(0xffffffffu, rs.mn, 1);
+        const float inv0 = (q & 1) ? inv_o : rs.inv, mn0 = (q & 1) ? mn_o : rs.mn;
+        const float inv1 = (q & 1) ? rs.inv : inv_o, mn1 = (q & 1) ? rs.mn : mn_o;
+        if (__any_sync(0xffffffffu, rs.tiny)) {        // rare: a subnormal scale somewhere in the tile
+            codes<true>(h0, mn0, inv0, 0, kw);
+            codes<true>(h1, mn1, inv1, 1, kw);
+        } else {
+            codes<false>(h0, mn0, inv0, 0, kw);
+            codes<false>(h1, mn1, inv1, 1, kw);
+        }
+    }
+};
+
+// ---- V side of one tile.  stage: the 16 V rows.  scratch: 16 float2 of shared memory owned by the warp.  Returns the
+// lane's words of the V code block in store order (see vfrag_byte_offset) and, in lanes g < 4, the {scale,
+// zero-point} word of slot 4 q + g.
+template <int CLS>
+struct FragV {
+    static constexpr int BITS = pool_bits(CLS), NW = 2 << CLS;
+    // word (in the lane's store vector) and bit position of the code of element e (0..3) of slot j, channel group i
+    __device__ static constexpr int pos(int i, int e) { return CLS == 0 ? i : CLS == 1 ? (e >> 1) * 2 + i : 4 * (e >> 1) + (e & 1) * 2 + i; }
+    __device__ static constexpr int shift(int j, int e) { return 8 * j + (CLS == 0 ? 2 * e : CLS == 1 ? 4 * (e & 1) : 0); }
+
+    template <bool CLAMP>
+    __device__ static __forceinline__ void codes(const __half2 (&h)[4][4], const float4 (&sc)[2], uint32_t (&vw)[NW]) {
+        uint32_t bias[NW];
+#pragma unroll
+        for (int w = 0; w < NW; ++w) bias[w] = 0;
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) bias[pos(i, e)] += 0x4B400000u << shift(j, e);
+#pragma unroll
+        for (int w = 0; w < NW; ++w) vw[w] = 0u - bias[w];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float inv = j == 0 ? sc[0].x : j == 1 ? sc[0].z : j == 2 ? sc[1].x : sc[1].z;
+            const float mn = j == 0 ? sc[0].y : j == 1 ? sc[0].w : j == 2 ? sc[1].y : sc[1].w;
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                for (int e = 0; e < 4; e += 2) {
+                    uint32_t b0, b1;
+                    code_pair<CLS, CLAMP>(h[j][2 * i + (e >> 1)], mn, inv, b0, b1);
+                    vw[pos(i, e)] += b0 << shift(j, e);
+                    vw[pos(i, e + 1)] += b1 << shift(j, e + 1);
+                }
+        }
+    }
+    __device__ static __forceinline__ void tile(const uint8_t* stage, float2* scratch, int g, int q, uint32_t (&vw)[NW],
+                                                uint32_t& meta) {
+        __half2 h[4][4];                               // [slot 4q + j][elements 4g..4g+3, then 32+4g..32+4g+3]
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int s = 4 * q + j;
+            *reinterpret_cast<uint2*>(&h[j][0]) = *reinterpret_cast<const uint2*>(stage + stage_piece_offset(s, g >> 1) + 8 * (g & 1));
+            *reinterpret_cast<uint2*>(&h[j][2]) =
+                *reinterpret_cast<const uint2*>(stage + stage_piece_offset(s, 4 + (g >> 1)) + 8 * (g & 1));
+        }
+        __half2 mm[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) mm[j] = shfl_min2(shfl_min2(shfl_min2(min_negmax(h[j]), 4), 8), 16);
+        // lanes g and g + 4 set up slot 4q + (g & 3); the results reach every lane through shared memory
+        const __half2 mine = (g & 3) == 0 ? mm[0] : (g & 3) == 1 ? mm[1] : (g & 3) == 2 ? mm[2] : mm[3];
+        const RowScale rs = row_scale<CLS>(__low2float(mine), -__high2float(mine));
+        meta = rs.meta;
+        __syncwarp();                                  // the scratch may still be read for the previous tile
+        if (g < 4) scratch[4 * q + g] = make_float2(rs.inv, rs.mn);
+        __syncwarp();
+        float4 sc[2];
+        sc[0] = *reinterpret_cast<const float4*>(scratch + 4 * q);
+        sc[1] = *reinterpret_cast<const float4*>(scratch + 4 * q + 2);
+        if (__any_sync(0xffffffffu, rs.tiny)) codes<true>(h, sc, vw);
+        else codes<false>(h, sc, vw);
+    }
+};
+
+// Store (or, for a tile that an earlier append call began, blend and store) a lane's words of one code block.
+// keep_k[i]: K block: the word of token i stays as it is.  keep_bytes: V block: mask of the bytes that stay.
+template <int NW>
+__device__ __forceinline__ void store_block(uint8_t* codes, int lane, const uint32_t (&w)[NW]) {
+    if (NW == 2) {
+        *reinterpret_cast<uint2*>(codes + lane * 8) = make_uint2(w[0], w[1]);
+    } else {
+#pragma unroll
+        for (int u = 0; u < NW / 4; ++u)
+            *reinterpret_cast<uint4*>(codes + (u * 32 + lane) * 16) = make_uint4(w[4 * u], w[4 * u + 1], w[4 * u + 2], w[4 * u + 3]);
+    }
+}
+template <int NW>
+__device__ __forceinline__ void load_block(const uint8_t* codes, int lane, uint32_t (&w)[NW]) {
+    if (NW == 2) {
+        const uint2 v = *reinterpret_cast<const uint2*>(codes + lane * 8);
+        w[0] = v.x; w[1] = v.y;
+    } else {
+#pragma unroll
+        for (int u = 0; u < NW / 4; ++u) {
+            const uint4 v = *reinterpret_cast<const uint4*>(codes + (u * 32 + lane) * 16);
+            w[4 * u] = v.x; w[4 * u + 1] = v.y; w[4 * u + 2] = v.z; w[4 * u + 3] = v.w;
+        }
+    }
+}
+
+// Work of a warp on one (tile, head) item whose rows sit in `stage`: quantize both tensors and store the record.
+// first_new: slots below it hold tokens of an earlier append call and stay as they are (0 for every other tile).
+template <int CLS>
+__device__ __forceinline__ void frag_item(const uint8_t* stage, float2* scratch, uint8_t* rec, int lane, int first_new) {
+    const int g = lane >> 2, q = lane & 3;
+    constexpr int NW = FragK<CLS>::NW;
+    uint32_t kw[NW], vw[NW], kmeta, vmeta;
+    FragK<CLS>::tile(stage, g, q, kw, kmeta);
+    FragV<CLS>::tile(stage + kStageTensorBytes, scratch, g, q, vw, vmeta);
+    uint8_t* vcodes = rec + pool_codes_bytes(CLS);
+    if (first_new > 0) {                               // warp-uniform, once per class and call at most
+        uint32_t ko[NW], vo[NW];
+        load_block<NW>(rec, lane, ko);
+        load_block<NW>(vcodes, lane, vo);
+        const int nb = min(max(first_new - 4 * q, 0), 4);              // bytes (slots 4q ..) of a V word that stay
+        const uint32_t keep = nb == 4 ? 0xffffffffu : ((1u << (8 * nb)) - 1u);
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+            const int i = CLS == 0 ? w : (w & 1);      // the token (g or g + 8) that K word w belongs to
+            if (g + 8 * i < first_new) kw[w] = ko[w];
+            vw[w] = (vw[w] & ~keep) | (vo[w] & keep);
+        }
+    }
+    store_block<NW>(rec, lane, kw);
+    store_block<NW>(vcodes, lane, vw);
+    if (q < 2 && g + 8 * q >= first_new) *reinterpret_cast<uint32_t*>(rec + meta_offset(CLS, 0, g + 8 * q)) = kmeta;
+    if (g < 4 && 4 * q + g >= first_new) *reinterpret_cast<uint32_t*>(rec + meta_offset(CLS, 1, 4 * q + g)) = vmeta;
+}
+
+// fp16 tile: the lane (half h, slot t) copies its 64 bytes of both rows (the unit layout of the fp16 pool).
+__device__ __forceinline__ void frag_item_fp16(const uint8_t* stage, uint8_t* rec, int lane, int first_new, uint32_t live_mask) {
+    const int half = lane >> 4, t = lane & 15;
+    if (t < first_new || !((live_mask >> t) & 1u)) return;
+    uint8_t* vcodes = rec + pool_codes_bytes(3);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        *reinterpret_cast<uint4*>(rec + unit_offset(3, half, u, t)) =
+            *reinterpret_cast<const uint4*>(stage + stage_piece_offset(t, 4 * half + u));
+        *reinterpret_cast<uint4*>(vcodes + unit_offset(3, half, u, t)) =
+            *reinterpret_cast<const uint4*>(stage + kStageTensorBytes + stage_piece_offset(t, 4 * half + u));
+    }
+}
+
+// The quantize-and-pack launch for caches with one scale group.  MODE as in k_quant_pack: 0 = classes from the
+// classify launch (several chunks per sequence), 1 = one chunk, classes from `bits`, 2 = one chunk, classes from
+// the controller.  grid = (nchunks, head_groups, batch), block = 256, dynamic smem = kFragRingBytes (+ controller).
+template <int MODE, int R = 1>
+__global__ void __launch_bounds__(kChunkTokens, KVQ_APPEND_MIN_CTAS)
+k_quant_pack_frag(AppendParams p) {
+    static_assert(MODE == 0 || R == 1, "single-chunk appends hold at most 256 tokens per sequence");
+    constexpr int CT = kChunkTokens * R;               // tokens per chunk
+    constexpr int NWARPS = kChunkTokens / 32;
+    extern __shared__ __align__(16) uint8_t dyn_smem[];   // [ring: warps x depth x 4 KB][controller block (MODE 2)]
+    float* sW = reinterpret_cast<float*>(dyn_smem + kFragRingBytes);
+    __shared__ uint32_t wtot[R][NWARPS][4];
+    __shared__ uint32_t base[4];
+    __shared__ uint16_t list[4][CT];                   // the chunk's tokens by class, in slot order
+    __shared__ uint32_t ext[4][kTileTokens];           // tokens of later chunks that complete the last owned tile (index in the call)
+    __shared__ uint32_t ext_n[4];
+    __shared__ float2 vscratch[NWARPS][kTileTokens];
+    const int chunk = blockIdx.x, hg = blockIdx.y, b = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_b = new_tokens_of(p, b);
+
+    // ---- classes of this thread's tokens (pass r: token r * 256 + thread of the chunk)
+    int c[R];
+    if (MODE == 2) {
+        controller_stage(sW, p.ctrl, p.hidden);
+        __syncthreads();
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int tok_i = chunk * CT + r * kChunkTokens + threadIdx.x;
+        const bool live = tok_i < n_b;
+        const size_t tok = (size_t)b * p.n_new + tok_i;
+        c[r] = -1;
+        if (MODE == 2) {
+            if (live) {
+                float4 f = reinterpret_cast<const float4*>(p.feats)[tok];
+                float lg[4];
+                c[r] = controller_decide_any(sW, p.hidden, f.x, f.y, f.z, f.w, lg);
+                if (p.bits_out && hg == 0) p.bits_out[tok] = (uint8_t)pool_bits(c[r]);
+            }
+        } else if (MODE == 1) {
+            if (live) c[r] = class_of_bits(p.bits[tok], p.store.flags);
+        } else {
+            if (live) c[r] = p.cls[tok];
+        }
+    }
+    // ---- fill of each pool before this chunk
+    if (warp == 0) {
+        uint4 h = make_uint4(0, 0, 0, 0);
+        if (MODE == 0) {
+            for (int cc = lane; cc < chunk; cc += 32) {
+                uint4 v = p.hist[(size_t)b * p.nchunks + cc];
+                h.x += v.x; h.y += v.y; h.z += v.z; h.w += v.w;
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                h.x += __shfl_xor_sync(0xffffffffu, h.x, d);
+                h.y += __shfl_xor_sync(0xffffffffu, h.y, d);
+                h.z += __shfl_xor_sync(0xffffffffu, h.z, d);
+                h.w += __shfl_xor_sync(0xffffffffu, h.w, d);
+            }
+        }
+        if (lane == 0) {
+            const uint32_t* ci = p.counts_in + (size_t)b * 4;
+            base[0] = ci[0] + h.x; base[1] = ci[1] + h.y; base[2] = ci[2] + h.z; base[3] = ci[3] + h.w;
+        }
+    }
+    // ---- rank inside the chunk: tokens of earlier passes, of earlier warps of the pass, of earlier lanes
+    uint32_t rank[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        rank[r] = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            uint32_t m = __ballot_sync(0xffffffffu, c[r] == k);
+            if (c[r] == k) rank[r] = __popc(m & ((1u << lane) - 1u));
+            if (lane == 0) wtot[r][warp][k] = __popc(m);
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        if (c[r] < 0) continue;
+        uint32_t before = rank[r];
+        for (int rr = 0; rr < r; ++rr)
+            for (int w = 0; w < NWARPS; ++w) before += wtot[rr][w][c[r]];
+        for (int w = 0; w < warp; ++w) before += wtot[r][w][c[r]];
+        const int in_chunk = r * kChunkTokens + threadIdx.x;
+        list[c[r]][before] = (uint16_t)in_chunk;
+        if (hg == 0)
+            p.store.index[((size_t)p.layer * p.store.batch + b) * p.store.max_ctx + first_pos_of(p, b) + chunk * CT + in_chunk] =
+                ((uint32_t)c[r] << 30) | (base[c[r]] + before);
+    }
+    uint32_t ncls[4];                                  // tokens of each class in this chunk
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        ncls[k] = 0;
+        for (int r = 0; r < R; ++r)
+            for (int w = 0; w < NWARPS; ++w) ncls[k] += wtot[r][w][k];
+    }
+    if (hg == 0 && chunk == p.nchunks - 1 && threadIdx.x < 4)
+        p.counts_out[(size_t)b * 4 + threadIdx.x] = base[threadIdx.x] + ncls[threadIdx.x];
+    const int h0 = hg * p.heads_per_group;
+    const int nh = min(p.heads_per_group, p.store.kv_heads - h0);
+    if (MODE != 0) {
+        // One chunk per sequence: this CTA is the only one that writes the streams of its heads, so it
+        // reserves the blocks they grow into itself (with several chunks the classify launch did it before).
+        if (warp < kNumPools) reserve_blocks(p.store, warp, p.layer, b, h0, nh, base[warp], base[warp] + ncls[warp], lane);
+    }
+
+    // ---- owned tiles of class k: first slot in [own0, base + n); the first chunk also owns the tile that an
+    //      earlier call left partly filled.  need[k]: tokens of later chunks that complete the last owned tile.
+    uint32_t first[4], pre[5], need[4];
+    pre[0] = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t own0 = chunk == 0 ? (base[k] & ~(uint32_t)(kTileTokens - 1)) : base[k];
+        const uint32_t t_first = (own0 + kTileTokens - 1) / kTileTokens, t_end = (base[k] + ncls[k] + kTileTokens - 1) / kTileTokens;
+        first[k] = t_first;
+        const uint32_t nt = t_end > t_first ? t_end - t_first : 0;
+        pre[k + 1] = pre[k] + nt;
+        need[k] = nt ? t_end * kTileTokens - (base[k] + ncls[k]) : 0;
+    }
+    if (MODE == 0 && warp < kNumPools) {               // warp k looks ahead for the class-k tokens that follow the chunk
+        const int k = warp;
+        const uint32_t want = need[k];
+        uint32_t found = 0;
+        for (int pos = (chunk + 1) * CT; found < want && pos < n_b; pos += 32) {
+            const int v = pos + lane < n_b ? (int)p.cls[(size_t)b * p.n_new + pos + lane] : -1;
+            const uint32_t m = __ballot_sync(0xffffffffu, v == k);
+            const uint32_t at = found + __popc(m & ((1u << lane) - 1u));
+            if (v == k && at < want) ext[k][at] = (uint32_t)(pos + lane);
+            found += __popc(m);
+        }
+        if (lane == 0) ext_n[k] = found < want ? found : want;
+    } else if (warp < kNumPools && lane == 0) {
+        ext_n[warp] = 0;
+    }
+    __syncthreads();
+
+    // ---- work items (owned tile tau, head hh), heads fastest, dealt round-robin to the warps.  The input rows of
+    // the next kAppendDepth items are kept in flight with 16-byte async copies into a per-warp ring: eight
+    // neighbouring lanes fetch one whole 128-byte row, slots without a token are filled with zeros.
+    struct Item {
+        int k;                                         // class, -1 = no more items
+        int first_new;                                 // slots below it belong to an earlier call
+        uint32_t live;                                 // bit s: slot s receives a token of this call
+        uint8_t* rec;
+    };
+    uint32_t tau = 0;
+    int hh = warp;
+    auto settle = [&]() {
+        while (hh >= nh) {
+            hh -= nh;
+            ++tau;
+        }
+    };
+    settle();
+    uint8_t* my_ring = dyn_smem + (size_t)warp * kAppendDepth * kFragStageBytes;
+    auto next_item = [&](int stage) {
+        Item it;
+        it.k = -1;
+        it.first_new = 0;
+        it.live = 0;
+        it.rec = nullptr;
+        if (tau < pre[4]) {
+            const int k = (tau >= pre[1]) + (tau >= pre[2]) + (tau >= pre[3]);
+            const uint32_t basek = k == 0 ? base[0] : k == 1 ? base[1] : k == 2 ? base[2] : base[3];
+            const uint32_t nk = (k == 0 ? ncls[0] : k == 1 ? ncls[1] : k == 2 ? ncls[2] : ncls[3]);
+            const uint32_t nke = nk + ext_n[k];
+            it.k = k;
+            const uint32_t tile = (k == 0 ? first[0] : k == 1 ? first[1] : k == 2 ? first[2] : first[3]) +
+                                  (tau - (k == 0 ? pre[0] : k == 1 ? pre[1] : k == 2 ? pre[2] : pre[3]));
+            const int r0 = (int)(tile * kTileTokens) - (int)basek;       // rank of the tile's slot 0 (negative: older slots)
+            it.first_new = r0 < 0 ? -r0 : 0;
+            const int h = h0 + hh;
+            it.rec = tile_ptr(p.store, k, stream_table(p.store, k, p.layer, b, h), tile, 1);
+            uint8_t* dst = my_ring + (size_t)stage * kFragStageBytes;
+            const int piece = lane & 7;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int s = (lane >> 3) + 4 * i;     // the slot whose row these eight lanes fetch
+                const int r = r0 + s;
+                const bool live = r >= 0 && (uint32_t)r < nke;
+                size_t tok_i = 0;
+                if (live) tok_i = (uint32_t)r < nk ? (size_t)chunk * CT + list[k][r] : (size_t)ext[k][(uint32_t)r - nk];
+                const size_t src = (((size_t)b * p.n_new + tok_i) * p.store.kv_heads + h) * kHeadDim;
+                const int off = stage_piece_offset(s, piece);
+                cp_async16_or_zero(dst + off, reinterpret_cast<const uint4*>(p.K + src) + piece, live);
+                cp_async16_or_zero(dst + kStageTensorBytes + off, reinterpret_cast<const uint4*>(p.V + src) + piece, live);
+            }
+            // slots that receive a token: ranks 0 .. nke-1 that fall into this tile
+            const int lo = r0 < 0 ? -r0 : 0, hi_ = min((int)kTileTokens, (int)nke - r0);
+            it.live = hi_ > lo ? (((1u << hi_) - 1u) & ~((1u << lo) - 1u)) : 0u;
+            hh += NWARPS;
+            settle();
+        }
+        cp_async_commit();                             // one group per call, possibly empty
+        return it;
+    };
+    Item items[kAppendDepth];
+#pragma unroll
+    for (int d = 0; d < kAppendDepth; ++d) items[d] = next_item(d);
+    int stage = 0;
+    while (items[0].k >= 0) {
+        cp_async_wait<kAppendDepth - 1>();             // this lane's copies of the oldest group have landed
+        __syncwarp();                                  // ... and so have the other lanes'
+        const Item cur = items[0];
+        const uint8_t* st = my_ring + (size_t)stage * kFragStageBytes;
+        if (cur.live != 0u) {                          // (a tile of an earlier call that this call adds nothing to)
+            switch (cur.k) {
+            case 0: frag_item<0>(st, vscratch[warp], cur.rec, lane, cur.first_new); break;
+            case 1: frag_item<1>(st, vscratch[warp], cur.rec, lane, cur.first_new); break;
+            case 2: frag_item<2>(st, vscratch[warp], cur.rec, lane, cur.first_new); break;
+            default: frag_item_fp16(st, cur.rec, lane, cur.first_new, cur.live); break;
+            }
+        }
+        __syncwarp();                                  // every lane has read the stage before it is refilled
+#pragma unroll
+        for (int d = 0; d + 1 < kAppendDepth; ++d) items[d] = items[d + 1];
+        items[kAppendDepth - 1] = next_item(stage);
+        if (++stage == kAppendDepth) stage = 0;
+    }
+    cp_async_wait<0>();
+}
+
+}  // namespace kvq

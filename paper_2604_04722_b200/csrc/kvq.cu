@@ -15,6 +15,7 @@
 #include "kvq_common.cuh"
 #include "k_controller.cuh"
 #include "k_append.cuh"
+#include "k_append_frag.cuh"
 #include "k_decode.cuh"
 #include "k_export.cuh"
 #include "k_features.cuh"
@@ -298,8 +299,8 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
         c->launches += 1;
     } else if (n_new <= kChunkTokens) {
         if (c->groups == 1) {
-            if (fused) k_quant_pack<2, 1><<<grid_q, kChunkTokens, kAppendRingBytes + smem, st>>>(p);
-            else k_quant_pack<1, 1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+            if (fused) k_quant_pack_frag<2><<<grid_q, kChunkTokens, kFragRingBytes + smem, st>>>(p);
+            else k_quant_pack_frag<1><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
         } else {
             if (fused) k_quant_pack<2, 2><<<grid_q, kChunkTokens, kAppendRingBytes + smem, st>>>(p);
             else k_quant_pack<1, 2><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
@@ -311,10 +312,10 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
         else k_classify<false><<<grid_c, kChunkTokens, 0, st>>>(p);
         k_reserve_blocks<<<c->batch, 128, 0, st>>>(p);
         if (p.tpt == 1) {
-            if (c->groups == 1) k_quant_pack<0, 1, 1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+            if (c->groups == 1) k_quant_pack_frag<0, 1><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
             else k_quant_pack<0, 2, 1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
         } else {
-            if (c->groups == 1) k_quant_pack<0, 1, KVQ_APPEND_TOKENS_PER_THREAD><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
+            if (c->groups == 1) k_quant_pack_frag<0, KVQ_APPEND_TOKENS_PER_THREAD><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
             else k_quant_pack<0, 2, KVQ_APPEND_TOKENS_PER_THREAD><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
         }
         c->launches += 3;
@@ -666,11 +667,12 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
         auto dyn_smem = [](auto kernel, int bytes) {
             return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
         };
-        ok = ok && dyn_smem(k_quant_pack<0, 1>, ring) && dyn_smem(k_quant_pack<0, 2>, ring);
-        ok = ok && dyn_smem(k_quant_pack<0, 1, KVQ_APPEND_TOKENS_PER_THREAD>, ring) &&
+        const int fring = (int)kFragRingBytes;
+        ok = ok && dyn_smem(k_quant_pack_frag<0, 1>, fring) && dyn_smem(k_quant_pack<0, 2>, ring);
+        ok = ok && dyn_smem(k_quant_pack_frag<0, KVQ_APPEND_TOKENS_PER_THREAD>, fring) &&
              dyn_smem(k_quant_pack<0, 2, KVQ_APPEND_TOKENS_PER_THREAD>, ring);
-        ok = ok && dyn_smem(k_quant_pack<1, 1>, ring) && dyn_smem(k_quant_pack<1, 2>, ring);
-        ok = ok && dyn_smem(k_quant_pack<2, 1>, ring + smem_max) && dyn_smem(k_quant_pack<2, 2>, ring + smem_max);
+        ok = ok && dyn_smem(k_quant_pack_frag<1>, fring) && dyn_smem(k_quant_pack<1, 2>, ring);
+        ok = ok && dyn_smem(k_quant_pack_frag<2>, fring + smem_max) && dyn_smem(k_quant_pack<2, 2>, ring + smem_max);
         ok = ok && dyn_smem(k_decode_attn<false, 1, GeomLarge>, (int)GeomLarge::kSmemBytes) &&
              dyn_smem(k_decode_attn<false, 2, GeomLarge>, (int)GeomLarge::kSmemBytes);
         ok = ok && dyn_smem(k_decode_attn<true, 1, GeomLarge>, (int)GeomLarge::kSmemBytes) &&
