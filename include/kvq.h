@@ -166,9 +166,11 @@ int kvq_append(kvq_ctx* ctx, int layer, const void* K, const void* V,
  * evaluated inside the kernels that quantize and pack (Eq. 24): feats is dev fp32
  * [batch][n_new][4].  bits_out_opt (dev uint8 [batch][n_new] or NULL) receives
  * the decisions.  Launches: one kernel for up to 256 new tokens per sequence (a
- * decode step included); a longer prefill runs three: the controller with a
- * class histogram per chunk of tokens, the reservation of arena blocks, and the
- * quantize-and-pack kernel, which reads the classes back from a scratch array.
+ * decode step included); a longer prefill runs two: the controller, which also
+ * counts the classes per chunk of tokens and reserves the arena blocks, and the
+ * quantize-and-pack kernel, which reads the classes (one byte per token) back
+ * from a scratch array because slots are handed out in position order across
+ * chunks.
  */
 int kvq_append_fused(kvq_ctx* ctx, int layer, const void* K, const void* V,
                      const float* feats, int n_new, uint8_t* bits_out_opt, void* stream);
@@ -182,7 +184,8 @@ int kvq_append_fused(kvq_ctx* ctx, int layer, const void* K, const void* V,
  * Afterwards the sequences of the layer differ in length: kvq_seq_lens reports them,
  * kvq_seq_len the longest, kvq_decode_attn attends for every sequence over what it holds
  * (a sequence that holds nothing gets a zero row), kvq_export_range and kvq_attend_last are
- * limited by the shortest.  Synchronizes the stream once (the lengths travel to the device).
+ * limited by the shortest.  Does not synchronize: host_lens is copied before the call returns (the caller may
+ * reuse it at once) and travels to the device behind the work already queued on `stream`.
  */
 int kvq_append_ragged(kvq_ctx* ctx, int layer, const void* K, const void* V, const uint8_t* bits,
                       const float* feats, int n_max, const int* host_lens, uint8_t* bits_out_opt,

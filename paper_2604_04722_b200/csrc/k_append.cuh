@@ -52,6 +52,7 @@ struct AppendParams {
     // n_new rows per sequence) and position of each sequence's first new token (nullptr: pos0 for all).
     const int* lens;
     const int* pos;
+    uint32_t* chunk_arrivals;          // [batch] classify CTAs of a sequence that have finished; zero between launches
 };
 
 __device__ __forceinline__ int new_tokens_of(const AppendParams& p, int b) { return p.lens ? p.lens[b] : p.n_new; }
@@ -67,7 +68,12 @@ __device__ __forceinline__ int class_of_bits(int bits, uint32_t* flags) {
     return c;
 }
 
-// Launch 1 (only when a sequence's new tokens span several chunks).
+__device__ __forceinline__ void reserve_blocks(const StoreView& s, int c, int layer, int b, int h0, int nh,
+                                               uint32_t n_old, uint32_t n_new, int lane);
+
+// Launch 1 (only when a sequence's new tokens span several chunks): class of every new token, a class histogram per
+// chunk, and -- by the CTA that finishes last for its sequence (an arrival counter, nobody waits) -- the arena blocks
+// that the sequence's streams grow into.
 template <bool FUSED>
 __global__ void __launch_bounds__(kChunkTokens)
 k_classify(AppendParams p) {
@@ -103,13 +109,31 @@ k_classify(AppendParams p) {
         for (int k = 0; k < 4; ++k) wtot[warp][k] = mine[k];
     }
     __syncthreads();
+    __shared__ uint32_t is_last;
     if (threadIdx.x == 0) {
         uint4 h = make_uint4(0, 0, 0, 0);
         for (int w = 0; w < kChunkTokens / 32; ++w) {
             h.x += wtot[w][0]; h.y += wtot[w][1]; h.z += wtot[w][2]; h.w += wtot[w][3];
         }
         p.hist[(size_t)b * p.nchunks + chunk] = h;
+        __threadfence();                               // the histogram is visible before this CTA is counted
+        is_last = atomicAdd(p.chunk_arrivals + b, 1u) + 1u == (uint32_t)p.nchunks;
     }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();                                   // the other chunks' histograms, counted before ours
+    if (warp < kNumPools) {                            // warp k reserves for class k
+        uint32_t add = 0;
+        for (int cc = lane; cc < p.nchunks; cc += 32) {
+            const uint4 v = __ldcg(p.hist + (size_t)b * p.nchunks + cc);
+            add += warp == 0 ? v.x : warp == 1 ? v.y : warp == 2 ? v.z : v.w;
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) add += __shfl_xor_sync(0xffffffffu, add, d);
+        const uint32_t n_old = p.counts_in[(size_t)b * 4 + warp];
+        reserve_blocks(p.store, warp, p.layer, b, 0, p.store.kv_heads, n_old, n_old + add, lane);
+    }
+    if (threadIdx.x == 0) p.chunk_arrivals[b] = 0;
 }
 
 constexpr float kRoundMagic = 12582912.0f;             // 1.5 * 2^23
@@ -294,22 +318,6 @@ __device__ __forceinline__ void reserve_blocks(const StoreView& s, int c, int la
     }
 }
 
-// Launch between k_classify and k_quant_pack<0> (several chunks per sequence): reserve the blocks every
-// stream of the layer grows into.  grid = batch, block = 128 (warp c handles class c).
-__global__ void __launch_bounds__(128)
-k_reserve_blocks(AppendParams p) {
-    const int b = blockIdx.x, c = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint32_t add = 0;
-    for (int cc = lane; cc < p.nchunks; cc += 32) {
-        const uint4 v = p.hist[(size_t)b * p.nchunks + cc];
-        add += c == 0 ? v.x : c == 1 ? v.y : c == 2 ? v.z : v.w;
-    }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) add += __shfl_xor_sync(0xffffffffu, add, d);
-    const uint32_t n_old = p.counts_in[(size_t)b * 4 + c];
-    reserve_blocks(p.store, c, p.layer, b, 0, p.store.kv_heads, n_old, n_old + add, lane);
-}
-
 // Launch 2.  MODE 0: classes come from k_classify (several chunks per sequence);
 // MODE 1: one chunk, classes from `bits`; MODE 2: one chunk, classes from the controller.
 // R: tokens per thread (= p.tpt): a chunk is 256 R tokens.  A 16-slot tile that a chunk only partly fills
@@ -417,7 +425,7 @@ k_quant_pack(AppendParams p) {
     const int nh = min(p.heads_per_group, p.store.kv_heads - h0);
     if (MODE != 0) {
         // One chunk per sequence: this CTA is the only one that writes the streams of its heads, so it
-        // reserves the blocks they grow into itself (with several chunks k_reserve_blocks did it before).
+        // reserves the blocks they grow into itself (with several chunks the classify launch did it before).
         if (warp < kNumPools) reserve_blocks(p.store, warp, p.layer, b, h0, nh, base[warp], base[warp] + ncls[warp], lane);
     }
     __syncthreads();
@@ -597,7 +605,7 @@ __device__ __forceinline__ void token_store(int c, const uint4 (&kraw)[4], const
 // One new token per sequence (a decode step): grid = (ceil(kv_heads / 16), batch), block = 32.
 // Lane l handles half-row l%2 of KV head 16*blockIdx.x + l/2.  Everything the warp needs (the K and V
 // rows, the pool fills, the features) is requested up front so the loads overlap the controller;
-// the decision is taken by the whole warp (FUSED, hidden width 32) or read from `bits`.
+// the decision is taken by the whole warp (FUSED, any hidden width) or read from `bits`.
 template <bool FUSED, int G>
 __global__ void __launch_bounds__(32)
 k_append_token(AppendParams p) {
@@ -631,7 +639,8 @@ k_append_token(AppendParams p) {
     int c;
     if (FUSED) {
         const float4 f = reinterpret_cast<const float4*>(p.feats)[b];
-        c = controller_decide_warp32(p.ctrl, f.x, f.y, f.z, f.w, lane);
+        c = p.hidden == 32 ? controller_decide_warp32(p.ctrl, f.x, f.y, f.z, f.w, lane)
+                           : controller_decide_warp(p.ctrl, p.hidden, f.x, f.y, f.z, f.w, lane);
     } else {
         c = class_of_bits(p.bits[b], p.store.flags);
     }

@@ -21,7 +21,16 @@
 #pragma once
 #include "k_append.cuh"
 
+#ifndef KVQ_APPEND_FRAG_MIN_CTAS
+#define KVQ_APPEND_FRAG_MIN_CTAS 2
+#endif
+#ifndef KVQ_APPEND_FRAG_DEPTH
+#define KVQ_APPEND_FRAG_DEPTH 2
+#endif
+
 namespace kvq {
+
+constexpr int kFragDepth = KVQ_APPEND_FRAG_DEPTH;      // items whose input rows are in flight per warp
 
 // Input stage of a work item in shared memory: [tensor][slot 0..15][piece 0..7] 16-byte pieces, the piece index
 // xor-ed with a function of the slot so that every read pattern below (and the fp16 copy) is free of bank
@@ -32,7 +41,7 @@ __host__ __device__ constexpr int stage_swizzle(int s) {
 __device__ __forceinline__ int stage_piece_offset(int s, int p) { return ((s << 3) + (p ^ stage_swizzle(s))) << 4; }
 constexpr int kStageTensorBytes = kTileTokens * kHeadDim * 2;            // 2 KB: 16 rows of one tensor
 constexpr int kFragStageBytes = 2 * kStageTensorBytes;                   // K rows, then V rows
-constexpr size_t kFragRingBytes = (size_t)(kChunkTokens / 32) * kAppendDepth * kFragStageBytes;
+constexpr size_t kFragRingBytes = (size_t)(kChunkTokens / 32) * kFragDepth * kFragStageBytes;
 
 // 16-byte async copy that writes zeros when `live` is false (the source is not read then).
 __device__ __forceinline__ void cp_async16_or_zero(void* smem_dst, const void* gmem_src, bool live) {
@@ -120,7 +129,6 @@ struct FragK {
                     *reinterpret_cast<const uint2*>(stage + stage_piece_offset(s, 2 * w + (q >> 1)) + 8 * (q & 1));
         }
     }
-    template <bool CLAMP>
     __device__ static __forceinline__ void codes(const __half2 (&h)[8], float mn, float inv, int i, uint32_t (&kw)[NW]) {
         uint32_t bias = 0;
 #pragma unroll
@@ -131,14 +139,16 @@ struct FragK {
 #pragma unroll
             for (int e = 0; e < EPW; e += 2) {
                 uint32_t b0, b1;
-                code_pair<CLS, CLAMP>(h[(w * EPW + e) / 2], mn, inv, b0, b1);
+                code_pair<CLS, false>(h[(w * EPW + e) / 2], mn, inv, b0, b1);
                 acc += b0 << (BITS * e);
                 acc += b1 << (BITS * (e + 1));
             }
             kw[pos(i, w)] = acc;
         }
     }
-    __device__ static __forceinline__ void tile(const uint8_t* stage, int g, int q, uint32_t (&kw)[NW], uint32_t& meta) {
+    // false: some row of the tile has a subnormal scale (its quotients need the clamp): the caller takes the
+    // compact general routine for the whole item instead.
+    __device__ static __forceinline__ bool tile(const uint8_t* stage, int g, int q, uint32_t (&kw)[NW], uint32_t& meta) {
         __half2 h0[8], h1[8];
         load_token(stage, g, q, h0);
         load_token(stage, g + 8, q, h1);
@@ -148,17 +158,12 @@ struct FragK {
         // even lanes set up slot g, odd lanes slot g + 8; the neighbour's result comes back through one exchange
         const __half2 mine = (q & 1) ? m1 : m0;
         const RowScale rs = row_scale<CLS>(__low2float(mine), -__high2float(mine));
+        if (__any_sync(0xffffffffu, rs.tiny)) return false;
         meta = rs.meta;
         const float inv_o = __shfl_xor_sync(0xffffffffu, rs.inv, 1), mn_o = __shfl_xor_sync(0xffffffffu, rs.mn, 1);
-        const float inv0 = (q & 1) ? inv_o : rs.inv, mn0 = (q & 1) ? mn_o : rs.mn;
-        const float inv1 = (q & 1) ? rs.inv : inv_o, mn1 = (q & 1) ? rs.mn : mn_o;
-        if (__any_sync(0xffffffffu, rs.tiny)) {        // rare: a subnormal scale somewhere in the tile
-            codes<true>(h0, mn0, inv0, 0, kw);
-            codes<true>(h1, mn1, inv1, 1, kw);
-        } else {
-            codes<false>(h0, mn0, inv0, 0, kw);
-            codes<false>(h1, mn1, inv1, 1, kw);
-        }
+        codes(h0, (q & 1) ? mn_o : rs.mn, (q & 1) ? inv_o : rs.inv, 0, kw);
+        codes(h1, (q & 1) ? rs.mn : mn_o, (q & 1) ? rs.inv : inv_o, 1, kw);
+        return true;
     }
 };
 
@@ -172,7 +177,6 @@ struct FragV {
     __device__ static constexpr int pos(int i, int e) { return CLS == 0 ? i : CLS == 1 ? (e >> 1) * 2 + i : 4 * (e >> 1) + (e & 1) * 2 + i; }
     __device__ static constexpr int shift(int j, int e) { return 8 * j + (CLS == 0 ? 2 * e : CLS == 1 ? 4 * (e & 1) : 0); }
 
-    template <bool CLAMP>
     __device__ static __forceinline__ void codes(const __half2 (&h)[4][4], const float4 (&sc)[2], uint32_t (&vw)[NW]) {
         uint32_t bias[NW];
 #pragma unroll
@@ -194,21 +198,21 @@ struct FragV {
 #pragma unroll
                 for (int e = 0; e < 4; e += 2) {
                     uint32_t b0, b1;
-                    code_pair<CLS, CLAMP>(h[j][2 * i + (e >> 1)], mn, inv, b0, b1);
+                    code_pair<CLS, false>(h[j][2 * i + (e >> 1)], mn, inv, b0, b1);
                     vw[pos(i, e)] += b0 << shift(j, e);
                     vw[pos(i, e + 1)] += b1 << shift(j, e + 1);
                 }
         }
     }
-    __device__ static __forceinline__ void tile(const uint8_t* stage, float2* scratch, int g, int q, uint32_t (&vw)[NW],
-                                                uint32_t& meta) {
+    // voff[j]: byte offset, inside the stage, of elements 4g .. 4g+3 of slot 4q + j (elements 32+4g .. sit 64 bytes
+    // further, xor-wise).  false: a subnormal scale in the tile (see FragK::tile).
+    __device__ static __forceinline__ bool tile(const uint8_t* stage, const int (&voff)[4], float2* scratch, int g, int q,
+                                                uint32_t (&vw)[NW], uint32_t& meta) {
         __half2 h[4][4];                               // [slot 4q + j][elements 4g..4g+3, then 32+4g..32+4g+3]
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int s = 4 * q + j;
-            *reinterpret_cast<uint2*>(&h[j][0]) = *reinterpret_cast<const uint2*>(stage + stage_piece_offset(s, g >> 1) + 8 * (g & 1));
-            *reinterpret_cast<uint2*>(&h[j][2]) =
-                *reinterpret_cast<const uint2*>(stage + stage_piece_offset(s, 4 + (g >> 1)) + 8 * (g & 1));
+            *reinterpret_cast<uint2*>(&h[j][0]) = *reinterpret_cast<const uint2*>(stage + voff[j]);
+            *reinterpret_cast<uint2*>(&h[j][2]) = *reinterpret_cast<const uint2*>(stage + (voff[j] ^ 64));
         }
         __half2 mm[4];
 #pragma unroll
@@ -216,6 +220,7 @@ struct FragV {
         // lanes g and g + 4 set up slot 4q + (g & 3); the results reach every lane through shared memory
         const __half2 mine = (g & 3) == 0 ? mm[0] : (g & 3) == 1 ? mm[1] : (g & 3) == 2 ? mm[2] : mm[3];
         const RowScale rs = row_scale<CLS>(__low2float(mine), -__high2float(mine));
+        if (__any_sync(0xffffffffu, rs.tiny)) return false;
         meta = rs.meta;
         __syncwarp();                                  // the scratch may still be read for the previous tile
         if (g < 4) scratch[4 * q + g] = make_float2(rs.inv, rs.mn);
@@ -223,8 +228,8 @@ struct FragV {
         float4 sc[2];
         sc[0] = *reinterpret_cast<const float4*>(scratch + 4 * q);
         sc[1] = *reinterpret_cast<const float4*>(scratch + 4 * q + 2);
-        if (__any_sync(0xffffffffu, rs.tiny)) codes<true>(h, sc, vw);
-        else codes<false>(h, sc, vw);
+        codes(h, sc, vw);
+        return true;
     }
 };
 
@@ -256,31 +261,94 @@ __device__ __forceinline__ void load_block(const uint8_t* codes, int lane, uint3
 
 // Work of a warp on one (tile, head) item whose rows sit in `stage`: quantize both tensors and store the record.
 // first_new: slots below it hold tokens of an earlier append call and stay as they are (0 for every other tile).
+// Returns false if a row of the tile needs the clamp (subnormal scale): the caller then runs general_item, which
+// rewrites whatever this routine has stored already with the same values.
 template <int CLS>
-__device__ __forceinline__ void frag_item(const uint8_t* stage, float2* scratch, uint8_t* rec, int lane, int first_new) {
+__device__ __forceinline__ bool frag_item(const uint8_t* stage, const int (&voff)[4], float2* scratch, uint8_t* rec, int lane,
+                                          int first_new) {
     const int g = lane >> 2, q = lane & 3;
     constexpr int NW = FragK<CLS>::NW;
-    uint32_t kw[NW], vw[NW], kmeta, vmeta;
-    FragK<CLS>::tile(stage, g, q, kw, kmeta);
-    FragV<CLS>::tile(stage + kStageTensorBytes, scratch, g, q, vw, vmeta);
     uint8_t* vcodes = rec + pool_codes_bytes(CLS);
-    if (first_new > 0) {                               // warp-uniform, once per class and call at most
-        uint32_t ko[NW], vo[NW];
-        load_block<NW>(rec, lane, ko);
-        load_block<NW>(vcodes, lane, vo);
-        const int nb = min(max(first_new - 4 * q, 0), 4);              // bytes (slots 4q ..) of a V word that stay
-        const uint32_t keep = nb == 4 ? 0xffffffffu : ((1u << (8 * nb)) - 1u);
+    {
+        uint32_t kw[NW], kmeta;
+        if (!FragK<CLS>::tile(stage, g, q, kw, kmeta)) return false;
+        if (first_new > 0) {                           // warp-uniform, once per class and call at most
+            uint32_t ko[NW];
+            load_block<NW>(rec, lane, ko);
 #pragma unroll
-        for (int w = 0; w < NW; ++w) {
-            const int i = CLS == 0 ? w : (w & 1);      // the token (g or g + 8) that K word w belongs to
-            if (g + 8 * i < first_new) kw[w] = ko[w];
-            vw[w] = (vw[w] & ~keep) | (vo[w] & keep);
+            for (int w = 0; w < NW; ++w)
+                if (g + 8 * (w & 1) < first_new) kw[w] = ko[w];       // K word w belongs to slot g (even w) or g + 8
         }
+        store_block<NW>(rec, lane, kw);
+        if (q < 2 && g + 8 * q >= first_new) *reinterpret_cast<uint32_t*>(rec + meta_offset(CLS, 0, g + 8 * q)) = kmeta;
     }
-    store_block<NW>(rec, lane, kw);
-    store_block<NW>(vcodes, lane, vw);
-    if (q < 2 && g + 8 * q >= first_new) *reinterpret_cast<uint32_t*>(rec + meta_offset(CLS, 0, g + 8 * q)) = kmeta;
-    if (g < 4 && 4 * q + g >= first_new) *reinterpret_cast<uint32_t*>(rec + meta_offset(CLS, 1, 4 * q + g)) = vmeta;
+    {
+        uint32_t vw[NW], vmeta;
+        if (!FragV<CLS>::tile(stage + kStageTensorBytes, voff, scratch, g, q, vw, vmeta)) return false;
+        if (first_new > 0) {
+            uint32_t vo[NW];
+            load_block<NW>(vcodes, lane, vo);
+            const int nb = min(max(first_new - 4 * q, 0), 4);          // bytes (slots 4q ..) of a V word that stay
+            const uint32_t keep = nb == 4 ? 0xffffffffu : ((1u << (8 * nb)) - 1u);
+#pragma unroll
+            for (int w = 0; w < NW; ++w) vw[w] = (vw[w] & ~keep) | (vo[w] & keep);
+        }
+        store_block<NW>(vcodes, lane, vw);
+        if (g < 4 && 4 * q + g >= first_new) *reinterpret_cast<uint32_t*>(rec + meta_offset(CLS, 1, 4 * q + g)) = vmeta;
+    }
+    return true;
+}
+
+// The general routine for one item: any class < 3, clamp included, every slot >= first_new written code word by
+// code word (K) and byte by byte (V).  Compact on purpose (loops are not unrolled): it runs only for tiles that
+// hold a row whose scale is a subnormal fp16.  Lane (half h, slot t) takes the half-row of 32 elements.
+__device__ __noinline__ void general_item(const uint8_t* stage, uint8_t* rec, int cls, int lane, int first_new) {
+    const int half = lane >> 4, t = lane & 15;
+    const int bits = pool_bits(cls), epw = 32 / bits;
+    const float levels = (float)((1 << bits) - 1);
+#pragma unroll 1
+    for (int tensor = 0; tensor < 2; ++tensor) {
+        const uint8_t* rows = stage + tensor * kStageTensorBytes;
+        uint8_t* codes = rec + tensor * pool_codes_bytes(cls);
+        float mn = INFINITY, mx = -INFINITY;
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i) {
+            const int e = 32 * half + i;
+            const float x = __half2float(*reinterpret_cast<const __half*>(rows + stage_piece_offset(t, e >> 3) + 2 * (e & 7)));
+            mn = fminf(mn, x);
+            mx = fmaxf(mx, x);
+        }
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 16));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+        if (mn == 0.0f) mn = 0.0f;
+        if (mx == 0.0f) mx = 0.0f;
+        const float s32 = __fdiv_rn(__fsub_rn(mx, mn), levels);
+        const __half s16 = __float2half_rn(s32);
+        const float sf = __half2float(s16);
+        const float inv = sf == 0.0f ? 0.0f : __frcp_rn(sf);
+        if (t < first_new) continue;                   // (after the shuffles: every lane takes part in them)
+        uint32_t word = 0;
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i) {
+            const int e = 32 * half + i;
+            const float x = __half2float(*reinterpret_cast<const __half*>(rows + stage_piece_offset(t, e >> 3) + 2 * (e & 7)));
+            const float v = fminf(__fmul_rn(__fsub_rn(x, mn), inv), levels);
+            const uint32_t code = __float_as_uint(__fadd_rn(v, kRoundMagic)) - 0x4B400000u;
+            word |= code << (bits * (e % epw));
+            if ((e + 1) % epw == 0) {                  // a canonical 32-bit word is complete
+                const int wq = e / epw;
+                if (tensor == 0) {
+                    *reinterpret_cast<uint32_t*>(codes + kfrag_word_offset(cls, t, wq)) = word;
+                } else {
+                    for (int b = 0; b < 4; ++b) codes[vfrag_byte_offset(cls, t, 4 * wq + b)] = (uint8_t)(word >> (8 * b));
+                }
+                word = 0;
+            }
+        }
+        if (half == 0)
+            *reinterpret_cast<uint32_t*>(rec + meta_offset(cls, tensor, t)) =
+                (uint32_t)__half_as_ushort(s16) | ((uint32_t)__half_as_ushort(__float2half_rn(mn)) << 16);
+    }
 }
 
 // fp16 tile: the lane (half h, slot t) copies its 64 bytes of both rows (the unit layout of the fp16 pool).
@@ -301,7 +369,7 @@ __device__ __forceinline__ void frag_item_fp16(const uint8_t* stage, uint8_t* re
 // classify launch (several chunks per sequence), 1 = one chunk, classes from `bits`, 2 = one chunk, classes from
 // the controller.  grid = (nchunks, head_groups, batch), block = 256, dynamic smem = kFragRingBytes (+ controller).
 template <int MODE, int R = 1>
-__global__ void __launch_bounds__(kChunkTokens, KVQ_APPEND_MIN_CTAS)
+__global__ void __launch_bounds__(kChunkTokens, KVQ_APPEND_FRAG_MIN_CTAS)
 k_quant_pack_frag(AppendParams p) {
     static_assert(MODE == 0 || R == 1, "single-chunk appends hold at most 256 tokens per sequence");
     constexpr int CT = kChunkTokens * R;               // tokens per chunk
@@ -438,7 +506,7 @@ k_quant_pack_frag(AppendParams p) {
     __syncthreads();
 
     // ---- work items (owned tile tau, head hh), heads fastest, dealt round-robin to the warps.  The input rows of
-    // the next kAppendDepth items are kept in flight with 16-byte async copies into a per-warp ring: eight
+    // the next kFragDepth items are kept in flight with 16-byte async copies into a per-warp ring: eight
     // neighbouring lanes fetch one whole 128-byte row, slots without a token are filled with zeros.
     struct Item {
         int k;                                         // class, -1 = no more items
@@ -455,7 +523,10 @@ k_quant_pack_frag(AppendParams p) {
         }
     };
     settle();
-    uint8_t* my_ring = dyn_smem + (size_t)warp * kAppendDepth * kFragStageBytes;
+    uint8_t* my_ring = dyn_smem + (size_t)warp * kFragDepth * kFragStageBytes;
+    int voff[4];                                       // where this lane's V elements of slots 4q .. 4q+3 sit in a stage
+#pragma unroll
+    for (int j = 0; j < 4; ++j) voff[j] = stage_piece_offset(4 * (lane & 3) + j, lane >> 3) + 8 * ((lane >> 2) & 1);
     auto next_item = [&](int stage) {
         Item it;
         it.k = -1;
@@ -497,28 +568,30 @@ k_quant_pack_frag(AppendParams p) {
         cp_async_commit();                             // one group per call, possibly empty
         return it;
     };
-    Item items[kAppendDepth];
+    Item items[kFragDepth];
 #pragma unroll
-    for (int d = 0; d < kAppendDepth; ++d) items[d] = next_item(d);
+    for (int d = 0; d < kFragDepth; ++d) items[d] = next_item(d);
     int stage = 0;
     while (items[0].k >= 0) {
-        cp_async_wait<kAppendDepth - 1>();             // this lane's copies of the oldest group have landed
+        cp_async_wait<kFragDepth - 1>();             // this lane's copies of the oldest group have landed
         __syncwarp();                                  // ... and so have the other lanes'
         const Item cur = items[0];
         const uint8_t* st = my_ring + (size_t)stage * kFragStageBytes;
         if (cur.live != 0u) {                          // (a tile of an earlier call that this call adds nothing to)
+            bool done = true;
             switch (cur.k) {
-            case 0: frag_item<0>(st, vscratch[warp], cur.rec, lane, cur.first_new); break;
-            case 1: frag_item<1>(st, vscratch[warp], cur.rec, lane, cur.first_new); break;
-            case 2: frag_item<2>(st, vscratch[warp], cur.rec, lane, cur.first_new); break;
+            case 0: done = frag_item<0>(st, voff, vscratch[warp], cur.rec, lane, cur.first_new); break;
+            case 1: done = frag_item<1>(st, voff, vscratch[warp], cur.rec, lane, cur.first_new); break;
+            case 2: done = frag_item<2>(st, voff, vscratch[warp], cur.rec, lane, cur.first_new); break;
             default: frag_item_fp16(st, cur.rec, lane, cur.first_new, cur.live); break;
             }
+            if (!done) general_item(st, cur.rec, cur.k, lane, cur.first_new);
         }
         __syncwarp();                                  // every lane has read the stage before it is refilled
 #pragma unroll
-        for (int d = 0; d + 1 < kAppendDepth; ++d) items[d] = items[d + 1];
-        items[kAppendDepth - 1] = next_item(stage);
-        if (++stage == kAppendDepth) stage = 0;
+        for (int d = 0; d + 1 < kFragDepth; ++d) items[d] = items[d + 1];
+        items[kFragDepth - 1] = next_item(stage);
+        if (++stage == kFragDepth) stage = 0;
     }
     cp_async_wait<0>();
 }

@@ -122,6 +122,85 @@ __device__ __forceinline__ int controller_decide_warp32(const float* __restrict_
     return cls;
 }
 
+// The same for any hidden width H <= kMaxHidden (the paper's 128 included): lane l owns the hidden units l, l + 32,
+// l + 64, l + 96.  Rows of W2 are streamed from global memory four inputs at a time while the first-layer outputs
+// come round by shuffle; every sum still runs in ascending input order with separately rounded products and sums.
+__device__ __forceinline__ int controller_decide_warp(const float* __restrict__ gW, int H, float x0, float x1, float x2,
+                                                      float x3, int lane) {
+    constexpr int M = kMaxHidden / 32;
+    const float* W1 = gW;
+    const float* b1 = W1 + 4 * H;
+    const float* W2 = b1 + H;
+    const float* b2 = W2 + H * H;
+    const float* W3 = b2 + H;
+    const float* b3 = W3 + 4 * H;
+    float h1[M], acc[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+        const int j = lane + 32 * m;
+        h1[m] = 0.0f;
+        acc[m] = 0.0f;
+        if (j < H) {
+            float a = __ldg(b1 + j);
+            a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 0), x0));
+            a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 1), x1));
+            a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 2), x2));
+            a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 3), x3));
+            h1[m] = a > 0.0f ? a : 0.0f;
+            acc[m] = __ldg(b2 + j);
+        }
+    }
+    const bool vec = (H & 3) == 0;                     // rows of W2 are then 16-byte aligned
+    for (int i0 = 0; i0 < H; i0 += 4) {
+        float w[M][4];
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            const int j = lane + 32 * m;
+            w[m][0] = w[m][1] = w[m][2] = w[m][3] = 0.0f;
+            if (j < H) {
+                if (vec) {
+                    const float4 v = __ldg(reinterpret_cast<const float4*>(W2 + (size_t)j * H + i0));
+                    w[m][0] = v.x; w[m][1] = v.y; w[m][2] = v.z; w[m][3] = v.w;
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (i0 + k < H) w[m][k] = __ldg(W2 + (size_t)j * H + i0 + k);
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int i = i0 + k;                      // warp-uniform
+            if (i >= H) break;
+            float src = h1[0];
+#pragma unroll
+            for (int m = 1; m < M; ++m) src = (i >> 5) == m ? h1[m] : src;
+            const float v = __shfl_sync(0xffffffffu, src, i & 31);
+#pragma unroll
+            for (int m = 0; m < M; ++m) acc[m] = __fadd_rn(acc[m], __fmul_rn(w[m][k], v));
+        }
+    }
+    float h2[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) h2[m] = acc[m] > 0.0f ? acc[m] : 0.0f;
+    float o = __ldg(b3 + (lane & 3));                  // lanes 0..3 hold the four logits (the others mirror them)
+    for (int j = 0; j < H; ++j) {
+        float src = h2[0];
+#pragma unroll
+        for (int m = 1; m < M; ++m) src = (j >> 5) == m ? h2[m] : src;
+        o = __fadd_rn(o, __fmul_rn(__ldg(W3 + (lane & 3) * H + j), __shfl_sync(0xffffffffu, src, j & 31)));
+    }
+    const float o0 = __shfl_sync(0xffffffffu, o, 0), o1 = __shfl_sync(0xffffffffu, o, 1);
+    const float o2 = __shfl_sync(0xffffffffu, o, 2), o3 = __shfl_sync(0xffffffffu, o, 3);
+    if (o0 != o0 || o1 != o1 || o2 != o2 || o3 != o3) return 3;
+    int cls = 0;
+    float best = o0;
+    if (o1 > best) { best = o1; cls = 1; }
+    if (o2 > best) { best = o2; cls = 2; }
+    if (o3 > best) { best = o3; cls = 3; }
+    return cls;
+}
+
 // kvq_select_bits: one thread per token.
 __global__ void __launch_bounds__(128)
 k_select_bits(const float* __restrict__ feats, int n, const float* __restrict__ gW, int H,

@@ -41,10 +41,18 @@ struct kvq_ctx {
     std::vector<int> len;                // host mirror: tokens of the longest sequence, per layer
     std::vector<int> lens;               // host mirror: tokens per (layer, sequence)
     std::vector<char> ragged;            // per layer: sequences differ in length
-    int* d_lens = nullptr;               // device scratch [3][batch]: this call's new tokens, first positions, lengths
+    // Per-sequence lengths of ragged calls travel through a small ring of page-locked host slots and matching
+    // device slots: one asynchronous copy per call, no synchronisation of the caller's stream.  A slot is reused
+    // only after the event recorded behind its last copy has completed (checked on the host).
+    static constexpr int kLenSlots = 8;
+    int* d_lens = nullptr;               // device [kLenSlots][3][batch]: a call's new tokens, first positions, lengths
+    int* h_lens = nullptr;               // page-locked host mirror of the same shape
+    cudaEvent_t len_ev[kLenSlots] = {};
+    int len_slot = 0;
     std::vector<int> cur;                // which counts buffer is current, per layer
     uint8_t* cls = nullptr;              // append scratch [batch][max_ctx]
     uint4* hist = nullptr;               // append scratch [batch][max chunks]
+    uint32_t* chunk_arrivals = nullptr;  // append scratch [batch], zero between launches
     float* ctrl = nullptr;               // controller parameter block
     int hidden = 0;
     float* part_o = nullptr;             // decode scratch [units][partial slots][64]
@@ -164,6 +172,12 @@ void launch_overlapped(void (*kernel)(Params), dim3 grid, unsigned block, size_t
 void free_all(kvq_ctx* c) {
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     c->prof_ev.clear();
+    for (cudaEvent_t& e : c->len_ev) {
+        if (e) cudaEventDestroy(e);
+        e = nullptr;
+    }
+    if (c->h_lens) cudaFreeHost(c->h_lens);
+    c->h_lens = nullptr;
     if (c->mem_mode != 0) return;                      // the buffers belong to the caller's workspace (or do not exist)
     cudaFree(c->arena);
     cudaFree(c->table);
@@ -172,6 +186,7 @@ void free_all(kvq_ctx* c) {
     cudaFree(c->counts);
     cudaFree(c->cls);
     cudaFree(c->hist);
+    cudaFree(c->chunk_arrivals);
     cudaFree(c->ctrl);
     cudaFree(c->part_o);
     cudaFree(c->part_ml);
@@ -202,6 +217,18 @@ const void* device_view(const void* p) {
     }
     if (a.type != cudaMemoryTypeHost || !a.devicePointer || !aligned16(a.devicePointer)) return nullptr;
     return a.devicePointer;
+}
+
+// The next slot of the lengths ring: host and device addresses.  Waits (on the host, for an event) only if the slot's
+// previous copy, kLenSlots ragged calls ago, has not run yet.
+int claim_len_slot(kvq_ctx* c, int** host, int** dev) {
+    const int s = c->len_slot;
+    c->len_slot = (s + 1) % kvq_ctx::kLenSlots;
+    if (cudaEventQuery(c->len_ev[s]) == cudaErrorNotReady) KVQ_CUDA(c, cudaEventSynchronize(c->len_ev[s]));
+    cudaGetLastError();
+    *host = c->h_lens + (size_t)s * 3 * c->batch;
+    *dev = c->d_lens + (size_t)s * 3 * c->batch;
+    return s;
 }
 
 inline uint32_t* counts_of(kvq_ctx* c, int which, int layer) {
@@ -250,21 +277,24 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
     p.bits_out = bits_out;
     p.cls = c->cls;
     p.hist = c->hist;
+    p.chunk_arrivals = c->chunk_arrivals;
     p.counts_in = counts_of(c, c->cur[layer], layer);
     p.counts_out = counts_of(c, c->cur[layer] ^ 1, layer);
     p.layer = layer;
     p.n_new = n_new;
     p.pos0 = c->len[layer];
     if (call_ragged || c->ragged[layer]) {             // per-sequence counts and positions travel with the call
-        std::vector<int> blk(2 * (size_t)c->batch);
+        int *h_slot = nullptr, *d_slot = nullptr;
+        const int slot = claim_len_slot(c, &h_slot, &d_slot);
+        if (slot < 0) return slot;
         for (int b = 0; b < c->batch; ++b) {
-            blk[b] = host_lens ? host_lens[b] : n_new;
-            blk[c->batch + b] = cur_lens[b];
+            h_slot[b] = host_lens ? host_lens[b] : n_new;
+            h_slot[c->batch + b] = cur_lens[b];
         }
-        KVQ_CUDA(c, cudaMemcpyAsync(c->d_lens, blk.data(), sizeof(int) * blk.size(), cudaMemcpyHostToDevice, st));
-        KVQ_CUDA(c, cudaStreamSynchronize(st));        // blk is pageable and about to go out of scope
-        p.lens = c->d_lens;
-        p.pos = c->d_lens + c->batch;
+        KVQ_CUDA(c, cudaMemcpyAsync(d_slot, h_slot, sizeof(int) * 2 * c->batch, cudaMemcpyHostToDevice, st));
+        KVQ_CUDA(c, cudaEventRecord(c->len_ev[slot], st));
+        p.lens = d_slot;
+        p.pos = d_slot + c->batch;
     }
     // Long prefills use chunks of 1024 tokens (fewer partly filled tiles at chunk ends), as long as that still
     // leaves several waves of CTAs once the KV heads are split into groups; everything else 256.
@@ -287,7 +317,7 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
 
     const size_t smem = fused ? controller_smem(c->hidden) : 0;
     dim3 grid_q(p.nchunks, groups, c->batch);
-    if (n_new == 1 && !call_ragged && (!fused || c->hidden == 32)) {   // a decode step: one warp per 16 heads
+    if (n_new == 1 && !call_ragged) {                  // a decode step: one warp per 16 heads
         dim3 grid_t((c->kv_heads + 15) / 16, c->batch);
         if (c->groups == 1) {
             if (fused) launch_overlapped(k_append_token<true, 1>, grid_t, 32, 0, st, p);
@@ -310,7 +340,6 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
         dim3 grid_c(p.nchunks, c->batch);
         if (fused) k_classify<true><<<grid_c, kChunkTokens, smem, st>>>(p);
         else k_classify<false><<<grid_c, kChunkTokens, 0, st>>>(p);
-        k_reserve_blocks<<<c->batch, 128, 0, st>>>(p);
         if (p.tpt == 1) {
             if (c->groups == 1) k_quant_pack_frag<0, 1><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
             else k_quant_pack<0, 2, 1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
@@ -318,7 +347,7 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
             if (c->groups == 1) k_quant_pack_frag<0, KVQ_APPEND_TOKENS_PER_THREAD><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
             else k_quant_pack<0, 2, KVQ_APPEND_TOKENS_PER_THREAD><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
         }
-        c->launches += 3;
+        c->launches += 2;
     }
     KVQ_CUDA(c, cudaGetLastError());
     c->cur[layer] ^= 1;
@@ -626,6 +655,7 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
     ok = ok && dev_alloc(c, &c->counts, sizeof(uint32_t) * 2 * (size_t)layers * batch * 4) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->cls, (size_t)batch * max_ctx) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->hist, sizeof(uint4) * batch * max_chunks) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->chunk_arrivals, sizeof(uint32_t) * batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->ctrl, controller_smem(kMaxHidden)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_o, sizeof(float) * max_partial_records(c) * kHeadDim) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_ml, sizeof(float2) * max_partial_records(c)) == cudaSuccess;
@@ -633,7 +663,7 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
     ok = ok && dev_alloc(c, &c->part_s2, sizeof(float) * max_partial_records(c)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->unit_var, sizeof(float) * units) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->vis, sizeof(uint32_t) * 4 * (size_t)batch * kMaxQueryRows) == cudaSuccess;
-    ok = ok && dev_alloc(c, &c->d_lens, sizeof(int) * 3 * (size_t)batch) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->d_lens, sizeof(int) * 3 * (size_t)batch * kvq_ctx::kLenSlots) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->flags, sizeof(uint32_t)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_feats, sizeof(float) * 4 * batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_K, sizeof(__half) * (size_t)batch * kv_heads * kHeadDim) == cudaSuccess;
@@ -648,6 +678,11 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
         return KVQ_OK;
     }
     if (ok) {
+        ok = cudaMallocHost(reinterpret_cast<void**>(&c->h_lens), sizeof(int) * 3 * (size_t)batch * kvq_ctx::kLenSlots) == cudaSuccess;
+        for (int i = 0; ok && i < kvq_ctx::kLenSlots; ++i)
+            ok = cudaEventCreateWithFlags(&c->len_ev[i], cudaEventDisableTiming) == cudaSuccess;
+    }
+    if (ok) {
         s.arena = c->arena;
         s.table = c->table;
         s.arena_used = c->arena_used;
@@ -658,6 +693,7 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
         ok = ok && cudaMemset(s.index, 0, sizeof(uint32_t) * (size_t)layers * batch * max_ctx) == cudaSuccess;
         ok = ok && cudaMemset(c->counts, 0, sizeof(uint32_t) * 2 * (size_t)layers * batch * 4) == cudaSuccess;
         ok = ok && cudaMemset(c->flags, 0, sizeof(uint32_t)) == cudaSuccess;
+        ok = ok && cudaMemset(c->chunk_arrivals, 0, sizeof(uint32_t) * batch) == cudaSuccess;
         ok = ok && cudaMemset(c->part_cnt, 0, sizeof(uint32_t) * units * kMaxQueryRows) == cudaSuccess;
         // the controller block may exceed the default 48 KB of dynamic shared memory
         const int smem_max = (int)controller_smem(kMaxHidden);
@@ -826,10 +862,13 @@ int kvq_attend_last(kvq_ctx* c, int layer, const void* Q, void* O, int n_queries
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int* d_len = nullptr;
     if (c->ragged[layer]) {
-        KVQ_CUDA(c, cudaMemcpyAsync(c->d_lens + 2 * c->batch, &c->lens[(size_t)layer * c->batch], sizeof(int) * c->batch,
-                                    cudaMemcpyHostToDevice, st));
-        KVQ_CUDA(c, cudaStreamSynchronize(st));
-        d_len = c->d_lens + 2 * c->batch;
+        int *h_slot = nullptr, *d_slot = nullptr;
+        const int slot = claim_len_slot(c, &h_slot, &d_slot);
+        if (slot < 0) return slot;
+        for (int b = 0; b < c->batch; ++b) h_slot[2 * c->batch + b] = c->lens[(size_t)layer * c->batch + b];
+        KVQ_CUDA(c, cudaMemcpyAsync(d_slot + 2 * c->batch, h_slot + 2 * c->batch, sizeof(int) * c->batch, cudaMemcpyHostToDevice, st));
+        KVQ_CUDA(c, cudaEventRecord(c->len_ev[slot], st));
+        d_len = d_slot + 2 * c->batch;
     }
     for (int t0 = 0; t0 < n_queries; t0 += kMaxQueryRows) {
         const int tq = n_queries - t0 < kMaxQueryRows ? n_queries - t0 : kMaxQueryRows;

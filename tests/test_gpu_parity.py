@@ -285,6 +285,32 @@ def test_decode_after_incremental_steps(gu, oracle):
             gu.assert_attention_close(g.decode(0, Q), oc.decode_attn(Q), "step %d" % step)
 
 
+@pytest.mark.parametrize("hidden,seed", [(32, 322), (128, 2), (7, 5), (100, 9)])
+def test_decode_steps_with_the_controller_inside_the_append(gu, oracle, hidden, seed):
+    """Decode steps through kvq_append_fused with one new token per sequence: the one-launch token append takes the
+    decision itself for every hidden width (the paper's 128 included), bit for bit the oracle's; store and attention
+    follow.  20 KV heads: two warps per sequence take the same decision."""
+    rng = np.random.default_rng(hidden)
+    cw = synth.controller_weights(seed, hidden)
+    B, Hq, H, steps = 3, 20, 20, 40
+    oc = oracle.OracleCache(B, Hq, H)
+    with gu.GpuCache(1, B, Hq, H, 64) as g:
+        g.set_controller(cw)
+        feats = synth.features_batch(seed, B, 0, steps)
+        want_bits, want_logits, gap = oracle.select_bits(feats, hidden, *cw.as_tuple())
+        got_bits = np.zeros_like(want_bits)
+        for step in range(steps):
+            K, V = _kv(rng, B, 1, H)
+            got_bits[:, step:step + 1] = g.append_fused(0, K, V, feats[:, step:step + 1])
+            oc.append(K, V, want_bits[:, step:step + 1])
+        near = gu.compare_decisions(got_bits, want_bits, want_logits, gap, "token append H=%d" % hidden)
+        assert all(r[3] == r[4] for r in near)
+        assert len(set(want_bits.ravel().tolist())) >= 2          # the weights do spread the tokens over classes
+        gu.assert_store_equals_oracle(g, 0, oc)
+        Q = rng.standard_normal((B, Hq, 64)).astype(np.float16)
+        gu.assert_attention_close(g.decode(0, Q), oc.decode_attn(Q), "H=%d" % hidden)
+
+
 @pytest.mark.parametrize("buffers", ["pageable", "page-locked", "page-locked but one", "page-locked, misaligned"])
 def test_decode_step_host_matches_device_path(gu, oracle, buffers):
     """The host-buffer entry point (fused append + attention, the step's inputs and result crossing the bus)
