@@ -346,3 +346,107 @@ class GroupedOracleCache:
                 p /= p.sum()
                 out[b, h] = p @ v
         return np.asarray(out, dtype=np.float16).view(np.uint16)          # fp64 -> fp16, round to nearest even
+
+
+def _unpack_codes(codes: np.ndarray, n: int, bits: int) -> np.ndarray:
+    """The first n codes of little-endian linear packed rows: codes u8 [..., bytes] -> u8 [..., n]."""
+    idx = np.arange(n) * bits
+    return (codes[..., idx // 8] >> (idx % 8).astype(np.uint8)) & np.uint8((1 << bits) - 1)
+
+
+def _pack_codes(c: np.ndarray, bits: int, row_bytes: int) -> np.ndarray:
+    """Codes u8 [..., n] -> little-endian linear packed rows u8 [..., row_bytes] (tail zero)."""
+    n = c.shape[-1]
+    out = np.zeros(c.shape[:-1] + (row_bytes,), dtype=np.uint8)
+    for i in range(n):
+        bp = i * bits
+        out[..., bp // 8] |= (c[..., i].astype(np.uint8) << np.uint8(bp % 8))
+    return out
+
+
+class PerChannelKCache:
+    """A cache whose KEYS are quantized per channel instead of per token (the granularity of the key quantizers in
+    the related work the paper cites in Section 2), values per token as in ``OracleCache``.
+
+    Reading.  Tokens go to the pool of their bit-width and take slots in position order as before.  The slots of a
+    (sequence, KV head, precision) stream are cut into WINDOWS of ``window`` = 16 consecutive slots.  In a complete
+    window every channel is a row for the row quantizer (the reading of Q_b in Eq. 24): its ``window`` key values,
+    one per token, get one {scale, zero-point} pair and codes by the same arithmetic.  The stream's last, still
+    incomplete window keeps its key rows in fp16 (they are quantized when the window fills); 16-bit tokens keep
+    fp16 rows as always.  Attention is Eq. 5 by its definition (fp64) over the dequantized rows.
+
+    Kept per token and KV head, for comparison with other implementations: ``k_state`` 0 = fp16 row (16-bit class or
+    open window), 1 = packed; ``kc`` the canonical row (packed codes in element order, or the fp16 row); per
+    (stream, window, channel) ``chan_meta`` {scale, zero-point} bit patterns."""
+
+    def __init__(self, batch: int, q_heads: int, kv_heads: int, head_dim: int = 64, window: int = 16):
+        self.B, self.Hq, self.Hkv, self.D, self.W = batch, q_heads, kv_heads, head_dim, window
+        self.bits = np.zeros((batch, 0), dtype=np.uint8)
+        self.K = np.zeros((batch, 0, kv_heads, head_dim), dtype=np.uint16)      # fp16 bit patterns as appended
+        self.vc = np.zeros((batch, 0, kv_heads, 2 * head_dim), dtype=np.uint8)
+        self.vm = np.zeros((batch, 0, kv_heads, 2), dtype=np.uint16)
+        self.counts = np.zeros((batch, 4), dtype=np.uint32)
+        self.pool_slot = np.zeros((batch, 0), dtype=np.uint32)
+
+    def __len__(self) -> int:
+        return self.bits.shape[1]
+
+    def append(self, K, V, bits) -> None:
+        bits = _c(bits, np.uint8)
+        _, _, vc, vm = append(V, V, bits)                          # values: the per-token row quantizer
+        ps = np.empty(bits.shape, dtype=np.uint32)
+        for b in range(self.B):
+            ps[b], self.counts[b] = assign_slots(bits[b], self.counts[b])
+        self.bits = np.concatenate([self.bits, bits], axis=1)
+        self.K = np.concatenate([self.K, _u16(K)], axis=1)
+        self.vc = np.concatenate([self.vc, vc], axis=1)
+        self.vm = np.concatenate([self.vm, vm], axis=1)
+        self.pool_slot = np.concatenate([self.pool_slot, ps], axis=1)
+
+    def key_state(self):
+        """(k_state u8 [B][n][Hkv], kc u8 [B][n][Hkv][2D], khat f32 [B][n][Hkv][D], chan_meta {(b, h, bits, window):
+        u16 [D][2]}) of the cache as it stands."""
+        B, n, H, D, W = self.B, len(self), self.Hkv, self.D, self.W
+        k_state = np.zeros((B, n, H), dtype=np.uint8)
+        kc = np.zeros((B, n, H, 2 * D), dtype=np.uint8)
+        khat = half_to_float(self.K)
+        kc[..., 0:2 * D:2] = (self.K & 0xFF).astype(np.uint8)          # fp16 rows, little-endian
+        kc[..., 1:2 * D:2] = (self.K >> 8).astype(np.uint8)
+        chan_meta = {}
+        for b in range(B):
+            for bt in (2, 4, 8):
+                pos = np.flatnonzero(self.bits[b] == bt)               # position order = slot order
+                for w in range(len(pos) // W):
+                    p = pos[w * W:(w + 1) * W]
+                    for h in range(H):
+                        # every channel's W values as one row of the row quantizer: [1][1][D][W]
+                        rows = np.ascontiguousarray(self.K[b, p, h, :].T)[None, None]
+                        cg, mg, _, _ = append(rows, rows, np.full((1, 1), bt, np.uint8))
+                        codes = _unpack_codes(cg[0, 0, :, :W * bt // 8], W, bt)       # [D][W]
+                        kc[b, p, h, :] = _pack_codes(np.ascontiguousarray(codes.T), bt, 2 * D)
+                        k_state[b, p, h] = 1
+                        chan_meta[(b, h, bt, w)] = mg[0, 0]
+                        for i in range(D):
+                            khat[b, p, h, i] = dequantize_row(cg[0, 0, i, :W * bt // 8], mg[0, 0, i], W, bt)
+        return k_state, kc, khat, chan_meta
+
+    def decode_attn(self, Q) -> np.ndarray:
+        """fp16 bit patterns [B][Hq][D]: Softmax(q K^T / sqrt(D)) V over the dequantized rows, in fp64."""
+        _, _, khat, _ = self.key_state()
+        q = half_to_float(_u16(Q)).astype(np.float64)
+        g = self.Hq // self.Hkv
+        out = np.empty((self.B, self.Hq, self.D), dtype=np.float64)
+        n = len(self)
+        for b in range(self.B):
+            vhat = np.empty((n, self.Hkv, self.D), dtype=np.float64)
+            for t in range(n):
+                bt = int(self.bits[b, t])
+                for h in range(self.Hkv):
+                    vhat[t, h] = dequantize_row(self.vc[b, t, h, :self.D * bt // 8], self.vm[b, t, h], self.D, bt)
+            for h in range(self.Hq):
+                k = khat[b, :, h // g].astype(np.float64)
+                z = k @ q[b, h] / np.sqrt(float(self.D))
+                p = np.exp(z - z.max())
+                p /= p.sum()
+                out[b, h] = p @ vhat[:, h // g]
+        return np.asarray(out, dtype=np.float16).view(np.uint16)
