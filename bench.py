@@ -358,7 +358,7 @@ def near_tie_report(bench, ctx, feats_d, n, max_rows=5):
     return {"threshold": NEAR_TIE_GAP, "decisions": int(n), "count": int(idx.numel()), "first": rows}
 
 
-def measure(bench, wl, *, steps, warmup, blocks, uniform_bits=0, scale_groups=1, e2e=True, e2e_blocks=3):
+def measure(bench, wl, *, steps, warmup, blocks, uniform_bits=0, scale_groups=1, e2e=True, e2e_blocks=3, k_per_channel=False):
     """Build the cache of `wl`, time its prefill, its decode steps and (optionally) the host-buffer steps."""
     torch, kq, dev, clib, stream = bench.torch, bench.kq, bench.dev, bench.clib, bench.stream
     W, K_steps = warmup, steps
@@ -388,7 +388,9 @@ def measure(bench, wl, *, steps, warmup, blocks, uniform_bits=0, scale_groups=1,
     t_gen = time.perf_counter() - t_gen
 
     to_dev = bench.to_dev
-    if scale_groups == 1:
+    if k_per_channel:
+        ctx = kq.kvq_create_perchannel(L, Hq, Hkv, D, ctx_len + total_steps, B)
+    elif scale_groups == 1:
         ctx = kq.kvq_create(L, Hq, Hkv, D, ctx_len + total_steps, B)
     else:
         ctx = kq.kvq_create_grouped(L, Hq, Hkv, D, ctx_len + total_steps, B, 0, scale_groups)
@@ -628,9 +630,9 @@ def cpu_leg(wl, steps, warmup=1):
 def run_ours(args, wl):
     bench = Bench()
     rank, world = bench.rank, bench.world
-    is_headline = wl.name == "cfg5" and not args.uniform_bits and args.scale_groups == 1
+    is_headline = wl.name == "cfg5" and not args.uniform_bits and args.scale_groups == 1 and not args.k_per_channel
     m = measure(bench, wl, steps=args.steps, warmup=args.warmup, blocks=args.blocks, uniform_bits=args.uniform_bits,
-                scale_groups=args.scale_groups)
+                scale_groups=args.scale_groups, k_per_channel=args.k_per_channel)
 
     others = None
     if is_headline and world == 1 and not args.no_other_workloads:
@@ -657,7 +659,7 @@ def run_ours(args, wl):
             "metric": METRIC, "value": m["bytes_job"] / (ms_step * 1e-3) / 1e9, "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(wl, args.uniform_bits, args.scale_groups),
+            "config": dict(workload_config(wl, args.uniform_bits, args.scale_groups), **({"k_per_channel": True} if args.k_per_channel else {})),
             "timing": {"blocks": args.blocks, "steps_per_block": args.steps,
                        "ms_per_step_median": ms_step, "ms_per_step_min": m["ms_step_min"], "ms_per_step_max": m["ms_step_max"],
                        "ms_per_step_of_each_block": m["ms_step_blocks"],
@@ -774,6 +776,8 @@ def main():
     ap.add_argument("--scale-groups", type=int, choices=[1, 2], default=1,
                     help="2: one scale / zero-point pair per 32 channels instead of per row (a variant, not the "
                          "quantizer the metric is quoted on)")
+    ap.add_argument("--k-per-channel", action="store_true",
+                    help="keys quantized per channel over windows of 16 slots (a variant, not the quantizer the metric is quoted on)")
     ap.add_argument("--batch", type=int, default=0,
                     help="fewer sequences than the workload's 16, likewise for profiler captures only")
     args = ap.parse_args()

@@ -106,6 +106,29 @@ int kvq_create_grouped(kvq_ctx** out, int layers, int q_heads, int kv_heads, int
                        int max_ctx, int batch, uint64_t arena_bytes, int scale_groups);
 
 /*
+ * The same with PER-CHANNEL KEYS, the granularity of the key quantizers in the related work the paper cites in
+ * Section 2 (Eq. 24 only names Q_b).  Tokens still go to the pool of their bit-width and take slots in position
+ * order; the slots of a (sequence, KV head, precision) stream are cut into windows of 16.  In a complete window
+ * every key CHANNEL is quantized by the row quantizer over its 16 values (one per token): one {scale,
+ * zero-point} pair per channel and window, codes as before.  The keys of the stream's last, incomplete window
+ * wait as fp16 rows and are packed when the window fills; the decode calls read them as they are.  Values keep
+ * one pair per token.  A stored row takes 52 / 84 / 148 / 256 bytes per token and KV head, plus 6 KB per stream
+ * for the waiting rows.  kvq_export_range returns, in k_codes, packed codes for keys in complete windows and the
+ * fp16 row otherwise, and {0,0} in k_meta; kvq_export_k_channels returns a window's pairs.  kvq_attend_last takes
+ * n_queries == 1 only and kvq_workspace_bytes / kvq_create_in do not offer this layout; everything else behaves
+ * as with kvq_create_arena.
+ */
+int kvq_create_perchannel(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim,
+                          int max_ctx, int batch, uint64_t arena_bytes);
+
+/*
+ * Per-channel keys: the 64 {scale, zero-point} pairs (fp16 bit patterns, host uint16 [64][2]) of window
+ * `window` (slots 16 window .. 16 window + 15) of the stream (layer, sequence b, kv_head, bits in {2,4,8}).
+ * KVQ_ERR_ARG if the window is not complete or the cache has another layout.  Synchronizes.
+ */
+int kvq_export_k_channels(kvq_ctx* ctx, int layer, int b, int kv_head, int bits, int window, uint16_t* host_meta);
+
+/*
  * The same cache inside device memory that the caller owns (for instance one torch tensor), so that
  * the library itself allocates no device memory for it.  kvq_workspace_bytes gives the size the other
  * arguments need (host uint64; it reads the current device's properties, allocates nothing).

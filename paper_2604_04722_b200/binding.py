@@ -34,6 +34,8 @@ SIGNATURES = {
     "kvq_create": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i]),
     "kvq_create_arena": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, C.c_uint64]),
     "kvq_create_grouped": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, C.c_uint64, _i]),
+    "kvq_create_perchannel": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, C.c_uint64]),
+    "kvq_export_k_channels": (_i, [_vp, _i, _i, _i, _i, _i, _vp]),
     "kvq_workspace_bytes": (_i, [_i, _i, _i, _i, _i, _i, C.c_uint64, _i, C.POINTER(C.c_uint64)]),
     "kvq_create_in": (_i, [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, C.c_uint64, _i, _vp, C.c_uint64]),
     "kvq_arena_usage": (_i, [_vp, _u64p, _u64p, _u64p]),
@@ -142,6 +144,22 @@ def kvq_create_grouped(layers: int, q_heads: int, kv_heads: int, head_dim: int, 
     check(lib().kvq_create_grouped(C.byref(h), layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes,
                                    scale_groups), "kvq_create_grouped")
     return h.value
+
+
+def kvq_create_perchannel(layers: int, q_heads: int, kv_heads: int, head_dim: int, max_ctx: int, batch: int,
+                          arena_bytes: int = 0) -> int:
+    h = _vp()
+    check(lib().kvq_create_perchannel(C.byref(h), layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes),
+          "kvq_create_perchannel")
+    return h.value
+
+
+def kvq_export_k_channels(ctx: int, layer: int, b: int, kv_head: int, bits: int, window: int):
+    """Returns the window's {scale, zero-point} pairs as numpy u16 [64][2]."""
+    import numpy as np
+    out = np.zeros((64, 2), np.uint16)
+    check(lib().kvq_export_k_channels(ctx, layer, b, kv_head, bits, window, out.ctypes.data), "kvq_export_k_channels")
+    return out
 
 
 def kvq_workspace_bytes(layers: int, q_heads: int, kv_heads: int, head_dim: int, max_ctx: int, batch: int,

@@ -602,6 +602,39 @@ __device__ __forceinline__ void token_store(int c, const uint4 (&kraw)[4], const
     }
 }
 
+// The stores of k_append_token for a cache with per-channel keys: the key half-row joins the fp16 residual rows of
+// its stream (it is packed when its window of 16 slots is complete, by k_pack_window); the value half-row is
+// quantized per token as in the other layouts.  kres: the stream's residual rows of class c, [16][64].
+__device__ __forceinline__ void token_store_pc(int c, const uint4 (&kraw)[4], const uint4 (&vraw)[4], bool active, int half,
+                                               int t, uint8_t* rec, __half* kres) {
+    uint8_t* vcodes = rec + pool_codes_bytes(c);
+    if (t == 0 && c < 3 && active && half == 0) {      // the token opens a tile: clear the tile's value {scale, zero-point} words
+        uint4* m = reinterpret_cast<uint4*>(rec + meta_offset(c, 1, 0, 0, kLayoutPerChannelK));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) m[i] = make_uint4(0, 0, 0, 0);
+    }
+    __syncwarp();
+    if (c < 3 && active) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) *reinterpret_cast<uint4*>(kres + t * kHeadDim + 32 * half + 8 * u) = kraw[u];
+    }
+    uint8_t* vmeta = rec + meta_offset(c < 3 ? c : 0, 1, t, 0, kLayoutPerChannelK);
+    switch (c) {
+    case 0: quantize_store_half_row<0, 1, 1, 1>(vraw, active, false, half, t, vcodes, vmeta); break;
+    case 1: quantize_store_half_row<1, 1, 1, 1>(vraw, active, false, half, t, vcodes, vmeta); break;
+    case 2: quantize_store_half_row<2, 1, 1, 1>(vraw, active, false, half, t, vcodes, vmeta); break;
+    default:
+        if (active) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                *reinterpret_cast<uint4*>(rec + unit_offset(3, half, u, t)) = kraw[u];
+                *reinterpret_cast<uint4*>(vcodes + unit_offset(3, half, u, t)) = vraw[u];
+            }
+        }
+        break;
+    }
+}
+
 // One new token per sequence (a decode step): grid = (ceil(kv_heads / 16), batch), block = 32.
 // Lane l handles half-row l%2 of KV head 16*blockIdx.x + l/2.  Everything the warp needs (the K and V
 // rows, the pool fills, the features) is requested up front so the loads overlap the controller;
@@ -663,12 +696,18 @@ k_append_token(AppendParams p) {
         id = __shfl_sync(0xffffffffu, id, lane & ~1);
         // the partner lane must not read the table before the entry is written: hand it the address instead
         uint8_t* rec_new = p.store.arena + (size_t)id * kBlockBytes;
-        token_store<G>(c, kraw, vraw, active, half, t, rec_new);
+        if constexpr (G == kLayoutPerChannelK)
+            token_store_pc(c, kraw, vraw, active, half, t, rec_new, c < 3 ? residual_rows(p.store, c, p.layer, b, active ? h : 0) : nullptr);
+        else
+            token_store<G>(c, kraw, vraw, active, half, t, rec_new);
         return;
     }
     const uint32_t id = c == 0 ? id0 : c == 1 ? id1 : c == 2 ? id2 : id3;
-    token_store<G>(c, kraw, vraw, active, half, t,
-                   p.store.arena + (size_t)id * kBlockBytes + (size_t)(tile % block_tiles(c, G)) * (uint32_t)pool_rec_bytes(c, G));
+    uint8_t* rec = p.store.arena + (size_t)id * kBlockBytes + (size_t)(tile % block_tiles(c, G)) * (uint32_t)pool_rec_bytes(c, G);
+    if constexpr (G == kLayoutPerChannelK)
+        token_store_pc(c, kraw, vraw, active, half, t, rec, c < 3 ? residual_rows(p.store, c, p.layer, b, active ? h : 0) : nullptr);
+    else
+        token_store<G>(c, kraw, vraw, active, half, t, rec);
 }
 
 }  // namespace kvq

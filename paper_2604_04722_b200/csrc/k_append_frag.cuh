@@ -177,6 +177,7 @@ struct FragV {
     __device__ static constexpr int pos(int i, int e) { return CLS == 0 ? i : CLS == 1 ? (e >> 1) * 2 + i : 4 * (e >> 1) + (e & 1) * 2 + i; }
     __device__ static constexpr int shift(int j, int e) { return 8 * j + (CLS == 0 ? 2 * e : CLS == 1 ? 4 * (e & 1) : 0); }
 
+    template <bool CLAMP>
     __device__ static __forceinline__ void codes(const __half2 (&h)[4][4], const float4 (&sc)[2], uint32_t (&vw)[NW]) {
         uint32_t bias[NW];
 #pragma unroll
@@ -198,14 +199,16 @@ struct FragV {
 #pragma unroll
                 for (int e = 0; e < 4; e += 2) {
                     uint32_t b0, b1;
-                    code_pair<CLS, false>(h[j][2 * i + (e >> 1)], mn, inv, b0, b1);
+                    code_pair<CLS, CLAMP>(h[j][2 * i + (e >> 1)], mn, inv, b0, b1);
                     vw[pos(i, e)] += b0 << shift(j, e);
                     vw[pos(i, e + 1)] += b1 << shift(j, e + 1);
                 }
         }
     }
     // voff[j]: byte offset, inside the stage, of elements 4g .. 4g+3 of slot 4q + j (elements 32+4g .. sit 64 bytes
-    // further, xor-wise).  false: a subnormal scale in the tile (see FragK::tile).
+    // further, xor-wise).  false: a subnormal scale in the tile (see FragK::tile); with CLAMP every quotient is
+    // clamped and the answer is always true.
+    template <bool CLAMP = false>
     __device__ static __forceinline__ bool tile(const uint8_t* stage, const int (&voff)[4], float2* scratch, int g, int q,
                                                 uint32_t (&vw)[NW], uint32_t& meta) {
         __half2 h[4][4];                               // [slot 4q + j][elements 4g..4g+3, then 32+4g..32+4g+3]
@@ -220,7 +223,7 @@ struct FragV {
         // lanes g and g + 4 set up slot 4q + (g & 3); the results reach every lane through shared memory
         const __half2 mine = (g & 3) == 0 ? mm[0] : (g & 3) == 1 ? mm[1] : (g & 3) == 2 ? mm[2] : mm[3];
         const RowScale rs = row_scale<CLS>(__low2float(mine), -__high2float(mine));
-        if (__any_sync(0xffffffffu, rs.tiny)) return false;
+        if (!CLAMP && __any_sync(0xffffffffu, rs.tiny)) return false;
         meta = rs.meta;
         __syncwarp();                                  // the scratch may still be read for the previous tile
         if (g < 4) scratch[4 * q + g] = make_float2(rs.inv, rs.mn);
@@ -228,8 +231,86 @@ struct FragV {
         float4 sc[2];
         sc[0] = *reinterpret_cast<const float4*>(scratch + 4 * q);
         sc[1] = *reinterpret_cast<const float4*>(scratch + 4 * q + 2);
-        codes(h, sc, vw);
+        codes<CLAMP>(h, sc, vw);
         return true;
+    }
+};
+
+// ---- K side of one COMPLETE tile of a cache with per-channel keys: every channel's 16 values (one per slot) are a
+// row for the row quantizer.  Lane (g, q) holds the same elements as in FragK (16 per slot, slots g and g + 8);
+// a channel's minimum and maximum meet through three xor-shuffles over g; the lane with g = k sets up the two
+// channels of its element pair k and all lanes fetch the pairs' {reciprocal, minimum} through shared memory
+// (chan: 4 x 16 float2 owned by the warp).  The quotient is always clamped (no separate routine for subnormal scales).
+template <int CLS>
+struct FragKPC {
+    static constexpr int BITS = pool_bits(CLS), EPW = 32 / BITS, WT = 16 / EPW, NW = 2 * WT;
+    // canonical element index of element 2k (and 2k + 1) of the lane's 16 elements
+    __device__ static constexpr int element(int q, int k) {
+        return CLS == 0 ? 16 * q + 2 * k : CLS == 1 ? 8 * q + 32 * (k >> 2) + 2 * (k & 3) : 4 * q + 16 * (k >> 1) + 2 * (k & 1);
+    }
+    __device__ static __forceinline__ void codes(const __half2 (&h)[8], const float4 (&sc)[8], int i, uint32_t (&kw)[NW]) {
+        constexpr float LEVELS = (float)((1 << BITS) - 1);
+        uint32_t bias = 0;
+#pragma unroll
+        for (int e = 0; e < EPW; ++e) bias += 0x4B400000u << (BITS * e);
+#pragma unroll
+        for (int w = 0; w < WT; ++w) {
+            uint32_t acc = 0u - bias;
+#pragma unroll
+            for (int e = 0; e < EPW; e += 2) {
+                const int k = (w * EPW + e) / 2;       // sc[k] = {inv, mn} of element 2k, {inv, mn} of element 2k + 1
+                const float2 f = __half22float2(h[k]);
+                const float r0 = __fadd_rn(fminf(__fmul_rn(__fsub_rn(f.x, sc[k].y), sc[k].x), LEVELS), kRoundMagic);
+                const float r1 = __fadd_rn(fminf(__fmul_rn(__fsub_rn(f.y, sc[k].w), sc[k].z), LEVELS), kRoundMagic);
+                acc += __float_as_uint(r0) << (BITS * e);
+                acc += __float_as_uint(r1) << (BITS * (e + 1));
+            }
+            kw[FragK<CLS>::pos(i, w)] = acc;
+        }
+    }
+    // chan_meta: the tile's 64 {scale, zero-point} words in the record.
+    __device__ static __forceinline__ void tile(const uint8_t* stage, float4* chan, uint32_t* chan_meta, int g, int q,
+                                                uint32_t (&kw)[NW]) {
+        __half2 h0[8], h1[8];
+        FragK<CLS>::load_token(stage, g, q, h0);
+        FragK<CLS>::load_token(stage, g + 8, q, h1);
+        float4 sc[8];
+        {
+            __half2 mn[8], mx[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                mn[k] = __hmin2(h0[k], h1[k]);
+                mx[k] = __hmax2(h0[k], h1[k]);
+#pragma unroll
+                for (int d = 4; d <= 16; d <<= 1) {
+                    uint32_t a = *reinterpret_cast<uint32_t*>(&mn[k]), b = *reinterpret_cast<uint32_t*>(&mx[k]);
+                    a = __shfl_xor_sync(0xffffffffu, a, d);
+                    b = __shfl_xor_sync(0xffffffffu, b, d);
+                    mn[k] = __hmin2(mn[k], *reinterpret_cast<__half2*>(&a));
+                    mx[k] = __hmax2(mx[k], *reinterpret_cast<__half2*>(&b));
+                }
+            }
+            __half2 my_mn = mn[0], my_mx = mx[0];      // the pair this lane sets up: k = g
+#pragma unroll
+            for (int k = 1; k < 8; ++k) {
+                my_mn = g == k ? mn[k] : my_mn;
+                my_mx = g == k ? mx[k] : my_mx;
+            }
+            const RowScale lo = row_scale<CLS>(__low2float(my_mn), __low2float(my_mx));
+            const RowScale hi = row_scale<CLS>(__high2float(my_mn), __high2float(my_mx));
+            int e0 = element(q, 0);
+#pragma unroll
+            for (int k = 1; k < 8; ++k) e0 = g == k ? element(q, k) : e0;
+            chan_meta[e0] = lo.meta;
+            chan_meta[e0 + 1] = hi.meta;
+            __syncwarp();                              // the scratch may still be read for the previous tile
+            chan[q * 8 + g] = make_float4(lo.inv, lo.mn, hi.inv, hi.mn);
+            __syncwarp();
+#pragma unroll
+            for (int k = 0; k < 8; ++k) sc[k] = chan[q * 8 + k];
+        }
+        codes(h0, sc, 0, kw);
+        codes(h1, sc, 1, kw);
     }
 };
 
@@ -297,6 +378,44 @@ __device__ __forceinline__ bool frag_item(const uint8_t* stage, const int (&voff
         if (g < 4 && 4 * q + g >= first_new) *reinterpret_cast<uint32_t*>(rec + meta_offset(CLS, 1, 4 * q + g)) = vmeta;
     }
     return true;
+}
+
+// The same for a cache with per-channel keys.  live: slots that receive a token of this call; the tile's keys are
+// packed only when it is complete (slots below first_new came from earlier calls: their rows were fetched from the
+// residual buffer into the stage), otherwise the new rows join the residual rows `kres` [16][64] of the stream.
+template <int CLS>
+__device__ __forceinline__ void frag_item_pc(const uint8_t* stage, const int (&voff)[4], float2* scratch, float4* chan,
+                                             uint8_t* rec, __half* kres, int lane, int first_new, uint32_t live) {
+    const int g = lane >> 2, q = lane & 3;
+    constexpr int NW = FragK<CLS>::NW;
+    const bool complete = (live | ((1u << first_new) - 1u)) == 0xffffu;
+    if (complete) {
+        uint32_t kw[NW];
+        FragKPC<CLS>::tile(stage, chan, reinterpret_cast<uint32_t*>(rec + chan_meta_offset(CLS, 0)), g, q, kw);
+        store_block<NW>(rec, lane, kw);
+    } else {
+        const int half = lane >> 4, t = lane & 15;
+        if ((live >> t) & 1u) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                *reinterpret_cast<uint4*>(kres + t * kHeadDim + 32 * half + 8 * u) =
+                    *reinterpret_cast<const uint4*>(stage + stage_piece_offset(t, 4 * half + u));
+        }
+    }
+    uint8_t* vcodes = rec + pool_codes_bytes(CLS);
+    uint32_t vw[NW], vmeta;
+    FragV<CLS>::template tile<true>(stage + kStageTensorBytes, voff, scratch, g, q, vw, vmeta);
+    if (first_new > 0) {
+        uint32_t vo[NW];
+        load_block<NW>(vcodes, lane, vo);
+        const int nb = min(max(first_new - 4 * q, 0), 4);
+        const uint32_t keep = nb == 4 ? 0xffffffffu : ((1u << (8 * nb)) - 1u);
+#pragma unroll
+        for (int w = 0; w < NW; ++w) vw[w] = (vw[w] & ~keep) | (vo[w] & keep);
+    }
+    store_block<NW>(vcodes, lane, vw);
+    if (g < 4 && 4 * q + g >= first_new)
+        *reinterpret_cast<uint32_t*>(rec + meta_offset(CLS, 1, 4 * q + g, 0, kLayoutPerChannelK)) = vmeta;
 }
 
 // The general routine for one item: any class < 3, clamp included, every slot >= first_new written code word by
@@ -368,9 +487,11 @@ __device__ __forceinline__ void frag_item_fp16(const uint8_t* stage, uint8_t* re
 // The quantize-and-pack launch for caches with one scale group.  MODE as in k_quant_pack: 0 = classes from the
 // classify launch (several chunks per sequence), 1 = one chunk, classes from `bits`, 2 = one chunk, classes from
 // the controller.  grid = (nchunks, head_groups, batch), block = 256, dynamic smem = kFragRingBytes (+ controller).
-template <int MODE, int R = 1>
+// PC: the cache keeps per-channel keys (layout kLayoutPerChannelK).
+template <int MODE, int R = 1, bool PC = false>
 __global__ void __launch_bounds__(kChunkTokens, KVQ_APPEND_FRAG_MIN_CTAS)
 k_quant_pack_frag(AppendParams p) {
+    constexpr int LAYOUT = PC ? kLayoutPerChannelK : 1;
     static_assert(MODE == 0 || R == 1, "single-chunk appends hold at most 256 tokens per sequence");
     constexpr int CT = kChunkTokens * R;               // tokens per chunk
     constexpr int NWARPS = kChunkTokens / 32;
@@ -382,6 +503,7 @@ k_quant_pack_frag(AppendParams p) {
     __shared__ uint32_t ext[4][kTileTokens];           // tokens of later chunks that complete the last owned tile (index in the call)
     __shared__ uint32_t ext_n[4];
     __shared__ float2 vscratch[NWARPS][kTileTokens];
+    __shared__ float4 kchan[PC ? NWARPS : 1][32];      // per-channel keys: {reciprocal, minimum} of a tile's channels
     const int chunk = blockIdx.x, hg = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_b = new_tokens_of(p, b);
@@ -513,6 +635,7 @@ k_quant_pack_frag(AppendParams p) {
         int first_new;                                 // slots below it belong to an earlier call
         uint32_t live;                                 // bit s: slot s receives a token of this call
         uint8_t* rec;
+        int h;                                         // KV head
     };
     uint32_t tau = 0;
     int hh = warp;
@@ -533,6 +656,7 @@ k_quant_pack_frag(AppendParams p) {
         it.first_new = 0;
         it.live = 0;
         it.rec = nullptr;
+        it.h = 0;
         if (tau < pre[4]) {
             const int k = (tau >= pre[1]) + (tau >= pre[2]) + (tau >= pre[3]);
             const uint32_t basek = k == 0 ? base[0] : k == 1 ? base[1] : k == 2 ? base[2] : base[3];
@@ -544,7 +668,8 @@ k_quant_pack_frag(AppendParams p) {
             const int r0 = (int)(tile * kTileTokens) - (int)basek;       // rank of the tile's slot 0 (negative: older slots)
             it.first_new = r0 < 0 ? -r0 : 0;
             const int h = h0 + hh;
-            it.rec = tile_ptr(p.store, k, stream_table(p.store, k, p.layer, b, h), tile, 1);
+            it.h = h;
+            it.rec = tile_ptr(p.store, k, stream_table(p.store, k, p.layer, b, h), tile, LAYOUT);
             uint8_t* dst = my_ring + (size_t)stage * kFragStageBytes;
             const int piece = lane & 7;
 #pragma unroll
@@ -556,7 +681,12 @@ k_quant_pack_frag(AppendParams p) {
                 if (live) tok_i = (uint32_t)r < nk ? (size_t)chunk * CT + list[k][r] : (size_t)ext[k][(uint32_t)r - nk];
                 const size_t src = (((size_t)b * p.n_new + tok_i) * p.store.kv_heads + h) * kHeadDim;
                 const int off = stage_piece_offset(s, piece);
-                cp_async16_or_zero(dst + off, reinterpret_cast<const uint4*>(p.K + src) + piece, live);
+                // a slot of an earlier call: its key row waits in the residual buffer -- read from the copy taken before this
+                // launch, because the rows of the stream's NEXT open window go to the same places during the launch
+                if (PC && r < 0 && k < 3)
+                    cp_async16_or_zero(dst + off, reinterpret_cast<const uint4*>(residual_rows_before(p.store, k, b, h) + s * kHeadDim) + piece, true);
+                else
+                    cp_async16_or_zero(dst + off, reinterpret_cast<const uint4*>(p.K + src) + piece, live);
                 cp_async16_or_zero(dst + kStageTensorBytes + off, reinterpret_cast<const uint4*>(p.V + src) + piece, live);
             }
             // slots that receive a token: ranks 0 .. nke-1 that fall into this tile
@@ -579,6 +709,15 @@ k_quant_pack_frag(AppendParams p) {
         const uint8_t* st = my_ring + (size_t)stage * kFragStageBytes;
         if (cur.live != 0u) {                          // (a tile of an earlier call that this call adds nothing to)
             bool done = true;
+            if (PC) {
+                __half* kres = cur.k < 3 ? residual_rows(p.store, cur.k, p.layer, b, cur.h) : nullptr;
+                switch (cur.k) {
+                case 0: frag_item_pc<0>(st, voff, vscratch[warp], kchan[PC ? warp : 0], cur.rec, kres, lane, cur.first_new, cur.live); break;
+                case 1: frag_item_pc<1>(st, voff, vscratch[warp], kchan[PC ? warp : 0], cur.rec, kres, lane, cur.first_new, cur.live); break;
+                case 2: frag_item_pc<2>(st, voff, vscratch[warp], kchan[PC ? warp : 0], cur.rec, kres, lane, cur.first_new, cur.live); break;
+                default: frag_item_fp16(st, cur.rec, lane, cur.first_new, cur.live); break;
+                }
+            } else
             switch (cur.k) {
             case 0: done = frag_item<0>(st, voff, vscratch[warp], cur.rec, lane, cur.first_new); break;
             case 1: done = frag_item<1>(st, voff, vscratch[warp], cur.rec, lane, cur.first_new); break;
@@ -594,6 +733,49 @@ k_quant_pack_frag(AppendParams p) {
         if (++stage == kFragDepth) stage = 0;
     }
     cp_async_wait<0>();
+}
+
+// Per-channel keys, after a one-token append: the token that took the last slot of a window completes it, and one
+// warp per (KV head, sequence) packs the window's 16 residual rows.  grid = (kv_heads, batch), block = 32.
+__global__ void __launch_bounds__(32)
+k_pack_window(AppendParams p) {
+    __shared__ __align__(16) uint8_t stage[kStageTensorBytes];
+    __shared__ float4 chan[32];
+    const int h = blockIdx.x, b = blockIdx.y, lane = threadIdx.x;
+    const StoreView& s = p.store;
+    const uint32_t word = s.index[((size_t)p.layer * s.batch + b) * s.max_ctx + first_pos_of(p, b)];
+    const int c = (int)(word >> 30);
+    const uint32_t slot = word & 0x3fffffffu;
+    if (c == 3 || (slot & (kTileTokens - 1)) != kTileTokens - 1) return;
+    const __half* rows = residual_rows(s, c, p.layer, b, h);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {                      // eight neighbouring lanes copy one 128-byte row
+        const int t = (lane >> 3) + 4 * i, piece = lane & 7;
+        *reinterpret_cast<uint4*>(stage + stage_piece_offset(t, piece)) = reinterpret_cast<const uint4*>(rows + t * kHeadDim)[piece];
+    }
+    __syncwarp();
+    uint8_t* rec = tile_ptr(s, c, stream_table(s, c, p.layer, b, h), slot / kTileTokens, kLayoutPerChannelK);
+    const int g = lane >> 2, q = lane & 3;
+    switch (c) {
+    case 0: {
+        uint32_t kw[FragK<0>::NW];
+        FragKPC<0>::tile(stage, chan, reinterpret_cast<uint32_t*>(rec + chan_meta_offset(0, 0)), g, q, kw);
+        store_block<FragK<0>::NW>(rec, lane, kw);
+        break;
+    }
+    case 1: {
+        uint32_t kw[FragK<1>::NW];
+        FragKPC<1>::tile(stage, chan, reinterpret_cast<uint32_t*>(rec + chan_meta_offset(1, 0)), g, q, kw);
+        store_block<FragK<1>::NW>(rec, lane, kw);
+        break;
+    }
+    default: {
+        uint32_t kw[FragK<2>::NW];
+        FragKPC<2>::tile(stage, chan, reinterpret_cast<uint32_t*>(rec + chan_meta_offset(2, 0)), g, q, kw);
+        store_block<FragK<2>::NW>(rec, lane, kw);
+        break;
+    }
+    }
 }
 
 }  // namespace kvq

@@ -498,9 +498,10 @@ struct ValueAcc {
     float ifix;                    // 2^(E-24)
 };
 
-template <int CLS>
+// LAYOUT: 1 = one {scale, zero-point} pair per key row, kLayoutPerChannelK = one pair per channel and tile.
+template <int CLS, int LAYOUT = 1>
 struct FragRows {
-    static constexpr int BITS = pool_bits(CLS), REC = pool_rec_bytes(CLS, 1);
+    static constexpr int BITS = pool_bits(CLS), REC = pool_rec_bytes(CLS, LAYOUT);
     static constexpr int NW = 2 << CLS;            // 32-bit words per lane of one tensor's codes: 2, 4, 8
     static constexpr int PLANES = 8 / BITS;        // codes per byte: 4, 2, 1
     static constexpr uint32_t MASK = CLS == 0 ? 0x03030303u : CLS == 1 ? 0x0f0f0f0fu : 0xffffffffu;
@@ -606,6 +607,11 @@ struct FragRows {
         float y = fmaf(km.x * (qi.inv_fix * kDotScale), dot, km.y * qi.sumq);
         y = valid ? y : -INFINITY;
 
+        finish_k_part(y, vm, q, slot, st, va, xbuf);
+    }
+    // The part of k_part that follows the logit: softmax weight, value weight on the grid, the rare grid changes.
+    template <class SM>
+    __device__ static __forceinline__ void finish_k_part(float y, float2 vm, int q, int slot, SM& st, ValueAcc& va, uint32_t* xbuf) {
         float e = fast_exp2(y - st.m);                 // the weight under the current maximum
         float x = (e * vm.x) * va.fix;                 // ... and its place on the current grid
         if (__builtin_expect(__any_sync(0xffffffffu, y > st.thr || !(x < kGridLimit)), 0)) {   // warp-uniform, rare
@@ -636,6 +642,118 @@ struct FragRows {
         if (SM::kStats) st.s2 = fmaf(e, e, st.s2);
         xbuf[(q >> 1) * kTileTokens + slot] = __float2uint_rn(x);
     }
+    // ---- per-channel keys.  khat_ti = c_ti s_i + z_i with one {s_i, z_i} per channel and TILE, so the scale moves to
+    // the query's side: q . khat_t = sum_i (q_i s_i) c_ti + sum_i q_i z_i, and the column operand of a tile's K products
+    // is the fixed-point form of q_i s_i, rebuilt for every tile (its own grid F: |q_i s_i F| < 2^22).  The lanes with
+    // g < 4 do that for tile A, the others for tile B (each lane the 16 channels of its operand registers).
+    // Position, among the lane's 16 channels, of the channel in byte j of operand register r of K product u; the
+    // channels are runs of 16 / 8 / 4 consecutive ones starting at pc_run(q, idx / run length).
+    __device__ static constexpr int pc_index(int u, int r, int j) {
+        return CLS == 0 ? 4 * j + 2 * u + r : CLS == 1 ? 8 * r + 2 * j + u : 4 * (2 * u + r) + j;
+    }
+    __device__ static constexpr int pc_channel(int q, int idx) {
+        return CLS == 0 ? 16 * q + idx : CLS == 1 ? 8 * q + 32 * (idx >> 3) + (idx & 7) : 4 * q + 16 * (idx >> 2) + (idx & 3);
+    }
+    __device__ static __forceinline__ void pc_load_query(const float* qrow, int q, float (&qe)[16]) {
+#pragma unroll
+        for (int idx = 0; idx < 16; ++idx) {
+            const int e = pc_channel(q, idx);
+            qe[idx] = qrow[(e >> 5) * (kHalfDim + 4) + (e & 31)];
+        }
+    }
+    // res_a / res_b: the tile's keys are still fp16 rows in kres (the open window of the stream): their logits are
+    // plain dot products, the tile's K products are ignored.
+    template <class SM>
+    __device__ static __forceinline__ void k_part_pc(const uint8_t* recA, const uint8_t* recB, bool valid, bool res_a, bool res_b,
+                                                     const __half* kres, const float* qrow, int lane, int g, int q,
+                                                     const float (&qe)[16], SM& st, ValueAcc& va, uint32_t* xbuf,
+                                                     uint32_t (&vwA)[NW], uint32_t (&vwB)[NW]) {
+        uint32_t kwA[NW], kwB[NW];
+        load_words(recA, lane, kwA);
+        load_words(recB, lane, kwB);
+        const int slot = g + 8 * (q & 1);
+        const uint8_t* rec_own = q < 2 ? recA : recB;
+        const float2 vm = meta_to_float2(*reinterpret_cast<const uint32_t*>(rec_own + meta_offset(CLS, 1, slot, 0, LAYOUT)));
+        load_words(recA + pool_codes_bytes(CLS), lane, vwA);
+        load_words(recB + pool_codes_bytes(CLS), lane, vwB);
+
+        // column operand of this lane's tile (A for g < 4, B otherwise)
+        const uint8_t* rec_x = g < 4 ? recA : recB;
+        float qs[16], zsum = 0.f, amax = 0.f;
+        constexpr int RUN = CLS == 0 ? 16 : CLS == 1 ? 8 : 4;
+#pragma unroll
+        for (int v4 = 0; v4 < 4; ++v4) {               // four {scale, zero-point} words per 16-byte load
+            const int e0 = pc_channel(q, 4 * v4);
+            const uint4 m4 = *reinterpret_cast<const uint4*>(rec_x + chan_meta_offset(CLS, e0));
+            const uint32_t m[4] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 sz = meta_to_float2(m[k]);
+                qs[4 * v4 + k] = qe[4 * v4 + k] * sz.x;
+                zsum = fmaf(qe[4 * v4 + k], sz.y, zsum);
+                amax = fmaxf(amax, fabsf(qs[4 * v4 + k]));
+            }
+        }
+        static_assert(RUN % 4 == 0, "a 16-byte load stays inside a run of consecutive channels");
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+        zsum += __shfl_xor_sync(0xffffffffu, zsum, 1);
+        zsum += __shfl_xor_sync(0xffffffffu, zsum, 2);
+        uint32_t ex = __float_as_uint(fmaxf(amax, 1.0e-30f)) >> 23;
+        ex = ex > 254u ? 254u : ex;                    // (garbage of a tile whose keys are residual rows)
+        const float fix = __uint_as_float((275u - ex) << 23), inv_fix = __uint_as_float((ex - 21u) << 23);
+        uint32_t bk[4];
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const float plane_scale = (float)(1 << (BITS * (PLANES - 1 - k_plane(u, r))));
+                uint32_t w = 0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int T = __float2int_rn(qs[pc_index(u, r, j)] * (fix * plane_scale));
+                    const int h0 = (T + 128) >> 8, d0 = T - (h0 << 8);
+                    const int h1 = (h0 + 128) >> 8, d1 = h0 - (h1 << 8);
+                    const int h2 = (h1 + 128) >> 8, d2 = h1 - (h2 << 8);
+                    const int dg = (g & 3) == 0 ? d0 : (g & 3) == 1 ? d1 : (g & 3) == 2 ? d2 : h2;
+                    w |= ((uint32_t)dg & 0xffu) << (8 * j);
+                }
+                bk[2 * u + r] = w;
+            }
+        uint32_t bkA[4], bkB[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            bkA[i] = g < 4 ? bk[i] : 0u;
+            bkB[i] = g < 4 ? 0u : bk[i];
+        }
+        int d[4] = {0, 0, 0, 0};
+        k_products(d, kwA, bkA);
+        k_products(d, kwB, bkB);
+        const float w0 = (q & 1) ? 65536.0f : 1.0f, w1 = (q & 1) ? 16777216.0f : 256.0f;
+        const float lo = fmaf((float)d[1], w1, (float)d[0] * w0), hi = fmaf((float)d[3], w1, (float)d[2] * w0);
+        const float dot = ((q & 1) ? hi : lo) + __shfl_xor_sync(0xffffffffu, (q & 1) ? lo : hi, 1);
+        // the owner's tile: its grid and its zero-point term sit with the lanes that built its operand
+        const int src = q < 2 ? 0 : 16;
+        const float inv_own = __shfl_sync(0xffffffffu, inv_fix, src), z_own = __shfl_sync(0xffffffffu, zsum, src);
+        float y = fmaf(inv_own * (kDotScale * kLogitScale), dot, z_own * kLogitScale);
+        if (res_a || res_b) {                          // warp-uniform: at most once per pool and segment
+            if (valid && (q < 2 ? res_a : res_b)) {
+                const __half2* row = reinterpret_cast<const __half2*>(kres + slot * kHeadDim);
+                float a = 0.f;
+#pragma unroll 8
+                for (int i = 0; i < kHeadDim / 2; ++i) {
+                    const float2 k2 = __half22float2(row[i]);
+                    const int e = 2 * i;
+                    a = fmaf(k2.x, qrow[(e >> 5) * (kHalfDim + 4) + (e & 31)], a);
+                    a = fmaf(k2.y, qrow[(e >> 5) * (kHalfDim + 4) + (e & 31) + 1], a);
+                }
+                y = a * kLogitScale;
+            }
+        }
+        y = valid ? y : -INFINITY;
+        finish_k_part(y, vm, q, slot, st, va, xbuf);
+    }
+
     // The four V products of one tile with the weights xs of its slots 4q .. 4q+3.
     __device__ static __forceinline__ void v_products(ValueAcc& va, const uint32_t (&vw)[NW], const uint4 xs, uint32_t sel) {
         const uint32_t bv = byte_perm(byte_perm(xs.x, xs.y, sel), byte_perm(xs.z, xs.w, sel), 0x5410u);
@@ -862,7 +980,7 @@ k_decode_attn(DecodeParams P) {
         QueryInfo qi;
         {
             const float qa = ws.q[lane], qb = ws.q[kQHalfStride + lane];
-            if (G == 1) {
+            if (G != 2) {
                 qi.sumq = warp_sum(qa + qb) * kLogitScale;         // sum_i q_i, in logit units
             } else {                                   // the sum over this lane's half: 32 elements over its 16 lanes
                 const float* qh_ = ws.q + half * kQHalfStride;
@@ -872,8 +990,8 @@ k_decode_attn(DecodeParams P) {
             const float qmax = fmaxf(warp_max(fmaxf(fabsf(qa), fabsf(qb))), 6.103515625e-05f);
             const uint32_t e = __float_as_uint(qmax) >> 23;        // biased exponent, 113..142
             // (the fragment path keeps one bit less: |q F| < 2^22, see FragRows)
-            qi.fix_scale = __uint_as_float(((G == 1 ? 275u : 276u) - e) << 23);
-            qi.inv_fix = __uint_as_float((e - (G == 1 ? 21u : 22u)) << 23) * kLogitScale;
+            qi.fix_scale = __uint_as_float(((G != 2 ? 275u : 276u) - e) << 23);
+            qi.inv_fix = __uint_as_float((e - (G != 2 ? 21u : 22u)) << 23) * kLogitScale;
             qi.q_half = ws.q + half * kQHalfStride;
         }
 
@@ -981,8 +1099,9 @@ k_decode_attn(DecodeParams P) {
         // a pair whose B is absent: it points at A's record again and every one of its slots counts as empty.
         auto walk_frag = [&](auto cls_tag) {
             constexpr int CLS = decltype(cls_tag)::value;
-            using C = FragRows<CLS>;
-            constexpr int TPS = Geo::tps(CLS, 1), BT = (int)block_tiles(CLS, 1);
+            constexpr bool PC = G == kLayoutPerChannelK;
+            using C = FragRows<CLS, PC ? kLayoutPerChannelK : 1>;
+            constexpr int TPS = Geo::tps(CLS, G), BT = (int)block_tiles(CLS, G);
             int tile0 = ws.lo[CLS];
             const int hi = ws.hi[CLS];
             if (tile0 >= hi || failed) return;
@@ -994,12 +1113,20 @@ k_decode_attn(DecodeParams P) {
             ChunkCursor cur;
             cur.start(tile0 % BT, TPS, BT);
             uint32_t bkA[4], bkB[4];
-            C::make_kb(ws.q, qi.fix_scale, g, q, bkA);
+            float qe[PC ? 16 : 1];                     // per-channel keys: the query channels of this lane's operand registers
+            if constexpr (PC) {
+                C::pc_load_query(ws.q, q, qe);
+            } else {
+                C::make_kb(ws.q, qi.fix_scale, g, q, bkA);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                bkB[i] = g >= 4 ? bkA[i] : 0u;
-                bkA[i] = g < 4 ? bkA[i] : 0u;
+                for (int i = 0; i < 4; ++i) {
+                    bkB[i] = g >= 4 ? bkA[i] : 0u;
+                    bkA[i] = g < 4 ? bkA[i] : 0u;
+                }
             }
+            // per-channel keys: the tile whose keys still wait as fp16 rows (the stream's open window), if any
+            const int res_tile = PC && (cnt & (kTileTokens - 1)) ? (int)(cnt / kTileTokens) : -1;
+            const __half* kres = PC ? residual_rows(P.store, CLS, P.layer, (int)b, kvh) : nullptr;
             ValueAcc va;
 #pragma unroll
             for (int m = 0; m < 4; ++m) va.d[m][0] = va.d[m][1] = va.d[m][2] = va.d[m][3] = 0;
@@ -1026,7 +1153,11 @@ k_decode_attn(DecodeParams P) {
                     const bool valid = (uint32_t)((tile0 + i) * kTileTokens) + my_slot < cnt && (q < 2 || has_b);
                     uint32_t vwA[C::NW], vwB[C::NW];
                     C::v_part(vpA, vpB, ws.x[pp ^ 1u], q, sel, va);
-                    C::k_part(recA, recB, valid, lane, g, q, bkA, bkB, qi, st, va, ws.x[pp], vwA, vwB);
+                    if constexpr (PC)
+                        C::k_part_pc(recA, recB, valid, tile0 + i == res_tile, has_b && tile0 + i + 1 == res_tile, kres, ws.q, lane, g,
+                                     q, qe, st, va, ws.x[pp], vwA, vwB);
+                    else
+                        C::k_part(recA, recB, valid, lane, g, q, bkA, bkB, qi, st, va, ws.x[pp], vwA, vwB);
                     __syncwarp();                      // the pair's weights are in shared memory
                     pp ^= 1u;
 #pragma unroll
@@ -1046,7 +1177,7 @@ k_decode_attn(DecodeParams P) {
             C::v_part(vpA, vpB, ws.x[pp ^ 1u], q, sel, va);     // the last pair's products
             C::flush(va, st, q);
         };
-        if constexpr (G == 1) {
+        if constexpr (G != 2) {
             walk_frag(std::integral_constant<int, 0>{});
             walk_frag(std::integral_constant<int, 1>{});
             walk_frag(std::integral_constant<int, 2>{});
@@ -1104,9 +1235,9 @@ k_decode_attn(DecodeParams P) {
         // (each half has its own zero-points: that sum stays inside the half).  One scale group: every token was
         // counted by exactly one lane; the quantized pools' part of the row sits with the lanes that own channels
         // and is gathered through shared memory.
-        const float l_w = (G == 1 ? 1.0f : 0.5f) * warp_sum(st.l);
-        const float b_w = G == 1 ? warp_sum(st.bsum) : half_sum(st.bsum);
-        if (G == 1) {
+        const float l_w = (G != 2 ? 1.0f : 0.5f) * warp_sum(st.l);
+        const float b_w = G != 2 ? warp_sum(st.bsum) : half_sum(st.bsum);
+        if (G != 2) {
             if ((lane & 3) < 2)
                 *reinterpret_cast<float4*>(ws.o + 4 * ((lane >> 2) + 8 * (lane & 3))) =
                     make_float4(st.of[0] + b_w, st.of[1] + b_w, st.of[2] + b_w, st.of[3] + b_w);
@@ -1119,7 +1250,7 @@ k_decode_attn(DecodeParams P) {
             r2[0] += b_w;
             r2[1] += b_w;
         }
-        const float s2_w = STATS ? (G == 1 ? 1.0f : 0.5f) * warp_sum(st.s2) : 0.f;
+        const float s2_w = STATS ? (G != 2 ? 1.0f : 0.5f) * warp_sum(st.s2) : 0.f;
 
         if (Geo::kCtaMerge && P.cta_parts) {
             // ---- all parts of the unit run in this CTA: partials and the arrival counter stay in shared memory

@@ -18,6 +18,7 @@ struct ExportParams {
     uint4* v_codes;
     uint16_t* k_meta;       // [nb][n][kv_heads][2 * scale groups]
     uint16_t* v_meta;
+    const uint32_t* counts; // [batch][4] pool fills of the layer (per-channel keys: which windows are complete)
 };
 
 // grid = (n, nb), block = 128.
@@ -43,7 +44,13 @@ k_export(ExportParams p) {
         const uint8_t* codes = tile_ptr(s, cls, stream_table(s, cls, p.layer, b, h), (uint32_t)tile, s.groups) +
                                (size_t)tensor * pool_codes_bytes(cls);
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (j < W && cls < 3 && s.groups == 1) {       // fragment layout: K rows word by word, V rows byte by byte
+        const bool frag = s.groups == 1 || s.groups == kLayoutPerChannelK;
+        // per-channel keys: a key row is packed only once its window of 16 slots is complete; until then it is an fp16 row
+        const bool open_window = s.groups == kLayoutPerChannelK && cls < 3 && tensor == 0 &&
+                                 (slot | (uint32_t)(kTileTokens - 1)) >= p.counts[(size_t)b * 4 + cls];
+        if (open_window) {
+            v = reinterpret_cast<const uint4*>(residual_rows(s, cls, p.layer, b, h) + t * kHeadDim)[j];
+        } else if (j < W && cls < 3 && frag) {         // fragment layout: K rows word by word, V rows byte by byte
             uint32_t w[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -69,15 +76,15 @@ k_export(ExportParams p) {
         }
         dst[(tok * s.kv_heads + h) * 8 + j] = v;
     }
-    const int G = s.groups;
+    const int G = s.groups == 2 ? 2 : 1;               // {scale, zero-point} pairs per row in the export format
     for (int it = threadIdx.x; it < s.kv_heads * 2 * G; it += blockDim.x) {
         const int g = it % G, tensor = (it / G) & 1, h = it / (2 * G);
         uint16_t* dst = tensor ? p.v_meta : p.k_meta;
         if (!dst) continue;
         uint32_t m = 0;
-        if (cls < 3) {
-            const uint8_t* rec = tile_ptr(s, cls, stream_table(s, cls, p.layer, b, h), (uint32_t)tile, G);
-            m = *reinterpret_cast<const uint32_t*>(rec + meta_offset(cls, tensor, t, g, G));
+        if (cls < 3 && !(s.groups == kLayoutPerChannelK && tensor == 0)) {      // (per-channel keys have no per-row pair)
+            const uint8_t* rec = tile_ptr(s, cls, stream_table(s, cls, p.layer, b, h), (uint32_t)tile, s.groups);
+            m = *reinterpret_cast<const uint32_t*>(rec + meta_offset(cls, tensor, t, g, s.groups));
         }
         dst[((tok * s.kv_heads + h) * G + g) * 2 + 0] = (uint16_t)(m & 0xffffu);
         dst[((tok * s.kv_heads + h) * G + g) * 2 + 1] = (uint16_t)(m >> 16);

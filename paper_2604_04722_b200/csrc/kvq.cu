@@ -38,6 +38,9 @@ struct kvq_ctx {
     uint32_t* table = nullptr;           // block tables of all streams
     uint32_t* arena_used = nullptr;      // device counter of blocks handed out
     uint32_t* counts = nullptr;          // [2][layers][batch][4], double-buffered pool fills
+    __half* kres = nullptr;              // per-channel keys: fp16 rows of the open windows (nullptr in the other layouts)
+    size_t kres_bytes = 0;
+    __half* kres_old = nullptr;          // copy of one layer's residual rows, taken before a multi-token append
     std::vector<int> len;                // host mirror: tokens of the longest sequence, per layer
     std::vector<int> lens;               // host mirror: tokens per (layer, sequence)
     std::vector<char> ragged;            // per layer: sequences differ in length
@@ -184,6 +187,8 @@ void free_all(kvq_ctx* c) {
     cudaFree(c->arena_used);
     cudaFree(c->store.index);
     cudaFree(c->counts);
+    cudaFree(c->kres);
+    cudaFree(c->kres_old);
     cudaFree(c->cls);
     cudaFree(c->hist);
     cudaFree(c->chunk_arrivals);
@@ -317,9 +322,21 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
 
     const size_t smem = fused ? controller_smem(c->hidden) : 0;
     dim3 grid_q(p.nchunks, groups, c->batch);
+    if (c->groups == kLayoutPerChannelK && !(n_new == 1 && !call_ragged) && c->len[layer] > 0) {
+        // Per-channel keys: the multi-token kernels read the rows of the windows left open by earlier calls from a
+        // copy, because the rows of each stream's next open window go to the same places during the launch.
+        const size_t slice = c->kres_bytes / c->layers;
+        KVQ_CUDA(c, cudaMemcpyAsync(c->kres_old, reinterpret_cast<const uint8_t*>(c->kres) + (size_t)layer * slice, slice,
+                                    cudaMemcpyDeviceToDevice, st));
+    }
     if (n_new == 1 && !call_ragged) {                  // a decode step: one warp per 16 heads
         dim3 grid_t((c->kv_heads + 15) / 16, c->batch);
-        if (c->groups == 1) {
+        if (c->groups == kLayoutPerChannelK) {         // keys wait as fp16 rows; a second small launch packs completed windows
+            if (fused) launch_overlapped(k_append_token<true, kLayoutPerChannelK>, grid_t, 32, 0, st, p);
+            else launch_overlapped(k_append_token<false, kLayoutPerChannelK>, grid_t, 32, 0, st, p);
+            k_pack_window<<<dim3(c->kv_heads, c->batch), 32, 0, st>>>(p);
+            c->launches += 1;
+        } else if (c->groups == 1) {
             if (fused) launch_overlapped(k_append_token<true, 1>, grid_t, 32, 0, st, p);
             else launch_overlapped(k_append_token<false, 1>, grid_t, 32, 0, st, p);
         } else {
@@ -328,7 +345,10 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
         }
         c->launches += 1;
     } else if (n_new <= kChunkTokens) {
-        if (c->groups == 1) {
+        if (c->groups == kLayoutPerChannelK) {
+            if (fused) k_quant_pack_frag<2, 1, true><<<grid_q, kChunkTokens, kFragRingBytes + smem, st>>>(p);
+            else k_quant_pack_frag<1, 1, true><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
+        } else if (c->groups == 1) {
             if (fused) k_quant_pack_frag<2><<<grid_q, kChunkTokens, kFragRingBytes + smem, st>>>(p);
             else k_quant_pack_frag<1><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
         } else {
@@ -341,10 +361,12 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
         if (fused) k_classify<true><<<grid_c, kChunkTokens, smem, st>>>(p);
         else k_classify<false><<<grid_c, kChunkTokens, 0, st>>>(p);
         if (p.tpt == 1) {
-            if (c->groups == 1) k_quant_pack_frag<0, 1><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
+            if (c->groups == kLayoutPerChannelK) k_quant_pack_frag<0, 1, true><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
+            else if (c->groups == 1) k_quant_pack_frag<0, 1><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
             else k_quant_pack<0, 2, 1><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
         } else {
-            if (c->groups == 1) k_quant_pack_frag<0, KVQ_APPEND_TOKENS_PER_THREAD><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
+            if (c->groups == kLayoutPerChannelK) k_quant_pack_frag<0, KVQ_APPEND_TOKENS_PER_THREAD, true><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
+            else if (c->groups == 1) k_quant_pack_frag<0, KVQ_APPEND_TOKENS_PER_THREAD><<<grid_q, kChunkTokens, kFragRingBytes, st>>>(p);
             else k_quant_pack<0, 2, KVQ_APPEND_TOKENS_PER_THREAD><<<grid_q, kChunkTokens, kAppendRingBytes, st>>>(p);
         }
         c->launches += 2;
@@ -511,7 +533,8 @@ template <bool STATS, class Geo>
 void launch_decode_geo(const kvq_ctx* c, const DecodeParams& p, cudaStream_t st) {
     const dim3 grid((p.gw + Geo::kWarps - 1) / Geo::kWarps);
     if (c->groups == 1) launch_overlapped(k_decode_attn<STATS, 1, Geo>, grid, Geo::kThreads, Geo::kSmemBytes, st, p);
-    else launch_overlapped(k_decode_attn<STATS, 2, Geo>, grid, Geo::kThreads, Geo::kSmemBytes, st, p);
+    else if (c->groups == 2) launch_overlapped(k_decode_attn<STATS, 2, Geo>, grid, Geo::kThreads, Geo::kSmemBytes, st, p);
+    else launch_overlapped(k_decode_attn<STATS, kLayoutPerChannelK, Geo>, grid, Geo::kThreads, Geo::kSmemBytes, st, p);
 }
 template <bool STATS>
 void launch_decode(const kvq_ctx* c, const DecodePlan& plan, const DecodeParams& p, cudaStream_t st) {
@@ -534,6 +557,7 @@ int export_impl(kvq_ctx* c, int layer, int b0, int nb, int pos0, int n, uint8_t*
     p.v_codes = static_cast<uint4*>(v_codes);
     p.k_meta = k_meta;
     p.v_meta = v_meta;
+    p.counts = counts_of(c, c->cur[layer], layer);
     k_export<<<dim3(n, nb), 128, 0, st>>>(p);
     c->launches += 1;
     KVQ_CUDA(c, cudaGetLastError());
@@ -559,12 +583,18 @@ int kvq_create_arena(kvq_ctx** out, int layers, int q_heads, int kv_heads, int h
 
 int kvq_create_grouped(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
                        uint64_t arena_bytes, int scale_groups) {
+    if (scale_groups != 1 && scale_groups != 2) return KVQ_ERR_ARG;
     return create_impl(out, layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes, scale_groups, 0, nullptr, 0, nullptr);
+}
+
+int kvq_create_perchannel(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
+                          uint64_t arena_bytes) {
+    return create_impl(out, layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes, kLayoutPerChannelK, 0, nullptr, 0, nullptr);
 }
 
 int kvq_workspace_bytes(int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch, uint64_t arena_bytes,
                         int scale_groups, uint64_t* bytes_out) {
-    if (!bytes_out) return KVQ_ERR_ARG;
+    if (!bytes_out || (scale_groups != 1 && scale_groups != 2)) return KVQ_ERR_ARG;
     kvq_ctx* none = nullptr;
     return create_impl(&none, layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes, scale_groups, 1, nullptr, 0,
                        bytes_out);
@@ -572,7 +602,7 @@ int kvq_workspace_bytes(int layers, int q_heads, int kv_heads, int head_dim, int
 
 int kvq_create_in(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_dim, int max_ctx, int batch,
                   uint64_t arena_bytes, int scale_groups, void* workspace, uint64_t workspace_bytes) {
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return KVQ_ERR_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 || (scale_groups != 1 && scale_groups != 2)) return KVQ_ERR_ARG;
     cudaPointerAttributes attr;                        // it has to be memory of a device, not of the host
     if (cudaPointerGetAttributes(&attr, workspace) != cudaSuccess) {
         cudaGetLastError();
@@ -592,7 +622,7 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
                 uint64_t* bytes_out) {
     if (!out) return KVQ_ERR_ARG;
     *out = nullptr;
-    if (scale_groups != 1 && scale_groups != 2) return KVQ_ERR_ARG;
+    if (scale_groups != 1 && scale_groups != 2 && scale_groups != kLayoutPerChannelK) return KVQ_ERR_ARG;
     if (layers < 1 || q_heads < 1 || kv_heads < 1 || batch < 1 || max_ctx < 1) return KVQ_ERR_ARG;
     if (head_dim != kHeadDim || q_heads % kv_heads != 0) return KVQ_ERR_ARG;
     if (max_ctx > (1 << 30) - 1 || batch > 65535 || q_heads > 65535) return KVQ_ERR_ARG;
@@ -653,6 +683,9 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
     ok = ok && dev_alloc(c, &c->arena_used, sizeof(uint32_t)) == cudaSuccess;
     ok = ok && dev_alloc(c, &s.index, sizeof(uint32_t) * (size_t)layers * batch * max_ctx) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->counts, sizeof(uint32_t) * 2 * (size_t)layers * batch * 4) == cudaSuccess;
+    c->kres_bytes = scale_groups == kLayoutPerChannelK ? sizeof(__half) * kResidualStreamHalves * streams : 0;
+    if (c->kres_bytes) ok = ok && dev_alloc(c, &c->kres, c->kres_bytes) == cudaSuccess;
+    if (c->kres_bytes) ok = ok && dev_alloc(c, &c->kres_old, c->kres_bytes / layers) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->cls, (size_t)batch * max_ctx) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->hist, sizeof(uint4) * batch * max_chunks) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->chunk_arrivals, sizeof(uint32_t) * batch) == cudaSuccess;
@@ -671,7 +704,7 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
     ok = ok && dev_alloc(c, &c->st_Q, sizeof(__half) * units * kHeadDim) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_O, sizeof(__half) * units * kHeadDim) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->st_bits, (size_t)batch) == cudaSuccess;
-    ok = ok && dev_alloc(c, &c->st_export, (size_t)kv_heads * (2 * KVQ_EXPORT_ROW_BYTES + 8 * scale_groups) + 16) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->st_export, (size_t)kv_heads * (2 * KVQ_EXPORT_ROW_BYTES + 8 * (scale_groups == 2 ? 2 : 1)) + 16) == cudaSuccess;
     if (ok && mem_mode == 1) {                         // only the size was asked for
         *bytes_out = c->slab_used;
         delete c;
@@ -684,6 +717,9 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
     }
     if (ok) {
         s.arena = c->arena;
+        s.kres = c->kres;
+        s.kres_old = c->kres_old;
+        if (c->kres_bytes) ok = ok && cudaMemset(c->kres, 0, c->kres_bytes) == cudaSuccess;
         s.table = c->table;
         s.arena_used = c->arena_used;
         s.flags = c->flags;
@@ -709,10 +745,16 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
              dyn_smem(k_quant_pack<0, 2, KVQ_APPEND_TOKENS_PER_THREAD>, ring);
         ok = ok && dyn_smem(k_quant_pack_frag<1>, fring) && dyn_smem(k_quant_pack<1, 2>, ring);
         ok = ok && dyn_smem(k_quant_pack_frag<2>, fring + smem_max) && dyn_smem(k_quant_pack<2, 2>, ring + smem_max);
+        ok = ok && dyn_smem(k_quant_pack_frag<0, 1, true>, fring) && dyn_smem(k_quant_pack_frag<0, KVQ_APPEND_TOKENS_PER_THREAD, true>, fring) &&
+             dyn_smem(k_quant_pack_frag<1, 1, true>, fring) && dyn_smem(k_quant_pack_frag<2, 1, true>, fring + smem_max);
         ok = ok && dyn_smem(k_decode_attn<false, 1, GeomLarge>, (int)GeomLarge::kSmemBytes) &&
              dyn_smem(k_decode_attn<false, 2, GeomLarge>, (int)GeomLarge::kSmemBytes);
         ok = ok && dyn_smem(k_decode_attn<true, 1, GeomLarge>, (int)GeomLarge::kSmemBytes) &&
              dyn_smem(k_decode_attn<true, 2, GeomLarge>, (int)GeomLarge::kSmemBytes);
+        ok = ok && dyn_smem(k_decode_attn<false, 3, GeomLarge>, (int)GeomLarge::kSmemBytes) &&
+             dyn_smem(k_decode_attn<true, 3, GeomLarge>, (int)GeomLarge::kSmemBytes) &&
+             dyn_smem(k_decode_attn<false, 3, GeomSmall>, (int)GeomSmall::kSmemBytes) &&
+             dyn_smem(k_decode_attn<true, 3, GeomSmall>, (int)GeomSmall::kSmemBytes);
         ok = ok && dyn_smem(k_decode_attn<false, 1, GeomSmall>, (int)GeomSmall::kSmemBytes) &&
              dyn_smem(k_decode_attn<false, 2, GeomSmall>, (int)GeomSmall::kSmemBytes);
         ok = ok && dyn_smem(k_decode_attn<true, 1, GeomSmall>, (int)GeomSmall::kSmemBytes) &&
@@ -856,6 +898,7 @@ int kvq_token_features(const void* logits, int logits_are_fp32, int n, int vocab
 
 int kvq_attend_last(kvq_ctx* c, int layer, const void* Q, void* O, int n_queries, void* stream) {
     if (check_layer(c, layer) != KVQ_OK || !Q || !O || n_queries < 1) return KVQ_ERR_ARG;
+    if (c->groups == kLayoutPerChannelK && n_queries > 1) return KVQ_ERR_ARG;   // an earlier row would see windows packed later
     if (c->len[layer] == 0) return KVQ_ERR_EMPTY;
     if (n_queries > min_len(c, layer)) return KVQ_ERR_ARG;
     DeviceGuard guard(c->device);
@@ -1024,7 +1067,7 @@ int kvq_export_token(kvq_ctx* c, int layer, int b, int pos, uint8_t* bits, uint3
         pos >= c->lens[(size_t)layer * c->batch + (b < 0 || b >= c->batch ? 0 : b)])
         return KVQ_ERR_ARG;
     DeviceGuard guard(c->device);
-    const size_t row = (size_t)c->kv_heads * KVQ_EXPORT_ROW_BYTES, meta = (size_t)c->kv_heads * 4 * c->groups;
+    const size_t row = (size_t)c->kv_heads * KVQ_EXPORT_ROW_BYTES, meta = (size_t)c->kv_heads * 4 * (c->groups == 2 ? 2 : 1);
     uint8_t* d_k = c->st_export;
     uint8_t* d_v = d_k + row;
     uint8_t* d_km = d_v + row;
@@ -1041,6 +1084,23 @@ int kvq_export_token(kvq_ctx* c, int layer, int b, int pos, uint8_t* bits, uint3
     if (pool_slot) KVQ_CUDA(c, cudaMemcpy(pool_slot, d_ps, 4, cudaMemcpyDeviceToHost));
     if (bits) KVQ_CUDA(c, cudaMemcpy(bits, d_ps + 4, 1, cudaMemcpyDeviceToHost));
     KVQ_CUDA(c, cudaDeviceSynchronize());
+    return KVQ_OK;
+}
+
+int kvq_export_k_channels(kvq_ctx* c, int layer, int b, int kv_head, int bits, int window, uint16_t* host_meta) {
+    if (check_layer(c, layer) != KVQ_OK || !host_meta || c->groups != kLayoutPerChannelK) return KVQ_ERR_ARG;
+    const int cls = bits == 2 ? 0 : bits == 4 ? 1 : bits == 8 ? 2 : -1;
+    if (cls < 0 || b < 0 || b >= c->batch || kv_head < 0 || kv_head >= c->kv_heads || window < 0) return KVQ_ERR_ARG;
+    DeviceGuard guard(c->device);
+    KVQ_CUDA(c, cudaDeviceSynchronize());
+    uint32_t fill[4];
+    KVQ_CUDA(c, cudaMemcpy(fill, counts_of(c, c->cur[layer], layer) + (size_t)b * 4, sizeof(fill), cudaMemcpyDeviceToHost));
+    if ((uint64_t)(window + 1) * kTileTokens > fill[cls]) return KVQ_ERR_ARG;           // the window is not complete
+    const uint32_t bt = block_tiles(cls, kLayoutPerChannelK);
+    uint32_t id = 0;
+    KVQ_CUDA(c, cudaMemcpy(&id, stream_table(c->store, cls, layer, b, kv_head) + (uint32_t)window / bt, sizeof(id), cudaMemcpyDeviceToHost));
+    const uint8_t* rec = c->arena + (size_t)id * kBlockBytes + (size_t)((uint32_t)window % bt) * pool_rec_bytes(cls, kLayoutPerChannelK);
+    KVQ_CUDA(c, cudaMemcpy(host_meta, rec + chan_meta_offset(cls, 0), 4 * kHeadDim, cudaMemcpyDeviceToHost));
     return KVQ_OK;
 }
 
@@ -1109,7 +1169,7 @@ int state_header(kvq_ctx* c, StateHeader& h) {
     h.counts_bytes = sizeof(uint32_t) * 2 * (uint64_t)c->layers * c->batch * 4;
     const uint64_t host_ints = (uint64_t)c->layers * 3 + (uint64_t)c->layers * c->batch;
     h.total_bytes = sizeof(StateHeader) + sizeof(int32_t) * host_ints + (uint64_t)(used + 1) * kBlockBytes + h.table_bytes +
-                    h.index_bytes + h.counts_bytes;
+                    h.index_bytes + h.counts_bytes + c->kres_bytes;
     return KVQ_OK;
 }
 }  // namespace
@@ -1152,6 +1212,8 @@ int kvq_save_state(kvq_ctx* c, void* host_buf, uint64_t host_bytes) {
     KVQ_CUDA(c, cudaMemcpy(out, c->store.index, h.index_bytes, cudaMemcpyDeviceToHost));
     out += h.index_bytes;
     KVQ_CUDA(c, cudaMemcpy(out, c->counts, h.counts_bytes, cudaMemcpyDeviceToHost));
+    out += h.counts_bytes;
+    if (c->kres_bytes) KVQ_CUDA(c, cudaMemcpy(out, c->kres, c->kres_bytes, cudaMemcpyDeviceToHost));
     return KVQ_OK;
 }
 
@@ -1172,7 +1234,7 @@ int kvq_load_state(kvq_ctx* c, const void* host_buf, uint64_t host_bytes) {
         return KVQ_ERR_ARG;
     const uint64_t host_ints = (uint64_t)c->layers * 3 + (uint64_t)c->layers * c->batch;
     if (h.total_bytes != sizeof(StateHeader) + sizeof(int32_t) * host_ints + ((uint64_t)h.blocks_used + 1) * kBlockBytes +
-                             h.table_bytes + h.index_bytes + h.counts_bytes)
+                             h.table_bytes + h.index_bytes + h.counts_bytes + c->kres_bytes)
         return KVQ_ERR_ARG;
     const uint8_t* in = static_cast<const uint8_t*>(host_buf) + sizeof(h);
     auto get_int = [&]() {
@@ -1256,6 +1318,8 @@ int kvq_load_state(kvq_ctx* c, const void* host_buf, uint64_t host_bytes) {
     KVQ_CUDA(c, cudaMemcpy(c->store.index, in, h.index_bytes, cudaMemcpyHostToDevice));
     in += h.index_bytes;
     KVQ_CUDA(c, cudaMemcpy(c->counts, in, h.counts_bytes, cudaMemcpyHostToDevice));
+    in += h.counts_bytes;
+    if (c->kres_bytes) KVQ_CUDA(c, cudaMemcpy(c->kres, in, c->kres_bytes, cudaMemcpyHostToDevice));
     KVQ_CUDA(c, cudaMemcpy(c->arena_used, &h.blocks_used, sizeof(uint32_t), cudaMemcpyHostToDevice));
     KVQ_CUDA(c, cudaMemset(c->flags, 0, sizeof(uint32_t)));
     return KVQ_OK;

@@ -49,12 +49,22 @@ __host__ __device__ constexpr int pool_half_bytes(int c) { return 8 << c; }     
 __host__ __device__ constexpr int pool_unit_bytes(int c) { return c == 0 ? 8 : 16; }
 __host__ __device__ constexpr int pool_units(int c) { return pool_half_bytes(c) / pool_unit_bytes(c); }   // 1,1,2,4
 __host__ __device__ constexpr int pool_codes_bytes(int c) { return 2 * pool_half_bytes(c) * kTileTokens; }  // per tile, per tensor
-// Scale groups g: 1 = one {scale, zero-point} pair per row (the default), 2 = one pair per half-row (32
-// channels), stored as two planes of 16 words per tensor: [K half 0][K half 1][V half 0][V half 1].
-__host__ __device__ constexpr int pool_meta_bytes(int c, int g = 1) { return pool_has_meta(c) ? 4 * kTileTokens * g : 0; }  // per tile, per tensor
-__host__ __device__ constexpr int pool_rec_bytes(int c, int g = 1) { return 2 * pool_codes_bytes(c) + 2 * pool_meta_bytes(c, g); }
+// Layout id g of a cache.  1 = one {scale, zero-point} pair per row (the default); 2 = one pair per half-row (32
+// channels), stored as two planes of 16 words per tensor: [K half 0][K half 1][V half 0][V half 1]; 3 = keys
+// quantized per CHANNEL over the 16 slots of a tile: [K: 64 channels x {scale, zero-point}][V: 16 slots x {..}].
+constexpr int kLayoutPerChannelK = 3;
+__host__ __device__ constexpr int pool_kmeta_bytes(int c, int g = 1) {
+    return !pool_has_meta(c) ? 0 : g == kLayoutPerChannelK ? 4 * kHeadDim : 4 * kTileTokens * g;
+}
+__host__ __device__ constexpr int pool_vmeta_bytes(int c, int g = 1) {
+    return !pool_has_meta(c) ? 0 : g == kLayoutPerChannelK ? 4 * kTileTokens : 4 * kTileTokens * g;
+}
+__host__ __device__ constexpr int pool_meta_bytes(int c, int g = 1) { return pool_vmeta_bytes(c, g); }   // per tile, V tensor (and K, layouts 1 and 2)
+__host__ __device__ constexpr int pool_rec_bytes(int c, int g = 1) {
+    return 2 * pool_codes_bytes(c) + pool_kmeta_bytes(c, g) + pool_vmeta_bytes(c, g);
+}
 __host__ __device__ constexpr int pool_row_bytes(int c, int g = 1) {             // K+V bytes per (token, KV head)
-    return pool_rec_bytes(c, g) / kTileTokens;                                   // 40, 72, 136, 256 (g = 2: 48, 80, 144, 256)
+    return pool_rec_bytes(c, g) / kTileTokens;                                   // 40, 72, 136, 256 (g = 2: 48, 80, 144, 256; g = 3: 52, 84, 148, 256)
 }
 // Byte offset, inside one tensor's code block of a tile, of unit u of half h of slot t.
 __host__ __device__ constexpr int unit_offset(int c, int h, int u, int t) {
@@ -63,8 +73,10 @@ __host__ __device__ constexpr int unit_offset(int c, int h, int u, int t) {
 // Byte offset, inside the record, of the {scale, zero-point} pair of slot t (tensor 0 = K, 1 = V).
 // With two scale groups `half` picks the plane of the half-row.
 __host__ __device__ constexpr int meta_offset(int c, int tensor, int t, int half = 0, int g = 1) {
-    return 2 * pool_codes_bytes(c) + tensor * pool_meta_bytes(c, g) + (g == 2 ? half * 4 * kTileTokens : 0) + 4 * t;
+    return 2 * pool_codes_bytes(c) + tensor * pool_kmeta_bytes(c, g) + (g == 2 ? half * 4 * kTileTokens : 0) + 4 * t;
 }
+// Per-channel keys: the {scale, zero-point} pair of channel i of the tile.
+__host__ __device__ constexpr int chan_meta_offset(int c, int i) { return 2 * pool_codes_bytes(c) + 4 * i; }
 
 // ---- Fragment layout of the quantized classes (caches with one scale group per row).
 //
@@ -111,9 +123,15 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 constexpr uint32_t kBlockBytes = 65536;
 // Tiles per block: a whole number of ring stages of the decode kernel (10 / 5 / 3 / 1 tiles).
 // (with two scale groups the records are 768 / 1280 / 2304 / 4096 bytes: 80 / 50 / 28 / 16 tiles)
+// (per-channel keys: 832 / 1344 / 2368 / 4096 bytes: 78 / 48 / 27 / 16 tiles)
 __host__ __device__ constexpr uint32_t block_tiles(int c, int g = 1) {
-    return g == 2 ? (c == 0 ? 80u : c == 1 ? 50u : c == 2 ? 28u : 16u) : (c == 0 ? 100u : c == 1 ? 55u : c == 2 ? 30u : 16u);
+    return g == 2   ? (c == 0 ? 80u : c == 1 ? 50u : c == 2 ? 28u : 16u)
+           : g == 3 ? (c == 0 ? 78u : c == 1 ? 48u : c == 2 ? 27u : 16u)
+                    : (c == 0 ? 100u : c == 1 ? 55u : c == 2 ? 30u : 16u);
 }
+// Per-channel keys: the fp16 key rows of the open (incomplete) window of every quantized stream wait here until the
+// window fills: [stream][class 0..2][slot 0..15][64].
+constexpr size_t kResidualStreamHalves = 3 * kTileTokens * kHeadDim;
 constexpr uint32_t kFlagArenaFull = 4u;
 
 // Everything a kernel needs to find a row.
@@ -123,7 +141,9 @@ struct StoreView {
     uint32_t* arena_used;         // blocks handed out so far (block ids are 1 + the old value)
     uint32_t arena_blocks;        // capacity in blocks, block 0 included
     uint32_t table_stride, table_off[kNumPools];
-    int groups;                   // scale groups per row: 1 or 2
+    int groups;                   // layout id: 1 or 2 scale groups per row, or kLayoutPerChannelK
+    __half* kres;                 // per-channel keys: residual rows (nullptr otherwise)
+    __half* kres_old;             // ... and a copy of the current layer's, taken before a multi-token append
     uint32_t* index;              // [layers][batch][max_ctx]   pool<<30 | slot
     uint32_t* flags;              // device flag word
     int layers, batch, kv_heads, q_heads, max_ctx, cap_tiles;
@@ -148,6 +168,15 @@ __device__ __forceinline__ uint32_t arena_take(const StoreView& s, uint32_t n) {
         return 0u;
     }
     return first;
+}
+// Residual rows of class c of stream (layer, b, h).
+__host__ __device__ inline __half* residual_rows(const StoreView& s, int c, int layer, int b, int h) {
+    const size_t stream = ((size_t)layer * s.batch + b) * s.kv_heads + h;
+    return s.kres + stream * kResidualStreamHalves + (size_t)c * kTileTokens * kHeadDim;
+}
+// The copy of the residual rows of class c of stream (b, h) of the layer being appended to (see kres_old).
+__host__ __device__ inline const __half* residual_rows_before(const StoreView& s, int c, int b, int h) {
+    return s.kres_old + ((size_t)b * s.kv_heads + h) * kResidualStreamHalves + (size_t)c * kTileTokens * kHeadDim;
 }
 // Blocks a stream of class c needs for n tokens.
 __host__ __device__ constexpr uint32_t blocks_for(int c, uint32_t n, int g = 1) {

@@ -24,10 +24,13 @@ def dev(a: np.ndarray) -> torch.Tensor:
 class GpuCache:
     """A kvq handle plus the shapes needed to size export buffers."""
 
-    def __init__(self, layers, batch, q_heads, kv_heads, max_ctx, head_dim=64, scale_groups=1, arena_bytes=0):
+    def __init__(self, layers, batch, q_heads, kv_heads, max_ctx, head_dim=64, scale_groups=1, arena_bytes=0,
+                 k_per_channel=False):
         self.L, self.B, self.Hq, self.Hkv, self.max_ctx = layers, batch, q_heads, kv_heads, max_ctx
         self.G = scale_groups
-        if scale_groups == 1 and arena_bytes == 0:
+        if k_per_channel:
+            self.ctx = kq.kvq_create_perchannel(layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes)
+        elif scale_groups == 1 and arena_bytes == 0:
             self.ctx = kq.kvq_create(layers, q_heads, kv_heads, head_dim, max_ctx, batch)
         else:
             self.ctx = kq.kvq_create_grouped(layers, q_heads, kv_heads, head_dim, max_ctx, batch, arena_bytes,
