@@ -635,16 +635,18 @@ __device__ __forceinline__ void token_store_pc(int c, const uint4 (&kraw)[4], co
     }
 }
 
-// One new token per sequence (a decode step): grid = (ceil(kv_heads / 16), batch), block = 32.
+// One new token per sequence (a decode step): grid = (ceil(kv_heads / 16), batch), block = 32 -- or 128 when the
+// controller is wider than 32 hidden units: the three extra warps only help with the decision.
 // Lane l handles half-row l%2 of KV head 16*blockIdx.x + l/2.  Everything the warp needs (the K and V
 // rows, the pool fills, the features) is requested up front so the loads overlap the controller;
 // the decision is taken by the whole warp (FUSED, any hidden width) or read from `bits`.
 template <bool FUSED, int G>
-__global__ void __launch_bounds__(32)
+__global__ void __launch_bounds__(128)
 k_append_token(AppendParams p) {
+    __shared__ float ctrl_sh[2 * kMaxHidden];
     pdl_launch_dependents();
     pdl_wait();                                        // the attention of the previous step still reads the store
-    const int lane = threadIdx.x, b = blockIdx.y;
+    const int lane = threadIdx.x & 31, b = blockIdx.y;
     const int h = blockIdx.x * 16 + (lane >> 1), half = lane & 1;
     const bool active = h < p.store.kv_heads;
     uint4 kraw[4], vraw[4];
@@ -672,8 +674,9 @@ k_append_token(AppendParams p) {
     int c;
     if (FUSED) {
         const float4 f = reinterpret_cast<const float4*>(p.feats)[b];
-        c = p.hidden == 32 ? controller_decide_warp32(p.ctrl, f.x, f.y, f.z, f.w, lane)
-                           : controller_decide_warp(p.ctrl, p.hidden, f.x, f.y, f.z, f.w, lane);
+        c = blockDim.x == 32 ? controller_decide_warp32(p.ctrl, f.x, f.y, f.z, f.w, lane)
+                             : controller_decide_cta128(p.ctrl, p.hidden, f.x, f.y, f.z, f.w, ctrl_sh);
+        if (threadIdx.x >= 32) return;                 // the helpers are done
     } else {
         c = class_of_bits(p.bits[b], p.store.flags);
     }

@@ -122,74 +122,71 @@ __device__ __forceinline__ int controller_decide_warp32(const float* __restrict_
     return cls;
 }
 
-// The same for any hidden width H <= kMaxHidden (the paper's 128 included): lane l owns the hidden units l, l + 32,
-// l + 64, l + 96.  Rows of W2 are streamed from global memory four inputs at a time while the first-layer outputs
-// come round by shuffle; every sum still runs in ascending input order with separately rounded products and sums.
-__device__ __forceinline__ int controller_decide_warp(const float* __restrict__ gW, int H, float x0, float x1, float x2,
-                                                      float x3, int lane) {
-    constexpr int M = kMaxHidden / 32;
+// The same decision taken by a CTA of 128 threads for ONE token, any hidden width H <= 128: thread j owns hidden
+// unit j.  First- and second-layer outputs cross shared memory (sh: 2 * kMaxHidden floats), every thread streams its
+// own row of W2 sixteen inputs ahead of their use; all sums in ascending input order with separately rounded
+// products and sums, so the result is bit-identical to controller_decide.  Every thread of the CTA must call it;
+// returns the class in every thread.
+__device__ __forceinline__ int controller_decide_cta128(const float* __restrict__ gW, int H, float x0, float x1, float x2,
+                                                        float x3, float* sh) {
+    const int j = threadIdx.x;
     const float* W1 = gW;
     const float* b1 = W1 + 4 * H;
     const float* W2 = b1 + H;
     const float* b2 = W2 + H * H;
     const float* W3 = b2 + H;
     const float* b3 = W3 + 4 * H;
-    float h1[M], acc[M];
-#pragma unroll
-    for (int m = 0; m < M; ++m) {
-        const int j = lane + 32 * m;
-        h1[m] = 0.0f;
-        acc[m] = 0.0f;
-        if (j < H) {
-            float a = __ldg(b1 + j);
-            a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 0), x0));
-            a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 1), x1));
-            a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 2), x2));
-            a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 3), x3));
-            h1[m] = a > 0.0f ? a : 0.0f;
-            acc[m] = __ldg(b2 + j);
-        }
-    }
-    const bool vec = (H & 3) == 0;                     // rows of W2 are then 16-byte aligned
-    for (int i0 = 0; i0 < H; i0 += 4) {
-        float w[M][4];
-#pragma unroll
-        for (int m = 0; m < M; ++m) {
-            const int j = lane + 32 * m;
-            w[m][0] = w[m][1] = w[m][2] = w[m][3] = 0.0f;
-            if (j < H) {
-                if (vec) {
-                    const float4 v = __ldg(reinterpret_cast<const float4*>(W2 + (size_t)j * H + i0));
-                    w[m][0] = v.x; w[m][1] = v.y; w[m][2] = v.z; w[m][3] = v.w;
-                } else {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (i0 + k < H) w[m][k] = __ldg(W2 + (size_t)j * H + i0 + k);
-                }
-            }
-        }
+    float* h1s = sh;
+    float* h2s = sh + kMaxHidden;
+    const bool mine = j < H;
+    const bool vec = (H & 3) == 0;
+    const float* row = W2 + (size_t)(mine ? j : 0) * H;
+    float4 cur[4], nxt[4];                             // sixteen weights of the row in use, sixteen on their way
+    auto fetch = [&](int i0, float4 (&w)[4]) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const int i = i0 + k;                      // warp-uniform
-            if (i >= H) break;
-            float src = h1[0];
-#pragma unroll
-            for (int m = 1; m < M; ++m) src = (i >> 5) == m ? h1[m] : src;
-            const float v = __shfl_sync(0xffffffffu, src, i & 31);
-#pragma unroll
-            for (int m = 0; m < M; ++m) acc[m] = __fadd_rn(acc[m], __fmul_rn(w[m][k], v));
+            const int i = i0 + 4 * k;
+            if (vec && i < H) {
+                w[k] = __ldg(reinterpret_cast<const float4*>(row + i));
+            } else {
+                w[k].x = i + 0 < H ? __ldg(row + i + 0) : 0.f;
+                w[k].y = i + 1 < H ? __ldg(row + i + 1) : 0.f;
+                w[k].z = i + 2 < H ? __ldg(row + i + 2) : 0.f;
+                w[k].w = i + 3 < H ? __ldg(row + i + 3) : 0.f;
+            }
         }
+    };
+    fetch(0, cur);
+    float acc = 0.f;
+    if (mine) {
+        float a = __ldg(b1 + j);
+        a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 0), x0));
+        a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 1), x1));
+        a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 2), x2));
+        a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 3), x3));
+        h1s[j] = a > 0.0f ? a : 0.0f;
+        acc = __ldg(b2 + j);
     }
-    float h2[M];
+    __syncthreads();
+    for (int i0 = 0; i0 < H; i0 += 16) {
+        if (i0 + 16 < H) fetch(i0 + 16, nxt);
 #pragma unroll
-    for (int m = 0; m < M; ++m) h2[m] = acc[m] > 0.0f ? acc[m] : 0.0f;
-    float o = __ldg(b3 + (lane & 3));                  // lanes 0..3 hold the four logits (the others mirror them)
-    for (int j = 0; j < H; ++j) {
-        float src = h2[0];
+        for (int k = 0; k < 4; ++k) {
+            const int i = i0 + 4 * k;
+            if (i + 0 < H) acc = __fadd_rn(acc, __fmul_rn(cur[k].x, h1s[i + 0]));
+            if (i + 1 < H) acc = __fadd_rn(acc, __fmul_rn(cur[k].y, h1s[i + 1]));
+            if (i + 2 < H) acc = __fadd_rn(acc, __fmul_rn(cur[k].z, h1s[i + 2]));
+            if (i + 3 < H) acc = __fadd_rn(acc, __fmul_rn(cur[k].w, h1s[i + 3]));
+        }
 #pragma unroll
-        for (int m = 1; m < M; ++m) src = (j >> 5) == m ? h2[m] : src;
-        o = __fadd_rn(o, __fmul_rn(__ldg(W3 + (lane & 3) * H + j), __shfl_sync(0xffffffffu, src, j & 31)));
+        for (int k = 0; k < 4; ++k) cur[k] = nxt[k];
     }
+    if (mine) h2s[j] = acc > 0.0f ? acc : 0.0f;
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    float o = __ldg(b3 + (lane & 3));                  // lanes 0..3 of every warp hold the four logits
+    const float* w3 = W3 + (lane & 3) * H;
+    for (int i = 0; i < H; ++i) o = __fadd_rn(o, __fmul_rn(__ldg(w3 + i), h2s[i]));
     const float o0 = __shfl_sync(0xffffffffu, o, 0), o1 = __shfl_sync(0xffffffffu, o, 1);
     const float o2 = __shfl_sync(0xffffffffu, o, 2), o3 = __shfl_sync(0xffffffffu, o, 3);
     if (o0 != o0 || o1 != o1 || o2 != o2 || o3 != o3) return 3;

@@ -55,6 +55,12 @@
 #pragma once
 #include "kvq_common.cuh"
 
+#ifndef KVQ_SMALL_WARPS
+#define KVQ_SMALL_WARPS 16
+#endif
+#ifndef KVQ_SMALL_STAGES
+#define KVQ_SMALL_STAGES 3
+#endif
 #ifndef KVQ_DECODE_FMA2
 #define KVQ_DECODE_FMA2 1          // fp16 pool: V-side accumulation with packed two-lane fp32 FMAs
 #endif
@@ -64,7 +70,7 @@ namespace kvq {
 // Launch geometry.  The kernel is instantiated twice:
 //   Large: 4 warps per CTA, 4 CTAs per SM, per-warp rings of two 6.5 KB stages -- the bandwidth configuration
 //          (16 resident warps per SM, 209 KB of rings);
-//   Small: 8 warps per CTA, 1 CTA per SM, per-warp rings of four 4.25 KB stages -- for launches of few warps,
+//   Small: 16 warps per CTA, 1 CTA per SM, per-warp rings of three 4.25 KB stages -- for launches of few warps,
 //          where a warp's whole share is in flight at once and the parts of a (sequence, query head) unit sit in
 //          one CTA, which merges them through shared memory (no partial records, no global counter).
 template <int WARPS, int STAGES, int STAGE_BYTES, int MIN_CTAS>
@@ -77,7 +83,7 @@ struct DecodeGeom {
     static_assert(STAGE_BYTES % 16 == 0 && STAGE_BYTES >= pool_rec_bytes(3), "a stage must hold one fp16 tile");
 };
 using GeomLarge = DecodeGeom<4, 2, 6528, 4>;          // 10 / 5 / 3 / 1 tiles of the four classes per stage
-using GeomSmall = DecodeGeom<8, 4, 4352, 1>;          //  6 / 3 / 2 / 1
+using GeomSmall = DecodeGeom<KVQ_SMALL_WARPS, KVQ_SMALL_STAGES, 4352, 1>;    //  6 / 3 / 2 / 1
 
 constexpr int kHalfDim = kHeadDim / 2;           // elements per lane
 constexpr float kLog2e = 1.4426950408889634f;
@@ -785,9 +791,9 @@ struct alignas(16) WarpScratch {
     int lo[kNumPools], hi[kNumPools];  // tile range of the segment in each pool
     uint32_t cnt[kNumPools];           // tokens in each pool
     uint32_t id[kNumPools];            // arena block that holds tile lo of each pool
-    float q[kHeadDim + 4];             // query row; half 1 starts at q[36] so the two halves sit in different banks
-    uint32_t x[2][2 * kTileTokens];    // fragment path: the value weights of a pair of tiles on the integer grid (two pairs alternate)
-    float o[kHeadDim];                 // the segment's output row (fragment path: gathered from the lanes that own channels;
+    alignas(16) float q[kHeadDim + 4]; // query row; half 1 starts at q[36] so the two halves sit in different banks
+    alignas(16) uint32_t x[2][2 * kTileTokens];    // (read 16 bytes at a time) fragment path: the value weights of a pair of tiles on the integer grid (two pairs alternate)
+    alignas(16) float o[kHeadDim];     // the segment's output row (fragment path: gathered from the lanes that own channels;
                                        // CTA merge: this warp's partial)
     float2 ml;                         // CTA merge: this warp's (m, l)
     float s2;                          //            and its sum of squared weights

@@ -331,17 +331,18 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
     }
     if (n_new == 1 && !call_ragged) {                  // a decode step: one warp per 16 heads
         dim3 grid_t((c->kv_heads + 15) / 16, c->batch);
+        const unsigned bt = fused && c->hidden != 32 ? 128 : 32;   // a controller of another width is evaluated by four warps
         if (c->groups == kLayoutPerChannelK) {         // keys wait as fp16 rows; a second small launch packs completed windows
-            if (fused) launch_overlapped(k_append_token<true, kLayoutPerChannelK>, grid_t, 32, 0, st, p);
-            else launch_overlapped(k_append_token<false, kLayoutPerChannelK>, grid_t, 32, 0, st, p);
+            if (fused) launch_overlapped(k_append_token<true, kLayoutPerChannelK>, grid_t, bt, 0, st, p);
+            else launch_overlapped(k_append_token<false, kLayoutPerChannelK>, grid_t, bt, 0, st, p);
             k_pack_window<<<dim3(c->kv_heads, c->batch), 32, 0, st>>>(p);
             c->launches += 1;
         } else if (c->groups == 1) {
-            if (fused) launch_overlapped(k_append_token<true, 1>, grid_t, 32, 0, st, p);
-            else launch_overlapped(k_append_token<false, 1>, grid_t, 32, 0, st, p);
+            if (fused) launch_overlapped(k_append_token<true, 1>, grid_t, bt, 0, st, p);
+            else launch_overlapped(k_append_token<false, 1>, grid_t, bt, 0, st, p);
         } else {
-            if (fused) launch_overlapped(k_append_token<true, 2>, grid_t, 32, 0, st, p);
-            else launch_overlapped(k_append_token<false, 2>, grid_t, 32, 0, st, p);
+            if (fused) launch_overlapped(k_append_token<true, 2>, grid_t, bt, 0, st, p);
+            else launch_overlapped(k_append_token<false, 2>, grid_t, bt, 0, st, p);
         }
         c->launches += 1;
     } else if (n_new <= kChunkTokens) {
@@ -402,6 +403,9 @@ constexpr int kMaxQueryRows = 8;       // query rows per sequence that one launc
 
 size_t max_partial_records(const kvq_ctx* c);
 
+#ifndef KVQ_SMALL_MAX_TILES_PER_WARP
+#define KVQ_SMALL_MAX_TILES_PER_WARP 40
+#endif
 // A launch plan: working warps, geometry, and (small geometry) parts per unit merged inside the CTA.
 struct DecodePlan {
     uint32_t gw = 0;
@@ -416,7 +420,7 @@ DecodePlan choose_plan(kvq_ctx* c, int len, uint64_t units, uint64_t room = 0) {
     if (room == 0) room = max_partial_records(c);
     auto fits = [&](uint64_t gw) { return units * (uint64_t)decode_pslots((uint32_t)units, (uint32_t)gw) <= room; };
     const uint64_t small_resident = (uint64_t)GeomSmall::kWarps * GeomSmall::kCtasPerSm * c->sm_count;
-    auto cta_mergeable = [&](uint64_t parts) { return parts == 1 || parts == 2 || parts == 4 || parts == 8; };
+    auto cta_mergeable = [&](uint64_t parts) { return parts >= 1 && parts <= (uint64_t)GeomSmall::kWarps && GeomSmall::kWarps % parts == 0; };
     if (c->splits_override > 0) {
         const uint64_t parts = (uint64_t)c->splits_override, gw = units * parts;
         if (gw <= small_resident && cta_mergeable(parts)) {
@@ -438,11 +442,11 @@ DecodePlan choose_plan(kvq_ctx* c, int len, uint64_t units, uint64_t room = 0) {
     if (tiles / 4 <= resident) {
         // A short cache is a chain of latencies, not a stream: a warp walks a tile in about kTileUs, parts merged
         // inside their CTA cost about kCtaMergeUs, parts merged through global partial records about kGlobalMergeUs
-        // (measured on warps' own timestamps).  Take the cheaper of: 8 / 4 / 2 / 1 parts per unit in the small
+        // (measured on warps' own timestamps).  Take the cheaper of: 16 / 8 / 4 / 2 / 1 parts per unit in the small
         // geometry, or as many parts as leave a warp four tiles, merged globally.
         const double kTileUs = 0.3, kCtaMergeUs = 0.5, kGlobalMergeUs = 3.0;
         double best_cost = 1e30;
-        for (uint64_t parts = 8; parts >= 1; parts /= 2) {
+        for (uint64_t parts = GeomSmall::kWarps; parts >= 1; parts /= 2) {
             if (units * parts > small_resident) continue;
             const double cost = kTileUs * (double)((tiles_per_unit + parts - 1) / parts) + kCtaMergeUs;
             if (cost < best_cost) {
@@ -464,6 +468,15 @@ DecodePlan choose_plan(kvq_ctx* c, int len, uint64_t units, uint64_t room = 0) {
             }
         }
         return plan;
+    }
+    {
+        const uint64_t parts = GeomSmall::kWarps;
+        if (units * parts <= small_resident && tiles_per_unit / parts <= KVQ_SMALL_MAX_TILES_PER_WARP) {
+            plan.gw = (uint32_t)(units * parts);       // a medium cache of few units: one CTA per unit, merged in shared memory
+            plan.small = true;
+            plan.cta_parts = (uint32_t)parts;
+            return plan;
+        }
     }
     if (!fits(units)) return plan;
     uint64_t cap = tiles / 8;
