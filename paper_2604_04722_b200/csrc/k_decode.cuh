@@ -26,32 +26,27 @@
 // mbarrier wait is bounded: on expiry the warp records KVQ_FLAG_WAIT_TIMEOUT
 // and stops.
 //
-// Work layout inside a warp: two lanes per token.  Lane l handles half l/16
-// (elements 32*(l/16) .. +32) of slot l%16 of a 16-token tile, so it keeps 32
-// pre-scaled query values and 32 output accumulators in registers (16 warps
-// stay resident per SM and hide the latency of the dependent FMA chains).  The
-// two half dot products meet through one xor-16 shuffle; the output
-// accumulators are per-lane partial sums reduced once per segment.
-//
-// Dequantization is hoisted out of the inner loops:
+// Arithmetic.  Dequantization is hoisted out of the inner loops:
 //   q.khat = s_k * sum_i q_i c_i + z_k * sum_i q_i
 //   sum_t p_t vhat_t = sum_t (p_t s_t) c_t + sum_t p_t z_t
+// so both sides are sums of products of small unsigned codes with a weight.
 //
-// K side: sum_i q_i c_i is an integer dot product.  q is put on a 24-bit fixed-point grid once
-// per segment: T_i = rint(q_i * 256 R), R the power of two that brings max|q| R just below 2^15
-// (an error below 2^-24 of max|q| per element, so elements up to 2^13 times smaller than the
-// largest keep fp16's own 11 bits), and T_i = 256 * hi_i + lo_i with a signed 16-bit hi and a
-// signed 8-bit lo.  The codes are masked IN PLACE into byte lanes (2-bit: four masks
-// 0x03030303 << 2k per word, 4-bit: two masks, 8-bit: none); dp2a multiplies two hi values by
-// two code bytes, dp4a four lo values by four code bytes, both accumulate exactly in int32, and
-// the planes' weights 4^k / 16^k are undone by a Horner step on the integer sums.  That is about
-// 1 / 1 / 0.75 issue slots per element instead of 2, on fewer of the half-rate integer ALU slots.
+// Caches with one {scale, zero-point} pair per row, and caches with per-channel keys, run both sums on the 8-bit
+// integer matrix instructions (FragRows below): the packed codes are the row operand as they are stored
+// (kvq_common.cuh stores them in operand order), byte planes cut out with one mask each, and the weights -- the
+// query for K, the softmax weights times the value scales for V -- are the column operand as balanced / unsigned
+// base-256 digits of a fixed-point number, one digit per column, int32 accumulation.  Two 16-slot tiles per
+// iteration, every lane owning one slot's logit and weight.
 //
-// V side: the integer codes enter fp32 FMAs without any int->float conversion: a bit field of a
-// packed word that lies inside bits [0,24) of a 32-bit word, read as an fp32 bit pattern, IS the
-// number code * 2^(k-149) (subnormal / first-binade encoding is linear), so one AND per element
-// isolates it and the power of two is folded into the accumulator's exponent.  Products stay in
-// the normal range, so the arithmetic is exact fp32 FMA work: 2 issue slots per element.
+// The fp16 pool, and the quantized pools of caches with two scale groups per row (Quantized below), use the older
+// lane mapping: two lanes per token, lane l handles half l/16 (elements 32*(l/16) .. +32) of slot l%16 of a tile,
+// with 32 pre-scaled query values and 32 output accumulators in registers; the two half dot products meet through
+// one xor-16 shuffle; the output accumulators are per-lane partial sums reduced once per segment.  There the K
+// side is an integer dot product over a 24-bit fixed-point query (a signed 16-bit limb through dp2a, a signed
+// 8-bit limb through dp4a, codes masked in place into byte planes, the planes' weights undone by a Horner step),
+// and the V side feeds masked bit fields to fp32 FMAs as they are: a bit field inside bits [0,24) of a 32-bit
+// word, read as an fp32 bit pattern, IS the number code * 2^(k-149) (the subnormal / first-binade encoding is
+// linear), so one AND per element isolates it and the power of two is folded into the accumulator's exponent.
 #pragma once
 #include "kvq_common.cuh"
 
