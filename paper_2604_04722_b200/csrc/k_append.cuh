@@ -215,11 +215,9 @@ __device__ __forceinline__ void pack_codes(const __half2* hp, float mn, float in
 // multiplies that zero with whatever a recycled block held before.
 // G: scale groups per row.  With G == 2 the half-row is a group of its own: no exchange with the partner lane,
 // and every lane stores (or clears) the {scale, zero-point} word of its own group at `meta`.
-// TENSOR: 0 = K, 1 = V.  With one scale group per row the codes go into the fragment layout of the decode
-// kernel (kvq_common.cuh): a K row's canonical words are scattered as 32-bit words; a V row's canonical bytes
-// sit slot-minor, four neighbouring slots per word, so in a tile-owning warp (PARTNER == 16) the four lanes of
-// slots 4q .. 4q+3 transpose their bytes among themselves first and store whole words where all four slots
-// belong to this append (single bytes otherwise: the other slots of the word hold tokens of an earlier call).
+// TENSOR: 0 = K, 1 = V.  With one scale group per row (G == 1: only the one-token append gets here, tiles go
+// through k_append_frag.cuh) the codes go into the fragment layout of the decode kernel (kvq_common.cuh): a K
+// row's canonical words as 32-bit words, a V row's canonical bytes one by one (they sit slot-minor).
 template <int CLS, int PARTNER = 16, int G = 1, int TENSOR = 0>
 __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], bool active, bool tail, int half, int t,
                                                         uint8_t* codes, uint8_t* meta) {
@@ -253,25 +251,6 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
     const bool tiny = sf != 0.0f && sf < 6.103515625e-05f;
     if (__any_sync(0xffffffffu, tiny)) pack_codes<CLS, true>(hp, mn, inv, w);
     else pack_codes<CLS, false>(hp, mn, inv, w);
-    if (G == 1 && TENSOR == 1 && PARTNER == 16) {
-        // 4 x 4 byte transposes among the lanes of slots 4q .. 4q+3 (same half): afterwards lane t holds, for every
-        // canonical word wi, byte t % 4 of that word from each of the four slots.  Every lane takes part.
-        const uint32_t group = (__ballot_sync(0xffffffffu, active) >> ((half * 16 + t) & ~3)) & 0xfu;
-        const uint32_t sel_a = (t & 2) ? 0x3276u : 0x5410u, sel_b = (t & 1) ? 0x3715u : 0x6240u;
-#pragma unroll
-        for (int wi = 0; wi < WORDS; ++wi) {
-            const uint32_t y = __byte_perm(w[wi], __shfl_xor_sync(0xffffffffu, w[wi], 2), sel_a);
-            const uint32_t o = __byte_perm(y, __shfl_xor_sync(0xffffffffu, y, 1), sel_b);
-            uint8_t* dst = codes + vfrag_byte_offset(CLS, t & ~3, 4 * (half * WORDS + wi) + (t & 3));
-            if (group == 0xfu) {
-                *reinterpret_cast<uint32_t*>(dst) = o;
-            } else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if (group & (1u << j)) dst[j] = (uint8_t)(o >> (8 * j));
-            }
-        }
-    }
     if (!active) {
         if (tail && (G == 2 || half == 0)) *reinterpret_cast<uint32_t*>(meta) = 0u;
         return;
@@ -280,14 +259,12 @@ __device__ __forceinline__ void quantize_store_half_row(const uint4 (&raw)[4], b
 #pragma unroll
         for (int wi = 0; wi < WORDS; ++wi)
             *reinterpret_cast<uint32_t*>(codes + kfrag_word_offset(CLS, t, half * WORDS + wi)) = w[wi];
-    } else if (G == 1 && PARTNER != 16) {              // a single token: its V bytes one by one
+    } else if (G == 1) {                               // a single token: its V bytes one by one
 #pragma unroll
         for (int wi = 0; wi < WORDS; ++wi)
 #pragma unroll
             for (int b = 0; b < 4; ++b)
                 codes[vfrag_byte_offset(CLS, t, 4 * (half * WORDS + wi) + b)] = (uint8_t)(w[wi] >> (8 * b));
-    } else if (G == 1) {
-        // stored above
     } else if (CLS == 0) {
         *reinterpret_cast<uint2*>(codes + unit_offset(0, half, 0, t)) = make_uint2(w[0], w[1]);
     } else {
@@ -643,7 +620,7 @@ __device__ __forceinline__ void token_store_pc(int c, const uint4 (&kraw)[4], co
 template <bool FUSED, int G>
 __global__ void __launch_bounds__(128)
 k_append_token(AppendParams p) {
-    __shared__ float ctrl_sh[2 * kMaxHidden];
+    extern __shared__ __align__(16) float ctrl_sh[];    // kControllerCtaSmemFloats floats when four warps evaluate the controller
     pdl_launch_dependents();
     pdl_wait();                                        // the attention of the previous step still reads the store
     const int lane = threadIdx.x & 31, b = blockIdx.y;

@@ -123,10 +123,13 @@ __device__ __forceinline__ int controller_decide_warp32(const float* __restrict_
 }
 
 // The same decision taken by a CTA of 128 threads for ONE token, any hidden width H <= 128: thread j owns hidden
-// unit j.  First- and second-layer outputs cross shared memory (sh: 2 * kMaxHidden floats), every thread streams its
-// own row of W2 sixteen inputs ahead of their use; all sums in ascending input order with separately rounded
-// products and sums, so the result is bit-identical to controller_decide.  Every thread of the CTA must call it;
-// returns the class in every thread.
+// unit j.  Every thread requests its whole row of W2 at once (16-byte async copies into shared memory, rows
+// padded by four floats so that neighbouring threads' rows fall into different banks), then first- and second-layer
+// outputs and W3 cross shared memory; all sums in ascending input order with separately rounded products and
+// sums, so the result is bit-identical to controller_decide.  Every thread of the CTA must call it; returns the
+// class in every thread.  sh: kControllerCtaSmemFloats floats, 16-byte aligned.
+constexpr int kW2RowStride = kMaxHidden + 4;
+constexpr int kControllerCtaSmemFloats = 6 * kMaxHidden + kMaxHidden * kW2RowStride;
 __device__ __forceinline__ int controller_decide_cta128(const float* __restrict__ gW, int H, float x0, float x1, float x2,
                                                         float x3, float* sh) {
     const int j = threadIdx.x;
@@ -138,25 +141,22 @@ __device__ __forceinline__ int controller_decide_cta128(const float* __restrict_
     const float* b3 = W3 + 4 * H;
     float* h1s = sh;
     float* h2s = sh + kMaxHidden;
+    float* w3s = sh + 2 * kMaxHidden;                  // the four rows of W3
+    float* w2s = sh + 6 * kMaxHidden + j * kW2RowStride;       // this thread's row of W2
     const bool mine = j < H;
-    const bool vec = (H & 3) == 0;
-    const float* row = W2 + (size_t)(mine ? j : 0) * H;
-    float4 cur[4], nxt[4];                             // sixteen weights of the row in use, sixteen on their way
-    auto fetch = [&](int i0, float4 (&w)[4]) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int i = i0 + 4 * k;
-            if (vec && i < H) {
-                w[k] = __ldg(reinterpret_cast<const float4*>(row + i));
-            } else {
-                w[k].x = i + 0 < H ? __ldg(row + i + 0) : 0.f;
-                w[k].y = i + 1 < H ? __ldg(row + i + 1) : 0.f;
-                w[k].z = i + 2 < H ? __ldg(row + i + 2) : 0.f;
-                w[k].w = i + 3 < H ? __ldg(row + i + 3) : 0.f;
-            }
+    const bool vec = (H & 3) == 0 && (reinterpret_cast<uintptr_t>(W2) & 15u) == 0;
+    if (mine) {
+        const float* row = W2 + (size_t)j * H;
+        if (vec) {
+            for (int i = 0; i < H; i += 4)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(w2s + i)), "l"(row + i)
+                             : "memory");
+        } else {
+            for (int i = 0; i < H; ++i) w2s[i] = __ldg(row + i);
         }
-    };
-    fetch(0, cur);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    for (int i = j; i < 4 * H; i += 128) w3s[i] = __ldg(W3 + i);
     float acc = 0.f;
     if (mine) {
         float a = __ldg(b1 + j);
@@ -167,26 +167,19 @@ __device__ __forceinline__ int controller_decide_cta128(const float* __restrict_
         h1s[j] = a > 0.0f ? a : 0.0f;
         acc = __ldg(b2 + j);
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
-    for (int i0 = 0; i0 < H; i0 += 16) {
-        if (i0 + 16 < H) fetch(i0 + 16, nxt);
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int i = i0 + 4 * k;
-            if (i + 0 < H) acc = __fadd_rn(acc, __fmul_rn(cur[k].x, h1s[i + 0]));
-            if (i + 1 < H) acc = __fadd_rn(acc, __fmul_rn(cur[k].y, h1s[i + 1]));
-            if (i + 2 < H) acc = __fadd_rn(acc, __fmul_rn(cur[k].z, h1s[i + 2]));
-            if (i + 3 < H) acc = __fadd_rn(acc, __fmul_rn(cur[k].w, h1s[i + 3]));
-        }
-#pragma unroll
-        for (int k = 0; k < 4; ++k) cur[k] = nxt[k];
+    if (mine) {
+#pragma unroll 8
+        for (int i = 0; i < H; ++i) acc = __fadd_rn(acc, __fmul_rn(w2s[i], h1s[i]));
+        h2s[j] = acc > 0.0f ? acc : 0.0f;
     }
-    if (mine) h2s[j] = acc > 0.0f ? acc : 0.0f;
     __syncthreads();
     const int lane = threadIdx.x & 31;
     float o = __ldg(b3 + (lane & 3));                  // lanes 0..3 of every warp hold the four logits
-    const float* w3 = W3 + (lane & 3) * H;
-    for (int i = 0; i < H; ++i) o = __fadd_rn(o, __fmul_rn(__ldg(w3 + i), h2s[i]));
+    const float* w3 = w3s + (lane & 3) * H;
+#pragma unroll 8
+    for (int i = 0; i < H; ++i) o = __fadd_rn(o, __fmul_rn(w3[i], h2s[i]));
     const float o0 = __shfl_sync(0xffffffffu, o, 0), o1 = __shfl_sync(0xffffffffu, o, 1);
     const float o2 = __shfl_sync(0xffffffffu, o, 2), o3 = __shfl_sync(0xffffffffu, o, 3);
     if (o0 != o0 || o1 != o1 || o2 != o2 || o3 != o3) return 3;

@@ -332,17 +332,18 @@ int append_impl(kvq_ctx* c, int layer, const void* K, const void* V, const uint8
     if (n_new == 1 && !call_ragged) {                  // a decode step: one warp per 16 heads
         dim3 grid_t((c->kv_heads + 15) / 16, c->batch);
         const unsigned bt = fused && c->hidden != 32 ? 128 : 32;   // a controller of another width is evaluated by four warps
+        const size_t ts = bt == 128 ? sizeof(float) * kControllerCtaSmemFloats : 0;
         if (c->groups == kLayoutPerChannelK) {         // keys wait as fp16 rows; a second small launch packs completed windows
-            if (fused) launch_overlapped(k_append_token<true, kLayoutPerChannelK>, grid_t, bt, 0, st, p);
-            else launch_overlapped(k_append_token<false, kLayoutPerChannelK>, grid_t, bt, 0, st, p);
+            if (fused) launch_overlapped(k_append_token<true, kLayoutPerChannelK>, grid_t, bt, ts, st, p);
+            else launch_overlapped(k_append_token<false, kLayoutPerChannelK>, grid_t, bt, ts, st, p);
             k_pack_window<<<dim3(c->kv_heads, c->batch), 32, 0, st>>>(p);
             c->launches += 1;
         } else if (c->groups == 1) {
-            if (fused) launch_overlapped(k_append_token<true, 1>, grid_t, bt, 0, st, p);
-            else launch_overlapped(k_append_token<false, 1>, grid_t, bt, 0, st, p);
+            if (fused) launch_overlapped(k_append_token<true, 1>, grid_t, bt, ts, st, p);
+            else launch_overlapped(k_append_token<false, 1>, grid_t, bt, ts, st, p);
         } else {
-            if (fused) launch_overlapped(k_append_token<true, 2>, grid_t, bt, 0, st, p);
-            else launch_overlapped(k_append_token<false, 2>, grid_t, bt, 0, st, p);
+            if (fused) launch_overlapped(k_append_token<true, 2>, grid_t, bt, ts, st, p);
+            else launch_overlapped(k_append_token<false, 2>, grid_t, bt, ts, st, p);
         }
         c->launches += 1;
     } else if (n_new <= kChunkTokens) {
@@ -752,6 +753,8 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
         auto dyn_smem = [](auto kernel, int bytes) {
             return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
         };
+        const int tsm = (int)(sizeof(float) * kControllerCtaSmemFloats);
+        ok = ok && dyn_smem(k_append_token<true, 1>, tsm) && dyn_smem(k_append_token<true, 2>, tsm) && dyn_smem(k_append_token<true, kLayoutPerChannelK>, tsm);
         const int fring = (int)kFragRingBytes;
         ok = ok && dyn_smem(k_quant_pack_frag<0, 1>, fring) && dyn_smem(k_quant_pack<0, 2>, ring);
         ok = ok && dyn_smem(k_quant_pack_frag<0, KVQ_APPEND_TOKENS_PER_THREAD>, fring) &&

@@ -120,3 +120,31 @@ def test_controller_inside_and_snapshot(gu, oracle):
         O = torch.zeros_like(Qd)
         with pytest.raises(kq.KvqError):
             kq.kvq_attend_last(g2.ctx, 0, torch.stack([Qd, Qd], dim=1).contiguous(), torch.zeros((B, 2, Hq, 64), dtype=Qd.dtype, device=Qd.device), 2)
+
+
+def test_ragged_appends_and_the_static_scratch_entry(gu, oracle):
+    """Sequences that grow by different amounts (one oracle cache per sequence), and kvq_decode_attn_static on this
+    layout: bit for bit what kvq_decode_attn returns."""
+    import torch
+    from paper_2604_04722_b200 import binding as kq
+    rng = np.random.default_rng(21)
+    B, Hq, H, n_max = 3, 4, 2, 90
+    ocs = [oracle.PerChannelKCache(1, Hq, H) for _ in range(B)]
+    with gu.GpuCache(1, B, Hq, H, 4 * n_max, k_per_channel=True) as g:
+        for call in range(4):
+            K, V = _kv(rng, B, n_max, H)
+            bits = BITS[rng.choice(4, size=(B, n_max), p=[.4, .3, .2, .1])]
+            lens = rng.integers(1, n_max + 1, size=B)
+            kq.kvq_append_ragged(g.ctx, 0, gu.dev(K.view(np.uint16)), gu.dev(V.view(np.uint16)), gu.dev(bits), None, n_max, lens)
+            for b in range(B):
+                ocs[b].append(K[b:b + 1, :lens[b]], V[b:b + 1, :lens[b]], bits[b:b + 1, :lens[b]])
+        Q = rng.standard_normal((B, Hq, 64)).astype(np.float16)
+        out = g.decode(0, Q)
+        for b in range(B):
+            gu.assert_attention_close(out[b:b + 1], ocs[b].decode_attn(Q[b:b + 1]), "sequence %d" % b)
+        Qd = gu.dev(Q.view(np.uint16))
+        got = torch.full_like(Qd, 0x7e00)
+        kq.kvq_decode_attn_static(g.ctx, 0, Qd, got)
+        torch.cuda.synchronize()
+        assert np.array_equal(got.cpu().numpy().view(np.uint16), out)
+        assert kq.kvq_device_status(g.ctx) == 0
