@@ -637,19 +637,59 @@ k_quant_pack_frag(AppendParams p) {
         uint8_t* rec;
         int h;                                         // KV head
     };
-    uint32_t tau = 0;
-    int hh = warp;
-    auto settle = [&]() {
-        while (hh >= nh) {
-            hh -= nh;
-            ++tau;
-        }
-    };
-    settle();
+    // Tiles are dealt round-robin to the warps; a warp takes a tile through all heads of the CTA's group, so what
+    // depends on the tile alone (class, ranks of its slots, the source rows of the four slots this lane fetches,
+    // the place of the record inside its arena block) is worked out once per tile.
+    uint32_t tau = (uint32_t)warp;
+    int hh = 0;
+    struct TileInfo {
+        int k, first_new;
+        uint32_t live, blk, rec_off;
+        size_t src[4];                                 // element offset of the row of slot (lane >> 3) + 4 i, head 0 (live slots)
+        uint32_t fetch;                                // bit i: that slot receives a token of this call; bit 4 + i: it is older
+    } ti;
+    ti.k = -1;
     uint8_t* my_ring = dyn_smem + (size_t)warp * kFragDepth * kFragStageBytes;
     int voff[4];                                       // where this lane's V elements of slots 4q .. 4q+3 sit in a stage
 #pragma unroll
     for (int j = 0; j < 4; ++j) voff[j] = stage_piece_offset(4 * (lane & 3) + j, lane >> 3) + 8 * ((lane >> 2) & 1);
+    const int piece = lane & 7;
+    int soff[4];                                       // where the piece this lane fetches of slot (lane >> 3) + 4 i goes
+#pragma unroll
+    for (int i = 0; i < 4; ++i) soff[i] = stage_piece_offset((lane >> 3) + 4 * i, piece);
+    const size_t row_stride = (size_t)p.store.kv_heads * kHeadDim;
+    const uint32_t* tab_b = p.store.table + ((size_t)p.layer * p.store.batch + b) * p.store.kv_heads * p.store.table_stride;
+    auto load_tile = [&]() {
+        const int k = (tau >= pre[1]) + (tau >= pre[2]) + (tau >= pre[3]);
+        const uint32_t basek = k == 0 ? base[0] : k == 1 ? base[1] : k == 2 ? base[2] : base[3];
+        const uint32_t nk = (k == 0 ? ncls[0] : k == 1 ? ncls[1] : k == 2 ? ncls[2] : ncls[3]);
+        const uint32_t nke = nk + ext_n[k];
+        const uint32_t tile = (k == 0 ? first[0] : k == 1 ? first[1] : k == 2 ? first[2] : first[3]) +
+                              (tau - (k == 0 ? pre[0] : k == 1 ? pre[1] : k == 2 ? pre[2] : pre[3]));
+        const int r0 = (int)(tile * kTileTokens) - (int)basek;           // rank of the tile's slot 0 (negative: older slots)
+        ti.k = k;
+        ti.first_new = r0 < 0 ? -r0 : 0;
+        switch (k) {                                   // (constant divisors)
+        case 0: ti.blk = tile / block_tiles(0, LAYOUT); ti.rec_off = (tile - ti.blk * block_tiles(0, LAYOUT)) * pool_rec_bytes(0, LAYOUT); break;
+        case 1: ti.blk = tile / block_tiles(1, LAYOUT); ti.rec_off = (tile - ti.blk * block_tiles(1, LAYOUT)) * pool_rec_bytes(1, LAYOUT); break;
+        case 2: ti.blk = tile / block_tiles(2, LAYOUT); ti.rec_off = (tile - ti.blk * block_tiles(2, LAYOUT)) * pool_rec_bytes(2, LAYOUT); break;
+        default: ti.blk = tile / block_tiles(3, LAYOUT); ti.rec_off = (tile - ti.blk * block_tiles(3, LAYOUT)) * pool_rec_bytes(3, LAYOUT); break;
+        }
+        ti.blk += p.store.table_off[k];
+        ti.fetch = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = r0 + (lane >> 3) + 4 * i;
+            const bool live = r >= 0 && (uint32_t)r < nke;
+            size_t tok_i = 0;
+            if (live) tok_i = (uint32_t)r < nk ? (size_t)chunk * CT + list[k][r] : (size_t)ext[k][(uint32_t)r - nk];
+            ti.src[i] = ((size_t)b * p.n_new + tok_i) * row_stride;
+            ti.fetch |= (live ? 1u : 0u) << i | (r < 0 ? 16u : 0u) << i;
+        }
+        // slots that receive a token: ranks 0 .. nke-1 that fall into this tile
+        const int lo = r0 < 0 ? -r0 : 0, hi_ = min((int)kTileTokens, (int)nke - r0);
+        ti.live = hi_ > lo ? (((1u << hi_) - 1u) & ~((1u << lo) - 1u)) : 0u;
+    };
     auto next_item = [&](int stage) {
         Item it;
         it.k = -1;
@@ -658,42 +698,31 @@ k_quant_pack_frag(AppendParams p) {
         it.rec = nullptr;
         it.h = 0;
         if (tau < pre[4]) {
-            const int k = (tau >= pre[1]) + (tau >= pre[2]) + (tau >= pre[3]);
-            const uint32_t basek = k == 0 ? base[0] : k == 1 ? base[1] : k == 2 ? base[2] : base[3];
-            const uint32_t nk = (k == 0 ? ncls[0] : k == 1 ? ncls[1] : k == 2 ? ncls[2] : ncls[3]);
-            const uint32_t nke = nk + ext_n[k];
+            if (hh == 0) load_tile();
+            const int k = ti.k, h = h0 + hh;
             it.k = k;
-            const uint32_t tile = (k == 0 ? first[0] : k == 1 ? first[1] : k == 2 ? first[2] : first[3]) +
-                                  (tau - (k == 0 ? pre[0] : k == 1 ? pre[1] : k == 2 ? pre[2] : pre[3]));
-            const int r0 = (int)(tile * kTileTokens) - (int)basek;       // rank of the tile's slot 0 (negative: older slots)
-            it.first_new = r0 < 0 ? -r0 : 0;
-            const int h = h0 + hh;
+            it.first_new = ti.first_new;
+            it.live = ti.live;
             it.h = h;
-            it.rec = tile_ptr(p.store, k, stream_table(p.store, k, p.layer, b, h), tile, LAYOUT);
+            it.rec = p.store.arena + (size_t)tab_b[(size_t)h * p.store.table_stride + ti.blk] * kBlockBytes + ti.rec_off;
             uint8_t* dst = my_ring + (size_t)stage * kFragStageBytes;
-            const int piece = lane & 7;
+            const size_t head_off = (size_t)h * kHeadDim;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int s = (lane >> 3) + 4 * i;     // the slot whose row these eight lanes fetch
-                const int r = r0 + s;
-                const bool live = r >= 0 && (uint32_t)r < nke;
-                size_t tok_i = 0;
-                if (live) tok_i = (uint32_t)r < nk ? (size_t)chunk * CT + list[k][r] : (size_t)ext[k][(uint32_t)r - nk];
-                const size_t src = (((size_t)b * p.n_new + tok_i) * p.store.kv_heads + h) * kHeadDim;
-                const int off = stage_piece_offset(s, piece);
+                const bool live = (ti.fetch >> i) & 1u;
+                const size_t src = ti.src[i] + head_off;
                 // a slot of an earlier call: its key row waits in the residual buffer -- read from the copy taken before this
                 // launch, because the rows of the stream's NEXT open window go to the same places during the launch
-                if (PC && r < 0 && k < 3)
-                    cp_async16_or_zero(dst + off, reinterpret_cast<const uint4*>(residual_rows_before(p.store, k, b, h) + s * kHeadDim) + piece, true);
+                if (PC && ((ti.fetch >> (4 + i)) & 1u) && k < 3)
+                    cp_async16_or_zero(dst + soff[i], reinterpret_cast<const uint4*>(residual_rows_before(p.store, k, b, h) + ((lane >> 3) + 4 * i) * kHeadDim) + piece, true);
                 else
-                    cp_async16_or_zero(dst + off, reinterpret_cast<const uint4*>(p.K + src) + piece, live);
-                cp_async16_or_zero(dst + kStageTensorBytes + off, reinterpret_cast<const uint4*>(p.V + src) + piece, live);
+                    cp_async16_or_zero(dst + soff[i], reinterpret_cast<const uint4*>(p.K + src) + piece, live);
+                cp_async16_or_zero(dst + kStageTensorBytes + soff[i], reinterpret_cast<const uint4*>(p.V + src) + piece, live);
             }
-            // slots that receive a token: ranks 0 .. nke-1 that fall into this tile
-            const int lo = r0 < 0 ? -r0 : 0, hi_ = min((int)kTileTokens, (int)nke - r0);
-            it.live = hi_ > lo ? (((1u << hi_) - 1u) & ~((1u << lo) - 1u)) : 0u;
-            hh += NWARPS;
-            settle();
+            if (++hh == nh) {
+                hh = 0;
+                tau += NWARPS;
+            }
         }
         cp_async_commit();                             // one group per call, possibly empty
         return it;
