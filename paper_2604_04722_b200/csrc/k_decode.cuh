@@ -72,7 +72,7 @@ template <int WARPS, int STAGES, int STAGE_BYTES, int MIN_CTAS>
 struct DecodeGeom {
     static constexpr int kWarps = WARPS, kThreads = WARPS * 32, kStages = STAGES, kStageBytes = STAGE_BYTES, kCtasPerSm = MIN_CTAS;
     static constexpr size_t kSmemBytes = (size_t)WARPS * STAGES * STAGE_BYTES;
-    static constexpr bool kCtaMerge = MIN_CTAS == 1;   // only the one-CTA-per-SM geometry merges inside the CTA
+    static constexpr bool kCtaMerge = true;            // units cut into a divisor of WARPS parts are merged inside their CTA
     // tiles of class c that fit one stage
     __host__ __device__ static constexpr int tps(int c, int g = 1) { return STAGE_BYTES / pool_rec_bytes(c, g); }
     static_assert(STAGE_BYTES % 16 == 0 && STAGE_BYTES >= pool_rec_bytes(3), "a stage must hold one fp16 tile");

@@ -430,6 +430,11 @@ DecodePlan choose_plan(kvq_ctx* c, int len, uint64_t units, uint64_t room = 0) {
             plan.cta_parts = (uint32_t)parts;
             return plan;
         }
+        if (GeomLarge::kWarps % parts == 0) {          // whole CTAs of the bandwidth geometry: no partial records either
+            plan.gw = (uint32_t)gw;
+            plan.cta_parts = (uint32_t)parts;
+            return plan;
+        }
         if (units * (parts + 1) <= room) {
             plan.gw = (uint32_t)gw;
             plan.small = gw <= small_resident;
@@ -509,6 +514,7 @@ DecodePlan choose_plan(kvq_ctx* c, int len, uint64_t units, uint64_t room = 0) {
         }
     }
     plan.gw = (uint32_t)best;
+    if (best % units == 0 && GeomLarge::kWarps % (best / units) == 0) plan.cta_parts = (uint32_t)(best / units);
     return plan;
 }
 
