@@ -36,7 +36,9 @@
  *   - All sequences of the batch advance together: every append adds the same
  *     number of tokens to each of the `batch` sequences of that layer.
  *   - fp16 tensors are IEEE binary16, row-major, innermost dimension last.
- *   - The handle is not thread-safe; use one handle from one thread at a time.
+ *   - The handle is not thread-safe; use one handle from one thread at a time, and queue its calls on one
+ *     stream (or order the streams yourself): the calls share scratch buffers of the handle (class bytes,
+ *     histograms and arrival counters of the append, partial records of the attention, the lengths ring).
  */
 #ifndef KVQ_H
 #define KVQ_H

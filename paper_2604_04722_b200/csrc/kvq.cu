@@ -142,7 +142,7 @@ constexpr int kProfMaxCalls = 1024;
 #define KVQ_APPEND_WAVES_SMALL 2
 #endif
 #ifndef KVQ_APPEND_WAVES
-#define KVQ_APPEND_WAVES 12
+#define KVQ_APPEND_WAVES 16
 #endif
 #ifndef KVQ_APPEND_TOKENS_PER_THREAD
 #define KVQ_APPEND_TOKENS_PER_THREAD 2
