@@ -86,6 +86,28 @@ k_classify(AppendParams p) {
         __syncthreads();
     }
     uint32_t mine[4] = {0, 0, 0, 0};                   // lane 0: this warp's tokens per class over all passes
+    if (FUSED && p.hidden == 32 && p.tpt == 2) {       // the usual prefill shape: both tokens of the thread at once
+        const int t0 = chunk * 2 * kChunkTokens + threadIdx.x, t1 = t0 + kChunkTokens;
+        const int n_b = new_tokens_of(p, b);
+        const bool live0 = t0 < n_b, live1 = t1 < n_b;
+        const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 f0 = live0 ? reinterpret_cast<const float4*>(p.feats)[(size_t)b * p.n_new + t0] : z;
+        const float4 f1 = live1 ? reinterpret_cast<const float4*>(p.feats)[(size_t)b * p.n_new + t1] : z;
+        int c0 = -1, c1 = -1;
+        if (__any_sync(0xffffffffu, live0 || live1)) controller_decide_two32(sW, f0, f1, c0, c1);
+        c0 = live0 ? c0 : -1;
+        c1 = live1 ? c1 : -1;
+        if (live0) {
+            p.cls[(size_t)b * p.n_new + t0] = (uint8_t)c0;
+            if (p.bits_out) p.bits_out[(size_t)b * p.n_new + t0] = (uint8_t)pool_bits(c0);
+        }
+        if (live1) {
+            p.cls[(size_t)b * p.n_new + t1] = (uint8_t)c1;
+            if (p.bits_out) p.bits_out[(size_t)b * p.n_new + t1] = (uint8_t)pool_bits(c1);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mine[k] += __popc(__ballot_sync(0xffffffffu, c0 == k)) + __popc(__ballot_sync(0xffffffffu, c1 == k));
+    } else
     for (int r = 0; r < p.tpt; ++r) {
         const int t = (chunk * p.tpt + r) * kChunkTokens + threadIdx.x;
         const bool live = t < new_tokens_of(p, b);

@@ -68,6 +68,64 @@ __device__ __forceinline__ int controller_decide(const float* sW, int Hrt, float
     return cls;
 }
 
+// Two tokens at once, hidden width 32: every weight is read from shared memory once for both and the two chains of
+// rounded products and sums are independent, so they overlap.  Same arithmetic and order per token as above.
+__device__ __forceinline__ void controller_decide_two32(const float* sW, const float4& xa, const float4& xb, int& cls_a,
+                                                        int& cls_b) {
+    constexpr int H = 32;
+    const float* W1 = sW;
+    const float* b1 = W1 + 4 * H;
+    const float* W2 = b1 + H;
+    const float* b2 = W2 + H * H;
+    const float* W3 = b2 + H;
+    const float* b3 = W3 + 4 * H;
+    float ha[H], hb[H];
+#pragma unroll
+    for (int j = 0; j < H; ++j) {
+        const float4 w = *reinterpret_cast<const float4*>(W1 + 4 * j);
+        float a = b1[j], b = a;
+        a = __fadd_rn(a, __fmul_rn(w.x, xa.x)); b = __fadd_rn(b, __fmul_rn(w.x, xb.x));
+        a = __fadd_rn(a, __fmul_rn(w.y, xa.y)); b = __fadd_rn(b, __fmul_rn(w.y, xb.y));
+        a = __fadd_rn(a, __fmul_rn(w.z, xa.z)); b = __fadd_rn(b, __fmul_rn(w.z, xb.z));
+        a = __fadd_rn(a, __fmul_rn(w.w, xa.w)); b = __fadd_rn(b, __fmul_rn(w.w, xb.w));
+        ha[j] = a > 0.0f ? a : 0.0f;
+        hb[j] = b > 0.0f ? b : 0.0f;
+    }
+    float oa[4], ob[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) oa[c] = ob[c] = b3[c];
+#pragma unroll 4
+    for (int j = 0; j < H; ++j) {
+        float a = b2[j], b = a;
+#pragma unroll
+        for (int i = 0; i < H; i += 4) {
+            const float4 w = *reinterpret_cast<const float4*>(W2 + j * H + i);
+            a = __fadd_rn(a, __fmul_rn(w.x, ha[i + 0])); b = __fadd_rn(b, __fmul_rn(w.x, hb[i + 0]));
+            a = __fadd_rn(a, __fmul_rn(w.y, ha[i + 1])); b = __fadd_rn(b, __fmul_rn(w.y, hb[i + 1]));
+            a = __fadd_rn(a, __fmul_rn(w.z, ha[i + 2])); b = __fadd_rn(b, __fmul_rn(w.z, hb[i + 2]));
+            a = __fadd_rn(a, __fmul_rn(w.w, ha[i + 3])); b = __fadd_rn(b, __fmul_rn(w.w, hb[i + 3]));
+        }
+        const float h2a = a > 0.0f ? a : 0.0f, h2b = b > 0.0f ? b : 0.0f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const float w = W3[c * H + j];
+            oa[c] = __fadd_rn(oa[c], __fmul_rn(w, h2a));
+            ob[c] = __fadd_rn(ob[c], __fmul_rn(w, h2b));
+        }
+    }
+    auto pick = [](const float (&o)[4]) {
+        if (o[0] != o[0] || o[1] != o[1] || o[2] != o[2] || o[3] != o[3]) return 3;
+        int cls = 0;
+        float best = o[0];
+        if (o[1] > best) { best = o[1]; cls = 1; }
+        if (o[2] > best) { best = o[2]; cls = 2; }
+        if (o[3] > best) { best = o[3]; cls = 3; }
+        return cls;
+    };
+    cls_a = pick(oa);
+    cls_b = pick(ob);
+}
+
 __device__ __forceinline__ int controller_decide_any(const float* sW, int H, float x0, float x1, float x2,
                                                      float x3, float logits[4]) {
     if (H == 32) return controller_decide<32>(sW, H, x0, x1, x2, x3, logits);
