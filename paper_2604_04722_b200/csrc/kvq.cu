@@ -761,6 +761,14 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
         };
         const int tsm = (int)(sizeof(float) * kControllerCtaSmemFloats);
         ok = ok && dyn_smem(k_append_token<true, 1>, tsm) && dyn_smem(k_append_token<true, 2>, tsm) && dyn_smem(k_append_token<true, kLayoutPerChannelK>, tsm);
+        // The kernels of a decode step alternate; the attention kernel needs almost all of an SM's shared memory, so the
+        // small ones ask for the same split of the L1 / shared-memory array and the SMs need not be reconfigured between them.
+        auto max_shared = [](auto kernel) {
+            return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+        };
+        ok = ok && max_shared(k_append_token<true, 1>) && max_shared(k_append_token<false, 1>) && max_shared(k_append_token<true, 2>) &&
+             max_shared(k_append_token<false, 2>) && max_shared(k_append_token<true, kLayoutPerChannelK>) &&
+             max_shared(k_append_token<false, kLayoutPerChannelK>) && max_shared(k_pack_window);
         const int fring = (int)kFragRingBytes;
         ok = ok && dyn_smem(k_quant_pack_frag<0, 1>, fring) && dyn_smem(k_quant_pack<0, 2>, ring);
         ok = ok && dyn_smem(k_quant_pack_frag<0, KVQ_APPEND_TOKENS_PER_THREAD>, fring) &&

@@ -419,3 +419,45 @@ def test_two_runs_give_the_same_bits(gu):
     for a, b in zip(runs[0][1], runs[1][1]):
         assert np.array_equal(a, b)
     assert np.array_equal(runs[0][1][0], runs[0][1][1]) and np.array_equal(runs[0][1][2], runs[0][1][3])
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_decode_with_extreme_value_scales_peaks_and_query_ranges(gu, oracle, seed):
+    """The value weights p * scale_v go through an integer grid shared by many tiles and the query through a
+    fixed-point grid: value rows whose scales differ by up to 2^22 from token to token, a single dominant key over a
+    flat background, query channels of very different size and very small or large queries must all stay within the
+    attention tolerance, for the automatic plan and for an explicit split count, in two appends."""
+    from paper_2604_04722_b200 import binding as kq
+    rng = np.random.default_rng(1000 + seed)
+    B, H = int(rng.choice([1, 2])), int(rng.choice([1, 3]))
+    Hq = H * int(rng.choice([1, 3]))
+    n = [5, 40, 333, 1500, 5000, 777][seed % 6]
+    mix = rng.dirichlet(np.ones(4) * 0.7)
+    kscale = [0.05, 1.0, 4.0, 12.0][seed % 4]
+    K = (rng.standard_normal((B, n, H, 64)) * kscale).astype(np.float16)
+    vs = np.exp2(rng.integers(-12, 11, size=(B, n, H, 1))).astype(np.float32)
+    V = np.clip(rng.standard_normal((B, n, H, 64)) * vs, -60000, 60000).astype(np.float16)
+    Q = rng.standard_normal((B, Hq, 64)).astype(np.float32)
+    mode = seed % 4
+    if mode == 1:                                            # one dominant key
+        for b in range(B):
+            for h in range(Hq):
+                K[b, int(rng.integers(0, n)), h // (Hq // H)] = (Q[b, h] * 4.0).astype(np.float16)
+    if mode == 2:
+        Q *= np.exp2(rng.integers(-8, 8, size=(B, Hq, 64)))
+    if mode == 3:
+        Q *= [1e-3, 30.0][seed % 2]
+    Q = Q.astype(np.float16)
+    bits = BITS[rng.choice(4, size=(B, n), p=mix)]
+    oc = oracle.OracleCache(B, Hq, H)
+    with gu.GpuCache(1, B, Hq, H, n) as g:
+        cut = int(rng.integers(1, n + 1))
+        for lo, hi in ((0, cut), (cut, n)):
+            if hi > lo:
+                g.append(0, K[:, lo:hi], V[:, lo:hi], bits[:, lo:hi])
+                oc.append(K[:, lo:hi], V[:, lo:hi], bits[:, lo:hi])
+        want = oc.decode_attn(Q)
+        for splits in (0, [1, 2, 5, 16, 64][seed % 5]):
+            kq.kvq_set_splits(g.ctx, splits)
+            gu.assert_attention_close(g.decode(0, Q), want, "seed %d splits %d" % (seed, splits))
+        assert kq.kvq_device_status(g.ctx) == 0
