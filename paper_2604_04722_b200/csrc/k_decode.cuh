@@ -489,6 +489,17 @@ __device__ __forceinline__ uint32_t byte_perm(uint32_t a, uint32_t b, uint32_t s
     return d;
 }
 
+// The four balanced base-256 digits of T (|T| < 2^31 - 2^23), one per byte, in two's complement: adding 128 to
+// each of the three low digits makes them unsigned without a borrow, so they are the bytes of the sum; flipping
+// bit 7 of each takes the 128 off again.  The top byte is the top digit as it stands.
+__device__ __forceinline__ uint32_t balanced_digits(int T) { return ((uint32_t)T + 0x00808080u) ^ 0x00808080u; }
+// Selector that picks byte n of both source words of a prmt into the two low bytes of its result.
+__device__ __forceinline__ uint32_t digit_selector(int n) { return (uint32_t)n | ((uint32_t)(4 + n) << 4); }
+// Byte n (through sel = digit_selector(n)) of u0, u1, u2, u3 as bytes 0..3 of one word.
+__device__ __forceinline__ uint32_t pick_bytes(uint32_t u0, uint32_t u1, uint32_t u2, uint32_t u3, uint32_t sel) {
+    return byte_perm(byte_perm(u0, u1, sel), byte_perm(u2, u3, sel), 0x5410u);
+}
+
 constexpr float kGridLimit = 16777215.0f;          // weights on the grid stay below 2^24
 constexpr int kFlushTiles = 1000;                  // int32 headroom: 16 slots * 255 * 255 per tile and accumulator
 
@@ -516,23 +527,19 @@ struct FragRows {
     // Column operand of the K products: digit g & 3 of the fixed-point query (the same words serve tile A from
     // the lanes with g < 4 and tile B from the lanes with g >= 4; see the walk).
     __device__ static __forceinline__ void make_kb(const float* qrow, float fix_scale, int g, int q, uint32_t (&bk)[4]) {
+        const uint32_t sel = digit_selector(g & 3);
 #pragma unroll
         for (int u = 0; u < 2; ++u)
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 const float plane_scale = (float)(1 << (BITS * (PLANES - 1 - k_plane(u, r))));
-                uint32_t w = 0;
+                uint32_t dgt[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int e = k_element(u, r, q, j);
-                    const int T = __float2int_rn(qrow[(e >> 5) * (kHalfDim + 4) + (e & 31)] * (fix_scale * plane_scale));
-                    const int h0 = (T + 128) >> 8, d0 = T - (h0 << 8);
-                    const int h1 = (h0 + 128) >> 8, d1 = h0 - (h1 << 8);
-                    const int h2 = (h1 + 128) >> 8, d2 = h1 - (h2 << 8);
-                    const int dg = (g & 3) == 0 ? d0 : (g & 3) == 1 ? d1 : (g & 3) == 2 ? d2 : h2;
-                    w |= ((uint32_t)dg & 0xffu) << (8 * j);
+                    dgt[j] = balanced_digits(__float2int_rn(qrow[(e >> 5) * (kHalfDim + 4) + (e & 31)] * (fix_scale * plane_scale)));
                 }
-                bk[2 * u + r] = w;
+                bk[2 * u + r] = pick_bytes(dgt[0], dgt[1], dgt[2], dgt[3], sel);
             }
     }
     __device__ static __forceinline__ void load_words(const uint8_t* codes, int lane, uint32_t (&w)[NW]) {
@@ -704,22 +711,17 @@ struct FragRows {
         ex = ex > 254u ? 254u : ex;                    // (garbage of a tile whose keys are residual rows)
         const float fix = __uint_as_float((275u - ex) << 23), inv_fix = __uint_as_float((ex - 21u) << 23);
         uint32_t bk[4];
+        const uint32_t sel = digit_selector(g & 3);
 #pragma unroll
         for (int u = 0; u < 2; ++u)
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 const float plane_scale = (float)(1 << (BITS * (PLANES - 1 - k_plane(u, r))));
-                uint32_t w = 0;
+                uint32_t dgt[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int T = __float2int_rn(qs[pc_index(u, r, j)] * (fix * plane_scale));
-                    const int h0 = (T + 128) >> 8, d0 = T - (h0 << 8);
-                    const int h1 = (h0 + 128) >> 8, d1 = h0 - (h1 << 8);
-                    const int h2 = (h1 + 128) >> 8, d2 = h1 - (h2 << 8);
-                    const int dg = (g & 3) == 0 ? d0 : (g & 3) == 1 ? d1 : (g & 3) == 2 ? d2 : h2;
-                    w |= ((uint32_t)dg & 0xffu) << (8 * j);
-                }
-                bk[2 * u + r] = w;
+                for (int j = 0; j < 4; ++j)
+                    dgt[j] = balanced_digits(__float2int_rn(qs[pc_index(u, r, j)] * (fix * plane_scale)));
+                bk[2 * u + r] = pick_bytes(dgt[0], dgt[1], dgt[2], dgt[3], sel);
             }
         uint32_t bkA[4], bkB[4];
 #pragma unroll
