@@ -644,6 +644,7 @@ __global__ void __launch_bounds__(128)
 k_append_token(AppendParams p) {
     extern __shared__ __align__(16) float ctrl_sh[];    // kControllerCtaSmemFloats floats when four warps evaluate the controller
     pdl_launch_dependents();
+    if (FUSED && blockDim.x != 32) controller_fetch_cta128(p.ctrl, p.hidden, ctrl_sh);   // no kernel writes the weights
     pdl_wait();                                        // the attention of the previous step still reads the store
     const int lane = threadIdx.x & 31, b = blockIdx.y;
     const int h = blockIdx.x * 16 + (lane >> 1), half = lane & 1;

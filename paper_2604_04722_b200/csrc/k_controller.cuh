@@ -181,40 +181,78 @@ __device__ __forceinline__ int controller_decide_warp32(const float* __restrict_
 }
 
 // The same decision taken by a CTA of 128 threads for ONE token, any hidden width H <= 128: thread j owns hidden
-// unit j.  Every thread requests its whole row of W2 at once (16-byte async copies into shared memory, rows
-// padded by four floats so that neighbouring threads' rows fall into different banks), then first- and second-layer
-// outputs and W3 cross shared memory; all sums in ascending input order with separately rounded products and
-// sums, so the result is bit-identical to controller_decide.  Every thread of the CTA must call it; returns the
-// class in every thread.  sh: kControllerCtaSmemFloats floats, 16-byte aligned.
+// unit j.  W2 and W3 come into shared memory with 16-byte async copies in which neighbouring threads take
+// neighbouring pieces of the matrices (whole 128-byte lines per request); their rows are padded by four floats
+// there, so that the 16-byte reads of the sums below (thread j reads row j of W2, lane l row l % 4 of W3) fall into
+// different banks.  First- and second-layer outputs cross shared memory; all sums in ascending input order with
+// separately rounded products and sums, so the result is bit-identical to controller_decide.  Every thread of
+// the CTA must call both parts; part 2 returns the class in every thread.  sh: kControllerCtaSmemFloats floats,
+// 16-byte aligned.
 constexpr int kW2RowStride = kMaxHidden + 4;
-constexpr int kControllerCtaSmemFloats = 6 * kMaxHidden + kMaxHidden * kW2RowStride;
+constexpr int kControllerCtaSmemFloats = 2 * kMaxHidden + 4 * kW2RowStride + kMaxHidden * kW2RowStride;
+// Whether W2 and W3 of the parameter block at gW can be moved and read in 16-byte pieces.
+__device__ __forceinline__ bool controller_rows_vectorized(const float* gW, int H) {
+    return (H & 3) == 0 && (reinterpret_cast<uintptr_t>(gW + 5 * H) & 15u) == 0 && (reinterpret_cast<uintptr_t>(gW + 6 * H + H * H) & 15u) == 0;
+}
+__device__ __forceinline__ void cp_async16_ca(float* smem_dst, const float* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+                 : "memory");
+}
+// acc + sum over i of w[i] * h[i], i ascending, every product and every sum rounded (w, h: 16-byte aligned when VEC).
+template <bool VEC>
+__device__ __forceinline__ float ordered_dot(float acc, const float* w, const float* h, int H) {
+    if (VEC) {
+#pragma unroll 4
+        for (int i = 0; i < H; i += 4) {
+            const float4 w4 = *reinterpret_cast<const float4*>(w + i), h4 = *reinterpret_cast<const float4*>(h + i);
+            acc = __fadd_rn(acc, __fmul_rn(w4.x, h4.x));
+            acc = __fadd_rn(acc, __fmul_rn(w4.y, h4.y));
+            acc = __fadd_rn(acc, __fmul_rn(w4.z, h4.z));
+            acc = __fadd_rn(acc, __fmul_rn(w4.w, h4.w));
+        }
+    } else {
+#pragma unroll 8
+        for (int i = 0; i < H; ++i) acc = __fadd_rn(acc, __fmul_rn(w[i], h[i]));
+    }
+    return acc;
+}
+// Part 1: request W2 and W3 (they are written by kvq_set_controller only, never by a kernel).
+__device__ __forceinline__ void controller_fetch_cta128(const float* __restrict__ gW, int H, float* sh) {
+    const int j = threadIdx.x;
+    const float* W2 = gW + 5 * H;
+    const float* W3 = W2 + H * H + H;
+    float* w3s = sh + 2 * kMaxHidden;                  // the four rows of W3, kW2RowStride apart
+    float* w2s = w3s + 4 * kW2RowStride;               // the H rows of W2, kW2RowStride apart
+    if (controller_rows_vectorized(gW, H)) {
+        const int per_row = H >> 2;                    // 16-byte pieces per row
+        for (int piece = j; piece < H * per_row; piece += 128) {
+            const int r = piece / per_row, c = (piece - r * per_row) << 2;
+            cp_async16_ca(w2s + r * kW2RowStride + c, W2 + (size_t)r * H + c);
+        }
+        for (int piece = j; piece < 4 * per_row; piece += 128) {
+            const int r = piece / per_row, c = (piece - r * per_row) << 2;
+            cp_async16_ca(w3s + r * kW2RowStride + c, W3 + (size_t)r * H + c);
+        }
+    } else {
+        for (int i = j; i < H * H; i += 128) w2s[(i / H) * kW2RowStride + i % H] = __ldg(W2 + i);
+        for (int i = j; i < 4 * H; i += 128) w3s[(i / H) * kW2RowStride + i % H] = __ldg(W3 + i);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+// Part 2: the decision, once controller_fetch_cta128 has been called with the same arguments.
 __device__ __forceinline__ int controller_decide_cta128(const float* __restrict__ gW, int H, float x0, float x1, float x2,
                                                         float x3, float* sh) {
     const int j = threadIdx.x;
     const float* W1 = gW;
     const float* b1 = W1 + 4 * H;
-    const float* W2 = b1 + H;
-    const float* b2 = W2 + H * H;
-    const float* W3 = b2 + H;
-    const float* b3 = W3 + 4 * H;
+    const float* b2 = b1 + H + H * H;
+    const float* b3 = b2 + H + 4 * H;
     float* h1s = sh;
     float* h2s = sh + kMaxHidden;
-    float* w3s = sh + 2 * kMaxHidden;                  // the four rows of W3
-    float* w2s = sh + 6 * kMaxHidden + j * kW2RowStride;       // this thread's row of W2
+    float* w3s = sh + 2 * kMaxHidden;
+    float* w2s = w3s + 4 * kW2RowStride;
     const bool mine = j < H;
-    const bool vec = (H & 3) == 0 && (reinterpret_cast<uintptr_t>(W2) & 15u) == 0;
-    if (mine) {
-        const float* row = W2 + (size_t)j * H;
-        if (vec) {
-            for (int i = 0; i < H; i += 4)
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(w2s + i)), "l"(row + i)
-                             : "memory");
-        } else {
-            for (int i = 0; i < H; ++i) w2s[i] = __ldg(row + i);
-        }
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    for (int i = j; i < 4 * H; i += 128) w3s[i] = __ldg(W3 + i);
+    const bool vec = controller_rows_vectorized(gW, H);
     float acc = 0.f;
     if (mine) {
         float a = __ldg(b1 + j);
@@ -225,19 +263,17 @@ __device__ __forceinline__ int controller_decide_cta128(const float* __restrict_
         h1s[j] = a > 0.0f ? a : 0.0f;
         acc = __ldg(b2 + j);
     }
+    const int lane = threadIdx.x & 31;
+    float o = __ldg(b3 + (lane & 3));                  // lanes 0..3 of every warp hold the four logits
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     if (mine) {
-#pragma unroll 8
-        for (int i = 0; i < H; ++i) acc = __fadd_rn(acc, __fmul_rn(w2s[i], h1s[i]));
+        acc = vec ? ordered_dot<true>(acc, w2s + j * kW2RowStride, h1s, H) : ordered_dot<false>(acc, w2s + j * kW2RowStride, h1s, H);
         h2s[j] = acc > 0.0f ? acc : 0.0f;
     }
     __syncthreads();
-    const int lane = threadIdx.x & 31;
-    float o = __ldg(b3 + (lane & 3));                  // lanes 0..3 of every warp hold the four logits
-    const float* w3 = w3s + (lane & 3) * H;
-#pragma unroll 8
-    for (int i = 0; i < H; ++i) o = __fadd_rn(o, __fmul_rn(w3[i], h2s[i]));
+    const float* w3 = w3s + (lane & 3) * kW2RowStride;
+    o = vec ? ordered_dot<true>(o, w3, h2s, H) : ordered_dot<false>(o, w3, h2s, H);
     const float o0 = __shfl_sync(0xffffffffu, o, 0), o1 = __shfl_sync(0xffffffffu, o, 1);
     const float o2 = __shfl_sync(0xffffffffu, o, 2), o3 = __shfl_sync(0xffffffffu, o, 3);
     if (o0 != o0 || o1 != o1 || o2 != o2 || o3 != o3) return 3;
