@@ -51,6 +51,7 @@ SIGNATURES = {
     "kvq_token_features": (_i, [_vp, _i, _i, _i, _vp, _vp, C.c_uint64, C.c_uint32, _vp, _vp, _vp]),
     "kvq_attend_last": (_i, [_vp, _i, _vp, _vp, _i, _vp]),
     "kvq_decode_attn_static": (_i, [_vp, _i, _vp, _vp, _vp]),
+    "kvq_decode_step": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvq_decode_step_host": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kvq_reset": (_i, [_vp, _vp]),
     "kvq_seq_len": (_i, [_vp, _i, C.POINTER(_i)]),
@@ -245,6 +246,12 @@ def kvq_attend_last(ctx: int, layer: int, Q, O, n_queries: int, stream=None) -> 
 def kvq_decode_attn_static(ctx: int, layer: int, Q, O, stream=None) -> None:
     """kvq_decode_attn with the split partials in the library's fixed device array: allocates nothing."""
     check(lib().kvq_decode_attn_static(ctx, layer, _ptr(Q), _ptr(O), _stream(stream)), "kvq_decode_attn_static")
+
+
+def kvq_decode_step(ctx: int, layer: int, feats, K, V, Q, O, bits_out=None, stream=None) -> None:
+    """One decode step on device buffers: kvq_append_fused of one token per sequence, then kvq_decode_attn."""
+    check(lib().kvq_decode_step(ctx, layer, _ptr(feats), _ptr(K), _ptr(V), _ptr(Q), _ptr(O), _ptr(bits_out),
+                                _stream(stream)), "kvq_decode_step")
 
 
 def kvq_decode_step_host(ctx: int, layer: int, feats, K, V, Q, O, bits_out=None, stream=None) -> None:

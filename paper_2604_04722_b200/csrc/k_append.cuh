@@ -634,20 +634,16 @@ __device__ __forceinline__ void token_store_pc(int c, const uint4 (&kraw)[4], co
     }
 }
 
-// One new token per sequence (a decode step): grid = (ceil(kv_heads / 16), batch), block = 32 -- or 128 when the
-// controller is wider than 32 hidden units: the three extra warps only help with the decision.
-// Lane l handles half-row l%2 of KV head 16*blockIdx.x + l/2.  Everything the warp needs (the K and V
-// rows, the pool fills, the features) is requested up front so the loads overlap the controller;
-// the decision is taken by the whole warp (FUSED, any hidden width) or read from `bits`.
+// One new token per sequence (a decode step), the work of one warp: the token of sequence b, KV heads
+// 16 bx .. 16 bx + 15; lane l handles half-row l % 2 of KV head 16 bx + l / 2.  Everything the warp needs (the K and
+// V rows, the pool fills, the features) is requested up front so the loads overlap the controller; the decision is
+// taken by the warp (FUSED) or read from `bits`.  wide: the warp is the first of a CTA of four whose other warps
+// help with a controller wider than 32 hidden units (they call this too and return after the decision;
+// controller_fetch_cta128 has been called by all of them).
 template <bool FUSED, int G>
-__global__ void __launch_bounds__(128)
-k_append_token(AppendParams p) {
-    extern __shared__ __align__(16) float ctrl_sh[];    // kControllerCtaSmemFloats floats when four warps evaluate the controller
-    pdl_launch_dependents();
-    if (FUSED && blockDim.x != 32) controller_fetch_cta128(p.ctrl, p.hidden, ctrl_sh);   // no kernel writes the weights
-    pdl_wait();                                        // the attention of the previous step still reads the store
-    const int lane = threadIdx.x & 31, b = blockIdx.y;
-    const int h = blockIdx.x * 16 + (lane >> 1), half = lane & 1;
+__device__ __forceinline__ void append_token_warp(const AppendParams& p, int bx, int b, bool wide, float* ctrl_sh) {
+    const int lane = threadIdx.x & 31;
+    const int h = bx * 16 + (lane >> 1), half = lane & 1;
     const bool active = h < p.store.kv_heads;
     uint4 kraw[4], vraw[4];
 #pragma unroll
@@ -674,14 +670,14 @@ k_append_token(AppendParams p) {
     int c;
     if (FUSED) {
         const float4 f = reinterpret_cast<const float4*>(p.feats)[b];
-        c = blockDim.x == 32 ? controller_decide_warp32(p.ctrl, f.x, f.y, f.z, f.w, lane)
-                             : controller_decide_cta128(p.ctrl, p.hidden, f.x, f.y, f.z, f.w, ctrl_sh);
-        if (threadIdx.x >= 32) return;                 // the helpers are done
+        c = !wide ? controller_decide_warp32(p.ctrl, f.x, f.y, f.z, f.w, lane)
+                  : controller_decide_cta128(p.ctrl, p.hidden, f.x, f.y, f.z, f.w, ctrl_sh);
+        if (wide && threadIdx.x >= 32) return;         // the helpers are done
     } else {
         c = class_of_bits(p.bits[b], p.store.flags);
     }
     const uint32_t slot = c == 0 ? fill.x : c == 1 ? fill.y : c == 2 ? fill.z : fill.w;
-    if (blockIdx.x == 0 && lane == 0) {
+    if (bx == 0 && lane == 0) {
         p.store.index[((size_t)p.layer * p.store.batch + b) * p.store.max_ctx + first_pos_of(p, b)] = ((uint32_t)c << 30) | slot;
         *reinterpret_cast<uint4*>(p.counts_out + (size_t)b * 4) =
             make_uint4(fill.x + (c == 0), fill.y + (c == 1), fill.z + (c == 2), fill.w + (c == 3));
@@ -711,6 +707,18 @@ k_append_token(AppendParams p) {
         token_store_pc(c, kraw, vraw, active, half, t, rec, c < 3 ? residual_rows(p.store, c, p.layer, b, active ? h : 0) : nullptr);
     else
         token_store<G>(c, kraw, vraw, active, half, t, rec);
+}
+
+// grid = (ceil(kv_heads / 16), batch), block = 32 -- or 128 when the controller is wider than 32 hidden units.
+template <bool FUSED, int G>
+__global__ void __launch_bounds__(128)
+k_append_token(AppendParams p) {
+    extern __shared__ __align__(16) float ctrl_sh[];    // kControllerCtaSmemFloats floats when four warps evaluate the controller
+    pdl_launch_dependents();
+    const bool wide = blockDim.x != 32;
+    if (FUSED && wide) controller_fetch_cta128(p.ctrl, p.hidden, ctrl_sh);   // no kernel writes the weights
+    pdl_wait();                                        // the attention of the previous step still reads the store
+    append_token_warp<FUSED, G>(p, (int)blockIdx.x, (int)blockIdx.y, wide, ctrl_sh);
 }
 
 }  // namespace kvq

@@ -49,6 +49,7 @@
 // linear), so one AND per element isolates it and the power of two is folded into the accumulator's exponent.
 #pragma once
 #include "kvq_common.cuh"
+#include "k_append.cuh"
 
 #ifndef KVQ_SMALL_WARPS
 #define KVQ_SMALL_WARPS 16
@@ -221,6 +222,22 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
     return v;
+}
+
+// What the store will hold for two elements of a 64-element row that the warp quantizes at class c (Eq. 24, the row
+// quantizer of k_append.cuh followed by x^ = code * scale + zero-point): every lane passes two of the row's elements,
+// all lanes the same c.  Class 3 keeps the fp16 values.
+__device__ __forceinline__ float2 row_values_as_stored(float2 x, int c) {
+    if (c == 3) return x;
+    float mn = -warp_max(-fminf(x.x, x.y)), mx = warp_max(fmaxf(x.x, x.y));
+    if (mn == 0.0f) mn = 0.0f;                         // -0 is stored as +0
+    if (mx == 0.0f) mx = 0.0f;
+    const float levels = c == 0 ? 3.0f : c == 1 ? 15.0f : 255.0f;
+    const float sf = __half2float(__float2half_rn(__fdiv_rn(__fsub_rn(mx, mn), levels)));
+    const float inv = sf == 0.0f ? 0.0f : __frcp_rn(sf);
+    const float c0 = rintf(fminf(__fmul_rn(__fsub_rn(x.x, mn), inv), levels));
+    const float c1 = rintf(fminf(__fmul_rn(__fsub_rn(x.y, mn), inv), levels));
+    return make_float2(__fadd_rn(__fmul_rn(c0, sf), mn), __fadd_rn(__fmul_rn(c1, sf), mn));
 }
 
 __device__ __forceinline__ float half_sum(float v) {    // over the 16 lanes of a half-warp
@@ -905,9 +922,15 @@ __device__ __forceinline__ void merge_partials(const DecodeParams& P, uint32_t u
 // STATS: also emit, per unit, the variance of its attention weights over the cached tokens.
 // P.cta_parts > 0: every unit is cut into that many parts (a divisor of Geo::kWarps), so all parts of a unit run in
 // one CTA, which merges them through shared memory.
-template <bool STATS, int G, class Geo>
-__global__ void __launch_bounds__(Geo::kThreads, Geo::kCtasPerSm)
-k_decode_attn(DecodeParams P) {
+//
+// STEP (one scale group per row only): the launch is a whole decode step.  `P.counts` are the pool fills BEFORE the
+// step's token, whose fp16 rows, features and controller come in A; other CTAs of the same launch store it (see
+// k_decode_step) and nobody waits for them: the warp that works on the last part of a unit evaluates the controller
+// itself, quantizes the token's K and V rows in registers the way the store does (row_values_as_stored) and adds the
+// token to its partial.  The slot the token is being written to lies beyond the fills this launch reads.
+template <bool STATS, int G, class Geo, bool STEP>
+__device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const AppendParams* A) {
+    static_assert(!STEP || (G == 1 && !STATS), "the one-launch step exists for the plain decode of one scale group per row");
     constexpr int kStages = Geo::kStages, kStageBytes = Geo::kStageBytes;
     extern __shared__ __align__(128) uint8_t ring[];   // [warps][stages][kStageBytes]
     __shared__ WarpScratch<kStages> scratch[Geo::kWarps];
@@ -949,6 +972,15 @@ k_decode_attn(DecodeParams P) {
         const uint32_t b = row / P.tq;                 // row = b * tq + (query row - t0)
         const size_t qo = (((size_t)b * P.t_total + P.t0 + (row - b * P.tq)) * P.store.q_heads + qh) * kHeadDim;
         const int kvh = (int)qh / P.group;
+        const bool adds_token = STEP && a1 == P.gw;    // this warp works on the unit's last part
+        __half2 k_new = __half2(), v_new = __half2();  // elements 2 lane, 2 lane + 1 of the step's token
+        if constexpr (STEP) {
+            if (adds_token) {
+                const size_t src = ((size_t)b * P.store.kv_heads + kvh) * kHeadDim;
+                k_new = reinterpret_cast<const __half2*>(A->K + src)[lane];
+                v_new = reinterpret_cast<const __half2*>(A->V + src)[lane];
+            }
+        }
         if (lane < kNumPools) {                        // lane c plans pool c
             const int c = lane;
             const uint32_t* tab = stream_table(P.store, c, P.layer, (int)b, kvh);
@@ -1254,6 +1286,23 @@ k_decode_attn(DecodeParams P) {
             r2[1] += b_w;
         }
         const float s2_w = STATS ? (G != 2 ? 1.0f : 0.5f) * warp_sum(st.s2) : 0.f;
+        float l_tot = l_w;
+        if constexpr (STEP) {
+            if (adds_token) {                          // warp-uniform
+                const float4 f = reinterpret_cast<const float4*>(A->feats)[b];
+                const int c = controller_decide_warp32(A->ctrl, f.x, f.y, f.z, f.w, lane);
+                const float2 kh = row_values_as_stored(__half22float2(k_new), c), vh = row_values_as_stored(__half22float2(v_new), c);
+                const int i = 2 * lane;
+                const float* qp = ws.q + (i >> 5) * kQHalfStride + (i & 31);
+                const float y = warp_sum(fmaf(kh.y, qp[1], kh.x * qp[0])) * kLogitScale;
+                const float m_new = fmaxf(st.m, y);
+                const float keep = fast_exp2(st.m - m_new), e = fast_exp2(y - m_new);
+                r2[0] = fmaf(r2[0], keep, e * vh.x);
+                r2[1] = fmaf(r2[1], keep, e * vh.y);
+                l_tot = fmaf(l_w, keep, e);
+                st.m = m_new;
+            }
+        }
 
         if (Geo::kCtaMerge && P.cta_parts) {
             // ---- all parts of the unit run in this CTA: partials and the arrival counter stay in shared memory
@@ -1261,7 +1310,7 @@ k_decode_attn(DecodeParams P) {
             const int wf = warp - (int)(j % parts);    // the unit's first warp in this CTA holds its counter
             reinterpret_cast<float2*>(ws.o)[lane] = make_float2(r2[0], r2[1]);
             if (lane == 0) {
-                ws.ml = make_float2(st.m, l_w);
+                ws.ml = make_float2(st.m, l_tot);
                 ws.s2 = s2_w;
             }
             __syncwarp();
@@ -1290,7 +1339,7 @@ k_decode_attn(DecodeParams P) {
         const uint32_t jf = decode_first_warp(u, P.units, P.gw);
         const size_t rec0 = (size_t)u * P.pslots;
         reinterpret_cast<float2*>(P.part_o + (rec0 + (j - jf)) * kHeadDim)[lane] = make_float2(r2[0], r2[1]);
-        if (lane == 0) P.part_ml[rec0 + (j - jf)] = make_float2(st.m, l_w);
+        if (lane == 0) P.part_ml[rec0 + (j - jf)] = make_float2(st.m, l_tot);
         if (STATS) {
             if (lane == 0) P.part_s2[rec0 + (j - jf)] = s2_w;
         }
@@ -1311,6 +1360,31 @@ k_decode_attn(DecodeParams P) {
             if (lane == 0) P.part_cnt[u] = 0;
         }
     }
+}
+
+template <bool STATS, int G, class Geo>
+__global__ void __launch_bounds__(Geo::kThreads, Geo::kCtasPerSm)
+k_decode_attn(DecodeParams P) {
+    decode_attn_body<STATS, G, Geo, false>(P, nullptr);
+}
+
+// One decode step (Eq. 4, then Eq. 5) in one launch: the first ceil(gw / Geo::kWarps) CTAs attend over the cache
+// as it was plus the step's token (decode_attn_body with STEP), the others store the token: every warp of theirs
+// is one warp of k_append_token.  Neither side reads what the other writes.  Controller width 32 only.
+// grid = ceil(gw / Geo::kWarps) + ceil(batch * ceil(kv_heads / 16) / Geo::kWarps).
+template <class Geo>
+__global__ void __launch_bounds__(Geo::kThreads, Geo::kCtasPerSm)
+k_decode_step(DecodeParams P, AppendParams A) {
+    const uint32_t attn_ctas = (P.gw + Geo::kWarps - 1) / Geo::kWarps;
+    if (blockIdx.x < attn_ctas) {
+        decode_attn_body<false, 1, Geo, true>(P, &A);
+        return;
+    }
+    pdl_launch_dependents();
+    pdl_wait();                                        // the attention of the previous step still reads the store
+    const int head_groups = (A.store.kv_heads + 15) / 16;
+    const int item = (int)(blockIdx.x - attn_ctas) * Geo::kWarps + (int)(threadIdx.x >> 5);
+    if (item < head_groups * A.store.batch) append_token_warp<true, 1>(A, item % head_groups, item / head_groups, false, nullptr);
 }
 
 // Pool fills each of the last t_total cached tokens may see when it asks as a query (causal

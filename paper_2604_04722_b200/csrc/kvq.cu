@@ -153,8 +153,8 @@ static_assert(KVQ_APPEND_TOKENS_PER_THREAD >= 1 && KVQ_APPEND_TOKENS_PER_THREAD 
 #endif
 // Launch with programmatic stream serialization (see pdl_wait): the kernel may be scheduled before the
 // kernel ahead of it in the stream has finished, if that kernel allows it; it waits inside for its end.
-template <class Params>
-void launch_overlapped(void (*kernel)(Params), dim3 grid, unsigned block, size_t smem, cudaStream_t st, const Params& p) {
+template <class... Params>
+void launch_overlapped(void (*kernel)(Params...), dim3 grid, unsigned block, size_t smem, cudaStream_t st, const Params&... p) {
 #if KVQ_OVERLAP_LAUNCHES
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
@@ -166,9 +166,9 @@ void launch_overlapped(void (*kernel)(Params), dim3 grid, unsigned block, size_t
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, kernel, p);
+    cudaLaunchKernelEx(&cfg, kernel, p...);
 #else
-    kernel<<<grid, block, smem, st>>>(p);
+    kernel<<<grid, block, smem, st>>>(p...);
 #endif
 }
 
@@ -789,6 +789,7 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
              dyn_smem(k_decode_attn<false, 2, GeomSmall>, (int)GeomSmall::kSmemBytes);
         ok = ok && dyn_smem(k_decode_attn<true, 1, GeomSmall>, (int)GeomSmall::kSmemBytes) &&
              dyn_smem(k_decode_attn<true, 2, GeomSmall>, (int)GeomSmall::kSmemBytes);
+        ok = ok && dyn_smem(k_decode_step<GeomSmall>, (int)GeomSmall::kSmemBytes);
         ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     }
     if (!ok) {
@@ -889,6 +890,67 @@ int kvq_decode_attn(kvq_ctx* c, int layer, const void* Q, void* O, void* stream)
     }
     c->launches += 1;
     KVQ_CUDA(c, cudaGetLastError());
+    return KVQ_OK;
+}
+
+int kvq_decode_step(kvq_ctx* c, int layer, const float* feats, const void* K, const void* V, const void* Q, void* O,
+                    uint8_t* bits_out_opt, void* stream) {
+    TraceRange trace("kvq_decode_step");
+    if (check_layer(c, layer) != KVQ_OK || !feats || !K || !V || !Q || !O) return KVQ_ERR_ARG;
+    if (!aligned16(K) || !aligned16(V) || !aligned16(feats)) return KVQ_ERR_ARG;
+    if (c->hidden == 0) return KVQ_ERR_NO_CONTROLLER;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // One launch when the attention is a chain of latencies rather than a stream (the plan takes the small geometry)
+    // and the warp that adds the token can evaluate the controller alone; otherwise the two calls, whose kernels
+    // overlap their launches.
+    const uint64_t units = (uint64_t)c->batch * c->q_heads;
+    DecodePlan plan;
+    bool one_launch = c->groups == 1 && c->hidden == 32 && !c->ragged[layer];
+    if (one_launch) {
+        plan = choose_plan(c, c->len[layer], units);
+        one_launch = plan.small && plan.gw > 0;
+    }
+    if (!one_launch) {
+        const int rc = append_impl(c, layer, K, V, nullptr, feats, bits_out_opt, 1, nullptr, st);
+        return rc != KVQ_OK ? rc : kvq_decode_attn(c, layer, Q, O, stream);
+    }
+    int* cur_lens = &c->lens[(size_t)layer * c->batch];
+    for (int b = 0; b < c->batch; ++b)
+        if (cur_lens[b] + 1 > c->max_ctx) return KVQ_ERR_CAPACITY;
+    DeviceGuard guard(c->device);
+    AppendParams a{};
+    a.store = c->store;
+    a.K = static_cast<const __half*>(K);
+    a.V = static_cast<const __half*>(V);
+    a.feats = feats;
+    a.ctrl = c->ctrl;
+    a.hidden = c->hidden;
+    a.bits_out = bits_out_opt;
+    a.counts_in = counts_of(c, c->cur[layer], layer);
+    a.counts_out = counts_of(c, c->cur[layer] ^ 1, layer);
+    a.layer = layer;
+    a.n_new = 1;
+    a.pos0 = c->len[layer];
+    a.tpt = 1;
+    a.nchunks = 1;
+    DecodeParams p{};
+    fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, plan, p);      // the fills before the step
+    const unsigned attn_ctas = (p.gw + GeomSmall::kWarps - 1) / GeomSmall::kWarps;
+    const unsigned items = (unsigned)c->batch * (unsigned)((c->kv_heads + 15) / 16);
+    const dim3 grid(attn_ctas + (items + GeomSmall::kWarps - 1) / GeomSmall::kWarps);
+    const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
+    cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 2] : nullptr;
+    if (rec) cudaEventRecord(ev[0], st);
+    launch_overlapped(k_decode_step<GeomSmall>, grid, GeomSmall::kThreads, GeomSmall::kSmemBytes, st, p, a);
+    if (rec) {
+        cudaEventRecord(ev[1], st);
+        c->prof_calls += 1;
+    }
+    c->launches += 1;
+    KVQ_CUDA(c, cudaGetLastError());
+    c->cur[layer] ^= 1;
+    for (int b = 0; b < c->batch; ++b) cur_lens[b] += 1;
+    c->len[layer] += 1;
     return KVQ_OK;
 }
 
@@ -1036,9 +1098,7 @@ int kvq_decode_step_host(kvq_ctx* c, int layer, const float* feats, const void* 
         d_Q = c->st_Q;
         d_O = c->st_O;
     }
-    int rc = kvq_append_fused(c, layer, d_K, d_V, static_cast<const float*>(d_feats), 1, c->st_bits, stream);
-    if (rc != KVQ_OK) return rc;
-    rc = kvq_decode_attn(c, layer, d_Q, d_O, stream);
+    const int rc = kvq_decode_step(c, layer, static_cast<const float*>(d_feats), d_K, d_V, d_Q, d_O, c->st_bits, stream);
     if (rc != KVQ_OK) return rc;
     if (!direct) KVQ_CUDA(c, cudaMemcpyAsync(O, c->st_O, q_bytes, cudaMemcpyDeviceToHost, st));
     if (bits_out_opt) KVQ_CUDA(c, cudaMemcpyAsync(bits_out_opt, c->st_bits, c->batch, cudaMemcpyDeviceToHost, st));

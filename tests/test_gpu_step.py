@@ -1,0 +1,176 @@
+"""GPU parity of kvq_decode_step: one decode step (controller decision, quantize-append of one
+token per sequence, attention over everything cached, Eq. 19-24, Eq. 4, Eq. 5) against the
+oracle, step by step.  Short caches with a controller of width 32 take the one-launch kernel (the
+attending warps add the step's token themselves from its fp16 rows); every other case runs the two
+kernels of kvq_append_fused + kvq_decode_attn behind the same call.  Both are compared with the
+oracle the same way: decisions and the whole store bit for bit, the attention output of EVERY
+step within the attention tolerance."""
+import numpy as np
+import pytest
+
+from paper_2604_04722_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+BITS = np.array([2, 4, 8, 16], dtype=np.uint8)
+
+
+@pytest.fixture(scope="module")
+def gu():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_04722_b200 import build
+    build.build()
+    import gpu_util
+    return gpu_util
+
+
+def _kv(rng, B, n, H, scale=1.0):
+    K = (rng.standard_normal((B, n, H, 64)) * scale).astype(np.float16)
+    V = (rng.standard_normal((B, n, H, 64)) * scale).astype(np.float16)
+    return K, V
+
+
+def _step(gu, g, layer, feats, K, V, Q):
+    """kvq_decode_step through the binding; returns (decisions [B], output [B][Hq][64] as uint16)."""
+    import torch
+    from paper_2604_04722_b200 import binding as kq
+    fd, Kd, Vd = gu.dev(feats.astype(np.float32)), gu.dev(K.view(np.uint16)), gu.dev(V.view(np.uint16))
+    Qd = gu.dev(Q.view(np.uint16))
+    O = torch.zeros_like(Qd)
+    bits = torch.zeros(feats.shape[0], dtype=torch.uint8, device=gu.DEV)
+    kq.kvq_decode_step(g.ctx, layer, fd, Kd, Vd, Qd, O, bits)
+    torch.cuda.synchronize()
+    return bits.cpu().numpy(), O.cpu().numpy().view(np.uint16)
+
+
+def _run_steps(gu, oracle, g, oc, cw, rng, B, Hq, H, steps, what, feat_seed=3, kscale=1.0, layer=0, first_pos=0):
+    from paper_2604_04722_b200 import binding as kq
+    feats = synth.features_batch(feat_seed, B, first_pos, steps)
+    want_bits, want_logits, gap = oracle.select_bits(feats, cw.hidden, *cw.as_tuple())
+    got_bits = np.zeros_like(want_bits)
+    launches0 = kq.kvq_launch_count(g.ctx)
+    for s in range(steps):
+        K, V = _kv(rng, B, 1, H, kscale)
+        Q = rng.standard_normal((B, Hq, 64)).astype(np.float16)
+        oc.append(K, V, want_bits[:, s:s + 1])
+        got_bits[:, s], out = _step(gu, g, layer, feats[:, s], K, V, Q)
+        gu.assert_attention_close(out, oc.decode_attn(Q), "%s, step %d" % (what, s))
+    near = gu.compare_decisions(got_bits, want_bits, want_logits, gap, what)
+    assert all(r[3] == r[4] for r in near)      # the oracle's store below was built from the oracle's decisions
+    assert kq.kvq_device_status(g.ctx) == 0
+    return kq.kvq_launch_count(g.ctx) - launches0
+
+
+@pytest.mark.parametrize("B,Hq,H", [(3, 6, 2), (1, 9, 3), (2, 20, 20)])
+def test_steps_from_an_empty_cache_take_one_launch_each(gu, oracle, B, Hq, H):
+    """From nothing cached: the first step attends over its own token only.  70 steps cross several tiles of every
+    pool; 20 KV heads need two storing warps per sequence."""
+    rng = np.random.default_rng(100 + B)
+    cw = synth.controller_weights(322, 32)
+    steps = 70
+    oc = oracle.OracleCache(B, Hq, H)
+    with gu.GpuCache(1, B, Hq, H, steps) as g:
+        g.set_controller(cw)
+        launches = _run_steps(gu, oracle, g, oc, cw, rng, B, Hq, H, steps, "step from empty B=%d" % B)
+        assert launches == steps                 # one kernel per step
+        gu.assert_store_equals_oracle(g, 0, oc)
+        assert len(set(oc.bits.ravel().tolist())) >= 3
+
+
+@pytest.mark.parametrize("splits", [0, 1, 2, 7, 16])
+def test_steps_after_a_prefill_for_every_way_of_cutting_the_work(gu, oracle, splits):
+    """Prefill of mixed precision, then steps; the split count decides whether the parts of a unit meet inside
+    their CTA (1, 2, 16, automatic) or through partial records (7): the token is added by the unit's last part."""
+    from paper_2604_04722_b200 import binding as kq
+    rng = np.random.default_rng(200 + splits)
+    cw = synth.controller_weights(98, 32)
+    B, Hq, H, n, steps = 2, 9, 3, 777, 24
+    oc = oracle.OracleCache(B, Hq, H)
+    with gu.GpuCache(2, B, Hq, H, n + steps) as g:
+        g.set_controller(cw)
+        kq.kvq_set_splits(g.ctx, splits)
+        K, V = _kv(rng, B, n, H, 1.5)
+        bits = BITS[rng.choice(4, size=(B, n))]
+        oc.append(K, V, bits)
+        g.append(1, K, V, bits)
+        launches = _run_steps(gu, oracle, g, oc, cw, rng, B, Hq, H, steps, "step after prefill, splits=%d" % splits,
+                              kscale=1.5, layer=1, first_pos=n)
+        assert launches == steps
+        gu.assert_store_equals_oracle(g, 1, oc)
+
+
+def test_steps_that_open_new_blocks_and_new_tiles(gu, oracle):
+    """All tokens in one class (a controller whose biases decide): the 2-bit stream of a sequence fills its first
+    64 KB block (102 tiles) during the steps and goes on in a second one."""
+    rng = np.random.default_rng(5)
+    H32 = 32
+    z = np.zeros
+    cw = synth.ControllerWeights(H32, z((H32, 4), np.float32), z(H32, np.float32), z((H32, H32), np.float32),
+                                 z(H32, np.float32), z((4, H32), np.float32), np.array([1, 0, 0, 0], np.float32))
+    B, Hq, H = 1, 2, 1
+    n = 102 * 16 - 5
+    steps = 12
+    oc = oracle.OracleCache(B, Hq, H)
+    with gu.GpuCache(1, B, Hq, H, n + steps) as g:
+        g.set_controller(cw)
+        K, V = _kv(rng, B, n, H)
+        bits = np.full((B, n), 2, np.uint8)
+        oc.append(K, V, bits)
+        g.append(0, K, V, bits)
+        _run_steps(gu, oracle, g, oc, cw, rng, B, Hq, H, steps, "steps across a block border", first_pos=n)
+        assert set(oc.bits.ravel().tolist()) == {2}
+        gu.assert_store_equals_oracle(g, 0, oc, pos0=n - 40, n=40 + steps)
+
+
+@pytest.mark.parametrize("case", ["hidden 128", "two scale groups", "per-channel keys", "long cache"])
+def test_steps_that_run_as_two_kernels(gu, oracle, case):
+    """The same call where the one-launch kernel does not apply: it must give the same results."""
+    rng = np.random.default_rng(len(case))
+    hidden = 128 if case == "hidden 128" else 32
+    cw = synth.controller_weights(2 if hidden == 128 else 322, hidden)
+    B, Hq, H, steps = 2, 4, 2, 20
+    n = 40000 if case == "long cache" else 300
+    if case == "two scale groups":
+        oc = oracle.GroupedOracleCache(B, Hq, H, 2)
+        g = gu.GpuCache(1, B, Hq, H, n + steps, scale_groups=2)
+    elif case == "per-channel keys":
+        oc = oracle.PerChannelKCache(B, Hq, H)
+        g = gu.GpuCache(1, B, Hq, H, n + steps, k_per_channel=True)
+    else:
+        oc = oracle.OracleCache(B, Hq, H)
+        g = gu.GpuCache(1, B, Hq, H, n + steps)
+    with g:
+        g.set_controller(cw)
+        K, V = _kv(rng, B, n, H)
+        bits = BITS[rng.choice(4, size=(B, n))]
+        oc.append(K, V, bits)
+        g.append(0, K, V, bits)
+        launches = _run_steps(gu, oracle, g, oc, cw, rng, B, Hq, H, steps, "two-kernel step, %s" % case, first_pos=n)
+        assert launches >= 2 * steps
+
+
+def test_step_argument_and_capacity_errors(gu):
+    import torch
+    from paper_2604_04722_b200 import binding as kq
+    B, Hq, H = 1, 2, 1
+    with gu.GpuCache(1, B, Hq, H, 2) as g:
+        f = torch.zeros((B, 4), device=gu.DEV)
+        K = torch.zeros((B, 1, H, 64), dtype=torch.float16, device=gu.DEV)
+        Q = torch.zeros((B, Hq, 64), dtype=torch.float16, device=gu.DEV)
+        O = torch.zeros_like(Q)
+        with pytest.raises(kq.KvqError) as e:
+            kq.kvq_decode_step(g.ctx, 0, f, K, K, Q, O)
+        assert e.value.code == kq.KVQ_ERR_NO_CONTROLLER
+        g.set_controller(synth.controller_weights(322, 32))
+        with pytest.raises(kq.KvqError) as e:
+            kq.kvq_decode_step(g.ctx, 3, f, K, K, Q, O)
+        assert e.value.code == kq.KVQ_ERR_ARG
+        kq.kvq_decode_step(g.ctx, 0, f, K, K, Q, O)
+        kq.kvq_decode_step(g.ctx, 0, f, K, K, Q, O)
+        with pytest.raises(kq.KvqError) as e:
+            kq.kvq_decode_step(g.ctx, 0, f, K, K, Q, O)
+        assert e.value.code == kq.KVQ_ERR_CAPACITY
+        torch.cuda.synchronize()
+        assert kq.kvq_device_status(g.ctx) == 0
