@@ -789,7 +789,7 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
              dyn_smem(k_decode_attn<false, 2, GeomSmall>, (int)GeomSmall::kSmemBytes);
         ok = ok && dyn_smem(k_decode_attn<true, 1, GeomSmall>, (int)GeomSmall::kSmemBytes) &&
              dyn_smem(k_decode_attn<true, 2, GeomSmall>, (int)GeomSmall::kSmemBytes);
-        ok = ok && dyn_smem(k_decode_step<GeomSmall>, (int)GeomSmall::kSmemBytes);
+        ok = ok && dyn_smem(k_decode_step<GeomSmall>, (int)GeomSmall::kSmemBytes) && dyn_smem(k_decode_step<GeomLarge>, (int)GeomLarge::kSmemBytes);
         ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     }
     if (!ok) {
@@ -900,15 +900,14 @@ int kvq_decode_step(kvq_ctx* c, int layer, const float* feats, const void* K, co
     if (!aligned16(K) || !aligned16(V) || !aligned16(feats)) return KVQ_ERR_ARG;
     if (c->hidden == 0) return KVQ_ERR_NO_CONTROLLER;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // One launch when the attention is a chain of latencies rather than a stream (the plan takes the small geometry)
-    // and the warp that adds the token can evaluate the controller alone; otherwise the two calls, whose kernels
-    // overlap their launches.
+    // One launch when the warp that adds the token can evaluate the controller alone (hidden width 32) and the
+    // layout is the plain one; otherwise the two calls, whose kernels overlap their launches.
     const uint64_t units = (uint64_t)c->batch * c->q_heads;
     DecodePlan plan;
     bool one_launch = c->groups == 1 && c->hidden == 32 && !c->ragged[layer];
     if (one_launch) {
         plan = choose_plan(c, c->len[layer], units);
-        one_launch = plan.small && plan.gw > 0;
+        one_launch = plan.gw > 0;
     }
     if (!one_launch) {
         const int rc = append_impl(c, layer, K, V, nullptr, feats, bits_out_opt, 1, nullptr, st);
@@ -935,13 +934,15 @@ int kvq_decode_step(kvq_ctx* c, int layer, const float* feats, const void* K, co
     a.nchunks = 1;
     DecodeParams p{};
     fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, plan, p);      // the fills before the step
-    const unsigned attn_ctas = (p.gw + GeomSmall::kWarps - 1) / GeomSmall::kWarps;
+    const unsigned cta_warps = plan.small ? GeomSmall::kWarps : GeomLarge::kWarps;
+    const unsigned attn_ctas = (p.gw + cta_warps - 1) / cta_warps;
     const unsigned items = (unsigned)c->batch * (unsigned)((c->kv_heads + 15) / 16);
-    const dim3 grid(attn_ctas + (items + GeomSmall::kWarps - 1) / GeomSmall::kWarps);
+    const dim3 grid(attn_ctas + (items + cta_warps - 1) / cta_warps);
     const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
     cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 2] : nullptr;
     if (rec) cudaEventRecord(ev[0], st);
-    launch_overlapped(k_decode_step<GeomSmall>, grid, GeomSmall::kThreads, GeomSmall::kSmemBytes, st, p, a);
+    if (plan.small) launch_overlapped(k_decode_step<GeomSmall>, grid, GeomSmall::kThreads, GeomSmall::kSmemBytes, st, p, a);
+    else launch_overlapped(k_decode_step<GeomLarge>, grid, GeomLarge::kThreads, GeomLarge::kSmemBytes, st, p, a);
     if (rec) {
         cudaEventRecord(ev[1], st);
         c->prof_calls += 1;

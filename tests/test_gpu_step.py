@@ -1,8 +1,8 @@
 """GPU parity of kvq_decode_step: one decode step (controller decision, quantize-append of one
 token per sequence, attention over everything cached, Eq. 19-24, Eq. 4, Eq. 5) against the
-oracle, step by step.  Short caches with a controller of width 32 take the one-launch kernel (the
-attending warps add the step's token themselves from its fp16 rows); every other case runs the two
-kernels of kvq_append_fused + kvq_decode_attn behind the same call.  Both are compared with the
+oracle, step by step.  With one scale group per row and a controller of width 32 the step is one
+launch (the attending warps add the step's token themselves from its fp16 rows); every other case
+runs the two kernels of kvq_append_fused + kvq_decode_attn behind the same call.  Both are compared with the
 oracle the same way: decisions and the whole store bit for bit, the attention output of EVERY
 step within the attention tolerance."""
 import numpy as np
@@ -124,14 +124,35 @@ def test_steps_that_open_new_blocks_and_new_tiles(gu, oracle):
         gu.assert_store_equals_oracle(g, 0, oc, pos0=n - 40, n=40 + steps)
 
 
-@pytest.mark.parametrize("case", ["hidden 128", "two scale groups", "per-channel keys", "long cache"])
+@pytest.mark.parametrize("splits", [0, 3, 4])
+def test_steps_on_a_long_cache_in_the_bandwidth_geometry(gu, oracle, splits):
+    """40 000 cached tokens per sequence: the launch takes the geometry of four-warp CTAs; parts of a unit meet
+    through partial records (automatic plan, 3) or inside their CTA (4)."""
+    from paper_2604_04722_b200 import binding as kq
+    rng = np.random.default_rng(300 + splits)
+    cw = synth.controller_weights(322, 32)
+    B, Hq, H, n, steps = 2, 4, 2, 40000, 10
+    oc = oracle.OracleCache(B, Hq, H)
+    with gu.GpuCache(1, B, Hq, H, n + steps) as g:
+        g.set_controller(cw)
+        kq.kvq_set_splits(g.ctx, splits)
+        K, V = _kv(rng, B, n, H)
+        bits = BITS[rng.choice(4, size=(B, n))]
+        oc.append(K, V, bits)
+        g.append(0, K, V, bits)
+        launches = _run_steps(gu, oracle, g, oc, cw, rng, B, Hq, H, steps, "step on a long cache, splits=%d" % splits, first_pos=n)
+        assert launches == steps
+        gu.assert_store_equals_oracle(g, 0, oc, pos0=n - 64, n=64 + steps)
+
+
+@pytest.mark.parametrize("case", ["hidden 128", "two scale groups", "per-channel keys"])
 def test_steps_that_run_as_two_kernels(gu, oracle, case):
     """The same call where the one-launch kernel does not apply: it must give the same results."""
     rng = np.random.default_rng(len(case))
     hidden = 128 if case == "hidden 128" else 32
     cw = synth.controller_weights(2 if hidden == 128 else 322, hidden)
     B, Hq, H, steps = 2, 4, 2, 20
-    n = 40000 if case == "long cache" else 300
+    n = 300
     if case == "two scale groups":
         oc = oracle.GroupedOracleCache(B, Hq, H, 2)
         g = gu.GpuCache(1, B, Hq, H, n + steps, scale_groups=2)
@@ -149,6 +170,41 @@ def test_steps_that_run_as_two_kernels(gu, oracle, case):
         g.append(0, K, V, bits)
         launches = _run_steps(gu, oracle, g, oc, cw, rng, B, Hq, H, steps, "two-kernel step, %s" % case, first_pos=n)
         assert launches >= 2 * steps
+
+
+def test_steps_on_a_layer_of_ragged_lengths_run_as_two_kernels(gu, oracle):
+    """Sequences of different lengths (one of them empty before the first step): every sequence against its own
+    oracle cache."""
+    from paper_2604_04722_b200 import binding as kq
+    rng = np.random.default_rng(77)
+    cw = synth.controller_weights(322, 32)
+    B, Hq, H, steps = 3, 6, 2, 9
+    lens = [200, 0, 57]
+    ocs = [oracle.OracleCache(1, Hq, H) for _ in range(B)]
+    with gu.GpuCache(1, B, Hq, H, 200 + steps) as g:
+        g.set_controller(cw)
+        K, V = _kv(rng, B, 200, H)
+        bits = BITS[rng.choice(4, size=(B, 200))]
+        kq.kvq_append_ragged(g.ctx, 0, gu.dev(K.view(np.uint16)), gu.dev(V.view(np.uint16)), gu.dev(bits), None, 200, lens)
+        for b in range(B):
+            if lens[b]:
+                ocs[b].append(K[b:b + 1, :lens[b]], V[b:b + 1, :lens[b]], bits[b:b + 1, :lens[b]])
+        feats = synth.features_batch(11, B, 0, steps)
+        want_bits, want_logits, gap = oracle.select_bits(feats, 32, *cw.as_tuple())
+        got_bits = np.zeros_like(want_bits)
+        launches0 = kq.kvq_launch_count(g.ctx)
+        for s in range(steps):
+            K, V = _kv(rng, B, 1, H)
+            Q = rng.standard_normal((B, Hq, 64)).astype(np.float16)
+            got_bits[:, s], out = _step(gu, g, 0, feats[:, s], K, V, Q)
+            for b in range(B):
+                ocs[b].append(K[b:b + 1], V[b:b + 1], want_bits[b:b + 1, s:s + 1])
+                gu.assert_attention_close(out[b:b + 1], ocs[b].decode_attn(Q[b:b + 1]), "ragged step %d seq %d" % (s, b))
+        near = gu.compare_decisions(got_bits, want_bits, want_logits, gap, "steps on ragged lengths")
+        assert all(r[3] == r[4] for r in near)
+        assert kq.kvq_launch_count(g.ctx) - launches0 >= 2 * steps
+        assert kq.kvq_seq_lens(g.ctx, 0, B).tolist() == [l + steps for l in lens]
+        assert kq.kvq_device_status(g.ctx) == 0
 
 
 def test_step_argument_and_capacity_errors(gu):
