@@ -900,11 +900,12 @@ int kvq_decode_step(kvq_ctx* c, int layer, const float* feats, const void* K, co
     if (!aligned16(K) || !aligned16(V) || !aligned16(feats)) return KVQ_ERR_ARG;
     if (c->hidden == 0) return KVQ_ERR_NO_CONTROLLER;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // One launch when the warp that adds the token can evaluate the controller alone (hidden width 32) and the
-    // layout is the plain one; otherwise the two calls, whose kernels overlap their launches.
+    // One launch when the warp that adds the token can evaluate the controller alone (hidden width 32: a wider
+    // one takes a single warp longer than the second launch costs) and the layout is the plain one; otherwise the
+    // two calls, whose kernels overlap their launches.
     const uint64_t units = (uint64_t)c->batch * c->q_heads;
     DecodePlan plan;
-    bool one_launch = c->groups == 1 && c->hidden == 32 && !c->ragged[layer];
+    bool one_launch = c->groups == 1 && c->hidden == 32;
     if (one_launch) {
         plan = choose_plan(c, c->len[layer], units);
         one_launch = plan.gw > 0;
@@ -932,6 +933,19 @@ int kvq_decode_step(kvq_ctx* c, int layer, const float* feats, const void* K, co
     a.pos0 = c->len[layer];
     a.tpt = 1;
     a.nchunks = 1;
+    if (c->ragged[layer]) {                            // every sequence's own position travels with the call
+        int *h_slot = nullptr, *d_slot = nullptr;
+        const int slot = claim_len_slot(c, &h_slot, &d_slot);
+        if (slot < 0) return slot;
+        for (int b = 0; b < c->batch; ++b) {
+            h_slot[b] = 1;
+            h_slot[c->batch + b] = cur_lens[b];
+        }
+        KVQ_CUDA(c, cudaMemcpyAsync(d_slot, h_slot, sizeof(int) * 2 * c->batch, cudaMemcpyHostToDevice, st));
+        KVQ_CUDA(c, cudaEventRecord(c->len_ev[slot], st));
+        a.lens = d_slot;
+        a.pos = d_slot + c->batch;
+    }
     DecodeParams p{};
     fill_decode_params(c, layer, Q, O, c->part_o, c->part_ml, c->part_cnt, plan, p);      // the fills before the step
     const unsigned cta_warps = plan.small ? GeomSmall::kWarps : GeomLarge::kWarps;

@@ -172,7 +172,7 @@ def test_steps_that_run_as_two_kernels(gu, oracle, case):
         assert launches >= 2 * steps
 
 
-def test_steps_on_a_layer_of_ragged_lengths_run_as_two_kernels(gu, oracle):
+def test_steps_on_a_layer_of_ragged_lengths(gu, oracle):
     """Sequences of different lengths (one of them empty before the first step): every sequence against its own
     oracle cache."""
     from paper_2604_04722_b200 import binding as kq
@@ -202,7 +202,13 @@ def test_steps_on_a_layer_of_ragged_lengths_run_as_two_kernels(gu, oracle):
                 gu.assert_attention_close(out[b:b + 1], ocs[b].decode_attn(Q[b:b + 1]), "ragged step %d seq %d" % (s, b))
         near = gu.compare_decisions(got_bits, want_bits, want_logits, gap, "steps on ragged lengths")
         assert all(r[3] == r[4] for r in near)
-        assert kq.kvq_launch_count(g.ctx) - launches0 >= 2 * steps
+        assert kq.kvq_launch_count(g.ctx) - launches0 == steps
+        for b in range(B):
+            for pos in sorted({0, lens[b] // 2, lens[b], lens[b] + steps - 1}):
+                bt, ps, kc, vc, km, vm = kq.kvq_export_token(g.ctx, 0, b, pos, H)
+                assert bt == int(ocs[b].bits[0, pos]) and ps == int(ocs[b].pool_slot[0, pos]), (b, pos)
+                assert np.array_equal(kc, ocs[b].kc[0, pos]) and np.array_equal(vc, ocs[b].vc[0, pos]), (b, pos)
+                assert np.array_equal(km, ocs[b].km[0, pos]) and np.array_equal(vm, ocs[b].vm[0, pos]), (b, pos)
         assert kq.kvq_seq_lens(g.ctx, 0, B).tolist() == [l + steps for l in lens]
         assert kq.kvq_device_status(g.ctx) == 0
 
