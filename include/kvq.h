@@ -312,8 +312,8 @@ int kvq_decode_attn_static(kvq_ctx* ctx, int layer, const void* Q, void* O, void
  * Q over everything cached in the layer, the new token included (Eq. 5).  Same result as
  * kvq_append_fused with n_new = 1 followed by kvq_decode_attn.  feats dev fp32 [batch][4];
  * K, V dev fp16 [batch][1][kv_heads][64]; Q, O dev fp16 [batch][q_heads][64]; bits_out_opt
- * dev uint8 [batch] or NULL.  Launches: ONE kernel when the handle has one scale group per
- * row and the controller has hidden width 32 (sequences of different lengths included): some
+ * dev uint8 [batch] or NULL.  Launches: ONE kernel when the keys are quantized per token (one
+ * or two scale groups) and the controller has hidden width 32, whatever the lengths: some
  * CTAs of the launch store the token while the others attend over the cache as it was and add
  * the token from its fp16 rows, quantized in registers exactly as it is stored, so neither
  * side waits for the other.  In every other case the two kernels of the two calls, whose

@@ -227,9 +227,17 @@ __device__ __forceinline__ float warp_sum(float v) {
 // What the store will hold for two elements of a 64-element row that the warp quantizes at class c (Eq. 24, the row
 // quantizer of k_append.cuh followed by x^ = code * scale + zero-point): every lane passes two of the row's elements,
 // all lanes the same c.  Class 3 keeps the fp16 values.
+// G = 2: the row has two scale groups of 32 elements, each quantized on its own; the lanes of a half-warp hold one.
+template <int G>
 __device__ __forceinline__ float2 row_values_as_stored(float2 x, int c) {
     if (c == 3) return x;
-    float mn = -warp_max(-fminf(x.x, x.y)), mx = warp_max(fmaxf(x.x, x.y));
+    float mn = -fminf(x.x, x.y), mx = fmaxf(x.x, x.y);
+#pragma unroll
+    for (int d = G == 2 ? 8 : 16; d > 0; d >>= 1) {
+        mn = fmaxf(mn, __shfl_xor_sync(0xffffffffu, mn, d));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+    }
+    mn = -mn;
     if (mn == 0.0f) mn = 0.0f;                         // -0 is stored as +0
     if (mx == 0.0f) mx = 0.0f;
     const float levels = c == 0 ? 3.0f : c == 1 ? 15.0f : 255.0f;
@@ -923,14 +931,14 @@ __device__ __forceinline__ void merge_partials(const DecodeParams& P, uint32_t u
 // P.cta_parts > 0: every unit is cut into that many parts (a divisor of Geo::kWarps), so all parts of a unit run in
 // one CTA, which merges them through shared memory.
 //
-// STEP (one scale group per row only): the launch is a whole decode step.  `P.counts` are the pool fills BEFORE the
+// STEP (not for per-channel keys): the launch is a whole decode step.  `P.counts` are the pool fills BEFORE the
 // step's token, whose fp16 rows, features and controller come in A; other CTAs of the same launch store it (see
 // k_decode_step) and nobody waits for them: the warp that works on the last part of a unit evaluates the controller
 // itself, quantizes the token's K and V rows in registers the way the store does (row_values_as_stored) and adds the
 // token to its partial.  The slot the token is being written to lies beyond the fills this launch reads.
 template <bool STATS, int G, class Geo, bool STEP>
 __device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const AppendParams* A) {
-    static_assert(!STEP || (G == 1 && !STATS), "the one-launch step exists for the plain decode of one scale group per row");
+    static_assert(!STEP || (G != kLayoutPerChannelK && !STATS), "the one-launch step exists for the plain decode with one pair per row or group");
     constexpr int kStages = Geo::kStages, kStageBytes = Geo::kStageBytes;
     extern __shared__ __align__(128) uint8_t ring[];   // [warps][stages][kStageBytes]
     __shared__ WarpScratch<kStages> scratch[Geo::kWarps];
@@ -1291,7 +1299,7 @@ __device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const Ap
             if (adds_token) {                          // warp-uniform
                 const float4 f = reinterpret_cast<const float4*>(A->feats)[b];
                 const int c = controller_decide_warp32(A->ctrl, f.x, f.y, f.z, f.w, lane);
-                const float2 kh = row_values_as_stored(__half22float2(k_new), c), vh = row_values_as_stored(__half22float2(v_new), c);
+                const float2 kh = row_values_as_stored<G>(__half22float2(k_new), c), vh = row_values_as_stored<G>(__half22float2(v_new), c);
                 const int i = 2 * lane;
                 const float* qp = ws.q + (i >> 5) * kQHalfStride + (i & 31);
                 const float y = warp_sum(fmaf(kh.y, qp[1], kh.x * qp[0])) * kLogitScale;
@@ -1372,19 +1380,19 @@ k_decode_attn(DecodeParams P) {
 // as it was plus the step's token (decode_attn_body with STEP), the others store the token: every warp of theirs
 // is one warp of k_append_token.  Neither side reads what the other writes.  Controller width 32 only.
 // grid = ceil(gw / Geo::kWarps) + ceil(batch * ceil(kv_heads / 16) / Geo::kWarps).
-template <class Geo>
+template <class Geo, int G>
 __global__ void __launch_bounds__(Geo::kThreads, Geo::kCtasPerSm)
 k_decode_step(DecodeParams P, AppendParams A) {
     const uint32_t attn_ctas = (P.gw + Geo::kWarps - 1) / Geo::kWarps;
     if (blockIdx.x < attn_ctas) {
-        decode_attn_body<false, 1, Geo, true>(P, &A);
+        decode_attn_body<false, G, Geo, true>(P, &A);
         return;
     }
     pdl_launch_dependents();
     pdl_wait();                                        // the attention of the previous step still reads the store
     const int head_groups = (A.store.kv_heads + 15) / 16;
     const int item = (int)(blockIdx.x - attn_ctas) * Geo::kWarps + (int)(threadIdx.x >> 5);
-    if (item < head_groups * A.store.batch) append_token_warp<true, 1>(A, item % head_groups, item / head_groups, false, nullptr);
+    if (item < head_groups * A.store.batch) append_token_warp<true, G>(A, item % head_groups, item / head_groups, false, nullptr);
 }
 
 // Pool fills each of the last t_total cached tokens may see when it asks as a query (causal

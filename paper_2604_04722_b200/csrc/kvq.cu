@@ -789,7 +789,8 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
              dyn_smem(k_decode_attn<false, 2, GeomSmall>, (int)GeomSmall::kSmemBytes);
         ok = ok && dyn_smem(k_decode_attn<true, 1, GeomSmall>, (int)GeomSmall::kSmemBytes) &&
              dyn_smem(k_decode_attn<true, 2, GeomSmall>, (int)GeomSmall::kSmemBytes);
-        ok = ok && dyn_smem(k_decode_step<GeomSmall>, (int)GeomSmall::kSmemBytes) && dyn_smem(k_decode_step<GeomLarge>, (int)GeomLarge::kSmemBytes);
+        ok = ok && dyn_smem(k_decode_step<GeomSmall, 1>, (int)GeomSmall::kSmemBytes) && dyn_smem(k_decode_step<GeomLarge, 1>, (int)GeomLarge::kSmemBytes) &&
+             dyn_smem(k_decode_step<GeomSmall, 2>, (int)GeomSmall::kSmemBytes) && dyn_smem(k_decode_step<GeomLarge, 2>, (int)GeomLarge::kSmemBytes);
         ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     }
     if (!ok) {
@@ -901,11 +902,11 @@ int kvq_decode_step(kvq_ctx* c, int layer, const float* feats, const void* K, co
     if (c->hidden == 0) return KVQ_ERR_NO_CONTROLLER;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // One launch when the warp that adds the token can evaluate the controller alone (hidden width 32: a wider
-    // one takes a single warp longer than the second launch costs) and the layout is the plain one; otherwise the
-    // two calls, whose kernels overlap their launches.
+    // one takes a single warp longer than the second launch costs) and keys have their scales per token (per-channel
+    // keys pack windows in a launch of their own); otherwise the two calls, whose kernels overlap their launches.
     const uint64_t units = (uint64_t)c->batch * c->q_heads;
     DecodePlan plan;
-    bool one_launch = c->groups == 1 && c->hidden == 32;
+    bool one_launch = c->groups != kLayoutPerChannelK && c->hidden == 32;
     if (one_launch) {
         plan = choose_plan(c, c->len[layer], units);
         one_launch = plan.gw > 0;
@@ -955,8 +956,10 @@ int kvq_decode_step(kvq_ctx* c, int layer, const float* feats, const void* K, co
     const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
     cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 2] : nullptr;
     if (rec) cudaEventRecord(ev[0], st);
-    if (plan.small) launch_overlapped(k_decode_step<GeomSmall>, grid, GeomSmall::kThreads, GeomSmall::kSmemBytes, st, p, a);
-    else launch_overlapped(k_decode_step<GeomLarge>, grid, GeomLarge::kThreads, GeomLarge::kSmemBytes, st, p, a);
+    if (plan.small && c->groups == 1) launch_overlapped(k_decode_step<GeomSmall, 1>, grid, GeomSmall::kThreads, GeomSmall::kSmemBytes, st, p, a);
+    else if (plan.small) launch_overlapped(k_decode_step<GeomSmall, 2>, grid, GeomSmall::kThreads, GeomSmall::kSmemBytes, st, p, a);
+    else if (c->groups == 1) launch_overlapped(k_decode_step<GeomLarge, 1>, grid, GeomLarge::kThreads, GeomLarge::kSmemBytes, st, p, a);
+    else launch_overlapped(k_decode_step<GeomLarge, 2>, grid, GeomLarge::kThreads, GeomLarge::kSmemBytes, st, p, a);
     if (rec) {
         cudaEventRecord(ev[1], st);
         c->prof_calls += 1;

@@ -1,6 +1,6 @@
 """GPU parity of kvq_decode_step: one decode step (controller decision, quantize-append of one
 token per sequence, attention over everything cached, Eq. 19-24, Eq. 4, Eq. 5) against the
-oracle, step by step.  With one scale group per row and a controller of width 32 the step is one
+oracle, step by step.  With keys quantized per token and a controller of width 32 the step is one
 launch (the attending warps add the step's token themselves from its fp16 rows); every other case
 runs the two kernels of kvq_append_fused + kvq_decode_attn behind the same call.  Both are compared with the
 oracle the same way: decisions and the whole store bit for bit, the attention output of EVERY
@@ -146,8 +146,9 @@ def test_steps_on_a_long_cache_in_the_bandwidth_geometry(gu, oracle, splits):
 
 
 @pytest.mark.parametrize("case", ["hidden 128", "two scale groups", "per-channel keys"])
-def test_steps_that_run_as_two_kernels(gu, oracle, case):
-    """The same call where the one-launch kernel does not apply: it must give the same results."""
+def test_steps_of_the_other_layouts_and_controller_widths(gu, oracle, case):
+    """Two scale groups per row take the one-launch kernel too; a wider controller and per-channel keys run the two
+    kernels behind the same call.  Same results either way."""
     rng = np.random.default_rng(len(case))
     hidden = 128 if case == "hidden 128" else 32
     cw = synth.controller_weights(2 if hidden == 128 else 322, hidden)
@@ -168,8 +169,10 @@ def test_steps_that_run_as_two_kernels(gu, oracle, case):
         bits = BITS[rng.choice(4, size=(B, n))]
         oc.append(K, V, bits)
         g.append(0, K, V, bits)
-        launches = _run_steps(gu, oracle, g, oc, cw, rng, B, Hq, H, steps, "two-kernel step, %s" % case, first_pos=n)
-        assert launches >= 2 * steps
+        launches = _run_steps(gu, oracle, g, oc, cw, rng, B, Hq, H, steps, "step, %s" % case, first_pos=n)
+        assert launches == steps if case == "two scale groups" else launches >= 2 * steps
+        if case != "per-channel keys":
+            gu.assert_store_equals_oracle(g, 0, oc)
 
 
 def test_steps_on_a_layer_of_ragged_lengths(gu, oracle):
