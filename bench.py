@@ -365,7 +365,7 @@ def measure(bench, wl, *, steps, warmup, blocks, uniform_bits=0, scale_groups=1,
     cold = flushes_l2(wl)
     e2e_warm = 3
     n_e2e = (e2e_warm + e2e_blocks * K_steps) if e2e else 0
-    total_steps = W + blocks * K_steps + K_steps + n_e2e + 1
+    total_steps = W + blocks * K_steps + 2 * K_steps + n_e2e + 1
     L, B, Hq, Hkv, D, ctx_len = wl.layers, wl.batch, wl.q_heads, wl.kv_heads, wl.head_dim, wl.context
     seed = wl.seed + 1000 * bench.rank                # replicas draw their own data
     cw = synth.controller_weights(wl.mlp_seed, wl.hidden)
@@ -487,18 +487,23 @@ def measure(bench, wl, *, steps, warmup, blocks, uniform_bits=0, scale_groups=1,
     launches_block = None
     if cold:
         # one pair of events per step; the flush runs between the pairs, outside the timed regions
-        kq.kvq_set_profiling(ctx, True)
-        kq.kvq_profile_read(ctx)
         for _ in range(blocks):
             ms_total = 0.0
             for _ in range(K_steps):
                 bench.flush_l2(step_no[0])
                 ms_total += bench.timed_block(one_step, 1)
-                a_ms, n = kq.kvq_profile_read(ctx)
-                attn_ms, ncalls = attn_ms + a_ms, ncalls + n
             block_ms.append(ms_total)
             if launches_block is None:
                 launches_block = kq.kvq_launch_count(ctx) - launches1
+        # one more block with the library's event pair around every launch (the pairs keep the launches of
+        # neighbouring layers from overlapping, so the steps above are timed without them)
+        kq.kvq_set_profiling(ctx, True)
+        kq.kvq_profile_read(ctx)
+        for _ in range(K_steps):
+            bench.flush_l2(step_no[0])
+            bench.timed_block(one_step, 1)
+            a_ms, n = kq.kvq_profile_read(ctx)
+            attn_ms, ncalls = attn_ms + a_ms, ncalls + n
         kq.kvq_set_profiling(ctx, False)
         warm_ms = bench.timed_block(one_step, K_steps)         # the same steps with whatever stays in L2
     else:
@@ -691,7 +696,7 @@ def run_ours(args, wl):
                          "timed_in": ("the timed blocks: steps x layers back-to-back launches of the step kernel between one pair of "
                                       "events; the event-pair figure is from the library's events around every single launch"
                                       if m["step_kernels"] == "k_decode_step" else
-                                      "the timed steps, one event pair per launch" if m["cold"] else
+                                      "one more block of steps (L2 flushed before each), one event pair per launch" if m["cold"] else
                                       "one more block of the same number of steps with an event pair around every launch"),
                          "frac_with_index_bytes": (m["launch_bytes"] + m["index_bytes"]) / (m["ms_launch"] * 1e-3) / 1e9 / m["peak"]},
             "cpu_baseline": cpu,
