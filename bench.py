@@ -53,10 +53,10 @@ L2_BYTES = 126e6
 NEAR_TIE_GAP = 1e-5
 ORACLE_SAMPLE_SEQS = 2                               # whole sequences of the workload the oracle legs run
 
-# DRAM traffic of one k_decode_attn launch (ncu: dram__bytes_read.sum + dram__bytes_write.sum) is kept in a
+# DRAM traffic of one launch of the step kernel (ncu: dram__bytes_read.sum + dram__bytes_write.sum) is kept in a
 # small text file beside the profile it comes from, together with a hash of the kernel sources it was
 # captured on; when the sources have changed since, the bench prints "traffic": null.
-TRAFFIC_FILE = os.path.join(ROOT, "profiles", "k_decode_attn_cfg5_traffic.txt")
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "k_decode_step_cfg5_traffic.txt")
 CSRC_DIR = os.path.join(ROOT, "paper_2604_04722_b200", "csrc")
 
 
