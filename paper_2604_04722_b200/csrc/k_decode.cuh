@@ -934,8 +934,8 @@ __device__ __forceinline__ void merge_partials(const DecodeParams& P, uint32_t u
 // STEP (not for per-channel keys): the launch is a whole decode step.  `P.counts` are the pool fills BEFORE the
 // step's token, whose fp16 rows, features and controller come in A; other CTAs of the same launch store it (see
 // k_decode_step) and nobody waits for them: the warp that works on the last part of a unit evaluates the controller
-// itself, quantizes the token's K and V rows in registers the way the store does (row_values_as_stored) and adds the
-// token to its partial.  The slot the token is being written to lies beyond the fills this launch reads.
+// itself and quantizes the token's K and V rows in registers the way the store does (row_values_as_stored) while its
+// first copies travel, and adds the token to its partial at the end.  The slot the token is being written to lies beyond the fills this launch reads.
 template <bool STATS, int G, class Geo, bool STEP>
 __device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const AppendParams* A) {
     static_assert(!STEP || (G != kLayoutPerChannelK && !STATS), "the one-launch step exists for the plain decode with one pair per row or group");
@@ -1085,6 +1085,21 @@ __device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const Ap
         };
         int in_flight = 0;
         for (; in_flight < kStages && p_left > 0; ++in_flight) issue_next();
+
+        // The step's token, worked out while the first copies travel: its logit and its two value elements as stored.
+        float y_new = 0.f;
+        float2 v_tok = make_float2(0.f, 0.f);
+        if constexpr (STEP) {
+            if (adds_token) {                          // warp-uniform
+                const float4 f = reinterpret_cast<const float4*>(A->feats)[b];
+                const int c = controller_decide_warp32(A->ctrl, f.x, f.y, f.z, f.w, lane);
+                const float2 kh = row_values_as_stored<G>(__half22float2(k_new), c);
+                v_tok = row_values_as_stored<G>(__half22float2(v_new), c);
+                const int i = 2 * lane;
+                const float* qp = ws.q + (i >> 5) * kQHalfStride + (i & 31);
+                y_new = warp_sum(fmaf(kh.y, qp[1], kh.x * qp[0])) * kLogitScale;
+            }
+        }
 
         SoftmaxT<STATS> st = {kNegBig, 0.f, 0.f, kNegBig, 0.f, {0.f, 0.f, 0.f, 0.f}};
         float acc[kHalfDim];
@@ -1296,17 +1311,11 @@ __device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const Ap
         const float s2_w = STATS ? (G != 2 ? 1.0f : 0.5f) * warp_sum(st.s2) : 0.f;
         float l_tot = l_w;
         if constexpr (STEP) {
-            if (adds_token) {                          // warp-uniform
-                const float4 f = reinterpret_cast<const float4*>(A->feats)[b];
-                const int c = controller_decide_warp32(A->ctrl, f.x, f.y, f.z, f.w, lane);
-                const float2 kh = row_values_as_stored<G>(__half22float2(k_new), c), vh = row_values_as_stored<G>(__half22float2(v_new), c);
-                const int i = 2 * lane;
-                const float* qp = ws.q + (i >> 5) * kQHalfStride + (i & 31);
-                const float y = warp_sum(fmaf(kh.y, qp[1], kh.x * qp[0])) * kLogitScale;
-                const float m_new = fmaxf(st.m, y);
-                const float keep = fast_exp2(st.m - m_new), e = fast_exp2(y - m_new);
-                r2[0] = fmaf(r2[0], keep, e * vh.x);
-                r2[1] = fmaf(r2[1], keep, e * vh.y);
+            if (adds_token) {                          // warp-uniform: one more online-softmax update
+                const float m_new = fmaxf(st.m, y_new);
+                const float keep = fast_exp2(st.m - m_new), e = fast_exp2(y_new - m_new);
+                r2[0] = fmaf(r2[0], keep, e * v_tok.x);
+                r2[1] = fmaf(r2[1], keep, e * v_tok.y);
                 l_tot = fmaf(l_w, keep, e);
                 st.m = m_new;
             }
