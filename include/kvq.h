@@ -324,7 +324,8 @@ int kvq_decode_step(kvq_ctx* ctx, int layer, const float* feats, const void* K, 
                     const void* Q, void* O, uint8_t* bits_out_opt, void* stream);
 
 /*
- * One decode step from HOST buffers, copies included: controller decision for
+ * One decode step from HOST buffers, copies included (kvq_decode_step on host
+ * memory, then a stream synchronization): controller decision for
  * the step's `batch` tokens, quantize-append of their K/V rows to `layer`,
  * attention of Q over the layer, result copied back.  feats host fp32
  * [batch][4]; K, V host fp16 [batch][1][kv_heads][64]; Q host fp16
