@@ -3,6 +3,8 @@ cached length (zero included), bit mix (degenerate mixes included), split count,
 and controller width are drawn per case; a prefill (bit-widths given or decided by the controller),
 then decode steps through kvq_decode_step, then kvq_decode_attn and its fixed-scratch variant.
 Decisions and the store are compared bit for bit, every attention output within the tolerance."""
+import os
+
 import numpy as np
 import pytest
 
@@ -11,7 +13,7 @@ from paper_2604_04722_b200 import synth
 pytestmark = pytest.mark.gpu
 
 BITS = np.array([2, 4, 8, 16], dtype=np.uint8)
-CASES = 36
+CASES = int(os.environ.get("KVQ_RANDOM_CASES", "36"))    # more seeds for a longer soak
 
 
 @pytest.fixture(scope="module")
