@@ -313,11 +313,14 @@ int kvq_decode_attn_static(kvq_ctx* ctx, int layer, const void* Q, void* O, void
  * kvq_append_fused with n_new = 1 followed by kvq_decode_attn.  feats dev fp32 [batch][4];
  * K, V dev fp16 [batch][1][kv_heads][64]; Q, O dev fp16 [batch][q_heads][64]; bits_out_opt
  * dev uint8 [batch] or NULL.  Launches: ONE kernel when the keys are quantized per token (one
- * or two scale groups) and the controller has hidden width 32, whatever the lengths: some
- * CTAs of the launch store the token while the others attend over the cache as it was and add
- * the token from its fp16 rows, quantized in registers exactly as it is stored, so neither
- * side waits for the other.  In every other case the two kernels of the two calls, whose
- * launches overlap.  Errors as for the two calls (an empty layer is fine: the step's token is
+ * or two scale groups), whatever the lengths and the controller's width: some CTAs of the
+ * launch store the token while the others attend over the cache as it was and add the token
+ * from its fp16 rows, quantized in registers exactly as it is stored, so the attention does
+ * not wait for the store.  (A controller of hidden width 32 is evaluated by every warp that
+ * needs the decision; a wider one by the storing CTAs, which publish the class for the
+ * attending warps of the same launch: those pick it up at the end of their work through a
+ * bounded wait, see KVQ_FLAG_WAIT_TIMEOUT.)  With per-channel keys the two kernels of the two
+ * calls, whose launches overlap.  Errors as for the two calls (an empty layer is fine: the step's token is
  * then all there is).
  */
 int kvq_decode_step(kvq_ctx* ctx, int layer, const float* feats, const void* K, const void* V,
@@ -423,7 +426,8 @@ int kvq_profile_read(kvq_ctx* ctx, double* attn_ms_total, int* calls);
 /* Device flags recorded by kernels since the last call (host uint32, cleared on read). */
 #define KVQ_FLAG_BAD_BITS 1u      /* a bit-width outside {2,4,8,16} was appended (stored as fp16) */
 #define KVQ_FLAG_ARENA_FULL 4u    /* an append ran out of arena blocks; the tokens that did not fit are lost */
-#define KVQ_FLAG_WAIT_TIMEOUT 2u  /* a bounded wait on an async copy expired in kvq_decode_attn; that
+#define KVQ_FLAG_WAIT_TIMEOUT 2u  /* a bounded wait expired in a decode call (on an async copy, or in
+                                     kvq_decode_step on the class that the storing CTAs publish); that
                                      call's output is invalid.  The warp that gave up still hands in an
                                      (empty) partial for the rest of its share, so every arrival counter
                                      the call used is back at zero when it ends and later calls on the

@@ -53,6 +53,10 @@ struct AppendParams {
     const int* lens;
     const int* pos;
     uint32_t* chunk_arrivals;          // [batch] classify CTAs of a sequence that have finished; zero between launches
+    // One-launch decode step with a controller wider than 32: the storing CTAs publish each sequence's class here as
+    // (step_serial << 2) | class for the attending warps of the same launch (nullptr: nobody asks).
+    uint32_t* step_cls;                // [batch]
+    uint32_t step_serial;
 };
 
 __device__ __forceinline__ int new_tokens_of(const AppendParams& p, int b) { return p.lens ? p.lens[b] : p.n_new; }
@@ -637,11 +641,14 @@ __device__ __forceinline__ void token_store_pc(int c, const uint4 (&kraw)[4], co
 // One new token per sequence (a decode step), the work of one warp: the token of sequence b, KV heads
 // 16 bx .. 16 bx + 15; lane l handles half-row l % 2 of KV head 16 bx + l / 2.  Everything the warp needs (the K and
 // V rows, the pool fills, the features) is requested up front so the loads overlap the controller; the decision is
-// taken by the warp (FUSED) or read from `bits`.  wide: the warp is the first of a CTA of four whose other warps
-// help with a controller wider than 32 hidden units (they call this too and return after the decision;
-// controller_fetch_cta128 has been called by all of them).
+// taken by the warp (FUSED) or read from `bits`.  ctl says who evaluates the controller: kCtlWarp32 the warp alone
+// (hidden width 32); kCtlCtaStaged / kCtlCtaDirect: the warp is the first of four (threads 0..127 of the CTA) that
+// evaluate a controller of any width together -- the other three call this too and return after the decision --
+// with W2 staged in shared memory (controller_fetch_cta128 has been called by all four; ctrl_sh holds
+// kControllerCtaSmemFloats floats) or read straight from global memory (kControllerDirectSmemFloats floats).
+constexpr int kCtlWarp32 = 0, kCtlCtaStaged = 1, kCtlCtaDirect = 2;
 template <bool FUSED, int G>
-__device__ __forceinline__ void append_token_warp(const AppendParams& p, int bx, int b, bool wide, float* ctrl_sh) {
+__device__ __forceinline__ void append_token_warp(const AppendParams& p, int bx, int b, int ctl, float* ctrl_sh) {
     const int lane = threadIdx.x & 31;
     const int h = bx * 16 + (lane >> 1), half = lane & 1;
     const bool active = h < p.store.kv_heads;
@@ -670,9 +677,14 @@ __device__ __forceinline__ void append_token_warp(const AppendParams& p, int bx,
     int c;
     if (FUSED) {
         const float4 f = reinterpret_cast<const float4*>(p.feats)[b];
-        c = !wide ? controller_decide_warp32(p.ctrl, f.x, f.y, f.z, f.w, lane)
-                  : controller_decide_cta128(p.ctrl, p.hidden, f.x, f.y, f.z, f.w, ctrl_sh);
-        if (wide && threadIdx.x >= 32) return;         // the helpers are done
+        c = ctl == kCtlWarp32    ? controller_decide_warp32(p.ctrl, f.x, f.y, f.z, f.w, lane)
+            : ctl == kCtlCtaStaged ? controller_decide_cta128(p.ctrl, p.hidden, f.x, f.y, f.z, f.w, ctrl_sh)
+                                   : controller_decide_cta_direct(p.ctrl, p.hidden, f.x, f.y, f.z, f.w, ctrl_sh);
+        if (p.step_cls && bx == 0 && threadIdx.x == 0) {       // for the attending warps of this launch
+            const uint32_t word = (p.step_serial << 2) | (uint32_t)c;
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.step_cls + b), "r"(word) : "memory");
+        }
+        if (ctl != kCtlWarp32 && threadIdx.x >= 32) return;    // the helpers are done
     } else {
         c = class_of_bits(p.bits[b], p.store.flags);
     }
@@ -718,7 +730,7 @@ k_append_token(AppendParams p) {
     const bool wide = blockDim.x != 32;
     if (FUSED && wide) controller_fetch_cta128(p.ctrl, p.hidden, ctrl_sh);   // no kernel writes the weights
     pdl_wait();                                        // the attention of the previous step still reads the store
-    append_token_warp<FUSED, G>(p, (int)blockIdx.x, (int)blockIdx.y, wide, ctrl_sh);
+    append_token_warp<FUSED, G>(p, (int)blockIdx.x, (int)blockIdx.y, wide ? kCtlCtaStaged : kCtlWarp32, ctrl_sh);
 }
 
 }  // namespace kvq

@@ -285,6 +285,80 @@ __device__ __forceinline__ int controller_decide_cta128(const float* __restrict_
     return cls;
 }
 
+// The same decision taken by the first 128 threads of a CTA (any CTA size) with a few KB of shared memory: thread j
+// owns hidden unit j and reads its row of W2 straight from global memory, 32 weights at a time (they are read by
+// every CTA of a launch and stay in L2).  The 128 threads meet at the named barrier 1, so the other threads of the
+// CTA need not take part.  Sums in ascending input order with separately rounded products and sums: bit-identical
+// to controller_decide.  Every one of the 128 threads must call it; returns the class in all of them.
+// sh: kControllerDirectSmemFloats floats, 16-byte aligned.
+constexpr int kControllerDirectSmemFloats = 2 * kMaxHidden + 4 * kW2RowStride;
+__device__ __forceinline__ void barrier_first_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ int controller_decide_cta_direct(const float* __restrict__ gW, int H, float x0, float x1, float x2,
+                                                            float x3, float* sh) {
+    const int j = threadIdx.x;
+    const float* W1 = gW;
+    const float* b1 = W1 + 4 * H;
+    const float* W2 = b1 + H;
+    const float* b2 = W2 + H * H;
+    const float* W3 = b2 + H;
+    const float* b3 = W3 + 4 * H;
+    float* h1s = sh;
+    float* h2s = sh + kMaxHidden;
+    float* w3s = sh + 2 * kMaxHidden;                  // the four rows of W3, kW2RowStride apart
+    const bool mine = j < H;
+    const bool vec = controller_rows_vectorized(gW, H);
+    for (int i = j; i < 4 * H; i += 128) w3s[(i / H) * kW2RowStride + i % H] = __ldg(W3 + i);
+    float acc = 0.f;
+    if (mine) {
+        float a = __ldg(b1 + j);
+        a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 0), x0));
+        a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 1), x1));
+        a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 2), x2));
+        a = __fadd_rn(a, __fmul_rn(__ldg(W1 + 4 * j + 3), x3));
+        h1s[j] = a > 0.0f ? a : 0.0f;
+        acc = __ldg(b2 + j);
+    }
+    barrier_first_128();
+    if (mine) {
+        const float* row = W2 + (size_t)j * H;
+        if (vec) {
+            for (int i0 = 0; i0 < H; i0 += 32) {       // 32 weights in flight, then their 32 ordered terms
+                float4 w[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) w[k] = i0 + 4 * k < H ? __ldg(reinterpret_cast<const float4*>(row + i0) + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (i0 + 4 * k < H) {
+                        const float4 h4 = *reinterpret_cast<const float4*>(h1s + i0 + 4 * k);
+                        acc = __fadd_rn(acc, __fmul_rn(w[k].x, h4.x));
+                        acc = __fadd_rn(acc, __fmul_rn(w[k].y, h4.y));
+                        acc = __fadd_rn(acc, __fmul_rn(w[k].z, h4.z));
+                        acc = __fadd_rn(acc, __fmul_rn(w[k].w, h4.w));
+                    }
+                }
+            }
+        } else {
+#pragma unroll 4
+            for (int i = 0; i < H; ++i) acc = __fadd_rn(acc, __fmul_rn(__ldg(row + i), h1s[i]));
+        }
+        h2s[j] = acc > 0.0f ? acc : 0.0f;
+    }
+    barrier_first_128();
+    const int lane = threadIdx.x & 31;
+    float o = __ldg(b3 + (lane & 3));                  // lanes 0..3 of every warp hold the four logits
+    const float* w3 = w3s + (lane & 3) * kW2RowStride;
+    o = (H & 3) == 0 ? ordered_dot<true>(o, w3, h2s, H) : ordered_dot<false>(o, w3, h2s, H);
+    const float o0 = __shfl_sync(0xffffffffu, o, 0), o1 = __shfl_sync(0xffffffffu, o, 1);
+    const float o2 = __shfl_sync(0xffffffffu, o, 2), o3 = __shfl_sync(0xffffffffu, o, 3);
+    if (o0 != o0 || o1 != o1 || o2 != o2 || o3 != o3) return 3;
+    int cls = 0;
+    float best = o0;
+    if (o1 > best) { best = o1; cls = 1; }
+    if (o2 > best) { best = o2; cls = 2; }
+    if (o3 > best) { best = o3; cls = 3; }
+    return cls;
+}
+
 // kvq_select_bits: one thread per token.
 __global__ void __launch_bounds__(128)
 k_select_bits(const float* __restrict__ feats, int n, const float* __restrict__ gW, int H,

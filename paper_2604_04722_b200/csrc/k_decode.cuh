@@ -108,6 +108,12 @@ struct DecodeParams {
     uint32_t gw;                   // working warps = parts the x axis is cut into
     uint32_t pslots;               // partial slots per unit = decode_pslots(units, gw)
     uint32_t cta_parts;            // > 0: gw = units * cta_parts and the parts of a unit share a CTA, which merges them itself
+    // One-launch decode step with a controller wider than 32 (k_decode_step<.., true>): the attending CTAs start at
+    // block cta0 (the storing CTAs come first) and read each sequence's class from step_cls, where a storing CTA of
+    // the same launch publishes it as (step_serial << 2) | class.
+    uint32_t cta0;
+    const uint32_t* step_cls;
+    uint32_t step_serial;
 };
 
 // Warps that can overlap one unit: ceil(gw/units) + 1.
@@ -936,7 +942,12 @@ __device__ __forceinline__ void merge_partials(const DecodeParams& P, uint32_t u
 // k_decode_step) and nobody waits for them: the warp that works on the last part of a unit evaluates the controller
 // itself and quantizes the token's K and V rows in registers the way the store does (row_values_as_stored) while its
 // first copies travel, and adds the token to its partial at the end.  The slot the token is being written to lies beyond the fills this launch reads.
-template <bool STATS, int G, class Geo, bool STEP>
+// STEP = 1: the controller has hidden width 32 and the warp evaluates it itself, early.  STEP = 2: any other width;
+// the storing CTAs of the launch (which come first in the grid, so that they are resident before any attending
+// CTA) evaluate it with 128 threads and publish the class; the attending warp picks it up at the END of its walk,
+// by when it has long been written: a bounded wait that has never been seen to spin, with the usual flag if it
+// should run out.
+template <bool STATS, int G, class Geo, int STEP>
 __device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const AppendParams* A) {
     static_assert(!STEP || (G != kLayoutPerChannelK && !STATS), "the one-launch step exists for the plain decode with one pair per row or group");
     constexpr int kStages = Geo::kStages, kStageBytes = Geo::kStageBytes;
@@ -944,7 +955,7 @@ __device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const Ap
     __shared__ WarpScratch<kStages> scratch[Geo::kWarps];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int half = lane >> 4, t = lane & 15;
-    const uint32_t j = blockIdx.x * Geo::kWarps + warp;
+    const uint32_t j = (STEP == 2 ? blockIdx.x - P.cta0 : blockIdx.x) * Geo::kWarps + warp;
     if (Geo::kCtaMerge && P.cta_parts) {               // the arrival counters of this CTA's units start at zero:
         if (lane == 0) scratch[warp].arrived = 0u;     // the only barrier of the kernel, before any warp can wait
         __syncthreads();
@@ -1089,7 +1100,7 @@ __device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const Ap
         // The step's token, worked out while the first copies travel: its logit and its two value elements as stored.
         float y_new = 0.f;
         float2 v_tok = make_float2(0.f, 0.f);
-        if constexpr (STEP) {
+        if constexpr (STEP == 1) {
             if (adds_token) {                          // warp-uniform
                 const float4 f = reinterpret_cast<const float4*>(A->feats)[b];
                 const int c = controller_decide_warp32(A->ctrl, f.x, f.y, f.z, f.w, lane);
@@ -1310,7 +1321,30 @@ __device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const Ap
         }
         const float s2_w = STATS ? (G != 2 ? 1.0f : 0.5f) * warp_sum(st.s2) : 0.f;
         float l_tot = l_w;
-        if constexpr (STEP) {
+        if constexpr (STEP == 2) {
+            if (adds_token) {                          // warp-uniform: the class comes from a storing CTA of this launch
+                uint32_t word = 0;
+                if (lane == 0) {
+                    bool found = false;
+                    for (uint32_t spin = 0; spin < kWaitLimit && !found; ++spin) {
+                        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(word) : "l"(P.step_cls + b) : "memory");
+                        found = (word >> 2) == P.step_serial;
+                        if (!found) __nanosleep(64);
+                    }
+                    if (!found) {
+                        atomicOr(P.store.flags, kFlagWaitTimeout);
+                        word = 3u;                     // keep the row as it is; the call's output is flagged invalid
+                    }
+                }
+                const int c = (int)(__shfl_sync(0xffffffffu, word, 0) & 3u);
+                const float2 kh = row_values_as_stored<G>(__half22float2(k_new), c);
+                v_tok = row_values_as_stored<G>(__half22float2(v_new), c);
+                const int i = 2 * lane;
+                const float* qp = ws.q + (i >> 5) * kQHalfStride + (i & 31);
+                y_new = warp_sum(fmaf(kh.y, qp[1], kh.x * qp[0])) * kLogitScale;
+            }
+        }
+        if constexpr (STEP != 0) {
             if (adds_token) {                          // warp-uniform: one more online-softmax update
                 const float m_new = fmaxf(st.m, y_new);
                 const float keep = fast_exp2(st.m - m_new), e = fast_exp2(y_new - m_new);
@@ -1382,26 +1416,43 @@ __device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const Ap
 template <bool STATS, int G, class Geo>
 __global__ void __launch_bounds__(Geo::kThreads, Geo::kCtasPerSm)
 k_decode_attn(DecodeParams P) {
-    decode_attn_body<STATS, G, Geo, false>(P, nullptr);
+    decode_attn_body<STATS, G, Geo, 0>(P, nullptr);
 }
 
 // One decode step (Eq. 4, then Eq. 5) in one launch: the first ceil(gw / Geo::kWarps) CTAs attend over the cache
 // as it was plus the step's token (decode_attn_body with STEP), the others store the token: every warp of theirs
-// is one warp of k_append_token.  Neither side reads what the other writes.  Controller width 32 only.
+// is one warp of k_append_token.  Neither side reads what the other writes.
 // grid = ceil(gw / Geo::kWarps) + ceil(batch * ceil(kv_heads / 16) / Geo::kWarps).
-template <class Geo, int G>
+// WIDE (a controller of another hidden width than 32): the storing CTAs come FIRST in the grid, one per (sequence,
+// group of 16 KV heads); their first 128 threads evaluate the controller together and publish the class for the
+// attending warps (see decode_attn_body).  grid = batch * ceil(kv_heads / 16) + ceil(gw / Geo::kWarps).
+template <class Geo, int G, bool WIDE>
 __global__ void __launch_bounds__(Geo::kThreads, Geo::kCtasPerSm)
 k_decode_step(DecodeParams P, AppendParams A) {
-    const uint32_t attn_ctas = (P.gw + Geo::kWarps - 1) / Geo::kWarps;
-    if (blockIdx.x < attn_ctas) {
-        decode_attn_body<false, G, Geo, true>(P, &A);
-        return;
-    }
-    pdl_launch_dependents();
-    pdl_wait();                                        // the attention of the previous step still reads the store
+    static_assert(sizeof(float) * kControllerDirectSmemFloats <= Geo::kSmemBytes, "the storing CTAs' controller scratch lies in the ring");
     const int head_groups = (A.store.kv_heads + 15) / 16;
-    const int item = (int)(blockIdx.x - attn_ctas) * Geo::kWarps + (int)(threadIdx.x >> 5);
-    if (item < head_groups * A.store.batch) append_token_warp<true, G>(A, item % head_groups, item / head_groups, false, nullptr);
+    if constexpr (WIDE) {
+        if (blockIdx.x >= P.cta0) {
+            decode_attn_body<false, G, Geo, 2>(P, &A);
+            return;
+        }
+        extern __shared__ __align__(128) uint8_t ring[];       // the storing CTAs use its start for the controller
+        pdl_launch_dependents();
+        pdl_wait();                                    // the attention of the previous step still reads the store
+        if (threadIdx.x < 128)
+            append_token_warp<true, G>(A, (int)blockIdx.x % head_groups, (int)blockIdx.x / head_groups, kCtlCtaDirect,
+                                       reinterpret_cast<float*>(ring));
+    } else {
+        const uint32_t attn_ctas = (P.gw + Geo::kWarps - 1) / Geo::kWarps;
+        if (blockIdx.x < attn_ctas) {
+            decode_attn_body<false, G, Geo, 1>(P, &A);
+            return;
+        }
+        pdl_launch_dependents();
+        pdl_wait();                                    // the attention of the previous step still reads the store
+        const int item = (int)(blockIdx.x - attn_ctas) * Geo::kWarps + (int)(threadIdx.x >> 5);
+        if (item < head_groups * A.store.batch) append_token_warp<true, G>(A, item % head_groups, item / head_groups, kCtlWarp32, nullptr);
+    }
 }
 
 // Pool fills each of the last t_total cached tokens may see when it asks as a query (causal

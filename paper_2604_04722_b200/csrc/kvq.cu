@@ -57,6 +57,8 @@ struct kvq_ctx {
     uint4* hist = nullptr;               // append scratch [batch][max chunks]
     uint32_t* chunk_arrivals = nullptr;  // append scratch [batch], zero between launches
     float* ctrl = nullptr;               // controller parameter block
+    uint32_t* step_cls = nullptr;        // [batch] class of the step's token, published inside a one-launch step (wide controllers)
+    uint32_t step_serial = 0;            // tag of the last such launch
     int hidden = 0;
     float* part_o = nullptr;             // decode scratch [units][partial slots][64]
     float2* part_ml = nullptr;           //                [units][partial slots]
@@ -193,6 +195,7 @@ void free_all(kvq_ctx* c) {
     cudaFree(c->hist);
     cudaFree(c->chunk_arrivals);
     cudaFree(c->ctrl);
+    cudaFree(c->step_cls);
     cudaFree(c->part_o);
     cudaFree(c->part_ml);
     cudaFree(c->part_cnt);
@@ -710,6 +713,7 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
     ok = ok && dev_alloc(c, &c->hist, sizeof(uint4) * batch * max_chunks) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->chunk_arrivals, sizeof(uint32_t) * batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->ctrl, controller_smem(kMaxHidden)) == cudaSuccess;
+    ok = ok && dev_alloc(c, &c->step_cls, sizeof(uint32_t) * batch) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_o, sizeof(float) * max_partial_records(c) * kHeadDim) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_ml, sizeof(float2) * max_partial_records(c)) == cudaSuccess;
     ok = ok && dev_alloc(c, &c->part_cnt, sizeof(uint32_t) * units * kMaxQueryRows) == cudaSuccess;
@@ -750,6 +754,7 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
         ok = ok && cudaMemset(c->counts, 0, sizeof(uint32_t) * 2 * (size_t)layers * batch * 4) == cudaSuccess;
         ok = ok && cudaMemset(c->flags, 0, sizeof(uint32_t)) == cudaSuccess;
         ok = ok && cudaMemset(c->chunk_arrivals, 0, sizeof(uint32_t) * batch) == cudaSuccess;
+        ok = ok && cudaMemset(c->step_cls, 0, sizeof(uint32_t) * batch) == cudaSuccess;
         ok = ok && cudaMemset(c->part_cnt, 0, sizeof(uint32_t) * units * kMaxQueryRows) == cudaSuccess;
         // the controller block may exceed the default 48 KB of dynamic shared memory
         const int smem_max = (int)controller_smem(kMaxHidden);
@@ -789,8 +794,10 @@ int create_impl(kvq_ctx** out, int layers, int q_heads, int kv_heads, int head_d
              dyn_smem(k_decode_attn<false, 2, GeomSmall>, (int)GeomSmall::kSmemBytes);
         ok = ok && dyn_smem(k_decode_attn<true, 1, GeomSmall>, (int)GeomSmall::kSmemBytes) &&
              dyn_smem(k_decode_attn<true, 2, GeomSmall>, (int)GeomSmall::kSmemBytes);
-        ok = ok && dyn_smem(k_decode_step<GeomSmall, 1>, (int)GeomSmall::kSmemBytes) && dyn_smem(k_decode_step<GeomLarge, 1>, (int)GeomLarge::kSmemBytes) &&
-             dyn_smem(k_decode_step<GeomSmall, 2>, (int)GeomSmall::kSmemBytes) && dyn_smem(k_decode_step<GeomLarge, 2>, (int)GeomLarge::kSmemBytes);
+        ok = ok && dyn_smem(k_decode_step<GeomSmall, 1, false>, (int)GeomSmall::kSmemBytes) && dyn_smem(k_decode_step<GeomLarge, 1, false>, (int)GeomLarge::kSmemBytes) &&
+             dyn_smem(k_decode_step<GeomSmall, 2, false>, (int)GeomSmall::kSmemBytes) && dyn_smem(k_decode_step<GeomLarge, 2, false>, (int)GeomLarge::kSmemBytes);
+        ok = ok && dyn_smem(k_decode_step<GeomSmall, 1, true>, (int)GeomSmall::kSmemBytes) && dyn_smem(k_decode_step<GeomLarge, 1, true>, (int)GeomLarge::kSmemBytes) &&
+             dyn_smem(k_decode_step<GeomSmall, 2, true>, (int)GeomSmall::kSmemBytes) && dyn_smem(k_decode_step<GeomLarge, 2, true>, (int)GeomLarge::kSmemBytes);
         ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     }
     if (!ok) {
@@ -901,12 +908,13 @@ int kvq_decode_step(kvq_ctx* c, int layer, const float* feats, const void* K, co
     if (!aligned16(K) || !aligned16(V) || !aligned16(feats)) return KVQ_ERR_ARG;
     if (c->hidden == 0) return KVQ_ERR_NO_CONTROLLER;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // One launch when the warp that adds the token can evaluate the controller alone (hidden width 32: a wider
-    // one takes a single warp longer than the second launch costs) and keys have their scales per token (per-channel
-    // keys pack windows in a launch of their own); otherwise the two calls, whose kernels overlap their launches.
+    // One launch when keys have their scales per token (per-channel keys pack windows in a launch of their own);
+    // otherwise the two calls, whose kernels overlap their launches.  With hidden width 32 the warp that adds the
+    // token evaluates the controller itself; a wider one is evaluated by the storing CTAs, which then come first in
+    // the grid and publish the class (tagged with a serial number that no earlier launch used).
     const uint64_t units = (uint64_t)c->batch * c->q_heads;
     DecodePlan plan;
-    bool one_launch = c->groups != kLayoutPerChannelK && c->hidden == 32;
+    bool one_launch = c->groups != kLayoutPerChannelK;
     if (one_launch) {
         plan = choose_plan(c, c->len[layer], units);
         one_launch = plan.gw > 0;
@@ -952,14 +960,30 @@ int kvq_decode_step(kvq_ctx* c, int layer, const float* feats, const void* K, co
     const unsigned cta_warps = plan.small ? GeomSmall::kWarps : GeomLarge::kWarps;
     const unsigned attn_ctas = (p.gw + cta_warps - 1) / cta_warps;
     const unsigned items = (unsigned)c->batch * (unsigned)((c->kv_heads + 15) / 16);
-    const dim3 grid(attn_ctas + (items + cta_warps - 1) / cta_warps);
+    const bool w32 = c->hidden == 32;
+    if (!w32) {
+        if (c->step_serial >= 0x3fffffffu) {           // the tag is about to repeat: forget the old ones first
+            KVQ_CUDA(c, cudaMemsetAsync(c->step_cls, 0, sizeof(uint32_t) * c->batch, st));
+            c->step_serial = 0;
+        }
+        a.step_cls = c->step_cls;
+        a.step_serial = ++c->step_serial;
+        p.cta0 = items;                                // one storing CTA per (sequence, group of 16 KV heads), first in the grid
+        p.step_cls = c->step_cls;
+        p.step_serial = a.step_serial;
+    }
+    const dim3 grid(w32 ? attn_ctas + (items + cta_warps - 1) / cta_warps : items + attn_ctas);
     const bool rec = c->profiling && c->prof_calls < kProfMaxCalls;
     cudaEvent_t* ev = rec ? &c->prof_ev[(size_t)c->prof_calls * 2] : nullptr;
     if (rec) cudaEventRecord(ev[0], st);
-    if (plan.small && c->groups == 1) launch_overlapped(k_decode_step<GeomSmall, 1>, grid, GeomSmall::kThreads, GeomSmall::kSmemBytes, st, p, a);
-    else if (plan.small) launch_overlapped(k_decode_step<GeomSmall, 2>, grid, GeomSmall::kThreads, GeomSmall::kSmemBytes, st, p, a);
-    else if (c->groups == 1) launch_overlapped(k_decode_step<GeomLarge, 1>, grid, GeomLarge::kThreads, GeomLarge::kSmemBytes, st, p, a);
-    else launch_overlapped(k_decode_step<GeomLarge, 2>, grid, GeomLarge::kThreads, GeomLarge::kSmemBytes, st, p, a);
+    auto launch = [&](auto small_kernel, auto large_kernel) {
+        if (plan.small) launch_overlapped(small_kernel, grid, GeomSmall::kThreads, GeomSmall::kSmemBytes, st, p, a);
+        else launch_overlapped(large_kernel, grid, GeomLarge::kThreads, GeomLarge::kSmemBytes, st, p, a);
+    };
+    if (c->groups == 1 && w32) launch(k_decode_step<GeomSmall, 1, false>, k_decode_step<GeomLarge, 1, false>);
+    else if (c->groups == 1) launch(k_decode_step<GeomSmall, 1, true>, k_decode_step<GeomLarge, 1, true>);
+    else if (w32) launch(k_decode_step<GeomSmall, 2, false>, k_decode_step<GeomLarge, 2, false>);
+    else launch(k_decode_step<GeomSmall, 2, true>, k_decode_step<GeomLarge, 2, true>);
     if (rec) {
         cudaEventRecord(ev[1], st);
         c->prof_calls += 1;

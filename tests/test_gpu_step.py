@@ -1,8 +1,8 @@
 """GPU parity of kvq_decode_step: one decode step (controller decision, quantize-append of one
 token per sequence, attention over everything cached, Eq. 19-24, Eq. 4, Eq. 5) against the
-oracle, step by step.  With keys quantized per token and a controller of width 32 the step is one
-launch (the attending warps add the step's token themselves from its fp16 rows); every other case
-runs the two kernels of kvq_append_fused + kvq_decode_attn behind the same call.  Both are compared with the
+oracle, step by step.  With keys quantized per token the step is one launch (the attending warps
+add the step's token themselves from its fp16 rows); per-channel keys run the two kernels of
+kvq_append_fused + kvq_decode_attn behind the same call.  Both are compared with the
 oracle the same way: decisions and the whole store bit for bit, the attention output of EVERY
 step within the attention tolerance."""
 import numpy as np
@@ -145,14 +145,41 @@ def test_steps_on_a_long_cache_in_the_bandwidth_geometry(gu, oracle, splits):
         gu.assert_store_equals_oracle(g, 0, oc, pos0=n - 64, n=64 + steps)
 
 
+@pytest.mark.parametrize("hidden,seed", [(128, 2), (100, 9), (7, 5), (1, 4)])
+@pytest.mark.parametrize("n", [150, 40000])
+def test_steps_with_controllers_of_other_widths_take_one_launch_each(gu, oracle, hidden, seed, n):
+    """The paper's hidden width (128) and ragged ones, on a short cache (16-warp CTAs) and on a long one (four-warp
+    CTAs): the storing CTAs of the launch evaluate the controller and publish the class, the attending warps pick it
+    up; decisions bit for bit the oracle's.  A controller set later takes over."""
+    rng = np.random.default_rng(hidden + n)
+    cw = synth.controller_weights(seed, hidden)
+    B, Hq, H, steps = 3, 6, 2, 12 if n > 1000 else 40
+    oc = oracle.OracleCache(B, Hq, H)
+    with gu.GpuCache(1, B, Hq, H, n + steps + 5) as g:
+        g.set_controller(cw)
+        K, V = _kv(rng, B, n, H)
+        bits = BITS[rng.choice(4, size=(B, n))]
+        oc.append(K, V, bits)
+        g.append(0, K, V, bits)
+        launches = _run_steps(gu, oracle, g, oc, cw, rng, B, Hq, H, steps, "step with hidden width %d, n=%d" % (hidden, n),
+                              feat_seed=seed, first_pos=n)
+        assert launches == steps
+        cw2 = synth.controller_weights(322, 32)
+        g.set_controller(cw2)
+        _run_steps(gu, oracle, g, oc, cw2, rng, B, Hq, H, 5, "step after a change of controller", first_pos=n + steps)
+        gu.assert_store_equals_oracle(g, 0, oc, pos0=max(0, n - 64), n=min(n, 64) + steps + 5)
+
+
 @pytest.mark.parametrize("case", ["hidden 128", "two scale groups", "per-channel keys"])
 def test_steps_of_the_other_layouts_and_controller_widths(gu, oracle, case):
-    """Two scale groups per row take the one-launch kernel too; a wider controller and per-channel keys run the two
-    kernels behind the same call.  Same results either way."""
+    """Two scale groups per row and a wider controller (20 KV heads: two storing CTAs per sequence) take the
+    one-launch kernel too; per-channel keys run the two kernels behind the same call.  Same results either way."""
     rng = np.random.default_rng(len(case))
     hidden = 128 if case == "hidden 128" else 32
     cw = synth.controller_weights(2 if hidden == 128 else 322, hidden)
     B, Hq, H, steps = 2, 4, 2, 20
+    if case == "hidden 128":
+        Hq = H = 20
     n = 300
     if case == "two scale groups":
         oc = oracle.GroupedOracleCache(B, Hq, H, 2)
@@ -170,7 +197,7 @@ def test_steps_of_the_other_layouts_and_controller_widths(gu, oracle, case):
         oc.append(K, V, bits)
         g.append(0, K, V, bits)
         launches = _run_steps(gu, oracle, g, oc, cw, rng, B, Hq, H, steps, "step, %s" % case, first_pos=n)
-        assert launches == steps if case == "two scale groups" else launches >= 2 * steps
+        assert launches >= 2 * steps if case == "per-channel keys" else launches == steps
         if case != "per-channel keys":
             gu.assert_store_equals_oracle(g, 0, oc)
 
