@@ -644,6 +644,29 @@ def cpu_leg(wl, steps, warmup=1):
             "append_prefill_tokens_per_s": leg["append_prefill_tokens_per_s"]}
 
 
+def measure_feature_kernels(bench, n=4096, vocab=49152, reps=5):
+    """The on-device feature kernel (Eq. 14-17: entropy, rarity, confidence of n tokens from their logits):
+    one pass over the logits, so its bound is HBM.  Synthetic logits (the kernel's time does not depend on
+    their values), larger than L2 in both types."""
+    torch, kq = bench.torch, bench.kq
+    peak, _ = measured_peak_gbs()
+    out = {"tokens": n, "vocab": vocab, "note": "kvq_token_features, one launch, logits resident in HBM; bytes = the logits"}
+    ids = torch.randint(0, vocab, (n,), dtype=torch.int32, device=bench.dev)
+    counts = torch.randint(0, 5000, (vocab,), dtype=torch.int32, device=bench.dev)
+    feats = torch.zeros((n, 4), dtype=torch.float32, device=bench.dev)
+    for name, dt in (("fp32", torch.float32), ("fp16", torch.float16)):
+        logits = (torch.randn((n, vocab), device=bench.dev, dtype=torch.float32) * 3).to(dt)
+        fn = lambda: kq.kvq_token_features(logits, dt == torch.float32, n, vocab, ids, counts, 10_000_000, vocab // 2, None, feats)
+        fn()
+        ms = bench.timed_block(fn, reps) / reps
+        nbytes = logits.numel() * logits.element_size()
+        out[name] = {"us_per_launch": ms * 1e3, "GBps": nbytes / (ms * 1e-3) / 1e9, "frac_of_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / peak,
+                     "logit_bytes": nbytes}
+        del logits
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args, wl):
     bench = Bench()
     rank, world = bench.rank, bench.world
@@ -662,6 +685,7 @@ def run_ours(args, wl):
                 cpu2 = cpu_leg(w2, 3)
             others[name + ("_all_%d_bit" % ub if ub else "")] = compact(m2, w2, cpu2)
         bench.kv_cache.clear()
+    features = measure_feature_kernels(bench) if is_headline and world == 1 and not args.no_other_workloads else None
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline and is_headline:
@@ -710,6 +734,7 @@ def run_ours(args, wl):
             "kv_bytes_per_layer": m["dec_bytes"], "expected_bits": m["expected_bits"],
             "device_flags": m["device_flags"], "input_generation_s": m["input_generation_s"],
             "other_workloads": others,
+            "feature_kernels": features,
         }
         print(json.dumps(line))
     bench.close()
