@@ -252,7 +252,9 @@ int kvq_decode_attn_var(kvq_ctx* ctx, int layer, const void* Q, void* O, float* 
  *               kvq_decode_attn_var
  *   feats       dev fp32 [n][4] in the order H, R, V, C of Eq. 17 (16-byte aligned)
  * The logits are read once; rows are read with 16-byte loads when vocab % 8 == 0 and the base
- * is 32-byte aligned.  The library treats the controller's inputs as four opaque numbers, so a
+ * is 32-byte aligned.  Masked entries (-inf) count as probability zero (p log p = 0); a row must
+ * keep at least one finite entry (a row that is masked throughout has no distribution: its H and C
+ * are unspecified).  fp32 logits below -1e28 are treated as masked.  The library treats the controller's inputs as four opaque numbers, so a
  * controller must have been trained on this order to be fed from here.
  */
 int kvq_token_features(const void* logits, int logits_are_fp32, int n, int vocab,
