@@ -103,14 +103,14 @@ def test_steps_after_a_prefill_for_every_way_of_cutting_the_work(gu, oracle, spl
 
 def test_steps_that_open_new_blocks_and_new_tiles(gu, oracle):
     """All tokens in one class (a controller whose biases decide): the 2-bit stream of a sequence fills its first
-    64 KB block (102 tiles) during the steps and goes on in a second one."""
+    64 KB block (100 tiles of 16 slots) during the steps and goes on in a second one."""
     rng = np.random.default_rng(5)
     H32 = 32
     z = np.zeros
     cw = synth.ControllerWeights(H32, z((H32, 4), np.float32), z(H32, np.float32), z((H32, H32), np.float32),
                                  z(H32, np.float32), z((4, H32), np.float32), np.array([1, 0, 0, 0], np.float32))
     B, Hq, H = 1, 2, 1
-    n = 102 * 16 - 5
+    n = 100 * 16 - 5
     steps = 12
     oc = oracle.OracleCache(B, Hq, H)
     with gu.GpuCache(1, B, Hq, H, n + steps) as g:
