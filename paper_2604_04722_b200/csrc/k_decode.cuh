@@ -57,6 +57,9 @@
 #ifndef KVQ_SMALL_STAGES
 #define KVQ_SMALL_STAGES 3
 #endif
+#ifndef KVQ_SMALL_END_TO_END
+#define KVQ_SMALL_END_TO_END 1
+#endif
 #ifndef KVQ_DECODE_FMA2
 #define KVQ_DECODE_FMA2 1          // fp16 pool: V-side accumulation with packed two-lane fp32 FMAs
 #endif
@@ -74,6 +77,10 @@ struct DecodeGeom {
     static constexpr int kWarps = WARPS, kThreads = WARPS * 32, kStages = STAGES, kStageBytes = STAGE_BYTES, kCtasPerSm = MIN_CTAS;
     static constexpr size_t kSmemBytes = (size_t)WARPS * STAGES * STAGE_BYTES;
     static constexpr bool kCtaMerge = true;            // units cut into a divisor of WARPS parts are merged inside their CTA
+    // One CTA per SM is the geometry of short caches, where a launch is a chain of latencies and a tile costs a warp
+    // the same time whatever its class: there a warp's share is a stretch of the unit's pools laid end to end.  In
+    // the bandwidth geometry every warp takes the same fraction of every pool, so that all warps move the same bytes.
+    static constexpr bool kPoolsEndToEnd = KVQ_SMALL_END_TO_END && MIN_CTAS == 1;
     // tiles of class c that fit one stage
     __host__ __device__ static constexpr int tps(int c, int g = 1) { return STAGE_BYTES / pool_rec_bytes(c, g); }
     static_assert(STAGE_BYTES % 16 == 0 && STAGE_BYTES >= pool_rec_bytes(3), "a stage must hold one fp16 tile");
@@ -829,6 +836,17 @@ struct alignas(16) WarpScratch {
 };
 constexpr int kQHalfStride = kHalfDim + 4;
 
+// Relative cost of a tile of each class to a warp of the short-cache geometry: a constant for the walk plus the
+// tile's share of a stage refill (6 / 3 / 2 / 1 tiles of the four classes fit a stage); the best of four sets
+// tried on the three short workloads, all within 4 % of one another.
+#ifndef KVQ_TILE_COST_2BIT
+#define KVQ_TILE_COST_2BIT 4u
+#define KVQ_TILE_COST_4BIT 5u
+#define KVQ_TILE_COST_8BIT 7u
+#define KVQ_TILE_COST_FP16 12u
+#endif
+__device__ constexpr uint32_t kTileCost[kNumPools] = {KVQ_TILE_COST_2BIT, KVQ_TILE_COST_4BIT, KVQ_TILE_COST_8BIT, KVQ_TILE_COST_FP16};
+
 // floor(n * a / g) for a <= g < 65536 in 32-bit arithmetic: n = q*g + r gives q*a + floor(r*a/g).
 __device__ __forceinline__ uint32_t scale_by_fraction(uint32_t n, uint32_t a, uint32_t g) {
     const uint32_t q = n / g, r = n - q * g;
@@ -1010,7 +1028,24 @@ __device__ __forceinline__ void decode_attn_body(const DecodeParams& P, const Ap
             const uint32_t nt = (n + kTileTokens - 1) / kTileTokens;
             ws.cnt[c] = n;
             int lo, hi;
-            if (P.gw < 65536u) {
+            if constexpr (Geo::kPoolsEndToEnd) {
+                // The four pools of the unit laid end to end and THAT axis cut into the warps' shares: a warp then
+                // walks one pool, or two where its share crosses a border, instead of a sliver of each of the four
+                // (every pool a warp enters costs it an operand set-up and a drained pipeline).
+                // A tile counts with what it costs a warp here (kTileCost: its walk plus its part of a stage refill).
+                const uint32_t cost = kTileCost[c];
+                uint32_t before = 0, total = 0;
+#pragma unroll
+                for (int k = 0; k < kNumPools; ++k) {
+                    const uint32_t wk = __shfl_sync(0xfu, nt * cost, k);
+                    before += k < c ? wk : 0u;
+                    total += wk;
+                }
+                const int r0 = (int)scale_by_fraction(total, a0, P.gw) - (int)before;
+                const int r1 = (int)scale_by_fraction(total, a1, P.gw) - (int)before;
+                lo = min(max(r0, 0) / (int)cost, (int)nt);       // the same rounding for a share's end and the next one's start
+                hi = a1 == P.gw ? (int)nt : min(max(r1, 0) / (int)cost, (int)nt);
+            } else if (P.gw < 65536u) {
                 lo = (int)scale_by_fraction(nt, a0, P.gw);
                 hi = (int)scale_by_fraction(nt, a1, P.gw);
             } else {
