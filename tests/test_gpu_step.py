@@ -202,6 +202,44 @@ def test_steps_of_the_other_layouts_and_controller_widths(gu, oracle, case):
             gu.assert_store_equals_oracle(g, 0, oc)
 
 
+@pytest.mark.parametrize("bits", [2, 4, 8, 16])
+def test_steps_with_degenerate_rows(gu, oracle, bits):
+    """Rows whose quantizer takes a special path (all zero, constant, +0 and -0 mixed, a range so small that the fp16
+    scale is subnormal or rounds to zero, values near the fp16 limit, one outlier channel), every token in the class
+    that a bias-only controller picks: the attending warps quantize the step's token themselves, so their copy of the
+    row quantizer must agree with the store's on these too."""
+    rng = np.random.default_rng(bits)
+    Hd = 32
+    z = np.zeros
+    b3 = np.zeros(4, np.float32)
+    b3[[2, 4, 8, 16].index(bits)] = 1.0
+    cw = synth.ControllerWeights(Hd, z((Hd, 4), np.float32), z(Hd, np.float32), z((Hd, Hd), np.float32),
+                                 z(Hd, np.float32), z((4, Hd), np.float32), b3)
+    B, Hq, H = 2, 4, 2
+    rows = [np.zeros(64), np.full(64, 0.3125), np.where(np.arange(64) % 2 == 0, 0.0, -0.0),
+            1e-4 + 1e-7 * np.arange(64), 3e-7 * (np.arange(64) % 3), np.where(np.arange(64) % 2 == 0, 60000.0, -60000.0),
+            np.where(np.arange(64) == 17, 40.0, 0.01 * rng.standard_normal(64)), rng.standard_normal(64)]
+    steps = len(rows)
+    n = 40
+    oc = oracle.OracleCache(B, Hq, H)
+    with gu.GpuCache(1, B, Hq, H, n + steps) as g:
+        g.set_controller(cw)
+        K, V = _kv(rng, B, n, H)
+        pre = np.full((B, n), bits, np.uint8)
+        oc.append(K, V, pre)
+        g.append(0, K, V, pre)
+        feats = synth.features_batch(1, B, n, steps)
+        for s, row in enumerate(rows):
+            K1 = np.broadcast_to(row.astype(np.float16), (B, 1, H, 64)).copy()
+            V1 = np.broadcast_to(rows[(s + 3) % steps].astype(np.float16), (B, 1, H, 64)).copy()
+            Q = rng.standard_normal((B, Hq, 64)).astype(np.float16)
+            oc.append(K1, V1, np.full((B, 1), bits, np.uint8))
+            got, out = _step(gu, g, 0, feats[:, s], K1, V1, Q)
+            assert np.all(got == bits)
+            gu.assert_attention_close(out, oc.decode_attn(Q), "degenerate rows, %d bits, step %d" % (bits, s))
+        gu.assert_store_equals_oracle(g, 0, oc)
+
+
 def test_steps_on_a_layer_of_ragged_lengths(gu, oracle):
     """Sequences of different lengths (one of them empty before the first step): every sequence against its own
     oracle cache."""
