@@ -10,6 +10,7 @@ heads, head_dim 64, batch 16, context 32768, bit-widths i.i.d. {2:50%, 4:30%, 8:
     python bench.py --gpus N --steps K --warmup W            # this library
     python bench.py --impl reference ...                     # the CPU oracle on a bounded sample
     python bench.py --sweep-splits                           # automatic launch plan against explicit split counts
+    python bench.py --features-only                          # the on-device feature kernel alone
 
 Timing protocol: after W warm-up steps a block of exactly K steps is timed with CUDA events between
 device synchronisations (and barriers when N > 1); the block is repeated `--blocks` times (default
@@ -810,6 +811,8 @@ def main():
                     help="skip the other workloads that the default line carries beside the headline one")
     ap.add_argument("--other-steps", type=int, default=10, help="steps per block of the other workloads")
     ap.add_argument("--other-blocks", type=int, default=5)
+    ap.add_argument("--features-only", action="store_true",
+                    help="time only the on-device feature kernel (the `feature_kernels` object of the default line)")
     ap.add_argument("--sweep-splits", action="store_true",
                     help="compare the automatic launch plan of the attention kernel with explicit split counts")
     ap.add_argument("--context", type=int, default=0,
@@ -839,6 +842,11 @@ def main():
         run_reference(args, wl)
     elif args.sweep_splits:
         run_sweep(args)
+    elif args.features_only:
+        b = Bench()
+        if b.rank == 0:
+            print(json.dumps({"feature_kernels": measure_feature_kernels(b)}))
+        b.close()
     else:
         run_ours(args, wl)
 
